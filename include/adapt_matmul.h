@@ -1,0 +1,184 @@
+/*
+ * adapt_matmul -- shape-adaptive dense GEMM for NVIDIA B200 (sm_100a).
+ *
+ *   C[M x N] = A[M x K] * B[K x N]      fp16 or bf16 operands, fp32 accumulation,
+ *                                        one round-to-nearest-even cast to the
+ *                                        16-bit output, every C element written once
+ *
+ * This is the problem the paper states in Section 4.1 and in the "Common" template
+ * paragraph (Eq. 2): 16-bit inputs, higher-precision on-chip accumulation, a single
+ * cast, minimum write volume 2*M*N bytes.  The library follows the paper's workflow
+ * (Section 3.2): a shape is classified in the 2D tiling taxonomy (Section 4.2), the
+ * legal kernel configurations are scored by an analytical latency model (Section 5.2,
+ * Eq. 6-11, 12-14), the winner is encoded in a 64-bit TilingKey and cached, and the
+ * online call is an O(1) lookup followed by the launch.
+ *
+ * Plain C ABI: no C++ or framework types cross this boundary.  Unless stated, a
+ * pointer argument is a HOST pointer; A, B, C and cuda_stream are the exceptions.
+ * All functions are thread-safe.  There is no CPU fallback: without a CUDA device
+ * the compute entry points fail with ADAPT_ERR_CUDA / ADAPT_ERR_NOT_INIT.
+ */
+#ifndef ADAPT_MATMUL_H
+#define ADAPT_MATMUL_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Opaque plan handle.  Owned by the library's plan cache, valid until
+ * adapt_shutdown(); the caller never frees it. */
+typedef struct adapt_plan_s* adapt_handle_t;
+
+/* Element type of A, B and C (they share it).  Accumulation is always fp32. */
+typedef enum { ADAPT_F16 = 0, ADAPT_BF16 = 1 } adapt_dtype_t;
+
+/* Storage of an operand, dense (leading dimension = inner extent).
+ * A is M x K: row-major means K contiguous, column-major means M contiguous.
+ * B is K x N: row-major means N contiguous, column-major means K contiguous.
+ * C is always row-major M x N. */
+typedef enum { ADAPT_ROW_MAJOR = 0, ADAPT_COL_MAJOR = 1 } adapt_layout_t;
+
+typedef enum {
+    ADAPT_OK = 0,
+    ADAPT_ERR_INVALID_ARG = 1,   /* negative size, NULL pointer, bad enum, aliasing C */
+    ADAPT_ERR_UNSUPPORTED = 2,   /* a dimension above 2^31-1, or a forced key that is illegal for the shape */
+    ADAPT_ERR_NOMEM = 3,         /* workspace allocation failed */
+    ADAPT_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed (message in adapt_last_error_message) */
+    ADAPT_ERR_TIMEOUT = 5,       /* a bounded device-side wait gave up (see adapt_poll_device_status) */
+    ADAPT_ERR_NOT_INIT = 6       /* compute call before a successful adapt_init */
+} adapt_status_t;
+
+/* The four templates of the taxonomy (Section 4.2). */
+typedef enum {
+    ADAPT_CLASS_COMMON = 0,              /* enough tiles, accumulator fits on chip */
+    ADAPT_CLASS_SINGLE_CORE_SPLIT_K = 1, /* enough tiles, tile larger than one SM's accumulator budget */
+    ADAPT_CLASS_MULTI_CORE_SPLIT_K = 2,  /* too few tiles, accumulator fits */
+    ADAPT_CLASS_HYBRID_SPLIT_K = 3       /* too few tiles and oversized tile */
+} adapt_class_t;
+
+/* Kernel families of the variant library. */
+typedef enum {
+    ADAPT_FAM_UMMA_1CTA = 0,  /* tcgen05 128 x BN tiles, TMEM accumulators, TMA ring; P_k > 1 adds split-K */
+    ADAPT_FAM_UMMA_2CTA = 1,  /* cta_group::2, 256 x BN tile on an SM pair */
+    ADAPT_FAM_SKINNY = 2,     /* warp-level kernel for M <= 16 or N <= 16, streams the large operand once */
+    ADAPT_FAM_SIMT = 3        /* CUDA-core tile kernel: legal for every shape and alignment */
+} adapt_family_t;
+
+/* How an operand reaches shared memory (the paper's Padding module, Table 2). */
+typedef enum {
+    ADAPT_SRC_TMA = 0,        /* TMA straight from the caller's buffer (needs 16 B pitch and base) */
+    ADAPT_SRC_PAD_COPY = 1,   /* prologue kernel re-pitches the operand into the workspace, then TMA */
+    ADAPT_SRC_LSU = 2         /* ordinary loads (skinny / SIMT families) */
+} adapt_source_t;
+
+/* Everything the selector decided for one shape.  Filled by adapt_plan_info and
+ * adapt_plan_candidates into caller-owned host memory. */
+typedef struct adapt_plan_info_s {
+    uint64_t tiling_key;      /* 64-bit TilingKey of this configuration (bit layout below) */
+    int64_t M, N, K;
+    int32_t dtype, layoutA, layoutB;
+    int32_t taxonomy_class;   /* adapt_class_t */
+    int32_t family;           /* adapt_family_t */
+    int32_t BM, BN, BK;       /* CTA (or CTA-pair) tile: the paper's m1, n1, k1 */
+    int32_t stages;           /* depth of the shared-memory ring (Multi-Buffer / Preloading depth) */
+    int32_t P_m, P_n, P_k;    /* task counts along M, N, K (Table 1) */
+    int32_t cluster;          /* CTAs per cluster (2 for the 2-CTA family) */
+    int32_t srcA, srcB;       /* adapt_source_t */
+    int32_t grid;             /* CTAs launched by the main kernel */
+    int32_t reserved;
+    int64_t workspace_bytes;  /* pad copies + split-K partials */
+    double flops;             /* 2*M*N*K */
+    double hbm_bytes;         /* modelled HBM traffic including workspace traffic */
+    double t_pro_us;          /* Eq. 7 terms of the prediction */
+    double t_main_us;
+    double t_epi_us;
+    double predicted_us;      /* T_pro + max_j T_main + T_epi + launch cost */
+} adapt_plan_info_t;
+
+/* TilingKey bit layout (Section 3.2 asks only for "a compact 64-bit key"; the fields are this
+ * library's): [63:62] taxonomy class, [61:59] family, [58:54] BM/16, [53:48] BN/16,
+ * [47:46] log2(BK/16), [45:42] stages, [41:32] P_k, [31] persistent tile loop,
+ * [30:29] srcA, [28:27] srcB, [26] dtype, [25] layoutA, [24] layoutB, [23:22] log2(cluster),
+ * [21:0] zero. */
+
+/* Select the device (cudaSetDevice), query it, and create the library state for
+ * it.  Idempotent.  Needed before adapt_matmul; planning works without it (the
+ * selector then assumes a B200: 148 SMs, 227 KB shared memory, 512 TMEM columns). */
+adapt_status_t adapt_init(int device);
+
+/* Free plans, workspaces and cached tensor maps.  Every handle becomes invalid. */
+void adapt_shutdown(void);
+
+/* Section 3.2 / 5.1 "offline" half, done on first sight of a shape and cached:
+ * classify (M,N,K), enumerate legal configurations, score each with the model,
+ * keep the argmin (Eq. 6).  Same arguments -> same handle (pointer-equal).
+ * Host work only, no GPU call.  A cache hit costs one hash probe.
+ * Returns NULL on error (adapt_last_error tells why).
+ * M, N, K >= 0 and <= 2^31-1.  M == 0 or N == 0 plans a no-op; K == 0 plans a zero fill. */
+adapt_handle_t adapt_matmul_plan(int64_t M, int64_t N, int64_t K,
+                                 adapt_dtype_t dtype, adapt_layout_t layoutA, adapt_layout_t layoutB);
+
+/* Section 3.2 "online" half: run the planned kernel(s).
+ * A, B, C: DEVICE pointers owned by the caller, 2-byte aligned at least (16-byte
+ * aligned buffers let TMA read them in place; others are re-pitched through the
+ * workspace first).  C must not overlap A or B.  cuda_stream is a cudaStream_t
+ * (NULL = default stream).  The call enqueues work and returns without
+ * synchronising.  The first call that needs a larger workspace than any before it
+ * allocates (cudaMalloc), so it must not happen inside a stream capture.
+ * Calls that share a stream may share the workspace; calls on different streams
+ * get different workspaces. */
+adapt_status_t adapt_matmul(adapt_handle_t plan, const void* A, const void* B, void* C, void* cuda_stream);
+
+/* Thread-local status of the last failing call on this thread, and its text. */
+adapt_status_t adapt_last_error(void);
+const char* adapt_last_error_message(void);
+const char* adapt_status_string(adapt_status_t s);
+
+/* Copy the plan's decision into *out (host memory). */
+adapt_status_t adapt_plan_info(adapt_handle_t plan, adapt_plan_info_t* out);
+
+/* Every legal configuration for the shape with its predicted time (Eq. 6's search
+ * set S(b(s)) after the capacity check), best first.  Writes at most cap entries
+ * to out (host memory) and returns the total number of legal candidates, or -1. */
+int adapt_plan_candidates(int64_t M, int64_t N, int64_t K,
+                          adapt_dtype_t dtype, adapt_layout_t layoutA, adapt_layout_t layoutB,
+                          adapt_plan_info_t* out, int cap);
+
+/* Bypass the model: a plan that runs exactly the configuration encoded in
+ * tiling_key (as reported by adapt_plan_candidates).  Used to time every legal
+ * variant (the paper's model-validation method, Section 6.6).  Cached per
+ * (shape, key).  NULL + ADAPT_ERR_UNSUPPORTED if the key is not legal for the shape. */
+adapt_handle_t adapt_matmul_plan_forced(int64_t M, int64_t N, int64_t K,
+                                        adapt_dtype_t dtype, adapt_layout_t layoutA, adapt_layout_t layoutB,
+                                        uint64_t tiling_key);
+
+/* The taxonomy by itself (Section 4.2), parameterised by the machine: returns the
+ * adapt_class_t of a shape tiled by m x n sub-tasks with an m1 x n1 accumulation
+ * tile on n_core cores with acc_bytes of fp32 accumulator per core; -1 on bad input. */
+int adapt_classify(int64_t M, int64_t N, int64_t m, int64_t n, int64_t m1, int64_t n1,
+                   int64_t n_core, int64_t acc_bytes);
+
+/* Closed-form building blocks of the model, exported for validation:
+ * Eq. 1 read volume, Eq. 2-5 write volumes (bytes), Eq. 12-14 pipeline times. */
+double adapt_model_read_volume(int64_t M, int64_t N, int64_t K, int64_t m1, int64_t n1);
+double adapt_model_write_volume(int cls, int64_t M, int64_t N, int64_t K, int64_t k, int64_t k1);
+double adapt_model_pipeline(int schedule /*0 baseline, 1 double buffer, 2 preload*/,
+                            int64_t Q, int64_t L, double t_M, double t_P, double T_drain);
+
+/* Synchronise the stream, then read and clear the device status word.  Returns
+ * ADAPT_ERR_TIMEOUT if a kernel's bounded barrier wait expired since the last
+ * poll, ADAPT_ERR_CUDA if the stream reports a fault, else ADAPT_OK. */
+adapt_status_t adapt_poll_device_status(void* cuda_stream);
+
+/* Number of plans in the cache (both selected and forced). */
+int64_t adapt_plan_cache_size(void);
+
+/* Count of kernels this library has launched since adapt_init (all streams). */
+int64_t adapt_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ADAPT_MATMUL_H */

@@ -1,0 +1,203 @@
+"""ctypes binding of ``libadaptmm.so``: the same names as ``include/adapt_matmul.h``.
+
+Argument marshalling only.  Every step of the GEMM path runs inside the CUDA
+library; there is no fallback.  If the shared object is missing, ``load()``
+raises and nothing else in this module works.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+F16, BF16 = 0, 1
+ROW_MAJOR, COL_MAJOR = 0, 1
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NOMEM, ERR_CUDA, ERR_TIMEOUT, ERR_NOT_INIT = range(7)
+CLASS_NAMES = ["Common", "SingleCoreSplitK", "MultiCoreSplitK", "HybridSplitK"]
+FAMILY_NAMES = ["umma_1cta", "umma_2cta", "skinny", "simt"]
+FAM_UMMA_1CTA, FAM_UMMA_2CTA, FAM_SKINNY, FAM_SIMT = range(4)
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libadaptmm.so")
+
+EXPORTS = [
+    "adapt_init", "adapt_shutdown", "adapt_matmul_plan", "adapt_matmul", "adapt_last_error",
+    "adapt_last_error_message", "adapt_status_string", "adapt_plan_info", "adapt_plan_candidates",
+    "adapt_matmul_plan_forced", "adapt_classify", "adapt_model_read_volume", "adapt_model_write_volume",
+    "adapt_model_pipeline", "adapt_poll_device_status", "adapt_plan_cache_size", "adapt_launch_count",
+]
+
+
+class PlanInfo(ctypes.Structure):
+    _fields_ = [
+        ("tiling_key", ctypes.c_uint64),
+        ("M", ctypes.c_int64), ("N", ctypes.c_int64), ("K", ctypes.c_int64),
+        ("dtype", ctypes.c_int32), ("layoutA", ctypes.c_int32), ("layoutB", ctypes.c_int32),
+        ("taxonomy_class", ctypes.c_int32), ("family", ctypes.c_int32),
+        ("BM", ctypes.c_int32), ("BN", ctypes.c_int32), ("BK", ctypes.c_int32),
+        ("stages", ctypes.c_int32),
+        ("P_m", ctypes.c_int32), ("P_n", ctypes.c_int32), ("P_k", ctypes.c_int32),
+        ("cluster", ctypes.c_int32), ("srcA", ctypes.c_int32), ("srcB", ctypes.c_int32),
+        ("grid", ctypes.c_int32), ("reserved", ctypes.c_int32),
+        ("workspace_bytes", ctypes.c_int64),
+        ("flops", ctypes.c_double), ("hbm_bytes", ctypes.c_double),
+        ("t_pro_us", ctypes.c_double), ("t_main_us", ctypes.c_double), ("t_epi_us", ctypes.c_double),
+        ("predicted_us", ctypes.c_double),
+    ]
+
+    def as_dict(self):
+        d = {k: getattr(self, k) for k, _ in self._fields_}
+        d["class_name"] = CLASS_NAMES[self.taxonomy_class]
+        d["family_name"] = FAMILY_NAMES[self.family] if 0 <= self.family < 4 else "?"
+        return d
+
+
+class AdaptError(RuntimeError):
+    def __init__(self, status, message):
+        super().__init__(f"adapt_matmul status {status}: {message}")
+        self.status = status
+
+
+_lib = None
+
+
+def load():
+    """Load the C-ABI library (built in-tree by ``paper_2608_10803_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise FileNotFoundError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2608_10803_b200.build`; there is no fallback path")
+    lib = ctypes.CDLL(LIB_PATH)
+    i64, i32, u64, vp, dbl = ctypes.c_int64, ctypes.c_int, ctypes.c_uint64, ctypes.c_void_p, ctypes.c_double
+    lib.adapt_init.restype = i32
+    lib.adapt_init.argtypes = [i32]
+    lib.adapt_shutdown.restype = None
+    lib.adapt_matmul_plan.restype = vp
+    lib.adapt_matmul_plan.argtypes = [i64, i64, i64, i32, i32, i32]
+    lib.adapt_matmul_plan_forced.restype = vp
+    lib.adapt_matmul_plan_forced.argtypes = [i64, i64, i64, i32, i32, i32, u64]
+    lib.adapt_matmul.restype = i32
+    lib.adapt_matmul.argtypes = [vp, vp, vp, vp, vp]
+    lib.adapt_last_error.restype = i32
+    lib.adapt_last_error_message.restype = ctypes.c_char_p
+    lib.adapt_status_string.restype = ctypes.c_char_p
+    lib.adapt_status_string.argtypes = [i32]
+    lib.adapt_plan_info.restype = i32
+    lib.adapt_plan_info.argtypes = [vp, ctypes.POINTER(PlanInfo)]
+    lib.adapt_plan_candidates.restype = i32
+    lib.adapt_plan_candidates.argtypes = [i64, i64, i64, i32, i32, i32, ctypes.POINTER(PlanInfo), i32]
+    lib.adapt_classify.restype = i32
+    lib.adapt_classify.argtypes = [i64] * 8
+    lib.adapt_model_read_volume.restype = dbl
+    lib.adapt_model_read_volume.argtypes = [i64] * 5
+    lib.adapt_model_write_volume.restype = dbl
+    lib.adapt_model_write_volume.argtypes = [i32] + [i64] * 5
+    lib.adapt_model_pipeline.restype = dbl
+    lib.adapt_model_pipeline.argtypes = [i32, i64, i64, dbl, dbl, dbl]
+    lib.adapt_poll_device_status.restype = i32
+    lib.adapt_poll_device_status.argtypes = [vp]
+    lib.adapt_plan_cache_size.restype = i64
+    lib.adapt_launch_count.restype = i64
+    _lib = lib
+    return lib
+
+
+def _check(status):
+    if status != OK:
+        raise AdaptError(status, load().adapt_last_error_message().decode())
+
+
+def adapt_init(device: int = 0):
+    _check(load().adapt_init(device))
+
+
+def adapt_shutdown():
+    load().adapt_shutdown()
+
+
+def adapt_matmul_plan(M, N, K, dtype, layoutA=ROW_MAJOR, layoutB=ROW_MAJOR):
+    h = load().adapt_matmul_plan(M, N, K, dtype, layoutA, layoutB)
+    if not h:
+        lib = load()
+        raise AdaptError(lib.adapt_last_error(), lib.adapt_last_error_message().decode())
+    return h
+
+
+def adapt_matmul_plan_forced(M, N, K, dtype, layoutA, layoutB, tiling_key):
+    h = load().adapt_matmul_plan_forced(M, N, K, dtype, layoutA, layoutB, tiling_key)
+    if not h:
+        lib = load()
+        raise AdaptError(lib.adapt_last_error(), lib.adapt_last_error_message().decode())
+    return h
+
+
+def adapt_matmul(plan, A_ptr: int, B_ptr: int, C_ptr: int, stream: int = 0):
+    """Enqueue C = A*B.  Pointers are raw device addresses (``tensor.data_ptr()``)."""
+    _check(load().adapt_matmul(plan, A_ptr, B_ptr, C_ptr, stream))
+
+
+def adapt_plan_info(plan) -> PlanInfo:
+    info = PlanInfo()
+    _check(load().adapt_plan_info(plan, ctypes.byref(info)))
+    return info
+
+
+def adapt_plan_candidates(M, N, K, dtype, layoutA=ROW_MAJOR, layoutB=ROW_MAJOR, cap: int = 512):
+    buf = (PlanInfo * cap)()
+    n = load().adapt_plan_candidates(M, N, K, dtype, layoutA, layoutB, buf, cap)
+    if n < 0:
+        lib = load()
+        raise AdaptError(lib.adapt_last_error(), lib.adapt_last_error_message().decode())
+    return [buf[i] for i in range(min(n, cap))]
+
+
+def adapt_classify(M, N, m, n, m1, n1, n_core, acc_bytes) -> int:
+    return load().adapt_classify(M, N, m, n, m1, n1, n_core, acc_bytes)
+
+
+def adapt_model_read_volume(M, N, K, m1, n1) -> float:
+    return load().adapt_model_read_volume(M, N, K, m1, n1)
+
+
+def adapt_model_write_volume(cls, M, N, K, k, k1) -> float:
+    return load().adapt_model_write_volume(cls, M, N, K, k, k1)
+
+
+def adapt_model_pipeline(schedule, Q, L, t_M, t_P, T_drain) -> float:
+    return load().adapt_model_pipeline(schedule, Q, L, t_M, t_P, T_drain)
+
+
+def adapt_poll_device_status(stream: int = 0):
+    _check(load().adapt_poll_device_status(stream))
+
+
+def adapt_plan_cache_size() -> int:
+    return load().adapt_plan_cache_size()
+
+
+def adapt_launch_count() -> int:
+    return load().adapt_launch_count()
+
+
+# ---- convenience for torch callers (memory and streams only) -------------------------------------
+
+def matmul(A, B, out=None, layoutA=ROW_MAJOR, layoutB=ROW_MAJOR, plan=None):
+    """C = A @ B for CUDA fp16/bf16 torch tensors through the library (row-major storage by default).
+
+    ``A`` holds M*K elements and ``B`` K*N elements in the stated layouts; shapes are read
+    as (M, K) and (K, N).  torch is used for the output allocation and the current stream.
+    """
+    import torch
+
+    assert A.is_cuda and B.is_cuda and A.dtype == B.dtype and A.is_contiguous() and B.is_contiguous()
+    dtype = F16 if A.dtype == torch.float16 else BF16
+    M, K = (A.shape if layoutA == ROW_MAJOR else (A.shape[1], A.shape[0]))
+    K2, N = (B.shape if layoutB == ROW_MAJOR else (B.shape[1], B.shape[0]))
+    assert K == K2
+    if out is None:
+        out = torch.empty((M, N), dtype=A.dtype, device=A.device)
+    if plan is None:
+        plan = adapt_matmul_plan(M, N, K, dtype, layoutA, layoutB)
+    adapt_matmul(plan, A.data_ptr(), B.data_ptr(), out.data_ptr(), torch.cuda.current_stream().cuda_stream)
+    return out

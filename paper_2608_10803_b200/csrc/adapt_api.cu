@@ -1,0 +1,687 @@
+// C ABI of the library: plan cache (online O(1) dispatch, Section 3.2), launch_map (TilingKey ->
+// compiled kernel), tensor-map construction, workspace management and the launches themselves.
+#include <atomic>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <string>
+#include <tuple>
+#include <unordered_map>
+#include <vector>
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <cudaTypedefs.h>
+
+#include "adapt_internal.h"
+#include "aux_kernels.cuh"
+#include "skinny_gemm.cuh"
+#include "umma_gemm.cuh"
+
+using namespace adapt;
+
+// ---------------------------------------------------------------------------------------------
+// error reporting (thread-local)
+// ---------------------------------------------------------------------------------------------
+static thread_local adapt_status_t tl_status = ADAPT_OK;
+static thread_local char tl_message[256] = "";
+
+static adapt_status_t fail(adapt_status_t st, const char* fmt, const char* detail = "")
+{
+    tl_status = st;
+    snprintf(tl_message, sizeof(tl_message), fmt, detail);
+    return st;
+}
+
+#define CUDA_TRY(expr)                                                        \
+    do {                                                                      \
+        cudaError_t e__ = (expr);                                             \
+        if (e__ != cudaSuccess) return fail(ADAPT_ERR_CUDA, #expr ": %s", cudaGetErrorString(e__)); \
+    } while (0)
+
+// ---------------------------------------------------------------------------------------------
+// plans and the plan cache
+// ---------------------------------------------------------------------------------------------
+struct MapSlot {
+    const void* ptr = nullptr;
+    int64_t pitch = 0;
+    CUtensorMap map;
+};
+
+struct adapt_plan_s {
+    Shape s;
+    Config c;
+    bool noop = false;        // M == 0 or N == 0
+    bool zero_fill = false;   // K == 0
+    std::mutex mu;            // guards the tensor-map slots
+    MapSlot mapA[2], mapB[2];
+    int nextA = 0, nextB = 0;
+};
+typedef adapt_plan_s Plan;
+
+namespace {
+
+// Open-addressing table keyed by a 64-bit shape word.  Readers take no lock: an entry's plan
+// pointer is published before its key.  Inserts and growth are serialised by a mutex; a grown
+// table replaces the old one, which is kept until shutdown so that concurrent readers stay valid.
+struct Table {
+    size_t cap;
+    std::atomic<uint64_t>* keys;
+    std::atomic<Plan*>* vals;
+    explicit Table(size_t c) : cap(c)
+    {
+        keys = new std::atomic<uint64_t>[c];
+        vals = new std::atomic<Plan*>[c];
+        for (size_t i = 0; i < c; ++i) { keys[i].store(0, std::memory_order_relaxed); vals[i].store(nullptr, std::memory_order_relaxed); }
+    }
+    ~Table() { delete[] keys; delete[] vals; }
+};
+
+inline uint64_t mix64(uint64_t x)
+{
+    x ^= x >> 33; x *= 0xff51afd7ed558ccdull; x ^= x >> 33; x *= 0xc4ceb9fe1a85ec53ull; x ^= x >> 33;
+    return x;
+}
+
+// dims below 2^20 pack into one word: [63] valid, [62] dtype, [61] layoutA, [60] layoutB, 3 x 20 bits
+inline bool shape_word(const Shape& s, uint64_t* w)
+{
+    if ((uint64_t)s.M >= (1u << 20) || (uint64_t)s.N >= (1u << 20) || (uint64_t)s.K >= (1u << 20)) return false;
+    *w = (1ull << 63) | ((uint64_t)s.dtype << 62) | ((uint64_t)s.layoutA << 61) | ((uint64_t)s.layoutB << 60) |
+         ((uint64_t)s.M << 40) | ((uint64_t)s.N << 20) | (uint64_t)s.K;
+    return true;
+}
+
+struct State {
+    std::mutex mu;                       // inserts, slow-path maps, workspace table, init
+    std::atomic<Table*> table{nullptr};
+    size_t count = 0;
+    std::vector<Table*> retired;
+    std::vector<Plan*> all_plans;
+    typedef std::tuple<int64_t, int64_t, int64_t, int, int, int, uint64_t> BigKey;
+    std::map<BigKey, Plan*> big;         // huge dims, and forced plans (last field = tiling key + 1)
+
+    bool inited = false;
+    int device = -1;
+    Machine machine;
+    Calib calib;
+    unsigned int* d_status = nullptr;
+    struct Workspace { void* ptr = nullptr; size_t bytes = 0; };
+    std::unordered_map<cudaStream_t, Workspace> ws;
+    PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+    std::atomic<int64_t> launches{0};
+    int log = 0;
+};
+
+State& st()
+{
+    static State* s = new State();     // never destroyed: handles stay valid during process exit
+    return *s;
+}
+
+void apply_env(State& S)
+{
+    if (const char* e = getenv("ADAPT_FAMILY_MASK")) S.machine.family_mask = (unsigned)strtoul(e, nullptr, 0);
+    if (const char* e = getenv("ADAPT_LOG")) S.log = atoi(e);
+    if (const char* e = getenv("ADAPT_WORKSPACE_LIMIT_MB")) S.machine.workspace_limit = (int64_t)atoll(e) << 20;
+}
+
+Plan* table_find(Table* t, uint64_t w)
+{
+    size_t i = (size_t)mix64(w) & (t->cap - 1);
+    for (;;) {
+        const uint64_t k = t->keys[i].load(std::memory_order_acquire);
+        if (k == w) return t->vals[i].load(std::memory_order_relaxed);
+        if (k == 0) return nullptr;
+        i = (i + 1) & (t->cap - 1);
+    }
+}
+
+void table_put(Table* t, uint64_t w, Plan* p)
+{
+    size_t i = (size_t)mix64(w) & (t->cap - 1);
+    while (t->keys[i].load(std::memory_order_relaxed) != 0) i = (i + 1) & (t->cap - 1);
+    t->vals[i].store(p, std::memory_order_relaxed);
+    t->keys[i].store(w, std::memory_order_release);
+}
+
+bool valid_shape(int64_t M, int64_t N, int64_t K, int dtype, int lA, int lB)
+{
+    const int64_t lim = 2147483647ll;
+    if (M < 0 || N < 0 || K < 0) { fail(ADAPT_ERR_INVALID_ARG, "negative dimension%s"); return false; }
+    if (M > lim || N > lim || K > lim) { fail(ADAPT_ERR_UNSUPPORTED, "dimension above 2^31-1%s"); return false; }
+    if ((dtype != 0 && dtype != 1) || (lA != 0 && lA != 1) || (lB != 0 && lB != 1)) {
+        fail(ADAPT_ERR_INVALID_ARG, "bad dtype or layout value%s");
+        return false;
+    }
+    return true;
+}
+
+Plan* make_plan(State& S, const Shape& s, const uint64_t* forced_key)
+{
+    Plan* p = new Plan();
+    p->s = s;
+    if (s.M == 0 || s.N == 0) { p->noop = true; return p; }
+    if (s.K == 0) { p->zero_fill = true; return p; }
+    if (forced_key) {
+        if (!config_from_key(s, *forced_key, S.machine, S.calib, &p->c)) {
+            delete p;
+            fail(ADAPT_ERR_UNSUPPORTED, "tiling key is not legal for this shape%s");
+            return nullptr;
+        }
+        return p;
+    }
+    std::vector<Config> cands;
+    enumerate_configs(s, S.machine, S.calib, &cands);
+    if (cands.empty()) {
+        delete p;
+        fail(ADAPT_ERR_UNSUPPORTED, "no legal configuration%s");
+        return nullptr;
+    }
+    p->c = cands[0];
+    if (S.log) {
+        fprintf(stderr, "[adapt] plan %lldx%lldx%lld dt%d: fam %d class %d tile %dx%dx%d st %d P_k %d src %d/%d pred %.2f us (%zu candidates)\n",
+                (long long)s.M, (long long)s.N, (long long)s.K, s.dtype, p->c.family, p->c.cls, p->c.BM, p->c.BN, p->c.BK,
+                p->c.stages, p->c.P_k, p->c.srcA, p->c.srcB, p->c.predicted_us, cands.size());
+    }
+    return p;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// C ABI: errors
+// ---------------------------------------------------------------------------------------------
+extern "C" adapt_status_t adapt_last_error(void) { return tl_status; }
+extern "C" const char* adapt_last_error_message(void) { return tl_message; }
+extern "C" const char* adapt_status_string(adapt_status_t s)
+{
+    switch (s) {
+        case ADAPT_OK: return "ok";
+        case ADAPT_ERR_INVALID_ARG: return "invalid argument";
+        case ADAPT_ERR_UNSUPPORTED: return "unsupported";
+        case ADAPT_ERR_NOMEM: return "out of memory";
+        case ADAPT_ERR_CUDA: return "CUDA error";
+        case ADAPT_ERR_TIMEOUT: return "device-side wait timed out";
+        case ADAPT_ERR_NOT_INIT: return "not initialised";
+    }
+    return "unknown";
+}
+
+// ---------------------------------------------------------------------------------------------
+// C ABI: planning
+// ---------------------------------------------------------------------------------------------
+extern "C" adapt_handle_t adapt_matmul_plan(int64_t M, int64_t N, int64_t K, adapt_dtype_t dtype,
+                                            adapt_layout_t layoutA, adapt_layout_t layoutB)
+{
+    State& S = st();
+    Shape s;
+    s.M = M; s.N = N; s.K = K; s.dtype = (int)dtype; s.layoutA = (int)layoutA; s.layoutB = (int)layoutB;
+    uint64_t w;
+    // fast path: a plain hash probe, no lock, no validation beyond what the key packing implies
+    if ((uint64_t)s.dtype < 2 && (uint64_t)s.layoutA < 2 && (uint64_t)s.layoutB < 2 && shape_word(s, &w)) {
+        Table* t = S.table.load(std::memory_order_acquire);
+        if (t) {
+            Plan* p = table_find(t, w);
+            if (p) return p;
+        }
+    }
+    if (!valid_shape(M, N, K, s.dtype, s.layoutA, s.layoutB)) return nullptr;
+    std::lock_guard<std::mutex> lock(S.mu);
+    if (!S.inited && S.all_plans.empty()) apply_env(S);
+    const bool small = shape_word(s, &w);
+    Table* t = S.table.load(std::memory_order_acquire);
+    if (small && t) {
+        Plan* p = table_find(t, w);
+        if (p) return p;
+    }
+    State::BigKey bk(M, N, K, s.dtype, s.layoutA, s.layoutB, 0);
+    if (!small) {
+        auto it = S.big.find(bk);
+        if (it != S.big.end()) return it->second;
+    }
+    Plan* p = make_plan(S, s, nullptr);
+    if (!p) return nullptr;
+    S.all_plans.push_back(p);
+    if (!small) { S.big[bk] = p; return p; }
+    if (!t || (S.count + 1) * 2 > t->cap) {
+        Table* nt = new Table(t ? t->cap * 2 : (size_t)1 << 14);
+        if (t) {
+            for (size_t i = 0; i < t->cap; ++i) {
+                const uint64_t k = t->keys[i].load(std::memory_order_relaxed);
+                if (k) table_put(nt, k, t->vals[i].load(std::memory_order_relaxed));
+            }
+            S.retired.push_back(t);
+        }
+        S.table.store(nt, std::memory_order_release);
+        t = nt;
+    }
+    table_put(t, w, p);
+    ++S.count;
+    return p;
+}
+
+extern "C" adapt_handle_t adapt_matmul_plan_forced(int64_t M, int64_t N, int64_t K, adapt_dtype_t dtype,
+                                                   adapt_layout_t layoutA, adapt_layout_t layoutB, uint64_t tiling_key)
+{
+    State& S = st();
+    if (!valid_shape(M, N, K, (int)dtype, (int)layoutA, (int)layoutB)) return nullptr;
+    if (M == 0 || N == 0 || K == 0) return adapt_matmul_plan(M, N, K, dtype, layoutA, layoutB);
+    Shape s;
+    s.M = M; s.N = N; s.K = K; s.dtype = (int)dtype; s.layoutA = (int)layoutA; s.layoutB = (int)layoutB;
+    std::lock_guard<std::mutex> lock(S.mu);
+    if (!S.inited && S.all_plans.empty()) apply_env(S);
+    State::BigKey bk(M, N, K, s.dtype, s.layoutA, s.layoutB, tiling_key + 1);
+    auto it = S.big.find(bk);
+    if (it != S.big.end()) return it->second;
+    // a forced plan may use any compiled family, whatever the selection mask says
+    Machine saved = S.machine;
+    S.machine.family_mask = 0xFu;
+    Plan* p = make_plan(S, s, &tiling_key);
+    S.machine = saved;
+    if (!p) return nullptr;
+    S.all_plans.push_back(p);
+    S.big[bk] = p;
+    return p;
+}
+
+extern "C" adapt_status_t adapt_plan_info(adapt_handle_t plan, adapt_plan_info_t* out)
+{
+    if (!plan || !out) return fail(ADAPT_ERR_INVALID_ARG, "null argument%s");
+    memset(out, 0, sizeof(*out));
+    if (plan->noop || plan->zero_fill) {
+        out->M = plan->s.M; out->N = plan->s.N; out->K = plan->s.K;
+        out->dtype = plan->s.dtype; out->layoutA = plan->s.layoutA; out->layoutB = plan->s.layoutB;
+        return ADAPT_OK;
+    }
+    fill_info(plan->s, plan->c, out);
+    return ADAPT_OK;
+}
+
+extern "C" int adapt_plan_candidates(int64_t M, int64_t N, int64_t K, adapt_dtype_t dtype, adapt_layout_t layoutA,
+                                     adapt_layout_t layoutB, adapt_plan_info_t* out, int cap)
+{
+    State& S = st();
+    if (!valid_shape(M, N, K, (int)dtype, (int)layoutA, (int)layoutB)) return -1;
+    Shape s;
+    s.M = M; s.N = N; s.K = K; s.dtype = (int)dtype; s.layoutA = (int)layoutA; s.layoutB = (int)layoutB;
+    Machine m;
+    {
+        std::lock_guard<std::mutex> lock(S.mu);
+        if (!S.inited && S.all_plans.empty()) apply_env(S);
+        m = S.machine;
+    }
+    m.family_mask = 0xFu;     // list every compiled family, selected or not
+    std::vector<Config> cands;
+    enumerate_configs(s, m, S.calib, &cands);
+    for (int i = 0; i < (int)cands.size() && i < cap && out; ++i) fill_info(s, cands[i], &out[i]);
+    return (int)cands.size();
+}
+
+extern "C" int adapt_classify(int64_t M, int64_t N, int64_t m, int64_t n, int64_t m1, int64_t n1, int64_t n_core, int64_t acc_bytes)
+{
+    return classify(M, N, m, n, m1, n1, n_core, acc_bytes);
+}
+extern "C" double adapt_model_read_volume(int64_t M, int64_t N, int64_t K, int64_t m1, int64_t n1)
+{
+    return read_volume(M, N, K, m1, n1);
+}
+extern "C" double adapt_model_write_volume(int cls, int64_t M, int64_t N, int64_t K, int64_t k, int64_t k1)
+{
+    return write_volume(cls, M, N, K, k, k1);
+}
+extern "C" double adapt_model_pipeline(int schedule, int64_t Q, int64_t L, double t_M, double t_P, double T_drain)
+{
+    return pipeline_time(schedule, Q, L, t_M, t_P, T_drain);
+}
+extern "C" int64_t adapt_plan_cache_size(void)
+{
+    State& S = st();
+    std::lock_guard<std::mutex> lock(S.mu);
+    return (int64_t)S.all_plans.size();
+}
+extern "C" int64_t adapt_launch_count(void) { return st().launches.load(); }
+
+// ---------------------------------------------------------------------------------------------
+// launch_map: (family, BN, A major, B major) -> compiled kernel
+// ---------------------------------------------------------------------------------------------
+typedef void (*UmmaKernel)(const CUtensorMap, const CUtensorMap, const UmmaParams);
+
+template <int CG>
+static UmmaKernel umma_lookup(int BN, bool a_mn, bool b_mn)
+{
+#define ADAPT_PICK(bn)                                                        \
+    if (BN == bn) {                                                           \
+        if (!a_mn && !b_mn) return umma_gemm_kernel<bn, false, false, CG>;    \
+        if (!a_mn && b_mn) return umma_gemm_kernel<bn, false, true, CG>;      \
+        if (a_mn && !b_mn) return umma_gemm_kernel<bn, true, false, CG>;      \
+        return umma_gemm_kernel<bn, true, true, CG>;                          \
+    }
+    if constexpr (CG == 1) { ADAPT_PICK(64) }
+    ADAPT_PICK(128)
+    ADAPT_PICK(256)
+#undef ADAPT_PICK
+    return nullptr;
+}
+
+static UmmaKernel launch_map_umma(int family, int BN, bool a_mn, bool b_mn)
+{
+    return family == ADAPT_FAM_UMMA_1CTA ? umma_lookup<1>(BN, a_mn, b_mn) : umma_lookup<2>(BN, a_mn, b_mn);
+}
+
+// ---------------------------------------------------------------------------------------------
+// init / shutdown
+// ---------------------------------------------------------------------------------------------
+extern "C" adapt_status_t adapt_init(int device)
+{
+    State& S = st();
+    std::lock_guard<std::mutex> lock(S.mu);
+    if (S.inited && S.device == device) return ADAPT_OK;
+    if (S.inited) return fail(ADAPT_ERR_INVALID_ARG, "already initialised on another device%s");
+    CUDA_TRY(cudaSetDevice(device));
+    cudaDeviceProp prop;
+    CUDA_TRY(cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) return fail(ADAPT_ERR_UNSUPPORTED, "device is not sm_100 (%s)", prop.name);
+    if (S.all_plans.empty()) apply_env(S);
+    S.machine.n_sm = prop.multiProcessorCount;
+    S.machine.smem_bytes = (int)prop.sharedMemPerBlockOptin;
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    CUDA_TRY(cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) return fail(ADAPT_ERR_CUDA, "cuTensorMapEncodeTiled not available%s");
+    S.encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
+    CUDA_TRY(cudaMalloc(&S.d_status, sizeof(unsigned int)));
+    CUDA_TRY(cudaMemset(S.d_status, 0, sizeof(unsigned int)));
+    // opt every tensor-core kernel into the full shared-memory carve-out
+    for (int fam = ADAPT_FAM_UMMA_1CTA; fam <= ADAPT_FAM_UMMA_2CTA; ++fam)
+        for (int BN : {64, 128, 256})
+            for (int a = 0; a < 2; ++a)
+                for (int b = 0; b < 2; ++b) {
+                    UmmaKernel k = launch_map_umma(fam, BN, a != 0, b != 0);
+                    if (!k) continue;
+                    CUDA_TRY(cudaFuncSetAttribute((const void*)k, cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
+                }
+    S.device = device;
+    S.inited = true;
+    return ADAPT_OK;
+}
+
+extern "C" void adapt_shutdown(void)
+{
+    State& S = st();
+    std::lock_guard<std::mutex> lock(S.mu);
+    if (S.inited) {
+        cudaDeviceSynchronize();
+        for (auto& kv : S.ws) if (kv.second.ptr) cudaFree(kv.second.ptr);
+        S.ws.clear();
+        if (S.d_status) cudaFree(S.d_status);
+        S.d_status = nullptr;
+    }
+    for (Plan* p : S.all_plans) delete p;
+    S.all_plans.clear();
+    S.big.clear();
+    Table* t = S.table.exchange(nullptr);
+    delete t;
+    for (Table* r : S.retired) delete r;
+    S.retired.clear();
+    S.count = 0;
+    S.inited = false;
+    S.device = -1;
+    S.launches.store(0);
+}
+
+extern "C" adapt_status_t adapt_poll_device_status(void* cuda_stream)
+{
+    State& S = st();
+    if (!S.inited) return fail(ADAPT_ERR_NOT_INIT, "adapt_init has not been called%s");
+    CUDA_TRY(cudaStreamSynchronize((cudaStream_t)cuda_stream));
+    unsigned int w = 0;
+    CUDA_TRY(cudaMemcpy(&w, S.d_status, sizeof(w), cudaMemcpyDeviceToHost));
+    if (w) {
+        CUDA_TRY(cudaMemset(S.d_status, 0, sizeof(unsigned int)));
+        return fail(ADAPT_ERR_TIMEOUT, "a kernel's bounded barrier wait expired%s");
+    }
+    return ADAPT_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// the online call
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+adapt_status_t get_workspace(State& S, cudaStream_t stream, size_t bytes, void** out)
+{
+    *out = nullptr;
+    if (bytes == 0) return ADAPT_OK;
+    std::lock_guard<std::mutex> lock(S.mu);
+    State::Workspace& w = S.ws[stream];
+    if (w.bytes < bytes) {
+        if (w.ptr) {
+            CUDA_TRY(cudaStreamSynchronize(stream));
+            CUDA_TRY(cudaFree(w.ptr));
+            w.ptr = nullptr;
+            w.bytes = 0;
+        }
+        const size_t want = (size_t)round_up((int64_t)bytes + (bytes >> 3), 1 << 20);
+        cudaError_t e = cudaMalloc(&w.ptr, want);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            w.ptr = nullptr;
+            return fail(ADAPT_ERR_NOMEM, "workspace allocation failed: %s", cudaGetErrorString(e));
+        }
+        w.bytes = want;
+    }
+    *out = w.ptr;
+    return ADAPT_OK;
+}
+
+// 2D tensor map over a dense 16-bit matrix [outer][pitch] whose logical inner extent is `inner`.
+adapt_status_t encode_map(State& S, CUtensorMap* map, const void* base, int dtype, int64_t inner, int64_t outer,
+                          int64_t pitch, int box_inner, int box_outer)
+{
+    const cuuint64_t gdim[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
+    const cuuint64_t gstride[1] = {(cuuint64_t)pitch * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)box_inner, (cuuint32_t)box_outer};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = S.encode(map, dtype == 0 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                                const_cast<void*>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char buf[32];
+        snprintf(buf, sizeof(buf), "%d", (int)r);
+        return fail(ADAPT_ERR_CUDA, "cuTensorMapEncodeTiled failed with CUresult %s", buf);
+    }
+    return ADAPT_OK;
+}
+
+adapt_status_t cached_map(State& S, Plan* pl, bool isA, const void* base, int64_t inner, int64_t outer, int64_t pitch,
+                          int box_inner, int box_outer, CUtensorMap* out)
+{
+    std::lock_guard<std::mutex> lock(pl->mu);
+    MapSlot* slots = isA ? pl->mapA : pl->mapB;
+    for (int i = 0; i < 2; ++i)
+        if (slots[i].ptr == base && slots[i].pitch == pitch) { *out = slots[i].map; return ADAPT_OK; }
+    int& next = isA ? pl->nextA : pl->nextB;
+    MapSlot& sl = slots[next];
+    next ^= 1;
+    adapt_status_t r = encode_map(S, &sl.map, base, pl->s.dtype, inner, outer, pitch, box_inner, box_outer);
+    if (r != ADAPT_OK) { sl.ptr = nullptr; return r; }
+    sl.ptr = base;
+    sl.pitch = pitch;
+    *out = sl.map;
+    return ADAPT_OK;
+}
+
+adapt_status_t launch_pad(State& S, const void* src, void* dst, int64_t outer, int64_t inner, int64_t pitch, cudaStream_t stream)
+{
+    const int64_t chunks = outer * (pitch / 8);
+    const int blocks = (int)std::min<int64_t>(ceil_div(chunks, 256), (int64_t)S.machine.n_sm * 16);
+    pad_copy_kernel<<<blocks, 256, 0, stream>>>((const unsigned short*)src, (unsigned short*)dst, outer, inner, pitch);
+    S.launches.fetch_add(1, std::memory_order_relaxed);
+    CUDA_TRY(cudaGetLastError());
+    return ADAPT_OK;
+}
+
+adapt_status_t launch_reduce(State& S, const float* partial, void* C, int64_t MN, int P_k, int dtype, cudaStream_t stream)
+{
+    const int64_t work = (MN + 3) / 4;
+    const int blocks = (int)std::min<int64_t>(ceil_div(work, 256), (int64_t)S.machine.n_sm * 8);
+    splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(partial, (unsigned short*)C, MN, P_k, dtype);
+    S.launches.fetch_add(1, std::memory_order_relaxed);
+    CUDA_TRY(cudaGetLastError());
+    return ADAPT_OK;
+}
+
+adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* C, cudaStream_t stream)
+{
+    const Shape& s = pl->s;
+    const Config& c = pl->c;
+    const bool a_mn = s.layoutA == ADAPT_COL_MAJOR;       // M contiguous
+    const bool b_mn = s.layoutB == ADAPT_ROW_MAJOR;       // N contiguous
+    const int64_t inA = a_mn ? s.M : s.K, outA = a_mn ? s.K : s.M;
+    const int64_t inB = b_mn ? s.N : s.K, outB = b_mn ? s.K : s.N;
+    const bool padA = c.srcA == ADAPT_SRC_PAD_COPY || ((uintptr_t)A & 15) != 0;
+    const bool padB = c.srcB == ADAPT_SRC_PAD_COPY || ((uintptr_t)B & 15) != 0;
+    const int64_t pitchA = padA ? padded_pitch(inA) : inA;
+    const int64_t pitchB = padB ? padded_pitch(inB) : inB;
+    const size_t szA = padA ? (size_t)round_up(outA * pitchA * 2, 256) : 0;
+    const size_t szB = padB ? (size_t)round_up(outB * pitchB * 2, 256) : 0;
+    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * s.N * 4, 256) : 0;
+    void* ws = nullptr;
+    adapt_status_t r = get_workspace(S, stream, szA + szB + szP, &ws);
+    if (r != ADAPT_OK) return r;
+    uint8_t* w8 = (uint8_t*)ws;
+    const void* a_src = A;
+    const void* b_src = B;
+    if (padA) {
+        if ((r = launch_pad(S, A, w8, outA, inA, pitchA, stream)) != ADAPT_OK) return r;
+        a_src = w8;
+    }
+    if (padB) {
+        if ((r = launch_pad(S, B, w8 + szA, outB, inB, pitchB, stream)) != ADAPT_OK) return r;
+        b_src = w8 + szA;
+    }
+    float* partial = c.P_k > 1 ? (float*)(w8 + szA + szB) : nullptr;
+
+    const int cg = c.cluster;
+    CUtensorMap tmA, tmB;
+    // K-major operand: one box of 64 k x (rows this CTA owns); MN-major operand: boxes of 64 x 64
+    if ((r = cached_map(S, pl, true, a_src, inA, outA, pitchA, 64, a_mn ? 64 : 128, &tmA)) != ADAPT_OK) return r;
+    if ((r = cached_map(S, pl, false, b_src, inB, outB, pitchB, 64, b_mn ? 64 : c.BN / cg, &tmB)) != ADAPT_OK) return r;
+
+    UmmaParams p;
+    p.M = (int)s.M; p.N = (int)s.N; p.K = (int)s.K;
+    p.P_m = c.P_m; p.P_n = c.P_n; p.P_k = c.P_k;
+    p.kb_total = (int)ceil_div(s.K, kUmmaBK);
+    p.kb_per_split = (int)ceil_div(p.kb_total, c.P_k);
+    p.num_units = c.P_m * c.P_n * c.P_k;
+    p.dtype = s.dtype;
+    p.stages = c.stages;
+    p.idesc = umma_idesc(s.dtype, a_mn, b_mn, 128 * cg, c.BN);
+    p.C = C;
+    p.partial = partial;
+    p.c_vec_ok = (s.N % 8 == 0 && ((uintptr_t)C & 15) == 0) ? 1 : 0;
+    p.status = S.d_status;
+
+    UmmaKernel k = launch_map_umma(c.family, c.BN, a_mn, b_mn);
+    if (!k) return fail(ADAPT_ERR_UNSUPPORTED, "no compiled kernel for this tiling key%s");
+    const int slots = S.machine.n_sm / cg;
+    const int grid = std::min(p.num_units, slots) * cg;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)grid, 1, 1);
+    cfg.blockDim = dim3(kUmmaThreads, 1, 1);
+    cfg.dynamicSmemBytes = (size_t)umma_smem_bytes(c.BN, cg, c.stages);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cg;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, k, tmA, tmB, p));
+    S.launches.fetch_add(1, std::memory_order_relaxed);
+    if (c.P_k > 1) return launch_reduce(S, partial, C, s.M * s.N, c.P_k, s.dtype, stream);
+    return ADAPT_OK;
+}
+
+adapt_status_t run_simt(State& S, Plan* pl, const void* A, const void* B, void* C, cudaStream_t stream)
+{
+    const Shape& s = pl->s;
+    const Config& c = pl->c;
+    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * s.N * 4, 256) : 0;
+    void* ws = nullptr;
+    adapt_status_t r = get_workspace(S, stream, szP, &ws);
+    if (r != ADAPT_OK) return r;
+    SimtParams p;
+    p.M = (int)s.M; p.N = (int)s.N; p.K = (int)s.K;
+    if (s.layoutA == ADAPT_ROW_MAJOR) { p.a_sm = s.K; p.a_sk = 1; } else { p.a_sm = 1; p.a_sk = s.M; }
+    if (s.layoutB == ADAPT_ROW_MAJOR) { p.b_sk = s.N; p.b_sn = 1; } else { p.b_sk = 1; p.b_sn = s.K; }
+    p.P_n = c.P_n;
+    p.P_k = c.P_k;
+    p.kb_per_split = (int)ceil_div(ceil_div(s.K, 16), c.P_k);
+    p.dtype = s.dtype;
+    p.C = (unsigned short*)C;
+    p.partial = (float*)ws;
+    dim3 grid((unsigned)((int64_t)c.P_m * c.P_n), (unsigned)c.P_k, 1);
+    simt_gemm_kernel<<<grid, 256, 0, stream>>>((const unsigned short*)A, (const unsigned short*)B, p);
+    S.launches.fetch_add(1, std::memory_order_relaxed);
+    CUDA_TRY(cudaGetLastError());
+    if (c.P_k > 1) return launch_reduce(S, (const float*)ws, C, s.M * s.N, c.P_k, s.dtype, stream);
+    return ADAPT_OK;
+}
+
+adapt_status_t run_skinny(State& S, Plan* pl, const void* A, const void* B, void* C, cudaStream_t stream)
+{
+    const Shape& s = pl->s;
+    const Config& c = pl->c;
+    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * s.N * 4, 256) : 0;
+    void* ws = nullptr;
+    adapt_status_t r = get_workspace(S, stream, szP, &ws);
+    if (r != ADAPT_OK) return r;
+    r = launch_skinny(s, c, A, B, C, (float*)ws, stream);
+    if (r != ADAPT_OK) return fail(r, "skinny kernel launch failed%s");
+    S.launches.fetch_add(1, std::memory_order_relaxed);
+    CUDA_TRY(cudaGetLastError());
+    if (c.P_k > 1) return launch_reduce(S, (const float*)ws, C, s.M * s.N, c.P_k, s.dtype, stream);
+    return ADAPT_OK;
+}
+
+bool overlaps(const void* a, size_t an, const void* b, size_t bn)
+{
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + bn && b0 < a0 + an;
+}
+
+}  // namespace
+
+extern "C" adapt_status_t adapt_matmul(adapt_handle_t plan, const void* A, const void* B, void* C, void* cuda_stream)
+{
+    State& S = st();
+    if (!plan) return fail(ADAPT_ERR_INVALID_ARG, "null plan%s");
+    if (!S.inited) return fail(ADAPT_ERR_NOT_INIT, "adapt_init has not been called%s");
+    Plan* pl = plan;
+    const Shape& s = pl->s;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (pl->noop) return ADAPT_OK;
+    if (!C) return fail(ADAPT_ERR_INVALID_ARG, "null C%s");
+    if (pl->zero_fill) {
+        CUDA_TRY(cudaMemsetAsync(C, 0, (size_t)s.M * s.N * 2, stream));
+        return ADAPT_OK;
+    }
+    if (!A || !B) return fail(ADAPT_ERR_INVALID_ARG, "null operand%s");
+    if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 1) return fail(ADAPT_ERR_INVALID_ARG, "operands must be 2-byte aligned%s");
+    const size_t nA = (size_t)s.M * s.K * 2, nB = (size_t)s.K * s.N * 2, nC = (size_t)s.M * s.N * 2;
+    if (overlaps(C, nC, A, nA) || overlaps(C, nC, B, nB)) return fail(ADAPT_ERR_INVALID_ARG, "C overlaps an input%s");
+    switch (pl->c.family) {
+        case ADAPT_FAM_UMMA_1CTA:
+        case ADAPT_FAM_UMMA_2CTA: return run_umma(S, pl, A, B, C, stream);
+        case ADAPT_FAM_SKINNY: return run_skinny(S, pl, A, B, C, stream);
+        case ADAPT_FAM_SIMT: return run_simt(S, pl, A, B, C, stream);
+    }
+    return fail(ADAPT_ERR_UNSUPPORTED, "unknown kernel family%s");
+}

@@ -1,0 +1,91 @@
+// Internal declarations shared by the host-side selector, the plan cache and the launchers.
+#pragma once
+
+#include <cstdint>
+#include <cstddef>
+#include <vector>
+
+#include "adapt_matmul.h"
+
+namespace adapt {
+
+// ---- machine description (paper Table 1: N_core, buffer capacities) ------------------------
+struct Machine {
+    int n_sm = 148;                     // N_core
+    int smem_bytes = 227 * 1024;        // per-CTA shared memory limit (the paper's L1 capacity)
+    int tmem_cols = 512;                // 128 lanes x 512 fp32 columns per SM (the paper's L0C)
+    int64_t workspace_limit = (int64_t)24 << 30;
+    unsigned family_mask = 0xFu;        // bit f set = family f may be selected
+};
+
+// ---- calibration constants of the latency model (Eq. 8: lambda_r, eta_r, BW_r) ------------
+// Measured on B200 with this library's own kernels (CUDA events); the paper's values are for
+// other hardware and are not printed, so these are this library's.
+struct Calib {
+    double launch_us = 2.2;             // one kernel launch on a busy stream (T_pro/T_epi launches too)
+    double hbm_bw = 6.2e12;             // B/s, large streaming transfers
+    double hbm_ramp_bytes = 24e6;       // bytes at which half of hbm_bw is reached (latency + ramp)
+    double l2_bw_per_sm = 90e9;         // B/s one SM can pull through TMA from L2
+    double tensor_flops = 1.55e15;      // whole chip, kind::f16, BN = 256
+    double eta_mma_bn128 = 0.92;        // relative tensor efficiency at BN = 128
+    double eta_mma_bn64 = 0.62;         // ... at BN = 64 (A-operand smem reads dominate)
+    double eta_2cta = 1.0;              // 2-CTA pairs share B: no extra tensor cost
+    double mem_latency_us = 1.0;        // TMA issue -> data visible (sets Delta_dep with few stages)
+    double tile_epilogue_us_per_kb = 0.012; // drain: TMEM -> registers -> global, per KB of C tile
+    double simt_flops = 12e12;          // CUDA-core tile kernel
+    double skinny_bw_eff = 0.80;        // fraction of hbm_bw the streaming kernel reaches
+    double skinny_mac_rate = 30e12;     // MAC/s ceiling of the warp-level kernel (m padded to 16)
+    double copy_bw_eff = 0.85;          // pad-copy and reduce kernels
+};
+
+// ---- one configuration x of the search set S(b(s)) (Eq. 6) ------------------------------------
+struct Config {
+    int family = ADAPT_FAM_SIMT;
+    int cls = ADAPT_CLASS_COMMON;
+    int BM = 64, BN = 64, BK = 16;
+    int stages = 1;
+    int P_m = 1, P_n = 1, P_k = 1;
+    int cluster = 1;
+    int persistent = 0;
+    int srcA = ADAPT_SRC_LSU, srcB = ADAPT_SRC_LSU;
+    int grid = 1;
+    int smem_bytes = 0;
+    int64_t workspace_bytes = 0;        // total
+    int64_t ws_padA = 0, ws_padB = 0, ws_partial = 0;  // sizes of the three regions
+    double hbm_bytes = 0, t_pro_us = 0, t_main_us = 0, t_epi_us = 0, predicted_us = 0;
+};
+
+struct Shape {
+    int64_t M = 0, N = 0, K = 0;
+    int dtype = 0, layoutA = 0, layoutB = 0;
+};
+
+// Section 4.2 predicate, parameterised by the machine.
+int classify(int64_t M, int64_t N, int64_t m, int64_t n, int64_t m1, int64_t n1, int64_t n_core, int64_t acc_bytes);
+
+// Closed forms (bytes; times in the caller's unit).
+double read_volume(int64_t M, int64_t N, int64_t K, int64_t m1, int64_t n1);                 // Eq. 1
+double write_volume(int cls, int64_t M, int64_t N, int64_t K, int64_t k, int64_t k1);       // Eq. 2-5
+double pipeline_time(int schedule, int64_t Q, int64_t L, double tM, double tP, double Td);  // Eq. 12-14
+
+uint64_t pack_tiling_key(const Shape& s, const Config& c);
+bool unpack_tiling_key(uint64_t key, Shape* flags, Config* c);   // fills the key's fields only
+
+// Enumerate the legal configurations for a shape (capacity and instruction-shape checks done),
+// each scored by the model, sorted best first with the deterministic tie-break.
+void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::vector<Config>* out);
+
+// Rebuild the full Config a key describes for this shape; false if it is not legal.
+bool config_from_key(const Shape& s, uint64_t key, const Machine& m, const Calib& cal, Config* out);
+
+void fill_info(const Shape& s, const Config& c, adapt_plan_info_t* out);
+
+inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
+
+// Operand pitch in elements after the Padding module (16-byte multiple).
+inline int64_t padded_pitch(int64_t inner) { return round_up(inner, 8); }
+
+const Calib& default_calib();
+
+}  // namespace adapt

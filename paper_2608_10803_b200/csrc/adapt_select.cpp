@@ -1,0 +1,478 @@
+// Host-side selector: taxonomy (Section 4.2), candidate enumeration with capacity checks
+// (Eq. 6), analytical latency model (Eq. 7-11 with the schedules of Eq. 12-14) and the 64-bit
+// TilingKey.  No CUDA here.
+#include "adapt_internal.h"
+
+#include <algorithm>
+#include <cmath>
+
+namespace adapt {
+
+const Calib& default_calib()
+{
+    static Calib c;
+    return c;
+}
+
+// ---- Section 4.2: two predicates, four templates ---------------------------------------------
+int classify(int64_t M, int64_t N, int64_t m, int64_t n, int64_t m1, int64_t n1, int64_t n_core, int64_t acc_bytes)
+{
+    if (M < 1 || N < 1 || m < 1 || n < 1 || m1 < 1 || n1 < 1 || n_core < 1 || acc_bytes < 1) return -1;
+    const int64_t P_m = ceil_div(M, m), P_n = ceil_div(N, n);
+    const bool enough_tasks = P_m * P_n >= n_core;            // X axis: spatial parallelism
+    const bool on_chip = m1 * n1 * 4 <= acc_bytes;            // Y axis: fp32 accumulation tile fits
+    if (enough_tasks) return on_chip ? ADAPT_CLASS_COMMON : ADAPT_CLASS_SINGLE_CORE_SPLIT_K;
+    return on_chip ? ADAPT_CLASS_MULTI_CORE_SPLIT_K : ADAPT_CLASS_HYBRID_SPLIT_K;
+}
+
+// ---- Eq. 1-5 ----------------------------------------------------------------------------------
+double read_volume(int64_t M, int64_t N, int64_t K, int64_t m1, int64_t n1)
+{
+    return 2.0 * (double)M * (double)N * (double)K * (1.0 / (double)m1 + 1.0 / (double)n1);
+}
+
+double write_volume(int cls, int64_t M, int64_t N, int64_t K, int64_t k, int64_t k1)
+{
+    const double MN = (double)M * (double)N;
+    switch (cls) {
+        case ADAPT_CLASS_COMMON: return 2.0 * MN;
+        case ADAPT_CLASS_SINGLE_CORE_SPLIT_K: return 4.0 * MN * (double)ceil_div(K, k1) + 2.0 * MN;
+        case ADAPT_CLASS_MULTI_CORE_SPLIT_K: return 4.0 * MN * (double)ceil_div(K, k) + 2.0 * MN;
+        case ADAPT_CLASS_HYBRID_SPLIT_K:
+            return (double)ceil_div(K, k) * (4.0 * MN * (double)ceil_div(k, k1)) + 2.0 * MN;
+        default: return -1.0;
+    }
+}
+
+// ---- Eq. 12-14 --------------------------------------------------------------------------------
+double pipeline_time(int schedule, int64_t Q, int64_t L, double tM, double tP, double Td)
+{
+    const double ii = std::max(tM, tP);
+    switch (schedule) {
+        case 0: return (double)Q * ((double)L * (tM + tP) + Td);                              // Eq. 12 per tile
+        case 1: return (double)Q * (tM + (double)(L - 1) * ii + tP + Td);                     // Eq. 13 per tile
+        case 2: return tM + ((double)Q * (double)L - 1.0) * ii + tP + (double)Q * Td;         // Eq. 14
+        default: return -1.0;
+    }
+}
+
+// ---- TilingKey --------------------------------------------------------------------------------
+static int ilog2(int v) { int r = 0; while ((1 << (r + 1)) <= v) ++r; return r; }
+
+uint64_t pack_tiling_key(const Shape& s, const Config& c)
+{
+    uint64_t k = 0;
+    k |= (uint64_t)(c.cls & 3) << 62;
+    k |= (uint64_t)(c.family & 7) << 59;
+    k |= (uint64_t)((c.BM / 16) & 31) << 54;
+    k |= (uint64_t)((c.BN / 16) & 63) << 48;
+    k |= (uint64_t)(ilog2(std::max(c.BK, 16) / 16) & 3) << 46;
+    k |= (uint64_t)(c.stages & 15) << 42;
+    k |= (uint64_t)(c.P_k & 1023) << 32;
+    k |= (uint64_t)(c.persistent & 1) << 31;
+    k |= (uint64_t)(c.srcA & 3) << 29;
+    k |= (uint64_t)(c.srcB & 3) << 27;
+    k |= (uint64_t)(s.dtype & 1) << 26;
+    k |= (uint64_t)(s.layoutA & 1) << 25;
+    k |= (uint64_t)(s.layoutB & 1) << 24;
+    k |= (uint64_t)(ilog2(std::max(c.cluster, 1)) & 3) << 22;
+    return k;
+}
+
+bool unpack_tiling_key(uint64_t k, Shape* s, Config* c)
+{
+    if (k & ((1ull << 22) - 1)) return false;
+    c->cls = (int)((k >> 62) & 3);
+    c->family = (int)((k >> 59) & 7);
+    c->BM = (int)((k >> 54) & 31) * 16;
+    c->BN = (int)((k >> 48) & 63) * 16;
+    c->BK = 16 << (int)((k >> 46) & 3);
+    c->stages = (int)((k >> 42) & 15);
+    c->P_k = (int)((k >> 32) & 1023);
+    c->persistent = (int)((k >> 31) & 1);
+    c->srcA = (int)((k >> 29) & 3);
+    c->srcB = (int)((k >> 27) & 3);
+    s->dtype = (int)((k >> 26) & 1);
+    s->layoutA = (int)((k >> 25) & 1);
+    s->layoutB = (int)((k >> 24) & 1);
+    c->cluster = 1 << (int)((k >> 22) & 3);
+    return true;
+}
+
+// ---- model --------------------------------------------------------------------------------------
+
+static const double kL2Bytes = 96e6;       // share of the 126 MB L2 one operand can expect to keep
+static const int kGroupM = 16;             // tile rasterisation: m-blocks per group (matches the kernel)
+
+static double copy_time_us(double bytes, const Calib& cal)
+{
+    return bytes / (cal.hbm_bw * cal.copy_bw_eff) * 1e6;
+}
+
+// Inner extent (contiguous dimension) of each operand in elements.
+static int64_t innerA(const Shape& s) { return s.layoutA == ADAPT_ROW_MAJOR ? s.K : s.M; }
+static int64_t outerA(const Shape& s) { return s.layoutA == ADAPT_ROW_MAJOR ? s.M : s.K; }
+static int64_t innerB(const Shape& s) { return s.layoutB == ADAPT_ROW_MAJOR ? s.N : s.K; }
+static int64_t outerB(const Shape& s) { return s.layoutB == ADAPT_ROW_MAJOR ? s.K : s.N; }
+
+static void finish_common(const Shape& s, Config& c, const Calib& cal)
+{
+    c.workspace_bytes = c.ws_padA + c.ws_padB + c.ws_partial;
+    c.predicted_us = cal.launch_us + c.t_pro_us + c.t_main_us + c.t_epi_us;
+    (void)s;
+}
+
+// Prologue (Section 5.2 "Prologue"): the Padding module re-pitches an operand whose rows are not
+// 16-byte multiples, reading it once and writing the padded copy once.
+static void model_prologue(const Shape& s, Config& c, const Calib& cal)
+{
+    c.t_pro_us = 0;
+    c.ws_padA = c.ws_padB = 0;
+    if (c.srcA == ADAPT_SRC_PAD_COPY) {
+        const double src = 2.0 * (double)s.M * (double)s.K;
+        c.ws_padA = round_up(outerA(s) * padded_pitch(innerA(s)) * 2, 256);
+        c.t_pro_us += cal.launch_us + copy_time_us(src + (double)c.ws_padA, cal);
+        c.hbm_bytes += src + (double)c.ws_padA;
+    }
+    if (c.srcB == ADAPT_SRC_PAD_COPY) {
+        const double src = 2.0 * (double)s.K * (double)s.N;
+        c.ws_padB = round_up(outerB(s) * padded_pitch(innerB(s)) * 2, 256);
+        c.t_pro_us += cal.launch_us + copy_time_us(src + (double)c.ws_padB, cal);
+        c.hbm_bytes += src + (double)c.ws_padB;
+    }
+}
+
+// Epilogue (Eq. 11): cross-CTA reduction of the fp32 partials (Eq. 4's extra 4*M*N*P_k bytes are
+// written by the main loop and read back here), then the single 16-bit write.
+static void model_epilogue(const Shape& s, Config& c, const Calib& cal)
+{
+    c.t_epi_us = 0;
+    c.ws_partial = 0;
+    if (c.P_k > 1) {
+        const double MN = (double)s.M * (double)s.N;
+        c.ws_partial = round_up((int64_t)c.P_k * s.M * s.N * 4, 256);
+        double part = 4.0 * MN * c.P_k;
+        // partials that fit in L2 are read back at L2 speed; model that as half the HBM cost
+        const double factor = part <= kL2Bytes ? 0.5 : 1.0;
+        c.t_epi_us = cal.launch_us + copy_time_us(part * factor + 2.0 * MN, cal);
+        c.hbm_bytes += part * (1.0 + factor);
+    }
+}
+
+static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Config& c)
+{
+    const int64_t kblocks = ceil_div(s.K, c.BK);
+    const int64_t L = ceil_div(kblocks, c.P_k);
+    const int64_t units = (int64_t)c.P_m * c.P_n * c.P_k;
+    const int64_t slots = m.n_sm / c.cluster;
+    const int64_t Q = ceil_div(units, slots);
+    c.grid = (int)(std::min(units, slots) * c.cluster);
+
+    const double MK = (double)s.M * s.K, KN = (double)s.K * s.N, MN = (double)s.M * s.N;
+    // HBM traffic: operands once, plus re-reads of B when it cannot stay in L2 across m-groups.
+    double rB = 1.0, rA = 1.0;
+    const int64_t rows_per_group = (int64_t)kGroupM * c.BM;
+    if (2.0 * KN > kL2Bytes) rB = (double)ceil_div(s.M, rows_per_group);
+    if (rB > 1.0 && 2.0 * MK <= kL2Bytes) {          // alternatively A stays resident and B streams once
+        rB = 1.0;
+    }
+    c.hbm_bytes = 2.0 * (MK * rA + KN * rB) + (c.P_k > 1 ? 0.0 : 2.0 * MN);
+
+    // per-SM stage: each CTA loads its 128 rows of A and its share of the BN columns of B
+    const double bn_per_cta = (double)c.BN / c.cluster;
+    const double stage_bytes = 2.0 * c.BK * (128.0 + bn_per_cta);
+    double tM = stage_bytes / cal.l2_bw_per_sm * 1e6;
+    double eta = c.BN >= 256 ? 1.0 : (c.BN >= 128 ? cal.eta_mma_bn128 : cal.eta_mma_bn64);
+    if (c.cluster == 2) eta *= cal.eta_2cta;
+    const double tP = 2.0 * 128.0 * c.BN * c.BK / (cal.tensor_flops / m.n_sm * eta) * 1e6;
+    // Delta_dep (Eq. 9): with S stages only S-1 loads are in flight while one is consumed, so a
+    // slice cannot issue faster than latency / (S-1); one stage serialises load and compute.
+    double pipe;
+    const double out_tile_kb = (c.P_k > 1 ? 4.0 : 2.0) * 128.0 * c.BN / 1024.0;
+    const double t_epi_tile = out_tile_kb * cal.tile_epilogue_us_per_kb;
+    if (c.stages <= 1) {
+        pipe = pipeline_time(0, Q, L, tM + cal.mem_latency_us, tP, t_epi_tile);
+    } else {
+        tM = std::max(tM, cal.mem_latency_us / (c.stages - 1));
+        const double ii = std::max(tM, tP);
+        // two TMEM accumulators: a tile's drain overlaps the next tile's main loop
+        const double exposed = std::max(0.0, t_epi_tile - (double)L * ii);
+        if (c.persistent) pipe = cal.mem_latency_us + pipeline_time(2, Q, L, tM, tP, exposed) + t_epi_tile;
+        else pipe = cal.mem_latency_us + pipeline_time(1, Q, L, tM, tP, t_epi_tile);
+    }
+    model_prologue(s, c, cal);
+    model_epilogue(s, c, cal);
+    const double t_hbm = c.hbm_bytes / cal.hbm_bw * 1e6 - c.t_pro_us - c.t_epi_us;
+    c.t_main_us = std::max(pipe, t_hbm);
+    finish_common(s, c, cal);
+}
+
+static void model_skinny(const Shape& s, const Machine& m, const Calib& cal, Config& c)
+{
+    const double MK = (double)s.M * s.K, KN = (double)s.K * s.N, MN = (double)s.M * s.N;
+    c.hbm_bytes = 2.0 * (MK + KN) + (c.P_k > 1 ? 0.0 : 2.0 * MN);
+    const int64_t units = (int64_t)c.P_m * c.P_n * c.P_k;
+    c.grid = (int)units;
+    const int64_t Q = ceil_div(units, (int64_t)m.n_sm * 2);      // two CTAs resident per SM
+    const double macs = (double)std::max(s.M, s.N) * s.K * 16.0;  // the small side is padded to 16
+    const double per_cta_bytes = 2.0 * ((double)c.BN * ceil_div(s.K, c.P_k));
+    const double t_cta = per_cta_bytes / (cal.l2_bw_per_sm * 0.5) * 1e6 + cal.mem_latency_us;
+    model_epilogue(s, c, cal);
+    const double t_stream = c.hbm_bytes / (cal.hbm_bw * cal.skinny_bw_eff) * 1e6 - c.t_epi_us;
+    const double t_alu = macs / cal.skinny_mac_rate * 1e6;
+    c.t_pro_us = 0;
+    c.t_main_us = std::max({t_stream, t_alu, (double)Q * t_cta});
+    finish_common(s, c, cal);
+}
+
+static void model_simt(const Shape& s, const Machine& m, const Calib& cal, Config& c)
+{
+    const double MK = (double)s.M * s.K, KN = (double)s.K * s.N, MN = (double)s.M * s.N;
+    const int64_t units = (int64_t)c.P_m * c.P_n * c.P_k;
+    c.grid = (int)units;
+    c.hbm_bytes = 2.0 * (MK + KN) + (c.P_k > 1 ? 0.0 : 2.0 * MN);
+    const int64_t resident = (int64_t)m.n_sm * 4;
+    const int64_t Q = ceil_div(units, resident);
+    // a full 64x64 tile costs the same whether or not the shape fills it
+    const double tile_flops = 2.0 * c.BM * c.BN * (double)ceil_div(s.K, c.P_k);
+    const double t_tile = tile_flops / (cal.simt_flops / resident) * 1e6 + cal.mem_latency_us;
+    model_epilogue(s, c, cal);
+    const double t_hbm = c.hbm_bytes / (cal.hbm_bw * 0.6) * 1e6 - c.t_epi_us;
+    c.t_pro_us = 0;
+    c.t_main_us = std::max((double)Q * t_tile, t_hbm);
+    finish_common(s, c, cal);
+}
+
+// ---- legality (the constraint M(b,x,s) <= C_limit of Eq. 6) -----------------------------------
+
+static int umma_smem_bytes(const Config& c)
+{
+    const int bn_per_cta = c.BN / c.cluster;
+    const int stage = 2 * c.BK * (128 + bn_per_cta);
+    return c.stages * stage + 1024 /*alignment slack*/ + 256 /*barriers, tmem pointer*/;
+}
+
+static bool aligned16(int64_t inner_elems) { return inner_elems % 8 == 0; }
+
+static bool legal_umma(const Shape& s, const Machine& m, Config& c)
+{
+    if (!(m.family_mask & (1u << c.family))) return false;
+    if (c.BK != 64) return false;
+    if (c.family == ADAPT_FAM_UMMA_1CTA) {
+        if (c.BM != 128 || c.cluster != 1) return false;
+        if (c.BN != 64 && c.BN != 128 && c.BN != 256) return false;
+    } else {
+        if (c.BM != 256 || c.cluster != 2) return false;
+        if (c.BN != 128 && c.BN != 256) return false;
+    }
+    if (c.BN % 16 != 0 || c.BN > 256) return false;                 // UMMA shape rule for M = 128/256
+    if (2 * c.BN > m.tmem_cols) return false;                       // two accumulator buffers in TMEM
+    if (c.stages < 1 || c.stages > 12) return false;
+    c.smem_bytes = umma_smem_bytes(c);
+    if (c.smem_bytes > m.smem_bytes) return false;
+    const int64_t kblocks = ceil_div(s.K, c.BK);
+    if (c.P_k < 1 || c.P_k > 1023 || c.P_k > kblocks) return false;
+    if (ceil_div(kblocks, ceil_div(kblocks, c.P_k)) != c.P_k) return false;   // no empty split
+    // operand sources: TMA needs a 16-byte row pitch
+    if (c.srcA == ADAPT_SRC_TMA && !aligned16(innerA(s))) return false;
+    if (c.srcB == ADAPT_SRC_TMA && !aligned16(innerB(s))) return false;
+    if (c.srcA == ADAPT_SRC_LSU || c.srcB == ADAPT_SRC_LSU) return false;
+    if (c.srcA == ADAPT_SRC_PAD_COPY && aligned16(innerA(s))) return false;    // nothing to pad
+    if (c.srcB == ADAPT_SRC_PAD_COPY && aligned16(innerB(s))) return false;
+    c.P_m = (int)ceil_div(s.M, c.BM);
+    c.P_n = (int)ceil_div(s.N, c.BN);
+    if ((int64_t)c.P_m * c.P_n * c.P_k > (int64_t)1 << 30) return false;
+    c.persistent = 1;
+    return true;
+}
+
+static bool legal_skinny(const Shape& s, const Machine& m, Config& c)
+{
+    if (!(m.family_mask & (1u << ADAPT_FAM_SKINNY))) return false;
+    if (std::min(s.M, s.N) > 16) return false;
+    if (c.BM != 16 || c.BK != 16 || c.cluster != 1) return false;
+    if (c.BN != 128 && c.BN != 256 && c.BN != 512) return false;     // streamed rows/columns per CTA
+    if (c.srcA != ADAPT_SRC_LSU || c.srcB != ADAPT_SRC_LSU) return false;
+    if (c.stages != 1) return false;
+    const int64_t ksteps = ceil_div(s.K, 256);                       // splits are whole staging chunks
+    if (c.P_k < 1 || c.P_k > 1023 || c.P_k > ksteps) return false;
+    if (ceil_div(ksteps, ceil_div(ksteps, c.P_k)) != c.P_k) return false;
+    c.P_m = 1;
+    c.P_n = (int)ceil_div(std::max(s.M, s.N), c.BN);
+    c.persistent = 0;
+    c.smem_bytes = 0;
+    return true;
+}
+
+static bool legal_simt(const Shape& s, const Machine& m, Config& c)
+{
+    if (!(m.family_mask & (1u << ADAPT_FAM_SIMT))) return false;
+    if (c.BM != 64 || c.BN != 64 || c.BK != 16 || c.cluster != 1 || c.stages != 1) return false;
+    if (c.srcA != ADAPT_SRC_LSU || c.srcB != ADAPT_SRC_LSU) return false;
+    const int64_t kblocks = ceil_div(s.K, c.BK);
+    if (c.P_k < 1 || c.P_k > 1023 || c.P_k > kblocks) return false;
+    if (ceil_div(kblocks, ceil_div(kblocks, c.P_k)) != c.P_k) return false;
+    c.P_m = (int)ceil_div(s.M, c.BM);
+    c.P_n = (int)ceil_div(s.N, c.BN);
+    if ((int64_t)c.P_m * c.P_n > (int64_t)1 << 30) return false;
+    c.persistent = 0;
+    c.smem_bytes = 0;
+    return true;
+}
+
+static bool finalize(const Shape& s, const Machine& m, const Calib& cal, Config& c)
+{
+    bool ok = false;
+    switch (c.family) {
+        case ADAPT_FAM_UMMA_1CTA:
+        case ADAPT_FAM_UMMA_2CTA: ok = legal_umma(s, m, c); break;
+        case ADAPT_FAM_SKINNY: ok = legal_skinny(s, m, c); break;
+        case ADAPT_FAM_SIMT: ok = legal_simt(s, m, c); break;
+        default: ok = false;
+    }
+    if (!ok) return false;
+    // taxonomy label: X axis from the spatial task count, Y axis from the fp32 tile against one
+    // SM's accumulator budget (half of TMEM, so that two accumulators can alternate)
+    const int64_t acc_budget = (int64_t)128 * (m.tmem_cols / 2) * 4;
+    const bool enough = (int64_t)c.P_m * c.P_n >= m.n_sm;
+    const bool on_chip = (int64_t)c.BM * c.BN * 4 <= acc_budget || c.family >= ADAPT_FAM_SKINNY;
+    c.cls = enough ? (on_chip ? ADAPT_CLASS_COMMON : ADAPT_CLASS_SINGLE_CORE_SPLIT_K)
+                   : (on_chip ? ADAPT_CLASS_MULTI_CORE_SPLIT_K : ADAPT_CLASS_HYBRID_SPLIT_K);
+    switch (c.family) {
+        case ADAPT_FAM_UMMA_1CTA:
+        case ADAPT_FAM_UMMA_2CTA: model_umma(s, m, cal, c); break;
+        case ADAPT_FAM_SKINNY: model_skinny(s, m, cal, c); break;
+        default: model_simt(s, m, cal, c); break;
+    }
+    if (c.workspace_bytes > m.workspace_limit) return false;
+    return true;
+}
+
+// P_k candidates: 1, and when the spatial tasks leave SMs idle, the counts that bring the grid to
+// about one or two CTAs per slot, plus powers of two in between.
+static void split_candidates(int64_t tiles_mn, int64_t slots, int64_t ksteps, int64_t min_steps, std::vector<int>* out)
+{
+    out->clear();
+    out->push_back(1);
+    if (tiles_mn >= 4 * slots) return;
+    const int64_t max_pk = std::min<int64_t>(1023, ksteps / std::max<int64_t>(1, min_steps));
+    std::vector<int64_t> want;
+    for (int64_t mult = 1; mult <= 4; mult *= 2) {
+        want.push_back(mult * slots / tiles_mn);
+        want.push_back(ceil_div(mult * slots, tiles_mn));
+    }
+    for (int64_t p = 2; p <= 1024; p *= 2) want.push_back(p);
+    want.push_back(3); want.push_back(6); want.push_back(12); want.push_back(24);
+    for (int64_t w : want) {
+        if (w < 2 || w > max_pk) continue;
+        // normalise so that no split is empty
+        const int64_t per = ceil_div(ksteps, w);
+        const int p = (int)ceil_div(ksteps, per);
+        if (p >= 2 && std::find(out->begin(), out->end(), p) == out->end()) out->push_back(p);
+    }
+    std::sort(out->begin(), out->end());
+}
+
+void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::vector<Config>* out)
+{
+    out->clear();
+    if (s.M < 1 || s.N < 1 || s.K < 1) return;
+    std::vector<int> pks;
+    // --- tcgen05 families ---
+    const int srcA = aligned16(innerA(s)) ? ADAPT_SRC_TMA : ADAPT_SRC_PAD_COPY;
+    const int srcB = aligned16(innerB(s)) ? ADAPT_SRC_TMA : ADAPT_SRC_PAD_COPY;
+    for (int fam = ADAPT_FAM_UMMA_1CTA; fam <= ADAPT_FAM_UMMA_2CTA; ++fam) {
+        const int BM = fam == ADAPT_FAM_UMMA_1CTA ? 128 : 256;
+        const int cluster = fam == ADAPT_FAM_UMMA_1CTA ? 1 : 2;
+        for (int BN : {64, 128, 256}) {
+            const int64_t tiles = ceil_div(s.M, BM) * ceil_div(s.N, BN);
+            split_candidates(tiles, m.n_sm / cluster, ceil_div(s.K, 64), 2, &pks);
+            // ring depth: the deepest that fits, and a double buffer (Eq. 13) for comparison
+            Config probe;
+            probe.family = fam; probe.BM = BM; probe.BN = BN; probe.BK = 64; probe.cluster = cluster;
+            int deepest = 0;
+            for (int st = 12; st >= 2; --st) {
+                probe.stages = st;
+                if (umma_smem_bytes(probe) <= m.smem_bytes) { deepest = st; break; }
+            }
+            if (deepest > 8) deepest = 8;
+            std::vector<int> depths = {deepest};
+            if (deepest > 4) depths.push_back(4);
+            if (deepest > 2) depths.push_back(2);
+            for (int st : depths) {
+                for (int pk : pks) {
+                    Config c;
+                    c.family = fam; c.BM = BM; c.BN = BN; c.BK = 64; c.cluster = cluster;
+                    c.stages = st; c.P_k = pk; c.srcA = srcA; c.srcB = srcB;
+                    if (finalize(s, m, cal, c)) out->push_back(c);
+                }
+            }
+        }
+    }
+    // --- warp-level streaming family ---
+    if (std::min(s.M, s.N) <= 16) {
+        for (int BN : {128, 256, 512}) {
+            const int64_t tiles = ceil_div(std::max(s.M, s.N), BN);
+            split_candidates(tiles, (int64_t)m.n_sm * 2, ceil_div(s.K, 256), 1, &pks);
+            for (int pk : pks) {
+                Config c;
+                c.family = ADAPT_FAM_SKINNY; c.BM = 16; c.BN = BN; c.BK = 16; c.stages = 1; c.P_k = pk;
+                c.srcA = c.srcB = ADAPT_SRC_LSU;
+                if (finalize(s, m, cal, c)) out->push_back(c);
+            }
+        }
+    }
+    // --- CUDA-core family: always legal ---
+    {
+        const int64_t tiles = ceil_div(s.M, 64) * ceil_div(s.N, 64);
+        split_candidates(tiles, (int64_t)m.n_sm * 4, ceil_div(s.K, 16), 4, &pks);
+        for (int pk : pks) {
+            Config c;
+            c.family = ADAPT_FAM_SIMT; c.BM = 64; c.BN = 64; c.BK = 16; c.stages = 1; c.P_k = pk;
+            c.srcA = c.srcB = ADAPT_SRC_LSU;
+            if (finalize(s, m, cal, c)) out->push_back(c);
+        }
+    }
+    // argmin of Eq. 6 with a deterministic tie-break: time, then fewer splits, then smaller
+    // workspace, then enumeration order (stable sort keeps it)
+    std::stable_sort(out->begin(), out->end(), [](const Config& a, const Config& b) {
+        if (a.predicted_us != b.predicted_us) return a.predicted_us < b.predicted_us;
+        if (a.P_k != b.P_k) return a.P_k < b.P_k;
+        return a.workspace_bytes < b.workspace_bytes;
+    });
+}
+
+bool config_from_key(const Shape& s, uint64_t key, const Machine& m, const Calib& cal, Config* out)
+{
+    Shape flags;
+    Config c;
+    if (!unpack_tiling_key(key, &flags, &c)) return false;
+    if (flags.dtype != s.dtype || flags.layoutA != s.layoutA || flags.layoutB != s.layoutB) return false;
+    if (s.M < 1 || s.N < 1 || s.K < 1) return false;
+    const int want_cls = c.cls;
+    Machine all = m;
+    all.family_mask = m.family_mask;
+    if (!finalize(s, all, cal, c)) return false;
+    if (c.cls != want_cls) return false;
+    if (pack_tiling_key(s, c) != key) return false;
+    *out = c;
+    return true;
+}
+
+void fill_info(const Shape& s, const Config& c, adapt_plan_info_t* o)
+{
+    o->tiling_key = pack_tiling_key(s, c);
+    o->M = s.M; o->N = s.N; o->K = s.K;
+    o->dtype = s.dtype; o->layoutA = s.layoutA; o->layoutB = s.layoutB;
+    o->taxonomy_class = c.cls; o->family = c.family;
+    o->BM = c.BM; o->BN = c.BN; o->BK = c.BK; o->stages = c.stages;
+    o->P_m = c.P_m; o->P_n = c.P_n; o->P_k = c.P_k; o->cluster = c.cluster;
+    o->srcA = c.srcA; o->srcB = c.srcB; o->grid = c.grid; o->reserved = 0;
+    o->workspace_bytes = c.workspace_bytes;
+    o->flops = 2.0 * (double)s.M * (double)s.N * (double)s.K;
+    o->hbm_bytes = c.hbm_bytes;
+    o->t_pro_us = c.t_pro_us; o->t_main_us = c.t_main_us; o->t_epi_us = c.t_epi_us;
+    o->predicted_us = c.predicted_us;
+}
+
+}  // namespace adapt

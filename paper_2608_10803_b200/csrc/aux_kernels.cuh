@@ -1,0 +1,181 @@
+// CUDA-core kernels around the tensor-core path: the Padding prologue (Table 2, Section 5.2
+// "Prologue"), the cross-CTA reduction of split-K partials (Eq. 4, Eq. 11 "T_cross_reduce"),
+// and the always-legal CUDA-core tile GEMM.
+#pragma once
+
+#include <cstdint>
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+
+namespace adapt {
+
+__device__ __forceinline__ float load16_as_float(const unsigned short* p, int dtype)
+{
+    const unsigned short v = *p;
+    if (dtype == 0) return __half2float(*reinterpret_cast<const __half*>(&v));
+    return __uint_as_float((uint32_t)v << 16);
+}
+__device__ __forceinline__ unsigned short float_to_16(float a, int dtype)
+{
+    if (dtype == 0) { __half h = __float2half_rn(a); return *reinterpret_cast<unsigned short*>(&h); }
+    __nv_bfloat16 h = __float2bfloat16_rn(a);
+    return *reinterpret_cast<unsigned short*>(&h);
+}
+
+// ---- Padding: re-pitch a dense [outer][inner] 16-bit matrix to [outer][pitch], pitch % 8 == 0 ----
+// One thread produces one 16-byte chunk of the destination.  The pad columns are never read by
+// the GEMM (the tensor map's extent stays `inner`), so they are written as zeros only to keep
+// the workspace deterministic.
+__global__ void __launch_bounds__(256)
+pad_copy_kernel(const unsigned short* __restrict__ src, unsigned short* __restrict__ dst,
+                int64_t outer, int64_t inner, int64_t pitch)
+{
+    const int64_t chunks_per_row = pitch / 8;
+    const int64_t total = outer * chunks_per_row;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = i / chunks_per_row;
+        const int64_t c = (i - row * chunks_per_row) * 8;
+        const unsigned short* s = src + row * inner + c;
+        unsigned short v[8];
+        if (c + 8 <= inner) {
+            if ((reinterpret_cast<uintptr_t>(s) & 3) == 0) {
+                const uint32_t* s32 = reinterpret_cast<const uint32_t*>(s);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t w = __ldg(s32 + j);
+                    v[2 * j] = (unsigned short)(w & 0xffffu);
+                    v[2 * j + 1] = (unsigned short)(w >> 16);
+                }
+            } else {
+                // 2-byte aligned only: one leading element, three aligned words, one trailing element
+                v[0] = __ldg(s);
+                const uint32_t* s32 = reinterpret_cast<const uint32_t*>(s + 1);
+#pragma unroll
+                for (int j = 0; j < 3; ++j) {
+                    const uint32_t w = __ldg(s32 + j);
+                    v[1 + 2 * j] = (unsigned short)(w & 0xffffu);
+                    v[2 + 2 * j] = (unsigned short)(w >> 16);
+                }
+                v[7] = __ldg(s + 7);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = (c + j < inner) ? __ldg(s + j) : (unsigned short)0;
+        }
+        uint4 o;
+        o.x = (uint32_t)v[0] | ((uint32_t)v[1] << 16);
+        o.y = (uint32_t)v[2] | ((uint32_t)v[3] << 16);
+        o.z = (uint32_t)v[4] | ((uint32_t)v[5] << 16);
+        o.w = (uint32_t)v[6] | ((uint32_t)v[7] << 16);
+        *reinterpret_cast<uint4*>(dst + row * pitch + c) = o;
+    }
+}
+
+// ---- split-K reduction: C = RN16( sum_{p = 0..P_k-1} partial[p] ), ascending p, fp32 ---------------
+// The order is fixed, so the result does not depend on which CTA finished first.
+__global__ void __launch_bounds__(256)
+splitk_reduce_kernel(const float* __restrict__ partial, unsigned short* __restrict__ C,
+                     int64_t MN, int P_k, int dtype)
+{
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    if ((MN & 3) == 0 && (reinterpret_cast<uintptr_t>(C) & 7) == 0) {
+        const int64_t n4 = MN >> 2;
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+            float4 acc = __ldcs(reinterpret_cast<const float4*>(partial) + i);
+            for (int p = 1; p < P_k; ++p) {
+                const float4 v = __ldcs(reinterpret_cast<const float4*>(partial + (int64_t)p * MN) + i);
+                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            }
+            uint2 o;
+            o.x = (uint32_t)float_to_16(acc.x, dtype) | ((uint32_t)float_to_16(acc.y, dtype) << 16);
+            o.y = (uint32_t)float_to_16(acc.z, dtype) | ((uint32_t)float_to_16(acc.w, dtype) << 16);
+            reinterpret_cast<uint2*>(C)[i] = o;
+        }
+    } else {
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < MN; i += stride) {
+            float acc = partial[i];
+            for (int p = 1; p < P_k; ++p) acc += partial[(int64_t)p * MN + i];
+            C[i] = float_to_16(acc, dtype);
+        }
+    }
+}
+
+// ---- CUDA-core tile GEMM: 64 x 64 tile, 256 threads, 4 x 4 outputs per thread ---------------------
+// Legal for every shape, layout and alignment (all accesses are element-wise and predicated).
+// fp32 FMA in ascending k.  blockIdx.x is the tile, blockIdx.y the k split; with P_k > 1 it writes fp32 partials.
+struct SimtParams {
+    int M, N, K;
+    int64_t a_sm, a_sk;          // element strides of A along m and k
+    int64_t b_sk, b_sn;          // element strides of B along k and n
+    int P_n, P_k, kb_per_split;  // n tiles; k splits; k-blocks of 16 per split
+    int dtype;
+    unsigned short* C;
+    float* partial;
+};
+
+__global__ void __launch_bounds__(256)
+simt_gemm_kernel(const unsigned short* __restrict__ A, const unsigned short* __restrict__ B, const SimtParams p)
+{
+    __shared__ float sA[16][64 + 4];
+    __shared__ float sB[16][64 + 4];
+    const int tid = threadIdx.x;
+    const int m0 = (int)(blockIdx.x / p.P_n) * 64, n0 = (int)(blockIdx.x % p.P_n) * 64;
+    const int split = blockIdx.y;
+    const int k_begin = split * p.kb_per_split * 16;
+    const int k_end = min(p.K, k_begin + p.kb_per_split * 16);
+    const int tx = tid & 15, ty = tid >> 4;       // thread's 4 columns: tx*4.., 4 rows: ty*4..
+    float acc[4][4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+    for (int k0 = k_begin; k0 < k_end; k0 += 16) {
+        // 64 x 16 elements of each operand, 4 per thread; index so that consecutive threads walk
+        // the contiguous dimension of the operand
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+            const int e = tid + it * 256;
+            int am, ak;
+            if (p.a_sk == 1) { ak = e & 15; am = e >> 4; } else { am = e & 63; ak = e >> 6; }
+            float va = 0.f;
+            if (m0 + am < p.M && k0 + ak < k_end)
+                va = load16_as_float(A + (int64_t)(m0 + am) * p.a_sm + (int64_t)(k0 + ak) * p.a_sk, p.dtype);
+            sA[ak][am] = va;
+            int bn, bk;
+            if (p.b_sn == 1) { bn = e & 63; bk = e >> 6; } else { bk = e & 15; bn = e >> 4; }
+            float vb = 0.f;
+            if (n0 + bn < p.N && k0 + bk < k_end)
+                vb = load16_as_float(B + (int64_t)(k0 + bk) * p.b_sk + (int64_t)(n0 + bn) * p.b_sn, p.dtype);
+            sB[bk][bn] = vb;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) a[i] = sA[kk][ty * 4 + i];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) b[j] = sB[kk][tx * 4 + j];
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + ty * 4 + i;
+        if (m >= p.M) continue;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int n = n0 + tx * 4 + j;
+            if (n >= p.N) continue;
+            if (p.P_k == 1) p.C[(int64_t)m * p.N + n] = float_to_16(acc[i][j], p.dtype);
+            else p.partial[((int64_t)split * p.M + m) * p.N + n] = acc[i][j];
+        }
+    }
+}
+
+}  // namespace adapt

@@ -1,0 +1,323 @@
+// tcgen05 GEMM kernel: the "Common" / "MultiCoreSplitK" templates (Section 4.2) on B200.
+//
+// One CTA (CG = 1) owns a 128 x BN output tile; a CTA pair (CG = 2) owns 256 x BN, each CTA
+// loading its own 128 rows of A and its own BN/2 columns of B (no multicast).  Pipeline
+// (Section 5.2, Eq. 9/13/14 restated for this machine):
+//
+//   producer warp : TMA, 128-byte swizzle, into an S-stage shared-memory ring   (the paper's MTE2)
+//   MMA warp      : one thread issues tcgen05.mma kind::f16, 128|256 x BN x 16,
+//                   fp32 accumulator in TMEM, two accumulator buffers           (Cube + L0C)
+//   4 epilogue warps: tcgen05.ld -> one RN-even cast -> global                  (FixPipe)
+//
+// The CTA is persistent: it walks its list of work units (tile x k-split) so the producer runs
+// ahead across tile boundaries (Preloading, Eq. 14) and the epilogue of unit u overlaps the main
+// loop of unit u+1.  With P_k > 1 a unit covers a fixed k-block range and writes an fp32 partial
+// tile to the workspace (Eq. 4); a separate kernel adds the partials in ascending split order.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+
+#include "ptx_sm100.cuh"
+
+namespace adapt {
+
+constexpr int kUmmaBK = 64;          // k-block: 64 elements = one 128-byte swizzle row
+constexpr int kUmmaThreads = 192;    // producer warp, MMA warp, four epilogue warps
+constexpr int kGroupM = 16;          // rasterisation: m-blocks per group
+
+struct UmmaParams {
+    int M, N, K;
+    int P_m, P_n, P_k;               // task counts (Table 1)
+    int kb_total, kb_per_split;      // k-blocks in K, k-blocks per split
+    int num_units;                   // P_m * P_n * P_k
+    int dtype;                       // ADAPT_F16 / ADAPT_BF16
+    int stages;
+    uint32_t idesc;                  // tcgen05 instruction descriptor
+    void* C;                         // 16-bit output, row-major M x N (used when P_k == 1)
+    float* partial;                  // fp32 [P_k][M][N] (used when P_k > 1)
+    int c_vec_ok;                    // C rows are 16-byte aligned (N % 8 == 0 and base aligned)
+    unsigned int* status;            // device status word: bit 0 = a bounded wait expired
+};
+
+// unit index -> (m block, n block, split).  Units of one output tile are adjacent in split;
+// tiles are visited in groups of kGroupM m-blocks so that concurrently running CTAs share B
+// columns and A rows in L2.
+__device__ __forceinline__ void decode_unit(const UmmaParams& p, int unit, int& mb, int& nb, int& split)
+{
+    split = unit % p.P_k;
+    const int t = unit / p.P_k;
+    const int group_size = kGroupM * p.P_n;
+    const int g = t / group_size;
+    const int first_m = g * kGroupM;
+    const int gm = min(p.P_m - first_m, kGroupM);
+    const int r = t - g * group_size;
+    mb = first_m + r % gm;
+    nb = r / gm;
+}
+
+__device__ __forceinline__ uint32_t pack16(float a, float b, int dtype)
+{
+    if (dtype == 0) {
+        __half2 h = __floats2half2_rn(a, b);
+        return *reinterpret_cast<uint32_t*>(&h);
+    }
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+__device__ __forceinline__ unsigned short cast16(float a, int dtype)
+{
+    if (dtype == 0) { __half h = __float2half_rn(a); return *reinterpret_cast<unsigned short*>(&h); }
+    __nv_bfloat16 h = __float2bfloat16_rn(a);
+    return *reinterpret_cast<unsigned short*>(&h);
+}
+
+template <int BN, bool A_MN, bool B_MN, int CG>
+__global__ void __launch_bounds__(kUmmaThreads, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const UmmaParams p)
+{
+    constexpr int BN_CTA = BN / CG;                       // B columns this CTA loads
+    constexpr int A_BYTES = 128 * kUmmaBK * 2;
+    constexpr int B_BYTES = BN_CTA * kUmmaBK * 2;
+    constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    constexpr int TMEM_COLS = 2 * BN;                     // two accumulator buffers
+    static_assert(TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "TMEM allocation is a power of two");
+    static_assert(BN_CTA % 64 == 0, "B is loaded in 64-column boxes");
+
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzle atoms are 1024-byte aligned
+    const int S = p.stages;
+    const uint32_t bar_base = smem_base + (uint32_t)S * STAGE_BYTES;
+    // barrier block: full[S], empty[S], tmem_full[2], tmem_empty[2], then the TMEM pointer and the abort flag
+    const uint32_t full_bar = bar_base;
+    const uint32_t empty_bar = bar_base + 8u * S;
+    const uint32_t tfull_bar = bar_base + 16u * S;
+    const uint32_t tempty_bar = tfull_bar + 16u;
+    const uint32_t tmem_slot = tempty_bar + 16u;
+    uint8_t* gen_base = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+    volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(gen_base + (size_t)S * STAGE_BYTES + 16 * S + 32);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + (size_t)S * STAGE_BYTES + 16 * S + 36);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t cta_rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;
+    const bool leader = cta_rank == 0;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+        for (int s = 0; s < S; ++s) {
+            ptx::mbar_init(full_bar + 8u * s, 1);          // one arrive.expect_tx per phase
+            ptx::mbar_init(empty_bar + 8u * s, 1);         // one tcgen05.commit per phase
+        }
+        for (int b = 0; b < 2; ++b) {
+            ptx::mbar_init(tfull_bar + 8u * b, 1);         // one tcgen05.commit per phase
+            ptx::mbar_init(tempty_bar + 8u * b, 4 * CG);   // one arrive per epilogue warp of every CTA of the group
+        }
+        ptx::fence_barrier_init();
+        ptx::fence_proxy_async_smem();
+        ptx::prefetch_tensormap(&tmA);
+        ptx::prefetch_tensormap(&tmB);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc<CG>(tmem_slot, TMEM_COLS);
+        ptx::tmem_relinquish<CG>();
+    }
+    ptx::tc_fence_before();
+    if (CG == 2) {
+        asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    } else {
+        __syncthreads();
+    }
+    ptx::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot_ptr;
+
+    const int unit0 = (CG == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int unit_step = (CG == 2) ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+
+    if (warp == 0) {
+        // ------------------------------ producer -----------------------------------------------
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            // the byte count of a stage is signalled on the leader's barrier (pair form)
+            uint32_t full_target = full_bar;
+            if (CG == 2) asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(full_target) : "r"(full_bar));
+            bool ok = true;
+            for (int unit = unit0; ok && unit < p.num_units; unit += unit_step) {
+                int mb, nb, split;
+                decode_unit(p, unit, mb, nb, split);
+                const int kb0 = split * p.kb_per_split;
+                const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+                const int row0 = mb * (128 * CG) + (int)cta_rank * 128;       // this CTA's A rows
+                const int col0 = nb * BN + (int)cta_rank * BN_CTA;            // this CTA's B columns
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    if (!ptx::mbar_wait(empty_bar + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
+                    const uint32_t sB = sA + A_BYTES;
+                    const uint32_t fb = full_target + 8u * stage;
+                    if (CG == 1) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, STAGE_BYTES);
+                    else if (leader) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, 2 * STAGE_BYTES);
+                    const int k0 = kb * kUmmaBK;
+                    if (!A_MN) {
+                        if (CG == 1) ptx::tma_load_2d(sA, &tmA, fb, k0, row0);
+                        else ptx::tma_load_2d_pair(sA, &tmA, fb, k0, row0);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 2; ++j) {
+                            if (CG == 1) ptx::tma_load_2d(sA + j * 8192, &tmA, fb, row0 + j * 64, k0);
+                            else ptx::tma_load_2d_pair(sA + j * 8192, &tmA, fb, row0 + j * 64, k0);
+                        }
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int j = 0; j < BN_CTA / 64; ++j) {
+                            if (CG == 1) ptx::tma_load_2d(sB + j * 8192, &tmB, fb, col0 + j * 64, k0);
+                            else ptx::tma_load_2d_pair(sB + j * 8192, &tmB, fb, col0 + j * 64, k0);
+                        }
+                    } else {
+                        if (CG == 1) ptx::tma_load_2d(sB, &tmB, fb, k0, col0);
+                        else ptx::tma_load_2d_pair(sB, &tmB, fb, k0, col0);
+                    }
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ---------------------------------------------
+        if (lane == 0 && leader) {
+            int stage = 0;
+            uint32_t phase = 0;
+            int buf = 0;
+            uint32_t buf_phase = 0;
+            // K-major operand: rows of 128 B, 8-row groups 1024 B apart, +32 B per 16-element k step.
+            // MN-major operand: 64-element blocks along M/N 8192 B apart (LBO), 8-row k groups
+            // 1024 B apart (SBO), +2048 B per 16-element k step.
+            const uint32_t a_lbo = A_MN ? 8192u : 16u, b_lbo = B_MN ? 8192u : 16u;
+            const uint32_t a_kstep = A_MN ? 2048u : 32u, b_kstep = B_MN ? 2048u : 32u;
+            bool ok = true;
+            for (int unit = unit0; ok && unit < p.num_units; unit += unit_step) {
+                int mb, nb, split;
+                decode_unit(p, unit, mb, nb, split);
+                const int kb0 = split * p.kb_per_split;
+                const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+                if (!ptx::mbar_wait(tempty_bar + 8u * buf, buf_phase ^ 1u, abort_flag)) { ok = false; break; }
+                ptx::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+                for (int kb = kb0; kb < kb1; ++kb) {
+                    if (!ptx::mbar_wait(full_bar + 8u * stage, phase, abort_flag)) { ok = false; break; }
+                    ptx::tc_fence_after();
+                    const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
+                    const uint32_t sB = sA + A_BYTES;
+#pragma unroll
+                    for (int k16 = 0; k16 < kUmmaBK / 16; ++k16) {
+                        const uint64_t adesc = ptx::smem_desc_sw128(sA + k16 * a_kstep, a_lbo, 1024u);
+                        const uint64_t bdesc = ptx::smem_desc_sw128(sB + k16 * b_kstep, b_lbo, 1024u);
+                        ptx::umma_f16<CG>(d_tmem, adesc, bdesc, p.idesc, (kb > kb0 || k16 > 0) ? 1u : 0u);
+                    }
+                    // free the stage (in both CTAs of a pair) once these MMAs have read it
+                    if (CG == 1) ptx::umma_commit_1(empty_bar + 8u * stage);
+                    else ptx::umma_commit_2(empty_bar + 8u * stage, 3);
+                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                if (CG == 1) ptx::umma_commit_1(tfull_bar + 8u * buf);
+                else ptx::umma_commit_2(tfull_bar + 8u * buf, 3);
+                buf ^= 1;
+                if (buf == 0) buf_phase ^= 1u;
+            }
+        }
+    } else {
+        // ------------------------------ epilogue -----------------------------------------------
+        const int q = warp & 3;                              // TMEM lane quarter this warp may read
+        int buf = 0;
+        uint32_t buf_phase = 0;
+        bool ok = true;
+        for (int unit = unit0; ok && unit < p.num_units; unit += unit_step) {
+            int mb, nb, split;
+            decode_unit(p, unit, mb, nb, split);
+            if (!ptx::mbar_wait(tfull_bar + 8u * buf, buf_phase, abort_flag)) { ok = false; break; }
+            ptx::tc_fence_after();
+            const int row = mb * (128 * CG) + (int)cta_rank * 128 + q * 32 + lane;
+            const int n0 = nb * BN;
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
+            const bool row_ok = row < p.M;
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                if (n0 + c0 >= p.N) break;                   // uniform across the warp
+                uint32_t r[32];
+                ptx::tmem_ld_32x32(t_row + (uint32_t)c0, r);
+                ptx::tmem_ld_wait();
+                if (!row_ok) continue;
+                const int col = n0 + c0;
+                if (p.P_k == 1) {
+                    unsigned short* crow = reinterpret_cast<unsigned short*>(p.C) + (size_t)row * p.N + col;
+                    if (p.c_vec_ok && col + 32 <= p.N) {
+#pragma unroll
+                        for (int v = 0; v < 4; ++v) {
+                            uint4 o;
+                            o.x = pack16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]), p.dtype);
+                            o.y = pack16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]), p.dtype);
+                            o.z = pack16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]), p.dtype);
+                            o.w = pack16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]), p.dtype);
+                            *reinterpret_cast<uint4*>(crow + 8 * v) = o;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col + j < p.N) crow[j] = cast16(__uint_as_float(r[j]), p.dtype);
+                    }
+                } else {
+                    float* prow = p.partial + ((size_t)split * p.M + row) * p.N + col;
+                    if ((p.N & 3) == 0 && col + 32 <= p.N) {
+#pragma unroll
+                        for (int v = 0; v < 8; ++v)
+                            *reinterpret_cast<uint4*>(prow + 4 * v) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (col + j < p.N) prow[j] = __uint_as_float(r[j]);
+                    }
+                }
+            }
+            // this warp has read its quarter of the accumulator: hand the buffer back to the MMA warp
+            ptx::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                if (CG == 1) ptx::mbar_arrive(tempty_bar + 8u * buf);
+                else ptx::mbar_arrive_cluster(tempty_bar + 8u * buf, 0);
+            }
+            buf ^= 1;
+            if (buf == 0) buf_phase ^= 1u;
+        }
+    }
+
+    // ------------------------------ common exit ----------------------------------------------
+    ptx::tc_fence_before();
+    if (CG == 2) {
+        asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+    } else {
+        __syncthreads();
+    }
+    if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, 1u);
+    if (warp == 1) {
+        ptx::tc_fence_after();
+        ptx::tmem_dealloc<CG>(tmem_base, TMEM_COLS);
+    }
+}
+
+// Instruction descriptor, kind::f16: [4,6) D format (1 = fp32), [7,10) A format, [10,13) B format
+// (0 = fp16, 1 = bf16), [15] A major, [16] B major (0 = K, 1 = MN), [17,23) N >> 3, [24,29) M >> 4.
+inline uint32_t umma_idesc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n)
+{
+    const uint32_t fmt = dtype == 0 ? 0u : 1u;
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+           ((uint32_t)(mma_n >> 3) << 17) | ((uint32_t)(mma_m >> 4) << 24);
+}
+
+inline int umma_smem_bytes(int BN, int cg, int stages)
+{
+    return stages * (128 * kUmmaBK * 2 + (BN / cg) * kUmmaBK * 2) + 1024 + 256;
+}
+
+}  // namespace adapt

@@ -1,0 +1,215 @@
+"""GPU parity tests: the CUDA path, called through the C ABI, against the CPU oracle."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_10803_b200 import binding as ab
+from paper_2608_10803_b200 import synth
+
+from gpu_util import TOL, check_case, compare_with_oracle, init, run_library, sample_rows
+
+pytestmark = pytest.mark.gpu
+
+ROW, COL = ab.ROW_MAJOR, ab.COL_MAJOR
+
+
+def draw(case):
+    return synth.draw_case(case, device="cuda")
+
+
+def every_variant(M, N, K, dtype, lA=ROW, lB=ROW, families=None, limit_per_family=40):
+    """(plan, info) of every legal configuration, optionally restricted to some families."""
+    out = []
+    count = {}
+    for c in ab.adapt_plan_candidates(M, N, K, dtype, lA, lB):
+        if families is not None and c.family not in families:
+            continue
+        count[c.family] = count.get(c.family, 0) + 1
+        if count[c.family] > limit_per_family:
+            continue
+        out.append((ab.adapt_matmul_plan_forced(M, N, K, dtype, lA, lB, c.tiling_key), c))
+    return out
+
+
+# ---- config 1: the 256^3 smoke case, full oracle, every variant ------------------------------------
+
+def test_config1_square_256_all_variants():
+    case = synth.config_square()[0]
+    A, B = draw(case)
+    for plan, c in every_variant(case.M, case.N, case.K, case.dtype):
+        check_case(case.M, case.N, case.K, case.dtype, A, B, plan=plan)
+    check_case(case.M, case.N, case.K, case.dtype, A, B)
+
+
+# ---- exact cases: small integers, position-coded, bit-identical to the oracle ---------------------
+
+EXACT_SHAPES = [
+    (256, 256, 256), (200, 264, 328), (131, 77, 259), (128, 128, 64), (129, 65, 65), (1, 8, 8), (5, 640, 1000),
+    (520, 3, 300), (16, 1024, 512), (1024, 16, 515), (300, 520, 8), (77, 50, 1), (384, 512, 2048), (64, 64, 8192),
+]
+
+
+@pytest.mark.parametrize("dtype", [ab.F16, ab.BF16])
+@pytest.mark.parametrize("shape", EXACT_SHAPES)
+def test_position_coded_integers_bit_exact_all_variants(shape, dtype):
+    M, N, K = shape
+    A = synth.position_coded(M, K, dtype, modulus=7, device="cuda")
+    B = synth.position_coded(K, N, dtype, modulus=5, device="cuda").contiguous()
+    for plan, c in every_variant(M, N, K, dtype, limit_per_family=12):
+        check_case(M, N, K, dtype, A, B, plan=plan, exact=True)
+    check_case(M, N, K, dtype, A, B, exact=True)
+
+
+@pytest.mark.parametrize("dtype", [ab.F16, ab.BF16])
+def test_random_integers_bit_exact(dtype):
+    M, N, K = 300, 200, 1500
+    A = synth.draw_operand(M, K, ("integer", -8, 8), 5, dtype, "cuda")
+    B = synth.draw_operand(K, N, ("integer", -8, 8), 6, dtype, "cuda")
+    for plan, c in every_variant(M, N, K, dtype, limit_per_family=6):
+        check_case(M, N, K, dtype, A, B, plan=plan, exact=True)
+
+
+# ---- layouts ------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("lA,lB", [(ROW, COL), (COL, ROW), (COL, COL)])
+@pytest.mark.parametrize("shape", [(256, 384, 512), (150, 90, 333), (8, 512, 640), (640, 8, 520)])
+def test_layouts_bit_exact(shape, lA, lB):
+    M, N, K = shape
+    dtype = ab.F16
+    A = synth.position_coded(M, K, dtype, 7, "cuda")
+    B = synth.position_coded(K, N, dtype, 5, "cuda")
+    A_st = A.t().contiguous() if lA == COL else A       # column-major storage of A is A^T row-major
+    B_st = B.t().contiguous() if lB == COL else B
+    for plan, c in every_variant(M, N, K, dtype, lA, lB, limit_per_family=4):
+        check_case(M, N, K, dtype, A_st, B_st, lA, lB, plan=plan, exact=True)
+
+
+# ---- edge tiles: one off the tile sizes, primes, ones --------------------------------------------------
+
+@pytest.mark.parametrize("shape", [(127, 255, 63), (129, 257, 65), (1, 1, 1), (2, 3, 5), (255, 129, 191),
+                                   (128, 256, 64), (17, 1031, 257), (1031, 17, 129), (97, 89, 83)])
+def test_edge_shapes_random_values(shape):
+    M, N, K = shape
+    for dtype in (ab.F16, ab.BF16):
+        A = synth.draw_operand(M, K, synth.U11, 101, dtype, "cuda")
+        B = synth.draw_operand(K, N, synth.U11, 102, dtype, "cuda")
+        for plan, c in every_variant(M, N, K, dtype, limit_per_family=6):
+            check_case(M, N, K, dtype, A, B, plan=plan)
+
+
+def test_degenerate_sizes():
+    init()
+    dtype = ab.F16
+    A = torch.ones((4, 0), dtype=torch.float16, device="cuda")
+    B = torch.ones((0, 6), dtype=torch.float16, device="cuda")
+    C = run_library(A, B, 4, 6, 0, dtype)                     # K = 0 -> zeros
+    torch.cuda.synchronize()
+    assert torch.count_nonzero(C).item() == 0 and not torch.isnan(C).any()
+    run_library(torch.empty((0, 8), dtype=torch.float16, device="cuda"),
+                torch.ones((8, 6), dtype=torch.float16, device="cuda"), 0, 6, 8, dtype)      # M = 0 -> no-op
+    run_library(torch.ones((4, 8), dtype=torch.float16, device="cuda"),
+                torch.empty((8, 0), dtype=torch.float16, device="cuda"), 4, 0, 8, dtype)      # N = 0 -> no-op
+    torch.cuda.synchronize()
+
+
+def test_argument_errors():
+    init()
+    h = ab.adapt_matmul_plan(64, 64, 64, ab.F16)
+    A = torch.ones((64, 64), dtype=torch.float16, device="cuda")
+    C = torch.empty((64, 64), dtype=torch.float16, device="cuda")
+    with pytest.raises(ab.AdaptError) as e:
+        ab.adapt_matmul(h, A.data_ptr(), A.data_ptr(), A.data_ptr(), 0)       # C aliases A
+    assert e.value.status == ab.ERR_INVALID_ARG
+    with pytest.raises(ab.AdaptError) as e:
+        ab.adapt_matmul(h, 0, A.data_ptr(), C.data_ptr(), 0)
+    assert e.value.status == ab.ERR_INVALID_ARG
+    with pytest.raises(ab.AdaptError) as e:
+        ab.adapt_matmul(h, A.data_ptr() + 1, A.data_ptr(), C.data_ptr(), 0)   # odd address
+    assert e.value.status == ab.ERR_INVALID_ARG
+
+
+def test_misaligned_pointers_take_the_repitch_path():
+    """Buffers that start 2 bytes off a 16-byte boundary still give the exact result."""
+    M, N, K = 256, 256, 512
+    dtype = ab.BF16
+    A = synth.position_coded(M, K, dtype, 7, "cuda")
+    B = synth.position_coded(K, N, dtype, 5, "cuda")
+    bufA = torch.zeros(M * K + 8, dtype=torch.bfloat16, device="cuda")
+    bufB = torch.zeros(K * N + 8, dtype=torch.bfloat16, device="cuda")
+    bufC = torch.zeros(M * N + 8, dtype=torch.bfloat16, device="cuda")
+    A1 = bufA[1:1 + M * K].view(M, K)
+    B1 = bufB[3:3 + K * N].view(K, N)
+    C1 = bufC[5:5 + M * N].view(M, N)
+    A1.copy_(A)
+    B1.copy_(B)
+    for plan, c in every_variant(M, N, K, dtype, limit_per_family=3):
+        C1.fill_(float("nan"))
+        run_library(A1, B1, M, N, K, dtype, plan=plan, out=C1)
+        torch.cuda.synchronize()
+        err, mism, n = compare_with_oracle(A1, B1, C1, M, N, K, dtype)
+        assert mism == 0, (ab.FAMILY_NAMES[c.family], c.BN, c.P_k, mism)
+    assert bufC[:5].abs().sum().item() == 0 and bufC[5 + M * N:].abs().sum().item() == 0   # no stray writes
+
+
+def test_run_twice_is_bit_identical():
+    for (M, N, K, dtype) in [(256, 256, 262144 // 8, ab.BF16), (7, 1024, 1024, ab.F16), (1000, 1024, 1024, ab.F16)]:
+        A = synth.draw_operand(M, K, synth.U11, 1, dtype, "cuda")
+        B = synth.draw_operand(K, N, synth.U11, 2, dtype, "cuda")
+        for plan, c in every_variant(M, N, K, dtype, limit_per_family=3):
+            C1 = run_library(A, B, M, N, K, dtype, plan=plan).clone()
+            C2 = run_library(A, B, M, N, K, dtype, plan=plan)
+            torch.cuda.synchronize()
+            assert torch.equal(C1.view(torch.int16), C2.view(torch.int16))
+
+
+# ---- the named workloads at full size, in the configuration bench.py times (model-selected plan) ----
+
+@pytest.mark.parametrize("case", synth.config_reco(), ids=lambda c: c.name)
+def test_config2_recommendation_shapes(case):
+    A, B = draw(case)
+    check_case(case.M, case.N, case.K, case.dtype, A, B, mac_budget=3e9)
+
+
+@pytest.mark.parametrize("case", synth.config_llm(), ids=lambda c: c.name)
+def test_config3_llm_layer_shapes(case):
+    A, B = draw(case)
+    check_case(case.M, case.N, case.K, case.dtype, A, B, mac_budget=1.5e10)
+
+
+@pytest.mark.parametrize("case", synth.config_large(), ids=lambda c: c.name)
+def test_config4_large_and_tall_k(case):
+    A, B = draw(case)
+    check_case(case.M, case.N, case.K, case.dtype, A, B, mac_budget=1.8e10)
+
+
+@pytest.mark.parametrize("case", synth.config_context(), ids=lambda c: c.name)
+def test_paper_named_shapes(case):
+    A, B = draw(case)
+    check_case(case.M, case.N, case.K, case.dtype, A, B, mac_budget=6e9)
+
+
+def test_sweep_oracle_subset():
+    """The seeded 200-shape subset of the 2,000-shape dynamic sweep; complete sampled rows on the
+    larger shapes so the CPU side stays within a minute or two."""
+    cases = synth.config_sweep()
+    worst = {ab.F16: 0.0, ab.BF16: 0.0}
+    for idx in synth.sweep_oracle_subset():
+        case = cases[idx]
+        A, B = draw(case)
+        err, _, _, _ = check_case(case.M, case.N, case.K, case.dtype, A, B, mac_budget=4e8, seed=idx)
+        worst[case.dtype] = max(worst[case.dtype], err)
+        del A, B
+    assert worst[ab.F16] <= TOL[ab.F16] and worst[ab.BF16] <= TOL[ab.BF16]
+
+
+def test_long_k_accumulation_error_stays_small():
+    """fp32 accumulation over a very long chain (no split): error must stay far below tolerance."""
+    M, N, K = 128, 128, 131072
+    dtype = ab.BF16
+    A = synth.draw_operand(M, K, synth.U11, 7, dtype, "cuda")
+    B = synth.draw_operand(K, N, synth.U11, 8, dtype, "cuda")
+    for plan, c in every_variant(M, N, K, dtype, families=[ab.FAM_UMMA_1CTA]):
+        if c.P_k != 1 or c.BN != 128:
+            continue
+        err, _, _, _ = check_case(M, N, K, dtype, A, B, plan=plan)
+        assert err < 4e-3

@@ -1,0 +1,201 @@
+"""Host-side logic of the C-ABI library, no GPU: exports, taxonomy, model closed forms,
+candidate legality, plan cache.  The library's classifier and formulas are compared with the
+oracle's (``oracle/taxonomy.py``), which is pinned to the paper separately."""
+import ctypes
+import os
+import re
+import time
+
+import pytest
+
+from oracle import taxonomy as tx
+from paper_2608_10803_b200 import binding as ab
+from paper_2608_10803_b200 import build as adapt_build
+from paper_2608_10803_b200 import synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+CLASS_ID = {tx.COMMON: 0, tx.SINGLE_CORE_SPLIT_K: 1, tx.MULTI_CORE_SPLIT_K: 2, tx.HYBRID_SPLIT_K: 3}
+
+
+@pytest.fixture(scope="module", autouse=True)
+def lib():
+    adapt_build.build()
+    return ab.load()
+
+
+def test_library_exports_every_declared_symbol(lib):
+    header = open(os.path.join(ROOT, "include", "adapt_matmul.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(adapt_[a-z_0-9]+)\s*\(", header))
+    assert declared, "no declarations found"
+    assert declared == set(ab.EXPORTS)
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_compute_without_device_fails_loudly(lib):
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("device present")
+    h = ab.adapt_matmul_plan(64, 64, 64, ab.F16)
+    with pytest.raises(ab.AdaptError) as e:
+        ab.adapt_matmul(h, 16, 16, 16, 0)
+    assert e.value.status == ab.ERR_NOT_INIT
+
+
+def worked_cases():
+    out = []
+    with open(os.path.join(ROOT, "tests", "golden", "taxonomy_cases.txt")) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            p = line.split()
+            out.append(tuple(int(x) for x in p[:12]) + (p[12],))
+    return out
+
+
+@pytest.mark.parametrize("case", worked_cases())
+def test_classifier_reproduces_worked_cases(case):
+    _, M, N, K, m, n, m1, n1, N_core, S, _, _, template = case
+    assert ab.adapt_classify(M, N, m, n, m1, n1, N_core, S) == CLASS_ID[template]
+
+
+def test_classifier_matches_oracle_on_a_grid():
+    for M in (1, 100, 1000, 5000, 100000):
+        for N in (1, 64, 777, 4096):
+            for (m, n) in ((128, 64), (128, 256), (256, 256)):
+                for (nc, acc) in ((16, 128 << 10), (148, 128 << 10), (74, 256 << 10)):
+                    want = CLASS_ID[tx.classify(M, N, m, n, m, n, nc, acc)]
+                    assert ab.adapt_classify(M, N, m, n, m, n, nc, acc) == want
+    assert ab.adapt_classify(0, 1, 1, 1, 1, 1, 1, 1) == -1
+
+
+def test_volume_formulas_match_oracle():
+    M, N, K = 12288, 688, 16991
+    for (m1, n1) in ((128, 256), (256, 256), (128, 64)):
+        assert ab.adapt_model_read_volume(M, N, K, m1, n1) == pytest.approx(float(tx.read_volume(M, N, K, m1, n1)), rel=1e-14)
+    assert ab.adapt_model_write_volume(0, M, N, K, K, 64) == tx.write_volume_common(M, N)
+    assert ab.adapt_model_write_volume(1, M, N, K, K, 512) == tx.write_volume_single_core_split_k(M, N, K, 512)
+    assert ab.adapt_model_write_volume(2, M, N, K, 1024, 64) == tx.write_volume_multi_core_split_k(M, N, K, 1024)
+    assert ab.adapt_model_write_volume(3, M, N, K, 1000, 300) == tx.write_volume_hybrid_split_k(M, N, K, 1000, 300)
+
+
+def test_pipeline_formulas_match_oracle():
+    for (Q, L, tM, tP, D) in ((1, 1, 3.0, 5.0, 1.0), (4, 9, 2.5, 1.5, 0.25), (7, 64, 1.0, 1.0, 3.0)):
+        assert ab.adapt_model_pipeline(0, Q, L, tM, tP, D) == pytest.approx(Q * tx.t_baseline(L, tM, tP, D))
+        assert ab.adapt_model_pipeline(1, Q, L, tM, tP, D) == pytest.approx(Q * tx.t_double_buffer(L, tM, tP, D))
+        assert ab.adapt_model_pipeline(2, Q, L, tM, tP, D) == pytest.approx(tx.t_preload(Q, L, tM, tP, D))
+
+
+def test_plan_is_cached_and_pointer_equal():
+    a = ab.adapt_matmul_plan(1000, 1024, 1024, ab.F16)
+    b = ab.adapt_matmul_plan(1000, 1024, 1024, ab.F16)
+    c = ab.adapt_matmul_plan(1000, 1024, 1024, ab.BF16)
+    d = ab.adapt_matmul_plan(1000, 1024, 1024, ab.F16, ab.COL_MAJOR, ab.ROW_MAJOR)
+    assert a == b and a != c and a != d
+    big = ab.adapt_matmul_plan(2_000_000, 8, 8, ab.F16)          # beyond the packed-key range
+    assert big == ab.adapt_matmul_plan(2_000_000, 8, 8, ab.F16)
+
+
+def test_plan_rejects_bad_arguments():
+    with pytest.raises(ab.AdaptError) as e:
+        ab.adapt_matmul_plan(-1, 4, 4, ab.F16)
+    assert e.value.status == ab.ERR_INVALID_ARG
+    with pytest.raises(ab.AdaptError) as e:
+        ab.adapt_matmul_plan(1 << 31, 4, 4, ab.F16)
+    assert e.value.status == ab.ERR_UNSUPPORTED
+    with pytest.raises(ab.AdaptError):
+        ab.adapt_matmul_plan(4, 4, 4, 7)
+
+
+def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
+    shapes = [(1, 1, 1), (1, 4096, 4096), (7, 1024, 1024), (8192, 8192, 8192), (256, 256, 262144),
+              (178, 71, 43035), (3067, 2, 75528), (6392, 8517, 4), (100000, 1024, 1024), (3, 256, 87087),
+              (12288, 688, 16991), (17, 17, 17), (99999, 3, 5)]
+    for (M, N, K) in shapes:
+        for dt in (ab.F16, ab.BF16):
+            cands = ab.adapt_plan_candidates(M, N, K, dt)
+            assert cands, (M, N, K)
+            assert all(cands[i].predicted_us <= cands[i + 1].predicted_us for i in range(len(cands) - 1))
+            info = ab.adapt_plan_info(ab.adapt_matmul_plan(M, N, K, dt))
+            assert (info.M, info.N, info.K, info.dtype) == (M, N, K, dt)
+            assert info.flops == 2.0 * M * N * K
+            assert info.P_k >= 1 and info.grid >= 1 and info.predicted_us > 0
+            for c in cands:
+                # capacity limits of Eq. 6
+                if c.family in (ab.FAM_UMMA_1CTA, ab.FAM_UMMA_2CTA):
+                    bn_cta = c.BN // c.cluster
+                    smem = c.stages * (128 * 64 * 2 + bn_cta * 64 * 2)
+                    assert smem <= 227 * 1024
+                    assert 2 * c.BN <= 512 and c.BN % 16 == 0
+                    assert c.P_k <= -(-K // 64)
+                    # unaligned operands are never handed to TMA directly (row-major: K for A, N for B)
+                    if K % 8:
+                        assert c.srcA == 1
+                    if N % 8:
+                        assert c.srcB == 1
+                if c.family == ab.FAM_SKINNY:
+                    assert min(M, N) <= 16
+                # taxonomy label follows the predicate (Section 4.2)
+                enough = c.P_m * c.P_n >= 148
+                assert (c.taxonomy_class in (0, 1)) == enough
+
+
+def test_forced_plan_round_trips_its_key():
+    M, N, K = 512, 768, 4096
+    cands = ab.adapt_plan_candidates(M, N, K, ab.BF16)
+    seen = set()
+    for c in cands:
+        assert c.tiling_key not in seen, "keys must identify configurations"
+        seen.add(c.tiling_key)
+        h = ab.adapt_matmul_plan_forced(M, N, K, ab.BF16, ab.ROW_MAJOR, ab.ROW_MAJOR, c.tiling_key)
+        info = ab.adapt_plan_info(h)
+        assert info.tiling_key == c.tiling_key
+        assert (info.family, info.BM, info.BN, info.stages, info.P_k) == (c.family, c.BM, c.BN, c.stages, c.P_k)
+    with pytest.raises(ab.AdaptError) as e:
+        ab.adapt_matmul_plan_forced(M, N, K, ab.BF16, ab.ROW_MAJOR, ab.ROW_MAJOR, 0x1234)
+    assert e.value.status == ab.ERR_UNSUPPORTED
+
+
+def test_split_k_is_chosen_for_small_mn_large_k_and_not_for_large_mn():
+    small = ab.adapt_plan_info(ab.adapt_matmul_plan(256, 256, 262144, ab.BF16))
+    assert small.P_k > 1 and small.taxonomy_class in (2, 3)
+    large = ab.adapt_plan_info(ab.adapt_matmul_plan(8192, 8192, 8192, ab.BF16))
+    assert large.P_k == 1 and large.taxonomy_class in (0, 1)
+    assert large.family in (ab.FAM_UMMA_1CTA, ab.FAM_UMMA_2CTA)
+
+
+def test_plan_is_deterministic_across_processes():
+    import subprocess
+    import sys
+    code = ("from paper_2608_10803_b200 import binding as ab;"
+            "print([ab.adapt_plan_info(ab.adapt_matmul_plan(*s, 0)).tiling_key for s in "
+            "[(7409,156,19633),(1657,12995,164),(64,1024,1024)]])")
+    outs = {subprocess.run([sys.executable, "-c", code], cwd=ROOT, capture_output=True, text=True, check=True).stdout
+            for _ in range(2)}
+    assert len(outs) == 1
+
+
+def test_cached_plan_lookup_is_fast():
+    """Dispatch target: a cached plan costs well under 2 microseconds (measured through ctypes,
+    whose own call overhead dominates; the C-level figure is reported by bench.py)."""
+    lib = ab.load()
+    shapes = synth.sweep_shapes()[:256]
+    for (M, N, K) in shapes:
+        ab.adapt_matmul_plan(M, N, K, ab.F16)
+    f = lib.adapt_matmul_plan
+    t0 = time.perf_counter()
+    reps = 20
+    for _ in range(reps):
+        for (M, N, K) in shapes:
+            f(M, N, K, 0, 0, 0)
+    per_call = (time.perf_counter() - t0) / (reps * len(shapes))
+    assert per_call < 5e-6, per_call
+
+
+def test_sweep_csv_matches_recipe():
+    shapes, draws = synth.draw_sweep_shapes()
+    assert draws == 2107
+    assert shapes == synth.sweep_shapes()
+    assert shapes[:5] == [(7409, 156, 19633), (3067, 2, 75528), (6392, 8517, 4), (178, 71, 43035), (1657, 12995, 164)]
+    assert len(synth.sweep_oracle_subset()) == 200
