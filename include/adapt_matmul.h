@@ -131,6 +131,17 @@ adapt_handle_t adapt_matmul_plan(int64_t M, int64_t N, int64_t K,
  * get different workspaces. */
 adapt_status_t adapt_matmul(adapt_handle_t plan, const void* A, const void* B, void* C, void* cuda_stream);
 
+/* The same call for operands that live in HOST memory (A_host, B_host inputs, C_host output,
+ * dense, in the plan's layouts; pinned memory makes the copies asynchronous).  Enqueues on the
+ * stream: copy A and B into a library-owned device staging buffer, the planned kernels, copy C
+ * back.  Returns without synchronising: the caller synchronises the stream before reading
+ * C_host or reusing A_host / B_host.  The staging buffer is per stream and grows on demand
+ * (cudaMalloc), like the workspace.  The paper has no counterpart (its operator takes device
+ * tensors); this entry exists so that end-to-end cost including the PCIe copies can be measured
+ * through one call. */
+adapt_status_t adapt_matmul_host(adapt_handle_t plan, const void* A_host, const void* B_host, void* C_host,
+                                 void* cuda_stream);
+
 /* Thread-local status of the last failing call on this thread, and its text. */
 adapt_status_t adapt_last_error(void);
 const char* adapt_last_error_message(void);

@@ -20,7 +20,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libadaptmm.so")
 
 EXPORTS = [
-    "adapt_init", "adapt_shutdown", "adapt_matmul_plan", "adapt_matmul", "adapt_last_error",
+    "adapt_init", "adapt_shutdown", "adapt_matmul_plan", "adapt_matmul", "adapt_matmul_host", "adapt_last_error",
     "adapt_last_error_message", "adapt_status_string", "adapt_plan_info", "adapt_plan_candidates",
     "adapt_matmul_plan_forced", "adapt_classify", "adapt_model_read_volume", "adapt_model_write_volume",
     "adapt_model_pipeline", "adapt_poll_device_status", "adapt_plan_cache_size", "adapt_launch_count",
@@ -79,6 +79,8 @@ def load():
     lib.adapt_matmul_plan_forced.argtypes = [i64, i64, i64, i32, i32, i32, u64]
     lib.adapt_matmul.restype = i32
     lib.adapt_matmul.argtypes = [vp, vp, vp, vp, vp]
+    lib.adapt_matmul_host.restype = i32
+    lib.adapt_matmul_host.argtypes = [vp, vp, vp, vp, vp]
     lib.adapt_last_error.restype = i32
     lib.adapt_last_error_message.restype = ctypes.c_char_p
     lib.adapt_status_string.restype = ctypes.c_char_p
@@ -135,6 +137,11 @@ def adapt_matmul_plan_forced(M, N, K, dtype, layoutA, layoutB, tiling_key):
 def adapt_matmul(plan, A_ptr: int, B_ptr: int, C_ptr: int, stream: int = 0):
     """Enqueue C = A*B.  Pointers are raw device addresses (``tensor.data_ptr()``)."""
     _check(load().adapt_matmul(plan, A_ptr, B_ptr, C_ptr, stream))
+
+
+def adapt_matmul_host(plan, A_host_ptr: int, B_host_ptr: int, C_host_ptr: int, stream: int = 0):
+    """Enqueue H2D(A, B), the GEMM and D2H(C) for host buffers (raw host addresses)."""
+    _check(load().adapt_matmul_host(plan, A_host_ptr, B_host_ptr, C_host_ptr, stream))
 
 
 def adapt_plan_info(plan) -> PlanInfo:

@@ -110,6 +110,7 @@ struct State {
     unsigned int* d_status = nullptr;
     struct Workspace { void* ptr = nullptr; size_t bytes = 0; };
     std::unordered_map<cudaStream_t, Workspace> ws;
+    std::unordered_map<cudaStream_t, Workspace> staging;   // device copies of host operands (adapt_matmul_host)
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
     std::atomic<int64_t> launches{0};
     int log = 0;
@@ -416,6 +417,8 @@ extern "C" void adapt_shutdown(void)
         cudaDeviceSynchronize();
         for (auto& kv : S.ws) if (kv.second.ptr) cudaFree(kv.second.ptr);
         S.ws.clear();
+        for (auto& kv : S.staging) if (kv.second.ptr) cudaFree(kv.second.ptr);
+        S.staging.clear();
         if (S.d_status) cudaFree(S.d_status);
         S.d_status = nullptr;
     }
@@ -451,12 +454,12 @@ extern "C" adapt_status_t adapt_poll_device_status(void* cuda_stream)
 // ---------------------------------------------------------------------------------------------
 namespace {
 
-adapt_status_t get_workspace(State& S, cudaStream_t stream, size_t bytes, void** out)
+adapt_status_t get_workspace(State& S, cudaStream_t stream, size_t bytes, void** out, bool staging = false)
 {
     *out = nullptr;
     if (bytes == 0) return ADAPT_OK;
     std::lock_guard<std::mutex> lock(S.mu);
-    State::Workspace& w = S.ws[stream];
+    State::Workspace& w = staging ? S.staging[stream] : S.ws[stream];
     if (w.bytes < bytes) {
         if (w.ptr) {
             CUDA_TRY(cudaStreamSynchronize(stream));
@@ -684,4 +687,30 @@ extern "C" adapt_status_t adapt_matmul(adapt_handle_t plan, const void* A, const
         case ADAPT_FAM_SIMT: return run_simt(S, pl, A, B, C, stream);
     }
     return fail(ADAPT_ERR_UNSUPPORTED, "unknown kernel family%s");
+}
+
+extern "C" adapt_status_t adapt_matmul_host(adapt_handle_t plan, const void* A_host, const void* B_host, void* C_host,
+                                            void* cuda_stream)
+{
+    State& S = st();
+    if (!plan) return fail(ADAPT_ERR_INVALID_ARG, "null plan%s");
+    if (!S.inited) return fail(ADAPT_ERR_NOT_INIT, "adapt_init has not been called%s");
+    const Shape& s = plan->s;
+    if (plan->noop) return ADAPT_OK;
+    if (!C_host || ((!A_host || !B_host) && !plan->zero_fill)) return fail(ADAPT_ERR_INVALID_ARG, "null operand%s");
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const size_t nA = (size_t)round_up(s.M * s.K * 2, 256), nB = (size_t)round_up(s.K * s.N * 2, 256);
+    const size_t nC = (size_t)round_up(s.M * s.N * 2, 256);
+    void* dev = nullptr;
+    adapt_status_t r = get_workspace(S, stream, nA + nB + nC, &dev, true);
+    if (r != ADAPT_OK) return r;
+    uint8_t* d8 = (uint8_t*)dev;
+    if (s.K > 0) {
+        CUDA_TRY(cudaMemcpyAsync(d8, A_host, (size_t)s.M * s.K * 2, cudaMemcpyHostToDevice, stream));
+        CUDA_TRY(cudaMemcpyAsync(d8 + nA, B_host, (size_t)s.K * s.N * 2, cudaMemcpyHostToDevice, stream));
+    }
+    r = adapt_matmul(plan, d8, d8 + nA, d8 + nA + nB, cuda_stream);
+    if (r != ADAPT_OK) return r;
+    CUDA_TRY(cudaMemcpyAsync(C_host, d8 + nA + nB, (size_t)s.M * s.N * 2, cudaMemcpyDeviceToHost, stream));
+    return ADAPT_OK;
 }
