@@ -528,11 +528,12 @@ adapt_status_t launch_pad(State& S, const void* src, void* dst, int64_t outer, i
     return ADAPT_OK;
 }
 
-adapt_status_t launch_reduce(State& S, const float* partial, void* C, int64_t MN, int P_k, int dtype, cudaStream_t stream)
+adapt_status_t launch_reduce(State& S, const float* partial, void* C, int64_t M, int64_t N, int P_k, int dtype, cudaStream_t stream)
 {
-    const int64_t work = (MN + 3) / 4;
+    const int64_t Np = round_up(N, 4);
+    const int64_t work = M * (Np / 4);
     const int blocks = (int)std::min<int64_t>(ceil_div(work, 256), (int64_t)S.machine.n_sm * 8);
-    splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(partial, (unsigned short*)C, MN, P_k, dtype);
+    splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(partial, (unsigned short*)C, (int)M, (int)N, (int)Np, P_k, dtype);
     S.launches.fetch_add(1, std::memory_order_relaxed);
     CUDA_TRY(cudaGetLastError());
     return ADAPT_OK;
@@ -552,7 +553,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     const int64_t pitchB = padB ? padded_pitch(inB) : inB;
     const size_t szA = padA ? (size_t)round_up(outA * pitchA * 2, 256) : 0;
     const size_t szB = padB ? (size_t)round_up(outB * pitchB * 2, 256) : 0;
-    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * s.N * 4, 256) : 0;
+    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * round_up(s.N, 4) * 4, 256) : 0;
     void* ws = nullptr;
     adapt_status_t r = get_workspace(S, stream, szA + szB + szP, &ws);
     if (r != ADAPT_OK) return r;
@@ -586,7 +587,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.idesc = umma_idesc(s.dtype, a_mn, b_mn, 128 * cg, c.BN);
     p.C = C;
     p.partial = partial;
-    p.c_vec_ok = (s.N % 8 == 0 && ((uintptr_t)C & 15) == 0) ? 1 : 0;
+    p.Np = (int)round_up(s.N, 4);
     p.status = S.d_status;
 
     UmmaKernel k = launch_map_umma(c.family, c.BN, a_mn, b_mn);
@@ -608,7 +609,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     cfg.numAttrs = 1;
     CUDA_TRY(cudaLaunchKernelEx(&cfg, k, tmA, tmB, p));
     S.launches.fetch_add(1, std::memory_order_relaxed);
-    if (c.P_k > 1) return launch_reduce(S, partial, C, s.M * s.N, c.P_k, s.dtype, stream);
+    if (c.P_k > 1) return launch_reduce(S, partial, C, s.M, s.N, c.P_k, s.dtype, stream);
     return ADAPT_OK;
 }
 
@@ -616,7 +617,7 @@ adapt_status_t run_simt(State& S, Plan* pl, const void* A, const void* B, void* 
 {
     const Shape& s = pl->s;
     const Config& c = pl->c;
-    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * s.N * 4, 256) : 0;
+    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * round_up(s.N, 4) * 4, 256) : 0;
     void* ws = nullptr;
     adapt_status_t r = get_workspace(S, stream, szP, &ws);
     if (r != ADAPT_OK) return r;
@@ -626,6 +627,7 @@ adapt_status_t run_simt(State& S, Plan* pl, const void* A, const void* B, void* 
     if (s.layoutB == ADAPT_ROW_MAJOR) { p.b_sk = s.N; p.b_sn = 1; } else { p.b_sk = 1; p.b_sn = s.K; }
     p.P_n = c.P_n;
     p.P_k = c.P_k;
+    p.Np = (int)round_up(s.N, 4);
     p.kb_per_split = (int)ceil_div(ceil_div(s.K, 16), c.P_k);
     p.dtype = s.dtype;
     p.C = (unsigned short*)C;
@@ -634,7 +636,7 @@ adapt_status_t run_simt(State& S, Plan* pl, const void* A, const void* B, void* 
     simt_gemm_kernel<<<grid, 256, 0, stream>>>((const unsigned short*)A, (const unsigned short*)B, p);
     S.launches.fetch_add(1, std::memory_order_relaxed);
     CUDA_TRY(cudaGetLastError());
-    if (c.P_k > 1) return launch_reduce(S, (const float*)ws, C, s.M * s.N, c.P_k, s.dtype, stream);
+    if (c.P_k > 1) return launch_reduce(S, (const float*)ws, C, s.M, s.N, c.P_k, s.dtype, stream);
     return ADAPT_OK;
 }
 
@@ -642,7 +644,7 @@ adapt_status_t run_skinny(State& S, Plan* pl, const void* A, const void* B, void
 {
     const Shape& s = pl->s;
     const Config& c = pl->c;
-    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * s.N * 4, 256) : 0;
+    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * round_up(s.N, 4) * 4, 256) : 0;
     void* ws = nullptr;
     adapt_status_t r = get_workspace(S, stream, szP, &ws);
     if (r != ADAPT_OK) return r;
@@ -650,7 +652,7 @@ adapt_status_t run_skinny(State& S, Plan* pl, const void* A, const void* B, void
     if (r != ADAPT_OK) return fail(r, "skinny kernel launch failed%s");
     S.launches.fetch_add(1, std::memory_order_relaxed);
     CUDA_TRY(cudaGetLastError());
-    if (c.P_k > 1) return launch_reduce(S, (const float*)ws, C, s.M * s.N, c.P_k, s.dtype, stream);
+    if (c.P_k > 1) return launch_reduce(S, (const float*)ws, C, s.M, s.N, c.P_k, s.dtype, stream);
     return ADAPT_OK;
 }
 

@@ -150,7 +150,7 @@ static void model_epilogue(const Shape& s, Config& c, const Calib& cal)
     c.ws_partial = 0;
     if (c.P_k > 1) {
         const double MN = (double)s.M * (double)s.N;
-        c.ws_partial = round_up((int64_t)c.P_k * s.M * s.N * 4, 256);
+        c.ws_partial = round_up((int64_t)c.P_k * s.M * round_up(s.N, 4) * 4, 256);
         double part = 4.0 * MN * c.P_k;
         // partials that fit in L2 are read back at L2 speed; model that as half the HBM cost
         const double factor = part <= kL2Bytes ? 0.5 : 1.0;
@@ -245,13 +245,6 @@ static void model_simt(const Shape& s, const Machine& m, const Calib& cal, Confi
 
 // ---- legality (the constraint M(b,x,s) <= C_limit of Eq. 6) -----------------------------------
 
-static int umma_smem_bytes(const Config& c)
-{
-    const int bn_per_cta = c.BN / c.cluster;
-    const int stage = 2 * c.BK * (128 + bn_per_cta);
-    return c.stages * stage + 1024 /*alignment slack*/ + 256 /*barriers, tmem pointer*/;
-}
-
 static bool aligned16(int64_t inner_elems) { return inner_elems % 8 == 0; }
 
 static bool legal_umma(const Shape& s, const Machine& m, Config& c)
@@ -268,7 +261,7 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     if (c.BN % 16 != 0 || c.BN > 256) return false;                 // UMMA shape rule for M = 128/256
     if (2 * c.BN > m.tmem_cols) return false;                       // two accumulator buffers in TMEM
     if (c.stages < 1 || c.stages > 12) return false;
-    c.smem_bytes = umma_smem_bytes(c);
+    c.smem_bytes = umma_smem_bytes(c.BN, c.cluster, c.stages);
     if (c.smem_bytes > m.smem_bytes) return false;
     const int64_t kblocks = ceil_div(s.K, c.BK);
     if (c.P_k < 1 || c.P_k > 1023 || c.P_k > kblocks) return false;
@@ -294,7 +287,7 @@ static bool legal_skinny(const Shape& s, const Machine& m, Config& c)
     if (c.BN != 128 && c.BN != 256 && c.BN != 512) return false;     // streamed rows/columns per CTA
     if (c.srcA != ADAPT_SRC_LSU || c.srcB != ADAPT_SRC_LSU) return false;
     if (c.stages != 1) return false;
-    const int64_t ksteps = ceil_div(s.K, 256);                       // splits are whole staging chunks
+    const int64_t ksteps = ceil_div(s.K, kSkinnyKChunk);             // splits are whole staging chunks
     if (c.P_k < 1 || c.P_k > 1023 || c.P_k > ksteps) return false;
     if (ceil_div(ksteps, ceil_div(ksteps, c.P_k)) != c.P_k) return false;
     c.P_m = 1;
@@ -393,7 +386,7 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
             int deepest = 0;
             for (int st = 12; st >= 2; --st) {
                 probe.stages = st;
-                if (umma_smem_bytes(probe) <= m.smem_bytes) { deepest = st; break; }
+                if (umma_smem_bytes(probe.BN, probe.cluster, st) <= m.smem_bytes) { deepest = st; break; }
             }
             if (deepest > 8) deepest = 8;
             std::vector<int> depths = {deepest};
@@ -413,7 +406,7 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
     if (std::min(s.M, s.N) <= 16) {
         for (int BN : {128, 256, 512}) {
             const int64_t tiles = ceil_div(std::max(s.M, s.N), BN);
-            split_candidates(tiles, (int64_t)m.n_sm * 2, ceil_div(s.K, 256), 1, &pks);
+            split_candidates(tiles, (int64_t)m.n_sm * 2, ceil_div(s.K, kSkinnyKChunk), 1, &pks);
             for (int pk : pks) {
                 Config c;
                 c.family = ADAPT_FAM_SKINNY; c.BM = 16; c.BN = BN; c.BK = 16; c.stages = 1; c.P_k = pk;

@@ -72,30 +72,37 @@ pad_copy_kernel(const unsigned short* __restrict__ src, unsigned short* __restri
 }
 
 // ---- split-K reduction: C = RN16( sum_{p = 0..P_k-1} partial[p] ), ascending p, fp32 ---------------
-// The order is fixed, so the result does not depend on which CTA finished first.
+// The order is fixed, so the result does not depend on which CTA finished first.  Partials are
+// stored [P_k][M][Np] with Np = N rounded up to 4, so every row starts on a 16-byte boundary and
+// one thread reduces four consecutive columns with 16-byte loads.
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float* __restrict__ partial, unsigned short* __restrict__ C,
-                     int64_t MN, int P_k, int dtype)
+                     int M, int N, int Np, int P_k, int dtype)
 {
+    const int groups = Np >> 2;
+    const int64_t total = (int64_t)M * groups;
+    const int64_t slab = (int64_t)M * Np;
     const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    if ((MN & 3) == 0 && (reinterpret_cast<uintptr_t>(C) & 7) == 0) {
-        const int64_t n4 = MN >> 2;
-        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
-            float4 acc = __ldcs(reinterpret_cast<const float4*>(partial) + i);
-            for (int p = 1; p < P_k; ++p) {
-                const float4 v = __ldcs(reinterpret_cast<const float4*>(partial + (int64_t)p * MN) + i);
-                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
-            }
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += stride) {
+        const int m = (int)(i / groups);
+        const int n = (int)(i - (int64_t)m * groups) * 4;
+        const float* src = partial + (int64_t)m * Np + n;
+        float4 acc = __ldcs(reinterpret_cast<const float4*>(src));
+        for (int p = 1; p < P_k; ++p) {
+            const float4 v = __ldcs(reinterpret_cast<const float4*>(src + (int64_t)p * slab));
+            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        }
+        unsigned short* dst = C + (int64_t)m * N + n;
+        if (n + 4 <= N && (reinterpret_cast<uintptr_t>(dst) & 7) == 0) {
             uint2 o;
             o.x = (uint32_t)float_to_16(acc.x, dtype) | ((uint32_t)float_to_16(acc.y, dtype) << 16);
             o.y = (uint32_t)float_to_16(acc.z, dtype) | ((uint32_t)float_to_16(acc.w, dtype) << 16);
-            reinterpret_cast<uint2*>(C)[i] = o;
-        }
-    } else {
-        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < MN; i += stride) {
-            float acc = partial[i];
-            for (int p = 1; p < P_k; ++p) acc += partial[(int64_t)p * MN + i];
-            C[i] = float_to_16(acc, dtype);
+            *reinterpret_cast<uint2*>(dst) = o;
+        } else {
+            const float a[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (n + j < N) dst[j] = float_to_16(a[j], dtype);
         }
     }
 }
@@ -108,6 +115,7 @@ struct SimtParams {
     int64_t a_sm, a_sk;          // element strides of A along m and k
     int64_t b_sk, b_sn;          // element strides of B along k and n
     int P_n, P_k, kb_per_split;  // n tiles; k splits; k-blocks of 16 per split
+    int Np;                      // row pitch of the partials (N rounded up to 4)
     int dtype;
     unsigned short* C;
     float* partial;
@@ -173,7 +181,7 @@ simt_gemm_kernel(const unsigned short* __restrict__ A, const unsigned short* __r
             const int n = n0 + tx * 4 + j;
             if (n >= p.N) continue;
             if (p.P_k == 1) p.C[(int64_t)m * p.N + n] = float_to_16(acc[i][j], p.dtype);
-            else p.partial[((int64_t)split * p.M + m) * p.N + n] = acc[i][j];
+            else p.partial[((int64_t)split * p.M + m) * p.Np + n] = acc[i][j];
         }
     }
 }

@@ -19,6 +19,7 @@
 #include <cuda_fp16.h>
 #include <cuda_bf16.h>
 
+#include "adapt_internal.h"
 #include "ptx_sm100.cuh"
 
 namespace adapt {
@@ -36,8 +37,8 @@ struct UmmaParams {
     int stages;
     uint32_t idesc;                  // tcgen05 instruction descriptor
     void* C;                         // 16-bit output, row-major M x N (used when P_k == 1)
-    float* partial;                  // fp32 [P_k][M][N] (used when P_k > 1)
-    int c_vec_ok;                    // C rows are 16-byte aligned (N % 8 == 0 and base aligned)
+    float* partial;                  // fp32 [P_k][M][Np], Np = N rounded up to 4 (used when P_k > 1)
+    int Np;                          // row pitch of the partials in elements
     unsigned int* status;            // device status word: bit 0 = a bounded wait expired
 };
 
@@ -98,6 +99,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     uint8_t* gen_base = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
     volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(gen_base + (size_t)S * STAGE_BYTES + 16 * S + 32);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + (size_t)S * STAGE_BYTES + 16 * S + 36);
+    // epilogue staging: per epilogue warp 32 rows x 72 16-bit elements (64 columns + up to 7 of shift)
+    uint8_t* stage_out = gen_base + (size_t)S * STAGE_BYTES + kUmmaBarrierBytes;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -238,38 +241,80 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             decode_unit(p, unit, mb, nb, split);
             if (!ptx::mbar_wait(tfull_bar + 8u * buf, buf_phase, abort_flag)) { ok = false; break; }
             ptx::tc_fence_after();
-            const int row = mb * (128 * CG) + (int)cta_rank * 128 + q * 32 + lane;
+            const int row0 = mb * (128 * CG) + (int)cta_rank * 128 + q * 32;   // first row of this warp's quarter
+            const int row = row0 + lane;
             const int n0 = nb * BN;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
             const bool row_ok = row < p.M;
+            if (p.P_k == 1) {
+                // 16-bit output, any N and any base alignment: a thread converts its row's 64 columns and
+                // stages them in shared memory shifted by the row's misalignment in C, so that 16-byte
+                // aligned chunks of the staged row are 16-byte aligned chunks of C; the warp then writes
+                // each row as contiguous aligned 16-byte stores (2-byte stores only at a row segment's ends).
+                uint8_t* stg = stage_out + (warp - 2) * kUmmaStageWarpBytes;
+                const uintptr_t c_base = reinterpret_cast<uintptr_t>(p.C);
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
-                if (n0 + c0 >= p.N) break;                   // uniform across the warp
-                uint32_t r[32];
-                ptx::tmem_ld_32x32(t_row + (uint32_t)c0, r);
-                ptx::tmem_ld_wait();
-                if (!row_ok) continue;
-                const int col = n0 + c0;
-                if (p.P_k == 1) {
-                    unsigned short* crow = reinterpret_cast<unsigned short*>(p.C) + (size_t)row * p.N + col;
-                    if (p.c_vec_ok && col + 32 <= p.N) {
+                for (int c0 = 0; c0 < BN; c0 += 64) {
+                    if (n0 + c0 >= p.N) break;                       // uniform across the warp
+                    const int ncols = min(64, p.N - (n0 + c0));
+                    const int m_r = (int)(((c_base + 2ull * ((size_t)row * p.N + n0 + c0)) & 15u) >> 1);
+                    unsigned short* srow = reinterpret_cast<unsigned short*>(stg + lane * kUmmaStageRowBytes);
 #pragma unroll
-                        for (int v = 0; v < 4; ++v) {
-                            uint4 o;
-                            o.x = pack16(__uint_as_float(r[8 * v + 0]), __uint_as_float(r[8 * v + 1]), p.dtype);
-                            o.y = pack16(__uint_as_float(r[8 * v + 2]), __uint_as_float(r[8 * v + 3]), p.dtype);
-                            o.z = pack16(__uint_as_float(r[8 * v + 4]), __uint_as_float(r[8 * v + 5]), p.dtype);
-                            o.w = pack16(__uint_as_float(r[8 * v + 6]), __uint_as_float(r[8 * v + 7]), p.dtype);
-                            *reinterpret_cast<uint4*>(crow + 8 * v) = o;
+                    for (int h = 0; h < 2; ++h) {
+                        if (n0 + c0 + 32 * h >= p.N) break;          // uniform
+                        uint32_t r[32];
+                        ptx::tmem_ld_32x32(t_row + (uint32_t)(c0 + 32 * h), r);
+                        ptx::tmem_ld_wait();
+                        const int o = m_r + 32 * h;                  // element offset inside the staged row
+                        if ((o & 1) == 0) {
+                            uint32_t* d = reinterpret_cast<uint32_t*>(srow + o);
+#pragma unroll
+                            for (int i = 0; i < 16; ++i)
+                                d[i] = pack16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]), p.dtype);
+                        } else {
+                            srow[o] = cast16(__uint_as_float(r[0]), p.dtype);
+                            uint32_t* d = reinterpret_cast<uint32_t*>(srow + o + 1);
+#pragma unroll
+                            for (int i = 0; i < 15; ++i)
+                                d[i] = pack16(__uint_as_float(r[2 * i + 1]), __uint_as_float(r[2 * i + 2]), p.dtype);
+                            srow[o + 31] = cast16(__uint_as_float(r[31]), p.dtype);
                         }
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (col + j < p.N) crow[j] = cast16(__uint_as_float(r[j]), p.dtype);
                     }
-                } else {
-                    float* prow = p.partial + ((size_t)split * p.M + row) * p.N + col;
-                    if ((p.N & 3) == 0 && col + 32 <= p.N) {
+                    __syncwarp();
+                    // 32 rows x 9 aligned chunks, spread over the lanes
+#pragma unroll 1
+                    for (int f = lane; f < 32 * 9; f += 32) {
+                        const int rr = f / 9, qc = f - rr * 9;
+                        const int grow = row0 + rr;
+                        if (grow >= p.M) continue;
+                        const uintptr_t g0 = c_base + 2ull * ((size_t)grow * p.N + n0 + c0);
+                        const int m = (int)((g0 & 15u) >> 1);
+                        const int lo = max(8 * qc, m), hi = min(8 * qc + 8, m + ncols);
+                        if (lo >= hi) continue;
+                        const uint8_t* src = stg + rr * kUmmaStageRowBytes;
+                        uint8_t* dst = reinterpret_cast<uint8_t*>(g0 - 2 * m);
+                        if (hi - lo == 8) {
+                            *reinterpret_cast<uint4*>(dst + 16 * qc) = *reinterpret_cast<const uint4*>(src + 16 * qc);
+                        } else {
+                            for (int j = lo; j < hi; ++j)
+                                reinterpret_cast<unsigned short*>(dst)[j] = reinterpret_cast<const unsigned short*>(src)[j];
+                        }
+                    }
+                    __syncwarp();
+                }
+            } else {
+                // fp32 partial tile: rows of the workspace are 16-byte aligned (pitch Np), so a thread
+                // writes its row's 32 columns as eight aligned 16-byte stores
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    if (n0 + c0 >= p.N) break;                       // uniform across the warp
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32(t_row + (uint32_t)c0, r);
+                    ptx::tmem_ld_wait();
+                    if (!row_ok) continue;
+                    const int col = n0 + c0;
+                    float* prow = p.partial + ((size_t)split * p.M + row) * p.Np + col;
+                    if (col + 32 <= p.Np) {
 #pragma unroll
                         for (int v = 0; v < 8; ++v)
                             *reinterpret_cast<uint4*>(prow + 4 * v) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
@@ -313,11 +358,6 @@ inline uint32_t umma_idesc(int dtype, bool a_mn, bool b_mn, int mma_m, int mma_n
     const uint32_t fmt = dtype == 0 ? 0u : 1u;
     return (1u << 4) | (fmt << 7) | (fmt << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
            ((uint32_t)(mma_n >> 3) << 17) | ((uint32_t)(mma_m >> 4) << 24);
-}
-
-inline int umma_smem_bytes(int BN, int cg, int stages)
-{
-    return stages * (128 * kUmmaBK * 2 + (BN / cg) * kUmmaBK * 2) + 1024 + 256;
 }
 
 }  // namespace adapt
