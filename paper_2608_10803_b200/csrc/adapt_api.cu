@@ -108,6 +108,7 @@ struct State {
     Machine machine;
     Calib calib;
     unsigned int* d_status = nullptr;
+    unsigned long long* d_trace = nullptr;   // diagnostic builds only
     struct Workspace { void* ptr = nullptr; size_t bytes = 0; };
     std::unordered_map<cudaStream_t, Workspace> ws;
     std::unordered_map<cudaStream_t, Workspace> staging;   // device copies of host operands (adapt_matmul_host)
@@ -395,6 +396,10 @@ extern "C" adapt_status_t adapt_init(int device)
     S.encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
     CUDA_TRY(cudaMalloc(&S.d_status, sizeof(unsigned int)));
     CUDA_TRY(cudaMemset(S.d_status, 0, sizeof(unsigned int)));
+#ifdef ADAPT_TRACE_BUILD
+    CUDA_TRY(cudaMalloc(&S.d_trace, 8 * 60002));
+    CUDA_TRY(cudaMemset(S.d_trace, 0, 8 * 60002));
+#endif
     // opt every tensor-core kernel into the full shared-memory carve-out
     for (int fam = ADAPT_FAM_UMMA_1CTA; fam <= ADAPT_FAM_UMMA_2CTA; ++fam)
         for (int BN : {64, 128, 256})
@@ -589,6 +594,10 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.partial = partial;
     p.Np = (int)round_up(s.N, 4);
     p.status = S.d_status;
+    p.trace = nullptr;
+#ifdef ADAPT_TRACE_BUILD
+    p.trace = S.d_trace;
+#endif
 
     UmmaKernel k = launch_map_umma(c.family, c.BN, a_mn, b_mn);
     if (!k) return fail(ADAPT_ERR_UNSUPPORTED, "no compiled kernel for this tiling key%s");
@@ -716,3 +725,15 @@ extern "C" adapt_status_t adapt_matmul_host(adapt_handle_t plan, const void* A_h
     CUDA_TRY(cudaMemcpyAsync(C_host, d8 + nA + nB, (size_t)s.M * s.N * 2, cudaMemcpyDeviceToHost, stream));
     return ADAPT_OK;
 }
+
+#ifdef ADAPT_TRACE_BUILD
+// Diagnostic builds only: copy the timestamp trace to the host and clear it.
+extern "C" int adapt_debug_trace(unsigned long long* out, int n_words)
+{
+    State& S = st();
+    cudaDeviceSynchronize();
+    cudaMemcpy(out, S.d_trace, (size_t)n_words * 8, cudaMemcpyDeviceToHost);
+    cudaMemset(S.d_trace, 0, 8 * 60002);
+    return 0;
+}
+#endif

@@ -90,14 +90,15 @@ const Calib& default_calib();
 
 // Shared-memory layout of the tcgen05 kernels, used by the capacity check and by the launcher:
 // S stages of (A: 128 x 64, B: BN/cluster x 64) 16-bit, a barrier block, the epilogue staging
-// (4 warps x 32 rows x 144 B), and slack to align the stages to 1024 B.
+// (one 144-byte row per epilogue thread), and slack to align the stages to 1024 B.
 constexpr int kSkinnyKChunk = 512;   // k values the warp-level kernel stages per chunk; its k splits are whole chunks
 constexpr int kUmmaBarrierBytes = 256;
-constexpr int kUmmaStageRowBytes = 144;
-constexpr int kUmmaStageWarpBytes = 32 * kUmmaStageRowBytes;
+constexpr int kUmmaEpilogueWarps = 8;
+constexpr int kUmmaStageRowBytes = 144;   // 72 16-bit elements: 64 columns + up to 7 of alignment shift
 inline int umma_smem_bytes(int BN, int cluster, int stages)
 {
-    return stages * (128 * 64 * 2 + (BN / cluster) * 64 * 2) + kUmmaBarrierBytes + 4 * kUmmaStageWarpBytes + 1024;
+    return stages * (128 * 64 * 2 + (BN / cluster) * 64 * 2) + kUmmaBarrierBytes +
+           kUmmaEpilogueWarps * 32 * kUmmaStageRowBytes + 1024;
 }
 
 }  // namespace adapt

@@ -259,7 +259,7 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
         if (c.BN != 128 && c.BN != 256) return false;
     }
     if (c.BN % 16 != 0 || c.BN > 256) return false;                 // UMMA shape rule for M = 128/256
-    if (2 * c.BN > m.tmem_cols) return false;                       // two accumulator buffers in TMEM
+    if (2 * c.BN > m.tmem_cols) return false;                       // at least two accumulator buffers in TMEM
     if (c.stages < 1 || c.stages > 12) return false;
     c.smem_bytes = umma_smem_bytes(c.BN, c.cluster, c.stages);
     if (c.smem_bytes > m.smem_bytes) return false;

@@ -6,8 +6,8 @@
 //
 //   producer warp : TMA, 128-byte swizzle, into an S-stage shared-memory ring   (the paper's MTE2)
 //   MMA warp      : one thread issues tcgen05.mma kind::f16, 128|256 x BN x 16,
-//                   fp32 accumulator in TMEM, two accumulator buffers           (Cube + L0C)
-//   4 epilogue warps: tcgen05.ld -> one RN-even cast -> global                  (FixPipe)
+//                   fp32 accumulator in TMEM, 2-4 accumulator buffers           (Cube + L0C)
+//   8 epilogue warps: tcgen05.ld -> one RN-even cast -> shared -> bulk copy out (FixPipe)
 //
 // The CTA is persistent: it walks its list of work units (tile x k-split) so the producer runs
 // ahead across tile boundaries (Preloading, Eq. 14) and the epilogue of unit u overlaps the main
@@ -25,7 +25,7 @@
 namespace adapt {
 
 constexpr int kUmmaBK = 64;          // k-block: 64 elements = one 128-byte swizzle row
-constexpr int kUmmaThreads = 192;    // producer warp, MMA warp, four epilogue warps
+constexpr int kUmmaThreads = 320;    // producer warp, MMA warp, eight epilogue warps
 constexpr int kGroupM = 16;          // rasterisation: m-blocks per group
 
 struct UmmaParams {
@@ -40,7 +40,20 @@ struct UmmaParams {
     float* partial;                  // fp32 [P_k][M][Np], Np = N rounded up to 4 (used when P_k > 1)
     int Np;                          // row pitch of the partials in elements
     unsigned int* status;            // device status word: bit 0 = a bounded wait expired
+    unsigned long long* trace;       // timestamp trace of CTA 0 (diagnostic builds only), else null
 };
+
+#ifdef ADAPT_TRACE_BUILD
+#define ADAPT_TRACE(ev, unit)                                                                         \
+    do {                                                                                              \
+        if (p.trace && blockIdx.x == 0) {                                                             \
+            const unsigned long long sl = atomicAdd(p.trace, 1ull);                                   \
+            if (sl < 30000) { p.trace[1 + 2 * sl] = ((unsigned long long)(ev) << 32) | (unsigned)(unit); p.trace[2 + 2 * sl] = ptx::globaltimer_ns(); } \
+        }                                                                                             \
+    } while (0)
+#else
+#define ADAPT_TRACE(ev, unit) do { } while (0)
+#endif
 
 // unit index -> (m block, n block, split).  Units of one output tile are adjacent in split;
 // tiles are visited in groups of kGroupM m-blocks so that concurrently running CTAs share B
@@ -82,25 +95,28 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     constexpr int A_BYTES = 128 * kUmmaBK * 2;
     constexpr int B_BYTES = BN_CTA * kUmmaBK * 2;
     constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    constexpr int TMEM_COLS = 2 * BN;                     // two accumulator buffers
-    static_assert(TMEM_COLS == 128 || TMEM_COLS == 256 || TMEM_COLS == 512, "TMEM allocation is a power of two");
+    constexpr int NBUF = (512 / BN) < 4 ? (512 / BN) : 4; // accumulator buffers in TMEM
+    constexpr int TMEM_COLS = NBUF * BN;
+    constexpr int PASSES = BN / 64;                       // 64-column epilogue passes per tile
+    static_assert(TMEM_COLS == 256 || TMEM_COLS == 512, "TMEM allocation is a power of two");
     static_assert(BN_CTA % 64 == 0, "B is loaded in 64-column boxes");
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzle atoms are 1024-byte aligned
     const int S = p.stages;
     const uint32_t bar_base = smem_base + (uint32_t)S * STAGE_BYTES;
-    // barrier block: full[S], empty[S], tmem_full[2], tmem_empty[2], then the TMEM pointer and the abort flag
+    // barrier block: full[S], empty[S], tmem_full[NBUF], tmem_empty[NBUF], the TMEM pointer, the abort flag
     const uint32_t full_bar = bar_base;
     const uint32_t empty_bar = bar_base + 8u * S;
     const uint32_t tfull_bar = bar_base + 16u * S;
-    const uint32_t tempty_bar = tfull_bar + 16u;
-    const uint32_t tmem_slot = tempty_bar + 16u;
+    const uint32_t tempty_bar = tfull_bar + 8u * NBUF;
+    const uint32_t tmem_slot = tempty_bar + 8u * NBUF;
     uint8_t* gen_base = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
-    volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(gen_base + (size_t)S * STAGE_BYTES + 16 * S + 32);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(gen_base + (size_t)S * STAGE_BYTES + 16 * S + 36);
-    // epilogue staging: per epilogue warp 32 rows x 72 16-bit elements (64 columns + up to 7 of shift)
-    uint8_t* stage_out = gen_base + (size_t)S * STAGE_BYTES + kUmmaBarrierBytes;
+    uint8_t* bar_gen = gen_base + (size_t)S * STAGE_BYTES;
+    volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(bar_gen + 16 * S + 16 * NBUF);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 16 * S + 16 * NBUF + 4);
+    // epilogue staging: one row of 72 16-bit elements (64 columns + up to 7 of shift) per epilogue thread
+    uint8_t* stage_out = bar_gen + kUmmaBarrierBytes;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -113,9 +129,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             ptx::mbar_init(full_bar + 8u * s, 1);          // one arrive.expect_tx per phase
             ptx::mbar_init(empty_bar + 8u * s, 1);         // one tcgen05.commit per phase
         }
-        for (int b = 0; b < 2; ++b) {
+        for (int b = 0; b < NBUF; ++b) {
             ptx::mbar_init(tfull_bar + 8u * b, 1);         // one tcgen05.commit per phase
-            ptx::mbar_init(tempty_bar + 8u * b, 4 * CG);   // one arrive per epilogue warp of every CTA of the group
+            ptx::mbar_init(tempty_bar + 8u * b, kUmmaEpilogueWarps * CG);   // one arrive per epilogue warp of the group
         }
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
@@ -184,6 +200,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
+                ADAPT_TRACE(1, unit);
             }
         }
     } else if (warp == 1) {
@@ -206,6 +223,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
                 if (!ptx::mbar_wait(tempty_bar + 8u * buf, buf_phase ^ 1u, abort_flag)) { ok = false; break; }
                 ptx::tc_fence_after();
+                ADAPT_TRACE(2, unit);
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (!ptx::mbar_wait(full_bar + 8u * stage, phase, abort_flag)) { ok = false; break; }
@@ -226,81 +244,102 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 if (!ok) break;
                 if (CG == 1) ptx::umma_commit_1(tfull_bar + 8u * buf);
                 else ptx::umma_commit_2(tfull_bar + 8u * buf, 3);
-                buf ^= 1;
-                if (buf == 0) buf_phase ^= 1u;
+                ADAPT_TRACE(3, unit);
+                if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
             }
         }
     } else {
         // ------------------------------ epilogue -----------------------------------------------
-        const int q = warp & 3;                              // TMEM lane quarter this warp may read
+        // Eight warps: warp w may read TMEM lanes 32*(w % 4) .. +31 only, so two warps share each lane
+        // quarter and take alternate 64-column passes (alternate tiles when a tile is one pass wide).
+        const int q = warp & 3;
+        const int half = (warp - 2) >> 2;
         int buf = 0;
         uint32_t buf_phase = 0;
+        int seq = 0;                                         // tiles this CTA has processed so far
         bool ok = true;
-        for (int unit = unit0; ok && unit < p.num_units; unit += unit_step) {
+        uint8_t* stg = stage_out + ((warp - 2) * 32 + lane) * kUmmaStageRowBytes;   // this thread's staging row
+        unsigned short* srow = reinterpret_cast<unsigned short*>(stg);
+        const uintptr_t c_base = reinterpret_cast<uintptr_t>(p.C);
+        for (int unit = unit0; ok && unit < p.num_units; unit += unit_step, ++seq) {
             int mb, nb, split;
             decode_unit(p, unit, mb, nb, split);
             if (!ptx::mbar_wait(tfull_bar + 8u * buf, buf_phase, abort_flag)) { ok = false; break; }
             ptx::tc_fence_after();
-            const int row0 = mb * (128 * CG) + (int)cta_rank * 128 + q * 32;   // first row of this warp's quarter
-            const int row = row0 + lane;
+            if (warp == 2 && lane == 0) ADAPT_TRACE(4, unit);
+            const int row = mb * (128 * CG) + (int)cta_rank * 128 + q * 32 + lane;
             const int n0 = nb * BN;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
             const bool row_ok = row < p.M;
             if (p.P_k == 1) {
-                // 16-bit output, any N and any base alignment: a thread converts its row's 64 columns and
-                // stages them in shared memory shifted by the row's misalignment in C, so that 16-byte
-                // aligned chunks of the staged row are 16-byte aligned chunks of C; the warp then writes
-                // each row as contiguous aligned 16-byte stores (2-byte stores only at a row segment's ends).
-                uint8_t* stg = stage_out + (warp - 2) * kUmmaStageWarpBytes;
-                const uintptr_t c_base = reinterpret_cast<uintptr_t>(p.C);
+                // 16-bit output, any N and any base alignment.  A thread converts 64 columns of its row
+                // and stages them in its own shared-memory row, shifted by the row's misalignment in C,
+                // so that 16-byte aligned chunks of the staged row are 16-byte aligned chunks of C.  The
+                // aligned interior of the row segment then leaves as one bulk copy (shared -> global);
+                // the at most 7 + 7 elements at its ends are 2-byte stores.  A thread touches only its
+                // own staging row, so no thread waits for another.
+                const uintptr_t g_tile = c_base + 2ull * ((size_t)row * p.N + n0);
 #pragma unroll 1
-                for (int c0 = 0; c0 < BN; c0 += 64) {
+                for (int pass = 0; pass < PASSES; ++pass) {
+                    const int c0 = pass * 64;
                     if (n0 + c0 >= p.N) break;                       // uniform across the warp
+                    if (((seq * PASSES + pass) & 1) != half) continue;   // the other warp of this quarter takes it
                     const int ncols = min(64, p.N - (n0 + c0));
-                    const int m_r = (int)(((c_base + 2ull * ((size_t)row * p.N + n0 + c0)) & 15u) >> 1);
-                    unsigned short* srow = reinterpret_cast<unsigned short*>(stg + lane * kUmmaStageRowBytes);
+                    const uintptr_t g0 = g_tile + 2u * c0;
+                    const int m_r = (int)((g0 & 15u) >> 1);
+                    uint32_t r0[32], r1[32];
+                    ptx::tmem_ld_32x32(t_row + (uint32_t)c0, r0);
+                    if (ncols > 32) ptx::tmem_ld_32x32(t_row + (uint32_t)(c0 + 32), r1);   // uniform
+                    ptx::tmem_ld_wait();
+                    if (warp == 2 && lane == 0) ADAPT_TRACE(5, unit);
+                    ptx::bulk_wait_read<0>();                        // the previous copy out of this row has read it
+                    if ((m_r & 1) == 0) {
+                        uint32_t* d = reinterpret_cast<uint32_t*>(srow + m_r);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        if (n0 + c0 + 32 * h >= p.N) break;          // uniform
-                        uint32_t r[32];
-                        ptx::tmem_ld_32x32(t_row + (uint32_t)(c0 + 32 * h), r);
-                        ptx::tmem_ld_wait();
-                        const int o = m_r + 32 * h;                  // element offset inside the staged row
-                        if ((o & 1) == 0) {
-                            uint32_t* d = reinterpret_cast<uint32_t*>(srow + o);
+                        for (int i = 0; i < 16; ++i)
+                            d[i] = pack16(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]), p.dtype);
+                        if (ncols > 32) {
 #pragma unroll
                             for (int i = 0; i < 16; ++i)
-                                d[i] = pack16(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]), p.dtype);
-                        } else {
-                            srow[o] = cast16(__uint_as_float(r[0]), p.dtype);
-                            uint32_t* d = reinterpret_cast<uint32_t*>(srow + o + 1);
+                                d[16 + i] = pack16(__uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]), p.dtype);
+                        }
+                    } else {
+                        srow[m_r] = cast16(__uint_as_float(r0[0]), p.dtype);
+                        uint32_t* d = reinterpret_cast<uint32_t*>(srow + m_r + 1);
+#pragma unroll
+                        for (int i = 0; i < 15; ++i)
+                            d[i] = pack16(__uint_as_float(r0[2 * i + 1]), __uint_as_float(r0[2 * i + 2]), p.dtype);
+                        if (ncols > 32) {
+                            d[15] = pack16(__uint_as_float(r0[31]), __uint_as_float(r1[0]), p.dtype);
 #pragma unroll
                             for (int i = 0; i < 15; ++i)
-                                d[i] = pack16(__uint_as_float(r[2 * i + 1]), __uint_as_float(r[2 * i + 2]), p.dtype);
-                            srow[o + 31] = cast16(__uint_as_float(r[31]), p.dtype);
-                        }
-                    }
-                    __syncwarp();
-                    // 32 rows x 9 aligned chunks, spread over the lanes
-#pragma unroll 1
-                    for (int f = lane; f < 32 * 9; f += 32) {
-                        const int rr = f / 9, qc = f - rr * 9;
-                        const int grow = row0 + rr;
-                        if (grow >= p.M) continue;
-                        const uintptr_t g0 = c_base + 2ull * ((size_t)grow * p.N + n0 + c0);
-                        const int m = (int)((g0 & 15u) >> 1);
-                        const int lo = max(8 * qc, m), hi = min(8 * qc + 8, m + ncols);
-                        if (lo >= hi) continue;
-                        const uint8_t* src = stg + rr * kUmmaStageRowBytes;
-                        uint8_t* dst = reinterpret_cast<uint8_t*>(g0 - 2 * m);
-                        if (hi - lo == 8) {
-                            *reinterpret_cast<uint4*>(dst + 16 * qc) = *reinterpret_cast<const uint4*>(src + 16 * qc);
+                                d[16 + i] = pack16(__uint_as_float(r1[2 * i + 1]), __uint_as_float(r1[2 * i + 2]), p.dtype);
+                            srow[m_r + 63] = cast16(__uint_as_float(r1[31]), p.dtype);
                         } else {
-                            for (int j = lo; j < hi; ++j)
-                                reinterpret_cast<unsigned short*>(dst)[j] = reinterpret_cast<const unsigned short*>(src)[j];
+                            srow[m_r + 31] = cast16(__uint_as_float(r0[31]), p.dtype);
                         }
                     }
-                    __syncwarp();
+                    if (row_ok) {
+                        const int end = m_r + ncols;                 // valid staged elements: [m_r, end)
+                        const int lo8 = (m_r + 7) & ~7, hi8 = end & ~7;
+                        unsigned short* grow = reinterpret_cast<unsigned short*>(g0 - 2 * m_r);   // 16-byte aligned
+                        if (hi8 > lo8) {
+                            ptx::fence_proxy_async_smem();
+                            ptx::bulk_store(grow + lo8, ptx::smem_u32(srow + lo8), (uint32_t)(2 * (hi8 - lo8)));
+                        }
+                        if (m_r | (end & 7)) {                       // ragged ends: at most 7 + 7 elements
+                            const int head_end = min(lo8, end);
+                            const int tail_begin = max(hi8, head_end);
+#pragma unroll
+                            for (int i = 0; i < 7; ++i) {
+                                const int jh = m_r + i, jt = tail_begin + i;
+                                if (jh < head_end) grow[jh] = srow[jh];
+                                if (jt < end) grow[jt] = srow[jt];
+                            }
+                        }
+                    }
+                    ptx::bulk_commit();
+                    if (warp == 2 && lane == 0) ADAPT_TRACE(6, unit);
                 }
             } else {
                 // fp32 partial tile: rows of the workspace are 16-byte aligned (pitch Np), so a thread
@@ -308,6 +347,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll 1
                 for (int c0 = 0; c0 < BN; c0 += 32) {
                     if (n0 + c0 >= p.N) break;                       // uniform across the warp
+                    if (((seq * (BN / 32) + (c0 >> 5)) & 1) != half) continue;
                     uint32_t r[32];
                     ptx::tmem_ld_32x32(t_row + (uint32_t)c0, r);
                     ptx::tmem_ld_wait();
@@ -325,16 +365,17 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     }
                 }
             }
-            // this warp has read its quarter of the accumulator: hand the buffer back to the MMA warp
+            // this warp has read its share of the accumulator: hand the buffer back to the MMA warp
             ptx::tc_fence_before();
             __syncwarp();
             if (lane == 0) {
                 if (CG == 1) ptx::mbar_arrive(tempty_bar + 8u * buf);
                 else ptx::mbar_arrive_cluster(tempty_bar + 8u * buf, 0);
+                if (warp == 2) ADAPT_TRACE(7, unit);
             }
-            buf ^= 1;
-            if (buf == 0) buf_phase ^= 1u;
+            if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
         }
+        ptx::bulk_wait_all();                                // this thread's output copies are complete
     }
 
     // ------------------------------ common exit ----------------------------------------------
