@@ -7,7 +7,7 @@
 //   producer warp : TMA, 128-byte swizzle, into an S-stage shared-memory ring   (the paper's MTE2)
 //   MMA warp      : one thread issues tcgen05.mma kind::f16, 128|256 x BN x 16,
 //                   fp32 accumulator in TMEM, 2-4 accumulator buffers           (Cube + L0C)
-//   8 epilogue warps: tcgen05.ld -> one RN-even cast -> shared -> bulk copy out (FixPipe)
+//   8 epilogue warps: tcgen05.ld -> one RN-even cast -> shared -> coalesced 16 B stores (FixPipe)
 //
 // The CTA is persistent: it walks its list of work units (tile x k-split) so the producer runs
 // ahead across tile boundaries (Preloading, Eq. 14) and the epilogue of unit u overlaps the main
@@ -273,26 +273,29 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             const bool row_ok = row < p.M;
             if (p.P_k == 1) {
                 // 16-bit output, any N and any base alignment.  A thread converts 64 columns of its row
-                // and stages them in its own shared-memory row, shifted by the row's misalignment in C,
-                // so that 16-byte aligned chunks of the staged row are 16-byte aligned chunks of C.  The
-                // aligned interior of the row segment then leaves as one bulk copy (shared -> global);
-                // the at most 7 + 7 elements at its ends are 2-byte stores.  A thread touches only its
-                // own staging row, so no thread waits for another.
-                const uintptr_t g_tile = c_base + 2ull * ((size_t)row * p.N + n0);
+                // and stages them in shared memory shifted by the row's misalignment in C, so that
+                // 16-byte aligned chunks of a staged row are 16-byte aligned chunks of C.  The warp then
+                // writes its 32 row segments cooperatively, consecutive lanes taking consecutive chunks
+                // of a row (aligned 16-byte stores, about 3.5 rows per instruction); the at most 7 + 7
+                // elements at a segment's ends are 2-byte stores by the row's own thread.
+                const int rowq0 = row - lane;                        // first row of this warp's quarter
+                const uintptr_t g_tile = c_base + 2ull * ((size_t)rowq0 * p.N + n0);
+                const uintptr_t row_bytes = 2ull * (uintptr_t)p.N;
 #pragma unroll 1
                 for (int pass = 0; pass < PASSES; ++pass) {
                     const int c0 = pass * 64;
                     if (n0 + c0 >= p.N) break;                       // uniform across the warp
                     if (((seq * PASSES + pass) & 1) != half) continue;   // the other warp of this quarter takes it
                     const int ncols = min(64, p.N - (n0 + c0));
-                    const uintptr_t g0 = g_tile + 2u * c0;
+                    const uintptr_t g_pass = g_tile + 2u * c0;       // row rowq0, column n0 + c0
+                    const uintptr_t g0 = g_pass + (uintptr_t)lane * row_bytes;
                     const int m_r = (int)((g0 & 15u) >> 1);
                     uint32_t r0[32], r1[32];
                     ptx::tmem_ld_32x32(t_row + (uint32_t)c0, r0);
                     if (ncols > 32) ptx::tmem_ld_32x32(t_row + (uint32_t)(c0 + 32), r1);   // uniform
                     ptx::tmem_ld_wait();
                     if (warp == 2 && lane == 0) ADAPT_TRACE(5, unit);
-                    ptx::bulk_wait_read<0>();                        // the previous copy out of this row has read it
+                    __syncwarp();                                    // the previous pass has been written out
                     if ((m_r & 1) == 0) {
                         uint32_t* d = reinterpret_cast<uint32_t*>(srow + m_r);
 #pragma unroll
@@ -319,26 +322,34 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             srow[m_r + 31] = cast16(__uint_as_float(r0[31]), p.dtype);
                         }
                     }
-                    if (row_ok) {
-                        const int end = m_r + ncols;                 // valid staged elements: [m_r, end)
+                    if (warp == 2 && lane == 0) ADAPT_TRACE(9, unit);
+                    const int end = m_r + ncols;                     // valid staged elements of this row: [m_r, end)
+                    if (row_ok && (m_r | (end & 7))) {               // ragged ends of this thread's own row
                         const int lo8 = (m_r + 7) & ~7, hi8 = end & ~7;
                         unsigned short* grow = reinterpret_cast<unsigned short*>(g0 - 2 * m_r);   // 16-byte aligned
-                        if (hi8 > lo8) {
-                            ptx::fence_proxy_async_smem();
-                            ptx::bulk_store(grow + lo8, ptx::smem_u32(srow + lo8), (uint32_t)(2 * (hi8 - lo8)));
-                        }
-                        if (m_r | (end & 7)) {                       // ragged ends: at most 7 + 7 elements
-                            const int head_end = min(lo8, end);
-                            const int tail_begin = max(hi8, head_end);
+                        const int head_end = min(lo8, end);
+                        const int tail_begin = max(hi8, head_end);
 #pragma unroll
-                            for (int i = 0; i < 7; ++i) {
-                                const int jh = m_r + i, jt = tail_begin + i;
-                                if (jh < head_end) grow[jh] = srow[jh];
-                                if (jt < end) grow[jt] = srow[jt];
-                            }
+                        for (int i = 0; i < 7; ++i) {
+                            const int jh = m_r + i, jt = tail_begin + i;
+                            if (jh < head_end) grow[jh] = srow[jh];
+                            if (jt < end) grow[jt] = srow[jt];
                         }
                     }
-                    ptx::bulk_commit();
+                    __syncwarp();                                    // every row of the warp is staged
+                    // 32 rows x 9 aligned chunks: lane + 32*it = 9*rr + qc
+                    int rr = lane / 9, qc = lane - 9 * rr;
+                    const uint8_t* stg_warp = stage_out + (warp - 2) * (32 * kUmmaStageRowBytes);
+#pragma unroll
+                    for (int it = 0; it < 9; ++it) {
+                        const uintptr_t g = g_pass + (uintptr_t)rr * row_bytes;
+                        const int m = (int)((g & 15u) >> 1);
+                        if (rowq0 + rr < p.M && 8 * qc >= m && 8 * qc + 8 <= m + ncols)
+                            *reinterpret_cast<uint4*>(g - 2 * m + 16 * qc) =
+                                *reinterpret_cast<const uint4*>(stg_warp + rr * kUmmaStageRowBytes + 16 * qc);
+                        rr += 3; qc += 5;
+                        if (qc >= 9) { qc -= 9; rr += 1; }
+                    }
                     if (warp == 2 && lane == 0) ADAPT_TRACE(6, unit);
                 }
             } else {
@@ -375,7 +386,6 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
             if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
         }
-        ptx::bulk_wait_all();                                // this thread's output copies are complete
     }
 
     // ------------------------------ common exit ----------------------------------------------
