@@ -142,6 +142,31 @@ adapt_status_t adapt_matmul(adapt_handle_t plan, const void* A, const void* B, v
 adapt_status_t adapt_matmul_host(adapt_handle_t plan, const void* A_host, const void* B_host, void* C_host,
                                  void* cuda_stream);
 
+/* C = A * B for callers that must not trigger a device allocation: code running where cudaMalloc is
+ * off limits, such as a latency-critical serving loop that forbids the implicit device
+ * synchronisation an allocation brings, a process whose memory pool has been handed over whole to
+ * another allocator, or a plug-in that is only given buffers and a stream.  The paper has no
+ * counterpart to this entry point; it exists for those callers only.
+ *
+ * It runs the CUDA-core split-K path (fp32 partial products per K split, then the fixed-order
+ * reduction with the single 16-bit cast) with the partials kept in a fixed 4 MiB array that is
+ * part of the library image, so every GPU that loads the library holds those 4 MiB until the
+ * process exits.  Limit: 2 * M * roundup(N, 4) * 4 bytes <= 4 MiB (at least two K splits must
+ * fit); larger outputs are rejected with ADAPT_ERR_UNSUPPORTED and a message, and K must be >= 1,
+ * M, N >= 1.  The number of splits is the largest that fits, at most 32 and at most ceil(K / 64).
+ *
+ * No cudaMalloc, cudaFree or other allocating call is made, neither adapt_init nor a plan is
+ * needed, and the current device is used.  The first call on a device looks up the array's device
+ * address (once per device); make that first call outside any stream capture.  All calls share
+ * the one array, whatever the stream: two calls that overlap on the GPU race on it, so keep calls
+ * on one stream or order them yourself.  The array keeps the previous call's partials; every
+ * element a call reads is first written by that call, so nothing needs clearing.
+ * A, B: DEVICE inputs in the stated layouts, C: DEVICE output, row-major M x N, 2-byte aligned.
+ * Enqueues two kernels on the stream and returns without synchronising. */
+adapt_status_t adapt_matmul_noalloc(int64_t M, int64_t N, int64_t K, adapt_dtype_t dtype,
+                                    adapt_layout_t layoutA, adapt_layout_t layoutB,
+                                    const void* A, const void* B, void* C, void* cuda_stream);
+
 /* Thread-local status of the last failing call on this thread, and its text. */
 adapt_status_t adapt_last_error(void);
 const char* adapt_last_error_message(void);

@@ -24,6 +24,7 @@ EXPORTS = [
     "adapt_last_error_message", "adapt_status_string", "adapt_plan_info", "adapt_plan_candidates",
     "adapt_matmul_plan_forced", "adapt_classify", "adapt_model_read_volume", "adapt_model_write_volume",
     "adapt_model_pipeline", "adapt_poll_device_status", "adapt_plan_cache_size", "adapt_launch_count",
+    "adapt_matmul_noalloc",
 ]
 
 
@@ -81,6 +82,8 @@ def load():
     lib.adapt_matmul.argtypes = [vp, vp, vp, vp, vp]
     lib.adapt_matmul_host.restype = i32
     lib.adapt_matmul_host.argtypes = [vp, vp, vp, vp, vp]
+    lib.adapt_matmul_noalloc.restype = i32
+    lib.adapt_matmul_noalloc.argtypes = [i64, i64, i64, i32, i32, i32, vp, vp, vp, vp]
     lib.adapt_last_error.restype = i32
     lib.adapt_last_error_message.restype = ctypes.c_char_p
     lib.adapt_status_string.restype = ctypes.c_char_p
@@ -142,6 +145,13 @@ def adapt_matmul(plan, A_ptr: int, B_ptr: int, C_ptr: int, stream: int = 0):
 def adapt_matmul_host(plan, A_host_ptr: int, B_host_ptr: int, C_host_ptr: int, stream: int = 0):
     """Enqueue H2D(A, B), the GEMM and D2H(C) for host buffers (raw host addresses)."""
     _check(load().adapt_matmul_host(plan, A_host_ptr, B_host_ptr, C_host_ptr, stream))
+
+
+def adapt_matmul_noalloc(M, N, K, dtype, layoutA, layoutB, A_ptr: int, B_ptr: int, C_ptr: int, stream: int = 0):
+    """C = A*B without any device allocation: split-K partials go to the library's fixed 4 MiB
+    scratch.  For callers that may not call cudaMalloc; the output must satisfy
+    2 * M * roundup(N, 4) * 4 bytes <= 4 MiB.  Calls that overlap on the GPU race on the scratch."""
+    _check(load().adapt_matmul_noalloc(M, N, K, dtype, layoutA, layoutB, A_ptr, B_ptr, C_ptr, stream))
 
 
 def adapt_plan_info(plan) -> PlanInfo:

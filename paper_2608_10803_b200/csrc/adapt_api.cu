@@ -737,3 +737,83 @@ extern "C" int adapt_debug_trace(unsigned long long* out, int n_words)
     return 0;
 }
 #endif
+
+// ---------------------------------------------------------------------------------------------
+// allocation-free entry point
+// ---------------------------------------------------------------------------------------------
+// Scratch for the fp32 split-K partials of adapt_matmul_noalloc.  It lives in the library image:
+// every device that loads the library carries it.  In host code the name below is only a handle
+// for cudaGetSymbolAddress, never a pointer a kernel may be given.
+constexpr size_t kNoAllocScratchBytes = (size_t)4 << 20;
+static __device__ __align__(256) unsigned char g_noalloc_scratch[kNoAllocScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::atomic<float*> g_noalloc_ptr[kMaxDevices];      // device address of the scratch, per device
+std::mutex g_noalloc_mu;
+}  // namespace
+
+extern "C" adapt_status_t adapt_matmul_noalloc(int64_t M, int64_t N, int64_t K, adapt_dtype_t dtype,
+                                               adapt_layout_t layoutA, adapt_layout_t layoutB,
+                                               const void* A, const void* B, void* C, void* cuda_stream)
+{
+    if (M < 1 || N < 1 || K < 1) return fail(ADAPT_ERR_INVALID_ARG, "adapt_matmul_noalloc needs M, N, K >= 1%s");
+    if (M > 2147483647ll || N > 2147483647ll || K > 2147483647ll) return fail(ADAPT_ERR_UNSUPPORTED, "dimension above 2^31-1%s");
+    if (((int)dtype != 0 && (int)dtype != 1) || ((int)layoutA != 0 && (int)layoutA != 1) || ((int)layoutB != 0 && (int)layoutB != 1))
+        return fail(ADAPT_ERR_INVALID_ARG, "bad dtype or layout value%s");
+    if (!A || !B || !C) return fail(ADAPT_ERR_INVALID_ARG, "null operand%s");
+    if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 1) return fail(ADAPT_ERR_INVALID_ARG, "operands must be 2-byte aligned%s");
+    const int64_t Np = round_up(N, 4);
+    const int64_t slab = M * Np * 4;                       // bytes of one split's partial
+    if (slab <= 0 || 2 * slab > (int64_t)kNoAllocScratchBytes)
+        return fail(ADAPT_ERR_UNSUPPORTED,
+                    "adapt_matmul_noalloc: output too large for the fixed 4 MiB scratch (needs 2 * M * roundup(N,4) * 4 bytes <= 4 MiB)%s");
+
+    int dev = -1;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return fail(ADAPT_ERR_UNSUPPORTED, "device ordinal out of range%s");
+    float* scratch = g_noalloc_ptr[dev].load(std::memory_order_acquire);
+    if (!scratch) {
+        // set-up, once per device, with that device current: ask the runtime for the DEVICE address
+        std::lock_guard<std::mutex> lock(g_noalloc_mu);
+        scratch = g_noalloc_ptr[dev].load(std::memory_order_acquire);
+        if (!scratch) {
+            void* ptr = nullptr;
+            cudaError_t e = cudaGetSymbolAddress(&ptr, g_noalloc_scratch);
+            if (e != cudaSuccess || !ptr) return fail(ADAPT_ERR_CUDA, "cudaGetSymbolAddress(scratch): %s", cudaGetErrorString(e));
+            scratch = (float*)ptr;
+            g_noalloc_ptr[dev].store(scratch, std::memory_order_release);
+        }
+    }
+
+    const int64_t kblocks = ceil_div(K, 16);
+    int64_t pk = std::min<int64_t>(32, (int64_t)kNoAllocScratchBytes / slab);
+    pk = std::min<int64_t>(pk, ceil_div(K, 64));
+    if (pk < 1) pk = 1;
+    if (pk > kblocks) pk = kblocks;
+    const int64_t per = ceil_div(kblocks, pk);
+    pk = ceil_div(kblocks, per);                           // no empty split
+
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    SimtParams p;
+    p.M = (int)M; p.N = (int)N; p.K = (int)K;
+    if (layoutA == ADAPT_ROW_MAJOR) { p.a_sm = K; p.a_sk = 1; } else { p.a_sm = 1; p.a_sk = M; }
+    if (layoutB == ADAPT_ROW_MAJOR) { p.b_sk = N; p.b_sn = 1; } else { p.b_sk = 1; p.b_sn = K; }
+    p.P_n = (int)ceil_div(N, 64);
+    p.P_k = 2;                                             // any value > 1: the kernel then writes fp32 partials
+    p.Np = (int)Np;
+    p.kb_per_split = (int)per;
+    p.dtype = (int)dtype;
+    p.C = (unsigned short*)C;
+    p.partial = scratch;
+    const int64_t tiles = ceil_div(M, 64) * ceil_div(N, 64);
+    dim3 grid((unsigned)tiles, (unsigned)pk, 1);
+    simt_gemm_kernel<<<grid, 256, 0, stream>>>((const unsigned short*)A, (const unsigned short*)B, p);
+    CUDA_TRY(cudaGetLastError());
+    const int64_t work = M * (Np / 4);
+    const int blocks = (int)std::min<int64_t>(ceil_div(work, 256), 148 * 8);
+    splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(scratch, (unsigned short*)C, (int)M, (int)N, (int)Np, (int)pk, (int)dtype);
+    CUDA_TRY(cudaGetLastError());
+    st().launches.fetch_add(2, std::memory_order_relaxed);
+    return ADAPT_OK;
+}
