@@ -281,76 +281,90 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 const int rowq0 = row - lane;                        // first row of this warp's quarter
                 const uintptr_t g_tile = c_base + 2ull * ((size_t)rowq0 * p.N + n0);
                 const uintptr_t row_bytes = 2ull * (uintptr_t)p.N;
+                // the two warps of a lane quarter take alternate tiles, so one thread sees all passes of
+                // its row and can carry the ragged tail of a pass into the head of the next one
+                if ((seq & 1) == half) {
+                    const uintptr_t g_row = g_tile + (uintptr_t)lane * row_bytes;   // this thread's row, column n0
+                    const int m_r = (int)((g_row & 15u) >> 1);           // the same in every pass: a pass is 128 bytes
+                    const int tile_cols = min(BN, p.N - n0);
 #pragma unroll 1
-                for (int pass = 0; pass < PASSES; ++pass) {
-                    const int c0 = pass * 64;
-                    if (n0 + c0 >= p.N) break;                       // uniform across the warp
-                    if (((seq * PASSES + pass) & 1) != half) continue;   // the other warp of this quarter takes it
-                    const int ncols = min(64, p.N - (n0 + c0));
-                    const uintptr_t g_pass = g_tile + 2u * c0;       // row rowq0, column n0 + c0
-                    const uintptr_t g0 = g_pass + (uintptr_t)lane * row_bytes;
-                    const int m_r = (int)((g0 & 15u) >> 1);
-                    uint32_t r0[32], r1[32];
-                    ptx::tmem_ld_32x32(t_row + (uint32_t)c0, r0);
-                    if (ncols > 32) ptx::tmem_ld_32x32(t_row + (uint32_t)(c0 + 32), r1);   // uniform
-                    ptx::tmem_ld_wait();
-                    if (warp == 2 && lane == 0) ADAPT_TRACE(5, unit);
-                    __syncwarp();                                    // the previous pass has been written out
-                    if ((m_r & 1) == 0) {
-                        uint32_t* d = reinterpret_cast<uint32_t*>(srow + m_r);
-#pragma unroll
-                        for (int i = 0; i < 16; ++i)
-                            d[i] = pack16(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]), p.dtype);
-                        if (ncols > 32) {
+                    for (int pass = 0; pass < PASSES; ++pass) {
+                        const int c0 = pass * 64;
+                        if (c0 >= tile_cols) break;                      // uniform across the warp
+                        const int ncols = min(64, tile_cols - c0);
+                        const bool last = c0 + 64 >= tile_cols;
+                        uint32_t r0[32], r1[32];
+                        ptx::tmem_ld_32x32(t_row + (uint32_t)c0, r0);
+                        if (ncols > 32) ptx::tmem_ld_32x32(t_row + (uint32_t)(c0 + 32), r1);   // uniform
+                        ptx::tmem_ld_wait();
+                        if (warp == 2 && lane == 0) ADAPT_TRACE(5, unit);
+                        __syncwarp();                                    // the previous pass has been written out
+                        // carry: elements 64..71 of the previous pass become elements 0..7 of this one
+                        if (pass > 0) *reinterpret_cast<uint4*>(srow) = *reinterpret_cast<const uint4*>(srow + 64);
+                        if ((m_r & 1) == 0) {
+                            uint32_t* d = reinterpret_cast<uint32_t*>(srow + m_r);
 #pragma unroll
                             for (int i = 0; i < 16; ++i)
-                                d[16 + i] = pack16(__uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]), p.dtype);
-                        }
-                    } else {
-                        srow[m_r] = cast16(__uint_as_float(r0[0]), p.dtype);
-                        uint32_t* d = reinterpret_cast<uint32_t*>(srow + m_r + 1);
+                                d[i] = pack16(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]), p.dtype);
+                            if (ncols > 32) {
 #pragma unroll
-                        for (int i = 0; i < 15; ++i)
-                            d[i] = pack16(__uint_as_float(r0[2 * i + 1]), __uint_as_float(r0[2 * i + 2]), p.dtype);
-                        if (ncols > 32) {
-                            d[15] = pack16(__uint_as_float(r0[31]), __uint_as_float(r1[0]), p.dtype);
+                                for (int i = 0; i < 16; ++i)
+                                    d[16 + i] = pack16(__uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]), p.dtype);
+                            }
+                        } else {
+                            srow[m_r] = cast16(__uint_as_float(r0[0]), p.dtype);
+                            uint32_t* d = reinterpret_cast<uint32_t*>(srow + m_r + 1);
 #pragma unroll
                             for (int i = 0; i < 15; ++i)
-                                d[16 + i] = pack16(__uint_as_float(r1[2 * i + 1]), __uint_as_float(r1[2 * i + 2]), p.dtype);
-                            srow[m_r + 63] = cast16(__uint_as_float(r1[31]), p.dtype);
-                        } else {
-                            srow[m_r + 31] = cast16(__uint_as_float(r0[31]), p.dtype);
-                        }
-                    }
-                    if (warp == 2 && lane == 0) ADAPT_TRACE(9, unit);
-                    const int end = m_r + ncols;                     // valid staged elements of this row: [m_r, end)
-                    if (row_ok && (m_r | (end & 7))) {               // ragged ends of this thread's own row
-                        const int lo8 = (m_r + 7) & ~7, hi8 = end & ~7;
-                        unsigned short* grow = reinterpret_cast<unsigned short*>(g0 - 2 * m_r);   // 16-byte aligned
-                        const int head_end = min(lo8, end);
-                        const int tail_begin = max(hi8, head_end);
+                                d[i] = pack16(__uint_as_float(r0[2 * i + 1]), __uint_as_float(r0[2 * i + 2]), p.dtype);
+                            if (ncols > 32) {
+                                d[15] = pack16(__uint_as_float(r0[31]), __uint_as_float(r1[0]), p.dtype);
 #pragma unroll
-                        for (int i = 0; i < 7; ++i) {
-                            const int jh = m_r + i, jt = tail_begin + i;
-                            if (jh < head_end) grow[jh] = srow[jh];
-                            if (jt < end) grow[jt] = srow[jt];
+                                for (int i = 0; i < 15; ++i)
+                                    d[16 + i] = pack16(__uint_as_float(r1[2 * i + 1]), __uint_as_float(r1[2 * i + 2]), p.dtype);
+                                srow[m_r + 63] = cast16(__uint_as_float(r1[31]), p.dtype);
+                            } else {
+                                srow[m_r + 31] = cast16(__uint_as_float(r0[31]), p.dtype);
+                            }
                         }
-                    }
-                    __syncwarp();                                    // every row of the warp is staged
-                    // 32 rows x 9 aligned chunks: lane + 32*it = 9*rr + qc
-                    int rr = lane / 9, qc = lane - 9 * rr;
-                    const uint8_t* stg_warp = stage_out + (warp - 2) * (32 * kUmmaStageRowBytes);
+                        if (warp == 2 && lane == 0) ADAPT_TRACE(9, unit);
+                        // staged row now holds valid elements [lo_valid, end): the carried tail makes the
+                        // head whole in every pass but the first
+                        const int lo_valid = pass == 0 ? m_r : 0;
+                        const int end = m_r + ncols;
+                        const uintptr_t g0 = g_row + 2u * c0;            // address of staged element m_r
+                        if (row_ok) {                                    // ragged ends of this thread's own row
+                            unsigned short* grow = reinterpret_cast<unsigned short*>(g0 - 2 * m_r);   // 16-byte aligned
+                            if (lo_valid) {
 #pragma unroll
-                    for (int it = 0; it < 9; ++it) {
-                        const uintptr_t g = g_pass + (uintptr_t)rr * row_bytes;
-                        const int m = (int)((g & 15u) >> 1);
-                        if (rowq0 + rr < p.M && 8 * qc >= m && 8 * qc + 8 <= m + ncols)
-                            *reinterpret_cast<uint4*>(g - 2 * m + 16 * qc) =
-                                *reinterpret_cast<const uint4*>(stg_warp + rr * kUmmaStageRowBytes + 16 * qc);
-                        rr += 3; qc += 5;
-                        if (qc >= 9) { qc -= 9; rr += 1; }
+                                for (int i = 0; i < 7; ++i)
+                                    if (lo_valid + i < min(8, end)) grow[lo_valid + i] = srow[lo_valid + i];
+                            }
+                            if (last && (end & 7)) {
+                                const int tail_begin = max(end & ~7, lo_valid ? min(8, end) : 0);
+#pragma unroll
+                                for (int i = 0; i < 7; ++i)
+                                    if (tail_begin + i < end) grow[tail_begin + i] = srow[tail_begin + i];
+                            }
+                        }
+                        __syncwarp();                                    // every row of the warp is staged
+                        // 32 rows x 9 aligned chunks: lane + 32*it = 9*rr + qc
+                        int rr = lane / 9, qc = lane - 9 * rr;
+                        const uint8_t* stg_warp = stage_out + (warp - 2) * (32 * kUmmaStageRowBytes);
+                        const uintptr_t g_pass = g_tile + 2u * c0;
+#pragma unroll
+                        for (int it = 0; it < 9; ++it) {
+                            const uintptr_t g = g_pass + (uintptr_t)rr * row_bytes;
+                            const int m = (int)((g & 15u) >> 1);
+                            const int lo_v = pass == 0 ? m : 0;
+                            if (rowq0 + rr < p.M && 8 * qc >= lo_v && 8 * qc + 8 <= m + ncols)
+                                *reinterpret_cast<uint4*>(g - 2 * m + 16 * qc) =
+                                    *reinterpret_cast<const uint4*>(stg_warp + rr * kUmmaStageRowBytes + 16 * qc);
+                            rr += 3; qc += 5;
+                            if (qc >= 9) { qc -= 9; rr += 1; }
+                        }
+                        if (warp == 2 && lane == 0) ADAPT_TRACE(6, unit);
                     }
-                    if (warp == 2 && lane == 0) ADAPT_TRACE(6, unit);
                 }
             } else {
                 // fp32 partial tile: rows of the workspace are 16-byte aligned (pitch Np), so a thread
