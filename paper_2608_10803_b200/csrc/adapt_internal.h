@@ -22,19 +22,25 @@ struct Machine {
 // Measured on B200 with this library's own kernels (CUDA events); the paper's values are for
 // other hardware and are not printed, so these are this library's.
 struct Calib {
-    double launch_us = 2.2;             // one kernel launch on a busy stream (T_pro/T_epi launches too)
+    double launch_us = 3.0;             // one kernel launch issued back to back on a stream (also per pad / reduce launch)
     double hbm_bw = 6.2e12;             // B/s, large streaming transfers
-    double hbm_ramp_bytes = 24e6;       // bytes at which half of hbm_bw is reached (latency + ramp)
-    double l2_bw_per_sm = 90e9;         // B/s one SM can pull through TMA from L2
-    double tensor_flops = 1.55e15;      // whole chip, kind::f16, BN = 256
-    double eta_mma_bn128 = 0.92;        // relative tensor efficiency at BN = 128
-    double eta_mma_bn64 = 0.62;         // ... at BN = 64 (A-operand smem reads dominate)
-    double eta_2cta = 1.0;              // 2-CTA pairs share B: no extra tensor cost
+    double l2_bw_per_sm = 100e9;        // B/s one SM pulls through TMA from L2 (8192^3, 128 x 256 tiles: 48 KB per 0.48 us)
+    double tensor_flops = 1.58e15;      // whole chip, kind::f16, BN = 256 (8192^3 on 256 x 256 pair tiles: 1.56e15)
+    double eta_mma_bn128 = 0.72;        // relative tensor efficiency at BN = 128 (0.29 us per 128 x 128 x 64 block)
+    double eta_mma_bn64 = 0.45;         // ... at BN = 64 (A-operand smem reads dominate)
+    double eta_2cta = 1.0;              // pair tiles share B: no extra tensor cost
     double mem_latency_us = 1.0;        // TMA issue -> data visible (sets Delta_dep with few stages)
-    double tile_epilogue_us_per_kb = 0.012; // drain: TMEM -> registers -> global, per KB of C tile
-    double simt_flops = 12e12;          // CUDA-core tile kernel
-    double skinny_bw_eff = 0.80;        // fraction of hbm_bw the streaming kernel reaches
-    double skinny_mac_rate = 30e12;     // MAC/s ceiling of the warp-level kernel (m padded to 16)
+    double umma_fixed_us = 2.5;         // barrier init, TMEM alloc, first load, last drain, TMEM free
+    // drain of one output tile through the epilogue warps (overlaps the next tile's main loop):
+    // fixed part per tile + part per KB written; rows of C that are not 16-byte aligned cost more
+    double epi_tile_fixed_us = 0.32, epi_us_per_kb = 0.0385;
+    double epi_tile_fixed_unaligned_us = 1.45, epi_us_per_kb_unaligned = 0.054;
+    double simt_flops = 15e12;          // CUDA-core tile kernel (1000^3: 17e12)
+    double simt_fixed_us = 1.5;
+    double skinny_bw_eff_aligned = 0.45;    // fraction of hbm_bw the warp-level streaming kernel reaches, 16-byte aligned rows
+    double skinny_bw_eff_unaligned = 0.14;  // ... rows assembled from two chunks
+    double skinny_fixed_us = 2.0;
+    double skinny_mac_rate = 30e12;     // MAC/s ceiling of the warp-level kernel (small side padded to 16)
     double copy_bw_eff = 0.85;          // pad-copy and reduce kernels
 };
 

@@ -185,21 +185,26 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     double eta = c.BN >= 256 ? 1.0 : (c.BN >= 128 ? cal.eta_mma_bn128 : cal.eta_mma_bn64);
     if (c.cluster == 2) eta *= cal.eta_2cta;
     const double tP = 2.0 * 128.0 * c.BN * c.BK / (cal.tensor_flops / m.n_sm * eta) * 1e6;
+    // Drain of one tile (the paper's T_drain: FixPipe cast and write).  With two or more TMEM
+    // accumulators it overlaps the next tile's main loop, so a tile costs max(L * II, T_drain).
+    const bool c_aligned = s.N % 8 == 0;
+    const double out_tile_kb = (c.P_k > 1 ? 4.0 : 2.0) * 128.0 * c.BN / 1024.0;
+    const double t_drain = (c.P_k > 1 || c_aligned)
+                               ? cal.epi_tile_fixed_us + cal.epi_us_per_kb * out_tile_kb
+                               : cal.epi_tile_fixed_unaligned_us + cal.epi_us_per_kb_unaligned * out_tile_kb;
     // Delta_dep (Eq. 9): with S stages only S-1 loads are in flight while one is consumed, so a
     // slice cannot issue faster than latency / (S-1); one stage serialises load and compute.
     double pipe;
-    const double out_tile_kb = (c.P_k > 1 ? 4.0 : 2.0) * 128.0 * c.BN / 1024.0;
-    const double t_epi_tile = out_tile_kb * cal.tile_epilogue_us_per_kb;
     if (c.stages <= 1) {
-        pipe = pipeline_time(0, Q, L, tM + cal.mem_latency_us, tP, t_epi_tile);
+        pipe = pipeline_time(0, Q, L, tM + cal.mem_latency_us, tP, t_drain);                  // Eq. 12
     } else {
         tM = std::max(tM, cal.mem_latency_us / (c.stages - 1));
         const double ii = std::max(tM, tP);
-        // two TMEM accumulators: a tile's drain overlaps the next tile's main loop
-        const double exposed = std::max(0.0, t_epi_tile - (double)L * ii);
-        if (c.persistent) pipe = cal.mem_latency_us + pipeline_time(2, Q, L, tM, tP, exposed) + t_epi_tile;
-        else pipe = cal.mem_latency_us + pipeline_time(1, Q, L, tM, tP, t_epi_tile);
+        const double t_tile = std::max((double)L * ii, t_drain);
+        // Eq. 14 with the drain overlapped: one fill, Q tiles back to back, the last drain exposed
+        pipe = tM + (double)Q * t_tile + tP + t_drain;
     }
+    pipe += cal.umma_fixed_us;
     model_prologue(s, c, cal);
     model_epilogue(s, c, cal);
     const double t_hbm = c.hbm_bytes / cal.hbm_bw * 1e6 - c.t_pro_us - c.t_epi_us;
@@ -215,13 +220,18 @@ static void model_skinny(const Shape& s, const Machine& m, const Calib& cal, Con
     c.grid = (int)units;
     const int64_t Q = ceil_div(units, (int64_t)m.n_sm * 2);      // two CTAs resident per SM
     const double macs = (double)std::max(s.M, s.N) * s.K * 16.0;  // the small side is padded to 16
+    // the streamed operand: B when M is the small side, else A; its rows are aligned when the
+    // contiguous extent is a multiple of 8 elements
+    const bool stream_is_B = s.M <= 16 && (s.M <= s.N || s.N > 16);
+    const int64_t inner = stream_is_B ? (s.layoutB == ADAPT_ROW_MAJOR ? s.N : s.K) : (s.layoutA == ADAPT_ROW_MAJOR ? s.K : s.M);
+    const double eff = inner % 8 == 0 ? cal.skinny_bw_eff_aligned : cal.skinny_bw_eff_unaligned;
+    // one CTA streams about hbm_bw * eff / (2 * n_sm) when the machine is full; fewer CTAs do not go faster
     const double per_cta_bytes = 2.0 * ((double)c.BN * ceil_div(s.K, c.P_k));
-    const double t_cta = per_cta_bytes / (cal.l2_bw_per_sm * 0.5) * 1e6 + cal.mem_latency_us;
+    const double t_cta = per_cta_bytes / (cal.hbm_bw * eff / (2.0 * m.n_sm)) * 1e6;
     model_epilogue(s, c, cal);
-    const double t_stream = c.hbm_bytes / (cal.hbm_bw * cal.skinny_bw_eff) * 1e6 - c.t_epi_us;
     const double t_alu = macs / cal.skinny_mac_rate * 1e6;
     c.t_pro_us = 0;
-    c.t_main_us = std::max({t_stream, t_alu, (double)Q * t_cta});
+    c.t_main_us = cal.skinny_fixed_us + std::max(t_alu, (double)Q * t_cta);
     finish_common(s, c, cal);
 }
 
@@ -235,7 +245,7 @@ static void model_simt(const Shape& s, const Machine& m, const Calib& cal, Confi
     const int64_t Q = ceil_div(units, resident);
     // a full 64x64 tile costs the same whether or not the shape fills it
     const double tile_flops = 2.0 * c.BM * c.BN * (double)ceil_div(s.K, c.P_k);
-    const double t_tile = tile_flops / (cal.simt_flops / resident) * 1e6 + cal.mem_latency_us;
+    const double t_tile = tile_flops / (cal.simt_flops / resident) * 1e6 + cal.simt_fixed_us;
     model_epilogue(s, c, cal);
     const double t_hbm = c.hbm_bytes / (cal.hbm_bw * 0.6) * 1e6 - c.t_epi_us;
     c.t_pro_us = 0;
