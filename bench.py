@@ -288,7 +288,7 @@ def ours(args):
 
     # ---- per-shape timing: R back-to-back calls between two events, rotating buffer sets ----
     per_shape = None
-    if rank == 0 or True:
+    if args.shape_passes > 0:
         reps = []
         for info, c in zip(infos, cases):
             reps.append(int(min(20, max(1, 60.0 / max(info.predicted_us, 1.0)))))
@@ -467,6 +467,55 @@ def e2e(args, cases, plans, pools, stream, world, dist):
             "api": "adapt_matmul_host (pinned host operands; H2D of A and B, kernels, D2H of C inside the timed region)"}
 
 
+def one_shape(args):
+    """Time a single GEMM shape (used for profiler captures and quick checks): prints one line."""
+    import torch
+    from paper_2608_10803_b200 import binding as ab
+    from paper_2608_10803_b200 import synth
+    M, N, K, dt = (int(x) for x in args.shape.split(","))
+    ab.adapt_init(0)
+    A = synth.draw_operand(M, K, synth.U11, 1, dt, "cuda")
+    B = synth.draw_operand(K, N, synth.U11, 2, dt, "cuda")
+    C = torch.empty((M, N), dtype=A.dtype, device="cuda")
+    if args.family >= 0:
+        cands = [c for c in ab.adapt_plan_candidates(M, N, K, dt) if c.family == args.family]
+        if args.bn:
+            cands = [c for c in cands if c.BN == args.bn]
+        if args.pk:
+            cands = [c for c in cands if c.P_k == args.pk]
+        plan = ab.adapt_matmul_plan_forced(M, N, K, dt, 0, 0, cands[0].tiling_key)
+    else:
+        plan = ab.adapt_matmul_plan(M, N, K, dt)
+    info = ab.adapt_plan_info(plan)
+    st = torch.cuda.current_stream().cuda_stream
+    ab.adapt_matmul(plan, A.data_ptr(), B.data_ptr(), C.data_ptr(), st)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.reps):
+        ab.adapt_matmul(plan, A.data_ptr(), B.data_ptr(), C.data_ptr(), st)
+    e1.record()
+    torch.cuda.synchronize()
+    ab.adapt_poll_device_status(st)
+    t = e0.elapsed_time(e1) / args.reps * 1e-3
+    byts = 2.0 * (M * K + K * N + M * N)
+    line = (f"{M}x{N}x{K} dt{dt} {ab.FAMILY_NAMES[info.family]} {info.BM}x{info.BN} st{info.stages} P_k{info.P_k} "
+            f"src{info.srcA}{info.srcB}: {t * 1e6:.1f} us  {2.0 * M * N * K / t / 1e12:.1f} TFLOP/s  {byts / t / 1e9:.0f} GB/s  "
+            f"predicted {info.predicted_us:.1f} us")
+    if args.cublas:
+        torch.matmul(A, B, out=C)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(args.reps):
+            torch.matmul(A, B, out=C)
+        e1.record()
+        torch.cuda.synchronize()
+        tc = e0.elapsed_time(e1) / args.reps * 1e-3
+        line += f"  | torch.matmul (cuBLAS, vendor reference) {tc * 1e6:.1f} us {2.0 * M * N * K / tc / 1e12:.1f} TFLOP/s"
+    print(line)
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -481,7 +530,15 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--dump", default="", help="write the per-shape table to this CSV")
+    ap.add_argument("--shape", default="", help="M,N,K,dtype: time this one shape only (dtype 0 = fp16, 1 = bf16)")
+    ap.add_argument("--reps", type=int, default=3)
+    ap.add_argument("--family", type=int, default=-1, help="with --shape: force a kernel family (0 umma_1cta, 1 umma_2cta, 2 skinny, 3 simt)")
+    ap.add_argument("--bn", type=int, default=0)
+    ap.add_argument("--pk", type=int, default=0)
+    ap.add_argument("--cublas", action="store_true", help="with --shape: also time torch.matmul as the vendor reference")
     args = ap.parse_args()
+    if args.shape:
+        return one_shape(args)
     if args.impl == "reference":
         return reference_arm(args)
     return ours(args)

@@ -37,6 +37,7 @@ struct Calib {
     double epi_tile_fixed_unaligned_us = 1.45, epi_us_per_kb_unaligned = 0.054;
     double simt_flops = 15e12;          // CUDA-core tile kernel (1000^3: 17e12)
     double simt_fixed_us = 1.5;
+    double simt_bw_eff = 0.15;          // fraction of hbm_bw its 2-byte accesses reach (K = 1 outer products: 0.13 measured)
     double skinny_bw_eff_aligned = 0.45;    // fraction of hbm_bw the warp-level streaming kernel reaches, 16-byte aligned rows
     double skinny_bw_eff_unaligned = 0.14;  // ... rows assembled from two chunks
     double skinny_fixed_us = 2.0;

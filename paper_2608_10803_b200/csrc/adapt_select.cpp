@@ -247,7 +247,8 @@ static void model_simt(const Shape& s, const Machine& m, const Calib& cal, Confi
     const double tile_flops = 2.0 * c.BM * c.BN * (double)ceil_div(s.K, c.P_k);
     const double t_tile = tile_flops / (cal.simt_flops / resident) * 1e6 + cal.simt_fixed_us;
     model_epilogue(s, c, cal);
-    const double t_hbm = c.hbm_bytes / (cal.hbm_bw * 0.6) * 1e6 - c.t_epi_us;
+    // element-wise 2-byte loads and stores: about a seventh of the HBM rate when memory-bound
+    const double t_hbm = c.hbm_bytes / (cal.hbm_bw * cal.simt_bw_eff) * 1e6 - c.t_epi_us;
     c.t_pro_us = 0;
     c.t_main_us = std::max((double)Q * t_tile, t_hbm);
     finish_common(s, c, cal);
