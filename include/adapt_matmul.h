@@ -70,7 +70,9 @@ typedef enum {
 typedef enum {
     ADAPT_SRC_TMA = 0,        /* TMA straight from the caller's buffer (needs 16 B pitch and base) */
     ADAPT_SRC_PAD_COPY = 1,   /* prologue kernel re-pitches the operand into the workspace, then TMA */
-    ADAPT_SRC_LSU = 2         /* ordinary loads (skinny / SIMT families) */
+    ADAPT_SRC_LSU = 2,        /* ordinary loads (skinny / SIMT families) */
+    ADAPT_SRC_TMA_CLASSES = 3 /* row-major A with K % 8 != 0 read in place: one TMA view per row class (row % 8),
+                                 tiles made of every 8th row; no copy, no workspace */
 } adapt_source_t;
 
 /* Everything the selector decided for one shape.  Filled by adapt_plan_info and

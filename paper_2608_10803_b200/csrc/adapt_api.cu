@@ -47,7 +47,8 @@ static adapt_status_t fail(adapt_status_t st, const char* fmt, const char* detai
 struct MapSlot {
     const void* ptr = nullptr;
     int64_t pitch = 0;
-    CUtensorMap map;
+    int count = 0;            // 1, or 8 for the per-row-class maps of A
+    CUtensorMap map[8];
 };
 
 struct adapt_plan_s {
@@ -349,17 +350,17 @@ extern "C" int64_t adapt_launch_count(void) { return st().launches.load(); }
 // ---------------------------------------------------------------------------------------------
 // launch_map: (family, BN, A major, B major) -> compiled kernel
 // ---------------------------------------------------------------------------------------------
-typedef void (*UmmaKernel)(const CUtensorMap, const CUtensorMap, const UmmaParams);
+typedef void (*UmmaKernel)(const TmapPack, const UmmaParams);
 
 template <int CG>
 static UmmaKernel umma_lookup(int BN, bool a_mn, bool b_mn)
 {
-#define ADAPT_PICK(bn)                                                        \
-    if (BN == bn) {                                                           \
-        if (!a_mn && !b_mn) return umma_gemm_kernel<bn, false, false, CG>;    \
-        if (!a_mn && b_mn) return umma_gemm_kernel<bn, false, true, CG>;      \
-        if (a_mn && !b_mn) return umma_gemm_kernel<bn, true, false, CG>;      \
-        return umma_gemm_kernel<bn, true, true, CG>;                          \
+#define ADAPT_PICK(bn)                                                               \
+    if (BN == bn) {                                                                  \
+        if (!a_mn && !b_mn) return umma_gemm_kernel<bn, false, false, CG, false>;    \
+        if (!a_mn && b_mn) return umma_gemm_kernel<bn, false, true, CG, false>;      \
+        if (a_mn && !b_mn) return umma_gemm_kernel<bn, true, false, CG, false>;      \
+        return umma_gemm_kernel<bn, true, true, CG, false>;                          \
     }
     if constexpr (CG == 1) { ADAPT_PICK(64) }
     ADAPT_PICK(128)
@@ -368,8 +369,14 @@ static UmmaKernel umma_lookup(int BN, bool a_mn, bool b_mn)
     return nullptr;
 }
 
-static UmmaKernel launch_map_umma(int family, int BN, bool a_mn, bool b_mn)
+static UmmaKernel launch_map_umma(int family, int BN, bool a_mn, bool b_mn, bool a_classes = false)
 {
+    if (a_classes) {                     // row-major A read through per-row-class maps (1-CTA tiles, row-major B)
+        if (BN == 64) return umma_gemm_kernel<64, false, true, 1, true>;
+        if (BN == 128) return umma_gemm_kernel<128, false, true, 1, true>;
+        if (BN == 256) return umma_gemm_kernel<256, false, true, 1, true>;
+        return nullptr;
+    }
     return family == ADAPT_FAM_UMMA_1CTA ? umma_lookup<1>(BN, a_mn, b_mn) : umma_lookup<2>(BN, a_mn, b_mn);
 }
 
@@ -409,6 +416,9 @@ extern "C" adapt_status_t adapt_init(int device)
                     if (!k) continue;
                     CUDA_TRY(cudaFuncSetAttribute((const void*)k, cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
                 }
+    for (int BN : {64, 128, 256})
+        CUDA_TRY(cudaFuncSetAttribute((const void*)launch_map_umma(ADAPT_FAM_UMMA_1CTA, BN, false, true, true),
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
     S.device = device;
     S.inited = true;
     return ADAPT_OK;
@@ -511,15 +521,42 @@ adapt_status_t cached_map(State& S, Plan* pl, bool isA, const void* base, int64_
     std::lock_guard<std::mutex> lock(pl->mu);
     MapSlot* slots = isA ? pl->mapA : pl->mapB;
     for (int i = 0; i < 2; ++i)
-        if (slots[i].ptr == base && slots[i].pitch == pitch) { *out = slots[i].map; return ADAPT_OK; }
+        if (slots[i].ptr == base && slots[i].pitch == pitch && slots[i].count == 1) { *out = slots[i].map[0]; return ADAPT_OK; }
     int& next = isA ? pl->nextA : pl->nextB;
     MapSlot& sl = slots[next];
     next ^= 1;
-    adapt_status_t r = encode_map(S, &sl.map, base, pl->s.dtype, inner, outer, pitch, box_inner, box_outer);
+    adapt_status_t r = encode_map(S, &sl.map[0], base, pl->s.dtype, inner, outer, pitch, box_inner, box_outer);
     if (r != ADAPT_OK) { sl.ptr = nullptr; return r; }
     sl.ptr = base;
     sl.pitch = pitch;
-    *out = sl.map;
+    sl.count = 1;
+    *out = sl.map[0];
+    return ADAPT_OK;
+}
+
+// Eight maps of a row-major A (M x K, K % 8 != 0, 16-byte aligned base), one per row class j = row % 8:
+// base rounded down to 16 bytes, rows 16*K bytes apart, inner extent K + sigma_j so that the k tail is
+// zero-filled; sigma_j = elements between the rounded base and the start of row j.
+adapt_status_t cached_class_maps(State& S, Plan* pl, const void* A, int64_t M, int64_t K, CUtensorMap* out, int* sigma)
+{
+    std::lock_guard<std::mutex> lock(pl->mu);
+    for (int j = 0; j < 8; ++j) sigma[j] = (int)(((2 * j * K) & 15) / 2);
+    MapSlot* slots = pl->mapA;
+    for (int i = 0; i < 2; ++i)
+        if (slots[i].ptr == A && slots[i].count == 8) { memcpy(out, slots[i].map, 8 * sizeof(CUtensorMap)); return ADAPT_OK; }
+    MapSlot& sl = slots[pl->nextA];
+    pl->nextA ^= 1;
+    sl.ptr = nullptr;
+    for (int j = 0; j < 8; ++j) {
+        const uint8_t* base = (const uint8_t*)A + ((2 * j * K) & ~(int64_t)15);
+        const int64_t rows = std::max<int64_t>(1, ceil_div(M - j, 8));
+        adapt_status_t r = encode_map(S, &sl.map[j], base, pl->s.dtype, K + sigma[j], rows, 8 * K, 64, 128);
+        if (r != ADAPT_OK) return r;
+    }
+    sl.ptr = A;
+    sl.pitch = K;
+    sl.count = 8;
+    memcpy(out, sl.map, 8 * sizeof(CUtensorMap));
     return ADAPT_OK;
 }
 
@@ -552,7 +589,9 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     const bool b_mn = s.layoutB == ADAPT_ROW_MAJOR;       // N contiguous
     const int64_t inA = a_mn ? s.M : s.K, outA = a_mn ? s.K : s.M;
     const int64_t inB = b_mn ? s.N : s.K, outB = b_mn ? s.K : s.N;
-    const bool padA = c.srcA == ADAPT_SRC_PAD_COPY || ((uintptr_t)A & 15) != 0;
+    // the copy-free class mode needs a 16-byte aligned A; otherwise fall back to the re-pitched copy
+    const bool classesA = c.srcA == ADAPT_SRC_TMA_CLASSES && ((uintptr_t)A & 15) == 0;
+    const bool padA = !classesA && (c.srcA != ADAPT_SRC_TMA || ((uintptr_t)A & 15) != 0);
     const bool padB = c.srcB == ADAPT_SRC_PAD_COPY || ((uintptr_t)B & 15) != 0;
     const int64_t pitchA = padA ? padded_pitch(inA) : inA;
     const int64_t pitchB = padB ? padded_pitch(inB) : inB;
@@ -576,17 +615,24 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     float* partial = c.P_k > 1 ? (float*)(w8 + szA + szB) : nullptr;
 
     const int cg = c.cluster;
-    CUtensorMap tmA, tmB;
-    // K-major operand: one box of 64 k x (rows this CTA owns); MN-major operand: boxes of 64 x 64
-    if ((r = cached_map(S, pl, true, a_src, inA, outA, pitchA, 64, a_mn ? 64 : 128, &tmA)) != ADAPT_OK) return r;
-    if ((r = cached_map(S, pl, false, b_src, inB, outB, pitchB, 64, b_mn ? 64 : c.BN / cg, &tmB)) != ADAPT_OK) return r;
-
+    TmapPack maps;
     UmmaParams p;
+    memset(p.a_sigma, 0, sizeof(p.a_sigma));
+    // K-major operand: one box of 64 k x (rows this CTA owns); MN-major operand: boxes of 64 x 64
+    if (classesA) {
+        if ((r = cached_class_maps(S, pl, A, s.M, s.K, maps.a, p.a_sigma)) != ADAPT_OK) return r;
+    } else {
+        if ((r = cached_map(S, pl, true, a_src, inA, outA, pitchA, 64, a_mn ? 64 : 128, &maps.a[0])) != ADAPT_OK) return r;
+    }
+    if ((r = cached_map(S, pl, false, b_src, inB, outB, pitchB, 64, b_mn ? 64 : c.BN / cg, &maps.b)) != ADAPT_OK) return r;
+
     p.M = (int)s.M; p.N = (int)s.N; p.K = (int)s.K;
-    p.P_m = c.P_m; p.P_n = c.P_n; p.P_k = c.P_k;
-    p.kb_total = (int)ceil_div(s.K, kUmmaBK);
+    // a plan made for class tiles that has to fall back to the copy (unaligned A pointer) uses plain tiles
+    p.P_m = (c.srcA == ADAPT_SRC_TMA_CLASSES && !classesA) ? (int)ceil_div(s.M, c.BM) : c.P_m;
+    p.P_n = c.P_n; p.P_k = c.P_k;
+    p.kb_total = (int)ceil_div(s.K + (classesA ? 7 : 0), kUmmaBK);
     p.kb_per_split = (int)ceil_div(p.kb_total, c.P_k);
-    p.num_units = c.P_m * c.P_n * c.P_k;
+    p.num_units = p.P_m * c.P_n * c.P_k;
     p.dtype = s.dtype;
     p.stages = c.stages;
     p.idesc = umma_idesc(s.dtype, a_mn, b_mn, 128 * cg, c.BN);
@@ -599,7 +645,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.trace = S.d_trace;
 #endif
 
-    UmmaKernel k = launch_map_umma(c.family, c.BN, a_mn, b_mn);
+    UmmaKernel k = launch_map_umma(c.family, c.BN, a_mn, b_mn, classesA);
     if (!k) return fail(ADAPT_ERR_UNSUPPORTED, "no compiled kernel for this tiling key%s");
     const int slots = S.machine.n_sm / cg;
     const int grid = std::min(p.num_units, slots) * cg;
@@ -616,7 +662,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, k, tmA, tmB, p));
+    CUDA_TRY(cudaLaunchKernelEx(&cfg, k, maps, p));
     S.launches.fetch_add(1, std::memory_order_relaxed);
     if (c.P_k > 1) return launch_reduce(S, partial, C, s.M, s.N, c.P_k, s.dtype, stream);
     return ADAPT_OK;

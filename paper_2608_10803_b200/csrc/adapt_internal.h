@@ -43,6 +43,7 @@ struct Calib {
     double skinny_fixed_us = 2.0;
     double skinny_mac_rate = 30e12;     // MAC/s ceiling of the warp-level kernel (small side padded to 16)
     double copy_bw_eff = 0.85;          // pad-copy and reduce kernels
+    double class_view_bw_eff = 0.65;    // HBM rate through the per-row-class TMA views of an unaligned A
 };
 
 // ---- one configuration x of the search set S(b(s)) (Eq. 6) ------------------------------------

@@ -161,7 +161,7 @@ static void model_epilogue(const Shape& s, Config& c, const Calib& cal)
 
 static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Config& c)
 {
-    const int64_t kblocks = ceil_div(s.K, c.BK);
+    const int64_t kblocks = ceil_div(s.K + (c.srcA == ADAPT_SRC_TMA_CLASSES ? 7 : 0), c.BK);
     const int64_t L = ceil_div(kblocks, c.P_k);
     const int64_t units = (int64_t)c.P_m * c.P_n * c.P_k;
     const int64_t slots = m.n_sm / c.cluster;
@@ -207,7 +207,9 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     pipe += cal.umma_fixed_us;
     model_prologue(s, c, cal);
     model_epilogue(s, c, cal);
-    const double t_hbm = c.hbm_bytes / cal.hbm_bw * 1e6 - c.t_pro_us - c.t_epi_us;
+    // strided row-class views stream A at a lower rate than a dense tensor (measured 3.5-4.1 TB/s)
+    const double bw = c.srcA == ADAPT_SRC_TMA_CLASSES ? cal.hbm_bw * cal.class_view_bw_eff : cal.hbm_bw;
+    const double t_hbm = c.hbm_bytes / bw * 1e6 - c.t_pro_us - c.t_epi_us;
     c.t_main_us = std::max(pipe, t_hbm);
     finish_common(s, c, cal);
 }
@@ -274,16 +276,23 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     if (c.stages < 1 || c.stages > 12) return false;
     c.smem_bytes = umma_smem_bytes(c.BN, c.cluster, c.stages);
     if (c.smem_bytes > m.smem_bytes) return false;
-    const int64_t kblocks = ceil_div(s.K, c.BK);
+    // in class mode the k index of a tile is shifted by up to 7 elements
+    const int64_t kblocks = ceil_div(s.K + (c.srcA == ADAPT_SRC_TMA_CLASSES ? 7 : 0), c.BK);
     if (c.P_k < 1 || c.P_k > 1023 || c.P_k > kblocks) return false;
     if (ceil_div(kblocks, ceil_div(kblocks, c.P_k)) != c.P_k) return false;   // no empty split
     // operand sources: TMA needs a 16-byte row pitch
     if (c.srcA == ADAPT_SRC_TMA && !aligned16(innerA(s))) return false;
     if (c.srcB == ADAPT_SRC_TMA && !aligned16(innerB(s))) return false;
-    if (c.srcA == ADAPT_SRC_LSU || c.srcB == ADAPT_SRC_LSU) return false;
+    if (c.srcA == ADAPT_SRC_LSU || c.srcB == ADAPT_SRC_LSU || c.srcB == ADAPT_SRC_TMA_CLASSES) return false;
+    const bool classes = c.srcA == ADAPT_SRC_TMA_CLASSES;
+    if (classes) {
+        // rows of one residue class share their misalignment: row-major A and B, one CTA per tile
+        if (c.family != ADAPT_FAM_UMMA_1CTA || s.layoutA != ADAPT_ROW_MAJOR || s.layoutB != ADAPT_ROW_MAJOR) return false;
+        if (aligned16(innerA(s)) || s.M < 8) return false;
+    }
     if (c.srcA == ADAPT_SRC_PAD_COPY && aligned16(innerA(s))) return false;    // nothing to pad
     if (c.srcB == ADAPT_SRC_PAD_COPY && aligned16(innerB(s))) return false;
-    c.P_m = (int)ceil_div(s.M, c.BM);
+    c.P_m = classes ? (int)(8 * ceil_div(s.M, 8 * c.BM)) : (int)ceil_div(s.M, c.BM);   // class tiles: 8 per 1024 rows
     c.P_n = (int)ceil_div(s.N, c.BN);
     if ((int64_t)c.P_m * c.P_n * c.P_k > (int64_t)1 << 30) return false;
     c.persistent = 1;
@@ -409,6 +418,12 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
                     c.family = fam; c.BM = BM; c.BN = BN; c.BK = 64; c.cluster = cluster;
                     c.stages = st; c.P_k = pk; c.srcA = srcA; c.srcB = srcB;
                     if (finalize(s, m, cal, c)) out->push_back(c);
+                    if (srcA == ADAPT_SRC_PAD_COPY && st == deepest) {        // the copy-free alternative for A
+                        Config d;
+                        d.family = fam; d.BM = BM; d.BN = BN; d.BK = 64; d.cluster = cluster;
+                        d.stages = st; d.P_k = pk; d.srcA = ADAPT_SRC_TMA_CLASSES; d.srcB = srcB;
+                        if (finalize(s, m, cal, d)) out->push_back(d);
+                    }
                 }
             }
         }

@@ -39,6 +39,7 @@ struct UmmaParams {
     void* C;                         // 16-bit output, row-major M x N (used when P_k == 1)
     float* partial;                  // fp32 [P_k][M][Np], Np = N rounded up to 4 (used when P_k > 1)
     int Np;                          // row pitch of the partials in elements
+    int a_sigma[8];                  // class mode: shift (elements) of row class j = row % 8 against its 16-byte aligned base
     unsigned int* status;            // device status word: bit 0 = a bounded wait expired
     unsigned long long* trace;       // timestamp trace of CTA 0 (diagnostic builds only), else null
 };
@@ -54,6 +55,13 @@ struct UmmaParams {
 #else
 #define ADAPT_TRACE(ev, unit) do { } while (0)
 #endif
+
+// Tensor maps of one launch.  a[0] is the map of A; in class mode (A_CLS) a[j] is the map of the
+// rows of A with row % 8 == j (see the kernel comment).
+struct TmapPack {
+    CUtensorMap a[8];
+    CUtensorMap b;
+};
 
 // unit index -> (m block, n block, split).  Units of one output tile are adjacent in split;
 // tiles are visited in groups of kGroupM m-blocks so that concurrently running CTAs share B
@@ -87,10 +95,21 @@ __device__ __forceinline__ unsigned short cast16(float a, int dtype)
     return *reinterpret_cast<unsigned short*>(&h);
 }
 
-template <int BN, bool A_MN, bool B_MN, int CG>
+// A_CLS ("row classes", the Padding module without a copy): A is row-major with K % 8 != 0, so its
+// rows are not 16-byte aligned and one tensor map cannot describe it.  Rows r and r + 8 do start
+// at the same offset from a 16-byte boundary (their distance is 16*K bytes), so the rows of one
+// residue class j = r % 8 form a tensor TMA can read: base rounded down to 16 bytes, row pitch
+// 16*K bytes, every row shifted by the same sigma_j elements.  An m-tile then takes 128 rows of
+// ONE class (rows 1024*g + j + 8*i), its k index runs over kappa = k + sigma_j, and B's k-rows
+// (an outer TMA coordinate, free of alignment rules) start at kappa - sigma_j; rows of B' with
+// kappa < sigma_j or k >= K are out of bounds and read as zero.  The sigma_j leading elements of
+// each A' row belong to the previous row of A: the MMA warp overwrites them with zeros in the
+// first k-block before the tensor core reads them.
+template <int BN, bool A_MN, bool B_MN, int CG, bool A_CLS>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
-umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const UmmaParams p)
+umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
 {
+    static_assert(!A_CLS || (!A_MN && B_MN && CG == 1), "class mode: row-major A and B, one CTA per tile");
     constexpr int BN_CTA = BN / CG;                       // B columns this CTA loads
     constexpr int A_BYTES = 128 * kUmmaBK * 2;
     constexpr int B_BYTES = BN_CTA * kUmmaBK * 2;
@@ -135,8 +154,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
-        ptx::prefetch_tensormap(&tmA);
-        ptx::prefetch_tensormap(&tmB);
+        ptx::prefetch_tensormap(&maps.a[0]);
+        ptx::prefetch_tensormap(&maps.b);
     }
     if (warp == 1) {
         ptx::tmem_alloc<CG>(tmem_slot, TMEM_COLS);
@@ -168,7 +187,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 decode_unit(p, unit, mb, nb, split);
                 const int kb0 = split * p.kb_per_split;
                 const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
-                const int row0 = mb * (128 * CG) + (int)cta_rank * 128;       // this CTA's A rows
+                // A rows of this CTA: consecutive rows, or in class mode rows 1024*g + j + 8*i read through
+                // map j at class-row index 128*g
+                const int cls = A_CLS ? (mb & 7) : 0;
+                const int row0 = A_CLS ? (mb >> 3) * 128 : mb * (128 * CG) + (int)cta_rank * 128;
+                const int kshift = A_CLS ? p.a_sigma[cls] : 0;                // B's k-rows lag A's kappa by sigma
+                const CUtensorMap* tmA = &maps.a[cls];
+                const CUtensorMap* tmB = &maps.b;
                 const int col0 = nb * BN + (int)cta_rank * BN_CTA;            // this CTA's B columns
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (!ptx::mbar_wait(empty_bar + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
@@ -179,24 +204,24 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                     else if (leader) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, 2 * STAGE_BYTES);
                     const int k0 = kb * kUmmaBK;
                     if (!A_MN) {
-                        if (CG == 1) ptx::tma_load_2d(sA, &tmA, fb, k0, row0);
-                        else ptx::tma_load_2d_pair(sA, &tmA, fb, k0, row0);
+                        if (CG == 1) ptx::tma_load_2d(sA, tmA, fb, k0, row0);
+                        else ptx::tma_load_2d_pair(sA, tmA, fb, k0, row0);
                     } else {
 #pragma unroll
                         for (int j = 0; j < 2; ++j) {
-                            if (CG == 1) ptx::tma_load_2d(sA + j * 8192, &tmA, fb, row0 + j * 64, k0);
-                            else ptx::tma_load_2d_pair(sA + j * 8192, &tmA, fb, row0 + j * 64, k0);
+                            if (CG == 1) ptx::tma_load_2d(sA + j * 8192, tmA, fb, row0 + j * 64, k0);
+                            else ptx::tma_load_2d_pair(sA + j * 8192, tmA, fb, row0 + j * 64, k0);
                         }
                     }
                     if (B_MN) {
 #pragma unroll
                         for (int j = 0; j < BN_CTA / 64; ++j) {
-                            if (CG == 1) ptx::tma_load_2d(sB + j * 8192, &tmB, fb, col0 + j * 64, k0);
-                            else ptx::tma_load_2d_pair(sB + j * 8192, &tmB, fb, col0 + j * 64, k0);
+                            if (CG == 1) ptx::tma_load_2d(sB + j * 8192, tmB, fb, col0 + j * 64, k0 - kshift);
+                            else ptx::tma_load_2d_pair(sB + j * 8192, tmB, fb, col0 + j * 64, k0 - kshift);
                         }
                     } else {
-                        if (CG == 1) ptx::tma_load_2d(sB, &tmB, fb, k0, col0);
-                        else ptx::tma_load_2d_pair(sB, &tmB, fb, k0, col0);
+                        if (CG == 1) ptx::tma_load_2d(sB, tmB, fb, k0, col0);
+                        else ptx::tma_load_2d_pair(sB, tmB, fb, k0, col0);
                     }
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
@@ -205,7 +230,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ---------------------------------------------
-        if (lane == 0 && leader) {
+        // one thread issues the MMAs; in class mode the whole warp runs the loop so that its other
+        // lanes can zero the stale leading elements of A' in the first k-block
+        if ((lane == 0 || A_CLS) && leader) {
             int stage = 0;
             uint32_t phase = 0;
             int buf = 0;
@@ -215,35 +242,62 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             // 1024 B apart (SBO), +2048 B per 16-element k step.
             const uint32_t a_lbo = A_MN ? 8192u : 16u, b_lbo = B_MN ? 8192u : 16u;
             const uint32_t a_kstep = A_MN ? 2048u : 32u, b_kstep = B_MN ? 2048u : 32u;
+            // in class mode all 32 lanes run this loop: lane 0 waits and the outcome is broadcast, so
+            // the lanes never part ways before a __syncwarp
+            auto mma_wait = [&](uint32_t bar, uint32_t parity) -> bool {
+                if (!A_CLS) return ptx::mbar_wait(bar, parity, abort_flag);
+                int w = 1;
+                if (lane == 0) w = ptx::mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+                return __shfl_sync(0xffffffffu, w, 0) != 0;
+            };
             bool ok = true;
             for (int unit = unit0; ok && unit < p.num_units; unit += unit_step) {
                 int mb, nb, split;
                 decode_unit(p, unit, mb, nb, split);
                 const int kb0 = split * p.kb_per_split;
                 const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
-                if (!ptx::mbar_wait(tempty_bar + 8u * buf, buf_phase ^ 1u, abort_flag)) { ok = false; break; }
+                if (!mma_wait(tempty_bar + 8u * buf, buf_phase ^ 1u)) { ok = false; break; }
                 ptx::tc_fence_after();
                 ADAPT_TRACE(2, unit);
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
                 for (int kb = kb0; kb < kb1; ++kb) {
-                    if (!ptx::mbar_wait(full_bar + 8u * stage, phase, abort_flag)) { ok = false; break; }
+                    if (!mma_wait(full_bar + 8u * stage, phase)) { ok = false; break; }
                     ptx::tc_fence_after();
                     const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
                     const uint32_t sB = sA + A_BYTES;
+                    if (A_CLS) {
+                        const int sigma = p.a_sigma[mb & 7];
+                        if (kb == 0 && sigma > 0) {
+                            // rows lane, lane+32, ...: chunk 0 of row r sits at r*128 + ((r & 7) << 4)
+                            uint8_t* genA = gen_base + (size_t)stage * STAGE_BYTES;
 #pragma unroll
-                    for (int k16 = 0; k16 < kUmmaBK / 16; ++k16) {
-                        const uint64_t adesc = ptx::smem_desc_sw128(sA + k16 * a_kstep, a_lbo, 1024u);
-                        const uint64_t bdesc = ptx::smem_desc_sw128(sB + k16 * b_kstep, b_lbo, 1024u);
-                        ptx::umma_f16<CG>(d_tmem, adesc, bdesc, p.idesc, (kb > kb0 || k16 > 0) ? 1u : 0u);
+                            for (int t = 0; t < 4; ++t) {
+                                const int r = lane + 32 * t;
+                                unsigned short* h = reinterpret_cast<unsigned short*>(genA + r * 128 + ((r & 7) << 4));
+                                for (int e = 0; e < sigma; ++e) h[e] = 0;
+                            }
+                            ptx::fence_proxy_async_smem();
+                        }
+                        __syncwarp();
                     }
-                    // free the stage (in both CTAs of a pair) once these MMAs have read it
-                    if (CG == 1) ptx::umma_commit_1(empty_bar + 8u * stage);
-                    else ptx::umma_commit_2(empty_bar + 8u * stage, 3);
+                    if (lane == 0) {
+#pragma unroll
+                        for (int k16 = 0; k16 < kUmmaBK / 16; ++k16) {
+                            const uint64_t adesc = ptx::smem_desc_sw128(sA + k16 * a_kstep, a_lbo, 1024u);
+                            const uint64_t bdesc = ptx::smem_desc_sw128(sB + k16 * b_kstep, b_lbo, 1024u);
+                            ptx::umma_f16<CG>(d_tmem, adesc, bdesc, p.idesc, (kb > kb0 || k16 > 0) ? 1u : 0u);
+                        }
+                        // free the stage (in both CTAs of a pair) once these MMAs have read it
+                        if (CG == 1) ptx::umma_commit_1(empty_bar + 8u * stage);
+                        else ptx::umma_commit_2(empty_bar + 8u * stage, 3);
+                    }
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
-                if (CG == 1) ptx::umma_commit_1(tfull_bar + 8u * buf);
-                else ptx::umma_commit_2(tfull_bar + 8u * buf, 3);
+                if (lane == 0) {
+                    if (CG == 1) ptx::umma_commit_1(tfull_bar + 8u * buf);
+                    else ptx::umma_commit_2(tfull_bar + 8u * buf, 3);
+                }
                 ADAPT_TRACE(3, unit);
                 if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
             }
@@ -267,7 +321,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             if (!ptx::mbar_wait(tfull_bar + 8u * buf, buf_phase, abort_flag)) { ok = false; break; }
             ptx::tc_fence_after();
             if (warp == 2 && lane == 0) ADAPT_TRACE(4, unit);
-            const int row = mb * (128 * CG) + (int)cta_rank * 128 + q * 32 + lane;
+            // row of C held by TMEM lane i of this CTA: consecutive rows, or every 8th row of one class
+            const int row_step = A_CLS ? 8 : 1;
+            const int row_base = A_CLS ? (mb >> 3) * 1024 + (mb & 7) : mb * (128 * CG) + (int)cta_rank * 128;
+            const int row = row_base + row_step * (q * 32 + lane);
             const int n0 = nb * BN;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
             const bool row_ok = row < p.M;
@@ -278,9 +335,9 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 // writes its 32 row segments cooperatively, consecutive lanes taking consecutive chunks
                 // of a row (aligned 16-byte stores, about 3.5 rows per instruction); the at most 7 + 7
                 // elements at a segment's ends are 2-byte stores by the row's own thread.
-                const int rowq0 = row - lane;                        // first row of this warp's quarter
+                const int rowq0 = row - row_step * lane;             // first row of this warp's quarter
                 const uintptr_t g_tile = c_base + 2ull * ((size_t)rowq0 * p.N + n0);
-                const uintptr_t row_bytes = 2ull * (uintptr_t)p.N;
+                const uintptr_t row_bytes = 2ull * (uintptr_t)p.N * row_step;   // distance between this warp's rows
                 // the two warps of a lane quarter take alternate tiles, so one thread sees all passes of
                 // its row and can carry the ragged tail of a pass into the head of the next one
                 if ((seq & 1) == half) {
@@ -357,7 +414,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                             const uintptr_t g = g_pass + (uintptr_t)rr * row_bytes;
                             const int m = (int)((g & 15u) >> 1);
                             const int lo_v = pass == 0 ? m : 0;
-                            if (rowq0 + rr < p.M && 8 * qc >= lo_v && 8 * qc + 8 <= m + ncols)
+                            if (rowq0 + row_step * rr < p.M && 8 * qc >= lo_v && 8 * qc + 8 <= m + ncols)
                                 *reinterpret_cast<uint4*>(g - 2 * m + 16 * qc) =
                                     *reinterpret_cast<const uint4*>(stg_warp + rr * kUmmaStageRowBytes + 16 * qc);
                             rr += 3; qc += 5;

@@ -213,3 +213,46 @@ def test_long_k_accumulation_error_stays_small():
             continue
         err, _, _, _ = check_case(M, N, K, dtype, A, B, plan=plan)
         assert err < 4e-3
+
+
+# ---- row-major A with K % 8 != 0 read in place through per-row-class TMA views --------------------
+
+def class_mode_variants(M, N, K, dtype, limit=6):
+    out = []
+    for c in ab.adapt_plan_candidates(M, N, K, dtype):
+        if c.srcA == 3 and len(out) < limit:
+            out.append((ab.adapt_matmul_plan_forced(M, N, K, dtype, ROW, ROW, c.tiling_key), c))
+    return out
+
+
+@pytest.mark.parametrize("dtype", [ab.F16, ab.BF16])
+@pytest.mark.parametrize("shape", [(131, 77, 259), (1030, 264, 331), (2500, 64, 1001), (8, 8, 9), (300, 520, 12),
+                                   (1024, 128, 4099), (77, 1000, 70), (4100, 16, 2047)])
+def test_row_class_views_bit_exact(shape, dtype):
+    M, N, K = shape
+    A = synth.position_coded(M, K, dtype, modulus=7, device="cuda")
+    B = synth.position_coded(K, N, dtype, modulus=5, device="cuda")
+    variants = class_mode_variants(M, N, K, dtype)
+    assert variants, "shape must offer the class-mode source for A"
+    for plan, c in variants:
+        check_case(M, N, K, dtype, A, B, plan=plan, exact=True)
+
+
+def test_row_class_views_do_not_leak_a_neighbouring_row():
+    """The elements in front of a class row's first element belong to the previous row of A; a
+    non-finite value there must not reach this row's result."""
+    M, N, K = 600, 136, 203
+    dtype = ab.F16
+    A = synth.position_coded(M, K, dtype, 7, "cuda")
+    B = synth.position_coded(K, N, dtype, 5, "cuda")
+    bad_rows = [4, 17, 300]
+    for r in bad_rows:
+        A[r, K - 1] = float("inf")            # the tail of row r precedes the head of row r + 1 in memory
+        A[r, K - 2] = float("nan")
+    keep = torch.tensor([i for i in range(M) if i not in bad_rows], device="cuda")
+    for plan, c in class_mode_variants(M, N, K, dtype):
+        C = run_library(A, B, M, N, K, dtype, plan=plan)
+        torch.cuda.synchronize()
+        assert torch.isfinite(C.index_select(0, keep)).all()
+        err, mism, n = compare_with_oracle(A, B, C, M, N, K, dtype, rows=keep.cpu().numpy())
+        assert mism == 0

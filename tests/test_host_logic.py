@@ -128,10 +128,12 @@ def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
                     smem = c.stages * (128 * 64 * 2 + bn_cta * 64 * 2)
                     assert smem <= 227 * 1024
                     assert 2 * c.BN <= 512 and c.BN % 16 == 0
-                    assert c.P_k <= -(-K // 64)
+                    assert c.P_k <= -(-(K + 7) // 64)
                     # unaligned operands are never handed to TMA directly (row-major: K for A, N for B)
                     if K % 8:
-                        assert c.srcA == 1
+                        assert c.srcA in (1, 3)      # re-pitched copy, or the per-row-class TMA views
+                    if c.srcA == 3:
+                        assert K % 8 and M >= 8 and c.family == ab.FAM_UMMA_1CTA and c.P_m == 8 * -(-M // 1024)
                     if N % 8:
                         assert c.srcB == 1
                 if c.family == ab.FAM_SKINNY:
