@@ -43,6 +43,7 @@ struct Calib {
     double skinny_fixed_us = 2.0;
     double skinny_mac_rate = 30e12;     // MAC/s ceiling of the warp-level kernel (small side padded to 16)
     double copy_bw_eff = 0.85;          // pad-copy and reduce kernels
+    double class_view_sm_eff = 0.7;     // per-SM rate through those views relative to l2_bw_per_sm (20000 x 8 x 60001 tail wave)
     double class_view_bw_eff = 0.65;    // HBM rate through the per-row-class TMA views of an unaligned A
 };
 

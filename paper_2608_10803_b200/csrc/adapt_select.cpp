@@ -181,7 +181,8 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     // per-SM stage: each CTA loads its 128 rows of A and its share of the BN columns of B
     const double bn_per_cta = (double)c.BN / c.cluster;
     const double stage_bytes = 2.0 * c.BK * (128.0 + bn_per_cta);
-    double tM = stage_bytes / cal.l2_bw_per_sm * 1e6;
+    // one SM pulls the strided row-class views at about half the rate of a dense tensor
+    double tM = stage_bytes / (cal.l2_bw_per_sm * (c.srcA == ADAPT_SRC_TMA_CLASSES ? cal.class_view_sm_eff : 1.0)) * 1e6;
     double eta = c.BN >= 256 ? 1.0 : (c.BN >= 128 ? cal.eta_mma_bn128 : cal.eta_mma_bn64);
     if (c.cluster == 2) eta *= cal.eta_2cta;
     const double tP = 2.0 * 128.0 * c.BN * c.BK / (cal.tensor_flops / m.n_sm * eta) * 1e6;
@@ -418,13 +419,24 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
                     c.family = fam; c.BM = BM; c.BN = BN; c.BK = 64; c.cluster = cluster;
                     c.stages = st; c.P_k = pk; c.srcA = srcA; c.srcB = srcB;
                     if (finalize(s, m, cal, c)) out->push_back(c);
-                    if (srcA == ADAPT_SRC_PAD_COPY && st == deepest) {        // the copy-free alternative for A
-                        Config d;
-                        d.family = fam; d.BM = BM; d.BN = BN; d.BK = 64; d.cluster = cluster;
-                        d.stages = st; d.P_k = pk; d.srcA = ADAPT_SRC_TMA_CLASSES; d.srcB = srcB;
-                        if (finalize(s, m, cal, d)) out->push_back(d);
-                    }
                 }
+            }
+        }
+    }
+    // --- tcgen05, A read in place through per-row-class views (row-major A, K % 8 != 0): 8 class
+    //     tiles per 1024 rows, so the split counts are drawn from that tile count ---
+    if (srcA == ADAPT_SRC_PAD_COPY && s.layoutA == ADAPT_ROW_MAJOR && s.layoutB == ADAPT_ROW_MAJOR && s.M >= 8) {
+        for (int BN : {64, 128, 256}) {
+            const int64_t tiles = 8 * ceil_div(s.M, 1024) * ceil_div(s.N, BN);
+            split_candidates(tiles, m.n_sm, ceil_div(s.K + 7, 64), 2, &pks);
+            int deepest = 0;
+            for (int st = 8; st >= 2; --st)
+                if (umma_smem_bytes(BN, 1, st) <= m.smem_bytes) { deepest = st; break; }
+            for (int pk : pks) {
+                Config d;
+                d.family = ADAPT_FAM_UMMA_1CTA; d.BM = 128; d.BN = BN; d.BK = 64; d.cluster = 1;
+                d.stages = deepest; d.P_k = pk; d.srcA = ADAPT_SRC_TMA_CLASSES; d.srcB = srcB;
+                if (deepest >= 2 && finalize(s, m, cal, d)) out->push_back(d);
             }
         }
     }

@@ -87,10 +87,16 @@ splitk_reduce_kernel(const float* __restrict__ partial, unsigned short* __restri
         const int m = (int)(i / groups);
         const int n = (int)(i - (int64_t)m * groups) * 4;
         const float* src = partial + (int64_t)m * Np + n;
-        float4 acc = __ldcs(reinterpret_cast<const float4*>(src));
-        for (int p = 1; p < P_k; ++p) {
-            const float4 v = __ldcs(reinterpret_cast<const float4*>(src + (int64_t)p * slab));
-            acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+        // loads are issued eight splits at a time; the additions stay in ascending split order
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int p0 = 0; p0 < P_k; p0 += 8) {
+            float4 v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (p0 + j < P_k) v[j] = __ldcs(reinterpret_cast<const float4*>(src + (int64_t)(p0 + j) * slab));
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (p0 + j < P_k) { acc.x += v[j].x; acc.y += v[j].y; acc.z += v[j].z; acc.w += v[j].w; }
         }
         unsigned short* dst = C + (int64_t)m * N + n;
         if (n + 4 <= N && (reinterpret_cast<uintptr_t>(dst) & 7) == 0) {
