@@ -181,8 +181,14 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     // per-SM stage: each CTA loads its 128 rows of A and its share of the BN columns of B
     const double bn_per_cta = (double)c.BN / c.cluster;
     const double stage_bytes = 2.0 * c.BK * (128.0 + bn_per_cta);
-    // one SM pulls the strided row-class views at about half the rate of a dense tensor
-    double tM = stage_bytes / (cal.l2_bw_per_sm * (c.srcA == ADAPT_SRC_TMA_CLASSES ? cal.class_view_sm_eff : 1.0)) * 1e6;
+    // One SM pulls operands that other SMs also use from L2 at l2_bw_per_sm (a little less through
+    // the strided row-class views); a stream that comes from HBM and is used once is bounded by the
+    // bytes one SM keeps in flight, about hbm_bw_per_sm.  The second case only shows in partial waves.
+    const double t_mma_all = 2.0 * (double)s.M * s.N * s.K / cal.tensor_flops;
+    const bool mem_bound = c.hbm_bytes / cal.hbm_bw > t_mma_all;
+    double sm_rate = cal.l2_bw_per_sm * (c.srcA == ADAPT_SRC_TMA_CLASSES ? cal.class_view_sm_eff : 1.0);
+    if (mem_bound && c.srcA == ADAPT_SRC_TMA_CLASSES) sm_rate = std::min(sm_rate, cal.hbm_bw_per_sm);   // measured for the views only
+    double tM = stage_bytes / sm_rate * 1e6;
     double eta = c.BN >= 256 ? 1.0 : (c.BN >= 128 ? cal.eta_mma_bn128 : cal.eta_mma_bn64);
     if (c.cluster == 2) eta *= cal.eta_2cta;
     const double tP = 2.0 * 128.0 * c.BN * c.BK / (cal.tensor_flops / m.n_sm * eta) * 1e6;
