@@ -537,7 +537,7 @@ adapt_status_t cached_map(State& S, Plan* pl, bool isA, const void* base, int64_
 // Eight maps of a row-major A (M x K, K % 8 != 0, 16-byte aligned base), one per row class j = row % 8:
 // base rounded down to 16 bytes, rows 16*K bytes apart, inner extent K + sigma_j so that the k tail is
 // zero-filled; sigma_j = elements between the rounded base and the start of row j.
-adapt_status_t cached_class_maps(State& S, Plan* pl, const void* A, int64_t M, int64_t K, CUtensorMap* out, int* sigma)
+adapt_status_t cached_class_maps(State& S, Plan* pl, const void* A, int64_t M, int64_t K, int box_rows, CUtensorMap* out, int* sigma)
 {
     std::lock_guard<std::mutex> lock(pl->mu);
     for (int j = 0; j < 8; ++j) sigma[j] = (int)(((2 * j * K) & 15) / 2);
@@ -550,7 +550,7 @@ adapt_status_t cached_class_maps(State& S, Plan* pl, const void* A, int64_t M, i
     for (int j = 0; j < 8; ++j) {
         const uint8_t* base = (const uint8_t*)A + ((2 * j * K) & ~(int64_t)15);
         const int64_t rows = std::max<int64_t>(1, ceil_div(M - j, 8));
-        adapt_status_t r = encode_map(S, &sl.map[j], base, pl->s.dtype, K + sigma[j], rows, 8 * K, 64, 128);
+        adapt_status_t r = encode_map(S, &sl.map[j], base, pl->s.dtype, K + sigma[j], rows, 8 * K, 64, box_rows);
         if (r != ADAPT_OK) return r;
     }
     sl.ptr = A;
@@ -617,12 +617,17 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     const int cg = c.cluster;
     TmapPack maps;
     UmmaParams p;
+    int a_box_rows = 128;
     memset(p.a_sigma, 0, sizeof(p.a_sigma));
     // K-major operand: one box of 64 k x (rows this CTA owns); MN-major operand: boxes of 64 x 64
     if (classesA) {
-        if ((r = cached_class_maps(S, pl, A, s.M, s.K, maps.a, p.a_sigma)) != ADAPT_OK) return r;
+        if (s.M < 1024) a_box_rows = (int)std::min<int64_t>(128, round_up(ceil_div(s.M, 8), 8));   // rows of the largest class
+        if ((r = cached_class_maps(S, pl, A, s.M, s.K, a_box_rows, maps.a, p.a_sigma)) != ADAPT_OK) return r;
     } else {
-        if ((r = cached_map(S, pl, true, a_src, inA, outA, pitchA, 64, a_mn ? 64 : 128, &maps.a[0])) != ADAPT_OK) return r;
+        // a K-major A of fewer than 128 rows is loaded with a box of just those rows (rounded up to 8):
+        // the rows of the stage it leaves untouched only feed accumulator rows that are never stored
+        if (!a_mn && cg == 1 && s.M < 128) a_box_rows = (int)round_up(s.M, 8);
+        if ((r = cached_map(S, pl, true, a_src, inA, outA, pitchA, 64, a_mn ? 64 : a_box_rows, &maps.a[0])) != ADAPT_OK) return r;
     }
     if ((r = cached_map(S, pl, false, b_src, inB, outB, pitchB, 64, b_mn ? 64 : c.BN / cg, &maps.b)) != ADAPT_OK) return r;
 
@@ -635,6 +640,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.num_units = p.P_m * c.P_n * c.P_k;
     p.dtype = s.dtype;
     p.stages = c.stages;
+    p.a_tx_bytes = a_box_rows * kUmmaBK * 2;
     p.idesc = umma_idesc(s.dtype, a_mn, b_mn, 128 * cg, c.BN);
     p.C = C;
     p.partial = partial;

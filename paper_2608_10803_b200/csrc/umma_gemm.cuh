@@ -39,6 +39,7 @@ struct UmmaParams {
     void* C;                         // 16-bit output, row-major M x N (used when P_k == 1)
     float* partial;                  // fp32 [P_k][M][Np], Np = N rounded up to 4 (used when P_k > 1)
     int Np;                          // row pitch of the partials in elements
+    int a_tx_bytes;                  // bytes one TMA load of A delivers per stage and CTA (a short box when M < 128)
     int a_sigma[8];                  // class mode: shift (elements) of row class j = row % 8 against its 16-byte aligned base
     unsigned int* status;            // device status word: bit 0 = a bounded wait expired
     unsigned long long* trace;       // timestamp trace of CTA 0 (diagnostic builds only), else null
@@ -200,7 +201,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
                     const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
                     const uint32_t sB = sA + A_BYTES;
                     const uint32_t fb = full_target + 8u * stage;
-                    if (CG == 1) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, STAGE_BYTES);
+                    if (CG == 1) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(p.a_tx_bytes + B_BYTES));
                     else if (leader) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, 2 * STAGE_BYTES);
                     const int k0 = kb * kUmmaBK;
                     if (!A_MN) {
