@@ -357,10 +357,10 @@ static UmmaKernel umma_lookup(int BN, bool a_mn, bool b_mn)
 {
 #define ADAPT_PICK(bn)                                                               \
     if (BN == bn) {                                                                  \
-        if (!a_mn && !b_mn) return umma_gemm_kernel<bn, false, false, CG, false>;    \
-        if (!a_mn && b_mn) return umma_gemm_kernel<bn, false, true, CG, false>;      \
-        if (a_mn && !b_mn) return umma_gemm_kernel<bn, true, false, CG, false>;      \
-        return umma_gemm_kernel<bn, true, true, CG, false>;                          \
+        if (!a_mn && !b_mn) return umma_gemm_kernel<bn, false, false, CG, 0>;    \
+        if (!a_mn && b_mn) return umma_gemm_kernel<bn, false, true, CG, 0>;      \
+        if (a_mn && !b_mn) return umma_gemm_kernel<bn, true, false, CG, 0>;      \
+        return umma_gemm_kernel<bn, true, true, CG, 0>;                          \
     }
     if constexpr (CG == 1) { ADAPT_PICK(64) }
     ADAPT_PICK(128)
@@ -369,14 +369,15 @@ static UmmaKernel umma_lookup(int BN, bool a_mn, bool b_mn)
     return nullptr;
 }
 
-static UmmaKernel launch_map_umma(int family, int BN, bool a_mn, bool b_mn, bool a_classes = false)
+static UmmaKernel launch_map_umma(int family, int BN, bool a_mn, bool b_mn, int mode = 0)
 {
-    if (a_classes) {                     // row-major A read through per-row-class maps (1-CTA tiles, row-major B)
-        if (BN == 64) return umma_gemm_kernel<64, false, true, 1, true>;
-        if (BN == 128) return umma_gemm_kernel<128, false, true, 1, true>;
-        if (BN == 256) return umma_gemm_kernel<256, false, true, 1, true>;
+    if (mode == 1) {                     // row-major A read through per-row-class maps (1-CTA tiles, row-major B)
+        if (BN == 64) return umma_gemm_kernel<64, false, true, 1, 1>;
+        if (BN == 128) return umma_gemm_kernel<128, false, true, 1, 1>;
+        if (BN == 256) return umma_gemm_kernel<256, false, true, 1, 1>;
         return nullptr;
     }
+    if (mode == 2) return BN == 64 ? umma_gemm_kernel<64, false, true, 1, 2> : nullptr;   // B through per-k-class maps
     return family == ADAPT_FAM_UMMA_1CTA ? umma_lookup<1>(BN, a_mn, b_mn) : umma_lookup<2>(BN, a_mn, b_mn);
 }
 
@@ -417,8 +418,10 @@ extern "C" adapt_status_t adapt_init(int device)
                     CUDA_TRY(cudaFuncSetAttribute((const void*)k, cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
                 }
     for (int BN : {64, 128, 256})
-        CUDA_TRY(cudaFuncSetAttribute((const void*)launch_map_umma(ADAPT_FAM_UMMA_1CTA, BN, false, true, true),
+        CUDA_TRY(cudaFuncSetAttribute((const void*)launch_map_umma(ADAPT_FAM_UMMA_1CTA, BN, false, true, 1),
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
+    CUDA_TRY(cudaFuncSetAttribute((const void*)launch_map_umma(ADAPT_FAM_UMMA_1CTA, 64, false, true, 2),
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
     S.device = device;
     S.inited = true;
     return ADAPT_OK;
@@ -534,27 +537,30 @@ adapt_status_t cached_map(State& S, Plan* pl, bool isA, const void* base, int64_
     return ADAPT_OK;
 }
 
-// Eight maps of a row-major A (M x K, K % 8 != 0, 16-byte aligned base), one per row class j = row % 8:
-// base rounded down to 16 bytes, rows 16*K bytes apart, inner extent K + sigma_j so that the k tail is
-// zero-filled; sigma_j = elements between the rounded base and the start of row j.
-adapt_status_t cached_class_maps(State& S, Plan* pl, const void* A, int64_t M, int64_t K, int box_rows, CUtensorMap* out, int* sigma)
+// Eight maps of a row-major matrix (rows x cols, cols % 8 != 0, 16-byte aligned base), one per row class
+// j = row % 8: base rounded down to 16 bytes, rows 16*cols bytes apart, inner extent cols + sigma_j so that
+// the tail is zero-filled; sigma_j = elements between the rounded base and the start of row j.  Used for
+// A (rows = M, cols = K) and, in k-class mode, for B (rows = K, cols = N).
+adapt_status_t cached_class_maps(State& S, Plan* pl, bool isA, const void* base_ptr, int64_t rows_total, int64_t cols,
+                                 int box_rows, CUtensorMap* out, int* sigma)
 {
     std::lock_guard<std::mutex> lock(pl->mu);
-    for (int j = 0; j < 8; ++j) sigma[j] = (int)(((2 * j * K) & 15) / 2);
-    MapSlot* slots = pl->mapA;
+    for (int j = 0; j < 8; ++j) sigma[j] = (int)(((2 * j * cols) & 15) / 2);
+    MapSlot* slots = isA ? pl->mapA : pl->mapB;
     for (int i = 0; i < 2; ++i)
-        if (slots[i].ptr == A && slots[i].count == 8) { memcpy(out, slots[i].map, 8 * sizeof(CUtensorMap)); return ADAPT_OK; }
-    MapSlot& sl = slots[pl->nextA];
-    pl->nextA ^= 1;
+        if (slots[i].ptr == base_ptr && slots[i].count == 8) { memcpy(out, slots[i].map, 8 * sizeof(CUtensorMap)); return ADAPT_OK; }
+    int& next = isA ? pl->nextA : pl->nextB;
+    MapSlot& sl = slots[next];
+    next ^= 1;
     sl.ptr = nullptr;
     for (int j = 0; j < 8; ++j) {
-        const uint8_t* base = (const uint8_t*)A + ((2 * j * K) & ~(int64_t)15);
-        const int64_t rows = std::max<int64_t>(1, ceil_div(M - j, 8));
-        adapt_status_t r = encode_map(S, &sl.map[j], base, pl->s.dtype, K + sigma[j], rows, 8 * K, 64, box_rows);
+        const uint8_t* base = (const uint8_t*)base_ptr + ((2 * j * cols) & ~(int64_t)15);
+        const int64_t rows = std::max<int64_t>(1, ceil_div(rows_total - j, 8));
+        adapt_status_t r = encode_map(S, &sl.map[j], base, pl->s.dtype, cols + sigma[j], rows, 8 * cols, 64, box_rows);
         if (r != ADAPT_OK) return r;
     }
-    sl.ptr = A;
-    sl.pitch = K;
+    sl.ptr = base_ptr;
+    sl.pitch = cols;
     sl.count = 8;
     memcpy(out, sl.map, 8 * sizeof(CUtensorMap));
     return ADAPT_OK;
@@ -585,26 +591,55 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
 {
     const Shape& s = pl->s;
     const Config& c = pl->c;
-    const bool a_mn = s.layoutA == ADAPT_COL_MAJOR;       // M contiguous
     const bool b_mn = s.layoutB == ADAPT_ROW_MAJOR;       // N contiguous
-    const int64_t inA = a_mn ? s.M : s.K, outA = a_mn ? s.K : s.M;
-    const int64_t inB = b_mn ? s.N : s.K, outB = b_mn ? s.K : s.N;
-    // the copy-free class mode needs a 16-byte aligned A; otherwise fall back to the re-pitched copy
+    // the copy-free class modes need 16-byte aligned base pointers; otherwise fall back to re-pitched copies
     const bool classesA = c.srcA == ADAPT_SRC_TMA_CLASSES && ((uintptr_t)A & 15) == 0;
-    const bool padA = !classesA && (c.srcA != ADAPT_SRC_TMA || ((uintptr_t)A & 15) != 0);
-    const bool padB = c.srcB == ADAPT_SRC_PAD_COPY || ((uintptr_t)B & 15) != 0;
+    const bool kclsB = c.srcB == ADAPT_SRC_TMA_CLASSES && ((uintptr_t)B & 15) == 0;
+    const bool a_mn = !kclsB && s.layoutA == ADAPT_COL_MAJOR;   // M contiguous (the regrouped A' is always K-major)
+    const int64_t Kc = round_up(ceil_div(s.K, 8), 64);          // k-class mode: padded class segment of A'
+    const int64_t inA = kclsB ? 8 * Kc : (a_mn ? s.M : s.K), outA = a_mn ? s.K : s.M;
+    const int64_t inB = b_mn ? s.N : s.K, outB = b_mn ? s.K : s.N;
+    const bool a_inner_ok = (s.layoutA == ADAPT_COL_MAJOR ? s.M : s.K) % 8 == 0;
+    const bool padA = !classesA && !kclsB && (!a_inner_ok || ((uintptr_t)A & 15) != 0);
+    const bool padB = !kclsB && (inB % 8 != 0 || ((uintptr_t)B & 15) != 0);
     const int64_t pitchA = padA ? padded_pitch(inA) : inA;
     const int64_t pitchB = padB ? padded_pitch(inB) : inB;
-    const size_t szA = padA ? (size_t)round_up(outA * pitchA * 2, 256) : 0;
+    const size_t szA = (padA || kclsB) ? (size_t)round_up(outA * pitchA * 2, 256) : 0;
     const size_t szB = padB ? (size_t)round_up(outB * pitchB * 2, 256) : 0;
-    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * round_up(s.N, 4) * 4, 256) : 0;
+
+    const int cg = c.cluster;
+    TmapPack maps;
+    UmmaParams p;
+    int a_box_rows = 128;
+    memset(p.a_sigma, 0, sizeof(p.a_sigma));
+    memset(p.b_sigma, 0, sizeof(p.b_sigma));
+    p.cls_kc = (int)Kc;
+    p.M = (int)s.M; p.N = (int)s.N; p.K = (int)s.K;
+    // a plan made for class tiles that has to fall back to copies (unaligned pointer) uses plain tiles
+    p.P_m = (c.srcA == ADAPT_SRC_TMA_CLASSES && !classesA) ? (int)ceil_div(s.M, c.BM) : c.P_m;
+    p.P_n = (c.srcB == ADAPT_SRC_TMA_CLASSES && !kclsB) ? (int)ceil_div(s.N, c.BN) : c.P_n;
+    p.kb_total = kclsB ? (int)(Kc / kUmmaBK) : (int)ceil_div(s.K + (classesA ? 7 : 0), kUmmaBK);
+    p.kb_per_split = (int)ceil_div(p.kb_total, c.P_k);
+    p.P_k = (int)ceil_div(p.kb_total, p.kb_per_split);    // equals the plan's count unless a fallback changed kb_total
+    p.num_units = p.P_m * p.P_n * p.P_k;
+
+    const size_t szP = p.P_k > 1 ? (size_t)round_up((int64_t)p.P_k * s.M * round_up(s.N, 4) * 4, 256) : 0;
     void* ws = nullptr;
     adapt_status_t r = get_workspace(S, stream, szA + szB + szP, &ws);
     if (r != ADAPT_OK) return r;
     uint8_t* w8 = (uint8_t*)ws;
     const void* a_src = A;
     const void* b_src = B;
-    if (padA) {
+    if (kclsB) {
+        const int64_t a_sm = s.layoutA == ADAPT_ROW_MAJOR ? s.K : 1, a_sk = s.layoutA == ADAPT_ROW_MAJOR ? 1 : s.M;
+        const int64_t work = s.M * Kc;                    // 16-byte chunks of A'
+        const int blocks = (int)std::min<int64_t>(ceil_div(work, 256), (int64_t)S.machine.n_sm * 16);
+        regroup_a_kernel<<<blocks, 256, 0, stream>>>((const unsigned short*)A, (unsigned short*)w8, (int)s.M, (int)s.K,
+                                                       (int)Kc, a_sm, a_sk);
+        S.launches.fetch_add(1, std::memory_order_relaxed);
+        CUDA_TRY(cudaGetLastError());
+        a_src = w8;
+    } else if (padA) {
         if ((r = launch_pad(S, A, w8, outA, inA, pitchA, stream)) != ADAPT_OK) return r;
         a_src = w8;
     }
@@ -612,32 +647,25 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
         if ((r = launch_pad(S, B, w8 + szA, outB, inB, pitchB, stream)) != ADAPT_OK) return r;
         b_src = w8 + szA;
     }
-    float* partial = c.P_k > 1 ? (float*)(w8 + szA + szB) : nullptr;
+    float* partial = p.P_k > 1 ? (float*)(w8 + szA + szB) : nullptr;
 
-    const int cg = c.cluster;
-    TmapPack maps;
-    UmmaParams p;
-    int a_box_rows = 128;
-    memset(p.a_sigma, 0, sizeof(p.a_sigma));
     // K-major operand: one box of 64 k x (rows this CTA owns); MN-major operand: boxes of 64 x 64
     if (classesA) {
         if (s.M < 1024) a_box_rows = (int)std::min<int64_t>(128, round_up(ceil_div(s.M, 8), 8));   // rows of the largest class
-        if ((r = cached_class_maps(S, pl, A, s.M, s.K, a_box_rows, maps.a, p.a_sigma)) != ADAPT_OK) return r;
+        if ((r = cached_class_maps(S, pl, true, A, s.M, s.K, a_box_rows, maps.a, p.a_sigma)) != ADAPT_OK) return r;
     } else {
         // a K-major A of fewer than 128 rows is loaded with a box of just those rows (rounded up to 8):
         // the rows of the stage it leaves untouched only feed accumulator rows that are never stored
         if (!a_mn && cg == 1 && s.M < 128) a_box_rows = (int)round_up(s.M, 8);
         if ((r = cached_map(S, pl, true, a_src, inA, outA, pitchA, 64, a_mn ? 64 : a_box_rows, &maps.a[0])) != ADAPT_OK) return r;
     }
-    if ((r = cached_map(S, pl, false, b_src, inB, outB, pitchB, 64, b_mn ? 64 : c.BN / cg, &maps.b)) != ADAPT_OK) return r;
+    if (kclsB) {
+        // rows of B (K x N, N % 8 != 0) by class k % 8: the same construction as A's row classes, 64 x 64 boxes
+        if ((r = cached_class_maps(S, pl, false, B, s.K, s.N, 64, maps.b, p.b_sigma)) != ADAPT_OK) return r;
+    } else {
+        if ((r = cached_map(S, pl, false, b_src, inB, outB, pitchB, 64, b_mn ? 64 : c.BN / cg, &maps.b[0])) != ADAPT_OK) return r;
+    }
 
-    p.M = (int)s.M; p.N = (int)s.N; p.K = (int)s.K;
-    // a plan made for class tiles that has to fall back to the copy (unaligned A pointer) uses plain tiles
-    p.P_m = (c.srcA == ADAPT_SRC_TMA_CLASSES && !classesA) ? (int)ceil_div(s.M, c.BM) : c.P_m;
-    p.P_n = c.P_n; p.P_k = c.P_k;
-    p.kb_total = (int)ceil_div(s.K + (classesA ? 7 : 0), kUmmaBK);
-    p.kb_per_split = (int)ceil_div(p.kb_total, c.P_k);
-    p.num_units = p.P_m * c.P_n * c.P_k;
     p.dtype = s.dtype;
     p.stages = c.stages;
     p.a_tx_bytes = a_box_rows * kUmmaBK * 2;
@@ -651,7 +679,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.trace = S.d_trace;
 #endif
 
-    UmmaKernel k = launch_map_umma(c.family, c.BN, a_mn, b_mn, classesA);
+    UmmaKernel k = launch_map_umma(c.family, c.BN, a_mn, b_mn, classesA ? 1 : (kclsB ? 2 : 0));
     if (!k) return fail(ADAPT_ERR_UNSUPPORTED, "no compiled kernel for this tiling key%s");
     const int slots = S.machine.n_sm / cg;
     const int grid = std::min(p.num_units, slots) * cg;
@@ -670,7 +698,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     cfg.numAttrs = 1;
     CUDA_TRY(cudaLaunchKernelEx(&cfg, k, maps, p));
     S.launches.fetch_add(1, std::memory_order_relaxed);
-    if (c.P_k > 1) return launch_reduce(S, partial, C, s.M, s.N, c.P_k, s.dtype, stream);
+    if (p.P_k > 1) return launch_reduce(S, partial, C, s.M, s.N, p.P_k, s.dtype, stream);
     return ADAPT_OK;
 }
 

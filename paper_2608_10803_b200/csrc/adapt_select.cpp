@@ -128,6 +128,14 @@ static void model_prologue(const Shape& s, Config& c, const Calib& cal)
 {
     c.t_pro_us = 0;
     c.ws_padA = c.ws_padB = 0;
+    if (c.srcB == ADAPT_SRC_TMA_CLASSES) {
+        // k-class mode: A is regrouped class-major (element-wise reads, 16-byte writes); B is read in place
+        const double src = 2.0 * (double)s.M * (double)s.K;
+        c.ws_padA = round_up(s.M * 8 * round_up(ceil_div(s.K, 8), 64) * 2, 256);
+        c.t_pro_us += cal.launch_us + (src + (double)c.ws_padA) / (cal.hbm_bw * cal.regroup_bw_eff) * 1e6;
+        c.hbm_bytes += src + (double)c.ws_padA;
+        return;
+    }
     if (c.srcA == ADAPT_SRC_PAD_COPY) {
         const double src = 2.0 * (double)s.M * (double)s.K;
         c.ws_padA = round_up(outerA(s) * padded_pitch(innerA(s)) * 2, 256);
@@ -161,8 +169,10 @@ static void model_epilogue(const Shape& s, Config& c, const Calib& cal)
 
 static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Config& c)
 {
-    const int64_t kblocks = ceil_div(s.K + (c.srcA == ADAPT_SRC_TMA_CLASSES ? 7 : 0), c.BK);
-    const int64_t L = ceil_div(kblocks, c.P_k);
+    const bool kclasses = c.srcB == ADAPT_SRC_TMA_CLASSES;
+    const int64_t kblocks = kclasses ? ceil_div(ceil_div(s.K, 8), c.BK)
+                                     : ceil_div(s.K + (c.srcA == ADAPT_SRC_TMA_CLASSES ? 7 : 0), c.BK);
+    const int64_t L = ceil_div(kblocks, c.P_k) * (kclasses ? 8 : 1);     // k-class mode: the split's blocks of all 8 classes
     const int64_t units = (int64_t)c.P_m * c.P_n * c.P_k;
     const int64_t slots = m.n_sm / c.cluster;
     const int64_t Q = ceil_div(units, slots);
@@ -176,7 +186,7 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     if (rB > 1.0 && 2.0 * MK <= kL2Bytes) {          // alternatively A stays resident and B streams once
         rB = 1.0;
     }
-    c.hbm_bytes = 2.0 * (MK * rA + KN * rB) + (c.P_k > 1 ? 0.0 : 2.0 * MN);
+    c.hbm_bytes = 2.0 * (MK * rA + KN * rB * (kclasses ? 64.0 / 56.0 : 1.0)) + (c.P_k > 1 ? 0.0 : 2.0 * MN);
 
     // per-SM stage: each CTA loads its 128 rows of A and its share of the BN columns of B
     const double bn_per_cta = (double)c.BN / c.cluster;
@@ -215,7 +225,7 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     model_prologue(s, c, cal);
     model_epilogue(s, c, cal);
     // strided row-class views stream A at a lower rate than a dense tensor (measured 3.5-4.1 TB/s)
-    const double bw = c.srcA == ADAPT_SRC_TMA_CLASSES ? cal.hbm_bw * cal.class_view_bw_eff : cal.hbm_bw;
+    const double bw = (c.srcA == ADAPT_SRC_TMA_CLASSES || kclasses) ? cal.hbm_bw * cal.class_view_bw_eff : cal.hbm_bw;
     const double t_hbm = c.hbm_bytes / bw * 1e6 - c.t_pro_us - c.t_epi_us;
     c.t_main_us = std::max(pipe, t_hbm);
     finish_common(s, c, cal);
@@ -284,23 +294,32 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     c.smem_bytes = umma_smem_bytes(c.BN, c.cluster, c.stages);
     if (c.smem_bytes > m.smem_bytes) return false;
     // in class mode the k index of a tile is shifted by up to 7 elements
-    const int64_t kblocks = ceil_div(s.K + (c.srcA == ADAPT_SRC_TMA_CLASSES ? 7 : 0), c.BK);
+    // k-class mode splits the blocks of one class; in row-class mode the k index is shifted by up to 7
+    const int64_t kblocks = c.srcB == ADAPT_SRC_TMA_CLASSES ? ceil_div(ceil_div(s.K, 8), c.BK)
+                                                              : ceil_div(s.K + (c.srcA == ADAPT_SRC_TMA_CLASSES ? 7 : 0), c.BK);
     if (c.P_k < 1 || c.P_k > 1023 || c.P_k > kblocks) return false;
     if (ceil_div(kblocks, ceil_div(kblocks, c.P_k)) != c.P_k) return false;   // no empty split
     // operand sources: TMA needs a 16-byte row pitch
     if (c.srcA == ADAPT_SRC_TMA && !aligned16(innerA(s))) return false;
     if (c.srcB == ADAPT_SRC_TMA && !aligned16(innerB(s))) return false;
-    if (c.srcA == ADAPT_SRC_LSU || c.srcB == ADAPT_SRC_LSU || c.srcB == ADAPT_SRC_TMA_CLASSES) return false;
+    if (c.srcA == ADAPT_SRC_LSU || c.srcB == ADAPT_SRC_LSU) return false;
     const bool classes = c.srcA == ADAPT_SRC_TMA_CLASSES;
+    const bool kclasses = c.srcB == ADAPT_SRC_TMA_CLASSES;
+    if (kclasses) {
+        // k-rows of one residue class share their misalignment: row-major B with N % 8 != 0, 64-column
+        // windows that own 56 columns, A regrouped class-major by a prologue copy (any layout of A)
+        if (c.family != ADAPT_FAM_UMMA_1CTA || s.layoutB != ADAPT_ROW_MAJOR || c.BN != 64) return false;
+        if (aligned16(innerB(s)) || s.K < 64 || c.srcA != ADAPT_SRC_PAD_COPY) return false;
+    }
     if (classes) {
         // rows of one residue class share their misalignment: row-major A and B, one CTA per tile
         if (c.family != ADAPT_FAM_UMMA_1CTA || s.layoutA != ADAPT_ROW_MAJOR || s.layoutB != ADAPT_ROW_MAJOR) return false;
         if (aligned16(innerA(s)) || s.M < 8) return false;
     }
-    if (c.srcA == ADAPT_SRC_PAD_COPY && aligned16(innerA(s))) return false;    // nothing to pad
+    if (c.srcA == ADAPT_SRC_PAD_COPY && aligned16(innerA(s)) && !kclasses) return false;    // nothing to pad
     if (c.srcB == ADAPT_SRC_PAD_COPY && aligned16(innerB(s))) return false;
     c.P_m = classes ? (int)(8 * ceil_div(s.M, 8 * c.BM)) : (int)ceil_div(s.M, c.BM);   // class tiles: 8 per 1024 rows
-    c.P_n = (int)ceil_div(s.N, c.BN);
+    c.P_n = (int)ceil_div(s.N, kclasses ? 56 : c.BN);
     if ((int64_t)c.P_m * c.P_n * c.P_k > (int64_t)1 << 30) return false;
     c.persistent = 1;
     return true;
@@ -444,6 +463,21 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
                 d.stages = deepest; d.P_k = pk; d.srcA = ADAPT_SRC_TMA_CLASSES; d.srcB = srcB;
                 if (deepest >= 2 && finalize(s, m, cal, d)) out->push_back(d);
             }
+        }
+    }
+    // --- tcgen05, B read in place through per-k-class views (row-major B, N % 8 != 0); A is regrouped by a
+    //     prologue copy, so this pays when A is the small operand ---
+    if (srcB == ADAPT_SRC_PAD_COPY && s.layoutB == ADAPT_ROW_MAJOR && s.K >= 64) {
+        const int64_t tiles = ceil_div(s.M, 128) * ceil_div(s.N, 56);
+        split_candidates(tiles, m.n_sm, ceil_div(ceil_div(s.K, 8), 64), 1, &pks);
+        int deepest = 0;
+        for (int st = 8; st >= 2; --st)
+            if (umma_smem_bytes(64, 1, st) <= m.smem_bytes) { deepest = st; break; }
+        for (int pk : pks) {
+            Config d;
+            d.family = ADAPT_FAM_UMMA_1CTA; d.BM = 128; d.BN = 64; d.BK = 64; d.cluster = 1;
+            d.stages = deepest; d.P_k = pk; d.srcA = ADAPT_SRC_PAD_COPY; d.srcB = ADAPT_SRC_TMA_CLASSES;
+            if (deepest >= 2 && finalize(s, m, cal, d)) out->push_back(d);
         }
     }
     // --- warp-level streaming family ---

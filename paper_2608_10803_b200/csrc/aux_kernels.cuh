@@ -71,6 +71,36 @@ pad_copy_kernel(const unsigned short* __restrict__ src, unsigned short* __restri
     }
 }
 
+// ---- k-class regrouping of A (prologue of the k-class mode) -----------------------------------------
+// A'[m][j * Kc + t] = A[m][8 t + j] for 8 t + j < K, else 0; j = 0..7, t < Kc.  A' is row-major with
+// pitch 8 * Kc (Kc a multiple of 64), so TMA reads the columns of one class as a dense K-major tile.
+// One thread writes eight consecutive t of one (m, j): a 16-byte store; A is read element-wise
+// (it is the small operand when this mode is chosen).
+__global__ void __launch_bounds__(256)
+regroup_a_kernel(const unsigned short* __restrict__ A, unsigned short* __restrict__ Ap,
+                 int M, int K, int Kc, int64_t a_sm, int64_t a_sk)
+{
+    const int chunks = Kc / 8;
+    const int64_t total = (int64_t)M * 8 * chunks;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % chunks);
+        const int j = (int)((i / chunks) & 7);
+        const int m = (int)(i / ((int64_t)8 * chunks));
+        unsigned short v[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const int k = 8 * (8 * c + e) + j;
+            v[e] = k < K ? __ldg(A + (int64_t)m * a_sm + (int64_t)k * a_sk) : (unsigned short)0;
+        }
+        uint4 o;
+        o.x = (uint32_t)v[0] | ((uint32_t)v[1] << 16);
+        o.y = (uint32_t)v[2] | ((uint32_t)v[3] << 16);
+        o.z = (uint32_t)v[4] | ((uint32_t)v[5] << 16);
+        o.w = (uint32_t)v[6] | ((uint32_t)v[7] << 16);
+        *reinterpret_cast<uint4*>(Ap + (int64_t)m * 8 * Kc + (int64_t)j * Kc + 8 * c) = o;
+    }
+}
+
 // ---- split-K reduction: C = RN16( sum_{p = 0..P_k-1} partial[p] ), ascending p, fp32 ---------------
 // The order is fixed, so the result does not depend on which CTA finished first.  Partials are
 // stored [P_k][M][Np] with Np = N rounded up to 4, so every row starts on a 16-byte boundary and

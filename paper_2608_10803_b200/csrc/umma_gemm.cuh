@@ -40,7 +40,9 @@ struct UmmaParams {
     float* partial;                  // fp32 [P_k][M][Np], Np = N rounded up to 4 (used when P_k > 1)
     int Np;                          // row pitch of the partials in elements
     int a_tx_bytes;                  // bytes one TMA load of A delivers per stage and CTA (a short box when M < 128)
-    int a_sigma[8];                  // class mode: shift (elements) of row class j = row % 8 against its 16-byte aligned base
+    int a_sigma[8];
+    int b_sigma[8];                  // k-class mode: column shift of B's row class j = k % 8
+    int cls_kc;                      // k-class mode: padded length of one class segment of A' (multiple of 64)                  // class mode: shift (elements) of row class j = row % 8 against its 16-byte aligned base
     unsigned int* status;            // device status word: bit 0 = a bounded wait expired
     unsigned long long* trace;       // timestamp trace of CTA 0 (diagnostic builds only), else null
 };
@@ -61,7 +63,7 @@ struct UmmaParams {
 // rows of A with row % 8 == j (see the kernel comment).
 struct TmapPack {
     CUtensorMap a[8];
-    CUtensorMap b;
+    CUtensorMap b[8];         // b[0] is the map of B; in k-class mode b[j] is the map of the k-rows with k % 8 == j
 };
 
 // unit index -> (m block, n block, split).  Units of one output tile are adjacent in split;
@@ -106,17 +108,30 @@ __device__ __forceinline__ unsigned short cast16(float a, int dtype)
 // kappa < sigma_j or k >= K are out of bounds and read as zero.  The sigma_j leading elements of
 // each A' row belong to the previous row of A: the MMA warp overwrites them with zeros in the
 // first k-block before the tensor core reads them.
-template <int BN, bool A_MN, bool B_MN, int CG, bool A_CLS>
+//
+// B_CLS (MODE 2, "k classes"): B is row-major with N % 8 != 0.  Its rows k and k + 8 share their
+// offset from a 16-byte boundary, so the k-rows of one residue class j = k % 8 form a tensor TMA can
+// read, every row shifted by the same sigma_j columns.  The contraction runs class by class: a
+// prologue kernel has regrouped A's columns class-major (A'[m][j][t] = A[m][8t + j], zero padded),
+// class j accumulates into its own TMEM buffer j (8 buffers of 64 columns) over the window
+// x' in [56*nb, 56*nb + 64) of shifted columns, and the epilogue adds the eight buffers with
+// buffer j read sigma_j columns to the right: C[m][56*nb + c] = sum_j acc_j[m][c + sigma_j], c < 56.
+// Columns of a buffer left of sigma_j hold products with the previous row's tail and are never read.
+template <int BN, bool A_MN, bool B_MN, int CG, int MODE>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
 {
-    static_assert(!A_CLS || (!A_MN && B_MN && CG == 1), "class mode: row-major A and B, one CTA per tile");
+    constexpr bool A_CLS = MODE == 1;
+    constexpr bool B_CLS = MODE == 2;
+    static_assert(MODE == 0 || (!A_MN && B_MN && CG == 1), "class modes: K-major A, row-major B, one CTA per tile");
+    static_assert(!B_CLS || BN == 64, "k-class mode uses 64-column windows");
+    constexpr int TILE_N = B_CLS ? 56 : BN;               // output columns a tile owns
     constexpr int BN_CTA = BN / CG;                       // B columns this CTA loads
     constexpr int A_BYTES = 128 * kUmmaBK * 2;
     constexpr int B_BYTES = BN_CTA * kUmmaBK * 2;
     constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    constexpr int NBUF = (512 / BN) < 4 ? (512 / BN) : 4; // accumulator buffers in TMEM
-    constexpr int TMEM_COLS = NBUF * BN;
+    constexpr int NBUF = B_CLS ? 1 : ((512 / BN) < 4 ? (512 / BN) : 4);   // accumulator buffers in TMEM
+    constexpr int TMEM_COLS = B_CLS ? 512 : NBUF * BN;    // k-class mode: eight class accumulators of 64 columns
     constexpr int PASSES = BN / 64;                       // 64-column epilogue passes per tile
     static_assert(TMEM_COLS == 256 || TMEM_COLS == 512, "TMEM allocation is a power of two");
     static_assert(BN_CTA % 64 == 0, "B is loaded in 64-column boxes");
@@ -156,7 +171,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
         ptx::prefetch_tensormap(&maps.a[0]);
-        ptx::prefetch_tensormap(&maps.b);
+        ptx::prefetch_tensormap(&maps.b[0]);
     }
     if (warp == 1) {
         ptx::tmem_alloc<CG>(tmem_slot, TMEM_COLS);
@@ -194,8 +209,21 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
                 const int row0 = A_CLS ? (mb >> 3) * 128 : mb * (128 * CG) + (int)cta_rank * 128;
                 const int kshift = A_CLS ? p.a_sigma[cls] : 0;                // B's k-rows lag A's kappa by sigma
                 const CUtensorMap* tmA = &maps.a[cls];
-                const CUtensorMap* tmB = &maps.b;
-                const int col0 = nb * BN + (int)cta_rank * BN_CTA;            // this CTA's B columns
+                const CUtensorMap* tmB = &maps.b[0];
+                const int col0 = nb * TILE_N + (int)cta_rank * BN_CTA;        // this CTA's B columns
+                if (B_CLS) {
+                    // class by class: A' columns j*Kc + 64*b .., B's class-j rows 64*b .. at shifted columns 56*nb ..
+                    for (int j = 0; ok && j < 8; ++j)
+                        for (int kb = kb0; kb < kb1; ++kb) {
+                            if (!ptx::mbar_wait(empty_bar + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                            const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
+                            ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(p.a_tx_bytes + B_BYTES));
+                            ptx::tma_load_2d(sA, tmA, full_bar + 8u * stage, j * p.cls_kc + kb * kUmmaBK, row0);
+                            ptx::tma_load_2d(sA + A_BYTES, &maps.b[j], full_bar + 8u * stage, col0, kb * kUmmaBK);
+                            if (++stage == S) { stage = 0; phase ^= 1u; }
+                        }
+                    continue;
+                }
                 for (int kb = kb0; kb < kb1; ++kb) {
                     if (!ptx::mbar_wait(empty_bar + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
@@ -261,7 +289,24 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
                 ptx::tc_fence_after();
                 ADAPT_TRACE(2, unit);
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-                for (int kb = kb0; kb < kb1; ++kb) {
+                if (B_CLS) {
+                    for (int j = 0; ok && j < 8; ++j)
+                        for (int kb = kb0; kb < kb1; ++kb) {
+                            if (!mma_wait(full_bar + 8u * stage, phase)) { ok = false; break; }
+                            ptx::tc_fence_after();
+                            const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
+                            const uint32_t sB = sA + A_BYTES;
+#pragma unroll
+                            for (int k16 = 0; k16 < kUmmaBK / 16; ++k16) {
+                                const uint64_t adesc = ptx::smem_desc_sw128(sA + k16 * a_kstep, a_lbo, 1024u);
+                                const uint64_t bdesc = ptx::smem_desc_sw128(sB + k16 * b_kstep, b_lbo, 1024u);
+                                ptx::umma_f16<CG>(tmem_base + 64u * j, adesc, bdesc, p.idesc, (kb > kb0 || k16 > 0) ? 1u : 0u);
+                            }
+                            ptx::umma_commit_1(empty_bar + 8u * stage);
+                            if (++stage == S) { stage = 0; phase ^= 1u; }
+                        }
+                }
+                for (int kb = kb0; !B_CLS && kb < kb1; ++kb) {
                     if (!mma_wait(full_bar + 8u * stage, phase)) { ok = false; break; }
                     ptx::tc_fence_after();
                     const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
@@ -326,8 +371,23 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
             const int row_step = A_CLS ? 8 : 1;
             const int row_base = A_CLS ? (mb >> 3) * 1024 + (mb & 7) : mb * (128 * CG) + (int)cta_rank * 128;
             const int row = row_base + row_step * (q * 32 + lane);
-            const int n0 = nb * BN;
+            const int n0 = nb * TILE_N;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
+            // k-class mode: columns [8c, 8c+8) of the tile = sum over the class buffers j (ascending), buffer j
+            // read sigma_j columns to the right
+            auto class_sum8 = [&](int c, uint32_t* out8) {
+                uint32_t v[8][8];
+#pragma unroll
+                for (int j = 0; j < 8; ++j) ptx::tmem_ld_32x8(t_row + (uint32_t)(64 * j + p.b_sigma[j] + 8 * c), v[j]);
+                ptx::tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    float acc = __uint_as_float(v[0][i]);
+#pragma unroll
+                    for (int j = 1; j < 8; ++j) acc += __uint_as_float(v[j][i]);
+                    out8[i] = __float_as_uint(acc);
+                }
+            };
             const bool row_ok = row < p.M;
             if (p.P_k == 1) {
                 // 16-bit output, any N and any base alignment.  A thread converts 64 columns of its row
@@ -341,10 +401,10 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
                 const uintptr_t row_bytes = 2ull * (uintptr_t)p.N * row_step;   // distance between this warp's rows
                 // the two warps of a lane quarter take alternate tiles, so one thread sees all passes of
                 // its row and can carry the ragged tail of a pass into the head of the next one
-                if ((seq & 1) == half) {
+                if (B_CLS ? half == 0 : (seq & 1) == half) {
                     const uintptr_t g_row = g_tile + (uintptr_t)lane * row_bytes;   // this thread's row, column n0
                     const int m_r = (int)((g_row & 15u) >> 1);           // the same in every pass: a pass is 128 bytes
-                    const int tile_cols = min(BN, p.N - n0);
+                    const int tile_cols = min(TILE_N, p.N - n0);
 #pragma unroll 1
                     for (int pass = 0; pass < PASSES; ++pass) {
                         const int c0 = pass * 64;
@@ -352,9 +412,18 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
                         const int ncols = min(64, tile_cols - c0);
                         const bool last = c0 + 64 >= tile_cols;
                         uint32_t r0[32], r1[32];
-                        ptx::tmem_ld_32x32(t_row + (uint32_t)c0, r0);
-                        if (ncols > 32) ptx::tmem_ld_32x32(t_row + (uint32_t)(c0 + 32), r1);   // uniform
-                        ptx::tmem_ld_wait();
+                        if (B_CLS) {
+#pragma unroll
+                            for (int c = 0; c < 4; ++c) class_sum8(c, r0 + 8 * c);
+#pragma unroll
+                            for (int c = 4; c < 7; ++c) class_sum8(c, r1 + 8 * (c - 4));
+#pragma unroll
+                            for (int i = 24; i < 32; ++i) r1[i] = 0;
+                        } else {
+                            ptx::tmem_ld_32x32(t_row + (uint32_t)c0, r0);
+                            if (ncols > 32) ptx::tmem_ld_32x32(t_row + (uint32_t)(c0 + 32), r1);   // uniform
+                            ptx::tmem_ld_wait();
+                        }
                         if (warp == 2 && lane == 0) ADAPT_TRACE(5, unit);
                         __syncwarp();                                    // the previous pass has been written out
                         // carry: elements 64..71 of the previous pass become elements 0..7 of this one
@@ -427,8 +496,29 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
             } else {
                 // fp32 partial tile: rows of the workspace are 16-byte aligned (pitch Np), so a thread
                 // writes its row's 32 columns as eight aligned 16-byte stores
+                if (B_CLS) {
+                    if (half == 0) {
 #pragma unroll 1
-                for (int c0 = 0; c0 < BN; c0 += 32) {
+                        for (int c = 0; c < 7; ++c) {
+                            if (n0 + 8 * c >= p.N) break;            // uniform across the warp
+                            uint32_t r8[8];
+                            class_sum8(c, r8);
+                            if (!row_ok) continue;
+                            const int col = n0 + 8 * c;
+                            float* prow = p.partial + ((size_t)split * p.M + row) * p.Np + col;
+                            if (col + 8 <= p.Np) {
+                                *reinterpret_cast<uint4*>(prow) = make_uint4(r8[0], r8[1], r8[2], r8[3]);
+                                *reinterpret_cast<uint4*>(prow + 4) = make_uint4(r8[4], r8[5], r8[6], r8[7]);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 8; ++j)
+                                    if (col + j < p.N) prow[j] = __uint_as_float(r8[j]);
+                            }
+                        }
+                    }
+                }
+#pragma unroll 1
+                for (int c0 = 0; !B_CLS && c0 < BN; c0 += 32) {
                     if (n0 + c0 >= p.N) break;                       // uniform across the warp
                     if (((seq * (BN / 32) + (c0 >> 5)) & 1) != half) continue;
                     uint32_t r[32];

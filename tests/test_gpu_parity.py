@@ -256,3 +256,65 @@ def test_row_class_views_do_not_leak_a_neighbouring_row():
         assert torch.isfinite(C.index_select(0, keep)).all()
         err, mism, n = compare_with_oracle(A, B, C, M, N, K, dtype, rows=keep.cpu().numpy())
         assert mism == 0
+
+
+# ---- row-major B with N % 8 != 0 read in place through per-k-class TMA views ----------------------
+
+def kclass_mode_variants(M, N, K, dtype, layoutA=ROW, limit=6):
+    out = []
+    for c in ab.adapt_plan_candidates(M, N, K, dtype, layoutA, ROW):
+        if c.srcB == 3 and len(out) < limit:
+            out.append((ab.adapt_matmul_plan_forced(M, N, K, dtype, layoutA, ROW, c.tiling_key), c))
+    return out
+
+
+@pytest.mark.parametrize("dtype", [ab.F16, ab.BF16])
+@pytest.mark.parametrize("shape", [(8, 3001, 4000), (100, 777, 1000), (131, 57, 64), (17, 55, 1031), (300, 9, 70),
+                                   (129, 1234, 513), (5, 113, 5003), (64, 20002, 300)])
+def test_k_class_views_bit_exact(shape, dtype):
+    M, N, K = shape
+    A = synth.position_coded(M, K, dtype, modulus=7, device="cuda")
+    B = synth.position_coded(K, N, dtype, modulus=5, device="cuda")
+    variants = kclass_mode_variants(M, N, K, dtype)
+    assert variants, "shape must offer the k-class source for B"
+    assert any(c.P_k > 1 for _, c in variants) or K < 1024
+    for plan, c in variants:
+        check_case(M, N, K, dtype, A, B, plan=plan, exact=True)
+
+
+def test_k_class_views_with_column_major_a_and_random_values():
+    M, N, K = 77, 1001, 2049
+    for dtype in (ab.F16, ab.BF16):
+        A = synth.draw_operand(K, M, synth.U11, 21, dtype, "cuda")      # storage of a column-major A
+        B = synth.draw_operand(K, N, synth.U11, 22, dtype, "cuda")
+        variants = kclass_mode_variants(M, N, K, dtype, layoutA=COL)
+        assert variants
+        for plan, c in variants[:3]:
+            err, _, _, _ = check_case(M, N, K, dtype, A, B, COL, ROW, plan=plan)
+            assert err <= TOL[dtype]
+
+
+def test_k_class_views_do_not_leak_a_neighbouring_row():
+    """The elements in front of a class row's first element belong to the previous row of B; they land
+    in accumulator columns that are never read, so a non-finite value in column N - 1 of a row of B may
+    only reach column N - 1 of the result."""
+    M, N, K = 40, 203, 600
+    dtype = ab.F16
+    A = synth.position_coded(M, K, dtype, 7, "cuda")
+    B = synth.position_coded(K, N, dtype, 5, "cuda")
+    ref = run_library(A, B, M, N, K, dtype).clone()                 # checked against the oracle below
+    err, mism, _ = compare_with_oracle(A, B, ref, M, N, K, dtype)
+    assert mism == 0
+    for r in (4, 17, 300):
+        B[r, N - 1] = float("inf")
+    variants = kclass_mode_variants(M, N, K, dtype)
+    assert variants
+    for plan, c in variants:
+        C = run_library(A, B, M, N, K, dtype, plan=plan)
+        torch.cuda.synchronize()
+        assert torch.isfinite(C[:, : N - 1]).all()
+        assert torch.equal(synth_bits(C[:, : N - 1]), synth_bits(ref[:, : N - 1]))
+
+
+def synth_bits(t):
+    return t.contiguous().view(torch.int16)

@@ -128,14 +128,18 @@ def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
                     smem = c.stages * (128 * 64 * 2 + bn_cta * 64 * 2)
                     assert smem <= 227 * 1024
                     assert 2 * c.BN <= 512 and c.BN % 16 == 0
-                    assert c.P_k <= -(-(K + 7) // 64)
+                    assert c.P_k <= (-(-(-(-K // 8)) // 64) if c.srcB == 3 else -(-(K + 7) // 64))
                     # unaligned operands are never handed to TMA directly (row-major: K for A, N for B)
                     if K % 8:
                         assert c.srcA in (1, 3)      # re-pitched copy, or the per-row-class TMA views
                     if c.srcA == 3:
                         assert K % 8 and M >= 8 and c.family == ab.FAM_UMMA_1CTA and c.P_m == 8 * -(-M // 1024)
                     if N % 8:
-                        assert c.srcB == 1
+                        assert c.srcB in (1, 3)      # re-pitched copy, or the per-k-class TMA views
+                    if c.srcB == 3:
+                        # k classes: A regrouped class-major, 56 output columns per tile
+                        assert N % 8 and K >= 64 and c.family == ab.FAM_UMMA_1CTA and c.BN == 64
+                        assert c.srcA == 1 and c.P_n == -(-N // 56)
                 if c.family == ab.FAM_SKINNY:
                     assert min(M, N) <= 16
                 # taxonomy label follows the predicate (Section 4.2)
