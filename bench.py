@@ -533,6 +533,10 @@ def one_shape(args):
             cands = [c for c in cands if c.BN == args.bn]
         if args.pk:
             cands = [c for c in cands if c.P_k == args.pk]
+        if args.stages:
+            cands = [c for c in cands if c.stages == args.stages]
+        if args.src:
+            cands = [c for c in cands if f"{c.srcA}{c.srcB}" == args.src]
         plan = ab.adapt_matmul_plan_forced(M, N, K, dt, 0, 0, cands[0].tiling_key)
     else:
         plan = ab.adapt_matmul_plan(M, N, K, dt)
@@ -638,6 +642,8 @@ def main():
     ap.add_argument("--family", type=int, default=-1, help="with --shape: force a kernel family (0 umma_1cta, 1 umma_2cta, 2 skinny, 3 simt)")
     ap.add_argument("--bn", type=int, default=0)
     ap.add_argument("--pk", type=int, default=0)
+    ap.add_argument("--stages", type=int, default=0)
+    ap.add_argument("--src", type=str, default="", help="with --family: operand sources as two digits, e.g. 13 = A copied, B through k-class views")
     ap.add_argument("--cublas", action="store_true", help="with --shape: also time torch.matmul as the vendor reference")
     args = ap.parse_args()
     if args.shape:

@@ -651,12 +651,12 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
 
     // K-major operand: one box of 64 k x (rows this CTA owns); MN-major operand: boxes of 64 x 64
     if (classesA) {
-        if (s.M < 1024) a_box_rows = (int)std::min<int64_t>(128, round_up(ceil_div(s.M, 8), 8));   // rows of the largest class
+        a_box_rows = umma_a_box_rows(s, cg, true, false);       // rows of the largest class
         if ((r = cached_class_maps(S, pl, true, A, s.M, s.K, a_box_rows, maps.a, p.a_sigma)) != ADAPT_OK) return r;
     } else {
         // a K-major A of fewer than 128 rows is loaded with a box of just those rows (rounded up to 8):
         // the rows of the stage it leaves untouched only feed accumulator rows that are never stored
-        if (!a_mn && cg == 1 && s.M < 128) a_box_rows = (int)round_up(s.M, 8);
+        a_box_rows = umma_a_box_rows(s, cg, false, kclsB);
         if ((r = cached_map(S, pl, true, a_src, inA, outA, pitchA, 64, a_mn ? 64 : a_box_rows, &maps.a[0])) != ADAPT_OK) return r;
     }
     if (kclsB) {
@@ -667,7 +667,9 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     }
 
     p.dtype = s.dtype;
+    // the plan's ring depth assumed its own A box; a fallback to copies may need a shallower ring
     p.stages = c.stages;
+    while (p.stages > 2 && umma_smem_bytes(c.BN, cg, p.stages, a_box_rows) > S.machine.smem_bytes) --p.stages;
     p.a_tx_bytes = a_box_rows * kUmmaBK * 2;
     p.idesc = umma_idesc(s.dtype, a_mn, b_mn, 128 * cg, c.BN);
     p.C = C;
@@ -687,7 +689,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
     cfg.blockDim = dim3(kUmmaThreads, 1, 1);
-    cfg.dynamicSmemBytes = (size_t)umma_smem_bytes(c.BN, cg, c.stages);
+    cfg.dynamicSmemBytes = (size_t)umma_smem_bytes(c.BN, cg, p.stages, a_box_rows);
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;

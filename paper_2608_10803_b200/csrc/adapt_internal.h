@@ -4,6 +4,7 @@
 #include <cstdint>
 #include <cstddef>
 #include <vector>
+#include <algorithm>
 
 #include "adapt_matmul.h"
 
@@ -103,13 +104,26 @@ const Calib& default_calib();
 // S stages of (A: 128 x 64, B: BN/cluster x 64) 16-bit, a barrier block, the epilogue staging
 // (one 144-byte row per epilogue thread), and slack to align the stages to 1024 B.
 constexpr int kSkinnyKChunk = 512;   // k values the warp-level kernel stages per chunk; its k splits are whole chunks
-constexpr int kUmmaBarrierBytes = 256;
+constexpr int kUmmaBarrierBytes = 512;
+constexpr int kUmmaMaxStages = 15;
 constexpr int kUmmaEpilogueWarps = 8;
 constexpr int kUmmaStageRowBytes = 144;   // 72 16-bit elements: 64 columns + up to 7 of alignment shift
-inline int umma_smem_bytes(int BN, int cluster, int stages)
+inline int umma_smem_bytes(int BN, int cluster, int stages, int a_rows = 128)
 {
-    return stages * (128 * 64 * 2 + (BN / cluster) * 64 * 2) + kUmmaBarrierBytes +
+    return stages * (a_rows * 64 * 2 + (BN / cluster) * 64 * 2) + kUmmaBarrierBytes +
            kUmmaEpilogueWarps * 32 * kUmmaStageRowBytes + 1024;
+}
+
+// Rows of A one TMA box brings per stage (a multiple of 8, so the stage stays a multiple of 1024 B).
+// A K-major A of fewer than 128 rows is loaded with a box of just those rows, and the stage's A
+// region shrinks with it: the MMA still reads 128 rows, but the rows past the box only feed
+// accumulator rows that are never stored.  Class tiles hold every 8th row of up to 1024.
+inline int umma_a_box_rows(const Shape& s, int cluster, bool row_classes, bool k_classes)
+{
+    const bool a_mn = !k_classes && s.layoutA == ADAPT_COL_MAJOR;
+    if (row_classes) return s.M < 1024 ? (int)std::min<int64_t>(128, round_up(ceil_div(s.M, 8), 8)) : 128;
+    if (!a_mn && cluster == 1 && s.M < 128) return (int)round_up(s.M, 8);
+    return 128;
 }
 
 }  // namespace adapt

@@ -190,7 +190,8 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
 
     // per-SM stage: each CTA loads its 128 rows of A and its share of the BN columns of B
     const double bn_per_cta = (double)c.BN / c.cluster;
-    const double stage_bytes = 2.0 * c.BK * (128.0 + bn_per_cta);
+    const double a_rows = umma_a_box_rows(s, c.cluster, c.srcA == ADAPT_SRC_TMA_CLASSES, kclasses);
+    const double stage_bytes = 2.0 * c.BK * (a_rows + bn_per_cta);
     // One SM pulls operands that other SMs also use from L2 at l2_bw_per_sm (a little less through
     // the strided row-class views); a stream that comes from HBM and is used once is bounded by the
     // bytes one SM keeps in flight, about hbm_bw_per_sm.  The second case only shows in partial waves.
@@ -290,8 +291,9 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     }
     if (c.BN % 16 != 0 || c.BN > 256) return false;                 // UMMA shape rule for M = 128/256
     if (2 * c.BN > m.tmem_cols) return false;                       // at least two accumulator buffers in TMEM
-    if (c.stages < 1 || c.stages > 12) return false;
-    c.smem_bytes = umma_smem_bytes(c.BN, c.cluster, c.stages);
+    if (c.stages < 1 || c.stages > kUmmaMaxStages) return false;
+    c.smem_bytes = umma_smem_bytes(c.BN, c.cluster, c.stages,
+                                   umma_a_box_rows(s, c.cluster, c.srcA == ADAPT_SRC_TMA_CLASSES, c.srcB == ADAPT_SRC_TMA_CLASSES));
     if (c.smem_bytes > m.smem_bytes) return false;
     // in class mode the k index of a tile is shifted by up to 7 elements
     // k-class mode splits the blocks of one class; in row-class mode the k index is shifted by up to 7
@@ -429,12 +431,13 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
             // ring depth: the deepest that fits, and a double buffer (Eq. 13) for comparison
             Config probe;
             probe.family = fam; probe.BM = BM; probe.BN = BN; probe.BK = 64; probe.cluster = cluster;
+            const int a_rows = umma_a_box_rows(s, cluster, false, false);
             int deepest = 0;
-            for (int st = 12; st >= 2; --st) {
+            for (int st = kUmmaMaxStages; st >= 2; --st) {
                 probe.stages = st;
-                if (umma_smem_bytes(probe.BN, probe.cluster, st) <= m.smem_bytes) { deepest = st; break; }
+                if (umma_smem_bytes(probe.BN, probe.cluster, st, a_rows) <= m.smem_bytes) { deepest = st; break; }
             }
-            if (deepest > 8) deepest = 8;
+            if (a_rows == 128 && deepest > 8) deepest = 8;
             std::vector<int> depths = {deepest};
             if (deepest > 4) depths.push_back(4);
             if (deepest > 2) depths.push_back(2);
@@ -455,8 +458,8 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
             const int64_t tiles = 8 * ceil_div(s.M, 1024) * ceil_div(s.N, BN);
             split_candidates(tiles, m.n_sm, ceil_div(s.K + 7, 64), 2, &pks);
             int deepest = 0;
-            for (int st = 8; st >= 2; --st)
-                if (umma_smem_bytes(BN, 1, st) <= m.smem_bytes) { deepest = st; break; }
+            for (int st = kUmmaMaxStages; st >= 2; --st)
+                if (umma_smem_bytes(BN, 1, st, umma_a_box_rows(s, 1, true, false)) <= m.smem_bytes) { deepest = st; break; }
             for (int pk : pks) {
                 Config d;
                 d.family = ADAPT_FAM_UMMA_1CTA; d.BM = 128; d.BN = BN; d.BK = 64; d.cluster = 1;
@@ -471,8 +474,8 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
         const int64_t tiles = ceil_div(s.M, 128) * ceil_div(s.N, 56);
         split_candidates(tiles, m.n_sm, ceil_div(ceil_div(s.K, 8), 64), 1, &pks);
         int deepest = 0;
-        for (int st = 8; st >= 2; --st)
-            if (umma_smem_bytes(64, 1, st) <= m.smem_bytes) { deepest = st; break; }
+        for (int st = kUmmaMaxStages; st >= 2; --st)
+            if (umma_smem_bytes(64, 1, st, umma_a_box_rows(s, 1, false, true)) <= m.smem_bytes) { deepest = st; break; }
         for (int pk : pks) {
             Config d;
             d.family = ADAPT_FAM_UMMA_1CTA; d.BM = 128; d.BN = 64; d.BK = 64; d.cluster = 1;

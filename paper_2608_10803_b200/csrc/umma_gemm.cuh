@@ -127,9 +127,10 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
     static_assert(!B_CLS || BN == 64, "k-class mode uses 64-column windows");
     constexpr int TILE_N = B_CLS ? 56 : BN;               // output columns a tile owns
     constexpr int BN_CTA = BN / CG;                       // B columns this CTA loads
-    constexpr int A_BYTES = 128 * kUmmaBK * 2;
+    // the A region of a stage holds the rows one box brings (128, or fewer for a short K-major A)
+    const int A_BYTES = (CG == 2) ? 128 * kUmmaBK * 2 : p.a_tx_bytes;
     constexpr int B_BYTES = BN_CTA * kUmmaBK * 2;
-    constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    const int STAGE_BYTES = A_BYTES + B_BYTES;
     constexpr int NBUF = B_CLS ? 1 : ((512 / BN) < 4 ? (512 / BN) : 4);   // accumulator buffers in TMEM
     constexpr int TMEM_COLS = B_CLS ? 512 : NBUF * BN;    // k-class mode: eight class accumulators of 64 columns
     constexpr int PASSES = BN / 64;                       // 64-column epilogue passes per tile
@@ -319,6 +320,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
 #pragma unroll
                             for (int t = 0; t < 4; ++t) {
                                 const int r = lane + 32 * t;
+                                if (r * 128 >= A_BYTES) break;           // rows past the box are not part of the stage
                                 unsigned short* h = reinterpret_cast<unsigned short*>(genA + r * 128 + ((r & 7) << 4));
                                 for (int e = 0; e < sigma; ++e) h[e] = 0;
                             }

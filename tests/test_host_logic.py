@@ -125,8 +125,14 @@ def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
                 # capacity limits of Eq. 6
                 if c.family in (ab.FAM_UMMA_1CTA, ab.FAM_UMMA_2CTA):
                     bn_cta = c.BN // c.cluster
-                    smem = c.stages * (128 * 64 * 2 + bn_cta * 64 * 2)
-                    assert smem <= 227 * 1024
+                    # a stage holds the rows of A one box brings (128, or fewer for a short A) and BN columns of B
+                    a_rows = 128
+                    if c.srcA == 3:
+                        a_rows = min(128, -(-(-(-M // 8)) // 8) * 8)
+                    elif c.cluster == 1 and M < 128:
+                        a_rows = -(-M // 8) * 8
+                    smem = c.stages * (a_rows * 64 * 2 + bn_cta * 64 * 2)
+                    assert smem <= 227 * 1024 and 2 <= c.stages <= 15
                     assert 2 * c.BN <= 512 and c.BN % 16 == 0
                     assert c.P_k <= (-(-(-(-K // 8)) // 64) if c.srcB == 3 else -(-(K + 7) // 64))
                     # unaligned operands are never handed to TMA directly (row-major: K for A, N for B)
