@@ -47,8 +47,8 @@ static adapt_status_t fail(adapt_status_t st, const char* fmt, const char* detai
 struct MapSlot {
     const void* ptr = nullptr;
     int64_t pitch = 0;
-    int count = 0;            // 1, or 8 for the per-row-class maps of A
-    CUtensorMap map[8];
+    int count = 0;            // 1, or the number of per-class maps (8 or 16)
+    CUtensorMap map[16];
 };
 
 struct adapt_plan_s {
@@ -57,9 +57,10 @@ struct adapt_plan_s {
     bool noop = false;        // M == 0 or N == 0
     bool zero_fill = false;   // K == 0
     std::mutex mu;            // guards the tensor-map slots
-    MapSlot mapA[2], mapB[2];
-    int nextA = 0, nextB = 0;
+    MapSlot maps[3][2];       // per operand (kMapA, kMapB, kMapC): the two most recent base pointers
+    int next[3] = {0, 0, 0};
 };
+enum { kMapA = 0, kMapB = 1, kMapC = 2 };
 typedef adapt_plan_s Plan;
 
 namespace {
@@ -350,17 +351,17 @@ extern "C" int64_t adapt_launch_count(void) { return st().launches.load(); }
 // ---------------------------------------------------------------------------------------------
 // launch_map: (family, BN, A major, B major) -> compiled kernel
 // ---------------------------------------------------------------------------------------------
-typedef void (*UmmaKernel)(const TmapPack, const UmmaParams);
+typedef const void* UmmaKernel;     // the parameter pack's type depends on the kernel mode: launched through cudaLaunchKernelExC
 
 template <int CG>
 static UmmaKernel umma_lookup(int BN, bool a_mn, bool b_mn)
 {
 #define ADAPT_PICK(bn)                                                               \
     if (BN == bn) {                                                                  \
-        if (!a_mn && !b_mn) return umma_gemm_kernel<bn, false, false, CG, 0>;    \
-        if (!a_mn && b_mn) return umma_gemm_kernel<bn, false, true, CG, 0>;      \
-        if (a_mn && !b_mn) return umma_gemm_kernel<bn, true, false, CG, 0>;      \
-        return umma_gemm_kernel<bn, true, true, CG, 0>;                          \
+        if (!a_mn && !b_mn) return (const void*)umma_gemm_kernel<bn, false, false, CG, 0>;    \
+        if (!a_mn && b_mn) return (const void*)umma_gemm_kernel<bn, false, true, CG, 0>;      \
+        if (a_mn && !b_mn) return (const void*)umma_gemm_kernel<bn, true, false, CG, 0>;      \
+        return (const void*)umma_gemm_kernel<bn, true, true, CG, 0>;                          \
     }
     if constexpr (CG == 1) { ADAPT_PICK(64) }
     ADAPT_PICK(128)
@@ -372,12 +373,15 @@ static UmmaKernel umma_lookup(int BN, bool a_mn, bool b_mn)
 static UmmaKernel launch_map_umma(int family, int BN, bool a_mn, bool b_mn, int mode = 0)
 {
     if (mode == 1) {                     // row-major A read through per-row-class maps (1-CTA tiles, row-major B)
-        if (BN == 64) return umma_gemm_kernel<64, false, true, 1, 1>;
-        if (BN == 128) return umma_gemm_kernel<128, false, true, 1, 1>;
-        if (BN == 256) return umma_gemm_kernel<256, false, true, 1, 1>;
+        if (BN == 64) return (const void*)umma_gemm_kernel<64, false, true, 1, 1>;
+        if (BN == 128) return (const void*)umma_gemm_kernel<128, false, true, 1, 1>;
+        if (BN == 256) return (const void*)umma_gemm_kernel<256, false, true, 1, 1>;
+        if (BN == 80) return (const void*)umma_gemm_kernel<80, false, true, 1, 1>;      // 64 / 128 / 192 owned + 16 halo columns
+        if (BN == 144) return (const void*)umma_gemm_kernel<144, false, true, 1, 1>;
+        if (BN == 208) return (const void*)umma_gemm_kernel<208, false, true, 1, 1>;
         return nullptr;
     }
-    if (mode == 2) return BN == 64 ? umma_gemm_kernel<64, false, true, 1, 2> : nullptr;   // B through per-k-class maps
+    if (mode == 2) return BN == 64 ? (const void*)umma_gemm_kernel<64, false, true, 1, 2> : nullptr;   // B through per-k-class maps
     return family == ADAPT_FAM_UMMA_1CTA ? umma_lookup<1>(BN, a_mn, b_mn) : umma_lookup<2>(BN, a_mn, b_mn);
 }
 
@@ -415,12 +419,12 @@ extern "C" adapt_status_t adapt_init(int device)
                 for (int b = 0; b < 2; ++b) {
                     UmmaKernel k = launch_map_umma(fam, BN, a != 0, b != 0);
                     if (!k) continue;
-                    CUDA_TRY(cudaFuncSetAttribute((const void*)k, cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
+                    CUDA_TRY(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
                 }
-    for (int BN : {64, 128, 256})
-        CUDA_TRY(cudaFuncSetAttribute((const void*)launch_map_umma(ADAPT_FAM_UMMA_1CTA, BN, false, true, 1),
+    for (int BN : {64, 128, 256, 80, 144, 208})
+        CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_1CTA, BN, false, true, 1),
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
-    CUDA_TRY(cudaFuncSetAttribute((const void*)launch_map_umma(ADAPT_FAM_UMMA_1CTA, 64, false, true, 2),
+    CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_1CTA, 64, false, true, 2),
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
     S.device = device;
     S.inited = true;
@@ -518,14 +522,14 @@ adapt_status_t encode_map(State& S, CUtensorMap* map, const void* base, int dtyp
     return ADAPT_OK;
 }
 
-adapt_status_t cached_map(State& S, Plan* pl, bool isA, const void* base, int64_t inner, int64_t outer, int64_t pitch,
+adapt_status_t cached_map(State& S, Plan* pl, int which, const void* base, int64_t inner, int64_t outer, int64_t pitch,
                           int box_inner, int box_outer, CUtensorMap* out)
 {
     std::lock_guard<std::mutex> lock(pl->mu);
-    MapSlot* slots = isA ? pl->mapA : pl->mapB;
+    MapSlot* slots = pl->maps[which];
     for (int i = 0; i < 2; ++i)
         if (slots[i].ptr == base && slots[i].pitch == pitch && slots[i].count == 1) { *out = slots[i].map[0]; return ADAPT_OK; }
-    int& next = isA ? pl->nextA : pl->nextB;
+    int& next = pl->next[which];
     MapSlot& sl = slots[next];
     next ^= 1;
     adapt_status_t r = encode_map(S, &sl.map[0], base, pl->s.dtype, inner, outer, pitch, box_inner, box_outer);
@@ -537,32 +541,45 @@ adapt_status_t cached_map(State& S, Plan* pl, bool isA, const void* base, int64_
     return ADAPT_OK;
 }
 
-// Eight maps of a row-major matrix (rows x cols, cols % 8 != 0, 16-byte aligned base), one per row class
-// j = row % 8: base rounded down to 16 bytes, rows 16*cols bytes apart, inner extent cols + sigma_j so that
-// the tail is zero-filled; sigma_j = elements between the rounded base and the start of row j.  Used for
-// A (rows = M, cols = K) and, in k-class mode, for B (rows = K, cols = N).
-adapt_status_t cached_class_maps(State& S, Plan* pl, bool isA, const void* base_ptr, int64_t rows_total, int64_t cols,
-                                 int box_rows, CUtensorMap* out, int* sigma)
+// Per-class maps of a row-major matrix (rows x cols, 16-byte aligned base): class j holds the rows with
+// row % ncls == j, which all start the same distance sigma_j (elements) after an `align`-byte boundary
+// (ncls * cols * 2 is a multiple of `align`: ncls = 8 for 16 bytes, 16 for 32).  Map j: base rounded down
+// to that boundary, rows ncls * cols * 2 bytes apart, inner extent cols + sigma_j, so a load reads zeros
+// past the row's end.  Used for A (rows = M, cols = K), in k-class mode for B (rows = K, cols = N), and for
+// C's stores: there `whole_units` cuts the extent down to whole `align`-byte units (returned in
+// extent[]), because TMA clips a stored row in 16-byte units and would overwrite the next row's head.
+adapt_status_t cached_class_maps(State& S, Plan* pl, int which, const void* base_ptr, int64_t rows_total, int64_t cols,
+                                 int box_rows, int ncls, int align, bool whole_units, CUtensorMap* out, int* sigma,
+                                 int* extent = nullptr)
 {
     std::lock_guard<std::mutex> lock(pl->mu);
-    for (int j = 0; j < 8; ++j) sigma[j] = (int)(((2 * j * cols) & 15) / 2);
-    MapSlot* slots = isA ? pl->mapA : pl->mapB;
+    const int unit = align / 2;                               // elements per aligned unit
+    for (int j = 0; j < ncls; ++j) {
+        sigma[j] = (int)(((2 * j * cols) & (align - 1)) / 2);
+        if (extent) extent[j] = (int)(whole_units ? (cols + sigma[j]) / unit * unit : cols + sigma[j]);
+    }
+    MapSlot* slots = pl->maps[which];
     for (int i = 0; i < 2; ++i)
-        if (slots[i].ptr == base_ptr && slots[i].count == 8) { memcpy(out, slots[i].map, 8 * sizeof(CUtensorMap)); return ADAPT_OK; }
-    int& next = isA ? pl->nextA : pl->nextB;
+        if (slots[i].ptr == base_ptr && slots[i].pitch == cols && slots[i].count == ncls) {
+            memcpy(out, slots[i].map, ncls * sizeof(CUtensorMap));
+            return ADAPT_OK;
+        }
+    int& next = pl->next[which];
     MapSlot& sl = slots[next];
     next ^= 1;
     sl.ptr = nullptr;
-    for (int j = 0; j < 8; ++j) {
-        const uint8_t* base = (const uint8_t*)base_ptr + ((2 * j * cols) & ~(int64_t)15);
-        const int64_t rows = std::max<int64_t>(1, ceil_div(rows_total - j, 8));
-        adapt_status_t r = encode_map(S, &sl.map[j], base, pl->s.dtype, cols + sigma[j], rows, 8 * cols, 64, box_rows);
+    for (int j = 0; j < ncls; ++j) {
+        const uint8_t* base = (const uint8_t*)base_ptr + ((2 * j * cols) & ~(int64_t)(align - 1));
+        const int64_t rows = std::max<int64_t>(1, ceil_div(rows_total - j, ncls));
+        int64_t inner = cols + sigma[j];
+        if (whole_units) inner = std::max<int64_t>(unit, inner / unit * unit);
+        adapt_status_t r = encode_map(S, &sl.map[j], base, pl->s.dtype, inner, rows, (int64_t)ncls * cols, 64, box_rows);
         if (r != ADAPT_OK) return r;
     }
     sl.ptr = base_ptr;
     sl.pitch = cols;
-    sl.count = 8;
-    memcpy(out, sl.map, 8 * sizeof(CUtensorMap));
+    sl.count = ncls;
+    memcpy(out, sl.map, ncls * sizeof(CUtensorMap));
     return ADAPT_OK;
 }
 
@@ -592,15 +609,17 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     const Shape& s = pl->s;
     const Config& c = pl->c;
     const bool b_mn = s.layoutB == ADAPT_ROW_MAJOR;       // N contiguous
-    // the copy-free class modes need 16-byte aligned base pointers; otherwise fall back to re-pitched copies
-    const bool classesA = c.srcA == ADAPT_SRC_TMA_CLASSES && ((uintptr_t)A & 15) == 0;
+    // class tiles read A through per-row-class maps: in place when its base is 16-byte aligned (whatever K
+    // is), else over a re-pitched copy; the k-class views of B need an aligned base, else B is copied
+    const bool classesA = c.srcA == ADAPT_SRC_TMA_CLASSES;
     const bool kclsB = c.srcB == ADAPT_SRC_TMA_CLASSES && ((uintptr_t)B & 15) == 0;
     const bool a_mn = !kclsB && s.layoutA == ADAPT_COL_MAJOR;   // M contiguous (the regrouped A' is always K-major)
     const int64_t Kc = round_up(ceil_div(s.K, 8), 64);          // k-class mode: padded class segment of A'
     const int64_t inA = kclsB ? 8 * Kc : (a_mn ? s.M : s.K), outA = a_mn ? s.K : s.M;
     const int64_t inB = b_mn ? s.N : s.K, outB = b_mn ? s.K : s.N;
     const bool a_inner_ok = (s.layoutA == ADAPT_COL_MAJOR ? s.M : s.K) % 8 == 0;
-    const bool padA = !classesA && !kclsB && (!a_inner_ok || ((uintptr_t)A & 15) != 0);
+    const bool padA = classesA ? ((uintptr_t)A & 15) != 0
+                               : (!kclsB && (!a_inner_ok || ((uintptr_t)A & 15) != 0));
     const bool padB = !kclsB && (inB % 8 != 0 || ((uintptr_t)B & 15) != 0);
     const int64_t pitchA = padA ? padded_pitch(inA) : inA;
     const int64_t pitchB = padB ? padded_pitch(inB) : inB;
@@ -608,15 +627,17 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     const size_t szB = padB ? (size_t)round_up(outB * pitchB * 2, 256) : 0;
 
     const int cg = c.cluster;
-    TmapPack maps;
+    const bool halo = classesA && c.BN % 64 != 0;           // class tiles with 16 halo columns (C's rows off 32-byte boundaries)
+    const int ncls = halo ? 16 : 8;                         // row classes of a class tile
+    struct { CUtensorMap a[16], b[8], c[16]; } maps;
     UmmaParams p;
     int a_box_rows = 128;
     memset(p.a_sigma, 0, sizeof(p.a_sigma));
     memset(p.b_sigma, 0, sizeof(p.b_sigma));
     p.cls_kc = (int)Kc;
     p.M = (int)s.M; p.N = (int)s.N; p.K = (int)s.K;
-    // a plan made for class tiles that has to fall back to copies (unaligned pointer) uses plain tiles
-    p.P_m = (c.srcA == ADAPT_SRC_TMA_CLASSES && !classesA) ? (int)ceil_div(s.M, c.BM) : c.P_m;
+    p.P_m = c.P_m;
+    // a plan made for k-class views that has to fall back to a copy of B (unaligned pointer) uses plain tiles
     p.P_n = (c.srcB == ADAPT_SRC_TMA_CLASSES && !kclsB) ? (int)ceil_div(s.N, c.BN) : c.P_n;
     p.kb_total = kclsB ? (int)(Kc / kUmmaBK) : (int)ceil_div(s.K + (classesA ? 7 : 0), kUmmaBK);
     p.kb_per_split = (int)ceil_div(p.kb_total, c.P_k);
@@ -651,19 +672,36 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
 
     // K-major operand: one box of 64 k x (rows this CTA owns); MN-major operand: boxes of 64 x 64
     if (classesA) {
-        a_box_rows = umma_a_box_rows(s, cg, true, false);       // rows of the largest class
-        if ((r = cached_class_maps(S, pl, true, A, s.M, s.K, a_box_rows, maps.a, p.a_sigma)) != ADAPT_OK) return r;
+        a_box_rows = umma_a_box_rows(s, cg, ncls, false);       // rows of the largest class
+        if ((r = cached_class_maps(S, pl, kMapA, a_src, s.M, padA ? pitchA : s.K, a_box_rows, ncls, 16, false, maps.a,
+                                   p.a_sigma)) != ADAPT_OK) return r;
     } else {
         // a K-major A of fewer than 128 rows is loaded with a box of just those rows (rounded up to 8):
         // the rows of the stage it leaves untouched only feed accumulator rows that are never stored
-        a_box_rows = umma_a_box_rows(s, cg, false, kclsB);
-        if ((r = cached_map(S, pl, true, a_src, inA, outA, pitchA, 64, a_mn ? 64 : a_box_rows, &maps.a[0])) != ADAPT_OK) return r;
+        a_box_rows = umma_a_box_rows(s, cg, 0, kclsB);
+        if ((r = cached_map(S, pl, kMapA, a_src, inA, outA, pitchA, 64, a_mn ? 64 : a_box_rows, &maps.a[0])) != ADAPT_OK) return r;
     }
     if (kclsB) {
         // rows of B (K x N, N % 8 != 0) by class k % 8: the same construction as A's row classes, 64 x 64 boxes
-        if ((r = cached_class_maps(S, pl, false, B, s.K, s.N, 64, maps.b, p.b_sigma)) != ADAPT_OK) return r;
+        if ((r = cached_class_maps(S, pl, kMapB, B, s.K, s.N, 64, 8, 16, false, maps.b, p.b_sigma)) != ADAPT_OK) return r;
     } else {
-        if ((r = cached_map(S, pl, false, b_src, inB, outB, pitchB, 64, b_mn ? 64 : c.BN / cg, &maps.b[0])) != ADAPT_OK) return r;
+        if ((r = cached_map(S, pl, kMapB, b_src, inB, outB, pitchB, 64, b_mn ? 64 : c.BN / cg, &maps.b[0])) != ADAPT_OK) return r;
+    }
+
+    // 16-bit output leaves through TMA stores (boxes of 64 elements x 32 rows, one epilogue warp) when the
+    // boxes cover whole 32-byte sectors: rows of C on 32-byte boundaries (N % 16 == 0; class tiles then use
+    // one map per row class), or halo class tiles, whose maps shift each class onto such a boundary
+    p.c_mode = 0;
+    memset(p.c_sigma, 0, sizeof(p.c_sigma));
+    memset(p.c_extent, 0, sizeof(p.c_extent));
+    if (p.P_k == 1 && !kclsB && (halo ? ((uintptr_t)C & 15) == 0 : (((uintptr_t)C & 31) == 0 && s.N % 16 == 0))) {
+        if (classesA) {
+            if ((r = cached_class_maps(S, pl, kMapC, C, s.M, s.N, 32, ncls, 32, true, maps.c, p.c_sigma, p.c_extent)) != ADAPT_OK)
+                return r;
+        } else {
+            if ((r = cached_map(S, pl, kMapC, C, s.N, s.M, s.N, 64, 32, &maps.c[0])) != ADAPT_OK) return r;
+        }
+        p.c_mode = 1;
     }
 
     p.dtype = s.dtype;
@@ -698,7 +736,22 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    CUDA_TRY(cudaLaunchKernelEx(&cfg, k, maps, p));
+    // the kernel takes the maps its mode uses
+    TmapPackT<0> pack0;
+    TmapPackT<1> pack1;
+    TmapPackT<2> pack2;
+    void* args[2] = {nullptr, &p};
+    if (classesA) {
+        memcpy(pack1.a, maps.a, sizeof(pack1.a)); pack1.b[0] = maps.b[0]; memcpy(pack1.c, maps.c, sizeof(pack1.c));
+        args[0] = &pack1;
+    } else if (kclsB) {
+        pack2.a[0] = maps.a[0]; memcpy(pack2.b, maps.b, sizeof(pack2.b)); pack2.c[0] = maps.c[0];
+        args[0] = &pack2;
+    } else {
+        pack0.a[0] = maps.a[0]; pack0.b[0] = maps.b[0]; pack0.c[0] = maps.c[0];
+        args[0] = &pack0;
+    }
+    CUDA_TRY(cudaLaunchKernelExC(&cfg, k, args));
     S.launches.fetch_add(1, std::memory_order_relaxed);
     if (p.P_k > 1) return launch_reduce(S, partial, C, s.M, s.N, p.P_k, s.dtype, stream);
     return ADAPT_OK;

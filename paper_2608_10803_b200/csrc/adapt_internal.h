@@ -34,7 +34,8 @@ struct Calib {
     double umma_fixed_us = 2.5;         // barrier init, TMEM alloc, first load, last drain, TMEM free
     // drain of one output tile through the epilogue warps (overlaps the next tile's main loop):
     // fixed part per tile + part per KB written; rows of C that are not 16-byte aligned cost more
-    double epi_tile_fixed_us = 0.32, epi_us_per_kb = 0.0385;
+    double epi_tile_fixed_us = 0.2, epi_us_per_kb = 0.0275;          // TMA stores (40000 x 40000 x 8: 4.8 TB/s)
+    double epi_partial_fixed_us = 0.32, epi_partial_us_per_kb = 0.0385;   // fp32 partials, stored by the epilogue threads
     double epi_tile_fixed_unaligned_us = 1.45, epi_us_per_kb_unaligned = 0.054;
     double simt_flops = 15e12;          // CUDA-core tile kernel (1000^3: 17e12)
     double simt_fixed_us = 1.5;
@@ -101,29 +102,34 @@ inline int64_t padded_pitch(int64_t inner) { return round_up(inner, 8); }
 const Calib& default_calib();
 
 // Shared-memory layout of the tcgen05 kernels, used by the capacity check and by the launcher:
-// S stages of (A: 128 x 64, B: BN/cluster x 64) 16-bit, a barrier block, the epilogue staging
-// (one 144-byte row per epilogue thread), and slack to align the stages to 1024 B.
+// S stages of (A: box rows x 64, B: BN/cluster x 64) 16-bit, a barrier block, the epilogue staging
+// (8 KB per epilogue warp), and slack to align the stages to 1024 B.
 constexpr int kSkinnyKChunk = 512;   // k values the warp-level kernel stages per chunk; its k splits are whole chunks
-constexpr int kUmmaBarrierBytes = 512;
+constexpr int kUmmaBarrierBytes = 1024;  // keeps the epilogue staging 1024-byte aligned (swizzled TMA boxes)
 constexpr int kUmmaMaxStages = 15;
 constexpr int kUmmaEpilogueWarps = 8;
 constexpr int kUmmaStageRowBytes = 144;   // 72 16-bit elements: 64 columns + up to 7 of alignment shift
+constexpr int kUmmaWarpStagingBytes = 8192;   // per epilogue warp: two 32 x 128 B boxes for TMA stores, or 32 shifted rows
 inline int umma_smem_bytes(int BN, int cluster, int stages, int a_rows = 128)
 {
-    return stages * (a_rows * 64 * 2 + (BN / cluster) * 64 * 2) + kUmmaBarrierBytes +
-           kUmmaEpilogueWarps * 32 * kUmmaStageRowBytes + 1024;
+    return stages * (a_rows * 64 * 2 + (int)round_up(BN / cluster, 64) * 64 * 2) + kUmmaBarrierBytes +
+           kUmmaEpilogueWarps * kUmmaWarpStagingBytes + 1024;
 }
 
 // Rows of A one TMA box brings per stage (a multiple of 8, so the stage stays a multiple of 1024 B).
 // A K-major A of fewer than 128 rows is loaded with a box of just those rows, and the stage's A
 // region shrinks with it: the MMA still reads 128 rows, but the rows past the box only feed
 // accumulator rows that are never stored.  Class tiles hold every 8th row of up to 1024.
-inline int umma_a_box_rows(const Shape& s, int cluster, bool row_classes, bool k_classes)
+inline int umma_a_box_rows(const Shape& s, int cluster, int row_classes, bool k_classes)
 {
     const bool a_mn = !k_classes && s.layoutA == ADAPT_COL_MAJOR;
-    if (row_classes) return s.M < 1024 ? (int)std::min<int64_t>(128, round_up(ceil_div(s.M, 8), 8)) : 128;
+    if (row_classes)    // 8 or 16 classes: a tile holds every 8th (16th) row of up to 1024 (2048)
+        return s.M < 128 * row_classes ? (int)std::min<int64_t>(128, round_up(ceil_div(s.M, row_classes), 8)) : 128;
     if (!a_mn && cluster == 1 && s.M < 128) return (int)round_up(s.M, 8);
     return 128;
 }
+
+// Row classes of a configuration's tiles: 0 (plain tiles), 8 (class tiles), 16 (class tiles with halo columns).
+inline int umma_row_classes(int srcA, int BN) { return srcA != ADAPT_SRC_TMA_CLASSES ? 0 : (BN % 64 ? 16 : 8); }
 
 }  // namespace adapt

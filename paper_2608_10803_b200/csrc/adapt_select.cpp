@@ -190,8 +190,8 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
 
     // per-SM stage: each CTA loads its 128 rows of A and its share of the BN columns of B
     const double bn_per_cta = (double)c.BN / c.cluster;
-    const double a_rows = umma_a_box_rows(s, c.cluster, c.srcA == ADAPT_SRC_TMA_CLASSES, kclasses);
-    const double stage_bytes = 2.0 * c.BK * (a_rows + bn_per_cta);
+    const double a_rows = umma_a_box_rows(s, c.cluster, umma_row_classes(c.srcA, c.BN), kclasses);
+    const double stage_bytes = 2.0 * c.BK * (a_rows + (double)round_up((int64_t)bn_per_cta, 64));
     // One SM pulls operands that other SMs also use from L2 at l2_bw_per_sm (a little less through
     // the strided row-class views); a stream that comes from HBM and is used once is bounded by the
     // bytes one SM keeps in flight, about hbm_bw_per_sm.  The second case only shows in partial waves.
@@ -200,16 +200,25 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     double sm_rate = cal.l2_bw_per_sm * (c.srcA == ADAPT_SRC_TMA_CLASSES ? cal.class_view_sm_eff : 1.0);
     if (mem_bound && c.srcA == ADAPT_SRC_TMA_CLASSES) sm_rate = std::min(sm_rate, cal.hbm_bw_per_sm);   // measured for the views only
     double tM = stage_bytes / sm_rate * 1e6;
-    double eta = c.BN >= 256 ? 1.0 : (c.BN >= 128 ? cal.eta_mma_bn128 : cal.eta_mma_bn64);
+    // relative tensor efficiency, measured at BN = 64, 128, 256 and interpolated for the halo tiles between them
+    double eta = c.BN >= 256 ? 1.0
+               : c.BN >= 128 ? cal.eta_mma_bn128 + (1.0 - cal.eta_mma_bn128) * (c.BN - 128) / 128.0
+                             : cal.eta_mma_bn64 + (cal.eta_mma_bn128 - cal.eta_mma_bn64) * (c.BN - 64) / 64.0;
     if (c.cluster == 2) eta *= cal.eta_2cta;
     const double tP = 2.0 * 128.0 * c.BN * c.BK / (cal.tensor_flops / m.n_sm * eta) * 1e6;
     // Drain of one tile (the paper's T_drain: FixPipe cast and write).  With two or more TMEM
     // accumulators it overlaps the next tile's main loop, so a tile costs max(L * II, T_drain).
-    const bool c_aligned = s.N % 8 == 0;
-    const double out_tile_kb = (c.P_k > 1 ? 4.0 : 2.0) * 128.0 * c.BN / 1024.0;
-    const double t_drain = (c.P_k > 1 || c_aligned)
-                               ? cal.epi_tile_fixed_us + cal.epi_us_per_kb * out_tile_kb
-                               : cal.epi_tile_fixed_unaligned_us + cal.epi_us_per_kb_unaligned * out_tile_kb;
+    // 16-bit tiles leave through TMA stores when C's rows are 16-byte aligned, or when class tiles with
+    // halo columns make their misalignment uniform; otherwise the epilogue threads store them, and fp32
+    // partials always go that way
+    const bool halo = c.BN % 64 != 0;
+    const int own_n = halo ? c.BN - 16 : c.BN;
+    const double out_tile_kb = (c.P_k > 1 ? 4.0 : 2.0) * 128.0 * own_n / 1024.0;
+    double t_drain;
+    if (c.P_k > 1) t_drain = cal.epi_partial_fixed_us + cal.epi_partial_us_per_kb * out_tile_kb;
+    else if (s.N % 16 == 0 || halo) t_drain = cal.epi_tile_fixed_us + cal.epi_us_per_kb * out_tile_kb;
+    else if (s.N % 8 == 0) t_drain = cal.epi_partial_fixed_us + cal.epi_partial_us_per_kb * out_tile_kb;   // aligned 16-byte stores by the threads
+    else t_drain = cal.epi_tile_fixed_unaligned_us + cal.epi_us_per_kb_unaligned * out_tile_kb;
     // Delta_dep (Eq. 9): with S stages only S-1 loads are in flight while one is consumed, so a
     // slice cannot issue faster than latency / (S-1); one stage serialises load and compute.
     double pipe;
@@ -284,7 +293,9 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     if (c.BK != 64) return false;
     if (c.family == ADAPT_FAM_UMMA_1CTA) {
         if (c.BM != 128 || c.cluster != 1) return false;
-        if (c.BN != 64 && c.BN != 128 && c.BN != 256) return false;
+        const bool halo_bn = c.BN == 80 || c.BN == 144 || c.BN == 208;    // class tiles: 64 / 128 / 192 owned + 16 halo columns
+        if (c.BN != 64 && c.BN != 128 && c.BN != 256 && !halo_bn) return false;
+        if (halo_bn && (c.srcA != ADAPT_SRC_TMA_CLASSES || s.N % 16 == 0 || s.M < 16)) return false;
     } else {
         if (c.BM != 256 || c.cluster != 2) return false;
         if (c.BN != 128 && c.BN != 256) return false;
@@ -293,7 +304,7 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     if (2 * c.BN > m.tmem_cols) return false;                       // at least two accumulator buffers in TMEM
     if (c.stages < 1 || c.stages > kUmmaMaxStages) return false;
     c.smem_bytes = umma_smem_bytes(c.BN, c.cluster, c.stages,
-                                   umma_a_box_rows(s, c.cluster, c.srcA == ADAPT_SRC_TMA_CLASSES, c.srcB == ADAPT_SRC_TMA_CLASSES));
+                                   umma_a_box_rows(s, c.cluster, umma_row_classes(c.srcA, c.BN), c.srcB == ADAPT_SRC_TMA_CLASSES));
     if (c.smem_bytes > m.smem_bytes) return false;
     // in class mode the k index of a tile is shifted by up to 7 elements
     // k-class mode splits the blocks of one class; in row-class mode the k index is shifted by up to 7
@@ -316,12 +327,15 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     if (classes) {
         // rows of one residue class share their misalignment: row-major A and B, one CTA per tile
         if (c.family != ADAPT_FAM_UMMA_1CTA || s.layoutA != ADAPT_ROW_MAJOR || s.layoutB != ADAPT_ROW_MAJOR) return false;
-        if (aligned16(innerA(s)) || s.M < 8) return false;
+        // they pay when A's rows are unaligned (no copy), or when C's rows do not start on 32-byte sector
+        // boundaries (halo tiles of 16 classes: uniform misalignment per tile, whole-sector TMA stores)
+        if ((aligned16(innerA(s)) && c.BN % 64 == 0) || s.M < 8) return false;
     }
     if (c.srcA == ADAPT_SRC_PAD_COPY && aligned16(innerA(s)) && !kclasses) return false;    // nothing to pad
     if (c.srcB == ADAPT_SRC_PAD_COPY && aligned16(innerB(s))) return false;
-    c.P_m = classes ? (int)(8 * ceil_div(s.M, 8 * c.BM)) : (int)ceil_div(s.M, c.BM);   // class tiles: 8 per 1024 rows
-    c.P_n = (int)ceil_div(s.N, kclasses ? 56 : c.BN);
+    const int ncls = umma_row_classes(c.srcA, c.BN);
+    c.P_m = classes ? (int)(ncls * ceil_div(s.M, ncls * c.BM)) : (int)ceil_div(s.M, c.BM);   // class tiles: 8 per 1024 rows, 16 per 2048
+    c.P_n = (int)ceil_div(s.N, kclasses ? 56 : (c.BN % 64 ? c.BN - 16 : c.BN));
     if ((int64_t)c.P_m * c.P_n * c.P_k > (int64_t)1 << 30) return false;
     c.persistent = 1;
     return true;
@@ -431,7 +445,7 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
             // ring depth: the deepest that fits, and a double buffer (Eq. 13) for comparison
             Config probe;
             probe.family = fam; probe.BM = BM; probe.BN = BN; probe.BK = 64; probe.cluster = cluster;
-            const int a_rows = umma_a_box_rows(s, cluster, false, false);
+            const int a_rows = umma_a_box_rows(s, cluster, 0, false);
             int deepest = 0;
             for (int st = kUmmaMaxStages; st >= 2; --st) {
                 probe.stages = st;
@@ -453,13 +467,16 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
     }
     // --- tcgen05, A read in place through per-row-class views (row-major A, K % 8 != 0): 8 class
     //     tiles per 1024 rows, so the split counts are drawn from that tile count ---
-    if (srcA == ADAPT_SRC_PAD_COPY && s.layoutA == ADAPT_ROW_MAJOR && s.layoutB == ADAPT_ROW_MAJOR && s.M >= 8) {
-        for (int BN : {64, 128, 256}) {
-            const int64_t tiles = 8 * ceil_div(s.M, 1024) * ceil_div(s.N, BN);
+    if ((srcA == ADAPT_SRC_PAD_COPY || s.N % 16 != 0) && s.layoutA == ADAPT_ROW_MAJOR && s.layoutB == ADAPT_ROW_MAJOR && s.M >= 8) {
+        for (int BN : {64, 128, 256, 80, 144, 208}) {
+            const bool halo = BN % 64 != 0;
+            if (halo && (s.N % 16 == 0 || s.M < 16)) continue;             // halo tiles serve a C off 32-byte boundaries only
+            if (!halo && srcA != ADAPT_SRC_PAD_COPY) continue;             // aligned A: class tiles only for their stores
+            const int64_t tiles = (halo ? 16 * ceil_div(s.M, 2048) : 8 * ceil_div(s.M, 1024)) * ceil_div(s.N, halo ? BN - 16 : BN);
             split_candidates(tiles, m.n_sm, ceil_div(s.K + 7, 64), 2, &pks);
             int deepest = 0;
             for (int st = kUmmaMaxStages; st >= 2; --st)
-                if (umma_smem_bytes(BN, 1, st, umma_a_box_rows(s, 1, true, false)) <= m.smem_bytes) { deepest = st; break; }
+                if (umma_smem_bytes(BN, 1, st, umma_a_box_rows(s, 1, BN % 64 ? 16 : 8, false)) <= m.smem_bytes) { deepest = st; break; }
             for (int pk : pks) {
                 Config d;
                 d.family = ADAPT_FAM_UMMA_1CTA; d.BM = 128; d.BN = BN; d.BK = 64; d.cluster = 1;
@@ -475,7 +492,7 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
         split_candidates(tiles, m.n_sm, ceil_div(ceil_div(s.K, 8), 64), 1, &pks);
         int deepest = 0;
         for (int st = kUmmaMaxStages; st >= 2; --st)
-            if (umma_smem_bytes(64, 1, st, umma_a_box_rows(s, 1, false, true)) <= m.smem_bytes) { deepest = st; break; }
+            if (umma_smem_bytes(64, 1, st, umma_a_box_rows(s, 1, 0, true)) <= m.smem_bytes) { deepest = st; break; }
         for (int pk : pks) {
             Config d;
             d.family = ADAPT_FAM_UMMA_1CTA; d.BM = 128; d.BN = 64; d.BK = 64; d.cluster = 1;

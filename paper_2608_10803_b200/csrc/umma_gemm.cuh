@@ -40,9 +40,14 @@ struct UmmaParams {
     float* partial;                  // fp32 [P_k][M][Np], Np = N rounded up to 4 (used when P_k > 1)
     int Np;                          // row pitch of the partials in elements
     int a_tx_bytes;                  // bytes one TMA load of A delivers per stage and CTA (a short box when M < 128)
-    int a_sigma[8];
+    int a_sigma[16];                 // class mode: shift (elements) of row class j against its 16-byte aligned base
     int b_sigma[8];                  // k-class mode: column shift of B's row class j = k % 8
-    int cls_kc;                      // k-class mode: padded length of one class segment of A' (multiple of 64)                  // class mode: shift (elements) of row class j = row % 8 against its 16-byte aligned base
+    int cls_kc;                      // k-class mode: padded length of one class segment of A' (multiple of 64)
+    int c_mode;                      // 16-bit output: 0 = stores by the epilogue threads (any N, any alignment),
+                                     // 1 = TMA stores through the maps of C (rows of C, or of the tile's row class,
+                                     //     start on 32-byte boundaries; class tiles with 16 halo columns shift them there)
+    int c_sigma[16];                 // halo class tiles: shift (elements) of C's row class j against its 32-byte aligned base
+    int c_extent[16];                // ... and the elements of a shifted row of that class that lie in whole 32-byte units
     unsigned int* status;            // device status word: bit 0 = a bounded wait expired
     unsigned long long* trace;       // timestamp trace of CTA 0 (diagnostic builds only), else null
 };
@@ -59,11 +64,16 @@ struct UmmaParams {
 #define ADAPT_TRACE(ev, unit) do { } while (0)
 #endif
 
-// Tensor maps of one launch.  a[0] is the map of A; in class mode (A_CLS) a[j] is the map of the
-// rows of A with row % 8 == j (see the kernel comment).
-struct TmapPack {
-    CUtensorMap a[8];
-    CUtensorMap b[8];         // b[0] is the map of B; in k-class mode b[j] is the map of the k-rows with k % 8 == j
+// Tensor maps of one launch, sized by the kernel mode (the pack is a kernel parameter, so the plain mode
+// passes three maps, not forty).  a[0] is the map of A; in class mode a[j] is the map of the rows of A in
+// row class j (see the kernel comment).  b[0] is the map of B; in k-class mode b[j] is the map of the
+// k-rows with k % 8 == j.  c[] are the maps of C for the TMA-store epilogue (c_mode != 0): c[0], or one
+// per row class.
+template <int MODE>
+struct TmapPackT {
+    CUtensorMap a[MODE == 1 ? 16 : 1];
+    CUtensorMap b[MODE == 2 ? 8 : 1];
+    CUtensorMap c[MODE == 1 ? 16 : 1];
 };
 
 // unit index -> (m block, n block, split).  Units of one output tile are adjacent in split;
@@ -119,23 +129,31 @@ __device__ __forceinline__ unsigned short cast16(float a, int dtype)
 // Columns of a buffer left of sigma_j hold products with the previous row's tail and are never read.
 template <int BN, bool A_MN, bool B_MN, int CG, int MODE>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
-umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
+umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams p)
 {
     constexpr bool A_CLS = MODE == 1;
     constexpr bool B_CLS = MODE == 2;
     static_assert(MODE == 0 || (!A_MN && B_MN && CG == 1), "class modes: K-major A, row-major B, one CTA per tile");
     static_assert(!B_CLS || BN == 64, "k-class mode uses 64-column windows");
-    constexpr int TILE_N = B_CLS ? 56 : BN;               // output columns a tile owns
+    // HALO: class tiles for a C whose rows do not start on 32-byte boundaries (N % 16 != 0) own 32-byte
+    // units of the shifted rows instead of columns, so they compute 16 columns more than they own (see
+    // the epilogue); they use 16 row classes, since rows 16 apart share their offset from such a boundary
+    constexpr bool HALO = A_CLS && (BN % 64 != 0);
+    static_assert(BN % 64 == 0 || (A_CLS && (BN - 16) % 64 == 0), "BN is a multiple of 64, plus 16 halo columns for class tiles");
+    constexpr int NCLS = HALO ? 16 : 8;                   // row classes of a class tile: rows NCLS*128*g + j + NCLS*i
+    constexpr int TILE_N = B_CLS ? 56 : (HALO ? BN - 16 : BN);   // output columns (HALO: chunk-aligned elements) a tile owns
     constexpr int BN_CTA = BN / CG;                       // B columns this CTA loads
     // the A region of a stage holds the rows one box brings (128, or fewer for a short K-major A)
     const int A_BYTES = (CG == 2) ? 128 * kUmmaBK * 2 : p.a_tx_bytes;
-    constexpr int B_BYTES = BN_CTA * kUmmaBK * 2;
+    constexpr int B_BOXES = (BN_CTA + 63) / 64;           // row-major B arrives in boxes of 64 columns
+    constexpr int B_BYTES = B_BOXES * 64 * kUmmaBK * 2;
     const int STAGE_BYTES = A_BYTES + B_BYTES;
     constexpr int NBUF = B_CLS ? 1 : ((512 / BN) < 4 ? (512 / BN) : 4);   // accumulator buffers in TMEM
-    constexpr int TMEM_COLS = B_CLS ? 512 : NBUF * BN;    // k-class mode: eight class accumulators of 64 columns
-    constexpr int PASSES = BN / 64;                       // 64-column epilogue passes per tile
+    constexpr int TMEM_COLS = (B_CLS || HALO) ? 512 : NBUF * BN;    // k-class mode: eight class accumulators of 64 columns
+    constexpr int PASSES = (TILE_N + 63) / 64;            // 64-column epilogue passes per tile
     static_assert(TMEM_COLS == 256 || TMEM_COLS == 512, "TMEM allocation is a power of two");
-    static_assert(BN_CTA % 64 == 0, "B is loaded in 64-column boxes");
+    static_assert(NBUF * BN <= TMEM_COLS, "accumulators fit the allocation");
+    static_assert(B_MN || BN_CTA % 64 == 0, "a K-major B tile is one box of BN rows");
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;   // swizzle atoms are 1024-byte aligned
@@ -206,8 +224,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
                 const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
                 // A rows of this CTA: consecutive rows, or in class mode rows 1024*g + j + 8*i read through
                 // map j at class-row index 128*g
-                const int cls = A_CLS ? (mb & 7) : 0;
-                const int row0 = A_CLS ? (mb >> 3) * 128 : mb * (128 * CG) + (int)cta_rank * 128;
+                const int cls = A_CLS ? (mb % NCLS) : 0;
+                const int row0 = A_CLS ? (mb / NCLS) * 128 : mb * (128 * CG) + (int)cta_rank * 128;
                 const int kshift = A_CLS ? p.a_sigma[cls] : 0;                // B's k-rows lag A's kappa by sigma
                 const CUtensorMap* tmA = &maps.a[cls];
                 const CUtensorMap* tmB = &maps.b[0];
@@ -220,7 +238,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
                             const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
                             ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(p.a_tx_bytes + B_BYTES));
                             ptx::tma_load_2d(sA, tmA, full_bar + 8u * stage, j * p.cls_kc + kb * kUmmaBK, row0);
-                            ptx::tma_load_2d(sA + A_BYTES, &maps.b[j], full_bar + 8u * stage, col0, kb * kUmmaBK);
+                            ptx::tma_load_2d(sA + A_BYTES, &maps.b[B_CLS ? j : 0], full_bar + 8u * stage, col0, kb * kUmmaBK);
                             if (++stage == S) { stage = 0; phase ^= 1u; }
                         }
                     continue;
@@ -245,7 +263,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
                     }
                     if (B_MN) {
 #pragma unroll
-                        for (int j = 0; j < BN_CTA / 64; ++j) {
+                        for (int j = 0; j < B_BOXES; ++j) {
                             if (CG == 1) ptx::tma_load_2d(sB + j * 8192, tmB, fb, col0 + j * 64, k0 - kshift);
                             else ptx::tma_load_2d_pair(sB + j * 8192, tmB, fb, col0 + j * 64, k0 - kshift);
                         }
@@ -313,7 +331,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
                     const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
                     const uint32_t sB = sA + A_BYTES;
                     if (A_CLS) {
-                        const int sigma = p.a_sigma[mb & 7];
+                        const int sigma = p.a_sigma[mb % NCLS];
                         if (kb == 0 && sigma > 0) {
                             // rows lane, lane+32, ...: chunk 0 of row r sits at r*128 + ((r & 7) << 4)
                             uint8_t* genA = gen_base + (size_t)stage * STAGE_BYTES;
@@ -359,8 +377,9 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
         int buf = 0;
         uint32_t buf_phase = 0;
         int seq = 0;                                         // tiles this CTA has processed so far
+        int tma_box = 0;                                     // TMA-store boxes this warp has issued so far
         bool ok = true;
-        uint8_t* stg = stage_out + ((warp - 2) * 32 + lane) * kUmmaStageRowBytes;   // this thread's staging row
+        uint8_t* stg = stage_out + (warp - 2) * kUmmaWarpStagingBytes + lane * kUmmaStageRowBytes;   // this thread's staging row
         unsigned short* srow = reinterpret_cast<unsigned short*>(stg);
         const uintptr_t c_base = reinterpret_cast<uintptr_t>(p.C);
         for (int unit = unit0; ok && unit < p.num_units; unit += unit_step, ++seq) {
@@ -370,8 +389,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
             ptx::tc_fence_after();
             if (warp == 2 && lane == 0) ADAPT_TRACE(4, unit);
             // row of C held by TMEM lane i of this CTA: consecutive rows, or every 8th row of one class
-            const int row_step = A_CLS ? 8 : 1;
-            const int row_base = A_CLS ? (mb >> 3) * 1024 + (mb & 7) : mb * (128 * CG) + (int)cta_rank * 128;
+            const int row_step = A_CLS ? NCLS : 1;
+            const int row_base = A_CLS ? (mb / NCLS) * (128 * NCLS) + (mb % NCLS) : mb * (128 * CG) + (int)cta_rank * 128;
             const int row = row_base + row_step * (q * 32 + lane);
             const int n0 = nb * TILE_N;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
@@ -403,7 +422,92 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
                 const uintptr_t row_bytes = 2ull * (uintptr_t)p.N * row_step;   // distance between this warp's rows
                 // the two warps of a lane quarter take alternate tiles, so one thread sees all passes of
                 // its row and can carry the ragged tail of a pass into the head of the next one
-                if (B_CLS ? half == 0 : (seq & 1) == half) {
+                if (!B_CLS && p.c_mode != 0) {
+                    // C through TMA stores.  A warp stages 32 rows x 64 elements as one 128B-swizzled box (row r
+                    // at r * 128, its 16-byte chunk c at position c ^ (r & 7): conflict-free 16-byte shared
+                    // stores) and one lane hands the box to TMA, which clips rows >= M and the end of the row.
+                    // Two boxes per warp alternate, so converting a pass overlaps the store of the one before.
+                    // The boxes must cover whole 32-byte sectors of C: rows that start 16 bytes off a sector
+                    // boundary halve the store rate, and TMA clips a row's end in 16-byte units, not elements.
+                    //
+                    // Rows on 32-byte boundaries (N % 16 == 0): boxes at columns n0 + 64 * pass of the plain map
+                    // (or of the class map, whose rows are every 8th row of C).
+                    // HALO (tiles of one of 16 row classes): all rows of the tile start sigma elements after a
+                    // 32-byte boundary, and the class map addresses them by x = n + sigma.  The tile owns the
+                    // units x in [16 + TILE_N * nb, 16 + TILE_N * (nb + 1)); it has computed columns
+                    // n >= TILE_N * nb, so element x sits in accumulator column x - sigma - TILE_N * nb
+                    // = (x - x_first) + 16 - sigma.  The first 16 - sigma elements of a row (x < 16) share their
+                    // unit with the previous row of C, the last (N + sigma) % 16 with the next one: the row's own
+                    // thread writes both with 2-byte stores (head: tile nb = 0; tail: the tile that owns the unit).
+                    if ((seq & 1) == half) {
+                        const int cls = A_CLS ? (mb % NCLS) : 0;
+                        const int sig = HALO ? p.c_sigma[cls] : 0;
+                        const int off = HALO ? 16 - sig : 0;
+                        const int y0 = A_CLS ? (mb / NCLS) * 128 + q * 32 : row_base + q * 32;
+                        const CUtensorMap* tmC = &maps.c[cls];
+                        uint8_t* wbuf = stage_out + (warp - 2) * kUmmaWarpStagingBytes;
+                        const int x_first = n0 + (HALO ? 16 : 0);
+                        const int x_end = HALO ? p.c_extent[cls] : p.N;  // end of the row's whole units
+                        if (HALO) {
+                            unsigned short* crow = reinterpret_cast<unsigned short*>(c_base) + (size_t)row * p.N;
+                            const int tail = (p.N + sig) - x_end;        // elements after the last whole unit
+                            const bool has_tail = x_end >= x_first && x_end < x_first + TILE_N && tail > 0;
+#pragma unroll
+                            for (int part = 0; part < 2; ++part) {       // 0: head of the row, 1: its tail (both uniform)
+                                if (part == 0 ? nb != 0 : !has_tail) continue;
+                                const int col = part == 0 ? 0 : off + (x_end - x_first);   // accumulator column
+                                const int n_first = part == 0 ? 0 : x_end - sig;
+                                const int count = part == 0 ? min(off, p.N) : tail;
+                                uint32_t e0[8], e1[8];
+                                ptx::tmem_ld_32x8(t_row + (uint32_t)col, e0);
+                                ptx::tmem_ld_32x8(t_row + (uint32_t)(col + 8), e1);
+                                ptx::tmem_ld_wait();
+                                if (row_ok) {
+#pragma unroll
+                                    for (int i = 0; i < 8; ++i) {
+                                        if (i < count) crow[n_first + i] = cast16(__uint_as_float(e0[i]), p.dtype);
+                                        if (8 + i < count) crow[n_first + 8 + i] = cast16(__uint_as_float(e1[i]), p.dtype);
+                                    }
+                                }
+                            }
+                        }
+#pragma unroll 1
+                        for (int pass = 0; pass < PASSES; ++pass) {
+                            const int x = x_first + 64 * pass;
+                            if (x >= x_end) break;                       // uniform across the warp
+                            const int ncols = min(64, x_end - x);
+                            uint8_t* box = wbuf + (tma_box & 1) * 4096;
+                            uint8_t* brow = box + lane * 128;
+#pragma unroll
+                            for (int h = 0; h < 2; ++h) {
+                                if (32 * h >= ncols) break;              // uniform; those elements lie beyond the row and are clipped
+                                uint32_t r[32];
+                                ptx::tmem_ld_32x32(t_row + (uint32_t)(off + 64 * pass + 32 * h), r);
+                                ptx::tmem_ld_wait();
+                                if (h == 0) {
+                                    if (lane == 0) ptx::bulk_wait_read<1>();   // the store that last used this box has read it
+                                    __syncwarp();
+                                }
+#pragma unroll
+                                for (int c = 0; c < 4; ++c) {
+                                    uint4 v;
+                                    v.x = pack16(__uint_as_float(r[8 * c + 0]), __uint_as_float(r[8 * c + 1]), p.dtype);
+                                    v.y = pack16(__uint_as_float(r[8 * c + 2]), __uint_as_float(r[8 * c + 3]), p.dtype);
+                                    v.z = pack16(__uint_as_float(r[8 * c + 4]), __uint_as_float(r[8 * c + 5]), p.dtype);
+                                    v.w = pack16(__uint_as_float(r[8 * c + 6]), __uint_as_float(r[8 * c + 7]), p.dtype);
+                                    *reinterpret_cast<uint4*>(brow + (((4 * h + c) ^ (lane & 7)) << 4)) = v;
+                                }
+                            }
+                            ptx::fence_proxy_async_smem();
+                            __syncwarp();
+                            if (lane == 0) {
+                                ptx::tma_store_2d(tmC, ptx::smem_u32(box), x, y0);
+                                ptx::bulk_commit();
+                            }
+                            ++tma_box;
+                        }
+                    }
+                } else if (B_CLS ? half == 0 : (seq & 1) == half) {
                     const uintptr_t g_row = g_tile + (uintptr_t)lane * row_bytes;   // this thread's row, column n0
                     const int m_r = (int)((g_row & 15u) >> 1);           // the same in every pass: a pass is 128 bytes
                     const int tile_cols = min(TILE_N, p.N - n0);
@@ -479,7 +583,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
                         __syncwarp();                                    // every row of the warp is staged
                         // 32 rows x 9 aligned chunks: lane + 32*it = 9*rr + qc
                         int rr = lane / 9, qc = lane - 9 * rr;
-                        const uint8_t* stg_warp = stage_out + (warp - 2) * (32 * kUmmaStageRowBytes);
+                        const uint8_t* stg_warp = stage_out + (warp - 2) * kUmmaWarpStagingBytes;
                         const uintptr_t g_pass = g_tile + 2u * c0;
 #pragma unroll
                         for (int it = 0; it < 9; ++it) {
@@ -520,9 +624,9 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
                     }
                 }
 #pragma unroll 1
-                for (int c0 = 0; !B_CLS && c0 < BN; c0 += 32) {
+                for (int c0 = 0; !B_CLS && c0 < TILE_N; c0 += 32) {
                     if (n0 + c0 >= p.N) break;                       // uniform across the warp
-                    if (((seq * (BN / 32) + (c0 >> 5)) & 1) != half) continue;
+                    if (((seq * (TILE_N / 32) + (c0 >> 5)) & 1) != half) continue;
                     uint32_t r[32];
                     ptx::tmem_ld_32x32(t_row + (uint32_t)c0, r);
                     ptx::tmem_ld_wait();
@@ -550,6 +654,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPack maps, const UmmaParams p)
             }
             if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
         }
+        if (lane == 0) ptx::bulk_wait_read<0>();             // TMA stores still reading this warp's staging boxes
     }
 
     // ------------------------------ common exit ----------------------------------------------

@@ -318,3 +318,70 @@ def test_k_class_views_do_not_leak_a_neighbouring_row():
 
 def synth_bits(t):
     return t.contiguous().view(torch.int16)
+
+
+# ---- class tiles with halo columns: C with N % 8 != 0 written through per-row-class TMA stores ------
+
+def halo_variants(M, N, K, dtype, limit=8):
+    """Class tiles with halo columns: up to limit/2 variants that store C themselves (P_k = 1, the TMA-store
+    epilogue) and as many that write fp32 partials."""
+    cands = [c for c in ab.adapt_plan_candidates(M, N, K, dtype) if c.srcA == 3 and c.BN % 64 != 0]
+    picked = [c for c in cands if c.P_k == 1][: limit // 2] + [c for c in cands if c.P_k > 1][: limit // 2]
+    return [(ab.adapt_matmul_plan_forced(M, N, K, dtype, ROW, ROW, c.tiling_key), c) for c in picked]
+
+
+@pytest.mark.parametrize("dtype", [ab.F16, ab.BF16])
+@pytest.mark.parametrize("shape", [(1030, 265, 328), (1030, 265, 331), (2500, 77, 1000), (4100, 1001, 64), (300, 521, 16),
+                                   (16, 9, 8), (129, 3, 40), (1024, 201, 4099), (3000, 40, 24), (2100, 8, 16), (77, 1537, 70), (2049, 193, 5)])
+def test_halo_class_tiles_bit_exact(shape, dtype):
+    M, N, K = shape
+    A = synth.position_coded(M, K, dtype, modulus=7, device="cuda")
+    B = synth.position_coded(K, N, dtype, modulus=5, device="cuda")
+    variants = halo_variants(M, N, K, dtype)
+    assert variants, "shape must offer class tiles with halo columns"
+    assert {c.BN for _, c in variants} <= {80, 144, 208}
+    for plan, c in variants:
+        check_case(M, N, K, dtype, A, B, plan=plan, exact=True)
+
+
+def test_halo_class_tiles_with_unaligned_pointers():
+    """A or C two bytes off a 16-byte boundary: A is then read through a re-pitched copy, C is stored by
+    the epilogue threads; the tiling stays the plan's."""
+    M, N, K = 1100, 333, 203
+    dtype = ab.F16
+    A = synth.position_coded(M, K, dtype, 7, "cuda")
+    B = synth.position_coded(K, N, dtype, 5, "cuda")
+    tdt = synth.torch_dtype(dtype)
+    a_buf = torch.zeros(M * K + 16, dtype=tdt, device="cuda")
+    A_off = a_buf[1:1 + M * K].view(M, K)
+    A_off.copy_(A)
+    assert A_off.data_ptr() % 16 == 2
+    variants = halo_variants(M, N, K, dtype, limit=4)
+    assert variants
+    for plan, c in variants:
+        for a_t, c_off in ((A_off, 0), (A, 1), (A_off, 1)):
+            c_buf = torch.full((M * N + 16,), float("nan"), dtype=tdt, device="cuda")
+            out = c_buf[c_off:c_off + M * N].view(M, N)
+            run_library(a_t, B, M, N, K, dtype, plan=plan, out=out)
+            torch.cuda.synchronize()
+            err, mism, _ = compare_with_oracle(A, B, out.contiguous(), M, N, K, dtype)
+            assert mism == 0
+            # nothing outside C was touched
+            assert torch.isnan(c_buf[:c_off]).all() and torch.isnan(c_buf[c_off + M * N:]).all()
+
+
+def test_tma_store_epilogue_leaves_neighbouring_memory_alone():
+    """Aligned and halo TMA stores clip at M and at the end of each row: guard elements around C stay."""
+    dtype = ab.BF16
+    tdt = synth.torch_dtype(dtype)
+    for (M, N, K) in [(200, 264, 64), (1031, 203, 72), (130, 72, 40)]:
+        A = synth.position_coded(M, K, dtype, 7, "cuda")
+        B = synth.position_coded(K, N, dtype, 5, "cuda")
+        c_buf = torch.full((M * N + 4096,), float("nan"), dtype=tdt, device="cuda")
+        out = c_buf[2048:2048 + M * N].view(M, N)
+        assert out.data_ptr() % 16 == 0
+        run_library(A, B, M, N, K, dtype, out=out)
+        torch.cuda.synchronize()
+        err, mism, _ = compare_with_oracle(A, B, out.contiguous(), M, N, K, dtype)
+        assert mism == 0
+        assert torch.isnan(c_buf[:2048]).all() and torch.isnan(c_buf[2048 + M * N:]).all()

@@ -126,20 +126,25 @@ def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
                 if c.family in (ab.FAM_UMMA_1CTA, ab.FAM_UMMA_2CTA):
                     bn_cta = c.BN // c.cluster
                     # a stage holds the rows of A one box brings (128, or fewer for a short A) and BN columns of B
+                    halo = c.BN % 64 != 0        # class tiles of 16 row classes that own 32-byte units of C's shifted rows
+                    ncls = 16 if halo else 8
                     a_rows = 128
                     if c.srcA == 3:
-                        a_rows = min(128, -(-(-(-M // 8)) // 8) * 8)
+                        a_rows = min(128, -(-(-(-M // ncls)) // 8) * 8)
                     elif c.cluster == 1 and M < 128:
                         a_rows = -(-M // 8) * 8
-                    smem = c.stages * (a_rows * 64 * 2 + bn_cta * 64 * 2)
+                    smem = c.stages * (a_rows * 64 * 2 + -(-bn_cta // 64) * 64 * 64 * 2)
                     assert smem <= 227 * 1024 and 2 <= c.stages <= 15
                     assert 2 * c.BN <= 512 and c.BN % 16 == 0
+                    if halo:
+                        assert c.BN in (80, 144, 208) and c.srcA == 3 and N % 16 and M >= 16 and c.P_n == -(-N // (c.BN - 16))
                     assert c.P_k <= (-(-(-(-K // 8)) // 64) if c.srcB == 3 else -(-(K + 7) // 64))
                     # unaligned operands are never handed to TMA directly (row-major: K for A, N for B)
                     if K % 8:
                         assert c.srcA in (1, 3)      # re-pitched copy, or the per-row-class TMA views
                     if c.srcA == 3:
-                        assert K % 8 and M >= 8 and c.family == ab.FAM_UMMA_1CTA and c.P_m == 8 * -(-M // 1024)
+                        assert (K % 8 or halo) and M >= 8 and c.family == ab.FAM_UMMA_1CTA
+                        assert c.P_m == ncls * -(-M // (128 * ncls))
                     if N % 8:
                         assert c.srcB in (1, 3)      # re-pitched copy, or the per-k-class TMA views
                     if c.srcB == 3:
