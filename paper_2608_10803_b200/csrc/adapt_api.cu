@@ -639,7 +639,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.P_m = c.P_m;
     // a plan made for k-class views that has to fall back to a copy of B (unaligned pointer) uses plain tiles
     p.P_n = (c.srcB == ADAPT_SRC_TMA_CLASSES && !kclsB) ? (int)ceil_div(s.N, c.BN) : c.P_n;
-    p.kb_total = kclsB ? (int)(Kc / kUmmaBK) : (int)ceil_div(s.K + (classesA ? 7 : 0), kUmmaBK);
+    p.kb_total = kclsB ? (int)(Kc / kUmmaBK) : (int)ceil_div(s.K + ((classesA && s.K % 8) ? 7 : 0), kUmmaBK);
     p.kb_per_split = (int)ceil_div(p.kb_total, c.P_k);
     p.P_k = (int)ceil_div(p.kb_total, p.kb_per_split);    // equals the plan's count unless a fallback changed kb_total
     p.num_units = p.P_m * p.P_n * p.P_k;

@@ -171,7 +171,7 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
 {
     const bool kclasses = c.srcB == ADAPT_SRC_TMA_CLASSES;
     const int64_t kblocks = kclasses ? ceil_div(ceil_div(s.K, 8), c.BK)
-                                     : ceil_div(s.K + (c.srcA == ADAPT_SRC_TMA_CLASSES ? 7 : 0), c.BK);
+                                     : ceil_div(s.K + ((c.srcA == ADAPT_SRC_TMA_CLASSES && s.K % 8) ? 7 : 0), c.BK);
     const int64_t L = ceil_div(kblocks, c.P_k) * (kclasses ? 8 : 1);     // k-class mode: the split's blocks of all 8 classes
     const int64_t units = (int64_t)c.P_m * c.P_n * c.P_k;
     const int64_t slots = m.n_sm / c.cluster;
@@ -196,7 +196,7 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     // the strided row-class views); a stream that comes from HBM and is used once is bounded by the
     // bytes one SM keeps in flight, about hbm_bw_per_sm.  The second case only shows in partial waves.
     const double t_mma_all = 2.0 * (double)s.M * s.N * s.K / cal.tensor_flops;
-    const bool mem_bound = c.hbm_bytes / cal.hbm_bw > t_mma_all;
+    const bool mem_bound = 2.0 * (MK * rA + KN * rB) / cal.hbm_bw > t_mma_all;   // the operand stream, not C, outweighs the MMAs
     double sm_rate = cal.l2_bw_per_sm * (c.srcA == ADAPT_SRC_TMA_CLASSES ? cal.class_view_sm_eff : 1.0);
     if (mem_bound && c.srcA == ADAPT_SRC_TMA_CLASSES) sm_rate = std::min(sm_rate, cal.hbm_bw_per_sm);   // measured for the views only
     double tM = stage_bytes / sm_rate * 1e6;
@@ -227,7 +227,10 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     } else {
         tM = std::max(tM, cal.mem_latency_us / (c.stages - 1));
         const double ii = std::max(tM, tP);
-        const double t_tile = std::max((double)L * ii, t_drain);
+        // class tiles pay a fixed cost per tile (strided row views; zeroing the heads of an unaligned A)
+        const double t_fixed = c.srcA != ADAPT_SRC_TMA_CLASSES ? 0.0
+                             : (s.K % 8 ? cal.class_tile_fixed_unaligned_us : cal.class_tile_fixed_us);
+        const double t_tile = std::max((double)L * ii + t_fixed, t_drain);
         // Eq. 14 with the drain overlapped: one fill, Q tiles back to back, the last drain exposed
         pipe = tM + (double)Q * t_tile + tP + t_drain;
     }
@@ -309,7 +312,7 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     // in class mode the k index of a tile is shifted by up to 7 elements
     // k-class mode splits the blocks of one class; in row-class mode the k index is shifted by up to 7
     const int64_t kblocks = c.srcB == ADAPT_SRC_TMA_CLASSES ? ceil_div(ceil_div(s.K, 8), c.BK)
-                                                              : ceil_div(s.K + (c.srcA == ADAPT_SRC_TMA_CLASSES ? 7 : 0), c.BK);
+                                                              : ceil_div(s.K + ((c.srcA == ADAPT_SRC_TMA_CLASSES && s.K % 8) ? 7 : 0), c.BK);
     if (c.P_k < 1 || c.P_k > 1023 || c.P_k > kblocks) return false;
     if (ceil_div(kblocks, ceil_div(kblocks, c.P_k)) != c.P_k) return false;   // no empty split
     // operand sources: TMA needs a 16-byte row pitch
@@ -473,7 +476,7 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
             if (halo && (s.N % 16 == 0 || s.M < 16)) continue;             // halo tiles serve a C off 32-byte boundaries only
             if (!halo && srcA != ADAPT_SRC_PAD_COPY) continue;             // aligned A: class tiles only for their stores
             const int64_t tiles = (halo ? 16 * ceil_div(s.M, 2048) : 8 * ceil_div(s.M, 1024)) * ceil_div(s.N, halo ? BN - 16 : BN);
-            split_candidates(tiles, m.n_sm, ceil_div(s.K + 7, 64), 2, &pks);
+            split_candidates(tiles, m.n_sm, ceil_div(s.K + (s.K % 8 ? 7 : 0), 64), 2, &pks);
             int deepest = 0;
             for (int st = kUmmaMaxStages; st >= 2; --st)
                 if (umma_smem_bytes(BN, 1, st, umma_a_box_rows(s, 1, BN % 64 ? 16 : 8, false)) <= m.smem_bytes) { deepest = st; break; }

@@ -485,8 +485,10 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                                 ptx::tmem_ld_32x32(t_row + (uint32_t)(off + 64 * pass + 32 * h), r);
                                 ptx::tmem_ld_wait();
                                 if (h == 0) {
+                                    if (warp == 2 && lane == 0) ADAPT_TRACE(5, unit);
                                     if (lane == 0) ptx::bulk_wait_read<1>();   // the store that last used this box has read it
                                     __syncwarp();
+                                    if (warp == 2 && lane == 0) ADAPT_TRACE(8, unit);
                                 }
 #pragma unroll
                                 for (int c = 0; c < 4; ++c) {
@@ -503,6 +505,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                             if (lane == 0) {
                                 ptx::tma_store_2d(tmC, ptx::smem_u32(box), x, y0);
                                 ptx::bulk_commit();
+                                if (warp == 2) ADAPT_TRACE(6, unit);
                             }
                             ++tma_box;
                         }

@@ -138,7 +138,7 @@ def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
                     assert 2 * c.BN <= 512 and c.BN % 16 == 0
                     if halo:
                         assert c.BN in (80, 144, 208) and c.srcA == 3 and N % 16 and M >= 16 and c.P_n == -(-N // (c.BN - 16))
-                    assert c.P_k <= (-(-(-(-K // 8)) // 64) if c.srcB == 3 else -(-(K + 7) // 64))
+                    assert c.P_k <= (-(-(-(-K // 8)) // 64) if c.srcB == 3 else -(-(K + (7 if K % 8 else 0)) // 64))
                     # unaligned operands are never handed to TMA directly (row-major: K for A, N for B)
                     if K % 8:
                         assert c.srcA in (1, 3)      # re-pitched copy, or the per-row-class TMA views
