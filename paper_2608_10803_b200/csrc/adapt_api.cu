@@ -381,7 +381,12 @@ static UmmaKernel launch_map_umma(int family, int BN, bool a_mn, bool b_mn, int 
         if (BN == 208) return (const void*)umma_gemm_kernel<208, false, true, 1, 1>;
         return nullptr;
     }
-    if (mode == 2) return BN == 64 ? (const void*)umma_gemm_kernel<64, false, true, 1, 2> : nullptr;   // B through per-k-class maps
+    if (mode == 2) {                     // B through per-k-class maps: eight accumulators (BN = 64), or classes as k splits
+        if (BN == 64) return (const void*)umma_gemm_kernel<64, false, true, 1, 2>;
+        if (BN == 128) return (const void*)umma_gemm_kernel<128, false, true, 1, 3>;
+        if (BN == 256) return (const void*)umma_gemm_kernel<256, false, true, 1, 3>;
+        return nullptr;
+    }
     return family == ADAPT_FAM_UMMA_1CTA ? umma_lookup<1>(BN, a_mn, b_mn) : umma_lookup<2>(BN, a_mn, b_mn);
 }
 
@@ -424,8 +429,9 @@ extern "C" adapt_status_t adapt_init(int device)
     for (int BN : {64, 128, 256, 80, 144, 208})
         CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_1CTA, BN, false, true, 1),
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
-    CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_1CTA, 64, false, true, 2),
-                                  cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
+    for (int BN : {64, 128, 256})
+        CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_1CTA, BN, false, true, 2),
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
     S.device = device;
     S.inited = true;
     return ADAPT_OK;
@@ -640,8 +646,14 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     // a plan made for k-class views that has to fall back to a copy of B (unaligned pointer) uses plain tiles
     p.P_n = (c.srcB == ADAPT_SRC_TMA_CLASSES && !kclsB) ? (int)ceil_div(s.N, c.BN) : c.P_n;
     p.kb_total = kclsB ? (int)(Kc / kUmmaBK) : (int)ceil_div(s.K + ((classesA && s.K % 8) ? 7 : 0), kUmmaBK);
-    p.kb_per_split = (int)ceil_div(p.kb_total, c.P_k);
-    p.P_k = (int)ceil_div(p.kb_total, p.kb_per_split);    // equals the plan's count unless a fallback changed kb_total
+    const bool ksplit_cls = kclsB && c.BN != 64;            // k classes as k splits: P_k = 8 * (splits per class)
+    if (ksplit_cls) {
+        p.kb_per_split = (int)ceil_div(p.kb_total, c.P_k / 8);
+        p.P_k = c.P_k;
+    } else {
+        p.kb_per_split = (int)ceil_div(p.kb_total, c.P_k);
+        p.P_k = (int)ceil_div(p.kb_total, p.kb_per_split);    // equals the plan's count unless a fallback changed kb_total
+    }
     p.num_units = p.P_m * p.P_n * p.P_k;
 
     const size_t szP = p.P_k > 1 ? (size_t)round_up((int64_t)p.P_k * s.M * round_up(s.N, 4) * 4, 256) : 0;
@@ -739,7 +751,8 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     // the kernel takes the maps its mode uses
     TmapPackT<0> pack0;
     TmapPackT<1> pack1;
-    TmapPackT<2> pack2;
+    TmapPackT<2> pack2;                                     // modes 2 and 3 take the same maps
+    static_assert(sizeof(TmapPackT<2>) == sizeof(TmapPackT<3>), "k-class packs share their layout");
     void* args[2] = {nullptr, &p};
     if (classesA) {
         memcpy(pack1.a, maps.a, sizeof(pack1.a)); pack1.b[0] = maps.b[0]; memcpy(pack1.c, maps.c, sizeof(pack1.c));

@@ -48,6 +48,7 @@ struct Calib {
     double hbm_bw_per_sm = 55e9;        // B/s one SM streams from HBM (tail wave of 20000 x 8 x 60001: 15 MB per tile in 0.3 ms)
     double class_view_sm_eff = 0.85;    // per-SM rate through those views relative to l2_bw_per_sm (20000 x 8 x 60001 tail wave)
     double class_tile_fixed_us = 0.5, class_tile_fixed_unaligned_us = 0.9;   // per class tile (44479 x 54634 x 16..72, 64-column tiles)
+    double class_split_bw_eff = 0.88;   // HBM rate through the k-class views of B with full-width tiles (classes as k splits)
     double regroup_bw_eff = 0.3;        // class-major regrouping of A (element-wise reads) relative to hbm_bw
     double class_view_bw_eff = 0.65;    // HBM rate through the per-row-class TMA views of an unaligned A
 };

@@ -172,7 +172,9 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     const bool kclasses = c.srcB == ADAPT_SRC_TMA_CLASSES;
     const int64_t kblocks = kclasses ? ceil_div(ceil_div(s.K, 8), c.BK)
                                      : ceil_div(s.K + ((c.srcA == ADAPT_SRC_TMA_CLASSES && s.K % 8) ? 7 : 0), c.BK);
-    const int64_t L = ceil_div(kblocks, c.P_k) * (kclasses ? 8 : 1);     // k-class mode: the split's blocks of all 8 classes
+    const bool ksplit_cls = kclasses && c.BN != 64;                       // each class a k split of its own
+    const int64_t L = ksplit_cls ? ceil_div(kblocks, c.P_k / 8)
+                                 : ceil_div(kblocks, c.P_k) * (kclasses ? 8 : 1);   // BN = 64: the split's blocks of all 8 classes
     const int64_t units = (int64_t)c.P_m * c.P_n * c.P_k;
     const int64_t slots = m.n_sm / c.cluster;
     const int64_t Q = ceil_div(units, slots);
@@ -186,7 +188,7 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     if (rB > 1.0 && 2.0 * MK <= kL2Bytes) {          // alternatively A stays resident and B streams once
         rB = 1.0;
     }
-    c.hbm_bytes = 2.0 * (MK * rA + KN * rB * (kclasses ? 64.0 / 56.0 : 1.0)) + (c.P_k > 1 ? 0.0 : 2.0 * MN);
+    c.hbm_bytes = 2.0 * (MK * rA + KN * rB * (kclasses ? c.BN / (c.BN - 8.0) : 1.0)) + (c.P_k > 1 ? 0.0 : 2.0 * MN);
 
     // per-SM stage: each CTA loads its 128 rows of A and its share of the BN columns of B
     const double bn_per_cta = (double)c.BN / c.cluster;
@@ -238,7 +240,8 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     model_prologue(s, c, cal);
     model_epilogue(s, c, cal);
     // strided row-class views stream A at a lower rate than a dense tensor (measured 3.5-4.1 TB/s)
-    const double bw = (c.srcA == ADAPT_SRC_TMA_CLASSES || kclasses) ? cal.hbm_bw * cal.class_view_bw_eff : cal.hbm_bw;
+    const double bw = ksplit_cls ? cal.hbm_bw * cal.class_split_bw_eff
+                    : (c.srcA == ADAPT_SRC_TMA_CLASSES || kclasses) ? cal.hbm_bw * cal.class_view_bw_eff : cal.hbm_bw;
     const double t_hbm = c.hbm_bytes / bw * 1e6 - c.t_pro_us - c.t_epi_us;
     c.t_main_us = std::max(pipe, t_hbm);
     finish_common(s, c, cal);
@@ -313,8 +316,12 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     // k-class mode splits the blocks of one class; in row-class mode the k index is shifted by up to 7
     const int64_t kblocks = c.srcB == ADAPT_SRC_TMA_CLASSES ? ceil_div(ceil_div(s.K, 8), c.BK)
                                                               : ceil_div(s.K + ((c.srcA == ADAPT_SRC_TMA_CLASSES && s.K % 8) ? 7 : 0), c.BK);
-    if (c.P_k < 1 || c.P_k > 1023 || c.P_k > kblocks) return false;
-    if (ceil_div(kblocks, ceil_div(kblocks, c.P_k)) != c.P_k) return false;   // no empty split
+    // k classes as k splits (k-class views of B with BN > 64): P_k = 8 * (splits of one class's blocks)
+    const bool ksplit_cls = c.srcB == ADAPT_SRC_TMA_CLASSES && c.BN != 64;
+    if (ksplit_cls && c.P_k % 8 != 0) return false;
+    const int64_t pk_blocks = ksplit_cls ? c.P_k / 8 : c.P_k;
+    if (c.P_k < 1 || c.P_k > 1023 || pk_blocks > kblocks) return false;
+    if (ceil_div(kblocks, ceil_div(kblocks, pk_blocks)) != pk_blocks) return false;   // no empty split
     // operand sources: TMA needs a 16-byte row pitch
     if (c.srcA == ADAPT_SRC_TMA && !aligned16(innerA(s))) return false;
     if (c.srcB == ADAPT_SRC_TMA && !aligned16(innerB(s))) return false;
@@ -324,7 +331,8 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     if (kclasses) {
         // k-rows of one residue class share their misalignment: row-major B with N % 8 != 0, 64-column
         // windows that own 56 columns, A regrouped class-major by a prologue copy (any layout of A)
-        if (c.family != ADAPT_FAM_UMMA_1CTA || s.layoutB != ADAPT_ROW_MAJOR || c.BN != 64) return false;
+        // (BN = 64: eight class accumulators per tile; BN = 128, 256: each class a k split, BN - 8 columns owned)
+        if (c.family != ADAPT_FAM_UMMA_1CTA || s.layoutB != ADAPT_ROW_MAJOR || c.BN % 64 != 0) return false;
         if (aligned16(innerB(s)) || s.K < 64 || c.srcA != ADAPT_SRC_PAD_COPY) return false;
     }
     if (classes) {
@@ -338,7 +346,7 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     if (c.srcB == ADAPT_SRC_PAD_COPY && aligned16(innerB(s))) return false;
     const int ncls = umma_row_classes(c.srcA, c.BN);
     c.P_m = classes ? (int)(ncls * ceil_div(s.M, ncls * c.BM)) : (int)ceil_div(s.M, c.BM);   // class tiles: 8 per 1024 rows, 16 per 2048
-    c.P_n = (int)ceil_div(s.N, kclasses ? 56 : (c.BN % 64 ? c.BN - 16 : c.BN));
+    c.P_n = (int)ceil_div(s.N, kclasses ? c.BN - 8 : (c.BN % 64 ? c.BN - 16 : c.BN));
     if ((int64_t)c.P_m * c.P_n * c.P_k > (int64_t)1 << 30) return false;
     c.persistent = 1;
     return true;
@@ -501,6 +509,23 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
             d.family = ADAPT_FAM_UMMA_1CTA; d.BM = 128; d.BN = 64; d.BK = 64; d.cluster = 1;
             d.stages = deepest; d.P_k = pk; d.srcA = ADAPT_SRC_PAD_COPY; d.srcB = ADAPT_SRC_TMA_CLASSES;
             if (deepest >= 2 && finalize(s, m, cal, d)) out->push_back(d);
+        }
+    }
+    // --- the same views with each class a k split: full-width tiles, 8 fp32 partials per output ---
+    if (srcB == ADAPT_SRC_PAD_COPY && s.layoutB == ADAPT_ROW_MAJOR && s.K >= 64) {
+        for (int BN : {128, 256}) {
+            const int64_t tiles = ceil_div(s.M, 128) * ceil_div(s.N, BN - 8);
+            split_candidates(tiles * 8, m.n_sm, ceil_div(ceil_div(s.K, 8), 64), 1, &pks);
+            if (std::find(pks.begin(), pks.end(), 1) == pks.end()) pks.insert(pks.begin(), 1);
+            int deepest = 0;
+            for (int st = kUmmaMaxStages; st >= 2; --st)
+                if (umma_smem_bytes(BN, 1, st, umma_a_box_rows(s, 1, 0, true)) <= m.smem_bytes) { deepest = st; break; }
+            for (int pkk : pks) {
+                Config d;
+                d.family = ADAPT_FAM_UMMA_1CTA; d.BM = 128; d.BN = BN; d.BK = 64; d.cluster = 1;
+                d.stages = deepest; d.P_k = 8 * pkk; d.srcA = ADAPT_SRC_PAD_COPY; d.srcB = ADAPT_SRC_TMA_CLASSES;
+                if (deepest >= 2 && 8 * pkk <= 1023 && finalize(s, m, cal, d)) out->push_back(d);
+            }
         }
     }
     // --- warp-level streaming family ---

@@ -72,7 +72,7 @@ struct UmmaParams {
 template <int MODE>
 struct TmapPackT {
     CUtensorMap a[MODE == 1 ? 16 : 1];
-    CUtensorMap b[MODE == 2 ? 8 : 1];
+    CUtensorMap b[MODE >= 2 ? 8 : 1];
     CUtensorMap c[MODE == 1 ? 16 : 1];
 };
 
@@ -127,12 +127,19 @@ __device__ __forceinline__ unsigned short cast16(float a, int dtype)
 // x' in [56*nb, 56*nb + 64) of shifted columns, and the epilogue adds the eight buffers with
 // buffer j read sigma_j columns to the right: C[m][56*nb + c] = sum_j acc_j[m][c + sigma_j], c < 56.
 // Columns of a buffer left of sigma_j hold products with the previous row's tail and are never read.
+//
+// B_SPLIT (MODE 3, "k classes as k splits"): the same views of B, but each class is a k split of its
+// own: unit (tile, split) with split = 8 * ks + j contracts the k-blocks of class j in range ks into one
+// accumulator of BN columns over the window x' in [(BN-8)*nb, (BN-8)*nb + BN) and writes the BN - 8
+// columns the tile owns as an fp32 partial (read sigma_j columns to the right); the reduction kernel adds
+// the 8 * P_kk slabs in ascending order.  Full-width tiles, at the price of 8 partials per output.
 template <int BN, bool A_MN, bool B_MN, int CG, int MODE>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams p)
 {
     constexpr bool A_CLS = MODE == 1;
     constexpr bool B_CLS = MODE == 2;
+    constexpr bool B_SPLIT = MODE == 3;                   // k classes as k splits (see below)
     static_assert(MODE == 0 || (!A_MN && B_MN && CG == 1), "class modes: K-major A, row-major B, one CTA per tile");
     static_assert(!B_CLS || BN == 64, "k-class mode uses 64-column windows");
     // HALO: class tiles for a C whose rows do not start on 32-byte boundaries (N % 16 != 0) own 32-byte
@@ -141,7 +148,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
     constexpr bool HALO = A_CLS && (BN % 64 != 0);
     static_assert(BN % 64 == 0 || (A_CLS && (BN - 16) % 64 == 0), "BN is a multiple of 64, plus 16 halo columns for class tiles");
     constexpr int NCLS = HALO ? 16 : 8;                   // row classes of a class tile: rows NCLS*128*g + j + NCLS*i
-    constexpr int TILE_N = B_CLS ? 56 : (HALO ? BN - 16 : BN);   // output columns (HALO: chunk-aligned elements) a tile owns
+    constexpr int TILE_N = B_CLS ? 56 : (B_SPLIT ? BN - 8 : (HALO ? BN - 16 : BN));   // output columns (HALO: chunk-aligned elements) a tile owns
     constexpr int BN_CTA = BN / CG;                       // B columns this CTA loads
     // the A region of a stage holds the rows one box brings (128, or fewer for a short K-major A)
     const int A_BYTES = (CG == 2) ? 128 * kUmmaBK * 2 : p.a_tx_bytes;
@@ -220,7 +227,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
             for (int unit = unit0; ok && unit < p.num_units; unit += unit_step) {
                 int mb, nb, split;
                 decode_unit(p, unit, mb, nb, split);
-                const int kb0 = split * p.kb_per_split;
+                const int kb0 = (B_SPLIT ? (split >> 3) : split) * p.kb_per_split;
                 const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
                 // A rows of this CTA: consecutive rows, or in class mode rows 1024*g + j + 8*i read through
                 // map j at class-row index 128*g
@@ -228,7 +235,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                 const int row0 = A_CLS ? (mb / NCLS) * 128 : mb * (128 * CG) + (int)cta_rank * 128;
                 const int kshift = A_CLS ? p.a_sigma[cls] : 0;                // B's k-rows lag A's kappa by sigma
                 const CUtensorMap* tmA = &maps.a[cls];
-                const CUtensorMap* tmB = &maps.b[0];
+                const CUtensorMap* tmB = &maps.b[B_SPLIT ? (split & 7) : 0];  // k classes as splits: the class's view of B
+                const int a_k_off = B_SPLIT ? (split & 7) * p.cls_kc : 0;     // ... and its segment of the regrouped A
                 const int col0 = nb * TILE_N + (int)cta_rank * BN_CTA;        // this CTA's B columns
                 if (B_CLS) {
                     // class by class: A' columns j*Kc + 64*b .., B's class-j rows 64*b .. at shifted columns 56*nb ..
@@ -252,8 +260,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     else if (leader) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, 2 * STAGE_BYTES);
                     const int k0 = kb * kUmmaBK;
                     if (!A_MN) {
-                        if (CG == 1) ptx::tma_load_2d(sA, tmA, fb, k0, row0);
-                        else ptx::tma_load_2d_pair(sA, tmA, fb, k0, row0);
+                        if (CG == 1) ptx::tma_load_2d(sA, tmA, fb, k0 + a_k_off, row0);
+                        else ptx::tma_load_2d_pair(sA, tmA, fb, k0 + a_k_off, row0);
                     } else {
 #pragma unroll
                         for (int j = 0; j < 2; ++j) {
@@ -302,7 +310,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
             for (int unit = unit0; ok && unit < p.num_units; unit += unit_step) {
                 int mb, nb, split;
                 decode_unit(p, unit, mb, nb, split);
-                const int kb0 = split * p.kb_per_split;
+                const int kb0 = (B_SPLIT ? (split >> 3) : split) * p.kb_per_split;
                 const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
                 if (!mma_wait(tempty_bar + 8u * buf, buf_phase ^ 1u)) { ok = false; break; }
                 ptx::tc_fence_after();
@@ -626,8 +634,44 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                         }
                     }
                 }
+                if (B_SPLIT) {
+                    // the tile's columns sit sigma_j columns to the right in the accumulator; BN - 8 of them:
+                    // chunks of 32 and a last one of 24, split between the two warps of the lane quarter
+                    const int sig = p.b_sigma[split & 7];
 #pragma unroll 1
-                for (int c0 = 0; !B_CLS && c0 < TILE_N; c0 += 32) {
+                    for (int c0 = 0; c0 < TILE_N; c0 += 32) {
+                        if (n0 + c0 >= p.N) break;                   // uniform across the warp
+                        if (((seq + (c0 >> 5)) & 1) != half) continue;
+                        uint32_t r[32];
+                        if (c0 + 32 <= TILE_N) {
+                            ptx::tmem_ld_32x32(t_row + (uint32_t)(sig + c0), r);
+                        } else {                                     // 24 columns: stay inside the accumulator
+                            uint32_t r8a[8], r8b[8], r8c[8];
+                            ptx::tmem_ld_32x8(t_row + (uint32_t)(sig + c0), r8a);
+                            ptx::tmem_ld_32x8(t_row + (uint32_t)(sig + c0 + 8), r8b);
+                            ptx::tmem_ld_32x8(t_row + (uint32_t)(sig + c0 + 16), r8c);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) { r[i] = r8a[i]; r[8 + i] = r8b[i]; r[16 + i] = r8c[i]; r[24 + i] = 0u; }
+                        }
+                        ptx::tmem_ld_wait();
+                        if (!row_ok) continue;
+                        const int col = n0 + c0;
+                        const int width = min(32, TILE_N - c0);
+                        float* prow = p.partial + ((size_t)split * p.M + row) * p.Np + col;
+                        if (col + width <= p.Np) {
+#pragma unroll
+                            for (int v = 0; v < 8; ++v)
+                                if (4 * v < width)
+                                    *reinterpret_cast<uint4*>(prow + 4 * v) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j < width && col + j < p.N) prow[j] = __uint_as_float(r[j]);
+                        }
+                    }
+                }
+#pragma unroll 1
+                for (int c0 = 0; !B_CLS && !B_SPLIT && c0 < TILE_N; c0 += 32) {
                     if (n0 + c0 >= p.N) break;                       // uniform across the warp
                     if (((seq * (TILE_N / 32) + (c0 >> 5)) & 1) != half) continue;
                     uint32_t r[32];

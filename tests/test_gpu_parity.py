@@ -260,12 +260,14 @@ def test_row_class_views_do_not_leak_a_neighbouring_row():
 
 # ---- row-major B with N % 8 != 0 read in place through per-k-class TMA views ----------------------
 
-def kclass_mode_variants(M, N, K, dtype, layoutA=ROW, limit=6):
-    out = []
-    for c in ab.adapt_plan_candidates(M, N, K, dtype, layoutA, ROW):
-        if c.srcB == 3 and len(out) < limit:
-            out.append((ab.adapt_matmul_plan_forced(M, N, K, dtype, layoutA, ROW, c.tiling_key), c))
-    return out
+def kclass_mode_variants(M, N, K, dtype, layoutA=ROW, limit=4):
+    """Up to `limit` variants each of the two forms: eight class accumulators per tile (BN = 64) and
+    classes as k splits (BN = 128, 256)."""
+    cands = [c for c in ab.adapt_plan_candidates(M, N, K, dtype, layoutA, ROW) if c.srcB == 3]
+    picked = [c for c in cands if c.BN == 64][:limit]
+    split = [c for c in cands if c.BN != 64]
+    picked += [c for c in split if c.P_k == 8][: limit // 2] + [c for c in split if c.P_k > 8][: limit // 2]
+    return [(ab.adapt_matmul_plan_forced(M, N, K, dtype, layoutA, ROW, c.tiling_key), c) for c in picked]
 
 
 @pytest.mark.parametrize("dtype", [ab.F16, ab.BF16])
@@ -278,6 +280,7 @@ def test_k_class_views_bit_exact(shape, dtype):
     variants = kclass_mode_variants(M, N, K, dtype)
     assert variants, "shape must offer the k-class source for B"
     assert any(c.P_k > 1 for _, c in variants) or K < 1024
+    assert any(c.BN != 64 for _, c in variants), "classes as k splits must be on offer"
     for plan, c in variants:
         check_case(M, N, K, dtype, A, B, plan=plan, exact=True)
 
@@ -289,7 +292,7 @@ def test_k_class_views_with_column_major_a_and_random_values():
         B = synth.draw_operand(K, N, synth.U11, 22, dtype, "cuda")
         variants = kclass_mode_variants(M, N, K, dtype, layoutA=COL)
         assert variants
-        for plan, c in variants[:3]:
+        for plan, c in variants:
             err, _, _, _ = check_case(M, N, K, dtype, A, B, COL, ROW, plan=plan)
             assert err <= TOL[dtype]
 

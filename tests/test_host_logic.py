@@ -138,7 +138,7 @@ def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
                     assert 2 * c.BN <= 512 and c.BN % 16 == 0
                     if halo:
                         assert c.BN in (80, 144, 208) and c.srcA == 3 and N % 16 and M >= 16 and c.P_n == -(-N // (c.BN - 16))
-                    assert c.P_k <= (-(-(-(-K // 8)) // 64) if c.srcB == 3 else -(-(K + (7 if K % 8 else 0)) // 64))
+                    assert c.P_k <= ((8 if c.BN != 64 else 1) * -(-(-(-K // 8)) // 64) if c.srcB == 3 else -(-(K + (7 if K % 8 else 0)) // 64))
                     # unaligned operands are never handed to TMA directly (row-major: K for A, N for B)
                     if K % 8:
                         assert c.srcA in (1, 3)      # re-pitched copy, or the per-row-class TMA views
@@ -148,9 +148,12 @@ def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
                     if N % 8:
                         assert c.srcB in (1, 3)      # re-pitched copy, or the per-k-class TMA views
                     if c.srcB == 3:
-                        # k classes: A regrouped class-major, 56 output columns per tile
-                        assert N % 8 and K >= 64 and c.family == ab.FAM_UMMA_1CTA and c.BN == 64
-                        assert c.srcA == 1 and c.P_n == -(-N // 56)
+                        # k classes: A regrouped class-major, BN - 8 output columns per tile; BN = 64 keeps eight
+                        # class accumulators per tile, BN = 128 / 256 makes each class a k split
+                        assert N % 8 and K >= 64 and c.family == ab.FAM_UMMA_1CTA and c.BN in (64, 128, 256)
+                        assert c.srcA == 1 and c.P_n == -(-N // (c.BN - 8))
+                        if c.BN != 64:
+                            assert c.P_k % 8 == 0
                 if c.family == ab.FAM_SKINNY:
                     assert min(M, N) <= 16
                 # taxonomy label follows the predicate (Section 4.2)
