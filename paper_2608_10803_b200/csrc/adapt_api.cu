@@ -129,6 +129,7 @@ void apply_env(State& S)
 {
     if (const char* e = getenv("ADAPT_FAMILY_MASK")) S.machine.family_mask = (unsigned)strtoul(e, nullptr, 0);
     if (const char* e = getenv("ADAPT_LOG")) S.log = atoi(e);
+    if (const char* e = getenv("ADAPT_NO_PDL")) pdl_enabled() = atoi(e) == 0;
     if (const char* e = getenv("ADAPT_WORKSPACE_LIMIT_MB")) S.machine.workspace_limit = (int64_t)atoll(e) << 20;
 }
 
@@ -593,7 +594,7 @@ adapt_status_t launch_pad(State& S, const void* src, void* dst, int64_t outer, i
 {
     const int64_t chunks = outer * (pitch / 8);
     const int blocks = (int)std::min<int64_t>(ceil_div(chunks, 256), (int64_t)S.machine.n_sm * 16);
-    pad_copy_kernel<<<blocks, 256, 0, stream>>>((const unsigned short*)src, (unsigned short*)dst, outer, inner, pitch);
+    CUDA_TRY(launch_pdl(pad_copy_kernel, dim3(blocks), dim3(256), 0, stream, (const unsigned short*)src, (unsigned short*)dst, outer, inner, pitch));
     S.launches.fetch_add(1, std::memory_order_relaxed);
     CUDA_TRY(cudaGetLastError());
     return ADAPT_OK;
@@ -604,7 +605,7 @@ adapt_status_t launch_reduce(State& S, const float* partial, void* C, int64_t M,
     const int64_t Np = round_up(N, 4);
     const int64_t work = M * (Np / 4);
     const int blocks = (int)std::min<int64_t>(ceil_div(work, 256), (int64_t)S.machine.n_sm * 8);
-    splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(partial, (unsigned short*)C, (int)M, (int)N, (int)Np, P_k, dtype);
+    CUDA_TRY(launch_pdl(splitk_reduce_kernel, dim3(blocks), dim3(256), 0, stream, (const float*)partial, (unsigned short*)C, (int)M, (int)N, (int)Np, (int)P_k, (int)dtype));
     S.launches.fetch_add(1, std::memory_order_relaxed);
     CUDA_TRY(cudaGetLastError());
     return ADAPT_OK;
@@ -667,8 +668,8 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
         const int64_t a_sm = s.layoutA == ADAPT_ROW_MAJOR ? s.K : 1, a_sk = s.layoutA == ADAPT_ROW_MAJOR ? 1 : s.M;
         const int64_t work = s.M * Kc;                    // 16-byte chunks of A'
         const int blocks = (int)std::min<int64_t>(ceil_div(work, 256), (int64_t)S.machine.n_sm * 16);
-        regroup_a_kernel<<<blocks, 256, 0, stream>>>((const unsigned short*)A, (unsigned short*)w8, (int)s.M, (int)s.K,
-                                                       (int)Kc, a_sm, a_sk);
+        CUDA_TRY(launch_pdl(regroup_a_kernel, dim3(blocks), dim3(256), 0, stream, (const unsigned short*)A, (unsigned short*)w8,
+                            (int)s.M, (int)s.K, (int)Kc, a_sm, a_sk));
         S.launches.fetch_add(1, std::memory_order_relaxed);
         CUDA_TRY(cudaGetLastError());
         a_src = w8;
@@ -741,13 +742,14 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     cfg.blockDim = dim3(kUmmaThreads, 1, 1);
     cfg.dynamicSmemBytes = (size_t)umma_smem_bytes(c.BN, cg, p.stages, a_box_rows);
     cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = (unsigned)cg;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    pdl_attribute(&attr[1]);
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = 2;
     // the kernel takes the maps its mode uses
     TmapPackT<0> pack0;
     TmapPackT<1> pack1;
@@ -790,7 +792,7 @@ adapt_status_t run_simt(State& S, Plan* pl, const void* A, const void* B, void* 
     p.C = (unsigned short*)C;
     p.partial = (float*)ws;
     dim3 grid((unsigned)((int64_t)c.P_m * c.P_n), (unsigned)c.P_k, 1);
-    simt_gemm_kernel<<<grid, 256, 0, stream>>>((const unsigned short*)A, (const unsigned short*)B, p);
+    CUDA_TRY(launch_pdl(simt_gemm_kernel, grid, dim3(256), 0, stream, (const unsigned short*)A, (const unsigned short*)B, p));
     S.launches.fetch_add(1, std::memory_order_relaxed);
     CUDA_TRY(cudaGetLastError());
     if (c.P_k > 1) return launch_reduce(S, (const float*)ws, C, s.M, s.N, c.P_k, s.dtype, stream);
@@ -956,11 +958,11 @@ extern "C" adapt_status_t adapt_matmul_noalloc(int64_t M, int64_t N, int64_t K, 
     p.partial = scratch;
     const int64_t tiles = ceil_div(M, 64) * ceil_div(N, 64);
     dim3 grid((unsigned)tiles, (unsigned)pk, 1);
-    simt_gemm_kernel<<<grid, 256, 0, stream>>>((const unsigned short*)A, (const unsigned short*)B, p);
+    CUDA_TRY(launch_pdl(simt_gemm_kernel, grid, dim3(256), 0, stream, (const unsigned short*)A, (const unsigned short*)B, p));
     CUDA_TRY(cudaGetLastError());
     const int64_t work = M * (Np / 4);
     const int blocks = (int)std::min<int64_t>(ceil_div(work, 256), 148 * 8);
-    splitk_reduce_kernel<<<blocks, 256, 0, stream>>>(scratch, (unsigned short*)C, (int)M, (int)N, (int)Np, (int)pk, (int)dtype);
+    CUDA_TRY(launch_pdl(splitk_reduce_kernel, dim3(blocks), dim3(256), 0, stream, (const float*)scratch, (unsigned short*)C, (int)M, (int)N, (int)Np, (int)pk, (int)dtype));
     CUDA_TRY(cudaGetLastError());
     st().launches.fetch_add(2, std::memory_order_relaxed);
     return ADAPT_OK;

@@ -7,6 +7,8 @@
 #include <cuda_fp16.h>
 #include <cuda_bf16.h>
 
+#include "launch_pdl.cuh"
+
 namespace adapt {
 
 __device__ __forceinline__ float load16_as_float(const unsigned short* p, int dtype)
@@ -30,6 +32,8 @@ __global__ void __launch_bounds__(256)
 pad_copy_kernel(const unsigned short* __restrict__ src, unsigned short* __restrict__ dst,
                 int64_t outer, int64_t inner, int64_t pitch)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int64_t chunks_per_row = pitch / 8;
     const int64_t total = outer * chunks_per_row;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
@@ -80,6 +84,8 @@ __global__ void __launch_bounds__(256)
 regroup_a_kernel(const unsigned short* __restrict__ A, unsigned short* __restrict__ Ap,
                  int M, int K, int Kc, int64_t a_sm, int64_t a_sk)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int chunks = Kc / 8;
     const int64_t total = (int64_t)M * 8 * chunks;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
@@ -109,6 +115,8 @@ __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float* __restrict__ partial, unsigned short* __restrict__ C,
                      int M, int N, int Np, int P_k, int dtype)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int groups = Np >> 2;
     const int64_t total = (int64_t)M * groups;
     const int64_t slab = (int64_t)M * Np;
@@ -162,6 +170,8 @@ simt_gemm_kernel(const unsigned short* __restrict__ A, const unsigned short* __r
 {
     __shared__ float sA[16][64 + 4];
     __shared__ float sB[16][64 + 4];
+    pdl_launch_dependents();
+    pdl_wait();
     const int tid = threadIdx.x;
     const int m0 = (int)(blockIdx.x / p.P_n) * 64, n0 = (int)(blockIdx.x % p.P_n) * 64;
     const int split = blockIdx.y;

@@ -25,6 +25,7 @@
 #include <cuda_runtime.h>
 
 #include "adapt_internal.h"
+#include "launch_pdl.cuh"
 
 namespace adapt {
 
@@ -144,6 +145,8 @@ __global__ void __launch_bounds__(kSkinnyThreads, 2)
 skinny_gemm_kernel(const SkinnyParams p)
 {
     __shared__ __align__(16) unsigned char s_raw[kSkinnySmemBytes];
+    pdl_launch_dependents();
+    pdl_wait();
     constexpr int PITCH = KC ? kSkinnyPitchKC : kSkinnyPitchRC;
     unsigned short (*s_small)[PITCH] = reinterpret_cast<unsigned short (*)[PITCH]>(s_raw);
     float* s_out = reinterpret_cast<float*>(s_raw);         // reused after the main loop
@@ -349,7 +352,7 @@ inline adapt_status_t launch_skinny(const Shape& s, const Config& c, const void*
     const bool aligned = (p.ld % 8 == 0) && ((uintptr_t)p.Str % 16 == 0);
     dim3 grid((unsigned)ceil_div(p.R, p.BNs), (unsigned)c.P_k, 1);
     SkinnyKernel k = kc ? skinny_pick<true>(s.dtype != 0, aligned) : skinny_pick<false>(s.dtype != 0, aligned);
-    k<<<grid, kSkinnyThreads, 0, stream>>>(p);
+    if (launch_pdl(k, grid, dim3(kSkinnyThreads, 1, 1), 0, stream, p) != cudaSuccess) return ADAPT_ERR_CUDA;
     return ADAPT_OK;
 }
 

@@ -21,6 +21,7 @@
 
 #include "adapt_internal.h"
 #include "ptx_sm100.cuh"
+#include "launch_pdl.cuh"
 
 namespace adapt {
 
@@ -179,6 +180,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
     // epilogue staging: one row of 72 16-bit elements (64 columns + up to 7 of shift) per epilogue thread
     uint8_t* stage_out = bar_gen + kUmmaBarrierBytes;
 
+    pdl_launch_dependents();
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t cta_rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;
@@ -211,6 +213,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
     }
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
+    // set-up done: from here on the kernel reads and writes global memory
+    pdl_wait();
 
     const int unit0 = (CG == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int unit_step = (CG == 2) ? (int)(gridDim.x >> 1) : (int)gridDim.x;
