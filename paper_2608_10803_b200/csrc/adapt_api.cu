@@ -385,7 +385,8 @@ static UmmaKernel launch_map_umma(int family, int BN, bool a_mn, bool b_mn, int 
     if (mode == 2) {                     // B through per-k-class maps: eight accumulators (BN = 64), or classes as k splits
         if (BN == 64) return (const void*)umma_gemm_kernel<64, false, true, 1, 2>;
         if (BN == 128) return (const void*)umma_gemm_kernel<128, false, true, 1, 3>;
-        if (BN == 256) return (const void*)umma_gemm_kernel<256, false, true, 1, 3>;
+        if (BN == 256) return family == ADAPT_FAM_UMMA_2CTA ? (const void*)umma_gemm_kernel<256, false, true, 2, 3>
+                                                             : (const void*)umma_gemm_kernel<256, false, true, 1, 3>;
         return nullptr;
     }
     return family == ADAPT_FAM_UMMA_1CTA ? umma_lookup<1>(BN, a_mn, b_mn) : umma_lookup<2>(BN, a_mn, b_mn);
@@ -433,6 +434,8 @@ extern "C" adapt_status_t adapt_init(int device)
     for (int BN : {64, 128, 256})
         CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_1CTA, BN, false, true, 2),
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
+    CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_2CTA, 256, false, true, 2),
+                                  cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
     S.device = device;
     S.inited = true;
     return ADAPT_OK;
@@ -602,7 +605,7 @@ adapt_status_t launch_pad(State& S, const void* src, void* dst, int64_t outer, i
 
 adapt_status_t launch_reduce(State& S, const float* partial, void* C, int64_t M, int64_t N, int P_k, int dtype, cudaStream_t stream)
 {
-    const int64_t Np = round_up(N, 4);
+    const int64_t Np = partial_pitch(N);
     const int64_t work = M * (Np / 4);
     const int blocks = (int)std::min<int64_t>(ceil_div(work, 256), (int64_t)S.machine.n_sm * 8);
     CUDA_TRY(launch_pdl(splitk_reduce_kernel, dim3(blocks), dim3(256), 0, stream, (const float*)partial, (unsigned short*)C, (int)M, (int)N, (int)Np, (int)P_k, (int)dtype));
@@ -657,7 +660,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     }
     p.num_units = p.P_m * p.P_n * p.P_k;
 
-    const size_t szP = p.P_k > 1 ? (size_t)round_up((int64_t)p.P_k * s.M * round_up(s.N, 4) * 4, 256) : 0;
+    const size_t szP = p.P_k > 1 ? (size_t)round_up((int64_t)p.P_k * s.M * partial_pitch(s.N) * 4, 256) : 0;
     void* ws = nullptr;
     adapt_status_t r = get_workspace(S, stream, szA + szB + szP, &ws);
     if (r != ADAPT_OK) return r;
@@ -720,12 +723,12 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.dtype = s.dtype;
     // the plan's ring depth assumed its own A box; a fallback to copies may need a shallower ring
     p.stages = c.stages;
-    while (p.stages > 2 && umma_smem_bytes(c.BN, cg, p.stages, a_box_rows) > S.machine.smem_bytes) --p.stages;
+    while (p.stages > 2 && umma_smem_bytes(c.BN, cg, p.stages, a_box_rows, p.P_k == 1) > S.machine.smem_bytes) --p.stages;
     p.a_tx_bytes = a_box_rows * kUmmaBK * 2;
     p.idesc = umma_idesc(s.dtype, a_mn, b_mn, 128 * cg, c.BN);
     p.C = C;
     p.partial = partial;
-    p.Np = (int)round_up(s.N, 4);
+    p.Np = (int)partial_pitch(s.N);
     p.status = S.d_status;
     p.trace = nullptr;
 #ifdef ADAPT_TRACE_BUILD
@@ -740,7 +743,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
     cfg.blockDim = dim3(kUmmaThreads, 1, 1);
-    cfg.dynamicSmemBytes = (size_t)umma_smem_bytes(c.BN, cg, p.stages, a_box_rows);
+    cfg.dynamicSmemBytes = (size_t)umma_smem_bytes(c.BN, cg, p.stages, a_box_rows, p.P_k == 1);
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -776,7 +779,7 @@ adapt_status_t run_simt(State& S, Plan* pl, const void* A, const void* B, void* 
 {
     const Shape& s = pl->s;
     const Config& c = pl->c;
-    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * round_up(s.N, 4) * 4, 256) : 0;
+    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * partial_pitch(s.N) * 4, 256) : 0;
     void* ws = nullptr;
     adapt_status_t r = get_workspace(S, stream, szP, &ws);
     if (r != ADAPT_OK) return r;
@@ -786,7 +789,7 @@ adapt_status_t run_simt(State& S, Plan* pl, const void* A, const void* B, void* 
     if (s.layoutB == ADAPT_ROW_MAJOR) { p.b_sk = s.N; p.b_sn = 1; } else { p.b_sk = 1; p.b_sn = s.K; }
     p.P_n = c.P_n;
     p.P_k = c.P_k;
-    p.Np = (int)round_up(s.N, 4);
+    p.Np = (int)partial_pitch(s.N);
     p.kb_per_split = (int)ceil_div(ceil_div(s.K, 16), c.P_k);
     p.dtype = s.dtype;
     p.C = (unsigned short*)C;
@@ -803,7 +806,7 @@ adapt_status_t run_skinny(State& S, Plan* pl, const void* A, const void* B, void
 {
     const Shape& s = pl->s;
     const Config& c = pl->c;
-    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * round_up(s.N, 4) * 4, 256) : 0;
+    const size_t szP = c.P_k > 1 ? (size_t)round_up((int64_t)c.P_k * s.M * partial_pitch(s.N) * 4, 256) : 0;
     void* ws = nullptr;
     adapt_status_t r = get_workspace(S, stream, szP, &ws);
     if (r != ADAPT_OK) return r;
@@ -913,7 +916,7 @@ extern "C" adapt_status_t adapt_matmul_noalloc(int64_t M, int64_t N, int64_t K, 
         return fail(ADAPT_ERR_INVALID_ARG, "bad dtype or layout value%s");
     if (!A || !B || !C) return fail(ADAPT_ERR_INVALID_ARG, "null operand%s");
     if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C) & 1) return fail(ADAPT_ERR_INVALID_ARG, "operands must be 2-byte aligned%s");
-    const int64_t Np = round_up(N, 4);
+    const int64_t Np = partial_pitch(N);
     const int64_t slab = M * Np * 4;                       // bytes of one split's partial
     if (slab <= 0 || 2 * slab > (int64_t)kNoAllocScratchBytes)
         return fail(ADAPT_ERR_UNSUPPORTED,

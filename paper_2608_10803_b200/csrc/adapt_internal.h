@@ -48,6 +48,7 @@ struct Calib {
     double hbm_bw_per_sm = 55e9;        // B/s one SM streams from HBM (tail wave of 20000 x 8 x 60001: 15 MB per tile in 0.3 ms)
     double class_view_sm_eff = 0.85;    // per-SM rate through those views relative to l2_bw_per_sm (20000 x 8 x 60001 tail wave)
     double class_tile_fixed_us = 0.5, class_tile_fixed_unaligned_us = 0.9;   // per class tile (44479 x 54634 x 16..72, 64-column tiles)
+    double kclass_view_sm_eff = 0.65;   // per-SM rate through the k-class views of B relative to l2_bw_per_sm (272 x 67839 x 6046: 48 KB per 0.75 us)
     double class_split_bw_eff = 0.88;   // HBM rate through the k-class views of B with full-width tiles (classes as k splits)
     double regroup_bw_eff = 0.3;        // class-major regrouping of A (element-wise reads) relative to hbm_bw
     double class_view_bw_eff = 0.65;    // HBM rate through the per-row-class TMA views of an unaligned A
@@ -98,6 +99,10 @@ void fill_info(const Shape& s, const Config& c, adapt_plan_info_t* out);
 inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
 
+// Row pitch (elements) of the fp32 split-K partials: rows start on 32-byte boundaries, so the tensor-core
+// kernels write whole 32-byte sectors (16-byte pieces of a sector halve the store rate).
+inline int64_t partial_pitch(int64_t N) { return round_up(N, 8); }
+
 // Operand pitch in elements after the Padding module (16-byte multiple).
 inline int64_t padded_pitch(int64_t inner) { return round_up(inner, 8); }
 
@@ -105,17 +110,29 @@ const Calib& default_calib();
 
 // Shared-memory layout of the tcgen05 kernels, used by the capacity check and by the launcher:
 // S stages of (A: box rows x 64, B: BN/cluster x 64) 16-bit, a barrier block, the epilogue staging
-// (8 KB per epilogue warp), and slack to align the stages to 1024 B.
+// (8 KB per epilogue warp, only when the kernel stores the 16-bit C), and slack to align the stages to 1024 B.
 constexpr int kSkinnyKChunk = 512;   // k values the warp-level kernel stages per chunk; its k splits are whole chunks
 constexpr int kUmmaBarrierBytes = 1024;  // keeps the epilogue staging 1024-byte aligned (swizzled TMA boxes)
 constexpr int kUmmaMaxStages = 15;
 constexpr int kUmmaEpilogueWarps = 8;
 constexpr int kUmmaStageRowBytes = 144;   // 72 16-bit elements: 64 columns + up to 7 of alignment shift
 constexpr int kUmmaWarpStagingBytes = 8192;   // per epilogue warp: two 32 x 128 B boxes for TMA stores, or 32 shifted rows
-inline int umma_smem_bytes(int BN, int cluster, int stages, int a_rows = 128)
+inline int umma_smem_bytes(int BN, int cluster, int stages, int a_rows, bool staging)
 {
-    return stages * (a_rows * 64 * 2 + (int)round_up(BN / cluster, 64) * 64 * 2) + kUmmaBarrierBytes +
-           kUmmaEpilogueWarps * kUmmaWarpStagingBytes + 1024;
+    const int stage = a_rows * 64 * 2 + (int)round_up(BN / cluster, 64) * 64 * 2;
+    const int used = stages * stage + kUmmaBarrierBytes + (staging ? kUmmaEpilogueWarps * kUmmaWarpStagingBytes : 0);
+    // the MMA reads 128 rows of A from every stage, also when the box brought fewer: the rows past the box
+    // of the last stage must still lie inside the allocation
+    const int read_end = (stages - 1) * stage + 128 * 64 * 2;
+    return std::max(used, read_end) + 1024;
+}
+// Deepest ring that fits (0 if not even two stages do).  Only a kernel that writes the 16-bit C itself
+// (P_k = 1) needs the epilogue staging; one that writes fp32 partials spends that space on stages.
+inline int umma_deepest_ring(int BN, int cluster, int a_rows, bool staging, int smem_limit, int cap = kUmmaMaxStages)
+{
+    for (int st = cap; st >= 2; --st)
+        if (umma_smem_bytes(BN, cluster, st, a_rows, staging) <= smem_limit) return st;
+    return 0;
 }
 
 // Rows of A one TMA box brings per stage (a multiple of 8, so the stage stays a multiple of 1024 B).

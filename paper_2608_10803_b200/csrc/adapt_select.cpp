@@ -158,7 +158,7 @@ static void model_epilogue(const Shape& s, Config& c, const Calib& cal)
     c.ws_partial = 0;
     if (c.P_k > 1) {
         const double MN = (double)s.M * (double)s.N;
-        c.ws_partial = round_up((int64_t)c.P_k * s.M * round_up(s.N, 4) * 4, 256);
+        c.ws_partial = round_up((int64_t)c.P_k * s.M * partial_pitch(s.N) * 4, 256);
         double part = 4.0 * MN * c.P_k;
         // partials that fit in L2 are read back at L2 speed; model that as half the HBM cost
         const double factor = part <= kL2Bytes ? 0.5 : 1.0;
@@ -199,7 +199,7 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     // bytes one SM keeps in flight, about hbm_bw_per_sm.  The second case only shows in partial waves.
     const double t_mma_all = 2.0 * (double)s.M * s.N * s.K / cal.tensor_flops;
     const bool mem_bound = 2.0 * (MK * rA + KN * rB) / cal.hbm_bw > t_mma_all;   // the operand stream, not C, outweighs the MMAs
-    double sm_rate = cal.l2_bw_per_sm * (c.srcA == ADAPT_SRC_TMA_CLASSES ? cal.class_view_sm_eff : 1.0);
+    double sm_rate = cal.l2_bw_per_sm * (c.srcA == ADAPT_SRC_TMA_CLASSES ? cal.class_view_sm_eff : (kclasses ? cal.kclass_view_sm_eff : 1.0));
     if (mem_bound && c.srcA == ADAPT_SRC_TMA_CLASSES) sm_rate = std::min(sm_rate, cal.hbm_bw_per_sm);   // measured for the views only
     double tM = stage_bytes / sm_rate * 1e6;
     // relative tensor efficiency, measured at BN = 64, 128, 256 and interpolated for the halo tiles between them
@@ -310,7 +310,8 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     if (2 * c.BN > m.tmem_cols) return false;                       // at least two accumulator buffers in TMEM
     if (c.stages < 1 || c.stages > kUmmaMaxStages) return false;
     c.smem_bytes = umma_smem_bytes(c.BN, c.cluster, c.stages,
-                                   umma_a_box_rows(s, c.cluster, umma_row_classes(c.srcA, c.BN), c.srcB == ADAPT_SRC_TMA_CLASSES));
+                                   umma_a_box_rows(s, c.cluster, umma_row_classes(c.srcA, c.BN), c.srcB == ADAPT_SRC_TMA_CLASSES),
+                                   c.P_k == 1);
     if (c.smem_bytes > m.smem_bytes) return false;
     // in class mode the k index of a tile is shifted by up to 7 elements
     // k-class mode splits the blocks of one class; in row-class mode the k index is shifted by up to 7
@@ -332,7 +333,8 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
         // k-rows of one residue class share their misalignment: row-major B with N % 8 != 0, 64-column
         // windows that own 56 columns, A regrouped class-major by a prologue copy (any layout of A)
         // (BN = 64: eight class accumulators per tile; BN = 128, 256: each class a k split, BN - 8 columns owned)
-        if (c.family != ADAPT_FAM_UMMA_1CTA || s.layoutB != ADAPT_ROW_MAJOR || c.BN % 64 != 0) return false;
+        if (s.layoutB != ADAPT_ROW_MAJOR || c.BN % 64 != 0) return false;
+        if (c.family != ADAPT_FAM_UMMA_1CTA && c.BN != 256) return false;    // pair tiles: classes as k splits, 256 columns
         if (aligned16(innerB(s)) || s.K < 64 || c.srcA != ADAPT_SRC_PAD_COPY) return false;
     }
     if (classes) {
@@ -454,24 +456,18 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
             const int64_t tiles = ceil_div(s.M, BM) * ceil_div(s.N, BN);
             split_candidates(tiles, m.n_sm / cluster, ceil_div(s.K, 64), 2, &pks);
             // ring depth: the deepest that fits, and a double buffer (Eq. 13) for comparison
-            Config probe;
-            probe.family = fam; probe.BM = BM; probe.BN = BN; probe.BK = 64; probe.cluster = cluster;
             const int a_rows = umma_a_box_rows(s, cluster, 0, false);
-            int deepest = 0;
-            for (int st = kUmmaMaxStages; st >= 2; --st) {
-                probe.stages = st;
-                if (umma_smem_bytes(probe.BN, probe.cluster, st, a_rows) <= m.smem_bytes) { deepest = st; break; }
-            }
-            if (a_rows == 128 && deepest > 8) deepest = 8;
-            std::vector<int> depths = {deepest};
-            if (deepest > 4) depths.push_back(4);
-            if (deepest > 2) depths.push_back(2);
-            for (int st : depths) {
-                for (int pk : pks) {
+            for (int pk : pks) {
+                int deepest = umma_deepest_ring(BN, cluster, a_rows, pk == 1, m.smem_bytes);
+                if (a_rows == 128 && deepest > 8) deepest = 8;
+                std::vector<int> depths = {deepest};
+                if (deepest > 4) depths.push_back(4);
+                if (deepest > 2) depths.push_back(2);
+                for (int st : depths) {
                     Config c;
                     c.family = fam; c.BM = BM; c.BN = BN; c.BK = 64; c.cluster = cluster;
                     c.stages = st; c.P_k = pk; c.srcA = srcA; c.srcB = srcB;
-                    if (finalize(s, m, cal, c)) out->push_back(c);
+                    if (st >= 2 && finalize(s, m, cal, c)) out->push_back(c);
                 }
             }
         }
@@ -485,10 +481,8 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
             if (!halo && srcA != ADAPT_SRC_PAD_COPY) continue;             // aligned A: class tiles only for their stores
             const int64_t tiles = (halo ? 16 * ceil_div(s.M, 2048) : 8 * ceil_div(s.M, 1024)) * ceil_div(s.N, halo ? BN - 16 : BN);
             split_candidates(tiles, m.n_sm, ceil_div(s.K + (s.K % 8 ? 7 : 0), 64), 2, &pks);
-            int deepest = 0;
-            for (int st = kUmmaMaxStages; st >= 2; --st)
-                if (umma_smem_bytes(BN, 1, st, umma_a_box_rows(s, 1, BN % 64 ? 16 : 8, false)) <= m.smem_bytes) { deepest = st; break; }
             for (int pk : pks) {
+                const int deepest = umma_deepest_ring(BN, 1, umma_a_box_rows(s, 1, halo ? 16 : 8, false), pk == 1, m.smem_bytes);
                 Config d;
                 d.family = ADAPT_FAM_UMMA_1CTA; d.BM = 128; d.BN = BN; d.BK = 64; d.cluster = 1;
                 d.stages = deepest; d.P_k = pk; d.srcA = ADAPT_SRC_TMA_CLASSES; d.srcB = srcB;
@@ -501,10 +495,8 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
     if (srcB == ADAPT_SRC_PAD_COPY && s.layoutB == ADAPT_ROW_MAJOR && s.K >= 64) {
         const int64_t tiles = ceil_div(s.M, 128) * ceil_div(s.N, 56);
         split_candidates(tiles, m.n_sm, ceil_div(ceil_div(s.K, 8), 64), 1, &pks);
-        int deepest = 0;
-        for (int st = kUmmaMaxStages; st >= 2; --st)
-            if (umma_smem_bytes(64, 1, st, umma_a_box_rows(s, 1, 0, true)) <= m.smem_bytes) { deepest = st; break; }
         for (int pk : pks) {
+            const int deepest = umma_deepest_ring(64, 1, umma_a_box_rows(s, 1, 0, true), pk == 1, m.smem_bytes);
             Config d;
             d.family = ADAPT_FAM_UMMA_1CTA; d.BM = 128; d.BN = 64; d.BK = 64; d.cluster = 1;
             d.stages = deepest; d.P_k = pk; d.srcA = ADAPT_SRC_PAD_COPY; d.srcB = ADAPT_SRC_TMA_CLASSES;
@@ -513,16 +505,17 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
     }
     // --- the same views with each class a k split: full-width tiles, 8 fp32 partials per output ---
     if (srcB == ADAPT_SRC_PAD_COPY && s.layoutB == ADAPT_ROW_MAJOR && s.K >= 64) {
-        for (int BN : {128, 256}) {
-            const int64_t tiles = ceil_div(s.M, 128) * ceil_div(s.N, BN - 8);
-            split_candidates(tiles * 8, m.n_sm, ceil_div(ceil_div(s.K, 8), 64), 1, &pks);
+        for (int v = 0; v < 3; ++v) {                               // 1-CTA tiles of 128 and 256 columns, pair tiles of 256
+            const int BN = v == 0 ? 128 : 256, cluster = v == 2 ? 2 : 1, BM = 128 * cluster;
+            const int64_t tiles = ceil_div(s.M, BM) * ceil_div(s.N, BN - 8);
+            split_candidates(tiles * 8, m.n_sm / cluster, ceil_div(ceil_div(s.K, 8), 64), 1, &pks);
             if (std::find(pks.begin(), pks.end(), 1) == pks.end()) pks.insert(pks.begin(), 1);
-            int deepest = 0;
-            for (int st = kUmmaMaxStages; st >= 2; --st)
-                if (umma_smem_bytes(BN, 1, st, umma_a_box_rows(s, 1, 0, true)) <= m.smem_bytes) { deepest = st; break; }
+            const int deepest = umma_deepest_ring(BN, cluster, umma_a_box_rows(s, cluster, 0, true), false, m.smem_bytes,
+                                                  cluster == 2 ? 8 : kUmmaMaxStages);
             for (int pkk : pks) {
                 Config d;
-                d.family = ADAPT_FAM_UMMA_1CTA; d.BM = 128; d.BN = BN; d.BK = 64; d.cluster = 1;
+                d.family = cluster == 2 ? ADAPT_FAM_UMMA_2CTA : ADAPT_FAM_UMMA_1CTA;
+                d.BM = BM; d.BN = BN; d.BK = 64; d.cluster = cluster;
                 d.stages = deepest; d.P_k = 8 * pkk; d.srcA = ADAPT_SRC_PAD_COPY; d.srcB = ADAPT_SRC_TMA_CLASSES;
                 if (deepest >= 2 && 8 * pkk <= 1023 && finalize(s, m, cal, d)) out->push_back(d);
             }

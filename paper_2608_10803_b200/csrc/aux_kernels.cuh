@@ -109,7 +109,7 @@ regroup_a_kernel(const unsigned short* __restrict__ A, unsigned short* __restric
 
 // ---- split-K reduction: C = RN16( sum_{p = 0..P_k-1} partial[p] ), ascending p, fp32 ---------------
 // The order is fixed, so the result does not depend on which CTA finished first.  Partials are
-// stored [P_k][M][Np] with Np = N rounded up to 4, so every row starts on a 16-byte boundary and
+// stored [P_k][M][Np] with Np = N rounded up to 8, so every row starts on a 32-byte boundary and
 // one thread reduces four consecutive columns with 16-byte loads.
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float* __restrict__ partial, unsigned short* __restrict__ C,
@@ -159,7 +159,7 @@ struct SimtParams {
     int64_t a_sm, a_sk;          // element strides of A along m and k
     int64_t b_sk, b_sn;          // element strides of B along k and n
     int P_n, P_k, kb_per_split;  // n tiles; k splits; k-blocks of 16 per split
-    int Np;                      // row pitch of the partials (N rounded up to 4)
+    int Np;                      // row pitch of the partials (N rounded up to 8)
     int dtype;
     unsigned short* C;
     float* partial;

@@ -326,7 +326,7 @@ inline adapt_status_t launch_skinny(const Shape& s, const Config& c, const void*
         kc = s.layoutB == ADAPT_COL_MAJOR;
         p.ld = kc ? s.K : s.N;
         p.out_ss = s.N; p.out_sr = 1;
-        p.part_ss = round_up(s.N, 4); p.part_sr = 1;
+        p.part_ss = partial_pitch(s.N); p.part_sr = 1;
     } else {
         // Small = B^T, streamed = A^T
         p.Small = (const unsigned short*)B;
@@ -336,7 +336,7 @@ inline adapt_status_t launch_skinny(const Shape& s, const Config& c, const void*
         kc = s.layoutA == ADAPT_ROW_MAJOR;
         p.ld = kc ? s.K : s.M;
         p.out_ss = 1; p.out_sr = s.N;
-        p.part_ss = 1; p.part_sr = round_up(s.N, 4);
+        p.part_ss = 1; p.part_sr = partial_pitch(s.N);
     }
     p.K = (int)s.K;
     p.BNs = c.BN;
@@ -347,7 +347,7 @@ inline adapt_status_t launch_skinny(const Shape& s, const Config& c, const void*
     p.dtype = s.dtype;
     p.C = (unsigned short*)C;
     p.partial = partial;
-    p.part_slab = s.M * round_up(s.N, 4);
+    p.part_slab = s.M * partial_pitch(s.N);
     // every group this kernel loads starts at Str + row * ld + (multiple of 8)
     const bool aligned = (p.ld % 8 == 0) && ((uintptr_t)p.Str % 16 == 0);
     dim3 grid((unsigned)ceil_div(p.R, p.BNs), (unsigned)c.P_k, 1);

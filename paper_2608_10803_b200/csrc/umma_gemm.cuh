@@ -38,7 +38,7 @@ struct UmmaParams {
     int stages;
     uint32_t idesc;                  // tcgen05 instruction descriptor
     void* C;                         // 16-bit output, row-major M x N (used when P_k == 1)
-    float* partial;                  // fp32 [P_k][M][Np], Np = N rounded up to 4 (used when P_k > 1)
+    float* partial;                  // fp32 [P_k][M][Np], Np = N rounded up to 8 (used when P_k > 1)
     int Np;                          // row pitch of the partials in elements
     int a_tx_bytes;                  // bytes one TMA load of A delivers per stage and CTA (a short box when M < 128)
     int a_sigma[16];                 // class mode: shift (elements) of row class j against its 16-byte aligned base
@@ -141,7 +141,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
     constexpr bool A_CLS = MODE == 1;
     constexpr bool B_CLS = MODE == 2;
     constexpr bool B_SPLIT = MODE == 3;                   // k classes as k splits (see below)
-    static_assert(MODE == 0 || (!A_MN && B_MN && CG == 1), "class modes: K-major A, row-major B, one CTA per tile");
+    static_assert(MODE == 0 || (!A_MN && B_MN), "class modes: K-major A, row-major B");
+    static_assert(MODE == 0 || MODE == 3 || CG == 1, "tiles of one row class and tiles with eight class accumulators: one CTA per tile");
     static_assert(!B_CLS || BN == 64, "k-class mode uses 64-column windows");
     // HALO: class tiles for a C whose rows do not start on 32-byte boundaries (N % 16 != 0) own 32-byte
     // units of the shifted rows instead of columns, so they compute 16 columns more than they own (see
@@ -615,8 +616,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     }
                 }
             } else {
-                // fp32 partial tile: rows of the workspace are 16-byte aligned (pitch Np), so a thread
-                // writes its row's 32 columns as eight aligned 16-byte stores
+                // fp32 partial tile: rows of the workspace are 32-byte aligned (pitch Np), so a thread
+                // writes its row's 32 columns as four aligned 32-byte stores (whole sectors)
                 if (B_CLS) {
                     if (half == 0) {
 #pragma unroll 1
@@ -628,8 +629,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                             const int col = n0 + 8 * c;
                             float* prow = p.partial + ((size_t)split * p.M + row) * p.Np + col;
                             if (col + 8 <= p.Np) {
-                                *reinterpret_cast<uint4*>(prow) = make_uint4(r8[0], r8[1], r8[2], r8[3]);
-                                *reinterpret_cast<uint4*>(prow + 4) = make_uint4(r8[4], r8[5], r8[6], r8[7]);
+                                ptx::st_global_v8(prow, r8);
                             } else {
 #pragma unroll
                                 for (int j = 0; j < 8; ++j)
@@ -664,9 +664,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                         float* prow = p.partial + ((size_t)split * p.M + row) * p.Np + col;
                         if (col + width <= p.Np) {
 #pragma unroll
-                            for (int v = 0; v < 8; ++v)
-                                if (4 * v < width)
-                                    *reinterpret_cast<uint4*>(prow + 4 * v) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                            for (int v = 0; v < 4; ++v)
+                                if (8 * v < width) ptx::st_global_v8(prow + 8 * v, r + 8 * v);
                         } else {
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
@@ -686,8 +685,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     float* prow = p.partial + ((size_t)split * p.M + row) * p.Np + col;
                     if (col + 32 <= p.Np) {
 #pragma unroll
-                        for (int v = 0; v < 8; ++v)
-                            *reinterpret_cast<uint4*>(prow + 4 * v) = make_uint4(r[4 * v], r[4 * v + 1], r[4 * v + 2], r[4 * v + 3]);
+                        for (int v = 0; v < 4; ++v) ptx::st_global_v8(prow + 8 * v, r + 8 * v);
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)

@@ -266,7 +266,10 @@ def kclass_mode_variants(M, N, K, dtype, layoutA=ROW, limit=4):
     cands = [c for c in ab.adapt_plan_candidates(M, N, K, dtype, layoutA, ROW) if c.srcB == 3]
     picked = [c for c in cands if c.BN == 64][:limit]
     split = [c for c in cands if c.BN != 64]
-    picked += [c for c in split if c.P_k == 8][: limit // 2] + [c for c in split if c.P_k > 8][: limit // 2]
+    one = [c for c in split if c.family == ab.FAM_UMMA_1CTA]
+    pair = [c for c in split if c.family == ab.FAM_UMMA_2CTA]
+    for group in (one, pair):
+        picked += [c for c in group if c.P_k == 8][: limit // 2] + [c for c in group if c.P_k > 8][: limit // 2]
     return [(ab.adapt_matmul_plan_forced(M, N, K, dtype, layoutA, ROW, c.tiling_key), c) for c in picked]
 
 
@@ -280,7 +283,8 @@ def test_k_class_views_bit_exact(shape, dtype):
     variants = kclass_mode_variants(M, N, K, dtype)
     assert variants, "shape must offer the k-class source for B"
     assert any(c.P_k > 1 for _, c in variants) or K < 1024
-    assert any(c.BN != 64 for _, c in variants), "classes as k splits must be on offer"
+    assert any(c.BN != 64 and c.family == ab.FAM_UMMA_1CTA for _, c in variants), "classes as k splits must be on offer"
+    assert any(c.family == ab.FAM_UMMA_2CTA for _, c in variants), "... and on pair tiles"
     for plan, c in variants:
         check_case(M, N, K, dtype, A, B, plan=plan, exact=True)
 

@@ -150,7 +150,7 @@ def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
                     if c.srcB == 3:
                         # k classes: A regrouped class-major, BN - 8 output columns per tile; BN = 64 keeps eight
                         # class accumulators per tile, BN = 128 / 256 makes each class a k split
-                        assert N % 8 and K >= 64 and c.family == ab.FAM_UMMA_1CTA and c.BN in (64, 128, 256)
+                        assert N % 8 and K >= 64 and c.BN in (64, 128, 256) and (c.family == ab.FAM_UMMA_1CTA or c.BN == 256)
                         assert c.srcA == 1 and c.P_n == -(-N // (c.BN - 8))
                         if c.BN != 64:
                             assert c.P_k % 8 == 0
