@@ -117,6 +117,7 @@ struct State {
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
     std::atomic<int64_t> launches{0};
     int log = 0;
+    bool class_promo128 = true;        // 128-byte L2 promotion for the strided class views (ADAPT_CLASS_PROMO128=0: 256 as for dense operands)
 };
 
 State& st()
@@ -130,6 +131,7 @@ void apply_env(State& S)
     if (const char* e = getenv("ADAPT_FAMILY_MASK")) S.machine.family_mask = (unsigned)strtoul(e, nullptr, 0);
     if (const char* e = getenv("ADAPT_LOG")) S.log = atoi(e);
     if (const char* e = getenv("ADAPT_NO_PDL")) pdl_enabled() = atoi(e) == 0;
+    if (const char* e = getenv("ADAPT_CLASS_PROMO128")) S.class_promo128 = atoi(e) != 0;
     if (const char* e = getenv("ADAPT_WORKSPACE_LIMIT_MB")) S.machine.workspace_limit = (int64_t)atoll(e) << 20;
 }
 
@@ -514,7 +516,7 @@ adapt_status_t get_workspace(State& S, cudaStream_t stream, size_t bytes, void**
 
 // 2D tensor map over a dense 16-bit matrix [outer][pitch] whose logical inner extent is `inner`.
 adapt_status_t encode_map(State& S, CUtensorMap* map, const void* base, int dtype, int64_t inner, int64_t outer,
-                          int64_t pitch, int box_inner, int box_outer)
+                          int64_t pitch, int box_inner, int box_outer, bool strided_view = false)
 {
     const cuuint64_t gdim[2] = {(cuuint64_t)inner, (cuuint64_t)outer};
     const cuuint64_t gstride[1] = {(cuuint64_t)pitch * 2};
@@ -522,7 +524,10 @@ adapt_status_t encode_map(State& S, CUtensorMap* map, const void* base, int dtyp
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = S.encode(map, dtype == 0 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
                                 const_cast<void*>(base), gdim, gstride, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                CU_TENSOR_MAP_SWIZZLE_128B,
+                                // the class views touch 128 bytes of a row and then jump 8 or 16 rows: fetching 256
+                                // bytes around each piece doubles their L2 traffic
+                                (strided_view && S.class_promo128) ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         char buf[32];
@@ -583,7 +588,7 @@ adapt_status_t cached_class_maps(State& S, Plan* pl, int which, const void* base
         const int64_t rows = std::max<int64_t>(1, ceil_div(rows_total - j, ncls));
         int64_t inner = cols + sigma[j];
         if (whole_units) inner = std::max<int64_t>(unit, inner / unit * unit);
-        adapt_status_t r = encode_map(S, &sl.map[j], base, pl->s.dtype, inner, rows, (int64_t)ncls * cols, 64, box_rows);
+        adapt_status_t r = encode_map(S, &sl.map[j], base, pl->s.dtype, inner, rows, (int64_t)ncls * cols, 64, box_rows, true);
         if (r != ADAPT_OK) return r;
     }
     sl.ptr = base_ptr;

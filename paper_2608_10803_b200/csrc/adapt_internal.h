@@ -31,6 +31,7 @@ struct Calib {
     double eta_mma_bn64 = 0.45;         // ... at BN = 64 (A-operand smem reads dominate)
     double eta_2cta = 1.0;              // pair tiles share B: no extra tensor cost
     double mem_latency_us = 1.0;        // TMA issue -> data visible (sets Delta_dep with few stages)
+    double hbm_latency_us = 2.7;        // the same under a full HBM stream (45312 x 5 x 96681: 6 stages of 16 KB reach 30 GB/s per SM)
     double umma_fixed_us = 2.5;         // barrier init, TMEM alloc, first load, last drain, TMEM free
     // drain of one output tile through the epilogue warps (overlaps the next tile's main loop):
     // fixed part per tile + part per KB written; rows of C that are not 16-byte aligned cost more
@@ -49,9 +50,9 @@ struct Calib {
     double class_view_sm_eff = 0.85;    // per-SM rate through those views relative to l2_bw_per_sm (20000 x 8 x 60001 tail wave)
     double class_tile_fixed_us = 0.5, class_tile_fixed_unaligned_us = 0.9;   // per class tile (44479 x 54634 x 16..72, 64-column tiles)
     double kclass_view_sm_eff = 0.65;   // per-SM rate through the k-class views of B relative to l2_bw_per_sm (272 x 67839 x 6046: 48 KB per 0.75 us)
-    double class_split_bw_eff = 0.88;   // HBM rate through the k-class views of B with full-width tiles (classes as k splits)
+    double class_split_bw_eff = 0.92;   // HBM rate through the k-class views of B with full-width tiles (classes as k splits)
     double regroup_bw_eff = 0.3;        // class-major regrouping of A (element-wise reads) relative to hbm_bw
-    double class_view_bw_eff = 0.65;    // HBM rate through the per-row-class TMA views of an unaligned A
+    double class_view_bw_eff = 0.8;     // HBM rate through the per-row-class TMA views of an unaligned A
 };
 
 // ---- one configuration x of the search set S(b(s)) (Eq. 6) ------------------------------------

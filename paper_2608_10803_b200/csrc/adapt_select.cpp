@@ -227,7 +227,8 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     if (c.stages <= 1) {
         pipe = pipeline_time(0, Q, L, tM + cal.mem_latency_us, tP, t_drain);                  // Eq. 12
     } else {
-        tM = std::max(tM, cal.mem_latency_us / (c.stages - 1));
+        // a stream that comes from HBM sees the loaded-memory latency, not the L2 one
+        tM = std::max(tM, (mem_bound ? cal.hbm_latency_us : cal.mem_latency_us) / (c.stages - 1));
         const double ii = std::max(tM, tP);
         // class tiles pay a fixed cost per tile (strided row views; zeroing the heads of an unaligned A)
         const double t_fixed = c.srcA != ADAPT_SRC_TMA_CLASSES ? 0.0
@@ -242,7 +243,16 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     // strided row-class views stream A at a lower rate than a dense tensor (measured 3.5-4.1 TB/s)
     const double bw = ksplit_cls ? cal.hbm_bw * cal.class_split_bw_eff
                     : (c.srcA == ADAPT_SRC_TMA_CLASSES || kclasses) ? cal.hbm_bw * cal.class_view_bw_eff : cal.hbm_bw;
-    const double t_hbm = c.hbm_bytes / bw * 1e6 - c.t_pro_us - c.t_epi_us;
+    // A row-major B arrives as k-rows of BN contiguous columns per tile: short pieces stream below the
+    // HBM rate (8 x 30016 x 40000: 3.6 / 5.5 / 6.9 TB/s at 128 / 256 / 512 bytes)
+    double t_b_extra = 0.0;
+    if (s.layoutB == ADAPT_ROW_MAJOR) {
+        const double piece = 2.0 * c.BN;
+        const double eff = piece >= 512 ? 1.0 : (piece >= 256 ? 0.8 + 0.2 * (piece - 256) / 256 : 0.52 + 0.28 * (piece - 128) / 128);
+        const double b_bytes = 2.0 * KN * rB * (kclasses ? c.BN / (c.BN - 8.0) : 1.0);
+        t_b_extra = b_bytes / bw * (1.0 / std::max(eff, 0.3) - 1.0) * 1e6;
+    }
+    const double t_hbm = c.hbm_bytes / bw * 1e6 + t_b_extra - c.t_pro_us - c.t_epi_us;
     c.t_main_us = std::max(pipe, t_hbm);
     finish_common(s, c, cal);
 }
@@ -431,6 +441,12 @@ static void split_candidates(int64_t tiles_mn, int64_t slots, int64_t ksteps, in
     }
     for (int64_t p = 2; p <= 1024; p *= 2) want.push_back(p);
     want.push_back(3); want.push_back(6); want.push_back(12); want.push_back(24);
+    // split counts that fill whole waves: the smallest few with at most 3 % of the last wave idle
+    int balanced = 0;
+    for (int64_t w = 2; w <= std::min<int64_t>(max_pk, 96) && balanced < 3; ++w) {
+        const int64_t units = tiles_mn * w, waves = ceil_div(units, slots);
+        if ((double)units >= 0.97 * (double)(waves * slots)) { want.push_back(w); ++balanced; }
+    }
     for (int64_t w : want) {
         if (w < 2 || w > max_pk) continue;
         // normalise so that no split is empty
