@@ -582,7 +582,8 @@ def validate_model(args):
     cases = synth.config_sweep()
     rng = np.random.default_rng(7)
     order = [int(i) for i in rng.permutation(len(cases))]
-    picked = [i for i in order if 5e-6 <= t_roof_nominal(cases[i]) and cases[i].bytes < 3e9][: args.validate_model]
+    picked = [i for i in order if args.validate_roof_us * 1e-6 <= t_roof_nominal(cases[i]) and cases[i].bytes < 3e9][: args.validate_model]
+    cand_rows = []
     hits, regrets, rows = 0, [], []
     for i in picked:
         c = cases[i]
@@ -602,6 +603,9 @@ def validate_model(args):
             e1.record()
             torch.cuda.synchronize()
             times.append(e0.elapsed_time(e1) / reps * 1e3)
+        for cand, t in zip(cands, times):
+            cand_rows.append((c.M, c.N, c.K, c.dtype, ab.FAMILY_NAMES[cand.family], cand.BN, cand.stages, cand.P_k, cand.srcA,
+                              cand.srcB, cand.predicted_us, cand.t_pro_us, cand.t_main_us, cand.t_epi_us, t))
         best = int(np.argmin(times))
         hits += int(best == 0 or times[0] <= 1.02 * times[best])
         regrets.append(times[0] / times[best])
@@ -612,6 +616,11 @@ def validate_model(args):
                                 "geomean_regret": geomean(regrets),
                                 "note": "regret = time of the model's pick / time of the fastest legal configuration; the paper reports 63.86 % exact hits on its own hardware"}}
     print(json.dumps(out))
+    if args.dump_candidates:
+        with open(args.dump_candidates, "w") as f:
+            f.write("M,N,K,dtype,family,BN,stages,P_k,srcA,srcB,pred_us,t_pro,t_main,t_epi,time_us\n")
+            for r in cand_rows:
+                f.write(",".join(f"{x:.3f}" if isinstance(x, float) else str(x) for x in r) + "\n")
     if args.dump:
         with open(args.dump, "w") as f:
             f.write("M,N,K,candidates,picked_us,best_us,predicted_us\n")
@@ -637,6 +646,8 @@ def main():
     ap.add_argument("--vendor", action="store_true", help="also time torch.matmul (cuBLAS) per shape as a vendor reference")
     ap.add_argument("--validate-model", type=int, default=0,
                     help="time every legal configuration of this many seeded sweep shapes and report how often the model's pick is the fastest")
+    ap.add_argument("--validate-roof-us", type=float, default=5.0, help="with --validate-model: only shapes whose nominal roofline time is at least this")
+    ap.add_argument("--dump-candidates", default="", help="with --validate-model: write every timed configuration (prediction and time) to this CSV")
     ap.add_argument("--shape", default="", help="M,N,K,dtype: time this one shape only (dtype 0 = fp16, 1 = bf16)")
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--family", type=int, default=-1, help="with --shape: force a kernel family (0 umma_1cta, 1 umma_2cta, 2 skinny, 3 simt)")
