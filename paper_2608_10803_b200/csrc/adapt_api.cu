@@ -406,7 +406,11 @@ extern "C" adapt_status_t adapt_init(int device)
     CUDA_TRY(cudaSetDevice(device));
     cudaDeviceProp prop;
     CUDA_TRY(cudaGetDeviceProperties(&prop, device));
-    if (prop.major != 10) return fail(ADAPT_ERR_UNSUPPORTED, "device is not sm_100 (%s)", prop.name);
+    if (prop.major != 10) {
+        char name[128];            // the message buffer holds 256 bytes
+        snprintf(name, sizeof(name), "%.120s", prop.name);
+        return fail(ADAPT_ERR_UNSUPPORTED, "device is not sm_100 (%s)", name);
+    }
     if (S.all_plans.empty()) apply_env(S);
     S.machine.n_sm = prop.multiProcessorCount;
     S.machine.smem_bytes = (int)prop.sharedMemPerBlockOptin;

@@ -254,9 +254,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                             ptx::tma_load_2d(sA + A_BYTES, &maps.b[B_CLS ? j : 0], full_bar + 8u * stage, col0, kb * kUmmaBK);
                             if (++stage == S) { stage = 0; phase ^= 1u; }
                         }
-                    continue;
                 }
-                for (int kb = kb0; kb < kb1; ++kb) {
+                for (int kb = kb0; !B_CLS && kb < kb1; ++kb) {
                     if (!ptx::mbar_wait(empty_bar + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                     const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
                     const uint32_t sB = sA + A_BYTES;
