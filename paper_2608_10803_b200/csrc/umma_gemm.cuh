@@ -41,6 +41,7 @@ struct UmmaParams {
     float* partial;                  // fp32 [P_k][M][Np], Np = N rounded up to 8 (used when P_k > 1)
     int Np;                          // row pitch of the partials in elements
     int a_tx_bytes;                  // bytes one TMA load of A delivers per stage and CTA (a short box when M < 128)
+    int a_shift_any;                 // class mode: some a_sigma[j] != 0 (the MMA warp then zeroes row heads)
     int a_sigma[16];                 // class mode: shift (elements) of row class j against its 16-byte aligned base
     int b_sigma[8];                  // k-class mode: column shift of B's row class j = k % 8
     int cls_kc;                      // k-class mode: padded length of one class segment of A' (multiple of 64)
@@ -292,7 +293,9 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
         // ------------------------------ MMA issuer ---------------------------------------------
         // one thread issues the MMAs; in class mode the whole warp runs the loop so that its other
         // lanes can zero the stale leading elements of A' in the first k-block
-        if ((lane == 0 || A_CLS) && leader) {
+        // (only when some class of A is shifted: with K % 8 == 0 every sigma is zero and one lane is enough)
+        const bool warp_wide = A_CLS && p.a_shift_any != 0;
+        if ((lane == 0 || warp_wide) && leader) {
             int stage = 0;
             uint32_t phase = 0;
             int buf = 0;
@@ -305,7 +308,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
             // in class mode all 32 lanes run this loop: lane 0 waits and the outcome is broadcast, so
             // the lanes never part ways before a __syncwarp
             auto mma_wait = [&](uint32_t bar, uint32_t parity) -> bool {
-                if (!A_CLS) return ptx::mbar_wait(bar, parity, abort_flag);
+                if (!warp_wide) return ptx::mbar_wait(bar, parity, abort_flag);
                 int w = 1;
                 if (lane == 0) w = ptx::mbar_wait(bar, parity, abort_flag) ? 1 : 0;
                 return __shfl_sync(0xffffffffu, w, 0) != 0;
@@ -342,7 +345,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     ptx::tc_fence_after();
                     const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
                     const uint32_t sB = sA + A_BYTES;
-                    if (A_CLS) {
+                    if (warp_wide) {
                         const int sigma = p.a_sigma[mb % NCLS];
                         if (kb == 0 && sigma > 0) {
                             // rows lane, lane+32, ...: chunk 0 of row r sits at r*128 + ((r & 7) << 4)
@@ -422,6 +425,16 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                 }
             };
             const bool row_ok = row < p.M;
+            bool released = false;
+            auto release_accumulator = [&]() {
+                ptx::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    if (CG == 1) ptx::mbar_arrive(tempty_bar + 8u * buf);
+                    else ptx::mbar_arrive_cluster(tempty_bar + 8u * buf, 0);
+                    if (warp == 2) ADAPT_TRACE(7, unit);
+                }
+            };
             if (p.P_k == 1) {
                 // 16-bit output, any N and any base alignment.  A thread converts 64 columns of its row
                 // and stages them in shared memory shifted by the row's misalignment in C, so that
@@ -496,6 +509,12 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                                 uint32_t r[32];
                                 ptx::tmem_ld_32x32(t_row + (uint32_t)(off + 64 * pass + 32 * h), r);
                                 ptx::tmem_ld_wait();
+                                if ((pass == PASSES - 1 || x + 64 >= x_end) && (h == 1 || ncols <= 32)) {
+                                    // the tile's last read of the accumulator: hand the buffer back now, so the MMA
+                                    // of the tile after next starts while this pass is still being packed and stored
+                                    release_accumulator();
+                                    released = true;
+                                }
                                 if (h == 0) {
                                     if (warp == 2 && lane == 0) ADAPT_TRACE(5, unit);
                                     if (lane == 0) ptx::bulk_wait_read<1>();   // the store that last used this box has read it
@@ -693,13 +712,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                 }
             }
             // this warp has read its share of the accumulator: hand the buffer back to the MMA warp
-            ptx::tc_fence_before();
-            __syncwarp();
-            if (lane == 0) {
-                if (CG == 1) ptx::mbar_arrive(tempty_bar + 8u * buf);
-                else ptx::mbar_arrive_cluster(tempty_bar + 8u * buf, 0);
-                if (warp == 2) ADAPT_TRACE(7, unit);
-            }
+            if (!released) release_accumulator();
             if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
         }
         if (lane == 0) ptx::bulk_wait_read<0>();             // TMA stores still reading this warp's staging boxes
