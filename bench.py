@@ -30,8 +30,29 @@ METRIC = "TFLOP/s and roofline fraction per shape (geomean over sweep) on 1 B200
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) over algorithmic bytes, from the ncu
 # captures summarised in profiles/kernels_ncu_full.md (small cases of the same kernels: traffic
 # grows with the bytes a launch moves, so the ratio is applied to the launch's algorithmic bytes).
-# umma_1cta: 16 x 65536 x 4096 stream 543.9 / 539.1 MB; umma_2cta: 4096^3 90.9 / 100.7 MB.
-NCU_TRAFFIC_RATIO = {"umma_1cta": 1.01, "umma_2cta": 0.90}
+# Keyed by kernel variant (family / tiling mode).
+NCU_TRAFFIC_RATIO = {
+    "umma_1cta/halo_class_tiles": 0.93,      # 20000 x 20001 x 12: 746.9 / 801.0 MB (part of C still in L2 at kernel end)
+    "umma_1cta/row_class_tiles": 1.02,       # 20000 x 8 x 60001: 2445.2 / 2401.3 MB
+    "umma_1cta/k_classes_as_splits": 1.04,   # 8 x 30001 x 8000: 497.6 / 480.6 MB
+    "umma_2cta/k_classes_as_splits": 1.04,
+    "umma_1cta/plain_tiles": 1.01,           # 16 x 65536 x 4096: 546.8 / 539.1 MB
+    "umma_2cta/plain_tiles": 0.87,           # 4096^3: 87.9 / 100.7 MB
+}
+
+
+def kernel_variant(ab, info):
+    """Kernel variant of a plan: family / tiling mode (the template instantiations that share an access pattern)."""
+    fam = ab.FAMILY_NAMES[info.family]
+    if not fam.startswith("umma"):
+        return fam
+    if info.srcB == 3:
+        mode = "k_class_accumulators" if info.BN == 64 else "k_classes_as_splits"
+    elif info.srcA == 3:
+        mode = "halo_class_tiles" if info.BN % 64 else "row_class_tiles"
+    else:
+        mode = "plain_tiles"
+    return f"{fam}/{mode}"
 
 
 def measured_peaks():
@@ -357,7 +378,8 @@ def ours(args):
 
     if rank == 0 and per_shape is not None:
         fr_nom, fr_meas, tf = [], [], []
-        fam_time, fam_bytes, fam_flops, fam_n = {}, {}, {}, {}
+        fam_time = {}
+        var_time, var_bytes, var_flops, var_n = {}, {}, {}, {}
         big = []
         for c, info, t in zip(cases, infos, per_shape):
             tr = t_roof_nominal(c)
@@ -366,15 +388,13 @@ def ours(args):
             tf.append(c.flops / t / 1e12)
             if tr >= 20e-6:
                 big.append(tr / t)
-            single = info.P_k == 1 and info.srcA != 1 and info.srcB != 1
             key = ab.FAMILY_NAMES[info.family]
             fam_time[key] = fam_time.get(key, 0.0) + t
-            if single:
-                k2 = key + "_single_launch"
-                fam_time[k2] = fam_time.get(k2, 0.0) + t
-                fam_bytes[k2] = fam_bytes.get(k2, 0.0) + c.bytes
-                fam_flops[k2] = fam_flops.get(k2, 0.0) + c.flops
-                fam_n[k2] = fam_n.get(k2, 0) + 1
+            k2 = kernel_variant(ab, info)
+            var_time[k2] = var_time.get(k2, 0.0) + t
+            var_bytes[k2] = var_bytes.get(k2, 0.0) + c.bytes
+            var_flops[k2] = var_flops.get(k2, 0.0) + c.flops
+            var_n[k2] = var_n.get(k2, 0) + 1
         total_t = sum(per_shape)
         if vendor is not None:
             sp = [v / t for v, t in zip(vendor, per_shape)]
@@ -389,33 +409,30 @@ def ours(args):
             "roofline_frac_geomean_troof_ge_20us": geomean(big), "shapes_troof_ge_20us": len(big),
             "tflops_geomean": geomean(tf), "sum_shape_time_ms": total_t * 1e3,
             "sum_t_roof_nominal_ms": sum(t_roof_nominal(c) for c in cases) * 1e3,
-            "time_share_by_family": {k: v / total_t for k, v in fam_time.items() if not k.endswith("_single_launch")},
+            "time_share_by_family": {k: v / total_t for k, v in fam_time.items()},
+            "time_share_by_kernel_variant": {k: v / total_t for k, v in sorted(var_time.items(), key=lambda kv: -kv[1])},
         }
-        # roofline of the dominant kernel: its launches that run alone (no pad prologue, no reduce)
-        # the dominant kernel is the family with the largest share of the pass; its roofline is taken
-        # over those of its launches that run as a single kernel
-        dom_family = max((k for k in fam_time if not k.endswith("_single_launch")), key=lambda k: fam_time[k])
-        dom = dom_family + "_single_launch"
-        ratio = NCU_TRAFFIC_RATIO.get(dom_family)
-        if dom in fam_time:
-            mem_t = fam_bytes[dom] / peaks["hbm"]
-            ten_t = fam_flops[dom] / peaks["tensor_sustained"]
-            if mem_t >= ten_t:
-                ach = fam_bytes[dom] / fam_time[dom] / 1e9
-                line["roofline"] = {"kernel": dom, "bound": "hbm", "achieved": ach, "peak": peaks["hbm"] / 1e9, "unit": "GB/s",
-                                    "frac": ach / (peaks["hbm"] / 1e9),
-                                    "traffic": ratio * fam_bytes[dom] / fam_n[dom] if ratio else None,
-                                    "peak_source": peaks["source"], "launches": fam_n[dom],
-                                    "avg_launch_us": fam_time[dom] / fam_n[dom] * 1e6,
-                                    "algorithmic_bytes_per_launch": fam_bytes[dom] / fam_n[dom]}
-            else:
-                ach = fam_flops[dom] / fam_time[dom] / 1e12
-                line["roofline"] = {"kernel": dom, "bound": "tensor", "achieved": ach, "peak": peaks["tensor_sustained"] / 1e12,
-                                    "unit": "TFLOP/s", "frac": ach / (peaks["tensor_sustained"] / 1e12),
-                                    "traffic": ratio * fam_bytes[dom] / fam_n[dom] if ratio else None,
-                                    "peak_source": peaks["source"], "launches": fam_n[dom],
-                                    "avg_launch_us": fam_time[dom] / fam_n[dom] * 1e6,
-                                    "algorithmic_flops_per_launch": fam_flops[dom] / fam_n[dom]}
+        # Roofline of the dominant kernel: the kernel variant (family / tiling mode) with the largest share of
+        # the pass.  achieved = sum of algorithmic bytes (or flops) of its calls / sum of their CUDA-event
+        # times; a call's time includes the small prologue (re-pitch of the small operand) or reduce launch
+        # where the variant has one, so the figure is a lower bound for the kernel itself.
+        dom = max(var_time, key=lambda k: var_time[k])
+        ratio = NCU_TRAFFIC_RATIO.get(dom)
+        mem_t = var_bytes[dom] / peaks["hbm"]
+        ten_t = var_flops[dom] / peaks["tensor_sustained"]
+        common = {"kernel": dom, "share_of_pass": var_time[dom] / total_t,
+                  "traffic": ratio * var_bytes[dom] / var_n[dom] if ratio else None,
+                  "peak_source": peaks["source"], "launches": var_n[dom],
+                  "avg_launch_us": var_time[dom] / var_n[dom] * 1e6}
+        if mem_t >= ten_t:
+            ach = var_bytes[dom] / var_time[dom] / 1e9
+            line["roofline"] = dict(common, bound="hbm", achieved=ach, peak=peaks["hbm"] / 1e9, unit="GB/s",
+                                    frac=ach / (peaks["hbm"] / 1e9), algorithmic_bytes_per_launch=var_bytes[dom] / var_n[dom])
+        else:
+            ach = var_flops[dom] / var_time[dom] / 1e12
+            line["roofline"] = dict(common, bound="tensor", achieved=ach, peak=peaks["tensor_sustained"] / 1e12, unit="TFLOP/s",
+                                    frac=ach / (peaks["tensor_sustained"] / 1e12),
+                                    algorithmic_flops_per_launch=var_flops[dom] / var_n[dom])
         if args.dump:
             os.makedirs(os.path.dirname(os.path.abspath(args.dump)), exist_ok=True)
             with open(args.dump, "w") as f:
