@@ -228,7 +228,8 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
         pipe = pipeline_time(0, Q, L, tM + cal.mem_latency_us, tP, t_drain);                  // Eq. 12
     } else {
         // a stream that comes from HBM sees the loaded-memory latency, not the L2 one
-        tM = std::max(tM, (mem_bound ? cal.hbm_latency_us : cal.mem_latency_us) / (c.stages - 1));
+        const bool views = c.srcA == ADAPT_SRC_TMA_CLASSES || kclasses;
+        tM = std::max(tM, (mem_bound ? (views ? cal.hbm_latency_views_us : cal.hbm_latency_us) : cal.mem_latency_us) / (c.stages - 1));
         const double ii = std::max(tM, tP);
         // class tiles pay a fixed cost per tile (strided row views; zeroing the heads of an unaligned A)
         const double t_fixed = c.srcA != ADAPT_SRC_TMA_CLASSES ? 0.0
