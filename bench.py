@@ -55,6 +55,21 @@ def kernel_variant(ab, info):
     return f"{fam}/{mode}"
 
 
+def max_over_ranks(x, dist, device):
+    """The slowest rank's value: a multi-GPU number is timed on the device as the maximum over ranks."""
+    if dist is None:
+        return x
+    import torch
+    t = torch.tensor([x], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replicas_value(units_per_rank, world, seconds):
+    """Whole-job throughput of `world` independent replicas (weak scaling, no data-path collective)."""
+    return units_per_rank * world / seconds
+
+
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -175,7 +190,7 @@ def reference_arm(args):
         return 0
     from paper_2608_10803_b200 import synth
     cases = synth.config_sweep()
-    sample, macs = oracle_sample(cases, 5e10)
+    sample, macs = oracle_sample(cases, args.ref_macs)
     one_pass, threads = run_oracle_sample(sample)
     for _ in range(args.warmup):
         one_pass()
@@ -308,13 +323,10 @@ def ours(args):
     ms_total = ev0.elapsed_time(ev1)
     launches = ab.adapt_launch_count() - launches0
     clocks = sampler.stop()
-    if dist is not None:
-        t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dist, "cuda")
     ms_step = ms_total / args.steps
     flops_pass = sum(c.flops for c in cases)
-    value = flops_pass * world / (ms_step * 1e-3) / 1e12
+    value = replicas_value(flops_pass, world, ms_step * 1e-3) / 1e12
 
     # ---- per-shape timing: R back-to-back calls between two events, rotating buffer sets ----
     per_shape = None
@@ -522,12 +534,9 @@ def e2e(args, cases, plans, pools, stream, world, dist):
     ev1.record()
     torch.cuda.synchronize()
     ms = ev0.elapsed_time(ev1)
-    if dist is not None:
-        t = torch.tensor([ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, dist, "cuda")
     fl = sum(cases[i].flops for i in keep)
-    return {"value": fl * world * args.e2e_steps / (ms * 1e-3) / 1e12, "unit": "TFLOP/s",
+    return {"value": replicas_value(fl * args.e2e_steps, world, ms * 1e-3) / 1e12, "unit": "TFLOP/s",
             "h2d_bytes_per_step": int(sum(2 * (cases[i].M * cases[i].K + cases[i].K * cases[i].N) for i in keep)),
             "d2h_bytes_per_step": int(sum(2 * cases[i].M * cases[i].N for i in keep)),
             "shapes": len(keep), "shapes_left_out": len(cases) - len(keep), "steps": args.e2e_steps, "ms_per_step": ms / args.e2e_steps,
@@ -665,6 +674,7 @@ def main():
                     help="time every legal configuration of this many seeded sweep shapes and report how often the model's pick is the fastest")
     ap.add_argument("--validate-roof-us", type=float, default=5.0, help="with --validate-model: only shapes whose nominal roofline time is at least this")
     ap.add_argument("--dump-candidates", default="", help="with --validate-model: write every timed configuration (prediction and time) to this CSV")
+    ap.add_argument("--ref-macs", type=float, default=5e10, help="with --impl reference: multiply-accumulates of the oracle's bounded sample per step")
     ap.add_argument("--shape", default="", help="M,N,K,dtype: time this one shape only (dtype 0 = fp16, 1 = bf16)")
     ap.add_argument("--reps", type=int, default=3)
     ap.add_argument("--family", type=int, default=-1, help="with --shape: force a kernel family (0 umma_1cta, 1 umma_2cta, 2 skinny, 3 simt)")
