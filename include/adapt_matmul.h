@@ -69,10 +69,17 @@ typedef enum {
 /* How an operand reaches shared memory (the paper's Padding module, Table 2). */
 typedef enum {
     ADAPT_SRC_TMA = 0,        /* TMA straight from the caller's buffer (needs 16 B pitch and base) */
-    ADAPT_SRC_PAD_COPY = 1,   /* prologue kernel re-pitches the operand into the workspace, then TMA */
+    ADAPT_SRC_PAD_COPY = 1,   /* prologue kernel re-pitches the operand into the workspace, then TMA (with srcB =
+                                 ADAPT_SRC_TMA_CLASSES: A is regrouped class-major instead) */
     ADAPT_SRC_LSU = 2,        /* ordinary loads (skinny / SIMT families) */
-    ADAPT_SRC_TMA_CLASSES = 3 /* row-major A with K % 8 != 0 read in place: one TMA view per row class (row % 8),
-                                 tiles made of every 8th row; no copy, no workspace */
+    ADAPT_SRC_TMA_CLASSES = 3 /* class views, no copy of that operand.
+                                 srcA: row-major A read in place through one TMA view per row class; tiles are made
+                                 of every 8th row (BN = 64, 128, 256; needs K % 8 != 0) or, with 16 halo columns
+                                 (BN = 80, 144, 208; needs N % 16 != 0, any K), of every 16th row, and C is then
+                                 written through per-class TMA stores.
+                                 srcB: row-major B with N % 8 != 0 read in place through one view per k class
+                                 (k % 8); BN = 64 keeps eight class accumulators per tile, BN = 128 / 256 makes
+                                 each class a k split (P_k is then a multiple of 8) */
 } adapt_source_t;
 
 /* Everything the selector decided for one shape.  Filled by adapt_plan_info and
