@@ -731,6 +731,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
 
     p.a_shift_any = 0;
     for (int j = 0; j < 16; ++j) p.a_shift_any |= p.a_sigma[j];
+    if (p.a_shift_any) p.a_shift_any = 1;
     p.dtype = s.dtype;
     // the plan's ring depth assumed its own A box; a fallback to copies may need a shallower ring
     p.stages = c.stages;

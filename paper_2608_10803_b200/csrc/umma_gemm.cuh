@@ -319,6 +319,38 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                 decode_unit(p, unit, mb, nb, split);
                 const int kb0 = (B_SPLIT ? (split >> 3) : split) * p.kb_per_split;
                 const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+                if (warp_wide && kb0 == 0 && kb1 > 0) {
+                    // Class tile whose rows are shifted: the sigma elements in front of each row of the first
+                    // k-block belong to the previous row of A and are zeroed before the tensor core reads them.
+                    // Done here, before the wait for a free accumulator: the loads run ahead of the drain, so
+                    // in the write-bound regime this work hides behind that wait.
+                    const int sigma = p.a_sigma[mb % NCLS];
+                    if (sigma > 0) {
+                        if (!mma_wait(full_bar + 8u * stage, phase)) { ok = false; break; }
+                        // rows lane, lane+32, ...: chunk 0 of row r (its first 8 elements) sits at
+                        // r*128 + ((r & 7) << 4); one masked 16-byte read-modify-write per row
+                        uint8_t* genA = gen_base + (size_t)stage * STAGE_BYTES;
+                        uint32_t keep[4];
+#pragma unroll
+                        for (int w = 0; w < 4; ++w)
+                            keep[w] = (2 * w >= sigma ? 0x0000ffffu : 0u) | (2 * w + 1 >= sigma ? 0xffff0000u : 0u);
+                        uint4 v[4];
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            const int r = lane + 32 * t;
+                            if (r * 128 < A_BYTES) v[t] = *reinterpret_cast<const uint4*>(genA + r * 128 + ((r & 7) << 4));
+                        }
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            const int r = lane + 32 * t;
+                            if (r * 128 < A_BYTES)               // rows past the box are not part of the stage
+                                *reinterpret_cast<uint4*>(genA + r * 128 + ((r & 7) << 4)) =
+                                    make_uint4(v[t].x & keep[0], v[t].y & keep[1], v[t].z & keep[2], v[t].w & keep[3]);
+                        }
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                    }
+                }
                 if (!mma_wait(tempty_bar + 8u * buf, buf_phase ^ 1u)) { ok = false; break; }
                 ptx::tc_fence_after();
                 ADAPT_TRACE(2, unit);
@@ -345,22 +377,6 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     ptx::tc_fence_after();
                     const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
                     const uint32_t sB = sA + A_BYTES;
-                    if (warp_wide) {
-                        const int sigma = p.a_sigma[mb % NCLS];
-                        if (kb == 0 && sigma > 0) {
-                            // rows lane, lane+32, ...: chunk 0 of row r sits at r*128 + ((r & 7) << 4)
-                            uint8_t* genA = gen_base + (size_t)stage * STAGE_BYTES;
-#pragma unroll
-                            for (int t = 0; t < 4; ++t) {
-                                const int r = lane + 32 * t;
-                                if (r * 128 >= A_BYTES) break;           // rows past the box are not part of the stage
-                                unsigned short* h = reinterpret_cast<unsigned short*>(genA + r * 128 + ((r & 7) << 4));
-                                for (int e = 0; e < sigma; ++e) h[e] = 0;
-                            }
-                            ptx::fence_proxy_async_smem();
-                        }
-                        __syncwarp();
-                    }
                     if (lane == 0) {
 #pragma unroll
                         for (int k16 = 0; k16 < kUmmaBK / 16; ++k16) {
