@@ -162,7 +162,8 @@ static void model_epilogue(const Shape& s, Config& c, const Calib& cal)
         double part = 4.0 * MN * c.P_k;
         // partials that fit in L2 are read back at L2 speed; model that as half the HBM cost
         const double factor = part <= kL2Bytes ? 0.5 : 1.0;
-        c.t_epi_us = cal.launch_us + copy_time_us(part * factor + 2.0 * MN, cal);
+        // the reduction kernel walks the P_k slabs eight at a time: one dependent trip to L2 / HBM per batch
+        c.t_epi_us = cal.launch_us + copy_time_us(part * factor + 2.0 * MN, cal) + cal.reduce_batch_us * (double)ceil_div(c.P_k, 8);
         c.hbm_bytes += part * (1.0 + factor);
     }
 }
@@ -234,7 +235,11 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
         // class tiles pay a fixed cost per tile (strided row views; zeroing the heads of an unaligned A)
         const double t_fixed = c.srcA != ADAPT_SRC_TMA_CLASSES ? 0.0
                              : (s.K % 8 ? cal.class_tile_fixed_unaligned_us : cal.class_tile_fixed_us);
-        const double t_tile = std::max((double)L * ii + t_fixed, t_drain);
+        // eight k-class accumulators fill TMEM: one tile at a time, its drain (eight-way sum, thread stores)
+        // is not overlapped with the next tile's main loop
+        const bool one_buffer = kclasses && !ksplit_cls;
+        const double t_tile = one_buffer ? (double)L * ii + cal.kclass_tile_drain_us
+                                         : std::max((double)L * ii + t_fixed, t_drain);
         // Eq. 14 with the drain overlapped: one fill, Q tiles back to back, the last drain exposed
         pipe = tM + (double)Q * t_tile + tP + t_drain;
     }
