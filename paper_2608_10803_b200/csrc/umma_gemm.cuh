@@ -48,6 +48,7 @@ struct UmmaParams {
     int c_mode;                      // 16-bit output: 0 = stores by the epilogue threads (any N, any alignment),
                                      // 1 = TMA stores through the maps of C (rows of C, or of the tile's row class,
                                      //     start on 32-byte boundaries; class tiles with 16 halo columns shift them there)
+    int c_hint;                      // TMA stores of C carry an evict-first L2 policy
     int c_sigma[16];                 // halo class tiles: shift (elements) of C's row class j against its 32-byte aligned base
     int c_extent[16];                // ... and the elements of a shifted row of that class that lie in whole 32-byte units
     unsigned int* status;            // device status word: bit 0 = a bounded wait expired
@@ -230,6 +231,11 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
             uint32_t full_target = full_bar;
             if (CG == 2) asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(full_target) : "r"(full_bar));
             bool ok = true;
+            auto load_a = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int x, int y) {
+                if (CG == 1) ptx::tma_load_2d(dst, tm, bar, x, y);
+                else ptx::tma_load_2d_pair(dst, tm, bar, x, y);
+            };
+            auto load_b = load_a;
             for (int unit = unit0; ok && unit < p.num_units; unit += unit_step) {
                 int mb, nb, split;
                 decode_unit(p, unit, mb, nb, split);
@@ -251,8 +257,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                             if (!ptx::mbar_wait(empty_bar + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
                             const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
                             ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(p.a_tx_bytes + B_BYTES));
-                            ptx::tma_load_2d(sA, tmA, full_bar + 8u * stage, j * p.cls_kc + kb * kUmmaBK, row0);
-                            ptx::tma_load_2d(sA + A_BYTES, &maps.b[B_CLS ? j : 0], full_bar + 8u * stage, col0, kb * kUmmaBK);
+                            load_a(sA, tmA, full_bar + 8u * stage, j * p.cls_kc + kb * kUmmaBK, row0);
+                            load_b(sA + A_BYTES, &maps.b[B_CLS ? j : 0], full_bar + 8u * stage, col0, kb * kUmmaBK);
                             if (++stage == S) { stage = 0; phase ^= 1u; }
                         }
                 }
@@ -265,24 +271,20 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     else if (leader) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, 2 * STAGE_BYTES);
                     const int k0 = kb * kUmmaBK;
                     if (!A_MN) {
-                        if (CG == 1) ptx::tma_load_2d(sA, tmA, fb, k0 + a_k_off, row0);
-                        else ptx::tma_load_2d_pair(sA, tmA, fb, k0 + a_k_off, row0);
+                        load_a(sA, tmA, fb, k0 + a_k_off, row0);
                     } else {
 #pragma unroll
                         for (int j = 0; j < 2; ++j) {
-                            if (CG == 1) ptx::tma_load_2d(sA + j * 8192, tmA, fb, row0 + j * 64, k0);
-                            else ptx::tma_load_2d_pair(sA + j * 8192, tmA, fb, row0 + j * 64, k0);
+                            load_a(sA + j * 8192, tmA, fb, row0 + j * 64, k0);
                         }
                     }
                     if (B_MN) {
 #pragma unroll
                         for (int j = 0; j < B_BOXES; ++j) {
-                            if (CG == 1) ptx::tma_load_2d(sB + j * 8192, tmB, fb, col0 + j * 64, k0 - kshift);
-                            else ptx::tma_load_2d_pair(sB + j * 8192, tmB, fb, col0 + j * 64, k0 - kshift);
+                            load_b(sB + j * 8192, tmB, fb, col0 + j * 64, k0 - kshift);
                         }
                     } else {
-                        if (CG == 1) ptx::tma_load_2d(sB, tmB, fb, k0, col0);
-                        else ptx::tma_load_2d_pair(sB, tmB, fb, k0, col0);
+                        load_b(sB, tmB, fb, k0, col0);
                     }
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
@@ -409,6 +411,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
         uint32_t buf_phase = 0;
         int seq = 0;                                         // tiles this CTA has processed so far
         int tma_box = 0;                                     // TMA-store boxes this warp has issued so far
+        const uint64_t c_policy = ptx::l2_policy_evict_first();
         bool ok = true;
         uint8_t* stg = stage_out + (warp - 2) * kUmmaWarpStagingBytes + lane * kUmmaStageRowBytes;   // this thread's staging row
         unsigned short* srow = reinterpret_cast<unsigned short*>(stg);
@@ -550,7 +553,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                             ptx::fence_proxy_async_smem();
                             __syncwarp();
                             if (lane == 0) {
-                                ptx::tma_store_2d(tmC, ptx::smem_u32(box), x, y0);
+                                if (p.c_hint) ptx::tma_store_2d_hint(tmC, ptx::smem_u32(box), x, y0, c_policy);
+                                else ptx::tma_store_2d(tmC, ptx::smem_u32(box), x, y0);
                                 ptx::bulk_commit();
                                 if (warp == 2) ADAPT_TRACE(6, unit);
                             }
