@@ -124,6 +124,12 @@ __device__ __forceinline__ void tma_store_2d(const void* tmap, uint32_t src, int
                  : "memory");
 }
 // One 32-byte store (a whole sector); p must be 32-byte aligned.
+__device__ __forceinline__ void st_global_v8_hint(void* p, const uint32_t* r, uint64_t policy)
+{
+    asm volatile("st.global.L2::cache_hint.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8}, %9;"
+                 ::"l"(p), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "l"(policy)
+                 : "memory");
+}
 __device__ __forceinline__ void st_global_v8(void* p, const uint32_t* r)
 {
     asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
@@ -136,6 +142,12 @@ __device__ __forceinline__ void tma_store_2d_hint(const void* tmap, uint32_t src
     asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group.L2::cache_hint [%0, {%2, %3}], [%1], %4;"
                  ::"l"(tmap), "r"(src), "r"(x), "r"(y), "l"(policy)
                  : "memory");
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
 }
 __device__ __forceinline__ uint64_t l2_policy_evict_first()
 {

@@ -49,6 +49,7 @@ struct UmmaParams {
                                      // 1 = TMA stores through the maps of C (rows of C, or of the tile's row class,
                                      //     start on 32-byte boundaries; class tiles with 16 halo columns shift them there)
     int c_hint;                      // TMA stores of C carry an evict-first L2 policy
+    int part_hint;                   // fp32 partials are stored with an evict-last L2 policy (they fit in L2)
     int c_sigma[16];                 // halo class tiles: shift (elements) of C's row class j against its 32-byte aligned base
     int c_extent[16];                // ... and the elements of a shifted row of that class that lie in whole 32-byte units
     unsigned int* status;            // device status word: bit 0 = a bounded wait expired
@@ -412,6 +413,12 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
         int seq = 0;                                         // tiles this CTA has processed so far
         int tma_box = 0;                                     // TMA-store boxes this warp has issued so far
         const uint64_t c_policy = ptx::l2_policy_evict_first();
+        // partials that fit in L2 are kept there for the reduction kernel (evict-last)
+        const uint64_t part_policy = ptx::l2_policy_evict_last();
+        auto store_partial8 = [&](float* dst, const uint32_t* r8x) {
+            if (p.part_hint) ptx::st_global_v8_hint(dst, r8x, part_policy);
+            else ptx::st_global_v8(dst, r8x);
+        };
         bool ok = true;
         uint8_t* stg = stage_out + (warp - 2) * kUmmaWarpStagingBytes + lane * kUmmaStageRowBytes;   // this thread's staging row
         unsigned short* srow = reinterpret_cast<unsigned short*>(stg);
@@ -667,7 +674,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                             const int col = n0 + 8 * c;
                             float* prow = p.partial + ((size_t)split * p.M + row) * p.Np + col;
                             if (col + 8 <= p.Np) {
-                                ptx::st_global_v8(prow, r8);
+                                store_partial8(prow, r8);
                             } else {
 #pragma unroll
                                 for (int j = 0; j < 8; ++j)
@@ -703,7 +710,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                         if (col + width <= p.Np) {
 #pragma unroll
                             for (int v = 0; v < 4; ++v)
-                                if (8 * v < width) ptx::st_global_v8(prow + 8 * v, r + 8 * v);
+                                if (8 * v < width) store_partial8(prow + 8 * v, r + 8 * v);
                         } else {
 #pragma unroll
                             for (int j = 0; j < 32; ++j)
@@ -723,7 +730,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     float* prow = p.partial + ((size_t)split * p.M + row) * p.Np + col;
                     if (col + 32 <= p.Np) {
 #pragma unroll
-                        for (int v = 0; v < 4; ++v) ptx::st_global_v8(prow + 8 * v, r + 8 * v);
+                        for (int v = 0; v < 4; ++v) store_partial8(prow + 8 * v, r + 8 * v);
                     } else {
 #pragma unroll
                         for (int j = 0; j < 32; ++j)
