@@ -936,7 +936,7 @@ extern "C" adapt_status_t adapt_matmul_noalloc(int64_t M, int64_t N, int64_t K, 
     const int64_t slab = M * Np * 4;                       // bytes of one split's partial
     if (slab <= 0 || 2 * slab > (int64_t)kNoAllocScratchBytes)
         return fail(ADAPT_ERR_UNSUPPORTED,
-                    "adapt_matmul_noalloc: output too large for the fixed 4 MiB scratch (needs 2 * M * roundup(N,4) * 4 bytes <= 4 MiB)%s");
+                    "adapt_matmul_noalloc: output too large for the fixed 4 MiB scratch (needs 2 * M * roundup(N,8) * 4 bytes <= 4 MiB)%s");
 
     int dev = -1;
     CUDA_TRY(cudaGetDevice(&dev));
