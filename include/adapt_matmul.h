@@ -160,7 +160,7 @@ adapt_status_t adapt_matmul_host(adapt_handle_t plan, const void* A_host, const 
  * It runs the CUDA-core split-K path (fp32 partial products per K split, then the fixed-order
  * reduction with the single 16-bit cast) with the partials kept in a fixed 4 MiB array that is
  * part of the library image, so every GPU that loads the library holds those 4 MiB until the
- * process exits.  Limit: 2 * M * roundup(N, 4) * 4 bytes <= 4 MiB (at least two K splits must
+ * process exits.  Limit: 2 * M * roundup(N, 8) * 4 bytes <= 4 MiB (at least two K splits must
  * fit); larger outputs are rejected with ADAPT_ERR_UNSUPPORTED and a message, and K must be >= 1,
  * M, N >= 1.  The number of splits is the largest that fits, at most 32 and at most ceil(K / 64).
  *
