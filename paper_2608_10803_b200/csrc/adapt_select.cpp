@@ -284,7 +284,11 @@ static void model_skinny(const Shape& s, const Machine& m, const Calib& cal, Con
     const double eff = inner % 8 == 0 ? cal.skinny_bw_eff_aligned : cal.skinny_bw_eff_unaligned;
     // one CTA streams about hbm_bw * eff / (2 * n_sm) when the machine is full; fewer CTAs do not go faster
     const double per_cta_bytes = 2.0 * ((double)c.BN * ceil_div(s.K, c.P_k));
-    const double t_cta = per_cta_bytes / (cal.hbm_bw * eff / (2.0 * m.n_sm)) * 1e6;
+    double t_cta = per_cta_bytes / (cal.hbm_bw * eff / (2.0 * m.n_sm)) * 1e6;
+    // unaligned rows are assembled from two dependent loads per k step: a CTA cannot go faster than that
+    // chain however few bytes it moves (3 x 98900 x 115: 28 us per CTA)
+    const bool k_is_outer = stream_is_B ? s.layoutB == ADAPT_ROW_MAJOR : s.layoutA == ADAPT_COL_MAJOR;   // one streamed row per k
+    if (inner % 8 != 0 && k_is_outer) t_cta = std::max(t_cta, cal.skinny_k_step_unaligned_us * (double)ceil_div(s.K, c.P_k));
     model_epilogue(s, c, cal);
     const double t_alu = macs / cal.skinny_mac_rate * 1e6;
     c.t_pro_us = 0;
