@@ -32,7 +32,7 @@ struct Calib {
     double eta_2cta = 1.0;              // pair tiles share B: no extra tensor cost
     double mem_latency_us = 1.0;        // TMA issue -> data visible (sets Delta_dep with few stages)
     double hbm_latency_us = 1.6;        // the same under a full HBM stream of a dense operand (128 x 128256 x 4096: 5 stages of 32 KB, 0.41 us each)
-    double hbm_latency_views_us = 2.7;  // ... through the strided class views (45312 x 5 x 96681: 6 stages of 16 KB reach 30 GB/s per SM)
+    double hbm_latency_views_us = 1.6;  // ... through the strided class views (79457 x 196 x 8325 with 3 stages: 0.75 us per stage)
     double umma_fixed_us = 2.5;         // barrier init, TMEM alloc, first load, last drain, TMEM free
     // drain of one output tile through the epilogue warps (overlaps the next tile's main loop):
     // fixed part per tile + part per KB written; rows of C that are not 16-byte aligned cost more
