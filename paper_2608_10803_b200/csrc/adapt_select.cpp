@@ -216,7 +216,9 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     // partials always go that way
     const bool halo = c.BN % 64 != 0;
     const int own_n = halo ? c.BN - 16 : c.BN;
-    const double out_tile_kb = (c.P_k > 1 ? 4.0 : 2.0) * 128.0 * own_n / 1024.0;
+    // rows of a tile that exist (short M: the rest is neither stored by the threads nor by TMA)
+    const double rows_valid = std::min(128.0, (double)s.M / ((double)c.P_m * c.cluster));
+    const double out_tile_kb = (c.P_k > 1 ? 4.0 : 2.0) * rows_valid * own_n / 1024.0;
     double t_drain;
     if (c.P_k > 1) t_drain = cal.epi_partial_fixed_us + cal.epi_partial_us_per_kb * out_tile_kb;
     else if (s.N % 16 == 0 || halo) t_drain = cal.epi_tile_fixed_us + cal.epi_us_per_kb * out_tile_kb;
