@@ -141,13 +141,18 @@ adapt_handle_t adapt_matmul_plan(int64_t M, int64_t N, int64_t K,
 adapt_status_t adapt_matmul(adapt_handle_t plan, const void* A, const void* B, void* C, void* cuda_stream);
 
 /* The same call for operands that live in HOST memory (A_host, B_host inputs, C_host output,
- * dense, in the plan's layouts; pinned memory makes the copies asynchronous).  Enqueues on the
- * stream: copy A and B into a library-owned device staging buffer, the planned kernels, copy C
- * back.  Returns without synchronising: the caller synchronises the stream before reading
- * C_host or reusing A_host / B_host.  The staging buffer is per stream and grows on demand
- * (cudaMalloc), like the workspace.  The paper has no counterpart (its operator takes device
- * tensors); this entry exists so that end-to-end cost including the PCIe copies can be measured
- * through one call. */
+ * dense, in the plan's layouts; pinned memory makes the copies asynchronous).  The library runs
+ * the call on a three-stage pipeline of its own streams (copy A and B into a device staging
+ * slot | the planned kernels | copy C back) with two staging slots per caller stream, so the
+ * copies of consecutive calls overlap the kernels and each other.  Returns without
+ * synchronising.  Ordering: the caller's stream is made to wait for the copy of C, so work
+ * enqueued on it after the call (and cudaStreamSynchronize on it) sees C_host complete; the
+ * host operands must be ready when the call is made (the copy in does NOT wait for earlier
+ * work on the caller's stream) and stay untouched until the stream has been synchronised.
+ * Calls that name the same stream must not be made from two threads at once.  The staging
+ * slots grow on demand (cudaMalloc), like the workspace.  The paper has no counterpart (its
+ * operator takes device tensors); this entry exists so that end-to-end cost including the PCIe
+ * copies can be measured through one call. */
 adapt_status_t adapt_matmul_host(adapt_handle_t plan, const void* A_host, const void* B_host, void* C_host,
                                  void* cuda_stream);
 

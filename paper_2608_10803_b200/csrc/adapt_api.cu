@@ -113,7 +113,16 @@ struct State {
     unsigned long long* d_trace = nullptr;   // diagnostic builds only
     struct Workspace { void* ptr = nullptr; size_t bytes = 0; };
     std::unordered_map<cudaStream_t, Workspace> ws;
-    std::unordered_map<cudaStream_t, Workspace> staging;   // device copies of host operands (adapt_matmul_host)
+    // adapt_matmul_host: one three-stage pipeline per caller stream (copy in | kernels | copy out, each on
+    // its own stream) with two staging slots, so the copies of consecutive calls overlap the kernels and
+    // each other (PCIe is full duplex)
+    struct HostPipe {
+        cudaStream_t in = nullptr, comp = nullptr, out = nullptr;
+        cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_comp[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
+        Workspace stage[2];
+        int next = 0;
+    };
+    std::unordered_map<cudaStream_t, HostPipe> pipes;
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
     std::atomic<int64_t> launches{0};
     int log = 0;
@@ -455,8 +464,19 @@ extern "C" void adapt_shutdown(void)
         cudaDeviceSynchronize();
         for (auto& kv : S.ws) if (kv.second.ptr) cudaFree(kv.second.ptr);
         S.ws.clear();
-        for (auto& kv : S.staging) if (kv.second.ptr) cudaFree(kv.second.ptr);
-        S.staging.clear();
+        for (auto& kv : S.pipes) {
+            State::HostPipe& hp = kv.second;
+            for (int b = 0; b < 2; ++b) {
+                if (hp.stage[b].ptr) cudaFree(hp.stage[b].ptr);
+                if (hp.ev_in[b]) cudaEventDestroy(hp.ev_in[b]);
+                if (hp.ev_comp[b]) cudaEventDestroy(hp.ev_comp[b]);
+                if (hp.ev_out[b]) cudaEventDestroy(hp.ev_out[b]);
+            }
+            if (hp.in) cudaStreamDestroy(hp.in);
+            if (hp.comp) cudaStreamDestroy(hp.comp);
+            if (hp.out) cudaStreamDestroy(hp.out);
+        }
+        S.pipes.clear();
         if (S.d_status) cudaFree(S.d_status);
         S.d_status = nullptr;
     }
@@ -492,12 +512,12 @@ extern "C" adapt_status_t adapt_poll_device_status(void* cuda_stream)
 // ---------------------------------------------------------------------------------------------
 namespace {
 
-adapt_status_t get_workspace(State& S, cudaStream_t stream, size_t bytes, void** out, bool staging = false)
+adapt_status_t get_workspace(State& S, cudaStream_t stream, size_t bytes, void** out)
 {
     *out = nullptr;
     if (bytes == 0) return ADAPT_OK;
     std::lock_guard<std::mutex> lock(S.mu);
-    State::Workspace& w = staging ? S.staging[stream] : S.ws[stream];
+    State::Workspace& w = S.ws[stream];
     if (w.bytes < bytes) {
         if (w.ptr) {
             CUDA_TRY(cudaStreamSynchronize(stream));
@@ -881,17 +901,56 @@ extern "C" adapt_status_t adapt_matmul_host(adapt_handle_t plan, const void* A_h
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     const size_t nA = (size_t)round_up(s.M * s.K * 2, 256), nB = (size_t)round_up(s.K * s.N * 2, 256);
     const size_t nC = (size_t)round_up(s.M * s.N * 2, 256);
-    void* dev = nullptr;
-    adapt_status_t r = get_workspace(S, stream, nA + nB + nC, &dev, true);
-    if (r != ADAPT_OK) return r;
-    uint8_t* d8 = (uint8_t*)dev;
-    if (s.K > 0) {
-        CUDA_TRY(cudaMemcpyAsync(d8, A_host, (size_t)s.M * s.K * 2, cudaMemcpyHostToDevice, stream));
-        CUDA_TRY(cudaMemcpyAsync(d8 + nA, B_host, (size_t)s.K * s.N * 2, cudaMemcpyHostToDevice, stream));
+    State::HostPipe* hp = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(S.mu);
+        hp = &S.pipes[stream];
+        if (!hp->in) {
+            CUDA_TRY(cudaStreamCreateWithFlags(&hp->in, cudaStreamNonBlocking));
+            CUDA_TRY(cudaStreamCreateWithFlags(&hp->comp, cudaStreamNonBlocking));
+            CUDA_TRY(cudaStreamCreateWithFlags(&hp->out, cudaStreamNonBlocking));
+            for (int b = 0; b < 2; ++b) {
+                CUDA_TRY(cudaEventCreateWithFlags(&hp->ev_in[b], cudaEventDisableTiming));
+                CUDA_TRY(cudaEventCreateWithFlags(&hp->ev_comp[b], cudaEventDisableTiming));
+                CUDA_TRY(cudaEventCreateWithFlags(&hp->ev_out[b], cudaEventDisableTiming));
+            }
+        }
     }
-    r = adapt_matmul(plan, d8, d8 + nA, d8 + nA + nB, cuda_stream);
+    const int b = hp->next;
+    hp->next ^= 1;
+    // the slot is free once the copy-out of the call that used it last (two calls ago) has finished
+    State::Workspace& w = hp->stage[b];
+    if (w.bytes < nA + nB + nC) {
+        CUDA_TRY(cudaStreamSynchronize(hp->out));
+        if (w.ptr) CUDA_TRY(cudaFree(w.ptr));
+        w.ptr = nullptr;
+        w.bytes = 0;
+        const size_t want = (size_t)round_up((int64_t)(nA + nB + nC) + (int64_t)((nA + nB + nC) >> 3), 1 << 20);
+        cudaError_t e = cudaMalloc(&w.ptr, want);
+        if (e != cudaSuccess) {
+            (void)cudaGetLastError();
+            w.ptr = nullptr;
+            return fail(ADAPT_ERR_NOMEM, "staging allocation failed: %s", cudaGetErrorString(e));
+        }
+        w.bytes = want;
+    } else {
+        CUDA_TRY(cudaStreamWaitEvent(hp->in, hp->ev_out[b], 0));
+    }
+    uint8_t* d8 = (uint8_t*)w.ptr;
+    if (s.K > 0) {
+        CUDA_TRY(cudaMemcpyAsync(d8, A_host, (size_t)s.M * s.K * 2, cudaMemcpyHostToDevice, hp->in));
+        CUDA_TRY(cudaMemcpyAsync(d8 + nA, B_host, (size_t)s.K * s.N * 2, cudaMemcpyHostToDevice, hp->in));
+    }
+    CUDA_TRY(cudaEventRecord(hp->ev_in[b], hp->in));
+    CUDA_TRY(cudaStreamWaitEvent(hp->comp, hp->ev_in[b], 0));
+    adapt_status_t r = adapt_matmul(plan, d8, d8 + nA, d8 + nA + nB, (void*)hp->comp);
     if (r != ADAPT_OK) return r;
-    CUDA_TRY(cudaMemcpyAsync(C_host, d8 + nA + nB, (size_t)s.M * s.N * 2, cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaEventRecord(hp->ev_comp[b], hp->comp));
+    CUDA_TRY(cudaStreamWaitEvent(hp->out, hp->ev_comp[b], 0));
+    CUDA_TRY(cudaMemcpyAsync(C_host, d8 + nA + nB, (size_t)s.M * s.N * 2, cudaMemcpyDeviceToHost, hp->out));
+    CUDA_TRY(cudaEventRecord(hp->ev_out[b], hp->out));
+    // work the caller enqueues on its stream after this call sees C_host complete
+    CUDA_TRY(cudaStreamWaitEvent(stream, hp->ev_out[b], 0));
     return ADAPT_OK;
 }
 

@@ -394,3 +394,42 @@ def test_tma_store_epilogue_leaves_neighbouring_memory_alone():
         err, mism, _ = compare_with_oracle(A, B, out.contiguous(), M, N, K, dtype)
         assert mism == 0
         assert torch.isnan(c_buf[:2048]).all() and torch.isnan(c_buf[2048 + M * N:]).all()
+
+
+# ---- host operands: the pipelined copy-in | kernels | copy-out entry point ------------------------------
+
+def test_host_entry_point_matches_the_oracle_over_a_run_of_calls():
+    """Seven calls back to back on one stream (both staging slots reused several times, growing and
+    shrinking shapes, both dtypes), results read only after one synchronisation at the end."""
+    shapes = [(131, 77, 259, ab.F16), (1030, 265, 331, ab.BF16), (8, 3001, 400, ab.F16), (256, 256, 256, ab.BF16),
+              (5, 640, 1000, ab.F16), (2049, 193, 5, ab.BF16), (300, 520, 12, ab.F16)]
+    st = torch.cuda.current_stream().cuda_stream
+    jobs = []
+    for (M, N, K, dtype) in shapes:
+        A = synth.position_coded(M, K, dtype, 7, "cpu").pin_memory()
+        B = synth.position_coded(K, N, dtype, 5, "cpu").pin_memory()
+        C = torch.full((M, N), float("nan"), dtype=synth.torch_dtype(dtype)).pin_memory()
+        plan = ab.adapt_matmul_plan(M, N, K, dtype)
+        ab.adapt_matmul_host(plan, A.data_ptr(), B.data_ptr(), C.data_ptr(), st)
+        jobs.append((M, N, K, dtype, A, B, C))
+    torch.cuda.synchronize()
+    ab.adapt_poll_device_status(st)
+    for (M, N, K, dtype, A, B, C) in jobs:
+        err, mism, _ = compare_with_oracle(A, B, C, M, N, K, dtype)
+        assert mism == 0, (M, N, K)
+
+
+def test_host_entry_point_twice_is_bit_identical_and_orders_the_callers_stream():
+    M, N, K, dtype = 777, 1001, 513, ab.BF16
+    A = synth.draw_operand(M, K, synth.U11, 5, dtype, "cpu").pin_memory()
+    B = synth.draw_operand(K, N, synth.U11, 6, dtype, "cpu").pin_memory()
+    C1 = torch.zeros((M, N), dtype=synth.torch_dtype(dtype)).pin_memory()
+    C2 = torch.zeros((M, N), dtype=synth.torch_dtype(dtype)).pin_memory()
+    plan = ab.adapt_matmul_plan(M, N, K, dtype)
+    s = torch.cuda.Stream()
+    ab.adapt_matmul_host(plan, A.data_ptr(), B.data_ptr(), C1.data_ptr(), s.cuda_stream)
+    ab.adapt_matmul_host(plan, A.data_ptr(), B.data_ptr(), C2.data_ptr(), s.cuda_stream)
+    s.synchronize()                       # the caller's stream alone: it waits for both copies of C
+    assert torch.equal(C1.view(torch.int16), C2.view(torch.int16))
+    err, _, _ = compare_with_oracle(A, B, C1, M, N, K, dtype)
+    assert err <= TOL[dtype]
