@@ -523,7 +523,7 @@ def e2e(args, cases, plans, pools, stream, world, dist):
             st = mh(plans[i], hA.data_ptr(), hB.data_ptr(), hC.data_ptr(), stream)
             if st != 0:
                 raise RuntimeError(lib.adapt_last_error_message().decode())
-    one_pass(order[:3])            # grows the staging buffer to its final size
+    one_pass(order[:6])            # grows the staging slots to their final sizes
     torch.cuda.synchronize()
     if dist is not None:
         dist.barrier()

@@ -115,11 +115,12 @@ struct State {
     std::unordered_map<cudaStream_t, Workspace> ws;
     // adapt_matmul_host: one three-stage pipeline per caller stream (copy in | kernels | copy out, each on
     // its own stream) with two staging slots, so the copies of consecutive calls overlap the kernels and
-    // each other (PCIe is full duplex)
+    // each other (PCIe is full duplex); a slot is reused once the copy-out of the call that used it last is done
+    static constexpr int kHostSlots = 2;
     struct HostPipe {
         cudaStream_t in = nullptr, comp = nullptr, out = nullptr;
-        cudaEvent_t ev_in[2] = {nullptr, nullptr}, ev_comp[2] = {nullptr, nullptr}, ev_out[2] = {nullptr, nullptr};
-        Workspace stage[2];
+        cudaEvent_t ev_in[kHostSlots] = {}, ev_comp[kHostSlots] = {}, ev_out[kHostSlots] = {};
+        Workspace stage[kHostSlots];
         int next = 0;
     };
     std::unordered_map<cudaStream_t, HostPipe> pipes;
@@ -466,7 +467,7 @@ extern "C" void adapt_shutdown(void)
         S.ws.clear();
         for (auto& kv : S.pipes) {
             State::HostPipe& hp = kv.second;
-            for (int b = 0; b < 2; ++b) {
+            for (int b = 0; b < State::kHostSlots; ++b) {
                 if (hp.stage[b].ptr) cudaFree(hp.stage[b].ptr);
                 if (hp.ev_in[b]) cudaEventDestroy(hp.ev_in[b]);
                 if (hp.ev_comp[b]) cudaEventDestroy(hp.ev_comp[b]);
@@ -909,7 +910,7 @@ extern "C" adapt_status_t adapt_matmul_host(adapt_handle_t plan, const void* A_h
             CUDA_TRY(cudaStreamCreateWithFlags(&hp->in, cudaStreamNonBlocking));
             CUDA_TRY(cudaStreamCreateWithFlags(&hp->comp, cudaStreamNonBlocking));
             CUDA_TRY(cudaStreamCreateWithFlags(&hp->out, cudaStreamNonBlocking));
-            for (int b = 0; b < 2; ++b) {
+            for (int b = 0; b < State::kHostSlots; ++b) {
                 CUDA_TRY(cudaEventCreateWithFlags(&hp->ev_in[b], cudaEventDisableTiming));
                 CUDA_TRY(cudaEventCreateWithFlags(&hp->ev_comp[b], cudaEventDisableTiming));
                 CUDA_TRY(cudaEventCreateWithFlags(&hp->ev_out[b], cudaEventDisableTiming));
@@ -917,8 +918,8 @@ extern "C" adapt_status_t adapt_matmul_host(adapt_handle_t plan, const void* A_h
         }
     }
     const int b = hp->next;
-    hp->next ^= 1;
-    // the slot is free once the copy-out of the call that used it last (two calls ago) has finished
+    hp->next = (hp->next + 1) % State::kHostSlots;
+    // the slot is free once the copy-out of the call that used it last has finished
     State::Workspace& w = hp->stage[b];
     if (w.bytes < nA + nB + nC) {
         CUDA_TRY(cudaStreamSynchronize(hp->out));
