@@ -290,7 +290,18 @@ static void model_skinny(const Shape& s, const Machine& m, const Calib& cal, Con
     // unaligned rows are assembled from two dependent loads per k step: a CTA cannot go faster than that
     // chain however few bytes it moves (3 x 98900 x 115: 28 us per CTA)
     const bool k_is_outer = stream_is_B ? s.layoutB == ADAPT_ROW_MAJOR : s.layoutA == ADAPT_COL_MAJOR;   // one streamed row per k
-    if (inner % 8 != 0 && k_is_outer) t_cta = std::max(t_cta, cal.skinny_k_step_unaligned_us * (double)ceil_div(s.K, c.P_k));
+    if (inner % 8 != 0 && k_is_outer) {
+        // Unaligned rows, one per k: the 8 warps of a CTA tile BN columns by 64 and share the k range among
+        // the rest in steps of 16; a step is a chain of dependent loads (about 2 us).  Within one staged
+        // chunk that chain is the whole cost (3 x 98900 x 115: 20 us); the bandwidth term above was
+        // measured on long k ranges and stays the floor there.
+        const int64_t k_split = ceil_div(s.K, c.P_k);
+        const int64_t wk = std::max<int64_t>(1, 8 / std::max(1, c.BN / 64));
+        const int64_t steps = round_up(ceil_div(std::min<int64_t>(k_split, kSkinnyKChunk), wk), 16) / 16 *
+                              ceil_div(k_split, kSkinnyKChunk);
+        const double t_chain = cal.skinny_step_unaligned_us * (double)steps;
+        t_cta = k_split <= kSkinnyKChunk ? t_chain : std::max(t_cta, t_chain);
+    }
     model_epilogue(s, c, cal);
     const double t_alu = macs / cal.skinny_mac_rate * 1e6;
     c.t_pro_us = 0;

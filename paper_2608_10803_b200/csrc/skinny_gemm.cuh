@@ -172,13 +172,15 @@ skinny_gemm_kernel(const SkinnyParams p)
 
     if (!KC) {
         const int r_warp = r_cta + wr * 64;
-        const int k_sub = kSkinnyKChunk / WK;            // k values one warp covers per chunk
         const int nv = p.R - (r_warp + 8 * g);           // valid columns of this lane's group
         const bool cols_full = r_warp + 64 <= p.R;
         for (int kc0 = k_begin; kc0 < k_end; kc0 += kSkinnyKChunk) {
             __syncthreads();                             // previous chunk fully consumed
             stage_small<PITCH>(p, s_small, kc0, k_end, tid);
             __syncthreads();
+            // the WK warps that share an r range split the chunk's k values evenly (in steps of 16), so a
+            // short k range still keeps all of them busy
+            const int k_sub = ((min(kSkinnyKChunk, k_end - kc0) + WK - 1) / WK + 15) & ~15;
             const int kw0 = kc0 + wk * k_sub;
             // a lane loads rows k+2t, +1, +8, +9 at columns r_warp + 8g .. +7
 #pragma unroll 2
