@@ -52,6 +52,7 @@ struct Calib {
     double class_view_sm_eff = 0.85;    // per-SM rate through those views relative to l2_bw_per_sm (20000 x 8 x 60001 tail wave)
     double class_tile_fixed_us = 0.5, class_tile_fixed_unaligned_us = 0.9;   // per class tile (44479 x 54634 x 16..72, 64-column tiles)
     double kclass_view_sm_eff = 0.55;   // per-SM rate through the k-class views of B relative to l2_bw_per_sm (272 x 67839 x 6046: 48 KB per 0.75 us)
+    double kclass_unit_fixed_us = 1.2;  // per unit of a k class run as a k split (1 x 80711 x 221: 18 units of one k-block in 37 us)
     double kclass_tile_drain_us = 2.5;  // drain of a tile with eight class accumulators (29 x 58492 x 94: 8 tile rounds in 35 us)
     double oob_box_penalty = 0.05;      // main-loop cost of one B box per stage that lies wholly beyond N
     double reduce_batch_us = 0.8;       // split-K reduction: one batch of eight slabs (13 x 420 x 43580: P_k 72 -> 24 saves 13 us)

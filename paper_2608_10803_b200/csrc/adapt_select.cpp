@@ -235,7 +235,9 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
         tM = std::max(tM, (mem_bound ? (views ? cal.hbm_latency_views_us : cal.hbm_latency_us) : cal.mem_latency_us) / (c.stages - 1));
         const double ii = std::max(tM, tP);
         // class tiles pay a fixed cost per tile (strided row views; zeroing the heads of an unaligned A)
-        const double t_fixed = c.srcA != ADAPT_SRC_TMA_CLASSES ? 0.0
+        // (the bubble between the units of a k class shrinks as the unit's main loop grows)
+        const double t_fixed = ksplit_cls ? std::max(0.0, cal.kclass_unit_fixed_us - 0.2 * (double)L * ii)
+                             : c.srcA != ADAPT_SRC_TMA_CLASSES ? 0.0
                              : (s.K % 8 ? cal.class_tile_fixed_unaligned_us : cal.class_tile_fixed_us);
         // eight k-class accumulators fill TMEM: one tile at a time, its drain (eight-way sum, thread stores)
         // is not overlapped with the next tile's main loop
