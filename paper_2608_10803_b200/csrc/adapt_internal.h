@@ -37,6 +37,7 @@ struct Calib {
     // drain of one output tile through the epilogue warps (overlaps the next tile's main loop):
     // fixed part per tile + part per KB written; rows of C that are not 16-byte aligned cost more
     double epi_tile_fixed_us = 0.2, epi_us_per_kb = 0.0275;          // TMA stores (40000 x 40000 x 8: 4.8 TB/s)
+    double pair_drain_factor = 1.15;    // 40000 x 40000 x 8: 780 us on pair tiles, 671 us on 1-CTA tiles
     double epi_partial_fixed_us = 0.32, epi_partial_us_per_kb = 0.0385;   // fp32 partials, stored by the epilogue threads
     double epi_tile_fixed_unaligned_us = 1.45, epi_us_per_kb_unaligned = 0.054;
     double simt_flops = 15e12;          // CUDA-core tile kernel (1000^3: 17e12)

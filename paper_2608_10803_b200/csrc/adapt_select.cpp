@@ -224,6 +224,8 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     else if (s.N % 16 == 0 || halo) t_drain = cal.epi_tile_fixed_us + cal.epi_us_per_kb * out_tile_kb;
     else if (s.N % 8 == 0) t_drain = cal.epi_partial_fixed_us + cal.epi_partial_us_per_kb * out_tile_kb;   // aligned 16-byte stores by the threads
     else t_drain = cal.epi_tile_fixed_unaligned_us + cal.epi_us_per_kb_unaligned * out_tile_kb;
+    // the two CTAs of a pair hand their accumulator back together: a drain-bound pair waits for its slower half
+    if (c.cluster == 2) t_drain *= cal.pair_drain_factor;
     // Delta_dep (Eq. 9): with S stages only S-1 loads are in flight while one is consumed, so a
     // slice cannot issue faster than latency / (S-1); one stage serialises load and compute.
     double pipe;
