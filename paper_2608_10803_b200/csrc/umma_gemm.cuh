@@ -7,12 +7,15 @@
 //   producer warp : TMA, 128-byte swizzle, into an S-stage shared-memory ring   (the paper's MTE2)
 //   MMA warp      : one thread issues tcgen05.mma kind::f16, 128|256 x BN x 16,
 //                   fp32 accumulator in TMEM, 2-4 accumulator buffers           (Cube + L0C)
-//   8 epilogue warps: tcgen05.ld -> one RN-even cast -> shared -> coalesced 16 B stores (FixPipe)
+//   8 epilogue warps: tcgen05.ld -> one RN-even cast -> shared -> TMA store of a 64 x 32 box, or
+//                   coalesced 16 B stores where C's rows rule TMA out                 (FixPipe)
 //
 // The CTA is persistent: it walks its list of work units (tile x k-split) so the producer runs
 // ahead across tile boundaries (Preloading, Eq. 14) and the epilogue of unit u overlaps the main
 // loop of unit u+1.  With P_k > 1 a unit covers a fixed k-block range and writes an fp32 partial
 // tile to the workspace (Eq. 4); a separate kernel adds the partials in ascending split order.
+// MODE selects how unaligned operands are reached without a copy (row classes of A, k classes of
+// B, halo class tiles for C): see the comment in front of the kernel.
 #pragma once
 
 #include <cuda.h>
