@@ -46,6 +46,7 @@ struct Calib {
     double skinny_bw_eff_aligned = 0.45;    // fraction of hbm_bw the warp-level streaming kernel reaches, 16-byte aligned rows
     double skinny_bw_eff_unaligned = 0.14;  // ... rows assembled from two chunks
     double skinny_fixed_us = 2.0;
+    double skinny_pass_us = 4.0;        // one 64-row pass over one staged chunk when the streamed rows are k-contiguous
     double skinny_step_unaligned_us = 2.0;   // one 16-k step of a warp when the streamed rows are unaligned
     double skinny_mac_rate = 30e12;     // MAC/s ceiling of the warp-level kernel (small side padded to 16)
     double copy_bw_eff = 0.85;          // pad-copy and reduce kernels

@@ -306,6 +306,12 @@ static void model_skinny(const Shape& s, const Machine& m, const Calib& cal, Con
         const double t_chain = cal.skinny_step_unaligned_us * (double)steps;
         t_cta = k_split <= kSkinnyKChunk ? t_chain : std::max(t_cta, t_chain);
     }
+    if (!k_is_outer) {
+        // k-contiguous stream: the CTA walks its rows in passes of 64, each a chain of dependent trips to
+        // memory per staged chunk (89274 x 16 x 23: two passes per CTA, three waves, 27 us)
+        const int64_t k_split = ceil_div(s.K, c.P_k);
+        t_cta = std::max(t_cta, cal.skinny_pass_us * (double)(c.BN / 64) * (double)ceil_div(k_split, kSkinnyKChunk));
+    }
     model_epilogue(s, c, cal);
     const double t_alu = macs / cal.skinny_mac_rate * 1e6;
     c.t_pro_us = 0;
