@@ -677,7 +677,7 @@ def main():
     ap.add_argument("--ref-macs", type=float, default=5e10, help="with --impl reference: multiply-accumulates of the oracle's bounded sample per step")
     ap.add_argument("--shape", default="", help="M,N,K,dtype: time this one shape only (dtype 0 = fp16, 1 = bf16)")
     ap.add_argument("--reps", type=int, default=3)
-    ap.add_argument("--family", type=int, default=-1, help="with --shape: force a kernel family (0 umma_1cta, 1 umma_2cta, 2 skinny, 3 simt)")
+    ap.add_argument("--family", type=int, default=-1, help="with --shape: force a kernel family (0 umma_1cta, 1 umma_2cta, 2 skinny, 3 simt, 4 cluster)")
     ap.add_argument("--bn", type=int, default=0)
     ap.add_argument("--pk", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)

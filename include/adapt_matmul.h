@@ -63,7 +63,10 @@ typedef enum {
     ADAPT_FAM_UMMA_1CTA = 0,  /* tcgen05 128 x BN tiles, TMEM accumulators, TMA ring; P_k > 1 adds split-K */
     ADAPT_FAM_UMMA_2CTA = 1,  /* cta_group::2, 256 x BN tile on an SM pair */
     ADAPT_FAM_SKINNY = 2,     /* warp-level kernel for M <= 16 or N <= 16, streams the large operand once */
-    ADAPT_FAM_SIMT = 3        /* CUDA-core tile kernel: legal for every shape and alignment */
+    ADAPT_FAM_SIMT = 3,       /* CUDA-core tile kernel: legal for every shape and alignment */
+    ADAPT_FAM_CLUSTER = 4     /* small problems in one launch: 64 x 64 tiles on mma.sync, any alignment, the k range
+                                 split over the CTAs of a cluster (P_k = cluster = 1, 2, 4, 8) and reduced through
+                                 distributed shared memory; no workspace */
 } adapt_family_t;
 
 /* How an operand reaches shared memory (the paper's Padding module, Table 2). */
@@ -71,7 +74,7 @@ typedef enum {
     ADAPT_SRC_TMA = 0,        /* TMA straight from the caller's buffer (needs 16 B pitch and base) */
     ADAPT_SRC_PAD_COPY = 1,   /* prologue kernel re-pitches the operand into the workspace, then TMA (with srcB =
                                  ADAPT_SRC_TMA_CLASSES: A is regrouped class-major instead) */
-    ADAPT_SRC_LSU = 2,        /* ordinary loads (skinny / SIMT families) */
+    ADAPT_SRC_LSU = 2,        /* ordinary loads (skinny / SIMT / cluster families) */
     ADAPT_SRC_TMA_CLASSES = 3 /* class views, no copy of that operand.
                                  srcA: row-major A read in place through one TMA view per row class; tiles are made
                                  of every 8th row (BN = 64, 128, 256; needs K % 8 != 0) or, with 16 halo columns

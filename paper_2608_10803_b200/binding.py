@@ -13,8 +13,8 @@ F16, BF16 = 0, 1
 ROW_MAJOR, COL_MAJOR = 0, 1
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_NOMEM, ERR_CUDA, ERR_TIMEOUT, ERR_NOT_INIT = range(7)
 CLASS_NAMES = ["Common", "SingleCoreSplitK", "MultiCoreSplitK", "HybridSplitK"]
-FAMILY_NAMES = ["umma_1cta", "umma_2cta", "skinny", "simt"]
-FAM_UMMA_1CTA, FAM_UMMA_2CTA, FAM_SKINNY, FAM_SIMT = range(4)
+FAMILY_NAMES = ["umma_1cta", "umma_2cta", "skinny", "simt", "cluster"]
+FAM_UMMA_1CTA, FAM_UMMA_2CTA, FAM_SKINNY, FAM_SIMT, FAM_CLUSTER = range(5)
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libadaptmm.so")

@@ -18,6 +18,7 @@
 #include "adapt_internal.h"
 #include "aux_kernels.cuh"
 #include "skinny_gemm.cuh"
+#include "cluster_gemm.cuh"
 #include "umma_gemm.cuh"
 
 using namespace adapt;
@@ -295,7 +296,7 @@ extern "C" adapt_handle_t adapt_matmul_plan_forced(int64_t M, int64_t N, int64_t
     if (it != S.big.end()) return it->second;
     // a forced plan may use any compiled family, whatever the selection mask says
     Machine saved = S.machine;
-    S.machine.family_mask = 0xFu;
+    S.machine.family_mask = 0x1Fu;
     Plan* p = make_plan(S, s, &tiling_key);
     S.machine = saved;
     if (!p) return nullptr;
@@ -330,7 +331,7 @@ extern "C" int adapt_plan_candidates(int64_t M, int64_t N, int64_t K, adapt_dtyp
         if (!S.inited && S.all_plans.empty()) apply_env(S);
         m = S.machine;
     }
-    m.family_mask = 0xFu;     // list every compiled family, selected or not
+    m.family_mask = 0x1Fu;    // list every compiled family, selected or not
     std::vector<Config> cands;
     enumerate_configs(s, m, S.calib, &cands);
     for (int i = 0; i < (int)cands.size() && i < cap && out; ++i) fill_info(s, cands[i], &out[i]);
@@ -452,6 +453,7 @@ extern "C" adapt_status_t adapt_init(int device)
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
     CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_2CTA, 256, false, true, 2),
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
+    CUDA_TRY(cluster_set_attributes());
     S.device = device;
     S.inited = true;
     return ADAPT_OK;
@@ -839,6 +841,14 @@ adapt_status_t run_simt(State& S, Plan* pl, const void* A, const void* B, void* 
     return ADAPT_OK;
 }
 
+adapt_status_t run_cluster(State& S, Plan* pl, const void* A, const void* B, void* C, cudaStream_t stream)
+{
+    if (launch_cluster(pl->s, pl->c, A, B, C, S.d_status, stream) != ADAPT_OK) return fail(ADAPT_ERR_CUDA, "cluster kernel launch failed%s");
+    S.launches.fetch_add(1, std::memory_order_relaxed);
+    CUDA_TRY(cudaGetLastError());
+    return ADAPT_OK;
+}
+
 adapt_status_t run_skinny(State& S, Plan* pl, const void* A, const void* B, void* C, cudaStream_t stream)
 {
     const Shape& s = pl->s;
@@ -886,6 +896,7 @@ extern "C" adapt_status_t adapt_matmul(adapt_handle_t plan, const void* A, const
         case ADAPT_FAM_UMMA_2CTA: return run_umma(S, pl, A, B, C, stream);
         case ADAPT_FAM_SKINNY: return run_skinny(S, pl, A, B, C, stream);
         case ADAPT_FAM_SIMT: return run_simt(S, pl, A, B, C, stream);
+        case ADAPT_FAM_CLUSTER: return run_cluster(S, pl, A, B, C, stream);
     }
     return fail(ADAPT_ERR_UNSUPPORTED, "unknown kernel family%s");
 }

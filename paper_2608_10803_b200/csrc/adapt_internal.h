@@ -16,7 +16,7 @@ struct Machine {
     int smem_bytes = 227 * 1024;        // per-CTA shared memory limit (the paper's L1 capacity)
     int tmem_cols = 512;                // 128 lanes x 512 fp32 columns per SM (the paper's L0C)
     int64_t workspace_limit = (int64_t)24 << 30;
-    unsigned family_mask = 0xFu;        // bit f set = family f may be selected
+    unsigned family_mask = 0x1Fu;        // bit f set = family f may be selected
 };
 
 // ---- calibration constants of the latency model (Eq. 8: lambda_r, eta_r, BW_r) ------------
@@ -49,6 +49,12 @@ struct Calib {
     double skinny_pass_us = 4.0;        // one 64-row pass over one staged chunk when the streamed rows are k-contiguous
     double skinny_step_unaligned_us = 2.0;   // one 16-k step of a warp when the streamed rows are unaligned
     double skinny_mac_rate = 30e12;     // MAC/s ceiling of the warp-level kernel (small side padded to 16)
+    // one-launch cluster kernel (64 x 64 tiles, k split over a cluster)
+    double cluster_fixed_us = 1.5;      // first trip to memory, last stage, rounding and store of the tile
+    double cluster_stage_us = 0.6;      // one 64-k stage of a CTA that has its SM to itself (a trip to L2 / HBM)
+    double cluster_stage_unaligned_us = 0.8;   // ... when the groups are assembled from two chunks
+    double cluster_reduce_us = 0.8;     // cluster barrier + reading the partial tiles of the peers
+    double cluster_bw_eff = 0.35;       // fraction of hbm_bw its register-staged loads reach when memory-bound
     double copy_bw_eff = 0.85;          // pad-copy and reduce kernels
     double hbm_bw_per_sm = 55e9;        // B/s one SM streams from HBM (tail wave of 20000 x 8 x 60001: 15 MB per tile in 0.3 ms)
     double class_view_sm_eff = 0.85;    // per-SM rate through those views relative to l2_bw_per_sm (20000 x 8 x 60001 tail wave)
@@ -120,6 +126,19 @@ const Calib& default_calib();
 // Shared-memory layout of the tcgen05 kernels, used by the capacity check and by the launcher:
 // S stages of (A: box rows x 64, B: BN/cluster x 64) 16-bit, a barrier block, the epilogue staging
 // (8 KB per epilogue warp, only when the kernel stores the 16-bit C), and slack to align the stages to 1024 B.
+// One-launch cluster kernel: a ring of raw stages (64 rows of 144 bytes per operand) plus two shifted stages.
+// The ring is as deep as the CTA's k range needs, capped so that the CTAs that share an SM all fit.
+constexpr int kClusterStageBytes = 2 * 64 * 144;
+constexpr int kClusterMaxRing = 6;
+inline int cluster_smem_bytes(int ring) { return (ring + 2) * kClusterStageBytes + 128; }   // + two shifted stages, barriers
+inline int cluster_ring(int64_t K, int cluster, int64_t tiles, int n_sm)
+{
+    const int64_t k_cta = (K + cluster - 1) / cluster;
+    const int64_t stages = ((k_cta + 15) / 16 * 16 + 63) / 64;
+    const int64_t per_sm = (tiles * cluster + n_sm - 1) / n_sm;
+    const int cap = per_sm <= 1 ? kClusterMaxRing : (per_sm == 2 ? 4 : 2);
+    return (int)std::max<int64_t>(1, std::min<int64_t>(stages, cap));
+}
 constexpr int kSkinnyKChunk = 512;   // k values the warp-level kernel stages per chunk; its k splits are whole chunks
 constexpr int kUmmaBarrierBytes = 1024;  // keeps the epilogue staging 1024-byte aligned (swizzled TMA boxes)
 constexpr int kUmmaMaxStages = 15;

@@ -338,6 +338,34 @@ static void model_simt(const Shape& s, const Machine& m, const Calib& cal, Confi
     finish_common(s, c, cal);
 }
 
+static bool aligned16(int64_t inner_elems);
+
+static void model_cluster(const Shape& s, const Machine& m, const Calib& cal, Config& c)
+{
+    const double MK = (double)s.M * s.K, KN = (double)s.K * s.N, MN = (double)s.M * s.N;
+    const int64_t tiles = (int64_t)c.P_m * c.P_n, units = tiles * c.cluster;
+    c.grid = (int)units;
+    // every tile row re-reads B and every tile column re-reads A, mostly from L2; HBM sees each once
+    c.hbm_bytes = 2.0 * (MK + KN + MN);
+    const int64_t per_sm = 4;                                   // CTAs resident per SM
+    const int64_t Q = ceil_div(units, (int64_t)m.n_sm * per_sm);
+    const int64_t k_cta = round_up(ceil_div(s.K, c.cluster), 16);
+    const int64_t stages = ceil_div(k_cta, 64);
+    const bool aligned = aligned16(innerA(s)) && aligned16(innerB(s));
+    // a CTA alone on its SM pays one trip to memory per stage; CTAs that share an SM overlap their trips
+    // until the SM's load path is the limit (16 KB per CTA and stage)
+    const double share = (double)std::min<int64_t>(per_sm, ceil_div(units, m.n_sm));
+    const double t_stage = std::max(aligned ? cal.cluster_stage_us : cal.cluster_stage_unaligned_us,
+                                    share * 16384.0 / cal.l2_bw_per_sm * 1e6 * (aligned ? 1.0 : 2.0));
+    const double t_cta = cal.cluster_fixed_us + (double)stages * t_stage + (c.cluster > 1 ? cal.cluster_reduce_us : 0.0);
+    const double l2_bytes = 2.0 * 64.0 * 64.0 * 2.0 * (double)stages * (double)units;   // what the CTAs pull in all
+    const double t_mem = std::max(c.hbm_bytes / (cal.hbm_bw * cal.cluster_bw_eff), l2_bytes / (cal.l2_bw_per_sm * m.n_sm)) * 1e6;
+    c.t_pro_us = 0;
+    c.t_epi_us = 0;
+    c.t_main_us = std::max((double)Q * t_cta, t_mem);
+    finish_common(s, c, cal);
+}
+
 // ---- legality (the constraint M(b,x,s) <= C_limit of Eq. 6) -----------------------------------
 
 static bool aligned16(int64_t inner_elems) { return inner_elems % 8 == 0; }
@@ -437,6 +465,23 @@ static bool legal_simt(const Shape& s, const Machine& m, Config& c)
     return true;
 }
 
+static bool legal_cluster(const Shape& s, const Machine& m, Config& c)
+{
+    if (!(m.family_mask & (1u << ADAPT_FAM_CLUSTER))) return false;
+    if (c.BM != 64 || c.BN != 64 || c.BK != 64) return false;
+    if (c.cluster != 1 && c.cluster != 2 && c.cluster != 4 && c.cluster != 8) return false;
+    if (c.P_k != c.cluster) return false;                            // the k splits are the cluster's CTAs
+    if (c.srcA != ADAPT_SRC_LSU || c.srcB != ADAPT_SRC_LSU) return false;
+    if ((c.cluster - 1) * round_up(ceil_div(s.K, c.cluster), 16) >= s.K) return false;   // no CTA without k values
+    c.P_m = (int)ceil_div(s.M, c.BM);
+    c.P_n = (int)ceil_div(s.N, c.BN);
+    if ((int64_t)c.P_m * c.P_n * c.cluster > (int64_t)1 << 24) return false;
+    if (c.stages != cluster_ring(s.K, c.cluster, (int64_t)c.P_m * c.P_n, m.n_sm)) return false;
+    c.persistent = 0;
+    c.smem_bytes = cluster_smem_bytes(c.stages);
+    return true;
+}
+
 static bool finalize(const Shape& s, const Machine& m, const Calib& cal, Config& c)
 {
     bool ok = false;
@@ -445,6 +490,7 @@ static bool finalize(const Shape& s, const Machine& m, const Calib& cal, Config&
         case ADAPT_FAM_UMMA_2CTA: ok = legal_umma(s, m, c); break;
         case ADAPT_FAM_SKINNY: ok = legal_skinny(s, m, c); break;
         case ADAPT_FAM_SIMT: ok = legal_simt(s, m, c); break;
+        case ADAPT_FAM_CLUSTER: ok = legal_cluster(s, m, c); break;
         default: ok = false;
     }
     if (!ok) return false;
@@ -459,6 +505,7 @@ static bool finalize(const Shape& s, const Machine& m, const Calib& cal, Config&
         case ADAPT_FAM_UMMA_1CTA:
         case ADAPT_FAM_UMMA_2CTA: model_umma(s, m, cal, c); break;
         case ADAPT_FAM_SKINNY: model_skinny(s, m, cal, c); break;
+        case ADAPT_FAM_CLUSTER: model_cluster(s, m, cal, c); break;
         default: model_simt(s, m, cal, c); break;
     }
     if (c.workspace_bytes > m.workspace_limit) return false;
@@ -599,6 +646,14 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
             c.srcA = c.srcB = ADAPT_SRC_LSU;
             if (finalize(s, m, cal, c)) out->push_back(c);
         }
+    }
+    // --- one-launch cluster family: always legal; meant for problems of a few microseconds ---
+    for (int cs : {1, 2, 4, 8}) {
+        Config c;
+        c.family = ADAPT_FAM_CLUSTER; c.BM = 64; c.BN = 64; c.BK = 64; c.P_k = cs; c.cluster = cs;
+        c.stages = cluster_ring(s.K, cs, ceil_div(s.M, 64) * ceil_div(s.N, 64), m.n_sm);
+        c.srcA = c.srcB = ADAPT_SRC_LSU;
+        if (finalize(s, m, cal, c)) out->push_back(c);
     }
     // argmin of Eq. 6 with a deterministic tie-break: time, then fewer splits, then smaller
     // workspace, then enumeration order (stable sort keeps it)

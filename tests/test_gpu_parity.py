@@ -396,6 +396,59 @@ def test_tma_store_epilogue_leaves_neighbouring_memory_alone():
         assert torch.isnan(c_buf[:2048]).all() and torch.isnan(c_buf[2048 + M * N:]).all()
 
 
+# ---- the one-launch cluster kernel: every cluster size, layout and alignment ---------------------------------
+
+def cluster_variants(M, N, K, dtype, lA=ROW, lB=ROW):
+    cands = [c for c in ab.adapt_plan_candidates(M, N, K, dtype, lA, lB) if c.family == ab.FAM_CLUSTER]
+    return [(ab.adapt_matmul_plan_forced(M, N, K, dtype, lA, lB, c.tiling_key), c) for c in cands]
+
+
+@pytest.mark.parametrize("lA,lB", [(ROW, ROW), (ROW, COL), (COL, ROW), (COL, COL)])
+@pytest.mark.parametrize("shape", [(64, 64, 64), (70, 130, 100), (200, 333, 1482), (129, 65, 17), (33, 7, 4099),
+                                   (1, 1, 1), (300, 264, 520), (3, 200, 129), (65, 63, 8)])
+def test_cluster_family_bit_exact(shape, lA, lB):
+    M, N, K = shape
+    for dtype in (ab.F16, ab.BF16):
+        A = synth.position_coded(M, K, dtype, 7, "cuda")
+        B = synth.position_coded(K, N, dtype, 5, "cuda")
+        A_st = A.t().contiguous() if lA == COL else A
+        B_st = B.t().contiguous() if lB == COL else B
+        variants = cluster_variants(M, N, K, dtype, lA, lB)
+        assert any(c.cluster == 1 and c.P_k == 1 for _, c in variants)
+        # every cluster size that leaves no CTA without k values (pieces are multiples of 16)
+        want = {cs for cs in (1, 2, 4, 8) if (cs - 1) * (-(-(-(-K // cs)) // 16) * 16) < K}
+        assert {c.cluster for _, c in variants} == want
+        for plan, c in variants:
+            assert c.P_k == c.cluster and c.workspace_bytes == 0
+            check_case(M, N, K, dtype, A_st, B_st, lA, lB, plan=plan, exact=True)
+
+
+def test_cluster_family_random_values_and_unaligned_pointers():
+    """Operands and C two bytes off a 16-byte boundary (rows of aligned pitch, misaligned base): the groups
+    are then assembled from two chunks; nothing outside C is written."""
+    M, N, K = 150, 200, 328
+    dtype = ab.BF16
+    tdt = synth.torch_dtype(dtype)
+    A = synth.draw_operand(M, K, synth.U11, 31, dtype, "cuda")
+    B = synth.draw_operand(K, N, synth.U11, 32, dtype, "cuda")
+    a_buf = torch.zeros(M * K + 16, dtype=tdt, device="cuda")
+    b_buf = torch.zeros(K * N + 16, dtype=tdt, device="cuda")
+    A_off = a_buf[1:1 + M * K].view(M, K)
+    B_off = b_buf[3:3 + K * N].view(K, N)
+    A_off.copy_(A)
+    B_off.copy_(B)
+    assert A_off.data_ptr() % 16 == 2 and B_off.data_ptr() % 16 == 6
+    for plan, c in cluster_variants(M, N, K, dtype):
+        for a_t, b_t, c_off in ((A, B, 0), (A_off, B, 1), (A, B_off, 0), (A_off, B_off, 3)):
+            c_buf = torch.full((M * N + 16,), float("nan"), dtype=tdt, device="cuda")
+            out = c_buf[c_off:c_off + M * N].view(M, N)
+            run_library(a_t, b_t, M, N, K, dtype, plan=plan, out=out)
+            torch.cuda.synchronize()
+            err, mism, _ = compare_with_oracle(A, B, out.contiguous(), M, N, K, dtype)
+            assert err <= 8e-3
+            assert torch.isnan(c_buf[:c_off]).all() and torch.isnan(c_buf[c_off + M * N:]).all()
+
+
 # ---- host operands: the pipelined copy-in | kernels | copy-out entry point ------------------------------
 
 def test_host_entry_point_matches_the_oracle_over_a_run_of_calls():
