@@ -41,7 +41,9 @@ struct Calib {
     double epi_partial_fixed_us = 0.32, epi_partial_us_per_kb = 0.0385;   // fp32 partials, stored by the epilogue threads
     double epi_tile_fixed_unaligned_us = 1.45, epi_us_per_kb_unaligned = 0.054;
     double simt_flops = 15e12;          // CUDA-core tile kernel (1000^3: 17e12)
-    double simt_fixed_us = 1.5;
+    double simt_fixed_us = 0.45;
+    double simt_step_us = 0.8;          // one 16-k step of a CTA alone on its SM (15 x 30 x 32: two steps, 4.85 us with the launch)
+    double halo_edge_tile_us = 3.4;     // row heads or tails of one halo tile, written element-wise
     double simt_bw_eff = 0.15;          // fraction of hbm_bw its 2-byte accesses reach (K = 1 outer products: 0.13 measured)
     double skinny_bw_eff_aligned = 0.45;    // fraction of hbm_bw the warp-level streaming kernel reaches, 16-byte aligned rows
     double skinny_bw_eff_unaligned = 0.14;  // ... rows assembled from two chunks
@@ -49,12 +51,14 @@ struct Calib {
     double skinny_pass_us = 4.0;        // one 64-row pass over one staged chunk when the streamed rows are k-contiguous
     double skinny_step_unaligned_us = 2.0;   // one 16-k step of a warp when the streamed rows are unaligned
     double skinny_mac_rate = 30e12;     // MAC/s ceiling of the warp-level kernel (small side padded to 16)
-    // one-launch cluster kernel (64 x 64 tiles, k split over a cluster)
-    double cluster_fixed_us = 1.5;      // first trip to memory, last stage, rounding and store of the tile
-    double cluster_stage_us = 0.6;      // one 64-k stage of a CTA that has its SM to itself (a trip to L2 / HBM)
-    double cluster_stage_unaligned_us = 0.8;   // ... when the groups are assembled from two chunks
-    double cluster_reduce_us = 0.8;     // cluster barrier + reading the partial tiles of the peers
-    double cluster_bw_eff = 0.35;       // fraction of hbm_bw its register-staged loads reach when memory-bound
+    // one-launch cluster kernel (64 x 64 tiles, k split over a cluster); least-squares fit over 180 timed
+    // configurations of 2,000-sweep shapes: 3.7 + 0.95 stages + 0.8 (cluster > 1) + crowd (1.6 + 0.44 stages) us
+    double cluster_fixed_us = 0.75;     // beyond the launch: barrier set-up, first trip to memory, rounding and store of the tile
+    double cluster_stage_us = 0.95;     // one 64-k stage: copy issue, shift pass, MMAs, each behind a CTA-wide barrier
+    double cluster_reduce_us = 0.8;     // cluster barriers + reading the partial tiles of the peers
+    double cluster_crowd_us = 1.56, cluster_crowd_stage_us = 0.44;   // per CTA per SM beyond one per two SMs
+    double cluster_wave_us = 5.5;       // each further round of clusters
+    double cluster_bw_eff = 0.35;       // fraction of hbm_bw its 16-byte copies reach when memory-bound
     double copy_bw_eff = 0.85;          // pad-copy and reduce kernels
     double hbm_bw_per_sm = 55e9;        // B/s one SM streams from HBM (tail wave of 20000 x 8 x 60001: 15 MB per tile in 0.3 ms)
     double class_view_sm_eff = 0.85;    // per-SM rate through those views relative to l2_bw_per_sm (20000 x 8 x 60001 tail wave)

@@ -250,6 +250,10 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
         pipe = tM + (double)Q * t_tile + tP + t_drain;
     }
     pipe += cal.umma_fixed_us;
+    // halo tiles: the first and the last tile of a row block write the elements before the first and after
+    // the last whole 32-byte unit of each row with 2-byte stores (48618 x 28 x 115: 384 such tiles, 17 us)
+    if (halo && c.P_k == 1)
+        pipe += 2.0 * cal.halo_edge_tile_us * (double)c.P_m / (double)std::min<int64_t>(m.n_sm, (int64_t)c.P_m * c.P_n);
     model_prologue(s, c, cal);
     model_epilogue(s, c, cal);
     // strided row-class views stream A at a lower rate than a dense tensor (measured 3.5-4.1 TB/s)
@@ -327,9 +331,13 @@ static void model_simt(const Shape& s, const Machine& m, const Calib& cal, Confi
     c.hbm_bytes = 2.0 * (MK + KN) + (c.P_k > 1 ? 0.0 : 2.0 * MN);
     const int64_t resident = (int64_t)m.n_sm * 4;
     const int64_t Q = ceil_div(units, resident);
-    // a full 64x64 tile costs the same whether or not the shape fills it
-    const double tile_flops = 2.0 * c.BM * c.BN * (double)ceil_div(s.K, c.P_k);
-    const double t_tile = tile_flops / (cal.simt_flops / resident) * 1e6 + cal.simt_fixed_us;
+    // A full 64 x 64 tile costs the same whether or not the shape fills it.  One step of 16 k values is a
+    // trip to memory for a CTA that has its SM to itself; CTAs that share an SM (up to 4) share its FMA rate
+    // (4 per SM: 2 * 64 * 64 * 16 flops per step at simt_flops / (4 n_sm) per CTA)
+    const double steps = (double)ceil_div(ceil_div(s.K, c.P_k), 16);
+    const double crowd = std::min(4.0, (double)units / m.n_sm);
+    const double t_step = std::max(cal.simt_step_us, crowd * 2.0 * 64 * 64 * 16 / (cal.simt_flops / m.n_sm) * 1e6);
+    const double t_tile = steps * t_step + cal.simt_fixed_us;
     model_epilogue(s, c, cal);
     // element-wise 2-byte loads and stores: about a seventh of the HBM rate when memory-bound
     const double t_hbm = c.hbm_bytes / (cal.hbm_bw * cal.simt_bw_eff) * 1e6 - c.t_epi_us;
@@ -347,22 +355,21 @@ static void model_cluster(const Shape& s, const Machine& m, const Calib& cal, Co
     c.grid = (int)units;
     // every tile row re-reads B and every tile column re-reads A, mostly from L2; HBM sees each once
     c.hbm_bytes = 2.0 * (MK + KN + MN);
-    const int64_t per_sm = 4;                                   // CTAs resident per SM
-    const int64_t Q = ceil_div(units, (int64_t)m.n_sm * per_sm);
     const int64_t k_cta = round_up(ceil_div(s.K, c.cluster), 16);
-    const int64_t stages = ceil_div(k_cta, 64);
-    const bool aligned = aligned16(innerA(s)) && aligned16(innerB(s));
-    // a CTA alone on its SM pays one trip to memory per stage; CTAs that share an SM overlap their trips
-    // until the SM's load path is the limit (16 KB per CTA and stage)
-    const double share = (double)std::min<int64_t>(per_sm, ceil_div(units, m.n_sm));
-    const double t_stage = std::max(aligned ? cal.cluster_stage_us : cal.cluster_stage_unaligned_us,
-                                    share * 16384.0 / cal.l2_bw_per_sm * 1e6 * (aligned ? 1.0 : 2.0));
-    const double t_cta = cal.cluster_fixed_us + (double)stages * t_stage + (c.cluster > 1 ? cal.cluster_reduce_us : 0.0);
-    const double l2_bytes = 2.0 * 64.0 * 64.0 * 2.0 * (double)stages * (double)units;   // what the CTAs pull in all
-    const double t_mem = std::max(c.hbm_bytes / (cal.hbm_bw * cal.cluster_bw_eff), l2_bytes / (cal.l2_bw_per_sm * m.n_sm)) * 1e6;
+    const double stages = (double)ceil_div(k_cta, 64);
+    // a cluster is placed inside one GPC (about 18 SMs): clusters of 4 and 8 leave SMs of a GPC unused, so
+    // fewer tiles run at a time; two CTAs share an SM when their rings fit
+    const int64_t per_sm = std::min<int64_t>(2, m.smem_bytes / cluster_smem_bytes(c.stages));
+    const int64_t at_a_time = (c.cluster == 1 ? (int64_t)m.n_sm : (int64_t)8 * (18 / c.cluster)) * std::max<int64_t>(1, per_sm);
+    const double waves = (double)ceil_div(tiles, at_a_time);
+    // CTAs beyond one per two SMs start to share the load path
+    const double crowd = std::max(0.0, (double)units / m.n_sm - 0.5);
+    const double t_cta = cal.cluster_fixed_us + cal.cluster_stage_us * stages + (c.cluster > 1 ? cal.cluster_reduce_us : 0.0) +
+                         crowd * (cal.cluster_crowd_us + cal.cluster_crowd_stage_us * stages) + cal.cluster_wave_us * (waves - 1.0);
+    const double t_mem = c.hbm_bytes / (cal.hbm_bw * cal.cluster_bw_eff) * 1e6;
     c.t_pro_us = 0;
     c.t_epi_us = 0;
-    c.t_main_us = std::max((double)Q * t_cta, t_mem);
+    c.t_main_us = std::max(t_cta, t_mem);
     finish_common(s, c, cal);
 }
 
@@ -475,7 +482,8 @@ static bool legal_cluster(const Shape& s, const Machine& m, Config& c)
     if ((c.cluster - 1) * round_up(ceil_div(s.K, c.cluster), 16) >= s.K) return false;   // no CTA without k values
     c.P_m = (int)ceil_div(s.M, c.BM);
     c.P_n = (int)ceil_div(s.N, c.BN);
-    if ((int64_t)c.P_m * c.P_n * c.cluster > (int64_t)1 << 24) return false;
+    // a kernel for problems of a few microseconds: at most two CTAs per SM in all
+    if ((int64_t)c.P_m * c.P_n * c.cluster > 2 * (int64_t)m.n_sm) return false;
     if (c.stages != cluster_ring(s.K, c.cluster, (int64_t)c.P_m * c.P_n, m.n_sm)) return false;
     c.persistent = 0;
     c.smem_bytes = cluster_smem_bytes(c.stages);
@@ -647,7 +655,7 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
             if (finalize(s, m, cal, c)) out->push_back(c);
         }
     }
-    // --- one-launch cluster family: always legal; meant for problems of a few microseconds ---
+    // --- one-launch cluster family: any shape, layout and alignment whose tiles fit the machine about once ---
     for (int cs : {1, 2, 4, 8}) {
         Config c;
         c.family = ADAPT_FAM_CLUSTER; c.BM = 64; c.BN = 64; c.BK = 64; c.P_k = cs; c.cluster = cs;
