@@ -65,7 +65,7 @@ typedef enum {
     ADAPT_FAM_SKINNY = 2,     /* warp-level kernel for M <= 16 or N <= 16, streams the large operand once */
     ADAPT_FAM_SIMT = 3,       /* CUDA-core tile kernel: legal for every shape and alignment */
     ADAPT_FAM_CLUSTER = 4     /* small problems in one launch: 64 x 64 tiles on mma.sync, any alignment, the k range
-                                 split over the CTAs of a cluster (P_k = cluster = 1, 2, 4, 8) and reduced through
+                                 split over the CTAs of a cluster (P_k = cluster = 1, 2, 4, 8, 16) and reduced through
                                  distributed shared memory; no workspace */
 } adapt_family_t;
 
@@ -112,8 +112,8 @@ typedef struct adapt_plan_info_s {
 /* TilingKey bit layout (Section 3.2 asks only for "a compact 64-bit key"; the fields are this
  * library's): [63:62] taxonomy class, [61:59] family, [58:54] BM/16, [53:48] BN/16,
  * [47:46] log2(BK/16), [45:42] stages, [41:32] P_k, [31] persistent tile loop,
- * [30:29] srcA, [28:27] srcB, [26] dtype, [25] layoutA, [24] layoutB, [23:22] log2(cluster),
- * [21:0] zero. */
+ * [30:29] srcA, [28:27] srcB, [26] dtype, [25] layoutA, [24] layoutB, [23:22] log2(cluster) mod 4,
+ * [21] log2(cluster) / 4, [20:0] zero. */
 
 /* Select the device (cudaSetDevice), query it, and create the library state for
  * it.  Idempotent.  Needed before adapt_matmul; planning works without it (the

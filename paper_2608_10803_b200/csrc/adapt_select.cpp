@@ -76,12 +76,13 @@ uint64_t pack_tiling_key(const Shape& s, const Config& c)
     k |= (uint64_t)(s.layoutA & 1) << 25;
     k |= (uint64_t)(s.layoutB & 1) << 24;
     k |= (uint64_t)(ilog2(std::max(c.cluster, 1)) & 3) << 22;
+    k |= (uint64_t)((ilog2(std::max(c.cluster, 1)) >> 2) & 1) << 21;
     return k;
 }
 
 bool unpack_tiling_key(uint64_t k, Shape* s, Config* c)
 {
-    if (k & ((1ull << 22) - 1)) return false;
+    if (k & ((1ull << 21) - 1)) return false;
     c->cls = (int)((k >> 62) & 3);
     c->family = (int)((k >> 59) & 7);
     c->BM = (int)((k >> 54) & 31) * 16;
@@ -95,7 +96,7 @@ bool unpack_tiling_key(uint64_t k, Shape* s, Config* c)
     s->dtype = (int)((k >> 26) & 1);
     s->layoutA = (int)((k >> 25) & 1);
     s->layoutB = (int)((k >> 24) & 1);
-    c->cluster = 1 << (int)((k >> 22) & 3);
+    c->cluster = 1 << (int)(((k >> 22) & 3) | (((k >> 21) & 1) << 2));
     return true;
 }
 
@@ -476,7 +477,7 @@ static bool legal_cluster(const Shape& s, const Machine& m, Config& c)
 {
     if (!(m.family_mask & (1u << ADAPT_FAM_CLUSTER))) return false;
     if (c.BM != 64 || c.BN != 64 || c.BK != 64) return false;
-    if (c.cluster != 1 && c.cluster != 2 && c.cluster != 4 && c.cluster != 8) return false;
+    if (c.cluster != 1 && c.cluster != 2 && c.cluster != 4 && c.cluster != 8 && c.cluster != 16) return false;
     if (c.P_k != c.cluster) return false;                            // the k splits are the cluster's CTAs
     if (c.srcA != ADAPT_SRC_LSU || c.srcB != ADAPT_SRC_LSU) return false;
     if ((c.cluster - 1) * round_up(ceil_div(s.K, c.cluster), 16) >= s.K) return false;   // no CTA without k values
@@ -656,7 +657,7 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
         }
     }
     // --- one-launch cluster family: any shape, layout and alignment whose tiles fit the machine about once ---
-    for (int cs : {1, 2, 4, 8}) {
+    for (int cs : {1, 2, 4, 8, 16}) {
         Config c;
         c.family = ADAPT_FAM_CLUSTER; c.BM = 64; c.BN = 64; c.BK = 64; c.P_k = cs; c.cluster = cs;
         c.stages = cluster_ring(s.K, cs, ceil_div(s.M, 64) * ceil_div(s.N, 64), m.n_sm);

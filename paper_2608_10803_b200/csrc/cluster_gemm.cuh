@@ -2,7 +2,7 @@
 //
 // The tensor-core kernel needs 16-byte aligned rows for its TMA loads and a second launch to add
 // split-K partials; on a problem of a few microseconds those extra launches are most of the time.
-// Here a 64 x 64 output tile belongs to a thread-block cluster of CS CTAs (CS = 1, 2, 4 or 8):
+// Here a 64 x 64 output tile belongs to a thread-block cluster of CS CTAs (CS = 1, 2, 4, 8 or 16):
 // CTA r of the cluster multiplies the r-th piece of the k range, the CS partial tiles are left in
 // each CTA's shared memory, and every CTA then adds its 64 / CS rows of the tile over all ranks
 // through distributed shared memory, in ascending rank order (the order of a split-K reduction,
@@ -346,6 +346,8 @@ inline cudaError_t cluster_set_attributes()
     for (int v = 0; v < 8; ++v) {
         cudaError_t e = cudaFuncSetAttribute(cluster_pick(v & 1, v & 2, v & 4), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              cluster_smem_bytes(kClusterMaxRing));
+        if (e != cudaSuccess) return e;
+        e = cudaFuncSetAttribute(cluster_pick(v & 1, v & 2, v & 4), cudaFuncAttributeNonPortableClusterSizeAllowed, 1);   // clusters of 16
         if (e != cudaSuccess) return e;
     }
     return cudaSuccess;
