@@ -156,6 +156,16 @@ def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
                             assert c.P_k % 8 == 0
                 if c.family == ab.FAM_SKINNY:
                     assert min(M, N) <= 16
+                if c.family == ab.FAM_CLUSTER:
+                    # one launch, no workspace: the k splits are the CTAs of the cluster, none without k values,
+                    # the whole grid at most two CTAs per SM, the ring inside the shared-memory limit
+                    assert c.cluster in (1, 2, 4, 8, 16) and c.P_k == c.cluster and c.workspace_bytes == 0
+                    assert (c.BM, c.BN, c.srcA, c.srcB) == (64, 64, 2, 2)
+                    k_cta = -(-(-(-K // c.cluster)) // 16) * 16
+                    assert (c.cluster - 1) * k_cta < K
+                    assert c.P_m * c.P_n * c.cluster <= 2 * 148 and c.grid == c.P_m * c.P_n * c.cluster
+                    assert 1 <= c.stages <= 6 and c.stages <= -(-k_cta // 64)
+                    assert (c.stages + 2) * 2 * 64 * 144 + 128 <= 227 * 1024
                 # taxonomy label follows the predicate (Section 4.2)
                 enough = c.P_m * c.P_n >= 148
                 assert (c.taxonomy_class in (0, 1)) == enough
@@ -175,6 +185,18 @@ def test_forced_plan_round_trips_its_key():
     with pytest.raises(ab.AdaptError) as e:
         ab.adapt_matmul_plan_forced(M, N, K, ab.BF16, ab.ROW_MAJOR, ab.ROW_MAJOR, 0x1234)
     assert e.value.status == ab.ERR_UNSUPPORTED
+
+
+def test_cluster_family_is_offered_for_small_grids_only_and_its_key_round_trips():
+    small = [c for c in ab.adapt_plan_candidates(50, 311, 3000, ab.F16) if c.family == ab.FAM_CLUSTER]
+    assert {c.cluster for c in small} == {1, 2, 4, 8, 16}           # 5 tiles x 16 CTAs still fit
+    for c in small:
+        info = ab.adapt_plan_info(ab.adapt_matmul_plan_forced(50, 311, 3000, ab.F16, ab.ROW_MAJOR, ab.ROW_MAJOR, c.tiling_key))
+        assert (info.family, info.cluster, info.P_k, info.stages) == (ab.FAM_CLUSTER, c.cluster, c.cluster, c.stages)
+    assert not [c for c in ab.adapt_plan_candidates(4096, 4096, 64, ab.F16) if c.family == ab.FAM_CLUSTER]
+    # a problem of a few tiles and a few hundred k values, unaligned everywhere: the one-launch kernel is the pick
+    pick = ab.adapt_plan_info(ab.adapt_matmul_plan(50, 311, 453, ab.F16))
+    assert pick.family == ab.FAM_CLUSTER and pick.workspace_bytes == 0
 
 
 def test_split_k_is_chosen_for_small_mn_large_k_and_not_for_large_mn():
