@@ -635,6 +635,26 @@ adapt_status_t launch_pad(State& S, const void* src, void* dst, int64_t outer, i
     return ADAPT_OK;
 }
 
+// A and B of one call re-pitched by one launch (blocks in proportion to the chunks of each).
+adapt_status_t launch_pad2(State& S, const void* srcA, void* dstA, int64_t outerA, int64_t innerA, int64_t pitchA,
+                           const void* srcB, void* dstB, int64_t outerB, int64_t innerB, int64_t pitchB, cudaStream_t stream)
+{
+    const int64_t cap = (int64_t)S.machine.n_sm * 16;
+    const int64_t chunksA = outerA * (pitchA / 8), chunksB = outerB * (pitchB / 8);
+    const int64_t blocks = std::min<int64_t>(ceil_div(chunksA, 256) + ceil_div(chunksB, 256), cap);
+    int64_t blocksA = std::max<int64_t>(1, std::min<int64_t>(blocks - 1, (blocks * chunksA + (chunksA + chunksB) / 2) / (chunksA + chunksB)));
+    blocksA = std::min<int64_t>(blocksA, ceil_div(chunksA, 256));
+    PadPair q;
+    q.src[0] = (const unsigned short*)srcA; q.dst[0] = (unsigned short*)dstA; q.outer[0] = outerA; q.inner[0] = innerA; q.pitch[0] = pitchA;
+    q.src[1] = (const unsigned short*)srcB; q.dst[1] = (unsigned short*)dstB; q.outer[1] = outerB; q.inner[1] = innerB; q.pitch[1] = pitchB;
+    q.blocks_a = (int)blocksA;
+    const int64_t blocksB = std::max<int64_t>(1, std::min<int64_t>(blocks - blocksA, ceil_div(chunksB, 256)));
+    CUDA_TRY(launch_pdl(pad_copy2_kernel, dim3((unsigned)(blocksA + blocksB)), dim3(256), 0, stream, q));
+    S.launches.fetch_add(1, std::memory_order_relaxed);
+    CUDA_TRY(cudaGetLastError());
+    return ADAPT_OK;
+}
+
 adapt_status_t launch_reduce(State& S, const float* partial, void* C, int64_t M, int64_t N, int P_k, int dtype, cudaStream_t stream)
 {
     const int64_t Np = partial_pitch(N);
@@ -708,11 +728,15 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
         S.launches.fetch_add(1, std::memory_order_relaxed);
         CUDA_TRY(cudaGetLastError());
         a_src = w8;
+    } else if (padA && padB) {
+        if ((r = launch_pad2(S, A, w8, outA, inA, pitchA, B, w8 + szA, outB, inB, pitchB, stream)) != ADAPT_OK) return r;
+        a_src = w8;
+        b_src = w8 + szA;
     } else if (padA) {
         if ((r = launch_pad(S, A, w8, outA, inA, pitchA, stream)) != ADAPT_OK) return r;
         a_src = w8;
     }
-    if (padB) {
+    if (padB && !(padA && !kclsB)) {
         if ((r = launch_pad(S, B, w8 + szA, outB, inB, pitchB, stream)) != ADAPT_OK) return r;
         b_src = w8 + szA;
     }

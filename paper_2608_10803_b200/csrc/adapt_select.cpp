@@ -146,7 +146,8 @@ static void model_prologue(const Shape& s, Config& c, const Calib& cal)
     if (c.srcB == ADAPT_SRC_PAD_COPY) {
         const double src = 2.0 * (double)s.K * (double)s.N;
         c.ws_padB = round_up(outerB(s) * padded_pitch(innerB(s)) * 2, 256);
-        c.t_pro_us += cal.launch_us + copy_time_us(src + (double)c.ws_padB, cal);
+        // both operands re-pitched: one launch does both
+        c.t_pro_us += (c.srcA == ADAPT_SRC_PAD_COPY ? 0.0 : cal.launch_us) + copy_time_us(src + (double)c.ws_padB, cal);
         c.hbm_bytes += src + (double)c.ws_padB;
     }
 }

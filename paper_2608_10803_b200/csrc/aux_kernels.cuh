@@ -28,15 +28,12 @@ __device__ __forceinline__ unsigned short float_to_16(float a, int dtype)
 // One thread produces one 16-byte chunk of the destination.  The pad columns are never read by
 // the GEMM (the tensor map's extent stays `inner`), so they are written as zeros only to keep
 // the workspace deterministic.
-__global__ void __launch_bounds__(256)
-pad_copy_kernel(const unsigned short* __restrict__ src, unsigned short* __restrict__ dst,
-                int64_t outer, int64_t inner, int64_t pitch)
+__device__ __forceinline__ void pad_copy_body(const unsigned short* __restrict__ src, unsigned short* __restrict__ dst,
+                                              int64_t outer, int64_t inner, int64_t pitch, int block, int blocks)
 {
-    pdl_launch_dependents();
-    pdl_wait();
     const int64_t chunks_per_row = pitch / 8;
     const int64_t total = outer * chunks_per_row;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    for (int64_t i = (int64_t)block * blockDim.x + threadIdx.x; i < total; i += (int64_t)blocks * blockDim.x) {
         const int64_t row = i / chunks_per_row;
         const int64_t c = (i - row * chunks_per_row) * 8;
         const unsigned short* s = src + row * inner + c;
@@ -73,6 +70,33 @@ pad_copy_kernel(const unsigned short* __restrict__ src, unsigned short* __restri
         o.w = (uint32_t)v[6] | ((uint32_t)v[7] << 16);
         *reinterpret_cast<uint4*>(dst + row * pitch + c) = o;
     }
+}
+
+__global__ void __launch_bounds__(256)
+pad_copy_kernel(const unsigned short* __restrict__ src, unsigned short* __restrict__ dst,
+                int64_t outer, int64_t inner, int64_t pitch)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    pad_copy_body(src, dst, outer, inner, pitch, (int)blockIdx.x, (int)gridDim.x);
+}
+
+// Both operands of one call in one launch: the first blocks_a blocks re-pitch A, the rest B.
+struct PadPair {
+    const unsigned short* src[2];
+    unsigned short* dst[2];
+    int64_t outer[2], inner[2], pitch[2];
+    int blocks_a;
+};
+__global__ void __launch_bounds__(256)
+pad_copy2_kernel(const PadPair q)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    if ((int)blockIdx.x < q.blocks_a)
+        pad_copy_body(q.src[0], q.dst[0], q.outer[0], q.inner[0], q.pitch[0], (int)blockIdx.x, q.blocks_a);
+    else
+        pad_copy_body(q.src[1], q.dst[1], q.outer[1], q.inner[1], q.pitch[1], (int)blockIdx.x - q.blocks_a, (int)gridDim.x - q.blocks_a);
 }
 
 // ---- k-class regrouping of A (prologue of the k-class mode) -----------------------------------------
