@@ -135,12 +135,23 @@ const Calib& default_calib();
 constexpr int kClusterStageBytes = 2 * 64 * 144;
 constexpr int kClusterMaxRing = 6;
 inline int cluster_smem_bytes(int ring) { return (ring + 2) * kClusterStageBytes + 128; }   // + two shifted stages, barriers
+// Clusters of a size the machine runs at a time with one CTA per SM (a cluster is placed inside one GPC, so
+// the larger sizes leave SMs unused): what cudaOccupancyMaxActiveClusters reports on a B200 for this kernel
+// with its deepest ring (148, 74, 33, 15, 7), scaled to other SM counts.  With two CTAs per SM (rings of up
+// to four stages; the kernel's registers allow no more) it is about twice that (296, 148, 71, 33, 14).
+inline int64_t cluster_slots(int cluster, int n_sm)
+{
+    const int64_t b200 = cluster == 1 ? 148 : cluster == 2 ? 74 : cluster == 4 ? 33 : cluster == 8 ? 15 : 7;
+    return std::max<int64_t>(1, b200 * n_sm / 148);
+}
+inline int cluster_ctas_per_sm(int ring, int smem_limit) { return std::max(1, std::min(2, smem_limit / cluster_smem_bytes(ring))); }
+// Depth of the raw ring: as deep as the CTA's k range needs, up to 6 stages when the tiles' clusters all run
+// at once with an SM per CTA, else up to 4 so that two CTAs share an SM.
 inline int cluster_ring(int64_t K, int cluster, int64_t tiles, int n_sm)
 {
     const int64_t k_cta = (K + cluster - 1) / cluster;
     const int64_t stages = ((k_cta + 15) / 16 * 16 + 63) / 64;
-    const int64_t per_sm = (tiles * cluster + n_sm - 1) / n_sm;
-    const int cap = per_sm <= 1 ? kClusterMaxRing : (per_sm == 2 ? 4 : 2);
+    const int cap = tiles <= cluster_slots(cluster, n_sm) ? kClusterMaxRing : 4;
     return (int)std::max<int64_t>(1, std::min<int64_t>(stages, cap));
 }
 constexpr int kSkinnyKChunk = 512;   // k values the warp-level kernel stages per chunk; its k splits are whole chunks

@@ -359,10 +359,9 @@ static void model_cluster(const Shape& s, const Machine& m, const Calib& cal, Co
     c.hbm_bytes = 2.0 * (MK + KN + MN);
     const int64_t k_cta = round_up(ceil_div(s.K, c.cluster), 16);
     const double stages = (double)ceil_div(k_cta, 64);
-    // a cluster is placed inside one GPC (about 18 SMs): clusters of 4 and 8 leave SMs of a GPC unused, so
-    // fewer tiles run at a time; two CTAs share an SM when their rings fit
-    const int64_t per_sm = std::min<int64_t>(2, m.smem_bytes / cluster_smem_bytes(c.stages));
-    const int64_t at_a_time = (c.cluster == 1 ? (int64_t)m.n_sm : (int64_t)8 * (18 / c.cluster)) * std::max<int64_t>(1, per_sm);
+    // a cluster is placed inside one GPC, so clusters of 4, 8 and 16 leave SMs unused and fewer tiles run at a
+    // time; two CTAs share an SM when their rings fit
+    const int64_t at_a_time = cluster_slots(c.cluster, m.n_sm) * cluster_ctas_per_sm(c.stages, m.smem_bytes);
     const double waves = (double)ceil_div(tiles, at_a_time);
     // CTAs beyond one per two SMs start to share the load path
     const double crowd = std::max(0.0, (double)units / m.n_sm - 0.5);

@@ -23,6 +23,8 @@
 
 #include <cstdint>
 #include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
 
 #include "adapt_internal.h"
 #include "launch_pdl.cuh"
