@@ -454,6 +454,7 @@ extern "C" adapt_status_t adapt_init(int device)
     CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_2CTA, 256, false, true, 2),
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
     CUDA_TRY(cluster_set_attributes());
+    S.machine.max_cluster = cluster_max_size();
     S.device = device;
     S.inited = true;
     return ADAPT_OK;

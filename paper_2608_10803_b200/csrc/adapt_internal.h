@@ -17,6 +17,7 @@ struct Machine {
     int tmem_cols = 512;                // 128 lanes x 512 fp32 columns per SM (the paper's L0C)
     int64_t workspace_limit = (int64_t)24 << 30;
     unsigned family_mask = 0x1Fu;        // bit f set = family f may be selected
+    int max_cluster = 16;               // largest thread-block cluster the one-launch kernel may ask for (queried at init)
 };
 
 // ---- calibration constants of the latency model (Eq. 8: lambda_r, eta_r, BW_r) ------------

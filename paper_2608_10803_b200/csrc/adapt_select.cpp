@@ -478,7 +478,7 @@ static bool legal_cluster(const Shape& s, const Machine& m, Config& c)
     if (!(m.family_mask & (1u << ADAPT_FAM_CLUSTER))) return false;
     if (c.BM != 64 || c.BN != 64 || c.BK != 64) return false;
     if (c.cluster != 1 && c.cluster != 2 && c.cluster != 4 && c.cluster != 8 && c.cluster != 16) return false;
-    if (c.P_k != c.cluster) return false;                            // the k splits are the cluster's CTAs
+    if (c.P_k != c.cluster || c.cluster > m.max_cluster) return false;    // the k splits are the cluster's CTAs
     if (c.srcA != ADAPT_SRC_LSU || c.srcB != ADAPT_SRC_LSU) return false;
     if ((c.cluster - 1) * round_up(ceil_div(s.K, c.cluster), 16) >= s.K) return false;   // no CTA without k values
     c.P_m = (int)ceil_div(s.M, c.BM);

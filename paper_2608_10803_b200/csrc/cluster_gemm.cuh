@@ -355,6 +355,28 @@ inline cudaError_t cluster_set_attributes()
     return cudaSuccess;
 }
 
+// Largest cluster size (16, 8, 4, 2, 1) of which the device runs at least one cluster with the deepest ring.
+inline int cluster_max_size()
+{
+    for (int cs = 16; cs > 1; cs >>= 1) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)cs, 1, 1);
+        cfg.blockDim = dim3(kClusterThreads, 1, 1);
+        cfg.dynamicSmemBytes = (size_t)cluster_smem_bytes(kClusterMaxRing);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)cs;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, (const void*)cluster_pick(true, false, false), &cfg) == cudaSuccess && n >= 1) return cs;
+        (void)cudaGetLastError();
+    }
+    return 1;
+}
+
 // Host launcher.  c.cluster = CS; c.stages = depth of the raw ring; the grid is CS CTAs per tile, the cluster spans blockIdx.x.
 inline adapt_status_t launch_cluster(const Shape& s, const Config& c, const void* A, const void* B, void* C,
                                      unsigned int* status, cudaStream_t stream)
