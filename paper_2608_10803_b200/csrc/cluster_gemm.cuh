@@ -280,6 +280,36 @@ cluster_gemm_kernel(const ClusterParams p)
     // a wait that gave up: the result is not valid; the host reads the status word
     if (!ok && lane == 0) atomicOr(p.status, 1u);
 
+    // a tile that is not shared with other CTAs is rounded and stored from the accumulators: a lane holds
+    // pairs of neighbouring columns
+    if (p.CS == 1) {
+#pragma unroll
+        for (int mi = 0; mi < 2; ++mi)
+#pragma unroll
+            for (int nj = 0; nj < 2; ++nj)
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    const int m = m0 + m_w + 16 * mi + g + 8 * h, n = n0 + n_w + 8 * nj + 2 * t;
+                    if (m >= p.M || n >= p.N) continue;
+                    unsigned short lo16, hi16;
+                    if (BF16) {
+                        __nv_bfloat16 a = __float2bfloat16_rn(acc[mi][nj][2 * h]), b = __float2bfloat16_rn(acc[mi][nj][2 * h + 1]);
+                        lo16 = *reinterpret_cast<unsigned short*>(&a); hi16 = *reinterpret_cast<unsigned short*>(&b);
+                    } else {
+                        __half a = __float2half_rn(acc[mi][nj][2 * h]), b = __float2half_rn(acc[mi][nj][2 * h + 1]);
+                        lo16 = *reinterpret_cast<unsigned short*>(&a); hi16 = *reinterpret_cast<unsigned short*>(&b);
+                    }
+                    unsigned short* dst = p.C + (int64_t)m * p.N + n;
+                    if (n + 1 < p.N && (reinterpret_cast<uintptr_t>(dst) & 3) == 0) {
+                        *reinterpret_cast<uint32_t*>(dst) = (uint32_t)lo16 | ((uint32_t)hi16 << 16);
+                    } else {
+                        dst[0] = lo16;
+                        if (n + 1 < p.N) dst[1] = hi16;
+                    }
+                }
+        return;
+    }
+
     // the CTA's partial tile, fp32, into its own shared memory
     __syncthreads();
 #pragma unroll
