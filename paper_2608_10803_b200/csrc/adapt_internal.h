@@ -24,7 +24,9 @@ struct Machine {
 // Measured on B200 with this library's own kernels (CUDA events); the paper's values are for
 // other hardware and are not printed, so these are this library's.
 struct Calib {
-    double launch_us = 3.0;             // one kernel launch issued back to back on a stream (also per pad / reduce launch)
+    double launch_us = 3.0;             // one kernel launch issued back to back on a stream (also per reduce launch)
+    double prologue_launch_us = 0.3;    // a re-pitch / regroup launch ahead of the GEMM: its launch overlaps the GEMM's own
+                                        // (programmatic dependent launch); fit over 910 timed small configurations: -0.2 us
     double hbm_bw = 6.2e12;             // B/s, large streaming transfers
     double l2_bw_per_sm = 100e9;        // B/s one SM pulls through TMA from L2 (8192^3, 128 x 256 tiles: 48 KB per 0.48 us)
     double tensor_flops = 1.58e15;      // whole chip, kind::f16, BN = 256 (8192^3 on 256 x 256 pair tiles: 1.56e15)
@@ -34,7 +36,7 @@ struct Calib {
     double mem_latency_us = 1.0;        // TMA issue -> data visible (sets Delta_dep with few stages)
     double hbm_latency_us = 1.6;        // the same under a full HBM stream of a dense operand (128 x 128256 x 4096: 5 stages of 32 KB, 0.41 us each)
     double hbm_latency_views_us = 1.6;  // ... through the strided class views (79457 x 196 x 8325 with 3 stages: 0.75 us per stage)
-    double umma_fixed_us = 2.5;         // barrier init, TMEM alloc, first load, last drain, TMEM free
+    double umma_fixed_us = 1.0;         // barrier init, TMEM alloc, first load, last drain, TMEM free (the same fit: 2.5 was 3 us high)
     // drain of one output tile through the epilogue warps (overlaps the next tile's main loop):
     // fixed part per tile + part per KB written; rows of C that are not 16-byte aligned cost more
     double epi_tile_fixed_us = 0.2, epi_us_per_kb = 0.0275;          // TMA stores (40000 x 40000 x 8: 4.8 TB/s)

@@ -133,21 +133,21 @@ static void model_prologue(const Shape& s, Config& c, const Calib& cal)
         // k-class mode: A is regrouped class-major (element-wise reads, 16-byte writes); B is read in place
         const double src = 2.0 * (double)s.M * (double)s.K;
         c.ws_padA = round_up(s.M * 8 * round_up(ceil_div(s.K, 8), 64) * 2, 256);
-        c.t_pro_us += cal.launch_us + (src + (double)c.ws_padA) / (cal.hbm_bw * cal.regroup_bw_eff) * 1e6;
+        c.t_pro_us += cal.prologue_launch_us + (src + (double)c.ws_padA) / (cal.hbm_bw * cal.regroup_bw_eff) * 1e6;
         c.hbm_bytes += src + (double)c.ws_padA;
         return;
     }
     if (c.srcA == ADAPT_SRC_PAD_COPY) {
         const double src = 2.0 * (double)s.M * (double)s.K;
         c.ws_padA = round_up(outerA(s) * padded_pitch(innerA(s)) * 2, 256);
-        c.t_pro_us += cal.launch_us + copy_time_us(src + (double)c.ws_padA, cal);
+        c.t_pro_us += cal.prologue_launch_us + copy_time_us(src + (double)c.ws_padA, cal);
         c.hbm_bytes += src + (double)c.ws_padA;
     }
     if (c.srcB == ADAPT_SRC_PAD_COPY) {
         const double src = 2.0 * (double)s.K * (double)s.N;
         c.ws_padB = round_up(outerB(s) * padded_pitch(innerB(s)) * 2, 256);
         // both operands re-pitched: one launch does both
-        c.t_pro_us += (c.srcA == ADAPT_SRC_PAD_COPY ? 0.0 : cal.launch_us) + copy_time_us(src + (double)c.ws_padB, cal);
+        c.t_pro_us += (c.srcA == ADAPT_SRC_PAD_COPY ? 0.0 : cal.prologue_launch_us) + copy_time_us(src + (double)c.ws_padB, cal);
         c.hbm_bytes += src + (double)c.ws_padB;
     }
 }
