@@ -48,11 +48,11 @@ struct Calib {
     double simt_step_us = 0.8;          // one 16-k step of a CTA alone on its SM (15 x 30 x 32: two steps, 4.85 us with the launch)
     double halo_edge_tile_us = 3.4;     // row heads or tails of one halo tile, written element-wise
     double simt_bw_eff = 0.15;          // fraction of hbm_bw its 2-byte accesses reach (K = 1 outer products: 0.13 measured)
-    double skinny_bw_eff_aligned = 0.45;    // fraction of hbm_bw the warp-level streaming kernel reaches, 16-byte aligned rows
-    double skinny_bw_eff_unaligned = 0.14;  // ... rows assembled from two chunks
+    double skinny_bw_eff_aligned = 0.32;    // fraction of hbm_bw the warp-level streaming kernel reaches, 16-byte aligned rows
+    double skinny_bw_eff_unaligned = 0.10;  // ... rows assembled from two chunks
     double skinny_fixed_us = 2.0;
-    double skinny_pass_us = 4.0;        // one 64-row pass over one staged chunk when the streamed rows are k-contiguous
-    double skinny_step_unaligned_us = 2.0;   // one 16-k step of a warp when the streamed rows are unaligned
+    double skinny_pass_us = 5.5;        // one 64-row pass over one staged chunk when the streamed rows are k-contiguous
+    double skinny_step_unaligned_us = 2.8;   // one 16-k step of a warp when the streamed rows are unaligned
     double skinny_mac_rate = 30e12;     // MAC/s ceiling of the warp-level kernel (small side padded to 16)
     // one-launch cluster kernel (64 x 64 tiles, k split over a cluster); least-squares fit over 180 timed
     // configurations of 2,000-sweep shapes: 3.7 + 0.95 stages + 0.8 (cluster > 1) + crowd (1.6 + 0.44 stages) us
