@@ -46,7 +46,7 @@ struct Calib {
     double simt_flops = 15e12;          // CUDA-core tile kernel (1000^3: 17e12)
     double simt_fixed_us = 0.45;
     double simt_step_us = 0.8;          // one 16-k step of a CTA alone on its SM (15 x 30 x 32: two steps, 4.85 us with the launch)
-    double halo_edge_tile_us = 3.4;     // row heads or tails of one halo tile, written element-wise
+    double halo_edge_tile_us = 0.8;     // row heads or tails of one halo tile (up to 15 elements per row, aligned stores of 2 to 16 bytes)
     double simt_bw_eff = 0.15;          // fraction of hbm_bw its 2-byte accesses reach (K = 1 outer products: 0.13 measured)
     double skinny_bw_eff_aligned = 0.32;    // fraction of hbm_bw the warp-level streaming kernel reaches, 16-byte aligned rows
     double skinny_bw_eff_unaligned = 0.10;  // ... rows assembled from two chunks

@@ -253,7 +253,7 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     }
     pipe += cal.umma_fixed_us;
     // halo tiles: the first and the last tile of a row block write the elements before the first and after
-    // the last whole 32-byte unit of each row with 2-byte stores (48618 x 28 x 115: 384 such tiles, 17 us)
+    // the last whole 32-byte unit of each row with narrow stores (48618 x 28 x 115: 384 such tiles)
     if (halo && c.P_k == 1)
         pipe += 2.0 * cal.halo_edge_tile_us * (double)c.P_m / (double)std::min<int64_t>(m.n_sm, (int64_t)c.P_m * c.P_n);
     model_prologue(s, c, cal);

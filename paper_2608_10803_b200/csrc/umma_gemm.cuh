@@ -115,6 +115,43 @@ __device__ __forceinline__ unsigned short cast16(float a, int dtype)
     return *reinterpret_cast<unsigned short*>(&h);
 }
 
+// Stores the casts of e[0 .. count), count <= 16, at dst .. dst + count as the fewest aligned stores of 16, 8, 4
+// and 2 bytes.  count and the alignment of dst are the same for every row of a tile, so the branches are
+// uniform; e is indexed with compile-time constants only.
+__device__ __forceinline__ void store_run16(unsigned short* dst, int count, const uint32_t (&e0)[8], const uint32_t (&e1)[8], int dtype)
+{
+    const int a = (int)((reinterpret_cast<uintptr_t>(dst) >> 1) & 7);     // element offset inside a 16-byte chunk
+    int next = 0;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        if (next != i || i >= count) continue;
+        const int pos = a + i, left = count - i;
+#define ADAPT_E(k) __uint_as_float((k) < 8 ? e0[(k) & 7] : e1[(k) & 7])
+        if (i + 8 <= 16 && (pos & 7) == 0 && left >= 8) {
+            uint4 v;
+            v.x = pack16(ADAPT_E(i), ADAPT_E(i + 1), dtype);
+            v.y = pack16(ADAPT_E(i + 2), ADAPT_E(i + 3), dtype);
+            v.z = pack16(ADAPT_E(i + 4), ADAPT_E(i + 5), dtype);
+            v.w = pack16(ADAPT_E(i + 6), ADAPT_E(i + 7), dtype);
+            *reinterpret_cast<uint4*>(dst + i) = v;
+            next = i + 8;
+        } else if (i + 4 <= 16 && (pos & 3) == 0 && left >= 4) {
+            uint2 v;
+            v.x = pack16(ADAPT_E(i), ADAPT_E(i + 1), dtype);
+            v.y = pack16(ADAPT_E(i + 2), ADAPT_E(i + 3), dtype);
+            *reinterpret_cast<uint2*>(dst + i) = v;
+            next = i + 4;
+        } else if (i + 2 <= 16 && (pos & 1) == 0 && left >= 2) {
+            *reinterpret_cast<uint32_t*>(dst + i) = pack16(ADAPT_E(i), ADAPT_E(i + 1), dtype);
+            next = i + 2;
+        } else {
+            dst[i] = cast16(ADAPT_E(i), dtype);
+            next = i + 1;
+        }
+#undef ADAPT_E
+    }
+}
+
 // A_CLS ("row classes", the Padding module without a copy): A is row-major with K % 8 != 0, so its
 // rows are not 16-byte aligned and one tensor map cannot describe it.  Rows r and r + 8 do start
 // at the same offset from a 16-byte boundary (their distance is 16*K bytes), so the rows of one
@@ -492,7 +529,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     // n >= TILE_N * nb, so element x sits in accumulator column x - sigma - TILE_N * nb
                     // = (x - x_first) + 16 - sigma.  The first 16 - sigma elements of a row (x < 16) share their
                     // unit with the previous row of C, the last (N + sigma) % 16 with the next one: the row's own
-                    // thread writes both with 2-byte stores (head: tile nb = 0; tail: the tile that owns the unit).
+                    // thread writes both with aligned stores of 2 to 16 bytes (head: tile nb = 0; tail: the tile that owns the unit).
                     if ((seq & 1) == half) {
                         const int cls = A_CLS ? (mb % NCLS) : 0;
                         const int sig = HALO ? p.c_sigma[cls] : 0;
@@ -516,13 +553,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                                 ptx::tmem_ld_32x8(t_row + (uint32_t)col, e0);
                                 ptx::tmem_ld_32x8(t_row + (uint32_t)(col + 8), e1);
                                 ptx::tmem_ld_wait();
-                                if (row_ok) {
-#pragma unroll
-                                    for (int i = 0; i < 8; ++i) {
-                                        if (i < count) crow[n_first + i] = cast16(__uint_as_float(e0[i]), p.dtype);
-                                        if (8 + i < count) crow[n_first + 8 + i] = cast16(__uint_as_float(e1[i]), p.dtype);
-                                    }
-                                }
+                                if (row_ok) store_run16(crow + n_first, count, e0, e1, p.dtype);
                             }
                         }
 #pragma unroll 1
