@@ -43,6 +43,8 @@ struct Calib {
     double pair_drain_factor = 1.15;    // 40000 x 40000 x 8: 780 us on pair tiles, 671 us on 1-CTA tiles
     double epi_partial_fixed_us = 0.32, epi_partial_us_per_kb = 0.0385;   // fp32 partials, stored by the epilogue threads
     double epi_tile_fixed_unaligned_us = 1.45, epi_us_per_kb_unaligned = 0.054;
+    double thread_store_exposed = 0.4;  // share of the main loop that a drain through the epilogue threads does not hide
+    double thread_store_exposed_pair = 0.25;   // ... on pair tiles (13835 x 3906 x 852 and 7111 x 97981 x 289 bracket it)
     double simt_flops = 15e12;          // CUDA-core tile kernel (1000^3: 17e12)
     double simt_fixed_us = 0.45;
     double simt_step_us = 0.8;          // one 16-k step of a CTA alone on its SM (15 x 30 x 32: two steps, 4.85 us with the launch)
