@@ -225,6 +225,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
     uint8_t* stage_out = bar_gen + kUmmaBarrierBytes;
 
     pdl_launch_dependents();
+    if (threadIdx.x == 0) ADAPT_TRACE(11, 0);
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const uint32_t cta_rank = (CG == 2) ? ptx::cluster_ctarank() : 0u;
@@ -258,25 +259,35 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
     // set-up done: from here on the kernel reads and writes global memory
+    if (threadIdx.x == 0) ADAPT_TRACE(12, 0);
     pdl_wait();
+    if (threadIdx.x == 0) ADAPT_TRACE(13, 0);
 
     const int unit0 = (CG == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int unit_step = (CG == 2) ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (warp == 0) {
         // ------------------------------ producer -----------------------------------------------
-        if (lane == 0) {
+        // One lane per TMA request of a k-block (A: one box, two when M-contiguous; B: one box, or one per 64
+        // columns when N-contiguous): the lanes run the loop together and issue their requests with one
+        // instruction.  A single lane issuing them one after the other spends about 0.1 us per request, which
+        // bounds a 128 x 256 tile with an N-contiguous B (five requests per k-block) at 0.5 us per k-block.
+        constexpr int NREQ_A = A_MN ? 2 : 1;
+        constexpr int NREQ = NREQ_A + (B_MN ? B_BOXES : 1);
+        constexpr uint32_t REQ_MASK = (1u << NREQ) - 1u;
+        if (lane < NREQ) {
             int stage = 0;
             uint32_t phase = 0;
             // the byte count of a stage is signalled on the leader's barrier (pair form)
             uint32_t full_target = full_bar;
             if (CG == 2) asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(full_target) : "r"(full_bar));
             bool ok = true;
-            auto load_a = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int x, int y) {
+            auto load = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int x, int y) {
                 if (CG == 1) ptx::tma_load_2d(dst, tm, bar, x, y);
                 else ptx::tma_load_2d_pair(dst, tm, bar, x, y);
             };
-            auto load_b = load_a;
+            const bool is_a = lane < NREQ_A;
+            const int jb = lane - NREQ_A;                                     // B box of this lane
             for (int unit = unit0; ok && unit < p.num_units; unit += unit_step) {
                 int mb, nb, split;
                 decode_unit(p, unit, mb, nb, split);
@@ -295,41 +306,45 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     // class by class: A' columns j*Kc + 64*b .., B's class-j rows 64*b .. at shifted columns 56*nb ..
                     for (int j = 0; ok && j < 8; ++j)
                         for (int kb = kb0; kb < kb1; ++kb) {
-                            if (!ptx::mbar_wait(empty_bar + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                            ok = __all_sync(REQ_MASK, ptx::mbar_wait(empty_bar + 8u * stage, phase ^ 1u, abort_flag));
+                            if (!ok) break;
                             const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
-                            ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(p.a_tx_bytes + B_BYTES));
-                            load_a(sA, tmA, full_bar + 8u * stage, j * p.cls_kc + kb * kUmmaBK, row0);
-                            load_b(sA + A_BYTES, &maps.b[B_CLS ? j : 0], full_bar + 8u * stage, col0, kb * kUmmaBK);
+                            if (lane == 0) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(p.a_tx_bytes + B_BYTES));
+                            __syncwarp(REQ_MASK);
+                            if (is_a) load(sA, tmA, full_bar + 8u * stage, j * p.cls_kc + kb * kUmmaBK, row0);
+                            else load(sA + A_BYTES, &maps.b[B_CLS ? j : 0], full_bar + 8u * stage, col0, kb * kUmmaBK);
                             if (++stage == S) { stage = 0; phase ^= 1u; }
                         }
                 }
                 for (int kb = kb0; !B_CLS && kb < kb1; ++kb) {
-                    if (!ptx::mbar_wait(empty_bar + 8u * stage, phase ^ 1u, abort_flag)) { ok = false; break; }
+                    ok = __all_sync(REQ_MASK, ptx::mbar_wait(empty_bar + 8u * stage, phase ^ 1u, abort_flag));
+                    if (!ok) break;
                     const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
                     const uint32_t sB = sA + A_BYTES;
                     const uint32_t fb = full_target + 8u * stage;
-                    if (CG == 1) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(p.a_tx_bytes + B_BYTES));
-                    else if (leader) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, 2 * STAGE_BYTES);
+                    if (lane == 0) {
+                        if (CG == 1) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(p.a_tx_bytes + B_BYTES));
+                        else if (leader) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, 2 * STAGE_BYTES);
+                    }
+                    __syncwarp(REQ_MASK);
                     const int k0 = kb * kUmmaBK;
-                    if (!A_MN) {
-                        load_a(sA, tmA, fb, k0 + a_k_off, row0);
+                    // this lane's request: where it lands, through which map, at which coordinates
+                    uint32_t dst;
+                    const CUtensorMap* tm;
+                    int x, y;
+                    if (is_a) {
+                        tm = tmA;
+                        if (!A_MN) { dst = sA; x = k0 + a_k_off; y = row0; }
+                        else { dst = sA + (uint32_t)lane * 8192u; x = row0 + lane * 64; y = k0; }
                     } else {
-#pragma unroll
-                        for (int j = 0; j < 2; ++j) {
-                            load_a(sA + j * 8192, tmA, fb, row0 + j * 64, k0);
-                        }
+                        tm = tmB;
+                        if (B_MN) { dst = sB + (uint32_t)jb * 8192u; x = col0 + jb * 64; y = k0 - kshift; }
+                        else { dst = sB; x = k0; y = col0; }
                     }
-                    if (B_MN) {
-#pragma unroll
-                        for (int j = 0; j < B_BOXES; ++j) {
-                            load_b(sB + j * 8192, tmB, fb, col0 + j * 64, k0 - kshift);
-                        }
-                    } else {
-                        load_b(sB, tmB, fb, k0, col0);
-                    }
+                    load(dst, tm, fb, x, y);
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
-                ADAPT_TRACE(1, unit);
+                if (lane == 0) ADAPT_TRACE(1, unit);
             }
         }
     } else if (warp == 1) {
@@ -787,6 +802,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
         __syncthreads();
     }
     if (threadIdx.x == 0 && *abort_flag) atomicOr(p.status, 1u);
+    if (threadIdx.x == 0) ADAPT_TRACE(14, 0);
     if (warp == 1) {
         ptx::tc_fence_after();
         ptx::tmem_dealloc<CG>(tmem_base, TMEM_COLS);
