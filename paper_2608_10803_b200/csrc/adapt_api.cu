@@ -722,7 +722,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     const void* b_src = B;
     if (kclsB) {
         const int64_t a_sm = s.layoutA == ADAPT_ROW_MAJOR ? s.K : 1, a_sk = s.layoutA == ADAPT_ROW_MAJOR ? 1 : s.M;
-        const int64_t work = s.M * Kc;                    // 16-byte chunks of A'
+        const int64_t work = a_sk == 1 ? s.M * (Kc / 8) : s.M * Kc;   // row-major A: a thread per 64 k of a row; else per 16-byte chunk of A'
         const int blocks = (int)std::min<int64_t>(ceil_div(work, 256), (int64_t)S.machine.n_sm * 16);
         CUDA_TRY(launch_pdl(regroup_a_kernel, dim3(blocks), dim3(256), 0, stream, (const unsigned short*)A, (unsigned short*)w8,
                             (int)s.M, (int)s.K, (int)Kc, a_sm, a_sk));

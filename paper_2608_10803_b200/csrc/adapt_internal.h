@@ -74,7 +74,7 @@ struct Calib {
     double oob_box_penalty = 0.05;      // main-loop cost of one B box per stage that lies wholly beyond N
     double reduce_batch_us = 0.8;       // split-K reduction: one batch of eight slabs (13 x 420 x 43580: P_k 72 -> 24 saves 13 us)
     double class_split_bw_eff = 0.92;   // HBM rate through the k-class views of B with full-width tiles (classes as k splits)
-    double regroup_bw_eff = 0.3;        // class-major regrouping of A (element-wise reads) relative to hbm_bw
+    double regroup_bw_eff = 0.85;       // class-major regrouping of a row-major A (20000 x 8000: 600 MB in 107 us) relative to hbm_bw
     double class_view_bw_eff = 0.8;     // HBM rate through the per-row-class TMA views of an unaligned A
 };
 

@@ -102,15 +102,74 @@ pad_copy2_kernel(const PadPair q)
 // ---- k-class regrouping of A (prologue of the k-class mode) -----------------------------------------
 // A'[m][j * Kc + t] = A[m][8 t + j] for 8 t + j < K, else 0; j = 0..7, t < Kc.  A' is row-major with
 // pitch 8 * Kc (Kc a multiple of 64), so TMA reads the columns of one class as a dense K-major tile.
-// One thread writes eight consecutive t of one (m, j): a 16-byte store; A is read element-wise
-// (it is the small operand when this mode is chosen).
+// Row-major A: one thread takes 64 consecutive k of one row (eight 16-byte loads, assembled from the two
+// covering aligned chunks when the row is not 16-byte aligned), transposes the 8 x 8 block of elements in
+// registers and writes one 16-byte chunk to each of the eight classes.  Any other A, and the ragged end
+// of a row: one thread writes eight consecutive t of one (m, j), reading A element-wise.
+__device__ __forceinline__ uint4 regroup_load8(const unsigned short* p)
+{
+    const uintptr_t a = reinterpret_cast<uintptr_t>(p);
+    const unsigned sh = (unsigned)(a & 15);
+    const uint4* q = reinterpret_cast<const uint4*>(a - sh);
+    const uint4 lo = __ldg(q);
+    if (sh == 0) return lo;
+    const uint4 hi = __ldg(q + 1);                    // holds the group's last bytes: inside the matrix
+    const unsigned ws = sh >> 2;
+    const unsigned sel = 0x3210u + 0x1111u * (sh & 3u);
+    const uint32_t w0 = ws == 0 ? lo.x : ws == 1 ? lo.y : ws == 2 ? lo.z : lo.w;
+    const uint32_t w1 = ws == 0 ? lo.y : ws == 1 ? lo.z : ws == 2 ? lo.w : hi.x;
+    const uint32_t w2 = ws == 0 ? lo.z : ws == 1 ? lo.w : ws == 2 ? hi.x : hi.y;
+    const uint32_t w3 = ws == 0 ? lo.w : ws == 1 ? hi.x : ws == 2 ? hi.y : hi.z;
+    const uint32_t w4 = ws == 0 ? hi.x : ws == 1 ? hi.y : ws == 2 ? hi.z : hi.w;
+    return make_uint4(__byte_perm(w0, w1, sel), __byte_perm(w1, w2, sel), __byte_perm(w2, w3, sel), __byte_perm(w3, w4, sel));
+}
+
 __global__ void __launch_bounds__(256)
 regroup_a_kernel(const unsigned short* __restrict__ A, unsigned short* __restrict__ Ap,
                  int M, int K, int Kc, int64_t a_sm, int64_t a_sk)
 {
     pdl_launch_dependents();
     pdl_wait();
-    const int chunks = Kc / 8;
+    const int chunks = Kc / 8;                       // 16-byte chunks per class segment = blocks of 64 k per row
+    if (a_sk == 1) {
+        const int64_t total = (int64_t)M * chunks;
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+            const int c = (int)(i % chunks);
+            const int m = (int)(i / chunks);
+            const unsigned short* row = A + (int64_t)m * a_sm;
+            unsigned short* dst = Ap + (int64_t)m * 8 * Kc + 8 * c;
+            const int k0 = 64 * c;
+            if (k0 + 64 <= K) {
+                uint4 in[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) in[e] = regroup_load8(row + k0 + 8 * e);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {        // element j of every group: word j / 2, half j % 2
+                    const uint32_t sel = (j & 1) ? 0x7632u : 0x5410u;
+                    uint32_t w[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e)
+                        w[e] = (j >> 1) == 0 ? in[e].x : (j >> 1) == 1 ? in[e].y : (j >> 1) == 2 ? in[e].z : in[e].w;
+                    *reinterpret_cast<uint4*>(dst + (int64_t)j * Kc) =
+                        make_uint4(__byte_perm(w[0], w[1], sel), __byte_perm(w[2], w[3], sel),
+                                   __byte_perm(w[4], w[5], sel), __byte_perm(w[6], w[7], sel));
+                }
+            } else {
+                for (int j = 0; j < 8; ++j) {        // the row's last block: element-wise, zeros past K
+                    unsigned short v[8];
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) {
+                        const int k = k0 + 8 * e + j;
+                        v[e] = k < K ? __ldg(row + k) : (unsigned short)0;
+                    }
+                    *reinterpret_cast<uint4*>(dst + (int64_t)j * Kc) =
+                        make_uint4((uint32_t)v[0] | ((uint32_t)v[1] << 16), (uint32_t)v[2] | ((uint32_t)v[3] << 16),
+                                   (uint32_t)v[4] | ((uint32_t)v[5] << 16), (uint32_t)v[6] | ((uint32_t)v[7] << 16));
+                }
+            }
+        }
+        return;
+    }
     const int64_t total = (int64_t)M * 8 * chunks;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
         const int c = (int)(i % chunks);
