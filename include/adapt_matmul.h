@@ -15,7 +15,13 @@
  *
  * Plain C ABI: no C++ or framework types cross this boundary.  Unless stated, a
  * pointer argument is a HOST pointer; A, B, C and cuda_stream are the exceptions.
- * All functions are thread-safe.  There is no CPU fallback: without a CUDA device
+ * Planning, the queries and the error functions may be called from any number of
+ * threads at once.  The compute calls (adapt_matmul, adapt_matmul_batch,
+ * adapt_matmul_host) may run concurrently on DIFFERENT streams; calls that name the
+ * same stream share that stream's workspace, which a call may have to grow (free and
+ * reallocate), so they must not be made from two threads at once: give each thread
+ * its own stream or serialise the calls.  The adapt_measure_* and adapt_selftest_*
+ * entries are single-threaded tools.  There is no CPU fallback: without a CUDA device
  * the compute entry points fail with ADAPT_ERR_CUDA / ADAPT_ERR_NOT_INIT.
  */
 #ifndef ADAPT_MATMUL_H
@@ -177,12 +183,67 @@ adapt_status_t adapt_matmul_host(adapt_handle_t plan, const void* A_host, const 
  * address (once per device); make that first call outside any stream capture.  All calls share
  * the one array, whatever the stream: two calls that overlap on the GPU race on it, so keep calls
  * on one stream or order them yourself.  The array keeps the previous call's partials; every
- * element a call reads is first written by that call, so nothing needs clearing.
+ * element that contributes to C is first written by the same call, so nothing needs clearing
+ * (the reduction also loads the up to 7 pad columns between N and roundup(N, 8) of each partial
+ * row, which no call writes, but it discards them unused).
  * A, B: DEVICE inputs in the stated layouts, C: DEVICE output, row-major M x N, 2-byte aligned.
  * Enqueues two kernels on the stream and returns without synchronising. */
 adapt_status_t adapt_matmul_noalloc(int64_t M, int64_t N, int64_t K, adapt_dtype_t dtype,
                                     adapt_layout_t layoutA, adapt_layout_t layoutB,
                                     const void* A, const void* B, void* C, void* cuda_stream);
+
+/* `count` independent GEMMs enqueued on one stream by one call: adapt_matmul(plans[i], A[i], B[i], C[i])
+ * for i = 0 .. count-1, in that order, stopping at the first failure.  plans, A, B and C are HOST arrays
+ * of `count` entries (the entries of A, B, C are device pointers).  It is the loop a caller would write,
+ * moved behind the boundary so that a caller in an interpreted language pays its foreign-call cost once per
+ * batch, not once per GEMM; each GEMM is still its own launch(es).  The paper replaces the vendor's
+ * MatMul / GroupMM operators in recommendation models (Section 6.5), whose layers issue exactly such
+ * lists of small GEMMs of different shapes. */
+adapt_status_t adapt_matmul_batch(int64_t count, const adapt_handle_t* plans, const void* const* A,
+                                  const void* const* B, void* const* C, void* cuda_stream);
+
+/* Harness support: `calls` back-to-back adapt_matmul calls of one plan, call i on operand set i % sets
+ * (A, B, C: HOST arrays of `sets` device pointers).  Used to time one shape with rotating buffers. */
+adapt_status_t adapt_matmul_repeat(adapt_handle_t plan, int sets, const void* const* A, const void* const* B,
+                                   void* const* C, int calls, void* cuda_stream);
+
+/* Host cost of the online call (Section 3.2 claims a "near-zero" dispatch; this measures it).
+ * Runs `calls` adapt_matmul calls of the plan on the given operands three ways and reports, per call,
+ * the host time (steady_clock around the calls, in batches of 128 with a stream synchronisation between
+ * batches so the launch queue never fills) and the device time (CUDA events around each batch):
+ * with the tensor-map cache on (the steady state of a caller that reuses buffers), with the cache
+ * bypassed (every call encodes its tensor maps: a caller whose pointers are new every time), and as
+ * bare launches: the kernels of one call, recorded with their exact configurations and arguments and
+ * replayed through cudaLaunchKernelExC with none of the library's logic around them.
+ * host_us_call - host_us_bare_launches is what the library adds to the launches themselves.
+ * The bare fields are -1 when a launch could not be recorded.  Synchronises the stream. */
+typedef struct adapt_dispatch_cost_s {
+    double host_us_call, host_us_call_map_miss, host_us_bare_launches;
+    double device_us_call, device_us_call_map_miss, device_us_bare_launches;
+    int32_t launches_per_call;   /* kernels one call enqueues (prologue + GEMM + reduce) */
+    int32_t maps_per_call;       /* tensor maps a call encodes when none is cached */
+} adapt_dispatch_cost_t;
+adapt_status_t adapt_measure_dispatch(adapt_handle_t plan, const void* A, const void* B, void* C,
+                                      void* cuda_stream, int calls, adapt_dispatch_cost_t* out);
+
+/* The launch floor: `launches` empty kernels back to back on the stream, with (programmatic != 0) or
+ * without programmatic dependent launch; per launch, the host time and the device time (same batching
+ * as above).  Every call of this library costs at least this much, whatever the kernel does. */
+adapt_status_t adapt_measure_empty_launch(int launches, int programmatic, void* cuda_stream,
+                                          double* host_us, double* device_us);
+
+/* Tensor maps encoded on the host since adapt_init; a call whose maps are cached encodes none.  Each plan
+ * keeps the encodings of its 8 most recent distinct (pointer, geometry) pairs per operand. */
+int64_t adapt_map_encode_count(void);
+/* enabled = 0 bypasses the tensor-map cache (every call encodes); 1 restores it.  Measurement only. */
+void adapt_set_map_cache(int enabled);
+
+/* Self-test of the bounded-wait path: enqueues a one-warp kernel that waits, with the same bounded wait
+ * the GEMM kernels use and a limit of limit_ns (at most 0.1 s), on a barrier nobody arrives on.  The wait
+ * gives up, the kernel ends normally and sets the device status word, and the next
+ * adapt_poll_device_status on the stream returns ADAPT_ERR_TIMEOUT (and clears the word).  Nothing is left
+ * waiting and the context stays usable.  The paper has no counterpart. */
+adapt_status_t adapt_selftest_wait_expiry(uint64_t limit_ns, void* cuda_stream);
 
 /* Thread-local status of the last failing call on this thread, and its text. */
 adapt_status_t adapt_last_error(void);

@@ -24,7 +24,8 @@ EXPORTS = [
     "adapt_last_error_message", "adapt_status_string", "adapt_plan_info", "adapt_plan_candidates",
     "adapt_matmul_plan_forced", "adapt_classify", "adapt_model_read_volume", "adapt_model_write_volume",
     "adapt_model_pipeline", "adapt_poll_device_status", "adapt_plan_cache_size", "adapt_launch_count",
-    "adapt_matmul_noalloc",
+    "adapt_matmul_noalloc", "adapt_matmul_batch", "adapt_matmul_repeat", "adapt_measure_dispatch",
+    "adapt_measure_empty_launch", "adapt_map_encode_count", "adapt_set_map_cache", "adapt_selftest_wait_expiry",
 ]
 
 
@@ -48,8 +49,21 @@ class PlanInfo(ctypes.Structure):
     def as_dict(self):
         d = {k: getattr(self, k) for k, _ in self._fields_}
         d["class_name"] = CLASS_NAMES[self.taxonomy_class]
-        d["family_name"] = FAMILY_NAMES[self.family] if 0 <= self.family < 4 else "?"
+        d["family_name"] = FAMILY_NAMES[self.family] if 0 <= self.family < len(FAMILY_NAMES) else "?"
         return d
+
+
+class DispatchCost(ctypes.Structure):
+    _fields_ = [
+        ("host_us_call", ctypes.c_double), ("host_us_call_map_miss", ctypes.c_double),
+        ("host_us_bare_launches", ctypes.c_double),
+        ("device_us_call", ctypes.c_double), ("device_us_call_map_miss", ctypes.c_double),
+        ("device_us_bare_launches", ctypes.c_double),
+        ("launches_per_call", ctypes.c_int32), ("maps_per_call", ctypes.c_int32),
+    ]
+
+    def as_dict(self):
+        return {k: getattr(self, k) for k, _ in self._fields_}
 
 
 class AdaptError(RuntimeError):
@@ -104,6 +118,19 @@ def load():
     lib.adapt_poll_device_status.argtypes = [vp]
     lib.adapt_plan_cache_size.restype = i64
     lib.adapt_launch_count.restype = i64
+    lib.adapt_map_encode_count.restype = i64
+    lib.adapt_set_map_cache.restype = None
+    lib.adapt_set_map_cache.argtypes = [i32]
+    lib.adapt_matmul_batch.restype = i32
+    lib.adapt_matmul_batch.argtypes = [i64, vp, vp, vp, vp, vp]
+    lib.adapt_matmul_repeat.restype = i32
+    lib.adapt_matmul_repeat.argtypes = [vp, i32, vp, vp, vp, i32, vp]
+    lib.adapt_measure_dispatch.restype = i32
+    lib.adapt_measure_dispatch.argtypes = [vp, vp, vp, vp, vp, i32, ctypes.POINTER(DispatchCost)]
+    lib.adapt_measure_empty_launch.restype = i32
+    lib.adapt_measure_empty_launch.argtypes = [i32, i32, vp, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
+    lib.adapt_selftest_wait_expiry.restype = i32
+    lib.adapt_selftest_wait_expiry.argtypes = [u64, vp]
     _lib = lib
     return lib
 
@@ -150,8 +177,50 @@ def adapt_matmul_host(plan, A_host_ptr: int, B_host_ptr: int, C_host_ptr: int, s
 def adapt_matmul_noalloc(M, N, K, dtype, layoutA, layoutB, A_ptr: int, B_ptr: int, C_ptr: int, stream: int = 0):
     """C = A*B without any device allocation: split-K partials go to the library's fixed 4 MiB
     scratch.  For callers that may not call cudaMalloc; the output must satisfy
-    2 * M * roundup(N, 4) * 4 bytes <= 4 MiB.  Calls that overlap on the GPU race on the scratch."""
+    2 * M * roundup(N, 8) * 4 bytes <= 4 MiB.  Calls that overlap on the GPU race on the scratch."""
     _check(load().adapt_matmul_noalloc(M, N, K, dtype, layoutA, layoutB, A_ptr, B_ptr, C_ptr, stream))
+
+
+def pointer_array(values):
+    """A host array of pointers (plans or device addresses) for the batched entry points."""
+    return (ctypes.c_void_p * len(values))(*values)
+
+
+def adapt_matmul_batch(plans, A_ptrs, B_ptrs, C_ptrs, stream: int = 0, count=None):
+    """adapt_matmul(plans[i], A[i], B[i], C[i]) for every i, one foreign call.  The arguments are
+    ``pointer_array`` objects (or sequences, converted here)."""
+    arrs = [a if isinstance(a, ctypes.Array) else pointer_array(list(a)) for a in (plans, A_ptrs, B_ptrs, C_ptrs)]
+    _check(load().adapt_matmul_batch(len(arrs[0]) if count is None else count, *arrs, stream))
+
+
+def adapt_matmul_repeat(plan, A_ptrs, B_ptrs, C_ptrs, calls: int, stream: int = 0):
+    arrs = [a if isinstance(a, ctypes.Array) else pointer_array(list(a)) for a in (A_ptrs, B_ptrs, C_ptrs)]
+    _check(load().adapt_matmul_repeat(plan, len(arrs[0]), *arrs, calls, stream))
+
+
+def adapt_measure_dispatch(plan, A_ptr: int, B_ptr: int, C_ptr: int, stream: int = 0, calls: int = 100000) -> DispatchCost:
+    out = DispatchCost()
+    _check(load().adapt_measure_dispatch(plan, A_ptr, B_ptr, C_ptr, stream, calls, ctypes.byref(out)))
+    return out
+
+
+def adapt_measure_empty_launch(launches: int, programmatic: bool, stream: int = 0):
+    """(host us, device us) per launch of an empty kernel issued back to back."""
+    h, d = ctypes.c_double(), ctypes.c_double()
+    _check(load().adapt_measure_empty_launch(launches, 1 if programmatic else 0, stream, ctypes.byref(h), ctypes.byref(d)))
+    return h.value, d.value
+
+
+def adapt_map_encode_count() -> int:
+    return load().adapt_map_encode_count()
+
+
+def adapt_set_map_cache(enabled: bool):
+    load().adapt_set_map_cache(1 if enabled else 0)
+
+
+def adapt_selftest_wait_expiry(limit_ns: int, stream: int = 0):
+    _check(load().adapt_selftest_wait_expiry(limit_ns, stream))
 
 
 def adapt_plan_info(plan) -> PlanInfo:

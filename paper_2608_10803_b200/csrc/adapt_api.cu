@@ -1,6 +1,7 @@
 // C ABI of the library: plan cache (online O(1) dispatch, Section 3.2), launch_map (TilingKey ->
 // compiled kernel), tensor-map construction, workspace management and the launches themselves.
 #include <atomic>
+#include <chrono>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -45,12 +46,21 @@ static adapt_status_t fail(adapt_status_t st, const char* fmt, const char* detai
 // ---------------------------------------------------------------------------------------------
 // plans and the plan cache
 // ---------------------------------------------------------------------------------------------
+// One cached encoding of an operand's tensor map(s).  The key is everything the encoding depends on: the base
+// pointer, the row pitch, the extents and the box (one plan can reach the same buffer with two geometries:
+// a k-class plan falls back to plain tiles when B's pointer is unaligned), and the number of maps.
 struct MapSlot {
     const void* ptr = nullptr;
-    int64_t pitch = 0;
+    int64_t pitch = 0, inner = 0, outer = 0;
+    int box_inner = 0, box_outer = 0;
     int count = 0;            // 1, or the number of per-class maps (8 or 16)
-    CUtensorMap map[16];
+    std::vector<CUtensorMap> map;
+    bool matches(const void* p, int64_t pi, int64_t in, int64_t ou, int bi, int bo, int n) const
+    {
+        return ptr == p && pitch == pi && inner == in && outer == ou && box_inner == bi && box_outer == bo && count == n;
+    }
 };
+constexpr int kMapSlots = 8;   // most recent distinct (pointer, geometry) pairs kept per operand and plan
 
 struct adapt_plan_s {
     Shape s;
@@ -58,7 +68,7 @@ struct adapt_plan_s {
     bool noop = false;        // M == 0 or N == 0
     bool zero_fill = false;   // K == 0
     std::mutex mu;            // guards the tensor-map slots
-    MapSlot maps[3][2];       // per operand (kMapA, kMapB, kMapC): the two most recent base pointers
+    std::vector<MapSlot> maps[3];   // per operand (kMapA, kMapB, kMapC): up to kMapSlots entries, replaced round-robin
     int next[3] = {0, 0, 0};
 };
 enum { kMapA = 0, kMapB = 1, kMapC = 2 };
@@ -127,6 +137,8 @@ struct State {
     std::unordered_map<cudaStream_t, HostPipe> pipes;
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
     std::atomic<int64_t> launches{0};
+    std::atomic<int64_t> map_encodes{0};   // tensor maps encoded on the host so far (a cached call encodes none)
+    std::atomic<int> map_cache{1};         // 0: every call encodes its maps afresh (measurement of the miss cost)
     int log = 0;
     bool class_promo128 = true;        // 128-byte L2 promotion for the strided class views (ADAPT_CLASS_PROMO128=0: 256 as for dense operands)
 };
@@ -361,6 +373,8 @@ extern "C" int64_t adapt_plan_cache_size(void)
     return (int64_t)S.all_plans.size();
 }
 extern "C" int64_t adapt_launch_count(void) { return st().launches.load(); }
+extern "C" int64_t adapt_map_encode_count(void) { return st().map_encodes.load(); }
+extern "C" void adapt_set_map_cache(int enabled) { st().map_cache.store(enabled ? 1 : 0); }
 
 // ---------------------------------------------------------------------------------------------
 // launch_map: (family, BN, A major, B major) -> compiled kernel
@@ -495,6 +509,8 @@ extern "C" void adapt_shutdown(void)
     S.inited = false;
     S.device = -1;
     S.launches.store(0);
+    S.map_encodes.store(0);
+    S.map_cache.store(1);
 }
 
 extern "C" adapt_status_t adapt_poll_device_status(void* cuda_stream)
@@ -565,21 +581,33 @@ adapt_status_t encode_map(State& S, CUtensorMap* map, const void* base, int dtyp
     return ADAPT_OK;
 }
 
+// The slot a new encoding goes to: a fresh one while fewer than kMapSlots exist, then round-robin.
+MapSlot& take_slot(Plan* pl, int which)
+{
+    std::vector<MapSlot>& slots = pl->maps[which];
+    if ((int)slots.size() < kMapSlots) { slots.emplace_back(); return slots.back(); }
+    int& next = pl->next[which];
+    MapSlot& sl = slots[next];
+    next = (next + 1) % kMapSlots;
+    return sl;
+}
+
 adapt_status_t cached_map(State& S, Plan* pl, int which, const void* base, int64_t inner, int64_t outer, int64_t pitch,
                           int box_inner, int box_outer, CUtensorMap* out)
 {
     std::lock_guard<std::mutex> lock(pl->mu);
-    MapSlot* slots = pl->maps[which];
-    for (int i = 0; i < 2; ++i)
-        if (slots[i].ptr == base && slots[i].pitch == pitch && slots[i].count == 1) { *out = slots[i].map[0]; return ADAPT_OK; }
-    int& next = pl->next[which];
-    MapSlot& sl = slots[next];
-    next ^= 1;
+    std::vector<MapSlot>& slots = pl->maps[which];
+    const bool use_cache = S.map_cache.load(std::memory_order_relaxed) != 0;
+    for (const MapSlot& sl : slots)
+        if (use_cache && sl.matches(base, pitch, inner, outer, box_inner, box_outer, 1)) { *out = sl.map[0]; return ADAPT_OK; }
+    S.map_encodes.fetch_add(1, std::memory_order_relaxed);
+    MapSlot& sl = take_slot(pl, which);
+    sl.ptr = nullptr;
+    sl.map.resize(1);
     adapt_status_t r = encode_map(S, &sl.map[0], base, pl->s.dtype, inner, outer, pitch, box_inner, box_outer);
-    if (r != ADAPT_OK) { sl.ptr = nullptr; return r; }
-    sl.ptr = base;
-    sl.pitch = pitch;
-    sl.count = 1;
+    if (r != ADAPT_OK) return r;
+    sl.ptr = base; sl.pitch = pitch; sl.inner = inner; sl.outer = outer;
+    sl.box_inner = box_inner; sl.box_outer = box_outer; sl.count = 1;
     *out = sl.map[0];
     return ADAPT_OK;
 }
@@ -601,16 +629,17 @@ adapt_status_t cached_class_maps(State& S, Plan* pl, int which, const void* base
         sigma[j] = (int)(((2 * j * cols) & (align - 1)) / 2);
         if (extent) extent[j] = (int)(whole_units ? (cols + sigma[j]) / unit * unit : cols + sigma[j]);
     }
-    MapSlot* slots = pl->maps[which];
-    for (int i = 0; i < 2; ++i)
-        if (slots[i].ptr == base_ptr && slots[i].pitch == cols && slots[i].count == ncls) {
-            memcpy(out, slots[i].map, ncls * sizeof(CUtensorMap));
+    std::vector<MapSlot>& slots = pl->maps[which];
+    const bool use_cache = S.map_cache.load(std::memory_order_relaxed) != 0;
+    for (const MapSlot& sl : slots)
+        if (use_cache && sl.matches(base_ptr, cols, whole_units ? 1 : 0, rows_total, 64, box_rows, ncls)) {
+            memcpy(out, sl.map.data(), ncls * sizeof(CUtensorMap));
             return ADAPT_OK;
         }
-    int& next = pl->next[which];
-    MapSlot& sl = slots[next];
-    next ^= 1;
+    S.map_encodes.fetch_add(ncls, std::memory_order_relaxed);
+    MapSlot& sl = take_slot(pl, which);
     sl.ptr = nullptr;
+    sl.map.resize(ncls);
     for (int j = 0; j < ncls; ++j) {
         const uint8_t* base = (const uint8_t*)base_ptr + ((2 * j * cols) & ~(int64_t)(align - 1));
         const int64_t rows = std::max<int64_t>(1, ceil_div(rows_total - j, ncls));
@@ -619,10 +648,9 @@ adapt_status_t cached_class_maps(State& S, Plan* pl, int which, const void* base
         adapt_status_t r = encode_map(S, &sl.map[j], base, pl->s.dtype, inner, rows, (int64_t)ncls * cols, 64, box_rows, true);
         if (r != ADAPT_OK) return r;
     }
-    sl.ptr = base_ptr;
-    sl.pitch = cols;
-    sl.count = ncls;
-    memcpy(out, sl.map, ncls * sizeof(CUtensorMap));
+    sl.ptr = base_ptr; sl.pitch = cols; sl.inner = whole_units ? 1 : 0; sl.outer = rows_total;
+    sl.box_inner = 64; sl.box_outer = box_rows; sl.count = ncls;
+    memcpy(out, sl.map.data(), ncls * sizeof(CUtensorMap));
     return ADAPT_OK;
 }
 
@@ -823,17 +851,20 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     TmapPackT<2> pack2;                                     // modes 2 and 3 take the same maps
     static_assert(sizeof(TmapPackT<2>) == sizeof(TmapPackT<3>), "k-class packs share their layout");
     void* args[2] = {nullptr, &p};
+    size_t arg_bytes[2] = {sizeof(pack0), sizeof(p)};
     if (classesA) {
+        arg_bytes[0] = sizeof(pack1);
         memcpy(pack1.a, maps.a, sizeof(pack1.a)); pack1.b[0] = maps.b[0]; memcpy(pack1.c, maps.c, sizeof(pack1.c));
         args[0] = &pack1;
     } else if (kclsB) {
+        arg_bytes[0] = sizeof(pack2);
         pack2.a[0] = maps.a[0]; memcpy(pack2.b, maps.b, sizeof(pack2.b)); pack2.c[0] = maps.c[0];
         args[0] = &pack2;
     } else {
         pack0.a[0] = maps.a[0]; pack0.b[0] = maps.b[0]; pack0.c[0] = maps.c[0];
         args[0] = &pack0;
     }
-    CUDA_TRY(cudaLaunchKernelExC(&cfg, k, args));
+    CUDA_TRY(launch_exc(&cfg, k, args, arg_bytes, 2));
     S.launches.fetch_add(1, std::memory_order_relaxed);
     if (p.P_k > 1) return launch_reduce(S, partial, C, s.M, s.N, p.P_k, s.dtype, stream);
     return ADAPT_OK;
@@ -988,6 +1019,150 @@ extern "C" adapt_status_t adapt_matmul_host(adapt_handle_t plan, const void* A_h
     CUDA_TRY(cudaEventRecord(hp->ev_out[b], hp->out));
     // work the caller enqueues on its stream after this call sees C_host complete
     CUDA_TRY(cudaStreamWaitEvent(stream, hp->ev_out[b], 0));
+    return ADAPT_OK;
+}
+
+
+// ---------------------------------------------------------------------------------------------
+// batched call, measurement support, self-test
+// ---------------------------------------------------------------------------------------------
+extern "C" adapt_status_t adapt_matmul_batch(int64_t count, const adapt_handle_t* plans, const void* const* A,
+                                             const void* const* B, void* const* C, void* cuda_stream)
+{
+    if (count < 0 || (count > 0 && (!plans || !A || !B || !C))) return fail(ADAPT_ERR_INVALID_ARG, "null array%s");
+    for (int64_t i = 0; i < count; ++i) {
+        const adapt_status_t r = adapt_matmul(plans[i], A[i], B[i], C[i], cuda_stream);
+        if (r != ADAPT_OK) return r;
+    }
+    return ADAPT_OK;
+}
+
+extern "C" adapt_status_t adapt_matmul_repeat(adapt_handle_t plan, int sets, const void* const* A, const void* const* B,
+                                              void* const* C, int calls, void* cuda_stream)
+{
+    if (sets < 1 || calls < 0 || !A || !B || !C) return fail(ADAPT_ERR_INVALID_ARG, "bad set count or null array%s");
+    for (int i = 0; i < calls; ++i) {
+        const int j = i % sets;
+        const adapt_status_t r = adapt_matmul(plan, A[j], B[j], C[j], cuda_stream);
+        if (r != ADAPT_OK) return r;
+    }
+    return ADAPT_OK;
+}
+
+namespace {
+double now_us()
+{
+    return std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now().time_since_epoch()).count();
+}
+}  // namespace
+
+extern "C" adapt_status_t adapt_measure_dispatch(adapt_handle_t plan, const void* A, const void* B, void* C,
+                                                 void* cuda_stream, int calls, adapt_dispatch_cost_t* out)
+{
+    State& S = st();
+    if (!plan || !out || calls < 1) return fail(ADAPT_ERR_INVALID_ARG, "null argument%s");
+    if (!S.inited) return fail(ADAPT_ERR_NOT_INIT, "adapt_init has not been called%s");
+    memset(out, 0, sizeof(*out));
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // warm-up (workspace, tensor maps), with the launches of one call written down for the bare replay
+    static thread_local LaunchRecord rec;
+    rec.n = 0;
+    adapt_status_t r = adapt_matmul(plan, A, B, C, cuda_stream);
+    if (r != ADAPT_OK) return r;
+    const int64_t l0 = S.launches.load(), e0 = S.map_encodes.load();
+    launch_recorder() = &rec;
+    r = adapt_matmul(plan, A, B, C, cuda_stream);
+    launch_recorder() = nullptr;
+    if (r != ADAPT_OK) return r;
+    out->launches_per_call = (int32_t)(S.launches.load() - l0);
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    cudaEvent_t ev0, ev1;
+    CUDA_TRY(cudaEventCreate(&ev0));
+    CUDA_TRY(cudaEventCreate(&ev1));
+    // batches short enough that the launch queue never fills: the host clock then sees host work only
+    const int batch = 128;
+    double host[3] = {0, 0, 0}, dev_ms[3] = {0, 0, 0};
+    for (int mode = 0; mode < 3; ++mode) {          // 0: cached maps, 1: maps encoded on every call, 2: bare launches
+        if (mode == 2 && rec.n != out->launches_per_call) { host[2] = -1.0; break; }
+        S.map_cache.store(mode == 1 ? 0 : 1);
+        const int64_t enc0 = S.map_encodes.load();
+        for (int done = 0; done < calls; done += batch) {
+            const int n = std::min(batch, calls - done);
+            CUDA_TRY(cudaEventRecord(ev0, stream));
+            const double t0 = now_us();
+            for (int i = 0; i < n; ++i) {
+                if (mode < 2) {
+                    r = adapt_matmul(plan, A, B, C, cuda_stream);
+                    if (r != ADAPT_OK) { S.map_cache.store(1); return r; }
+                } else {
+                    for (int l = 0; l < rec.n; ++l) CUDA_TRY(launch_replay(rec.launch[l], stream));
+                }
+            }
+            host[mode] += now_us() - t0;
+            CUDA_TRY(cudaEventRecord(ev1, stream));
+            CUDA_TRY(cudaStreamSynchronize(stream));
+            float ms = 0.f;
+            CUDA_TRY(cudaEventElapsedTime(&ms, ev0, ev1));
+            dev_ms[mode] += ms;
+        }
+        if (mode == 1) out->maps_per_call = (int32_t)((S.map_encodes.load() - enc0) / calls);
+    }
+    S.map_cache.store(1);
+    (void)e0;
+    cudaEventDestroy(ev0);
+    cudaEventDestroy(ev1);
+    out->host_us_call = host[0] / calls;
+    out->host_us_call_map_miss = host[1] / calls;
+    out->host_us_bare_launches = host[2] < 0 ? -1.0 : host[2] / calls;
+    out->device_us_call = dev_ms[0] * 1e3 / calls;
+    out->device_us_call_map_miss = dev_ms[1] * 1e3 / calls;
+    out->device_us_bare_launches = host[2] < 0 ? -1.0 : dev_ms[2] * 1e3 / calls;
+    return ADAPT_OK;
+}
+
+extern "C" adapt_status_t adapt_measure_empty_launch(int launches, int programmatic, void* cuda_stream,
+                                                     double* host_us, double* device_us)
+{
+    if (launches < 1 || !host_us || !device_us) return fail(ADAPT_ERR_INVALID_ARG, "bad argument%s");
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const bool saved = pdl_enabled();
+    pdl_enabled() = programmatic != 0;
+    cudaEvent_t ev0, ev1;
+    CUDA_TRY(cudaEventCreate(&ev0));
+    CUDA_TRY(cudaEventCreate(&ev1));
+    for (int i = 0; i < 16; ++i) (void)launch_pdl(empty_kernel, dim3(1), dim3(32), 0, stream, 0);
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    const int batch = 128;
+    double host = 0, dev_ms = 0;
+    for (int done = 0; done < launches; done += batch) {
+        const int n = std::min(batch, launches - done);
+        CUDA_TRY(cudaEventRecord(ev0, stream));
+        const double t0 = now_us();
+        for (int i = 0; i < n; ++i) (void)launch_pdl(empty_kernel, dim3(1), dim3(32), 0, stream, i);
+        host += now_us() - t0;
+        CUDA_TRY(cudaEventRecord(ev1, stream));
+        CUDA_TRY(cudaStreamSynchronize(stream));
+        float ms = 0.f;
+        CUDA_TRY(cudaEventElapsedTime(&ms, ev0, ev1));
+        dev_ms += ms;
+    }
+    pdl_enabled() = saved;
+    cudaEventDestroy(ev0);
+    cudaEventDestroy(ev1);
+    CUDA_TRY(cudaGetLastError());
+    *host_us = host / launches;
+    *device_us = dev_ms * 1e3 / launches;
+    return ADAPT_OK;
+}
+
+extern "C" adapt_status_t adapt_selftest_wait_expiry(uint64_t limit_ns, void* cuda_stream)
+{
+    State& S = st();
+    if (!S.inited) return fail(ADAPT_ERR_NOT_INIT, "adapt_init has not been called%s");
+    if (limit_ns > 100000000ull) return fail(ADAPT_ERR_INVALID_ARG, "the self-test's wait limit is at most 0.1 s%s");
+    CUDA_TRY(launch_pdl(wait_expiry_kernel, dim3(1), dim3(32), 0, (cudaStream_t)cuda_stream, S.d_status, (unsigned long long)limit_ns));
+    S.launches.fetch_add(1, std::memory_order_relaxed);
+    CUDA_TRY(cudaGetLastError());
     return ADAPT_OK;
 }
 

@@ -8,6 +8,7 @@
 #include <cuda_bf16.h>
 
 #include "launch_pdl.cuh"
+#include "ptx_sm100.cuh"
 
 namespace adapt {
 
@@ -313,6 +314,36 @@ simt_gemm_kernel(const unsigned short* __restrict__ A, const unsigned short* __r
             else p.partial[((int64_t)split * p.M + m) * p.Np + n] = acc[i][j];
         }
     }
+}
+
+// ---- measurement and self-test kernels ---------------------------------------------------------------
+// The cheapest kernel this library can launch: the launch floor that every call pays.
+__global__ void empty_kernel(int dummy)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    (void)dummy;
+}
+
+// One warp waits, with the library's bounded wait and a caller-chosen limit, on a barrier that nobody ever
+// arrives on.  The wait must give up, raise the abort flag and let the kernel end normally with bit 0 of the
+// status word set: the same path a tensor-core kernel takes when a load or an MMA never signals.  No TMA, no
+// TMEM, nothing left in flight.
+__global__ void wait_expiry_kernel(unsigned int* status, unsigned long long limit_ns)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    __shared__ int abort_flag;
+    pdl_launch_dependents();
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        ptx::mbar_init(ptx::smem_u32(&bar), 1);
+        ptx::fence_barrier_init();
+    }
+    __syncthreads();
+    pdl_wait();
+    const bool ok = ptx::mbar_wait_limit(ptx::smem_u32(&bar), 0u, &abort_flag, limit_ns);
+    __syncthreads();
+    if (threadIdx.x == 0 && (!ok || abort_flag)) atomicOr(status, 1u);
 }
 
 }  // namespace adapt

@@ -8,12 +8,12 @@
 // through distributed shared memory, in ascending rank order (the order of a split-K reduction,
 // fixed, so the result does not depend on timing), rounds once and stores C.  No workspace.
 //
-// Operands come in as one bulk copy (cp.async.bulk) per 64-element row into a ring of raw stages (64 x 64
-// of each operand per stage, kept in the operand's own orientation), each stage completing on an mbarrier:
-// the whole ring is in flight before the first wait, so a CTA pays about one trip to memory for 64 x ring
-// values of k.  A row is copied as the aligned 16-byte chunks that hold it, whatever its alignment, and
-// shifted into place by byte permutes, shared memory to shared memory, masked at the ragged edges, so no
-// access is element-wise.  ldmatrix (transposing when the operand's contiguous dimension is not k) feeds
+// Operands come in as 16-byte cp.async.cg copies into a ring of raw stages (64 x 64 of each operand per
+// stage, kept in the operand's own orientation); every thread's copies of a stage arrive on the stage's
+// mbarrier (cp.async.mbarrier.arrive.noinc): the whole ring is in flight before the first wait, so a CTA
+// pays about one trip to memory for 64 x ring values of k.  A row is copied as the up to nine aligned
+// 16-byte chunks that hold it, whatever its alignment, and shifted into place by byte permutes, shared
+// memory to shared memory, masked at the ragged edges, so no access is element-wise.  ldmatrix (transposing when the operand's contiguous dimension is not k) feeds
 // mma.sync.m16n8k16 with fp32 accumulation.
 #pragma once
 
@@ -243,11 +243,13 @@ cluster_gemm_kernel(const ClusterParams p)
     for (int s = 0; s < n_stages; ++s) {
         const int slot = s % S, buf = s & 1;
         const int k0 = k_begin + s * kClusterKS;
-        // bounded wait for the stage's rows; a warp leaves the loop as one
+        // bounded wait for the stage's rows.  The decision to leave is taken by the CTA as a whole: every thread
+        // reaches the barrier below in every iteration, whether its own wait succeeded or gave up, so the barrier
+        // counts of the warps never drift apart and all of them take the same path to the common exit.
         const bool landed = ptx::mbar_wait(bar0 + 8u * slot, (uint32_t)((s / S) & 1), abort_flag);
-        if (!__all_sync(0xffffffffu, landed)) { ok = false; break; }
-        shift_stage(slot, buf, k0);
-        __syncthreads();            // shifted stage complete; raw slot free; every warp is past the MMAs of stage s - 1
+        if (landed) shift_stage(slot, buf, k0);
+        // shifted stage complete; raw slot free; every warp is past the MMAs of stage s - 1
+        if (__syncthreads_or(landed ? 0 : 1)) { ok = false; break; }
         if (s + S < n_stages) issue_stage(slot, k0 + S * kClusterKS);
         const uint32_t sa = fin0 + (uint32_t)(buf * STAGE), sb = sa + (uint32_t)OPND;
         auto k_step = [&](int kk) {
@@ -277,8 +279,9 @@ cluster_gemm_kernel(const ClusterParams p)
             for (int kk = 0; k0 + kk < k_end; kk += 16) k_step(kk);
         }
     }
-    // a wait that gave up: the result is not valid; the host reads the status word
-    if (!ok && lane == 0) atomicOr(p.status, 1u);
+    // a wait that gave up: the result is not valid; the host reads the status word.  `ok` is the same in every
+    // thread of the CTA, and the CTA still runs the barriers below (the cluster barriers too: its peers count on them).
+    if (!ok && tid == 0) atomicOr(p.status, 1u);
 
     // a tile that is not shared with other CTAs is rounded and stored from the accumulators: a lane holds
     // pairs of neighbouring columns
@@ -425,6 +428,7 @@ inline adapt_status_t launch_cluster(const Shape& s, const Config& c, const void
     p.ring = c.stages;
     p.status = status;
     cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)((int64_t)c.P_m * c.P_n * c.cluster), 1, 1);
     cfg.blockDim = dim3(kClusterThreads, 1, 1);
     cfg.dynamicSmemBytes = (size_t)cluster_smem_bytes(c.stages);
@@ -437,7 +441,9 @@ inline adapt_status_t launch_cluster(const Shape& s, const Config& c, const void
     attr[1].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = c.cluster > 1 ? 2 : 1;
-    if (cudaLaunchKernelEx(&cfg, cluster_pick(a_kc, b_kc, s.dtype != 0), p) != cudaSuccess) return ADAPT_ERR_CUDA;
+    void* args[1] = {&p};
+    const size_t arg_bytes[1] = {sizeof(p)};
+    if (launch_exc(&cfg, (const void*)cluster_pick(a_kc, b_kc, s.dtype != 0), args, arg_bytes, 1) != cudaSuccess) return ADAPT_ERR_CUDA;
     return ADAPT_OK;
 }
 

@@ -8,6 +8,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <cstring>
 #include <utility>
 
 namespace adapt {
@@ -31,10 +32,71 @@ inline void pdl_attribute(cudaLaunchAttribute* attr)
     attr->val.programmaticStreamSerializationAllowed = pdl_enabled() ? 1 : 0;
 }
 
+// Launch recorder (measurement support): while a thread has one armed, every launch it makes through
+// launch_exc is also written down (configuration, attributes, kernel, a copy of the argument bytes), so that
+// the same launches can be replayed bare and the host cost of a library call be compared with the cost of
+// its launches alone.
+struct LaunchRecord {
+    static constexpr int kMax = 4;
+    static constexpr size_t kArgBytes = 6144;
+    int n = 0;
+    struct One {
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attrs[4];
+        const void* func;
+        int nargs;
+        size_t off[8];
+        alignas(64) unsigned char bytes[kArgBytes];
+    } launch[kMax];
+};
+inline LaunchRecord*& launch_recorder()
+{
+    static thread_local LaunchRecord* r = nullptr;
+    return r;
+}
+
+// Every launch of the library goes through here: cudaLaunchKernelExC with the arguments as an array of
+// pointers (arg_bytes gives their sizes for the recorder).
+inline cudaError_t launch_exc(const cudaLaunchConfig_t* cfg, const void* func, void** args, const size_t* arg_bytes, int nargs)
+{
+    LaunchRecord* rec = launch_recorder();
+    if (rec && rec->n < LaunchRecord::kMax && nargs <= 8 && cfg->numAttrs <= 4) {
+        LaunchRecord::One& o = rec->launch[rec->n];
+        size_t off = 0;
+        bool fits = true;
+        for (int i = 0; i < nargs; ++i) {
+            off = (off + 63) & ~(size_t)63;
+            if (off + arg_bytes[i] > LaunchRecord::kArgBytes) { fits = false; break; }
+            o.off[i] = off;
+            memcpy(o.bytes + off, args[i], arg_bytes[i]);
+            off += arg_bytes[i];
+        }
+        if (fits) {
+            o.cfg = *cfg;
+            for (unsigned i = 0; i < cfg->numAttrs; ++i) o.attrs[i] = cfg->attrs[i];
+            o.cfg.attrs = o.attrs;
+            o.func = func;
+            o.nargs = nargs;
+            ++rec->n;
+        }
+    }
+    return cudaLaunchKernelExC(cfg, func, args);
+}
+
+inline cudaError_t launch_replay(LaunchRecord::One& o, cudaStream_t stream)
+{
+    void* args[8];
+    for (int i = 0; i < o.nargs; ++i) args[i] = o.bytes + o.off[i];
+    o.cfg.stream = stream;
+    o.cfg.attrs = o.attrs;
+    return cudaLaunchKernelExC(&o.cfg, o.func, args);
+}
+
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream, Args&&... args)
 {
     cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = grid;
     cfg.blockDim = block;
     cfg.dynamicSmemBytes = smem;
@@ -43,7 +105,12 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     pdl_attribute(&attr[0]);
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+    // the arguments converted to the kernel's parameter types, then passed by address
+    return [&](KArgs... coerced) {
+        void* argv[] = {(void*)&coerced...};
+        const size_t sizes[] = {sizeof(KArgs)...};
+        return launch_exc(&cfg, (const void*)kernel, argv, sizes, (int)sizeof...(KArgs));
+    }(std::forward<Args>(args)...);
 }
 
 }  // namespace adapt

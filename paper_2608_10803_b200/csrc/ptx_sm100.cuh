@@ -74,7 +74,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // up (abort flag in shared memory); the caller then leaves its loop and falls through to the
 // kernel's common exit.
 constexpr uint64_t kWaitLimitNs = 2000000000ull;   // 2 s: orders of magnitude above any legitimate wait
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint64_t limit_ns)
 {
     if (mbar_try_wait(bar, parity)) return true;
     uint32_t spins = 0;
@@ -84,10 +84,14 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
             if (*abort_flag) return false;
             const uint64_t now = globaltimer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+            else if (now - t0 > limit_ns) { *abort_flag = 1; return false; }
         }
     }
     return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    return mbar_wait_limit(bar, parity, abort_flag, kWaitLimitNs);
 }
 
 // ---- TMA -------------------------------------------------------------------------------------
@@ -210,11 +214,15 @@ __device__ __forceinline__ void umma_commit_1(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// Pair form: arrive on the barrier at this offset in every CTA of `cta_mask`.
-__device__ __forceinline__ void umma_commit_2(uint32_t bar, uint16_t cta_mask)
+// Pair form, issued by the leader (CTA 0 of the pair): arrive on the barrier at this offset in BOTH CTAs once
+// all MMAs issued so far have completed.  Two plain commits, one per barrier address (the leader's own and the
+// peer's, mapped into the cluster window), so every CTA-pair signal in this library is a unicast arrive.
+__device__ __forceinline__ void umma_commit_2(uint32_t bar)
 {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-                 ::"r"(bar), "h"(cta_mask) : "memory");
+    uint32_t peer;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, 1;" : "=r"(peer) : "r"(bar));
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(peer) : "memory");
 }
 
 // 32 lanes x 32 columns of fp32: thread t of the warp receives lane (base lane + t), columns c..c+31.

@@ -444,14 +444,14 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                         }
                         // free the stage (in both CTAs of a pair) once these MMAs have read it
                         if (CG == 1) ptx::umma_commit_1(empty_bar + 8u * stage);
-                        else ptx::umma_commit_2(empty_bar + 8u * stage, 3);
+                        else ptx::umma_commit_2(empty_bar + 8u * stage);
                     }
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
                 if (!ok) break;
                 if (lane == 0) {
                     if (CG == 1) ptx::umma_commit_1(tfull_bar + 8u * buf);
-                    else ptx::umma_commit_2(tfull_bar + 8u * buf, 3);
+                    else ptx::umma_commit_2(tfull_bar + 8u * buf);
                 }
                 ADAPT_TRACE(3, unit);
                 if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }

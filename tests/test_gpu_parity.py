@@ -71,11 +71,11 @@ def test_random_integers_bit_exact(dtype):
 
 # ---- layouts ------------------------------------------------------------------------------------------
 
+@pytest.mark.parametrize("dtype", [ab.F16, ab.BF16])
 @pytest.mark.parametrize("lA,lB", [(ROW, COL), (COL, ROW), (COL, COL)])
 @pytest.mark.parametrize("shape", [(256, 384, 512), (150, 90, 333), (8, 512, 640), (640, 8, 520)])
-def test_layouts_bit_exact(shape, lA, lB):
+def test_layouts_bit_exact(shape, lA, lB, dtype):
     M, N, K = shape
-    dtype = ab.F16
     A = synth.position_coded(M, K, dtype, 7, "cuda")
     B = synth.position_coded(K, N, dtype, 5, "cuda")
     A_st = A.t().contiguous() if lA == COL else A       # column-major storage of A is A^T row-major
@@ -487,3 +487,113 @@ def test_host_entry_point_twice_is_bit_identical_and_orders_the_callers_stream()
     assert torch.equal(C1.view(torch.int16), C2.view(torch.int16))
     err, _, _ = compare_with_oracle(A, B, C1, M, N, K, dtype)
     assert err <= TOL[dtype]
+
+
+# ---- plan-cache key beyond the packed range; tensor-map cache; the bounded-wait path ----------------------
+
+@pytest.mark.parametrize("shape", [((1 << 20) + 3, 8, 24), (16, (1 << 20) + 8, 40), (9, 24, (1 << 20) + 5)])
+def test_dimension_beyond_the_packed_shape_key(shape):
+    """A dimension of 2^20 or more does not fit the packed 64-bit shape word: the plan comes from the slow-path
+    table, is still cached (same handle) and runs like any other."""
+    M, N, K = shape
+    dtype = ab.BF16
+    init()
+    h1 = ab.adapt_matmul_plan(M, N, K, dtype)
+    h2 = ab.adapt_matmul_plan(M, N, K, dtype)
+    assert h1 == h2
+    A = synth.draw_operand(M, K, ("integer", -3, 3), 31, dtype, "cuda")
+    B = synth.draw_operand(K, N, ("integer", -3, 3), 32, dtype, "cuda")
+    check_case(M, N, K, dtype, A, B, plan=h1, exact=True, mac_budget=2e9)
+
+
+def test_tensor_map_cache_keeps_geometries_apart():
+    """One plan can reach the same workspace address with two tile geometries: a k-class plan (B read in place
+    through per-class views, A regrouped into the workspace) falls back to re-pitched copies when B's pointer
+    is not 16-byte aligned, and with a column-major A the two layouts of the workspace copy of A can share
+    base pointer and pitch.  The cache must not hand the map of one to the other, in either order."""
+    M, K, N = 510, 260, 1003                 # padded_pitch(M) = 512 = 8 * Kc with Kc = 64 ... checked below
+    dtype = ab.F16
+    init()
+    cands = [c for c in ab.adapt_plan_candidates(M, N, K, dtype, COL, ROW) if c.srcB == 3]
+    assert cands, "expected a k-class configuration for this shape"
+    A = synth.position_coded(M, K, dtype, 7, "cuda")
+    B = synth.position_coded(K, N, dtype, 5, "cuda")
+    A_st = A.t().contiguous()
+    bufB = torch.zeros(K * N + 8, dtype=torch.float16, device="cuda")
+    B_off = bufB[1:1 + K * N].view(K, N)
+    B_off.copy_(B)
+    for c in cands[:3]:
+        plan = ab.adapt_matmul_plan_forced(M, N, K, dtype, COL, ROW, c.tiling_key)
+        for order in ((B, B_off, B), (B_off, B, B_off)):
+            for Bx in order:
+                C = run_library(A_st, Bx, M, N, K, dtype, COL, ROW, plan=plan)
+                torch.cuda.synchronize()
+                ab.adapt_poll_device_status(torch.cuda.current_stream().cuda_stream)
+                err, mism, n = compare_with_oracle(A_st, Bx, C, M, N, K, dtype, COL, ROW)
+                assert mism == 0, (c.BN, c.P_k, mism)
+
+
+def test_tensor_map_cache_hits_after_the_first_call_and_holds_eight_pointer_sets():
+    init()
+    M, N, K, dtype = 512, 512, 512, ab.BF16
+    plan = ab.adapt_matmul_plan(M, N, K, dtype)
+    st = torch.cuda.current_stream().cuda_stream
+    sets = [(synth.draw_operand(M, K, synth.U11, 40 + i, dtype, "cuda"), synth.draw_operand(K, N, synth.U11, 60 + i, dtype, "cuda"),
+             torch.empty((M, N), dtype=torch.bfloat16, device="cuda")) for i in range(8)]
+    for a, b, c in sets:
+        ab.adapt_matmul(plan, a.data_ptr(), b.data_ptr(), c.data_ptr(), st)
+    before = ab.adapt_map_encode_count()
+    for _ in range(3):
+        for a, b, c in sets:
+            ab.adapt_matmul(plan, a.data_ptr(), b.data_ptr(), c.data_ptr(), st)
+    torch.cuda.synchronize()
+    assert ab.adapt_map_encode_count() == before, "a rotation over eight pointer sets must not encode a tensor map"
+    ref = sets[0][2].clone()
+    ab.adapt_set_map_cache(False)
+    try:
+        ab.adapt_matmul(plan, sets[0][0].data_ptr(), sets[0][1].data_ptr(), sets[0][2].data_ptr(), st)
+        torch.cuda.synchronize()
+        assert ab.adapt_map_encode_count() > before
+    finally:
+        ab.adapt_set_map_cache(True)
+    assert torch.equal(ref.view(torch.int16), sets[0][2].view(torch.int16))
+
+
+def test_bounded_wait_expires_and_reports_a_timeout():
+    """A wait on a barrier nobody arrives on gives up after its limit: the kernel ends normally, the status word
+    is set, the poll reports ADAPT_ERR_TIMEOUT once, and the library keeps working afterwards."""
+    init()
+    st = torch.cuda.current_stream().cuda_stream
+    ab.adapt_poll_device_status(st)                       # clean to begin with
+    ab.adapt_selftest_wait_expiry(1_000_000, st)          # 1 ms
+    with pytest.raises(ab.AdaptError) as e:
+        ab.adapt_poll_device_status(st)
+    assert e.value.status == ab.ERR_TIMEOUT
+    ab.adapt_poll_device_status(st)                       # the word was cleared by the failing poll
+    M, N, K, dtype = 256, 256, 256, ab.F16
+    A = synth.position_coded(M, K, dtype, 7, "cuda")
+    B = synth.position_coded(K, N, dtype, 5, "cuda")
+    check_case(M, N, K, dtype, A, B, exact=True)
+
+
+def test_batched_entry_point_matches_single_calls():
+    init()
+    st = torch.cuda.current_stream().cuda_stream
+    shapes = [(131, 77, 259, ab.BF16), (512, 512, 2048, ab.BF16), (8, 3001, 400, ab.F16), (1, 1, 1, ab.F16), (300, 520, 12, ab.F16)]
+    plans, As, Bs, C1, C2 = [], [], [], [], []
+    for i, (M, N, K, dt) in enumerate(shapes):
+        plans.append(ab.adapt_matmul_plan(M, N, K, dt))
+        As.append(synth.draw_operand(M, K, synth.U11, 70 + i, dt, "cuda"))
+        Bs.append(synth.draw_operand(K, N, synth.U11, 90 + i, dt, "cuda"))
+        C1.append(torch.full((M, N), float("nan"), dtype=As[-1].dtype, device="cuda"))
+        C2.append(torch.full((M, N), float("nan"), dtype=As[-1].dtype, device="cuda"))
+        ab.adapt_matmul(plans[-1], As[-1].data_ptr(), Bs[-1].data_ptr(), C1[-1].data_ptr(), st)
+    ab.adapt_matmul_batch(plans, [a.data_ptr() for a in As], [b.data_ptr() for b in Bs], [c.data_ptr() for c in C2], st)
+    ab.adapt_matmul_repeat(plans[0], [As[0].data_ptr()] * 2, [Bs[0].data_ptr()] * 2, [C2[0].data_ptr()] * 2, 3, st)
+    torch.cuda.synchronize()
+    ab.adapt_poll_device_status(st)
+    for a, b in zip(C1, C2):
+        assert torch.equal(a.view(torch.int16), b.view(torch.int16))
+    (M, N, K, dt) = shapes[1]
+    err, mism, n = compare_with_oracle(As[1], Bs[1], C2[1], M, N, K, dt)
+    assert err <= TOL[dt]
