@@ -288,23 +288,34 @@ def ours(args):
         slots.append(s)
 
     lib = ab.load()
-    mm = lib.adapt_matmul
+    # Pointer policy, the same in the headline pass and in the per-shape pass: every shape owns up to eight
+    # operand sets (enough to exceed L2 twice over) and consecutive calls of a shape rotate through them.  The
+    # library keeps the tensor-map encodings of the eight most recent pointer sets per plan, so after the
+    # warm-up passes no call encodes a map (checked below through adapt_map_encode_count); what a call with
+    # never-seen pointers pays is measured separately (dispatch_cost: host_us_call_map_miss).
+    n_rot = max(len(s) for s in slots)
+    plan_arr = ab.pointer_array(plans)
+    rot = []
+    for r in range(n_rot):
+        rot.append(tuple(ab.pointer_array([s[r % len(s)][j] for s in slots]) for j in range(3)))
+    pass_no = [0]
 
     def one_pass():
-        for h, s in zip(plans, slots):
-            a, b, c_ = s[0][:3]
-            st = mm(h, a, b, c_, stream)
-            if st != 0:
-                raise RuntimeError(f"adapt_matmul failed: {lib.adapt_last_error_message().decode()}")
+        a, b, c_ = rot[pass_no[0] % n_rot]
+        pass_no[0] += 1
+        st = lib.adapt_matmul_batch(len(plans), plan_arr, a, b, c_, stream)
+        if st != 0:
+            raise RuntimeError(f"adapt_matmul failed: {lib.adapt_last_error_message().decode()}")
 
     def barrier():
         if dist is not None:
             dist.barrier()
 
-    for _ in range(max(3, args.warmup)):
+    for _ in range(max(3, args.warmup, n_rot)):
         one_pass()
     torch.cuda.synchronize()
     ab.adapt_poll_device_status(stream)
+    encodes0 = ab.adapt_map_encode_count()
 
     sampler = ClockSampler(local)
     sampler.start()
@@ -335,20 +346,46 @@ def ours(args):
         for info, c in zip(infos, cases):
             reps.append(int(min(20, max(1, 60.0 / max(info.predicted_us, 1.0)))))
         passes = []
+        sets = [tuple(ab.pointer_array([x[j] for x in s]) for j in range(3)) for s in slots]
         for _ in range(args.shape_passes):
             evs = []
-            for h, s, r in zip(plans, slots, reps):
+            for h, s, st3, r in zip(plans, slots, sets, reps):
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
-                for j in range(r):
-                    a, b, c_ = s[j % len(s)][:3]
-                    mm(h, a, b, c_, stream)
+                lib.adapt_matmul_repeat(h, len(s), st3[0], st3[1], st3[2], r, stream)
                 e1.record()
                 evs.append((e0, e1))
             torch.cuda.synchronize()
             passes.append([e0.elapsed_time(e1) * 1e-3 / r for (e0, e1), r in zip(evs, reps)])
         per_shape = [statistics.median(p[i] for p in passes) for i in range(len(cases))]
     ab.adapt_poll_device_status(stream)
+    map_encodes_timed = ab.adapt_map_encode_count() - encodes0
+
+    # ---- the launch floor and the host cost of the online call (timed inside the library, in C) ----
+    floor = None
+    dispatch = None
+    if rank == 0 and not args.no_dispatch:
+        h_pdl, d_pdl = ab.adapt_measure_empty_launch(20000, True, stream)
+        h_np, d_np = ab.adapt_measure_empty_launch(20000, False, stream)
+        floor = {"empty_kernel_us_pdl": d_pdl, "empty_kernel_us_no_pdl": d_np, "host_us_per_launch_pdl": h_pdl,
+                 "host_us_per_launch_no_pdl": h_np,
+                 "how": "20,000 empty kernels back to back on the stream in batches of 128, CUDA events around each batch (device) and steady_clock around the launches (host)"}
+        dispatch = {}
+        seen_kinds = {}
+        for i, (c, info) in enumerate(zip(cases, infos)):
+            kind = kernel_variant(ab, info) + ("+reduce" if info.P_k > 1 and info.family != ab.FAM_CLUSTER else "")
+            if kind in seen_kinds or c.bytes > 64e6:
+                continue
+            seen_kinds[kind] = i
+        want = ["umma_1cta/plain_tiles", "umma_1cta/halo_class_tiles", "umma_1cta/row_class_tiles", "cluster", "simt",
+                "umma_1cta/plain_tiles+reduce", "umma_1cta/k_classes_as_splits+reduce"]
+        for kind in want:
+            if kind not in seen_kinds:
+                continue
+            i = seen_kinds[kind]
+            a, b, c_ = slots[i][0][:3]
+            dc = ab.adapt_measure_dispatch(plans[i], a, b, c_, stream, 20000 if cases[i].bytes < 4e6 else 2000)
+            dispatch[kind] = dict(dc.as_dict(), shape=[cases[i].M, cases[i].N, cases[i].K])
 
     # ---- vendor-library reference (context, not the product): torch.matmul on the same buffers ----
     vendor = None
@@ -386,7 +423,13 @@ def ours(args):
                    "timing": "CUDA events on the launching stream around K passes; per-shape: events around R back-to-back calls with rotated buffers, median of passes"},
         "clocks": clocks, "gpu_launches": int(launches), "host_wall_ms_per_step": wall / args.steps * 1e3,
         "plan_ms_cold_total": plan_ms,
+        "pointer_policy": {"operand_sets_per_shape_max": n_rot, "map_cache_slots_per_plan": 8,
+                           "tensor_maps_encoded_in_timed_regions": int(map_encodes_timed),
+                           "note": "headline pass p uses set p mod n of every shape, the per-shape pass rotates the same sets; all sets fit the per-plan tensor-map cache, so no timed call encodes a map; the cost of a miss is in dispatch_cost"},
     }
+    if floor is not None:
+        line["launch_floor"] = floor
+        line["dispatch_cost"] = dispatch
 
     if rank == 0 and per_shape is not None:
         fr_nom, fr_meas, tf = [], [], []
@@ -415,7 +458,30 @@ def ours(args):
                                         "geomean_time_ratio_vendor_over_ours": geomean(sp),
                                         "geomean_time_ratio_troof_ge_20us": geomean(bigsp),
                                         "sum_vendor_time_ms": sum(vendor) * 1e3, "sum_our_time_ms": sum(per_shape) * 1e3}
+        # the same fractions against roofline time + the launch floor (what a perfect kernel behind one launch
+        # would reach), and by bucket of nominal roofline time
+        floor_us = floor["empty_kernel_us_pdl"] if floor else None
+        buckets = []
+        edges = [0.0, 0.1e-6, 1e-6, 5e-6, 20e-6, 100e-6, float("inf")]
+        for lo, hi in zip(edges[:-1], edges[1:]):
+            idx = [i for i, c in enumerate(cases) if lo <= t_roof_nominal(c) < hi]
+            if not idx:
+                continue
+            b = {"t_roof_us": [lo * 1e6, hi * 1e6 if hi != float("inf") else None], "shapes": len(idx),
+                 "median_call_us": statistics.median(per_shape[i] for i in idx) * 1e6,
+                 "geomean_frac_nominal": geomean([fr_nom[i] for i in idx]),
+                 "sum_call_ms": sum(per_shape[i] for i in idx) * 1e3}
+            if floor_us is not None:
+                b["geomean_frac_vs_troof_plus_launch"] = geomean([(t_roof_nominal(cases[i]) + floor_us * 1e-6) / per_shape[i] for i in idx])
+            if vendor is not None:
+                b["geomean_time_ratio_vendor_over_ours"] = geomean([vendor[i] / per_shape[i] for i in idx])
+            buckets.append(b)
         line["sweep"] = {
+            "roofline_frac_geomean_vs_troof_plus_launch":
+                geomean([(t_roof_nominal(c) + floor_us * 1e-6) / t for c, t in zip(cases, per_shape)]) if floor_us is not None else None,
+            "roofline_frac_geomean_if_every_call_took_troof_plus_launch":
+                geomean([t_roof_nominal(c) / (t_roof_nominal(c) + floor_us * 1e-6) for c in cases]) if floor_us is not None else None,
+            "by_t_roof_bucket": buckets,
             "roofline_frac_geomean_nominal": geomean(fr_nom),
             "roofline_frac_geomean_measured_peaks": geomean(fr_meas),
             "roofline_frac_geomean_troof_ge_20us": geomean(big), "shapes_troof_ge_20us": len(big),
@@ -668,6 +734,7 @@ def main():
     ap.add_argument("--limit", type=int, default=0)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--no-dispatch", action="store_true", help="skip the launch-floor and dispatch-cost measurements")
     ap.add_argument("--dump", default="", help="write the per-shape table to this CSV")
     ap.add_argument("--vendor", action="store_true", help="also time torch.matmul (cuBLAS) per shape as a vendor reference")
     ap.add_argument("--validate-model", type=int, default=0,

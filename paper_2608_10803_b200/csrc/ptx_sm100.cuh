@@ -94,6 +94,52 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return mbar_wait_limit(bar, parity, abort_flag, kWaitLimitNs);
 }
 
+// The same wait with cluster-scope acquire: for barriers that CTAs of the cluster arrive on after writing
+// shared memory this CTA is about to read through the cluster window (and the reverse hand-back).
+__device__ __forceinline__ bool mbar_try_wait_cluster(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint32_t bar, uint32_t parity, volatile int* abort_flag)
+{
+    if (mbar_try_wait_cluster(bar, parity)) return true;
+    uint32_t spins = 0;
+    uint64_t t0 = 0;
+    while (!mbar_try_wait_cluster(bar, parity)) {
+        if ((++spins & 0xff) == 0) {
+            if (*abort_flag) return false;
+            const uint64_t now = globaltimer_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+        }
+    }
+    return true;
+}
+// 16 bytes from the shared memory of CTA `rank` of this cluster, at the offset of `local_addr` in this CTA.
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t local_addr, uint32_t rank)
+{
+    uint32_t remote;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(local_addr), "r"(rank));
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(remote) : "memory");
+    return v;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 // ---- TMA -------------------------------------------------------------------------------------
 // 2D tiled load into this CTA's shared memory; x is the innermost coordinate (elements) and
 // must make x * element size a multiple of 16 bytes.  Completion is counted in bytes on `bar`.
