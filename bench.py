@@ -35,6 +35,9 @@ NCU_TRAFFIC_RATIO = {
     "umma_1cta/halo_class_tiles": 0.93,      # 20000 x 20001 x 12: 746.9 / 801.0 MB (part of C still in L2 at kernel end)
     "umma_1cta/row_class_tiles": 1.02,       # 20000 x 8 x 60001: 2445.2 / 2401.3 MB
     "umma_1cta/k_classes_as_splits": 1.04,   # 8 x 30001 x 8000: 497.6 / 480.6 MB
+    "umma_1cta/k_classes_as_splits+fused_reduce": 1.04,
+    "umma_1cta/row_class_tiles+fused_reduce": 1.02,
+    "umma_1cta/plain_tiles+fused_reduce": 1.01,
     "umma_2cta/k_classes_as_splits": 1.04,
     "umma_1cta/plain_tiles": 1.01,           # 16 x 65536 x 4096: 546.8 / 539.1 MB
     "umma_2cta/plain_tiles": 0.87,           # 4096^3: 87.9 / 100.7 MB
@@ -52,7 +55,7 @@ def kernel_variant(ab, info):
         mode = "halo_class_tiles" if info.BN % 64 else "row_class_tiles"
     else:
         mode = "plain_tiles"
-    return f"{fam}/{mode}"
+    return f"{fam}/{mode}" + ("+fused_reduce" if info.fused else "")
 
 
 def max_over_ranks(x, dist, device):
@@ -373,12 +376,13 @@ def ours(args):
         dispatch = {}
         seen_kinds = {}
         for i, (c, info) in enumerate(zip(cases, infos)):
-            kind = kernel_variant(ab, info) + ("+reduce" if info.P_k > 1 and info.family != ab.FAM_CLUSTER else "")
+            kind = kernel_variant(ab, info) + ("+reduce" if info.P_k > 1 and info.family != ab.FAM_CLUSTER and not info.fused else "")
             if kind in seen_kinds or c.bytes > 64e6:
                 continue
             seen_kinds[kind] = i
         want = ["umma_1cta/plain_tiles", "umma_1cta/halo_class_tiles", "umma_1cta/row_class_tiles", "cluster", "simt",
-                "umma_1cta/plain_tiles+reduce", "umma_1cta/k_classes_as_splits+reduce"]
+                "umma_1cta/plain_tiles+reduce", "umma_1cta/k_classes_as_splits+reduce", "umma_1cta/plain_tiles+fused_reduce",
+                "umma_1cta/k_classes_as_splits+fused_reduce", "umma_1cta/row_class_tiles+fused_reduce"]
         for kind in want:
             if kind not in seen_kinds:
                 continue
@@ -514,11 +518,11 @@ def ours(args):
         if args.dump:
             os.makedirs(os.path.dirname(os.path.abspath(args.dump)), exist_ok=True)
             with open(args.dump, "w") as f:
-                f.write("index,M,N,K,dtype,family,class,BM,BN,stages,P_k,srcA,srcB,pred_us,time_us,tflops,frac_nominal,t_roof_us,vendor_us\n")
+                f.write("index,M,N,K,dtype,family,class,BM,BN,stages,P_k,fused,srcA,srcB,pred_us,time_us,tflops,frac_nominal,t_roof_us,vendor_us\n")
                 for i, (c, info, t) in enumerate(zip(cases, infos, per_shape)):
                     vu = f"{vendor[i] * 1e6:.3f}" if vendor is not None else ""
                     f.write(f"{i},{c.M},{c.N},{c.K},{c.dtype},{ab.FAMILY_NAMES[info.family]},{info.taxonomy_class},{info.BM},{info.BN},"
-                            f"{info.stages},{info.P_k},{info.srcA},{info.srcB},{info.predicted_us:.3f},{t * 1e6:.3f},"
+                            f"{info.stages},{info.P_k},{info.fused},{info.srcA},{info.srcB},{info.predicted_us:.3f},{t * 1e6:.3f},"
                             f"{c.flops / t / 1e12:.4f},{t_roof_nominal(c) / t:.5f},{t_roof_nominal(c) * 1e6:.4f},{vu}\n")
 
     # ---- dispatch overhead of a cached plan (host clock, C call through ctypes) ----
@@ -629,6 +633,8 @@ def one_shape(args):
             cands = [c for c in cands if c.stages == args.stages]
         if args.src:
             cands = [c for c in cands if f"{c.srcA}{c.srcB}" == args.src]
+        if args.fused >= 0:
+            cands = [c for c in cands if c.fused == args.fused]
         plan = ab.adapt_matmul_plan_forced(M, N, K, dt, 0, 0, cands[0].tiling_key)
     else:
         plan = ab.adapt_matmul_plan(M, N, K, dt)
@@ -646,7 +652,7 @@ def one_shape(args):
     t = e0.elapsed_time(e1) / args.reps * 1e-3
     byts = 2.0 * (M * K + K * N + M * N)
     line = (f"{M}x{N}x{K} dt{dt} {ab.FAMILY_NAMES[info.family]} {info.BM}x{info.BN} st{info.stages} P_k{info.P_k} "
-            f"src{info.srcA}{info.srcB}: {t * 1e6:.1f} us  {2.0 * M * N * K / t / 1e12:.1f} TFLOP/s  {byts / t / 1e9:.0f} GB/s  "
+            f"src{info.srcA}{info.srcB}{' fused' if info.fused else ''}: {t * 1e6:.1f} us  {2.0 * M * N * K / t / 1e12:.1f} TFLOP/s  {byts / t / 1e9:.0f} GB/s  "
             f"predicted {info.predicted_us:.1f} us")
     if args.cublas:
         torch.matmul(A, B, out=C)
@@ -749,6 +755,7 @@ def main():
     ap.add_argument("--pk", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--src", type=str, default="", help="with --family: operand sources as two digits, e.g. 13 = A copied, B through k-class views")
+    ap.add_argument("--fused", type=int, default=-1, help="with --family: 1 = only fused split-K configurations, 0 = only unfused")
     ap.add_argument("--cublas", action="store_true", help="with --shape: also time torch.matmul as the vendor reference")
     args = ap.parse_args()
     if args.shape:

@@ -105,7 +105,9 @@ typedef struct adapt_plan_info_s {
     int32_t cluster;          /* CTAs per cluster (2 for the 2-CTA family) */
     int32_t srcA, srcB;       /* adapt_source_t */
     int32_t grid;             /* CTAs launched by the main kernel */
-    int32_t reserved;
+    int32_t fused;            /* 1: tcgen05 split-K whose P_k splits are the CTAs of one thread-block cluster and whose
+                                 partial tiles are added through distributed shared memory inside the GEMM launch
+                                 (no workspace, no reduction launch); 0 otherwise */
     int64_t workspace_bytes;  /* pad copies + split-K partials */
     double flops;             /* 2*M*N*K */
     double hbm_bytes;         /* modelled HBM traffic including workspace traffic */
@@ -119,7 +121,7 @@ typedef struct adapt_plan_info_s {
  * library's): [63:62] taxonomy class, [61:59] family, [58:54] BM/16, [53:48] BN/16,
  * [47:46] log2(BK/16), [45:42] stages, [41:32] P_k, [31] persistent tile loop,
  * [30:29] srcA, [28:27] srcB, [26] dtype, [25] layoutA, [24] layoutB, [23:22] log2(cluster) mod 4,
- * [21] log2(cluster) / 4, [20:0] zero. */
+ * [21] log2(cluster) / 4, [20] fused in-cluster split-K reduction, [19:0] zero. */
 
 /* Select the device (cudaSetDevice), query it, and create the library state for
  * it.  Idempotent.  Needed before adapt_matmul; planning works without it (the

@@ -398,8 +398,38 @@ static UmmaKernel umma_lookup(int BN, bool a_mn, bool b_mn)
     return nullptr;
 }
 
-static UmmaKernel launch_map_umma(int family, int BN, bool a_mn, bool b_mn, int mode = 0)
+// fused split-K instantiations (1-CTA tiles; the k splits of a tile are one cluster)
+static UmmaKernel umma_lookup_fused(int BN, bool a_mn, bool b_mn)
 {
+#define ADAPT_PICK(bn)                                                                         \
+    if (BN == bn) {                                                                            \
+        if (!a_mn && !b_mn) return (const void*)umma_gemm_kernel<bn, false, false, 1, 0, true>; \
+        if (!a_mn && b_mn) return (const void*)umma_gemm_kernel<bn, false, true, 1, 0, true>;   \
+        if (a_mn && !b_mn) return (const void*)umma_gemm_kernel<bn, true, false, 1, 0, true>;   \
+        return (const void*)umma_gemm_kernel<bn, true, true, 1, 0, true>;                       \
+    }
+    ADAPT_PICK(64)
+    ADAPT_PICK(128)
+    ADAPT_PICK(256)
+#undef ADAPT_PICK
+    return nullptr;
+}
+
+static UmmaKernel launch_map_umma(int family, int BN, bool a_mn, bool b_mn, int mode = 0, bool fused = false)
+{
+    if (fused) {
+        if (family != ADAPT_FAM_UMMA_1CTA) return nullptr;
+        if (mode == 0) return umma_lookup_fused(BN, a_mn, b_mn);
+        if (mode == 1) {
+            if (BN == 64) return (const void*)umma_gemm_kernel<64, false, true, 1, 1, true>;
+            if (BN == 128) return (const void*)umma_gemm_kernel<128, false, true, 1, 1, true>;
+            if (BN == 256) return (const void*)umma_gemm_kernel<256, false, true, 1, 1, true>;
+            return nullptr;
+        }
+        if (BN == 128) return (const void*)umma_gemm_kernel<128, false, true, 1, 3, true>;
+        if (BN == 256) return (const void*)umma_gemm_kernel<256, false, true, 1, 3, true>;
+        return nullptr;
+    }
     if (mode == 1) {                     // row-major A read through per-row-class maps (1-CTA tiles, row-major B)
         if (BN == 64) return (const void*)umma_gemm_kernel<64, false, true, 1, 1>;
         if (BN == 128) return (const void*)umma_gemm_kernel<128, false, true, 1, 1>;
@@ -467,6 +497,37 @@ extern "C" adapt_status_t adapt_init(int device)
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
     CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_2CTA, 256, false, true, 2),
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
+    for (int BN : {64, 128, 256}) {
+        for (int a = 0; a < 2; ++a)
+            for (int b = 0; b < 2; ++b)
+                CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_1CTA, BN, a != 0, b != 0, 0, true),
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
+        CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_1CTA, BN, false, true, 1, true),
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
+        if (BN != 64)
+            CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_1CTA, BN, false, true, 2, true),
+                                          cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
+    }
+    // clusters of 2, 4, 8 CTAs of the tcgen05 kernel (one CTA per SM) that the device runs at a time
+    for (int i = 0; i < 3; ++i) {
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        const int cs = 2 << i;
+        cfg.gridDim = dim3((unsigned)(cs * S.machine.n_sm), 1, 1);
+        cfg.blockDim = dim3(kUmmaThreads, 1, 1);
+        cfg.dynamicSmemBytes = (size_t)160 * 1024;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)cs;
+        attr[0].val.clusterDim.y = 1;
+        attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, launch_map_umma(ADAPT_FAM_UMMA_1CTA, 128, false, true, 0, true), &cfg) == cudaSuccess && n >= 1)
+            S.machine.umma_clusters[i] = n;
+        (void)cudaGetLastError();
+    }
     CUDA_TRY(cluster_set_attributes());
     S.machine.max_cluster = cluster_max_size();
     S.device = device;
@@ -741,7 +802,9 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     }
     p.num_units = p.P_m * p.P_n * p.P_k;
 
-    const size_t szP = p.P_k > 1 ? (size_t)round_up((int64_t)p.P_k * s.M * partial_pitch(s.N) * 4, 256) : 0;
+    // the plan's fused reduction stands unless a fallback changed the tiling (then: partials in the workspace)
+    const bool fused = c.fused != 0 && p.P_k == c.P_k && !(c.srcB == ADAPT_SRC_TMA_CLASSES && !kclsB);
+    const size_t szP = (p.P_k > 1 && !fused) ? (size_t)round_up((int64_t)p.P_k * s.M * partial_pitch(s.N) * 4, 256) : 0;
     void* ws = nullptr;
     adapt_status_t r = get_workspace(S, stream, szA + szB + szP, &ws);
     if (r != ADAPT_OK) return r;
@@ -769,7 +832,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
         if ((r = launch_pad(S, B, w8 + szA, outB, inB, pitchB, stream)) != ADAPT_OK) return r;
         b_src = w8 + szA;
     }
-    float* partial = p.P_k > 1 ? (float*)(w8 + szA + szB) : nullptr;
+    float* partial = (p.P_k > 1 && !fused) ? (float*)(w8 + szA + szB) : nullptr;
 
     // K-major operand: one box of 64 k x (rows this CTA owns); MN-major operand: boxes of 64 x 64
     if (classesA) {
@@ -815,7 +878,10 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.dtype = s.dtype;
     // the plan's ring depth assumed its own A box; a fallback to copies may need a shallower ring
     p.stages = c.stages;
-    while (p.stages > 2 && umma_smem_bytes(c.BN, cg, p.stages, a_box_rows, p.P_k == 1) > S.machine.smem_bytes) --p.stages;
+    const int fused_bytes = fused ? umma_fused_bytes(c.BN, a_box_rows) : 0;
+    p.x_rows = a_box_rows;
+    p.x_pitch = umma_fused_pitch(c.BN);
+    while (p.stages > 2 && umma_smem_bytes(c.BN, cg, p.stages, a_box_rows, p.P_k == 1, fused_bytes) > S.machine.smem_bytes) --p.stages;
     p.a_tx_bytes = a_box_rows * kUmmaBK * 2;
     p.idesc = umma_idesc(s.dtype, a_mn, b_mn, 128 * cg, c.BN);
     p.C = C;
@@ -827,19 +893,20 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.trace = S.d_trace;
 #endif
 
-    UmmaKernel k = launch_map_umma(c.family, c.BN, a_mn, b_mn, classesA ? 1 : (kclsB ? 2 : 0));
+    UmmaKernel k = launch_map_umma(c.family, c.BN, a_mn, b_mn, classesA ? 1 : (kclsB ? 2 : 0), fused);
     if (!k) return fail(ADAPT_ERR_UNSUPPORTED, "no compiled kernel for this tiling key%s");
-    const int slots = S.machine.n_sm / cg;
-    const int grid = std::min(p.num_units, slots) * cg;
+    const int slots = fused ? umma_cluster_slots(S.machine, p.P_k) : S.machine.n_sm / cg;
+    const int launch_cluster = fused ? p.P_k : cg;            // fused split-K: the splits of a tile are one cluster
+    const int grid = fused ? std::min(p.P_m * p.P_n, slots) * p.P_k : std::min(p.num_units, slots) * cg;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)grid, 1, 1);
     cfg.blockDim = dim3(kUmmaThreads, 1, 1);
-    cfg.dynamicSmemBytes = (size_t)umma_smem_bytes(c.BN, cg, p.stages, a_box_rows, p.P_k == 1);
+    cfg.dynamicSmemBytes = (size_t)umma_smem_bytes(c.BN, cg, p.stages, a_box_rows, p.P_k == 1, fused_bytes);
     cfg.stream = stream;
     cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = (unsigned)cg;
+    attr[0].val.clusterDim.x = (unsigned)launch_cluster;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     pdl_attribute(&attr[1]);
@@ -866,7 +933,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     }
     CUDA_TRY(launch_exc(&cfg, k, args, arg_bytes, 2));
     S.launches.fetch_add(1, std::memory_order_relaxed);
-    if (p.P_k > 1) return launch_reduce(S, partial, C, s.M, s.N, p.P_k, s.dtype, stream);
+    if (p.P_k > 1 && !fused) return launch_reduce(S, partial, C, s.M, s.N, p.P_k, s.dtype, stream);
     return ADAPT_OK;
 }
 

@@ -18,7 +18,14 @@ struct Machine {
     int64_t workspace_limit = (int64_t)24 << 30;
     unsigned family_mask = 0x1Fu;        // bit f set = family f may be selected
     int max_cluster = 16;               // largest thread-block cluster the one-launch kernel may ask for (queried at init)
+    // clusters of 2, 4, 8 CTAs of the tcgen05 kernel (one CTA per SM) the device runs at a time; a cluster sits inside
+    // one GPC, so the larger sizes leave SMs unused (B200: 74, 33, 15; queried at init)
+    int umma_clusters[3] = {74, 33, 15};
 };
+inline int umma_cluster_slots(const Machine& m, int cluster)
+{
+    return cluster == 2 ? m.umma_clusters[0] : cluster == 4 ? m.umma_clusters[1] : cluster == 8 ? m.umma_clusters[2] : m.n_sm;
+}
 
 // ---- calibration constants of the latency model (Eq. 8: lambda_r, eta_r, BW_r) ------------
 // Measured on B200 with this library's own kernels (CUDA events); the paper's values are for
@@ -64,6 +71,11 @@ struct Calib {
     double cluster_crowd_us = 1.56, cluster_crowd_stage_us = 0.44;   // per CTA per SM beyond one per two SMs
     double cluster_wave_us = 5.5;       // each further round of clusters
     double cluster_bw_eff = 0.35;       // fraction of hbm_bw its 16-byte copies reach when memory-bound
+    double fused_reduce_us = 2.5;       // fused split-K: cluster scheduling, drain to shared memory, two cluster-wide barrier rounds,
+                                        // first remote reads (1 x 4096 x 4096, 128 x 128 tiles, P_k 4: 12.1 us fused, 11.3 us with the reduce launch)
+    double fused_wave_us = 3.5;         // each further round of clusters starts cold (1 x 4096 x 4096, P_k 8: 3 rounds 26 us, 2 rounds 20 us)
+    double reduce_launch_us = 1.5;      // the reduce launch behind the GEMM: programmatic dependent launch hides about half of a launch
+    double dsmem_bw_per_sm = 60e9;      // B/s one SM reads from its peers' shared memory during the fused reduction
     double copy_bw_eff = 0.85;          // pad-copy and reduce kernels
     double hbm_bw_per_sm = 55e9;        // B/s one SM streams from HBM (tail wave of 20000 x 8 x 60001: 15 MB per tile in 0.3 ms)
     double class_view_sm_eff = 0.85;    // per-SM rate through those views relative to l2_bw_per_sm (20000 x 8 x 60001 tail wave)
@@ -86,6 +98,8 @@ struct Config {
     int stages = 1;
     int P_m = 1, P_n = 1, P_k = 1;
     int cluster = 1;
+    int fused = 0;                      // tcgen05 split-K with the k splits as one thread-block cluster, reduced through
+                                        // distributed shared memory inside the GEMM launch (no partials in global memory)
     int persistent = 0;
     int srcA = ADAPT_SRC_LSU, srcB = ADAPT_SRC_LSU;
     int grid = 1;
@@ -165,10 +179,14 @@ constexpr int kUmmaMaxStages = 15;
 constexpr int kUmmaEpilogueWarps = 8;
 constexpr int kUmmaStageRowBytes = 144;   // 72 16-bit elements: 64 columns + up to 7 of alignment shift
 constexpr int kUmmaWarpStagingBytes = 8192;   // per epilogue warp: two 32 x 128 B boxes for TMA stores, or 32 shifted rows
-inline int umma_smem_bytes(int BN, int cluster, int stages, int a_rows, bool staging)
+// fp32 partial tile a CTA of a fused split-K cluster keeps for the exchange: x_rows rows of BN + 4 elements
+// (the 16 bytes of padding spread the rows of a warp over the banks)
+inline int umma_fused_pitch(int BN) { return BN + 4; }
+inline int umma_fused_bytes(int BN, int x_rows) { return x_rows * umma_fused_pitch(BN) * 4; }
+inline int umma_smem_bytes(int BN, int cluster, int stages, int a_rows, bool staging, int fused_bytes = 0)
 {
     const int stage = a_rows * 64 * 2 + (int)round_up(BN / cluster, 64) * 64 * 2;
-    const int used = stages * stage + kUmmaBarrierBytes + (staging ? kUmmaEpilogueWarps * kUmmaWarpStagingBytes : 0);
+    const int used = stages * stage + kUmmaBarrierBytes + (staging ? kUmmaEpilogueWarps * kUmmaWarpStagingBytes : 0) + fused_bytes;
     // the MMA reads 128 rows of A from every stage, also when the box brought fewer: the rows past the box
     // of the last stage must still lie inside the allocation
     const int read_end = (stages - 1) * stage + 128 * 64 * 2;
@@ -176,10 +194,10 @@ inline int umma_smem_bytes(int BN, int cluster, int stages, int a_rows, bool sta
 }
 // Deepest ring that fits (0 if not even two stages do).  Only a kernel that writes the 16-bit C itself
 // (P_k = 1) needs the epilogue staging; one that writes fp32 partials spends that space on stages.
-inline int umma_deepest_ring(int BN, int cluster, int a_rows, bool staging, int smem_limit, int cap = kUmmaMaxStages)
+inline int umma_deepest_ring(int BN, int cluster, int a_rows, bool staging, int smem_limit, int cap = kUmmaMaxStages, int fused_bytes = 0)
 {
     for (int st = cap; st >= 2; --st)
-        if (umma_smem_bytes(BN, cluster, st, a_rows, staging) <= smem_limit) return st;
+        if (umma_smem_bytes(BN, cluster, st, a_rows, staging, fused_bytes) <= smem_limit) return st;
     return 0;
 }
 

@@ -77,12 +77,13 @@ uint64_t pack_tiling_key(const Shape& s, const Config& c)
     k |= (uint64_t)(s.layoutB & 1) << 24;
     k |= (uint64_t)(ilog2(std::max(c.cluster, 1)) & 3) << 22;
     k |= (uint64_t)((ilog2(std::max(c.cluster, 1)) >> 2) & 1) << 21;
+    k |= (uint64_t)(c.fused & 1) << 20;
     return k;
 }
 
 bool unpack_tiling_key(uint64_t k, Shape* s, Config* c)
 {
-    if (k & ((1ull << 21) - 1)) return false;
+    if (k & ((1ull << 20) - 1)) return false;
     c->cls = (int)((k >> 62) & 3);
     c->family = (int)((k >> 59) & 7);
     c->BM = (int)((k >> 54) & 31) * 16;
@@ -97,6 +98,7 @@ bool unpack_tiling_key(uint64_t k, Shape* s, Config* c)
     s->layoutA = (int)((k >> 25) & 1);
     s->layoutB = (int)((k >> 24) & 1);
     c->cluster = 1 << (int)(((k >> 22) & 3) | (((k >> 21) & 1) << 2));
+    c->fused = (int)((k >> 20) & 1);
     return true;
 }
 
@@ -158,6 +160,13 @@ static void model_epilogue(const Shape& s, Config& c, const Calib& cal)
 {
     c.t_epi_us = 0;
     c.ws_partial = 0;
+    if (c.fused) {
+        // Eq. 11 with the cross-core exchange on chip: each CTA reads one tile's worth of fp32 partials from its
+        // peers' shared memory (its share of the rows over all ranks); no second launch, no workspace
+        // (its time is the tile drain of the main kernel, so nothing is added here)
+        c.hbm_bytes += 2.0 * (double)s.M * (double)s.N;
+        return;
+    }
     if (c.P_k > 1) {
         const double MN = (double)s.M * (double)s.N;
         c.ws_partial = round_up((int64_t)c.P_k * s.M * partial_pitch(s.N) * 4, 256);
@@ -165,7 +174,7 @@ static void model_epilogue(const Shape& s, Config& c, const Calib& cal)
         // partials that fit in L2 are read back at L2 speed; model that as half the HBM cost
         const double factor = part <= kL2Bytes ? 0.5 : 1.0;
         // the reduction kernel walks the P_k slabs eight at a time: one dependent trip to L2 / HBM per batch
-        c.t_epi_us = cal.launch_us + copy_time_us(part * factor + 2.0 * MN, cal) + cal.reduce_batch_us * (double)ceil_div(c.P_k, 8);
+        c.t_epi_us = cal.reduce_launch_us + copy_time_us(part * factor + 2.0 * MN, cal) + cal.reduce_batch_us * (double)ceil_div(c.P_k, 8);
         c.hbm_bytes += part * (1.0 + factor);
     }
 }
@@ -178,10 +187,11 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     const bool ksplit_cls = kclasses && c.BN != 64;                       // each class a k split of its own
     const int64_t L = ksplit_cls ? ceil_div(kblocks, c.P_k / 8)
                                  : ceil_div(kblocks, c.P_k) * (kclasses ? 8 : 1);   // BN = 64: the split's blocks of all 8 classes
-    const int64_t units = (int64_t)c.P_m * c.P_n * c.P_k;
-    const int64_t slots = m.n_sm / c.cluster;
+    // fused split-K: a tile is a cluster of P_k CTAs, and only so many clusters of that size run at a time
+    const int64_t units = c.fused ? (int64_t)c.P_m * c.P_n : (int64_t)c.P_m * c.P_n * c.P_k;
+    const int64_t slots = c.fused ? umma_cluster_slots(m, c.P_k) : m.n_sm / c.cluster;
     const int64_t Q = ceil_div(units, slots);
-    c.grid = (int)(std::min(units, slots) * c.cluster);
+    c.grid = (int)(std::min(units, slots) * (c.fused ? c.P_k : c.cluster));
 
     const double MK = (double)s.M * s.K, KN = (double)s.K * s.N, MN = (double)s.M * s.N;
     // HBM traffic: operands once, plus re-reads of B when it cannot stay in L2 across m-groups.
@@ -222,7 +232,8 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     const double rows_valid = std::min(128.0, (double)s.M / ((double)c.P_m * c.cluster));
     const double out_tile_kb = (c.P_k > 1 ? 4.0 : 2.0) * rows_valid * own_n / 1024.0;
     double t_drain;
-    if (c.P_k > 1) t_drain = cal.epi_partial_fixed_us + cal.epi_partial_us_per_kb * out_tile_kb;
+    if (c.fused) t_drain = cal.fused_reduce_us + 4.0 * rows_valid * c.BN / cal.dsmem_bw_per_sm * 1e6;   // exchange + reduce + store, per tile
+    else if (c.P_k > 1) t_drain = cal.epi_partial_fixed_us + cal.epi_partial_us_per_kb * out_tile_kb;
     else if (s.N % 16 == 0 || halo) t_drain = cal.epi_tile_fixed_us + cal.epi_us_per_kb * out_tile_kb;
     else if (s.N % 8 == 0) t_drain = cal.epi_partial_fixed_us + cal.epi_partial_us_per_kb * out_tile_kb;   // aligned 16-byte stores by the threads
     else t_drain = cal.epi_tile_fixed_unaligned_us + cal.epi_us_per_kb_unaligned * out_tile_kb;
@@ -257,6 +268,7 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
         pipe = tM + (double)Q * t_tile + tP + t_drain;
     }
     pipe += cal.umma_fixed_us;
+    if (c.fused) pipe += cal.fused_wave_us * (double)(Q - 1);
     // halo tiles: the first and the last tile of a row block write the elements before the first and after
     // the last whole 32-byte unit of each row with narrow stores (48618 x 28 x 115: 384 such tiles)
     if (halo && c.P_k == 1)
@@ -399,9 +411,14 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     if (c.BN % 16 != 0 || c.BN > 256) return false;                 // UMMA shape rule for M = 128/256
     if (2 * c.BN > m.tmem_cols) return false;                       // at least two accumulator buffers in TMEM
     if (c.stages < 1 || c.stages > kUmmaMaxStages) return false;
-    c.smem_bytes = umma_smem_bytes(c.BN, c.cluster, c.stages,
-                                   umma_a_box_rows(s, c.cluster, umma_row_classes(c.srcA, c.BN), c.srcB == ADAPT_SRC_TMA_CLASSES),
-                                   c.P_k == 1);
+    const int a_rows_box = umma_a_box_rows(s, c.cluster, umma_row_classes(c.srcA, c.BN), c.srcB == ADAPT_SRC_TMA_CLASSES);
+    if (c.fused) {
+        // the k splits of a tile form one cluster: 1-CTA tiles, a portable cluster size, no halo tiles, not the
+        // eight-accumulator k-class tiles
+        if (c.family != ADAPT_FAM_UMMA_1CTA || (c.P_k != 2 && c.P_k != 4 && c.P_k != 8) || c.BN % 64 != 0) return false;
+        if (c.srcB == ADAPT_SRC_TMA_CLASSES && c.BN == 64) return false;
+    }
+    c.smem_bytes = umma_smem_bytes(c.BN, c.cluster, c.stages, a_rows_box, c.P_k == 1, c.fused ? umma_fused_bytes(c.BN, a_rows_box) : 0);
     if (c.smem_bytes > m.smem_bytes) return false;
     // in class mode the k index of a tile is shifted by up to 7 elements
     // k-class mode splits the blocks of one class; in row-class mode the k index is shifted by up to 7
@@ -585,6 +602,14 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
                     c.stages = st; c.P_k = pk; c.srcA = srcA; c.srcB = srcB;
                     if (st >= 2 && finalize(s, m, cal, c)) out->push_back(c);
                 }
+                // the same split with its reduction fused into the launch (the splits of a tile as one cluster)
+                if (fam == ADAPT_FAM_UMMA_1CTA && (pk == 2 || pk == 4 || pk == 8)) {
+                    Config c;
+                    c.family = fam; c.BM = BM; c.BN = BN; c.BK = 64; c.cluster = cluster; c.fused = 1;
+                    c.stages = umma_deepest_ring(BN, 1, a_rows, false, m.smem_bytes, a_rows == 128 ? 8 : kUmmaMaxStages, umma_fused_bytes(BN, a_rows));
+                    c.P_k = pk; c.srcA = srcA; c.srcB = srcB;
+                    if (c.stages >= 2 && finalize(s, m, cal, c)) out->push_back(c);
+                }
             }
         }
     }
@@ -603,6 +628,13 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
                 d.family = ADAPT_FAM_UMMA_1CTA; d.BM = 128; d.BN = BN; d.BK = 64; d.cluster = 1;
                 d.stages = deepest; d.P_k = pk; d.srcA = ADAPT_SRC_TMA_CLASSES; d.srcB = srcB;
                 if (deepest >= 2 && finalize(s, m, cal, d)) out->push_back(d);
+                if (!halo && (pk == 2 || pk == 4 || pk == 8)) {
+                    const int rows = umma_a_box_rows(s, 1, 8, false);
+                    Config f = d;
+                    f.fused = 1;
+                    f.stages = umma_deepest_ring(BN, 1, rows, false, m.smem_bytes, kUmmaMaxStages, umma_fused_bytes(BN, rows));
+                    if (f.stages >= 2 && finalize(s, m, cal, f)) out->push_back(f);
+                }
             }
         }
     }
@@ -634,6 +666,13 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
                 d.BM = BM; d.BN = BN; d.BK = 64; d.cluster = cluster;
                 d.stages = deepest; d.P_k = 8 * pkk; d.srcA = ADAPT_SRC_PAD_COPY; d.srcB = ADAPT_SRC_TMA_CLASSES;
                 if (deepest >= 2 && 8 * pkk <= 1023 && finalize(s, m, cal, d)) out->push_back(d);
+                if (cluster == 1 && pkk == 1) {                     // the eight classes of a tile as one cluster
+                    const int rows = umma_a_box_rows(s, 1, 0, true);
+                    Config f = d;
+                    f.fused = 1;
+                    f.stages = umma_deepest_ring(BN, 1, rows, false, m.smem_bytes, kUmmaMaxStages, umma_fused_bytes(BN, rows));
+                    if (f.stages >= 2 && finalize(s, m, cal, f)) out->push_back(f);
+                }
             }
         }
     }
@@ -703,7 +742,7 @@ void fill_info(const Shape& s, const Config& c, adapt_plan_info_t* o)
     o->taxonomy_class = c.cls; o->family = c.family;
     o->BM = c.BM; o->BN = c.BN; o->BK = c.BK; o->stages = c.stages;
     o->P_m = c.P_m; o->P_n = c.P_n; o->P_k = c.P_k; o->cluster = c.cluster;
-    o->srcA = c.srcA; o->srcB = c.srcB; o->grid = c.grid; o->reserved = 0;
+    o->srcA = c.srcA; o->srcB = c.srcB; o->grid = c.grid; o->fused = c.fused;
     o->workspace_bytes = c.workspace_bytes;
     o->flops = 2.0 * (double)s.M * (double)s.N * (double)s.K;
     o->hbm_bytes = c.hbm_bytes;

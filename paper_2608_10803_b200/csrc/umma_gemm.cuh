@@ -55,6 +55,8 @@ struct UmmaParams {
     int part_hint;                   // fp32 partials are stored with an evict-last L2 policy (they fit in L2)
     int c_sigma[16];                 // halo class tiles: shift (elements) of C's row class j against its 32-byte aligned base
     int c_extent[16];                // ... and the elements of a shifted row of that class that lie in whole 32-byte units
+    int x_rows, x_pitch;             // fused split-K: rows and row pitch (fp32 elements) of the partial tile each CTA of the
+                                     // cluster keeps in its shared memory for the exchange
     unsigned int* status;            // device status word: bit 0 = a bounded wait expired
     unsigned long long* trace;       // timestamp trace of CTA 0 (diagnostic builds only), else null
 };
@@ -177,10 +179,19 @@ __device__ __forceinline__ void store_run16(unsigned short* dst, int count, cons
 // accumulator of BN columns over the window x' in [(BN-8)*nb, (BN-8)*nb + BN) and writes the BN - 8
 // columns the tile owns as an fp32 partial (read sigma_j columns to the right); the reduction kernel adds
 // the 8 * P_kk slabs in ascending order.  Full-width tiles, at the price of 8 partials per output.
-template <int BN, bool A_MN, bool B_MN, int CG, int MODE>
+//
+// FUSE ("MultiCoreSplitK" in one launch, Eq. 4 / Eq. 11 without the trip through global memory): the P_k splits
+// of a tile are the CTAs of one thread-block cluster (P_k = 2, 4 or 8; rank = split).  Each CTA drains its fp32
+// accumulator into its own shared memory; when all have (mbarrier arrivals across the cluster), the CTAs share
+// the tile's (row, 4-column) groups evenly, and each adds its groups over ranks 0 .. P_k-1 in ascending order
+// through distributed shared memory, rounds once and stores C.  The order is the one splitk_reduce_kernel
+// uses, so a shape gives the same bits with either path and from run to run.
+template <int BN, bool A_MN, bool B_MN, int CG, int MODE, bool FUSE = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams p)
 {
+    static_assert(!FUSE || (CG == 1 && (MODE == 0 || MODE == 1 || MODE == 3)), "the fused reduction: 1-CTA tiles, clusters made of the k splits");
+    static_assert(!FUSE || BN % 64 == 0, "the fused reduction has no halo tiles");
     constexpr bool A_CLS = MODE == 1;
     constexpr bool B_CLS = MODE == 2;
     constexpr bool B_SPLIT = MODE == 3;                   // k classes as k splits (see below)
@@ -222,7 +233,10 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
     volatile uint32_t* tmem_slot_ptr = reinterpret_cast<volatile uint32_t*>(bar_gen + 16 * S + 16 * NBUF);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bar_gen + 16 * S + 16 * NBUF + 4);
     // epilogue staging: one row of 72 16-bit elements (64 columns + up to 7 of shift) per epilogue thread
+    // (fused split-K: the CTA's fp32 partial tile instead)
     uint8_t* stage_out = bar_gen + kUmmaBarrierBytes;
+    // fused split-K: "every rank's partial is in place" / "every rank has read mine", at fixed offsets of the barrier block
+    const uint32_t xfull_bar = bar_base + 512u, xempty_bar = bar_base + 520u;
 
     pdl_launch_dependents();
     if (threadIdx.x == 0) ADAPT_TRACE(11, 0);
@@ -241,6 +255,10 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
             ptx::mbar_init(tfull_bar + 8u * b, 1);         // one tcgen05.commit per phase
             ptx::mbar_init(tempty_bar + 8u * b, kUmmaEpilogueWarps * CG);   // one arrive per epilogue warp of the group
         }
+        if (FUSE) {
+            ptx::mbar_init(xfull_bar, (uint32_t)(kUmmaEpilogueWarps * p.P_k));     // one arrive per epilogue warp of every rank
+            ptx::mbar_init(xempty_bar, (uint32_t)(kUmmaEpilogueWarps * p.P_k));
+        }
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
         ptx::prefetch_tensormap(&maps.a[0]);
@@ -251,7 +269,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
         ptx::tmem_relinquish<CG>();
     }
     ptx::tc_fence_before();
-    if (CG == 2) {
+    if (CG == 2 || FUSE) {      // peers arrive on this CTA's barriers: they must all exist first
         asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
     } else {
         __syncthreads();
@@ -516,7 +534,79 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     if (warp == 2) ADAPT_TRACE(7, unit);
                 }
             };
-            if (p.P_k == 1) {
+            if constexpr (FUSE) {
+                // ---- fused split-K: partial -> own shared memory -> sum over the cluster's ranks -> C ----
+                const uint32_t xphase = (uint32_t)(seq & 1);
+                const uint32_t my_rank = ptx::cluster_ctarank();
+                float* X = reinterpret_cast<float*>(stage_out);
+                // every rank has finished reading the partial this CTA wrote for its previous tile
+                if (!ptx::mbar_wait_cluster(xempty_bar, xphase ^ 1u, abort_flag)) { ok = false; break; }
+                const int r_in_tile = q * 32 + lane;
+                const int sig = B_SPLIT ? p.b_sigma[split & 7] : 0;      // k classes as splits: the tile's columns sit sigma to the right
+#pragma unroll 1
+                for (int c0 = 0; c0 < TILE_N; c0 += 32) {
+                    if (n0 + c0 >= p.N) break;                           // uniform across the warp
+                    if (((seq * ((TILE_N + 31) / 32) + (c0 >> 5)) & 1) != half) continue;
+                    uint32_t r[32];
+                    if (c0 + 32 <= TILE_N) {
+                        ptx::tmem_ld_32x32(t_row + (uint32_t)(sig + c0), r);
+                    } else {                                             // 24 columns (k-class tiles own BN - 8): stay inside the accumulator
+                        uint32_t r8a[8], r8b[8], r8c[8];
+                        ptx::tmem_ld_32x8(t_row + (uint32_t)(sig + c0), r8a);
+                        ptx::tmem_ld_32x8(t_row + (uint32_t)(sig + c0 + 8), r8b);
+                        ptx::tmem_ld_32x8(t_row + (uint32_t)(sig + c0 + 16), r8c);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) { r[i] = r8a[i]; r[8 + i] = r8b[i]; r[16 + i] = r8c[i]; r[24 + i] = 0u; }
+                    }
+                    ptx::tmem_ld_wait();
+                    if (r_in_tile < p.x_rows) {
+                        float4* dst = reinterpret_cast<float4*>(X + (size_t)r_in_tile * p.x_pitch + c0);
+#pragma unroll
+                        for (int v = 0; v < 8; ++v)
+                            dst[v] = make_float4(__uint_as_float(r[4 * v]), __uint_as_float(r[4 * v + 1]),
+                                                 __uint_as_float(r[4 * v + 2]), __uint_as_float(r[4 * v + 3]));
+                    }
+                }
+                release_accumulator();
+                released = true;
+                // this warp's share of the partial is written: tell every rank (release at cluster scope)
+                __syncwarp();
+                if (lane == 0)
+                    for (int rk = 0; rk < p.P_k; ++rk) ptx::mbar_arrive_cluster(xfull_bar, (uint32_t)rk);
+                if (!ptx::mbar_wait_cluster(xfull_bar, xphase, abort_flag)) { ok = false; break; }
+                // rows and 4-column groups of this tile that exist; rank r takes the r-th share of them
+                const int rows_here = A_CLS ? min(128, (p.M - row_base + row_step - 1) / row_step) : min(128, p.M - row_base);
+                const int tile_cols = min(TILE_N, p.N - n0);
+                const int groups = (tile_cols + 3) >> 2;
+                const int total = rows_here * groups;
+                const int per = (total + p.P_k - 1) / p.P_k;
+                const int e_end = min(total, ((int)my_rank + 1) * per);
+                const uint32_t x_addr = ptx::smem_u32(X);
+                unsigned short* c16 = reinterpret_cast<unsigned short*>(p.C);
+                for (int e = (int)my_rank * per + (warp - 2) * 32 + lane; e < e_end; e += kUmmaEpilogueWarps * 32) {
+                    const int rr = e / groups, g = e - rr * groups;
+                    const uint32_t a = x_addr + (uint32_t)((rr * p.x_pitch + 4 * g) * 4);
+                    float4 sum = ptx::ld_cluster_f4(a, 0u);
+                    for (int rk = 1; rk < p.P_k; ++rk) {
+                        const float4 v = ptx::ld_cluster_f4(a, (uint32_t)rk);
+                        sum.x += v.x; sum.y += v.y; sum.z += v.z; sum.w += v.w;
+                    }
+                    const int n = n0 + 4 * g;
+                    unsigned short* dst = c16 + (size_t)(row_base + row_step * rr) * p.N + n;
+                    if (n + 4 <= p.N && (reinterpret_cast<uintptr_t>(dst) & 7) == 0) {
+                        *reinterpret_cast<uint2*>(dst) = make_uint2(pack16(sum.x, sum.y, p.dtype), pack16(sum.z, sum.w, p.dtype));
+                    } else {
+                        const float o[4] = {sum.x, sum.y, sum.z, sum.w};
+#pragma unroll
+                        for (int j = 0; j < 4; ++j)
+                            if (n + j < p.N) dst[j] = cast16(o[j], p.dtype);
+                    }
+                }
+                // done reading every rank's partial: each may overwrite it for its next tile
+                __syncwarp();
+                if (lane == 0)
+                    for (int rk = 0; rk < p.P_k; ++rk) ptx::mbar_arrive_cluster(xempty_bar, (uint32_t)rk);
+            } else if (p.P_k == 1) {
                 // 16-bit output, any N and any base alignment.  A thread converts 64 columns of its row
                 // and stages them in shared memory shifted by the row's misalignment in C, so that
                 // 16-byte aligned chunks of a staged row are 16-byte aligned chunks of C.  The warp then
@@ -796,7 +886,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
 
     // ------------------------------ common exit ----------------------------------------------
     ptx::tc_fence_before();
-    if (CG == 2) {
+    if (CG == 2 || FUSE) {      // no CTA leaves while a peer may still read its shared memory or arrive on its barriers
         asm volatile("barrier.cluster.arrive.release.aligned;\nbarrier.cluster.wait.acquire.aligned;" ::: "memory");
     } else {
         __syncthreads();

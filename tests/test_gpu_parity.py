@@ -597,3 +597,67 @@ def test_batched_entry_point_matches_single_calls():
     (M, N, K, dt) = shapes[1]
     err, mism, n = compare_with_oracle(As[1], Bs[1], C2[1], M, N, K, dt)
     assert err <= TOL[dt]
+
+
+# ---- split-K with the reduction fused into the GEMM launch (the k splits of a tile as one cluster) ----------
+
+def fused_variants(M, N, K, dtype, lA=ROW, lB=ROW):
+    return [(ab.adapt_matmul_plan_forced(M, N, K, dtype, lA, lB, c.tiling_key), c)
+            for c in ab.adapt_plan_candidates(M, N, K, dtype, lA, lB) if c.fused]
+
+
+@pytest.mark.parametrize("dtype", [ab.F16, ab.BF16])
+@pytest.mark.parametrize("shape", [(1, 1024, 4096), (16, 512, 2048), (128, 384, 1024), (200, 264, 1328), (131, 77, 2590),
+                                   (2048, 1024, 512), (8, 3001, 4000), (1030, 264, 1331), (300, 520, 390), (64, 64, 8192)])
+def test_fused_split_k_bit_exact(shape, dtype):
+    """Every fused configuration (cluster sizes 2, 4, 8; plain tiles, row-class tiles, k classes as the cluster's
+    ranks; one tile per cluster and several) against the oracle on position-coded integers."""
+    M, N, K = shape
+    A = synth.position_coded(M, K, dtype, modulus=7, device="cuda")
+    B = synth.position_coded(K, N, dtype, modulus=5, device="cuda").contiguous()
+    variants = fused_variants(M, N, K, dtype)
+    assert variants, "expected fused configurations for this shape"
+    seen = set()
+    for plan, c in variants:
+        check_case(M, N, K, dtype, A, B, plan=plan, exact=True)
+        seen.add(c.P_k)
+    assert seen & {2, 4, 8}
+
+
+@pytest.mark.parametrize("lA,lB", [(ROW, COL), (COL, ROW), (COL, COL)])
+def test_fused_split_k_layouts(lA, lB):
+    M, N, K = 136, 256, 2048
+    for dtype in (ab.F16, ab.BF16):
+        A = synth.position_coded(M, K, dtype, 7, "cuda")
+        B = synth.position_coded(K, N, dtype, 5, "cuda")
+        A_st = A.t().contiguous() if lA == COL else A
+        B_st = B.t().contiguous() if lB == COL else B
+        variants = fused_variants(M, N, K, dtype, lA, lB)
+        assert variants
+        for plan, c in variants:
+            check_case(M, N, K, dtype, A_st, B_st, lA, lB, plan=plan, exact=True)
+
+
+def test_fused_split_k_matches_the_two_launch_path_bit_for_bit_on_random_values():
+    """Same split count, same ascending order of the additions: the fused reduction and the workspace reduction
+    give the same bits, and the fused one is the same from run to run."""
+    for (M, N, K, dtype) in [(16, 4096, 4096, ab.BF16), (128, 1024, 4096, ab.F16), (300, 200, 3000, ab.BF16)]:
+        A = synth.draw_operand(M, K, synth.U11, 21, dtype, "cuda")
+        B = synth.draw_operand(K, N, synth.U11, 22, dtype, "cuda")
+        cands = ab.adapt_plan_candidates(M, N, K, dtype)
+        for f in [c for c in cands if c.fused][:6]:
+            twin = [c for c in cands if not c.fused and c.family == f.family and c.BN == f.BN and c.P_k == f.P_k
+                    and c.srcA == f.srcA and c.srcB == f.srcB]
+            pf = ab.adapt_matmul_plan_forced(M, N, K, dtype, ROW, ROW, f.tiling_key)
+            C1 = run_library(A, B, M, N, K, dtype, plan=pf).clone()
+            C2 = run_library(A, B, M, N, K, dtype, plan=pf)
+            torch.cuda.synchronize()
+            assert torch.equal(C1.view(torch.int16), C2.view(torch.int16))
+            if twin:
+                pt = ab.adapt_matmul_plan_forced(M, N, K, dtype, ROW, ROW, twin[0].tiling_key)
+                C3 = run_library(A, B, M, N, K, dtype, plan=pt)
+                torch.cuda.synchronize()
+                assert torch.equal(C1.view(torch.int16), C3.view(torch.int16)), (f.BN, f.P_k)
+            err, mism, n = compare_with_oracle(A, B, C1, M, N, K, dtype)
+            assert err <= TOL[dtype]
+        ab.adapt_poll_device_status(torch.cuda.current_stream().cuda_stream)
