@@ -668,6 +668,44 @@ def one_shape(args):
     return 0
 
 
+def store_ceiling(args):
+    """Write-only ceiling of the GEMM's store path: the epilogue's store pattern with nothing in front of it
+    (TMA box stores, 3-d TMA stores, plain 32-byte stores), on a 0.8 GB and a 13 GB output."""
+    import torch
+    from paper_2608_10803_b200 import binding as ab
+    ab.adapt_init(0)
+    st = torch.cuda.current_stream().cuda_stream
+    out = {"store_ceiling": []}
+    for rows, cols in ((20000, 20032), (94851, 69952)):
+        buf = torch.empty(rows * cols, dtype=torch.float16, device="cuda")
+        gb = rows * cols * 2 / 1e9
+        for mode, name in ((0, "tma_box_32x64"), (1, "tma_3d_32xtile"), (2, "st_global_v8")):
+            for tile_cols in (192, 256):
+                for order in (0, 1):
+                    for hint in (False, True):
+                        if mode == 2 and hint:
+                            continue
+                        us = ab.adapt_measure_store_rate(buf.data_ptr(), rows, cols, mode, tile_cols, order, hint, 3, st)
+                        out["store_ceiling"].append({"rows": rows, "cols": cols, "GB": round(gb, 2), "mode": name, "tile_cols": tile_cols,
+                                                     "order": "gemm_raster" if order == 0 else "row_block_major",
+                                                     "evict_first": hint, "us": round(us, 1), "TBps": round(gb / us * 1e3, 3)})
+        # context: the same bytes through cudaMemset-like torch fill
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        buf.fill_(1.0)
+        e0.record()
+        for _ in range(3):
+            buf.fill_(1.0)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / 3 * 1e3
+        out["store_ceiling"].append({"rows": rows, "cols": cols, "GB": round(gb, 2), "mode": "torch.fill_ (context)", "us": round(us, 1),
+                                     "TBps": round(gb / us * 1e3, 3)})
+        del buf
+    print(json.dumps(out))
+    return 0
+
+
 def validate_model(args):
     """The paper's model check (Section 6.6): time every legal configuration of a shape, call the
     fastest the oracle configuration, and count how often the analytical model picked it."""
@@ -756,10 +794,13 @@ def main():
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--src", type=str, default="", help="with --family: operand sources as two digits, e.g. 13 = A copied, B through k-class views")
     ap.add_argument("--fused", type=int, default=-1, help="with --family: 1 = only fused split-K configurations, 0 = only unfused")
+    ap.add_argument("--store-ceiling", action="store_true", help="measure the write-only ceiling of the store path (0.8 GB and 13 GB outputs)")
     ap.add_argument("--cublas", action="store_true", help="with --shape: also time torch.matmul as the vendor reference")
     args = ap.parse_args()
     if args.shape:
         return one_shape(args)
+    if args.store_ceiling:
+        return store_ceiling(args)
     if args.validate_model:
         return validate_model(args)
     if args.impl == "reference":

@@ -234,6 +234,17 @@ adapt_status_t adapt_measure_dispatch(adapt_handle_t plan, const void* A, const 
 adapt_status_t adapt_measure_empty_launch(int launches, int programmatic, void* cuda_stream,
                                           double* host_us, double* device_us);
 
+/* The write-only ceiling of the GEMM's store path (Eq. 2: a Common-template GEMM with a short K is a write of
+ * 2*M*N bytes and little else).  Writes a 16-bit matrix [rows][cols] (DEVICE buffer of rows*cols*2 bytes, 32-byte
+ * aligned, cols a multiple of 64; its contents are overwritten with a constant) `passes` times, tile by tile
+ * (128 rows x tile_cols columns, tile_cols = 64, 128, 192 or 256) from persistent CTAs laid out like the GEMM's
+ * epilogue warps, with nothing in front of the stores: mode 0 = TMA stores of 32 x 64 boxes (what the epilogue
+ * issues), 1 = one 3-d TMA store of 32 rows x tile_cols per warp and tile, 2 = plain 32-byte stores.
+ * order 0 visits the tiles in the GEMM's rasterisation, 1 row-block by row-block; hint != 0 stores with the
+ * evict-first L2 policy.  *device_us = time of one pass (CUDA events).  Synchronises the stream. */
+adapt_status_t adapt_measure_store_rate(void* buffer, int64_t rows, int64_t cols, int mode, int tile_cols,
+                                        int order, int hint, int passes, void* cuda_stream, double* device_us);
+
 /* Tensor maps encoded on the host since adapt_init; a call whose maps are cached encodes none.  Each plan
  * keeps the encodings of its 8 most recent distinct (pointer, geometry) pairs per operand. */
 int64_t adapt_map_encode_count(void);

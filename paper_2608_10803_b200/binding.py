@@ -26,6 +26,7 @@ EXPORTS = [
     "adapt_model_pipeline", "adapt_poll_device_status", "adapt_plan_cache_size", "adapt_launch_count",
     "adapt_matmul_noalloc", "adapt_matmul_batch", "adapt_matmul_repeat", "adapt_measure_dispatch",
     "adapt_measure_empty_launch", "adapt_map_encode_count", "adapt_set_map_cache", "adapt_selftest_wait_expiry",
+    "adapt_measure_store_rate",
 ]
 
 
@@ -129,6 +130,8 @@ def load():
     lib.adapt_measure_dispatch.argtypes = [vp, vp, vp, vp, vp, i32, ctypes.POINTER(DispatchCost)]
     lib.adapt_measure_empty_launch.restype = i32
     lib.adapt_measure_empty_launch.argtypes = [i32, i32, vp, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
+    lib.adapt_measure_store_rate.restype = i32
+    lib.adapt_measure_store_rate.argtypes = [vp, i64, i64, i32, i32, i32, i32, i32, vp, ctypes.POINTER(dbl)]
     lib.adapt_selftest_wait_expiry.restype = i32
     lib.adapt_selftest_wait_expiry.argtypes = [u64, vp]
     _lib = lib
@@ -209,6 +212,15 @@ def adapt_measure_empty_launch(launches: int, programmatic: bool, stream: int = 
     h, d = ctypes.c_double(), ctypes.c_double()
     _check(load().adapt_measure_empty_launch(launches, 1 if programmatic else 0, stream, ctypes.byref(h), ctypes.byref(d)))
     return h.value, d.value
+
+
+def adapt_measure_store_rate(buf_ptr: int, rows: int, cols: int, mode: int, tile_cols: int = 192, order: int = 0,
+                             hint: bool = False, passes: int = 3, stream: int = 0) -> float:
+    """Device microseconds of one write-only pass over a [rows][cols] 16-bit matrix (see the header)."""
+    us = ctypes.c_double()
+    _check(load().adapt_measure_store_rate(buf_ptr, rows, cols, mode, tile_cols, order, 1 if hint else 0, passes, stream,
+                                           ctypes.byref(us)))
+    return us.value
 
 
 def adapt_map_encode_count() -> int:

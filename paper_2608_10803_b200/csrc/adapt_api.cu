@@ -784,6 +784,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     struct { CUtensorMap a[16], b[8], c[16]; } maps;
     UmmaParams p;
     int a_box_rows = 128;
+    int b_box_k = 64;                                       // k rows one box of a row-major B brings
     memset(p.a_sigma, 0, sizeof(p.a_sigma));
     memset(p.b_sigma, 0, sizeof(p.b_sigma));
     p.cls_kc = (int)Kc;
@@ -849,7 +850,10 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
         // rows of B (K x N, N % 8 != 0) by class k % 8: the same construction as A's row classes, 64 x 64 boxes
         if ((r = cached_class_maps(S, pl, kMapB, B, s.K, s.N, 64, 8, 16, false, maps.b, p.b_sigma)) != ADAPT_OK) return r;
     } else {
-        if ((r = cached_map(S, pl, kMapB, b_src, inB, outB, pitchB, 64, b_mn ? 64 : c.BN / cg, &maps.b[0])) != ADAPT_OK) return r;
+        // a row-major B whose K fits one k-block is loaded with boxes of just the k rows that exist (rounded up to 8; class
+        // tiles shift B's rows by up to 7): boxes of 64 rows that lie mostly beyond K load several times slower when B is wide
+        if (b_mn && p.kb_total == 1) b_box_k = (int)std::min<int64_t>(64, round_up(s.K + ((classesA && s.K % 8) ? 7 : 0), 8));
+        if ((r = cached_map(S, pl, kMapB, b_src, inB, outB, pitchB, 64, b_mn ? b_box_k : c.BN / cg, &maps.b[0])) != ADAPT_OK) return r;
     }
 
     // 16-bit output leaves through TMA stores (boxes of 64 elements x 32 rows, one epilogue warp) when the
@@ -872,6 +876,12 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
         p.c_mode = 1;
     }
 
+    // write-bound shapes (C outweighs the operands) walk the tiles row block by row block
+    // (2048 x 97328 x 64: 80 -> 71 us, 94851 x 69977 x 12: 2740 -> 2580 us), unless K is so short that the one A tile all
+    // concurrent CTAs of a row block then read is a handful of cache lines (2048 x 97328 x 8: 86 -> 124 us that way)
+    p.raster = (p.P_k == 1 && (double)s.M * (double)s.N >= (double)s.K * ((double)s.M + (double)s.N) &&
+                (s.K >= 32 || p.P_n <= 64 || classesA)) ? 1 : 0;
+    if (const char* e = getenv("ADAPT_RASTER")) p.raster = atoi(e);
     p.a_shift_any = 0;
     for (int j = 0; j < 16; ++j) p.a_shift_any |= p.a_sigma[j];
     if (p.a_shift_any) p.a_shift_any = 1;
@@ -883,6 +893,10 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.x_pitch = umma_fused_pitch(c.BN);
     while (p.stages > 2 && umma_smem_bytes(c.BN, cg, p.stages, a_box_rows, p.P_k == 1, fused_bytes) > S.machine.smem_bytes) --p.stages;
     p.a_tx_bytes = a_box_rows * kUmmaBK * 2;
+    {
+        const int bn_cta = c.BN / cg;
+        p.b_tx_bytes = b_mn ? ((bn_cta + 63) / 64) * 64 * b_box_k * 2 : bn_cta * kUmmaBK * 2;
+    }
     p.idesc = umma_idesc(s.dtype, a_mn, b_mn, 128 * cg, c.BN);
     p.C = C;
     p.partial = partial;
@@ -1219,6 +1233,60 @@ extern "C" adapt_status_t adapt_measure_empty_launch(int launches, int programma
     CUDA_TRY(cudaGetLastError());
     *host_us = host / launches;
     *device_us = dev_ms * 1e3 / launches;
+    return ADAPT_OK;
+}
+
+extern "C" adapt_status_t adapt_measure_store_rate(void* buffer, int64_t rows, int64_t cols, int mode, int tile_cols,
+                                                   int order, int hint, int passes, void* cuda_stream, double* device_us)
+{
+    State& S = st();
+    if (!S.inited) return fail(ADAPT_ERR_NOT_INIT, "adapt_init has not been called%s");
+    if (!buffer || !device_us || rows < 1 || cols < 64 || cols % 64 != 0 || mode < 0 || mode > 2 || passes < 1 ||
+        tile_cols < 64 || tile_cols > 256 || tile_cols % 64 != 0 || ((uintptr_t)buffer & 31) != 0 || rows > 2147483647ll || cols > 2147483647ll)
+        return fail(ADAPT_ERR_INVALID_ARG, "store-rate measurement: rows >= 1, cols a multiple of 64, tile_cols 64..256, a 32-byte aligned buffer%s");
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    CUtensorMap map2d, map3d;
+    adapt_status_t r = encode_map(S, &map2d, buffer, 0, cols, rows, cols, 64, 32);
+    if (r != ADAPT_OK) return r;
+    {
+        const cuuint64_t gdim[3] = {64, (cuuint64_t)rows, (cuuint64_t)(cols / 64)};
+        const cuuint64_t gstride[2] = {(cuuint64_t)cols * 2, 128};
+        const cuuint32_t box[3] = {64, 32, (cuuint32_t)(tile_cols / 64)};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        const CUresult cr = S.encode(&map3d, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 3, buffer, gdim, gstride, box, estr,
+                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (cr != CUDA_SUCCESS) {
+            if (mode == 1) return fail(ADAPT_ERR_CUDA, "cuTensorMapEncodeTiled refused the 3-d store map%s");
+            map3d = map2d;
+        }
+    }
+    FillParams p;
+    p.C = (unsigned short*)buffer; p.rows = (int)rows; p.cols = (int)cols; p.tile_cols = tile_cols; p.order = order; p.hint = hint;
+    const void* k = mode == 0 ? (const void*)fill_kernel<0> : mode == 1 ? (const void*)fill_kernel<1> : (const void*)fill_kernel<2>;
+    const size_t smem = 8 * 16384 + 1024;
+    CUDA_TRY(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cudaEvent_t ev0, ev1;
+    CUDA_TRY(cudaEventCreate(&ev0));
+    CUDA_TRY(cudaEventCreate(&ev1));
+    for (int i = 0; i < passes + 1; ++i) {
+        if (i == 1) CUDA_TRY(cudaEventRecord(ev0, stream));
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof(cfg));
+        cfg.gridDim = dim3((unsigned)S.machine.n_sm, 1, 1);
+        cfg.blockDim = dim3(256, 1, 1);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        void* args[3] = {&map2d, &map3d, &p};
+        CUDA_TRY(cudaLaunchKernelExC(&cfg, k, args));
+    }
+    CUDA_TRY(cudaEventRecord(ev1, stream));
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    float ms = 0.f;
+    CUDA_TRY(cudaEventElapsedTime(&ms, ev0, ev1));
+    cudaEventDestroy(ev0);
+    cudaEventDestroy(ev1);
+    *device_us = (double)ms * 1e3 / passes;
     return ADAPT_OK;
 }
 

@@ -4,6 +4,7 @@
 #pragma once
 
 #include <cstdint>
+#include <cuda.h>
 #include <cuda_fp16.h>
 #include <cuda_bf16.h>
 
@@ -344,6 +345,86 @@ __global__ void wait_expiry_kernel(unsigned int* status, unsigned long long limi
     const bool ok = ptx::mbar_wait_limit(ptx::smem_u32(&bar), 0u, &abort_flag, limit_ns);
     __syncthreads();
     if (threadIdx.x == 0 && (!ok || abort_flag)) atomicOr(status, 1u);
+}
+
+// ---- write-only ceiling: the GEMM's store pattern with nothing in front of it -------------------------
+// A 16-bit matrix [rows][cols] (cols a multiple of 64, rows of 32 bytes alignment) is written tile by tile
+// (128 rows x tile_cols columns, tile_cols a multiple of 64) by persistent CTAs of eight warps, exactly as the GEMM
+// epilogue leaves its tiles: warp w takes the tiles of its CTA with parity w / 4 and the 32 rows of quarter w % 4.
+// MODE 0: one TMA store per 32 x 64 box (4 KB) from a 128B-swizzled staging box, two boxes in flight per warp
+//         (what the epilogue does).
+// MODE 1: one TMA store per 32 rows x tile_cols (a 3-d box over 64-column blocks), issued once per tile and warp.
+// MODE 2: plain stores, 32 bytes per lane, the warp covering 8 rows x 128 bytes per instruction.
+// order = 0 visits the tiles m-fastest in groups of 16 m-blocks (the GEMM's rasterisation), 1 visits them
+// n-fastest (neighbouring CTAs write neighbouring column blocks of the same rows).
+struct FillParams {
+    unsigned short* C;
+    int rows, cols, tile_cols, order, hint;
+};
+template <int MODE>
+__global__ void __launch_bounds__(256, 1)
+fill_kernel(const __grid_constant__ CUtensorMap map2d, const __grid_constant__ CUtensorMap map3d, const FillParams p)
+{
+    extern __shared__ uint8_t fill_smem[];
+    const uint32_t base = (ptx::smem_u32(fill_smem) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int q = warp & 3, half = warp >> 2;
+    const uint32_t wbuf = base + (uint32_t)warp * 16384u;      // up to four 4 KB boxes per warp
+    // something to store: the staging holds a pattern, written once
+    for (uint32_t i = threadIdx.x; i < 8u * 16384u / 16u; i += blockDim.x) {
+        const uint32_t v = 0x3c003c00u;
+        asm volatile("st.shared.v4.b32 [%0], {%1, %1, %1, %1};" ::"r"(base + 16u * i), "r"(v) : "memory");
+    }
+    ptx::fence_proxy_async_smem();
+    __syncthreads();
+    const int P_m = (p.rows + 127) / 128, P_n = (p.cols + p.tile_cols - 1) / p.tile_cols;
+    const int tiles = P_m * P_n;
+    const uint64_t pol = ptx::l2_policy_evict_first();
+    int seq = 0, box = 0;
+    for (int t = blockIdx.x; t < tiles; t += gridDim.x, ++seq) {
+        if ((seq & 1) != half) continue;
+        int mb, nb;
+        if (p.order == 0) {
+            const int group = 16 * P_n, g = t / group, first_m = g * 16, gm = min(P_m - first_m, 16), r = t - g * group;
+            mb = first_m + r % gm; nb = r / gm;
+        } else {
+            mb = t / P_n; nb = t - mb * P_n;
+        }
+        const int y0 = mb * 128 + q * 32, x0 = nb * p.tile_cols;
+        if (y0 >= p.rows) continue;
+        const int passes = min(p.tile_cols, p.cols - x0) / 64;
+        if (MODE == 0) {
+            for (int pass = 0; pass < passes; ++pass) {
+                if (lane == 0) {
+                    ptx::bulk_wait_read<1>();
+                    const uint32_t src = wbuf + (uint32_t)(box & 1) * 4096u;
+                    if (p.hint) ptx::tma_store_2d_hint(&map2d, src, x0 + 64 * pass, y0, pol);
+                    else ptx::tma_store_2d(&map2d, src, x0 + 64 * pass, y0);
+                    ptx::bulk_commit();
+                }
+                ++box;
+                __syncwarp();
+            }
+        } else if (MODE == 1) {
+            if (lane == 0) {
+                ptx::bulk_wait_read<0>();
+                asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                             ::"l"(&map3d), "r"(wbuf), "r"(0), "r"(y0), "r"(x0 / 64) : "memory");
+                ptx::bulk_commit();
+            }
+            __syncwarp();
+        } else {
+            const uint32_t r8[8] = {0x3c003c00u, 0x3c003c00u, 0x3c003c00u, 0x3c003c00u, 0x3c003c00u, 0x3c003c00u, 0x3c003c00u, 0x3c003c00u};
+            for (int pass = 0; pass < passes; ++pass)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int row = y0 + 8 * i + (lane >> 2);
+                    if (row < p.rows)
+                        ptx::st_global_v8(p.C + (size_t)row * p.cols + x0 + 64 * pass + 16 * (lane & 3), r8);
+                }
+        }
+    }
+    if (lane == 0) ptx::bulk_wait_read<0>();
 }
 
 }  // namespace adapt

@@ -44,6 +44,9 @@ struct UmmaParams {
     float* partial;                  // fp32 [P_k][M][Np], Np = N rounded up to 8 (used when P_k > 1)
     int Np;                          // row pitch of the partials in elements
     int a_tx_bytes;                  // bytes one TMA load of A delivers per stage and CTA (a short box when M < 128)
+    int b_tx_bytes;                  // bytes the TMA loads of B deliver per stage and CTA: the full boxes, or, for a row-major B
+                                     // when K fits one k-block, boxes of just the k rows that exist (rounded up to 8); the rows of
+                                     // the stage they leave untouched are zeroed once at kernel start
     int a_shift_any;                 // class mode: some a_sigma[j] != 0 (the MMA warp then zeroes row heads)
     int a_sigma[16];                 // class mode: shift (elements) of row class j against its 16-byte aligned base
     int b_sigma[8];                  // k-class mode: column shift of B's row class j = k % 8
@@ -51,6 +54,9 @@ struct UmmaParams {
     int c_mode;                      // 16-bit output: 0 = stores by the epilogue threads (any N, any alignment),
                                      // 1 = TMA stores through the maps of C (rows of C, or of the tile's row class,
                                      //     start on 32-byte boundaries; class tiles with 16 halo columns shift them there)
+    int raster;                      // tile visiting order: 0 = m-fastest inside groups of kGroupM m-blocks (operand reuse in L2),
+                                     // 1 = n-fastest, row block by row block (write-bound shapes: neighbouring CTAs write
+                                     //     neighbouring column blocks of the same rows, and a CTA's consecutive class tiles share their maps)
     int c_hint;                      // TMA stores of C carry an evict-first L2 policy
     int part_hint;                   // fp32 partials are stored with an evict-last L2 policy (they fit in L2)
     int c_sigma[16];                 // halo class tiles: shift (elements) of C's row class j against its 32-byte aligned base
@@ -92,6 +98,11 @@ __device__ __forceinline__ void decode_unit(const UmmaParams& p, int unit, int& 
 {
     split = unit % p.P_k;
     const int t = unit / p.P_k;
+    if (p.raster == 1) {
+        mb = t / p.P_n;
+        nb = t - mb * p.P_n;
+        return;
+    }
     const int group_size = kGroupM * p.P_n;
     const int g = t / group_size;
     const int first_m = g * kGroupM;
@@ -261,12 +272,27 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
         }
         ptx::fence_barrier_init();
         ptx::fence_proxy_async_smem();
-        ptx::prefetch_tensormap(&maps.a[0]);
-        ptx::prefetch_tensormap(&maps.b[0]);
+        // the maps this CTA's first unit goes through (a class tile reads A and writes C through its class's maps)
+        int mb0 = 0, nb0 = 0, sp0 = 0;
+        const int first_unit = (CG == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+        if (first_unit < p.num_units) decode_unit(p, first_unit, mb0, nb0, sp0);
+        ptx::prefetch_tensormap(&maps.a[A_CLS ? (mb0 % NCLS) : 0]);
+        ptx::prefetch_tensormap(&maps.b[(B_SPLIT || B_CLS) ? (sp0 & 7) : 0]);
+        if (p.c_mode != 0) ptx::prefetch_tensormap(&maps.c[A_CLS ? (mb0 % NCLS) : 0]);
     }
     if (warp == 1) {
         ptx::tmem_alloc<CG>(tmem_slot, TMEM_COLS);
         ptx::tmem_relinquish<CG>();
+    } else if (p.b_tx_bytes < B_BYTES) {
+        // Short-K boxes of B: a load then brings only the k rows that exist, so the rest of every stage's B region is
+        // zeroed here, once (no load ever writes it; the tensor core multiplies it with the zero-filled k tail of A).
+        // Boxes made of 64 k rows of which most lie beyond K cost a wide B several times the load time of full ones.
+        const int t = threadIdx.x >= 64 ? (int)threadIdx.x - 32 : (int)threadIdx.x;     // 288 threads, warp 1 left out
+        for (int st = 0; st < S; ++st) {
+            uint4* dst = reinterpret_cast<uint4*>(gen_base + (size_t)st * STAGE_BYTES + A_BYTES);
+            for (int i = t; i < B_BYTES / 16; i += kUmmaThreads - 32) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+        }
+        ptx::fence_proxy_async_smem();
     }
     ptx::tc_fence_before();
     if (CG == 2 || FUSE) {      // peers arrive on this CTA's barriers: they must all exist first
@@ -318,6 +344,13 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                 const int kshift = A_CLS ? p.a_sigma[cls] : 0;                // B's k-rows lag A's kappa by sigma
                 const CUtensorMap* tmA = &maps.a[cls];
                 const CUtensorMap* tmB = &maps.b[B_SPLIT ? (split & 7) : 0];  // k classes as splits: the class's view of B
+                if ((A_CLS || B_SPLIT) && lane == 0 && unit + unit_step < p.num_units) {
+                    // the next unit may go through other maps: fetch their descriptors while this unit loads
+                    int mb2, nb2, sp2;
+                    decode_unit(p, unit + unit_step, mb2, nb2, sp2);
+                    if (A_CLS && (mb2 % NCLS) != cls) ptx::prefetch_tensormap(&maps.a[mb2 % NCLS]);
+                    if (B_SPLIT && (sp2 & 7) != (split & 7)) ptx::prefetch_tensormap(&maps.b[sp2 & 7]);
+                }
                 const int a_k_off = B_SPLIT ? (split & 7) * p.cls_kc : 0;     // ... and its segment of the regrouped A
                 const int col0 = nb * TILE_N + (int)cta_rank * BN_CTA;        // this CTA's B columns
                 if (B_CLS) {
@@ -327,7 +360,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                             ok = __all_sync(REQ_MASK, ptx::mbar_wait(empty_bar + 8u * stage, phase ^ 1u, abort_flag));
                             if (!ok) break;
                             const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
-                            if (lane == 0) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(p.a_tx_bytes + B_BYTES));
+                            if (lane == 0) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(p.a_tx_bytes + p.b_tx_bytes));
                             __syncwarp(REQ_MASK);
                             if (is_a) load(sA, tmA, full_bar + 8u * stage, j * p.cls_kc + kb * kUmmaBK, row0);
                             else load(sA + A_BYTES, &maps.b[B_CLS ? j : 0], full_bar + 8u * stage, col0, kb * kUmmaBK);
@@ -341,8 +374,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     const uint32_t sB = sA + A_BYTES;
                     const uint32_t fb = full_target + 8u * stage;
                     if (lane == 0) {
-                        if (CG == 1) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(p.a_tx_bytes + B_BYTES));
-                        else if (leader) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, 2 * STAGE_BYTES);
+                        if (CG == 1) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(p.a_tx_bytes + p.b_tx_bytes));
+                        else if (leader) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(2 * (A_BYTES + p.b_tx_bytes)));
                     }
                     __syncwarp(REQ_MASK);
                     const int k0 = kb * kUmmaBK;
@@ -635,6 +668,12 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     // = (x - x_first) + 16 - sigma.  The first 16 - sigma elements of a row (x < 16) share their
                     // unit with the previous row of C, the last (N + sigma) % 16 with the next one: the row's own
                     // thread writes both with aligned stores of 2 to 16 bytes (head: tile nb = 0; tail: the tile that owns the unit).
+                    if (A_CLS && (seq & 1) != half && lane == 0 && unit + unit_step < p.num_units) {
+                        // the other warp of the quarter stores this tile; this one stores the next: fetch its map's descriptor now
+                        int mb2, nb2, sp2;
+                        decode_unit(p, unit + unit_step, mb2, nb2, sp2);
+                        ptx::prefetch_tensormap(&maps.c[mb2 % NCLS]);
+                    }
                     if ((seq & 1) == half) {
                         const int cls = A_CLS ? (mb % NCLS) : 0;
                         const int sig = HALO ? p.c_sigma[cls] : 0;
