@@ -41,6 +41,8 @@ NCU_TRAFFIC_RATIO = {
     "umma_2cta/k_classes_as_splits": 1.04,
     "umma_1cta/plain_tiles": 1.01,           # 16 x 65536 x 4096: 546.8 / 539.1 MB
     "umma_2cta/plain_tiles": 0.87,           # 4096^3: 87.9 / 100.7 MB
+    "umma_2cta/plain_tiles+stream_k": 0.87,
+    "umma_1cta/plain_tiles+stream_k": 1.01,
 }
 
 
@@ -55,7 +57,7 @@ def kernel_variant(ab, info):
         mode = "halo_class_tiles" if info.BN % 64 else "row_class_tiles"
     else:
         mode = "plain_tiles"
-    return f"{fam}/{mode}" + ("+fused_reduce" if info.fused else "")
+    return f"{fam}/{mode}" + ("+fused_reduce" if info.fused else "") + ("+stream_k" if info.streamk else "")
 
 
 def max_over_ranks(x, dist, device):
@@ -518,11 +520,11 @@ def ours(args):
         if args.dump:
             os.makedirs(os.path.dirname(os.path.abspath(args.dump)), exist_ok=True)
             with open(args.dump, "w") as f:
-                f.write("index,M,N,K,dtype,family,class,BM,BN,stages,P_k,fused,srcA,srcB,pred_us,time_us,tflops,frac_nominal,t_roof_us,vendor_us\n")
+                f.write("index,M,N,K,dtype,family,class,BM,BN,stages,P_k,fused,streamk,srcA,srcB,pred_us,time_us,tflops,frac_nominal,t_roof_us,vendor_us\n")
                 for i, (c, info, t) in enumerate(zip(cases, infos, per_shape)):
                     vu = f"{vendor[i] * 1e6:.3f}" if vendor is not None else ""
                     f.write(f"{i},{c.M},{c.N},{c.K},{c.dtype},{ab.FAMILY_NAMES[info.family]},{info.taxonomy_class},{info.BM},{info.BN},"
-                            f"{info.stages},{info.P_k},{info.fused},{info.srcA},{info.srcB},{info.predicted_us:.3f},{t * 1e6:.3f},"
+                            f"{info.stages},{info.P_k},{info.fused},{info.streamk},{info.srcA},{info.srcB},{info.predicted_us:.3f},{t * 1e6:.3f},"
                             f"{c.flops / t / 1e12:.4f},{t_roof_nominal(c) / t:.5f},{t_roof_nominal(c) * 1e6:.4f},{vu}\n")
 
     # ---- dispatch overhead of a cached plan (host clock, C call through ctypes) ----
@@ -635,6 +637,8 @@ def one_shape(args):
             cands = [c for c in cands if f"{c.srcA}{c.srcB}" == args.src]
         if args.fused >= 0:
             cands = [c for c in cands if c.fused == args.fused]
+        if args.streamk >= 0:
+            cands = [c for c in cands if c.streamk == args.streamk]
         plan = ab.adapt_matmul_plan_forced(M, N, K, dt, 0, 0, cands[0].tiling_key)
     else:
         plan = ab.adapt_matmul_plan(M, N, K, dt)
@@ -652,7 +656,7 @@ def one_shape(args):
     t = e0.elapsed_time(e1) / args.reps * 1e-3
     byts = 2.0 * (M * K + K * N + M * N)
     line = (f"{M}x{N}x{K} dt{dt} {ab.FAMILY_NAMES[info.family]} {info.BM}x{info.BN} st{info.stages} P_k{info.P_k} "
-            f"src{info.srcA}{info.srcB}{' fused' if info.fused else ''}: {t * 1e6:.1f} us  {2.0 * M * N * K / t / 1e12:.1f} TFLOP/s  {byts / t / 1e9:.0f} GB/s  "
+            f"src{info.srcA}{info.srcB}{' fused' if info.fused else ''}{' stream-K' if info.streamk else ''}: {t * 1e6:.1f} us  {2.0 * M * N * K / t / 1e12:.1f} TFLOP/s  {byts / t / 1e9:.0f} GB/s  "
             f"predicted {info.predicted_us:.1f} us")
     if args.cublas:
         torch.matmul(A, B, out=C)
@@ -793,6 +797,7 @@ def main():
     ap.add_argument("--pk", type=int, default=0)
     ap.add_argument("--stages", type=int, default=0)
     ap.add_argument("--src", type=str, default="", help="with --family: operand sources as two digits, e.g. 13 = A copied, B through k-class views")
+    ap.add_argument("--streamk", type=int, default=-1, help="with --family: 1 = only stream-K configurations, 0 = none of them")
     ap.add_argument("--fused", type=int, default=-1, help="with --family: 1 = only fused split-K configurations, 0 = only unfused")
     ap.add_argument("--store-ceiling", action="store_true", help="measure the write-only ceiling of the store path (0.8 GB and 13 GB outputs)")
     ap.add_argument("--cublas", action="store_true", help="with --shape: also time torch.matmul as the vendor reference")

@@ -108,7 +108,11 @@ typedef struct adapt_plan_info_s {
     int32_t fused;            /* 1: tcgen05 split-K whose P_k splits are the CTAs of one thread-block cluster and whose
                                  partial tiles are added through distributed shared memory inside the GEMM launch
                                  (no workspace, no reduction launch); 0 otherwise */
-    int64_t workspace_bytes;  /* pad copies + split-K partials */
+    int32_t streamk;          /* 1: tcgen05 stream-K: the k-blocks of the tiles that do not fill a whole wave of SMs are shared
+                                 evenly by all CTAs; partial tiles go through the workspace and are added by the tile's owner in
+                                 ascending k order inside the same launch; 0 otherwise */
+    int32_t reserved;
+    int64_t workspace_bytes;  /* pad copies + split-K / stream-K partials */
     double flops;             /* 2*M*N*K */
     double hbm_bytes;         /* modelled HBM traffic including workspace traffic */
     double t_pro_us;          /* Eq. 7 terms of the prediction */
@@ -121,7 +125,7 @@ typedef struct adapt_plan_info_s {
  * library's): [63:62] taxonomy class, [61:59] family, [58:54] BM/16, [53:48] BN/16,
  * [47:46] log2(BK/16), [45:42] stages, [41:32] P_k, [31] persistent tile loop,
  * [30:29] srcA, [28:27] srcB, [26] dtype, [25] layoutA, [24] layoutB, [23:22] log2(cluster) mod 4,
- * [21] log2(cluster) / 4, [20] fused in-cluster split-K reduction, [19:0] zero. */
+ * [21] log2(cluster) / 4, [20] fused in-cluster split-K reduction, [19] stream-K, [18:0] zero. */
 
 /* Select the device (cudaSetDevice), query it, and create the library state for
  * it.  Idempotent.  Needed before adapt_matmul; planning works without it (the

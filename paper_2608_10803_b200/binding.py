@@ -41,6 +41,7 @@ class PlanInfo(ctypes.Structure):
         ("P_m", ctypes.c_int32), ("P_n", ctypes.c_int32), ("P_k", ctypes.c_int32),
         ("cluster", ctypes.c_int32), ("srcA", ctypes.c_int32), ("srcB", ctypes.c_int32),
         ("grid", ctypes.c_int32), ("fused", ctypes.c_int32),
+        ("streamk", ctypes.c_int32), ("reserved", ctypes.c_int32),
         ("workspace_bytes", ctypes.c_int64),
         ("flops", ctypes.c_double), ("hbm_bytes", ctypes.c_double),
         ("t_pro_us", ctypes.c_double), ("t_main_us", ctypes.c_double), ("t_epi_us", ctypes.c_double),

@@ -122,7 +122,7 @@ struct State {
     Calib calib;
     unsigned int* d_status = nullptr;
     unsigned long long* d_trace = nullptr;   // diagnostic builds only
-    struct Workspace { void* ptr = nullptr; size_t bytes = 0; };
+    struct Workspace { void* ptr = nullptr; size_t bytes = 0; unsigned int epoch = 0; };
     std::unordered_map<cudaStream_t, Workspace> ws;
     // adapt_matmul_host: one three-stage pipeline per caller stream (copy in | kernels | copy out, each on
     // its own stream) with two staging slots, so the copies of consecutive calls overlap the kernels and
@@ -415,6 +415,28 @@ static UmmaKernel umma_lookup_fused(int BN, bool a_mn, bool b_mn)
     return nullptr;
 }
 
+// stream-K instantiations (plain tiles, both families)
+template <int CG>
+static UmmaKernel umma_lookup_sk(int BN, bool a_mn, bool b_mn)
+{
+#define ADAPT_PICK(bn)                                                                                \
+    if (BN == bn) {                                                                                   \
+        if (!a_mn && !b_mn) return (const void*)umma_gemm_kernel<bn, false, false, CG, 0, false, true>; \
+        if (!a_mn && b_mn) return (const void*)umma_gemm_kernel<bn, false, true, CG, 0, false, true>;   \
+        if (a_mn && !b_mn) return (const void*)umma_gemm_kernel<bn, true, false, CG, 0, false, true>;   \
+        return (const void*)umma_gemm_kernel<bn, true, true, CG, 0, false, true>;                       \
+    }
+    if constexpr (CG == 1) { ADAPT_PICK(64) }
+    ADAPT_PICK(128)
+    ADAPT_PICK(256)
+#undef ADAPT_PICK
+    return nullptr;
+}
+static UmmaKernel launch_map_umma_sk(int family, int BN, bool a_mn, bool b_mn)
+{
+    return family == ADAPT_FAM_UMMA_1CTA ? umma_lookup_sk<1>(BN, a_mn, b_mn) : umma_lookup_sk<2>(BN, a_mn, b_mn);
+}
+
 static UmmaKernel launch_map_umma(int family, int BN, bool a_mn, bool b_mn, int mode = 0, bool fused = false)
 {
     if (fused) {
@@ -508,6 +530,13 @@ extern "C" adapt_status_t adapt_init(int device)
             CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_1CTA, BN, false, true, 2, true),
                                           cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
     }
+    for (int fam = ADAPT_FAM_UMMA_1CTA; fam <= ADAPT_FAM_UMMA_2CTA; ++fam)
+        for (int BN : {64, 128, 256})
+            for (int a = 0; a < 2; ++a)
+                for (int b = 0; b < 2; ++b) {
+                    UmmaKernel k = launch_map_umma_sk(fam, BN, a != 0, b != 0);
+                    if (k) CUDA_TRY(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
+                }
     // clusters of 2, 4, 8 CTAs of the tcgen05 kernel (one CTA per SM) that the device runs at a time
     for (int i = 0; i < 3; ++i) {
         cudaLaunchConfig_t cfg;
@@ -593,12 +622,20 @@ extern "C" adapt_status_t adapt_poll_device_status(void* cuda_stream)
 // ---------------------------------------------------------------------------------------------
 namespace {
 
-adapt_status_t get_workspace(State& S, cudaStream_t stream, size_t bytes, void** out)
+// The stream's workspace, at least `bytes` large.  Its first kUmmaFlagBytes are the stream-K flag words: zeroed when the
+// workspace is allocated, afterwards only ever set to the epoch of a launch, and *epoch (if asked for) is a value no
+// earlier launch on this workspace has used.  The caller's regions start at *out (after the flags).
+adapt_status_t get_workspace(State& S, cudaStream_t stream, size_t bytes, void** out, unsigned int* epoch = nullptr, void** flags = nullptr)
 {
     *out = nullptr;
-    if (bytes == 0) return ADAPT_OK;
+    if (bytes == 0 && !epoch) return ADAPT_OK;
+    bytes += kUmmaFlagBytes;
     std::lock_guard<std::mutex> lock(S.mu);
     State::Workspace& w = S.ws[stream];
+    if (epoch) {
+        if (++w.epoch == 0) ++w.epoch;       // 0 is what fresh flags hold
+        *epoch = w.epoch;
+    }
     if (w.bytes < bytes) {
         if (w.ptr) {
             CUDA_TRY(cudaStreamSynchronize(stream));
@@ -614,8 +651,10 @@ adapt_status_t get_workspace(State& S, cudaStream_t stream, size_t bytes, void**
             return fail(ADAPT_ERR_NOMEM, "workspace allocation failed: %s", cudaGetErrorString(e));
         }
         w.bytes = want;
+        CUDA_TRY(cudaMemsetAsync(w.ptr, 0, kUmmaFlagBytes, stream));
     }
-    *out = w.ptr;
+    *out = (uint8_t*)w.ptr + kUmmaFlagBytes;
+    if (flags) *flags = w.ptr;
     return ADAPT_OK;
 }
 
@@ -806,8 +845,14 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     // the plan's fused reduction stands unless a fallback changed the tiling (then: partials in the workspace)
     const bool fused = c.fused != 0 && p.P_k == c.P_k && !(c.srcB == ADAPT_SRC_TMA_CLASSES && !kclsB);
     const size_t szP = (p.P_k > 1 && !fused) ? (size_t)round_up((int64_t)p.P_k * s.M * partial_pitch(s.N) * 4, 256) : 0;
+    // stream-K stands unless a fallback changed the tiling; one fp32 partial tile per CTA
+    const bool streamk = c.streamk != 0 && p.P_k == 1 && !classesA && !kclsB;
+    const int sk_slots = S.machine.n_sm / c.cluster;
+    const size_t szS = streamk ? (size_t)sk_slots * c.cluster * 128 * c.BN * 4 : 0;
     void* ws = nullptr;
-    adapt_status_t r = get_workspace(S, stream, szA + szB + szP, &ws);
+    void* ws_flags = nullptr;
+    unsigned int epoch = 0;
+    adapt_status_t r = get_workspace(S, stream, szA + szB + szP + szS, &ws, streamk ? &epoch : nullptr, &ws_flags);
     if (r != ADAPT_OK) return r;
     uint8_t* w8 = (uint8_t*)ws;
     const void* a_src = A;
@@ -891,6 +936,16 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     const int fused_bytes = fused ? umma_fused_bytes(c.BN, a_box_rows) : 0;
     p.x_rows = a_box_rows;
     p.x_pitch = umma_fused_pitch(c.BN);
+    p.sk_tiles = p.sk_q0 = p.sk_rem = 0;
+    p.sk_partial = nullptr;
+    p.sk_flags = (unsigned int*)ws_flags;
+    p.sk_epoch = epoch;
+    if (streamk) {
+        const StreamK sk = streamk_schedule(p.num_units, sk_slots, p.kb_total);
+        p.sk_tiles = (int)sk.sk_tiles; p.sk_q0 = (int)sk.q0; p.sk_rem = (int)sk.rem;
+        p.sk_partial = (float*)(w8 + szA + szB + szP);
+        p.part_hint = 1;                                    // the partial tiles are read back within microseconds: keep them in L2
+    }
     while (p.stages > 2 && umma_smem_bytes(c.BN, cg, p.stages, a_box_rows, p.P_k == 1, fused_bytes) > S.machine.smem_bytes) --p.stages;
     p.a_tx_bytes = a_box_rows * kUmmaBK * 2;
     {
@@ -903,15 +958,18 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.Np = (int)partial_pitch(s.N);
     p.status = S.d_status;
     p.trace = nullptr;
+    p.trace_cta = 0;
 #ifdef ADAPT_TRACE_BUILD
     p.trace = S.d_trace;
+    if (const char* e = getenv("ADAPT_TRACE_CTA")) p.trace_cta = atoi(e);
 #endif
 
-    UmmaKernel k = launch_map_umma(c.family, c.BN, a_mn, b_mn, classesA ? 1 : (kclsB ? 2 : 0), fused);
+    UmmaKernel k = streamk ? launch_map_umma_sk(c.family, c.BN, a_mn, b_mn)
+                           : launch_map_umma(c.family, c.BN, a_mn, b_mn, classesA ? 1 : (kclsB ? 2 : 0), fused);
     if (!k) return fail(ADAPT_ERR_UNSUPPORTED, "no compiled kernel for this tiling key%s");
     const int slots = fused ? umma_cluster_slots(S.machine, p.P_k) : S.machine.n_sm / cg;
     const int launch_cluster = fused ? p.P_k : cg;            // fused split-K: the splits of a tile are one cluster
-    const int grid = fused ? std::min(p.P_m * p.P_n, slots) * p.P_k : std::min(p.num_units, slots) * cg;
+    const int grid = fused ? std::min(p.P_m * p.P_n, slots) * p.P_k : (streamk ? slots : std::min(p.num_units, slots)) * cg;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)grid, 1, 1);

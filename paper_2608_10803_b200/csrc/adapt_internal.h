@@ -71,6 +71,9 @@ struct Calib {
     double cluster_crowd_us = 1.56, cluster_crowd_stage_us = 0.44;   // per CTA per SM beyond one per two SMs
     double cluster_wave_us = 5.5;       // each further round of clusters
     double cluster_bw_eff = 0.35;       // fraction of hbm_bw its 16-byte copies reach when memory-bound
+    double streamk_fixup_us = 10.0;     // stream-K: partial tile out (5 us) and its fence, the flag, the owner's exposed last drain ...
+    double streamk_peer_us = 3.0;       // ... and its additions, per slot that shares the tile (2560 x 4096 x 4096, 6 sharers: 87 us
+                                        // against 55 us of main loop; 5120 x 4096 x 8192, 3 sharers: 246 us against 226 us)
     double fused_reduce_us = 2.5;       // fused split-K: cluster scheduling, drain to shared memory, two cluster-wide barrier rounds,
                                         // first remote reads (1 x 4096 x 4096, 128 x 128 tiles, P_k 4: 12.1 us fused, 11.3 us with the reduce launch)
     double fused_wave_us = 3.5;         // each further round of clusters starts cold (1 x 4096 x 4096, P_k 8: 3 rounds 26 us, 2 rounds 20 us)
@@ -100,6 +103,8 @@ struct Config {
     int cluster = 1;
     int fused = 0;                      // tcgen05 split-K with the k splits as one thread-block cluster, reduced through
                                         // distributed shared memory inside the GEMM launch (no partials in global memory)
+    int streamk = 0;                    // tcgen05, P_k = 1: the k-blocks of the tiles that do not fill a whole wave of slots are
+                                        // shared evenly by all slots (deterministic stream-K)
     int persistent = 0;
     int srcA = ADAPT_SRC_LSU, srcB = ADAPT_SRC_LSU;
     int grid = 1;
@@ -173,6 +178,22 @@ inline int cluster_ring(int64_t K, int cluster, int64_t tiles, int n_sm)
     const int cap = tiles <= cluster_slots(cluster, n_sm) ? kClusterMaxRing : 4;
     return (int)std::max<int64_t>(1, std::min<int64_t>(stages, cap));
 }
+// Stream-K schedule of a shape: W whole waves of tiles stay data-parallel, the R = tiles - W * slots tiles left over
+// (all tiles when there are fewer than slots) are cut into k-block ranges, sk_q0 (+1 for the first sk_rem slots) per slot.
+struct StreamK {
+    int64_t tiles, slots, waves, sk_tiles, q0, rem;
+};
+inline StreamK streamk_schedule(int64_t tiles, int64_t slots, int64_t kblocks)
+{
+    StreamK k;
+    k.tiles = tiles; k.slots = slots;
+    k.waves = tiles / slots;
+    k.sk_tiles = tiles - k.waves * slots;
+    k.q0 = k.sk_tiles * kblocks / slots;
+    k.rem = k.sk_tiles * kblocks - k.q0 * slots;
+    return k;
+}
+constexpr int kUmmaFlagBytes = 4096;     // head of every workspace: stream-K flag words (one per CTA), zeroed when the workspace is allocated
 constexpr int kSkinnyKChunk = 512;   // k values the warp-level kernel stages per chunk; its k splits are whole chunks
 constexpr int kUmmaBarrierBytes = 1024;  // keeps the epilogue staging 1024-byte aligned (swizzled TMA boxes)
 constexpr int kUmmaMaxStages = 15;

@@ -78,12 +78,13 @@ uint64_t pack_tiling_key(const Shape& s, const Config& c)
     k |= (uint64_t)(ilog2(std::max(c.cluster, 1)) & 3) << 22;
     k |= (uint64_t)((ilog2(std::max(c.cluster, 1)) >> 2) & 1) << 21;
     k |= (uint64_t)(c.fused & 1) << 20;
+    k |= (uint64_t)(c.streamk & 1) << 19;
     return k;
 }
 
 bool unpack_tiling_key(uint64_t k, Shape* s, Config* c)
 {
-    if (k & ((1ull << 20) - 1)) return false;
+    if (k & ((1ull << 19) - 1)) return false;
     c->cls = (int)((k >> 62) & 3);
     c->family = (int)((k >> 59) & 7);
     c->BM = (int)((k >> 54) & 31) * 16;
@@ -99,6 +100,7 @@ bool unpack_tiling_key(uint64_t k, Shape* s, Config* c)
     s->layoutB = (int)((k >> 24) & 1);
     c->cluster = 1 << (int)(((k >> 22) & 3) | (((k >> 21) & 1) << 2));
     c->fused = (int)((k >> 20) & 1);
+    c->streamk = (int)((k >> 19) & 1);
     return true;
 }
 
@@ -160,6 +162,11 @@ static void model_epilogue(const Shape& s, Config& c, const Calib& cal)
 {
     c.t_epi_us = 0;
     c.ws_partial = 0;
+    if (c.streamk) {
+        // one fp32 partial tile per CTA, written and read back once at most (they stay in L2); no second launch
+        c.ws_partial = (int64_t)c.grid * 128 * c.BN * 4;
+        return;
+    }
     if (c.fused) {
         // Eq. 11 with the cross-core exchange on chip: each CTA reads one tile's worth of fp32 partials from its
         // peers' shared memory (its share of the rows over all ranks); no second launch, no workspace
@@ -191,7 +198,7 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     const int64_t units = c.fused ? (int64_t)c.P_m * c.P_n : (int64_t)c.P_m * c.P_n * c.P_k;
     const int64_t slots = c.fused ? umma_cluster_slots(m, c.P_k) : m.n_sm / c.cluster;
     const int64_t Q = ceil_div(units, slots);
-    c.grid = (int)(std::min(units, slots) * (c.fused ? c.P_k : c.cluster));
+    c.grid = c.streamk ? (int)(slots * c.cluster) : (int)(std::min(units, slots) * (c.fused ? c.P_k : c.cluster));
 
     const double MK = (double)s.M * s.K, KN = (double)s.K * s.N, MN = (double)s.M * s.N;
     // HBM traffic: operands once, plus re-reads of B when it cannot stay in L2 across m-groups.
@@ -266,6 +273,18 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
                                            : std::max((double)L * ii + t_fixed, t_drain);
         // Eq. 14 with the drain overlapped: one fill, Q tiles back to back, the last drain exposed
         pipe = tM + (double)Q * t_tile + tP + t_drain;
+        if (c.streamk) {
+            // whole waves as above; the leftover tiles' k-blocks shared evenly by all slots, then the owners' fix-up
+            // While a slot works on its share of the leftover tiles it is at a k position of its own: nothing it loads is
+            // shared with the other slots at that moment, so all of them together pull slots x stage bytes per k-block
+            // from HBM (8192^3: 74 pairs x 64 KB per 0.41 us = 11.5 TB/s asked for), and the shared part runs at that rate
+            const StreamK sk = streamk_schedule(units, slots, L);
+            const double shared = (double)(sk.q0 + (sk.rem ? 1 : 0));
+            const double ii_shared = std::max(ii, (double)slots * c.cluster * stage_bytes / cal.hbm_bw * 1e6);
+            pipe = tM + std::max((double)sk.waves * (double)L * ii + shared * ii_shared + (double)(sk.waves + 1) * t_fixed,
+                                 (double)(sk.waves + 2) * t_drain) + tP + t_drain + cal.streamk_fixup_us +
+                   cal.streamk_peer_us * (double)L / (double)std::max<int64_t>(1, sk.q0);
+        }
     }
     pipe += cal.umma_fixed_us;
     if (c.fused) pipe += cal.fused_wave_us * (double)(Q - 1);
@@ -411,6 +430,10 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     if (c.BN % 16 != 0 || c.BN > 256) return false;                 // UMMA shape rule for M = 128/256
     if (2 * c.BN > m.tmem_cols) return false;                       // at least two accumulator buffers in TMEM
     if (c.stages < 1 || c.stages > kUmmaMaxStages) return false;
+    if (c.streamk) {
+        // plain tiles, one split, not fused; needs leftover tiles and at least two k-blocks per slot in the shared part
+        if (c.P_k != 1 || c.fused || c.srcA == ADAPT_SRC_TMA_CLASSES || c.srcB == ADAPT_SRC_TMA_CLASSES || c.stages < 2) return false;
+    }
     const int a_rows_box = umma_a_box_rows(s, c.cluster, umma_row_classes(c.srcA, c.BN), c.srcB == ADAPT_SRC_TMA_CLASSES);
     if (c.fused) {
         // the k splits of a tile form one cluster: 1-CTA tiles, a portable cluster size, no halo tiles, not the
@@ -457,6 +480,12 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     c.P_m = classes ? (int)(ncls * ceil_div(s.M, ncls * c.BM)) : (int)ceil_div(s.M, c.BM);   // class tiles: 8 per 1024 rows, 16 per 2048
     c.P_n = (int)ceil_div(s.N, kclasses ? c.BN - 8 : (c.BN % 64 ? c.BN - 16 : c.BN));
     if ((int64_t)c.P_m * c.P_n * c.P_k > (int64_t)1 << 30) return false;
+    if (c.streamk) {
+        const int64_t kb = ceil_div(s.K, c.BK);
+        const StreamK sk = streamk_schedule((int64_t)c.P_m * c.P_n, m.n_sm / c.cluster, kb);
+        // at most about eight slots per shared tile: its owner adds their partials one after the other
+        if (sk.sk_tiles == 0 || sk.q0 < 2 || kb < 4 || sk.q0 * 8 < kb) return false;
+    }
     c.persistent = 1;
     return true;
 }
@@ -602,6 +631,13 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
                     c.stages = st; c.P_k = pk; c.srcA = srcA; c.srcB = srcB;
                     if (st >= 2 && finalize(s, m, cal, c)) out->push_back(c);
                 }
+                // one split, the leftover wave shared by all slots (stream-K)
+                if (pk == 1) {
+                    Config c;
+                    c.family = fam; c.BM = BM; c.BN = BN; c.BK = 64; c.cluster = cluster; c.streamk = 1;
+                    c.stages = deepest; c.P_k = 1; c.srcA = srcA; c.srcB = srcB;
+                    if (deepest >= 2 && finalize(s, m, cal, c)) out->push_back(c);
+                }
                 // the same split with its reduction fused into the launch (the splits of a tile as one cluster)
                 if (fam == ADAPT_FAM_UMMA_1CTA && (pk == 2 || pk == 4 || pk == 8)) {
                     Config c;
@@ -742,7 +778,7 @@ void fill_info(const Shape& s, const Config& c, adapt_plan_info_t* o)
     o->taxonomy_class = c.cls; o->family = c.family;
     o->BM = c.BM; o->BN = c.BN; o->BK = c.BK; o->stages = c.stages;
     o->P_m = c.P_m; o->P_n = c.P_n; o->P_k = c.P_k; o->cluster = c.cluster;
-    o->srcA = c.srcA; o->srcB = c.srcB; o->grid = c.grid; o->fused = c.fused;
+    o->srcA = c.srcA; o->srcB = c.srcB; o->grid = c.grid; o->fused = c.fused; o->streamk = c.streamk; o->reserved = 0;
     o->workspace_bytes = c.workspace_bytes;
     o->flops = 2.0 * (double)s.M * (double)s.N * (double)s.K;
     o->hbm_bytes = c.hbm_bytes;

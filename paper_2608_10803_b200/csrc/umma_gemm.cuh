@@ -61,16 +61,23 @@ struct UmmaParams {
     int part_hint;                   // fp32 partials are stored with an evict-last L2 policy (they fit in L2)
     int c_sigma[16];                 // halo class tiles: shift (elements) of C's row class j against its 32-byte aligned base
     int c_extent[16];                // ... and the elements of a shifted row of that class that lie in whole 32-byte units
+    // stream-K (SK kernels): the first sk_tiles tiles are cut into k-block ranges shared evenly by all slots (a slot is a
+    // CTA, or a CTA pair): slot s takes sk_q0 (+1 for s < sk_rem) consecutive k-blocks of the tile-major sequence
+    int sk_tiles, sk_q0, sk_rem;
+    float* sk_partial;               // one fp32 partial tile [128][BN] per CTA (slot * CTAs per slot + rank in the pair)
+    unsigned int* sk_flags;          // one word per CTA: the epoch of the launch whose partial is complete there
+    unsigned int sk_epoch;           // this launch's epoch (unique per workspace)
     int x_rows, x_pitch;             // fused split-K: rows and row pitch (fp32 elements) of the partial tile each CTA of the
                                      // cluster keeps in its shared memory for the exchange
     unsigned int* status;            // device status word: bit 0 = a bounded wait expired
-    unsigned long long* trace;       // timestamp trace of CTA 0 (diagnostic builds only), else null
+    unsigned long long* trace;       // timestamp trace of one CTA (diagnostic builds only), else null
+    int trace_cta;
 };
 
 #ifdef ADAPT_TRACE_BUILD
 #define ADAPT_TRACE(ev, unit)                                                                         \
     do {                                                                                              \
-        if (p.trace && blockIdx.x == 0) {                                                             \
+        if (p.trace && (int)blockIdx.x == p.trace_cta) {                                                             \
             const unsigned long long sl = atomicAdd(p.trace, 1ull);                                   \
             if (sl < 30000) { p.trace[1 + 2 * sl] = ((unsigned long long)(ev) << 32) | (unsigned)(unit); p.trace[2 + 2 * sl] = ptx::globaltimer_ns(); } \
         }                                                                                             \
@@ -110,6 +117,69 @@ __device__ __forceinline__ void decode_unit(const UmmaParams& p, int unit, int& 
     const int r = t - g * group_size;
     mb = first_m + r % gm;
     nb = r / gm;
+}
+
+// One entry of a slot's work list.  kind 0: the whole k range of a tile (or one split of it), stored the usual way;
+// kind 1 (stream-K): a k range that does not start at 0: an fp32 partial tile for the slot that owns the tile's start;
+// kind 2 (stream-K): the start of a tile whose later k ranges `npeers` following slots contribute.
+struct WorkItem {
+    int unit, mb, nb, split, kb0, kb1, kind, npeers;
+};
+
+// The it-th work item of slot `slot` (of `n_slots`).  Without stream-K: unit slot + it * n_slots.  With stream-K
+// (Section 4.2's StreamK remark, made deterministic): first the slot's share of the stream-K tiles (at most two
+// ranges: the end of one tile, then the start of the next), then whole tiles sk_tiles + slot + j * n_slots.
+template <bool SK, bool B_SPLIT>
+__device__ __forceinline__ bool next_item(const UmmaParams& p, int slot, int n_slots, int it, WorkItem& w)
+{
+    w.kind = 0;
+    w.npeers = 0;
+    if (!SK) {
+        w.unit = slot + it * n_slots;
+        if (w.unit >= p.num_units) return false;
+        decode_unit(p, w.unit, w.mb, w.nb, w.split);
+        w.kb0 = (B_SPLIT ? (w.split >> 3) : w.split) * p.kb_per_split;
+        w.kb1 = min(p.kb_total, w.kb0 + p.kb_per_split);
+        return true;
+    }
+    const int L = p.kb_total;
+    const int begin = slot * p.sk_q0 + min(slot, p.sk_rem);
+    const int len = p.sk_q0 + (slot < p.sk_rem ? 1 : 0);
+    const int t1 = begin / L, a = begin - t1 * L;
+    const bool crosses = a + len > L;
+    // The slot's share is at most two ranges: the END of tile t1 (when it does not start at k-block 0) and the START of
+    // the next tile.  The end range comes first: its partial is what the previous slot will need.  The start range comes
+    // LAST, after the slot's whole tiles: by then the slots that hold the rest of that tile have long written theirs.
+    const int n_first = (len > 0 && a != 0) ? 1 : 0;
+    const int n_last = (len > 0 && (a == 0 || crosses)) ? 1 : 0;
+    const int first_dp = p.sk_tiles + slot;
+    const int n_dp = first_dp < p.num_units ? (p.num_units - first_dp + n_slots - 1) / n_slots : 0;
+    int tile;
+    if (it < n_first) {
+        tile = t1; w.kb0 = a; w.kb1 = min(L, a + len);
+        w.kind = 1;
+    } else if (it < n_first + n_dp) {
+        tile = first_dp + (it - n_first) * n_slots;
+        w.kb0 = 0;
+        w.kb1 = L;
+    } else if (it < n_first + n_dp + n_last) {
+        if (a == 0) { tile = t1; w.kb1 = len; }
+        else { tile = t1 + 1; w.kb1 = a + len - L; }
+        w.kb0 = 0;
+        if (w.kb1 != L) {
+            // the slots after this one that hold the rest of the tile: up to the owner of its last k-block
+            const int last = (tile + 1) * L - 1;
+            const int cut = p.sk_rem * (p.sk_q0 + 1);
+            const int owner = last < cut ? last / (p.sk_q0 + 1) : p.sk_rem + (last - cut) / p.sk_q0;
+            w.kind = 2;
+            w.npeers = owner - slot;
+        }
+    } else {
+        return false;
+    }
+    w.unit = tile;
+    decode_unit(p, tile, w.mb, w.nb, w.split);
+    return true;
 }
 
 __device__ __forceinline__ uint32_t pack16(float a, float b, int dtype)
@@ -197,10 +267,18 @@ __device__ __forceinline__ void store_run16(unsigned short* dst, int count, cons
 // the tile's (row, 4-column) groups evenly, and each adds its groups over ranks 0 .. P_k-1 in ascending order
 // through distributed shared memory, rounds once and stores C.  The order is the one splitk_reduce_kernel
 // uses, so a shape gives the same bits with either path and from run to run.
-template <int BN, bool A_MN, bool B_MN, int CG, int MODE, bool FUSE = false>
+//
+// SK (stream-K, plain tiles, P_k = 1): when the tiles do not fill whole waves of slots, the k-blocks of the first
+// sk_tiles tiles are shared evenly by all slots.  A slot's share is one run of the tile-major k-block sequence: the end
+// of one tile (written as an fp32 partial, then a flag), then the start of the next, whose remaining k ranges the
+// following slots computed FIRST; the slot adds their partials to its accumulator in ascending k order and stores the
+// tile.  The assignment and the order of the additions are fixed by the shape, so the result is too.  Every wait on a
+// flag is bounded like the barrier waits.
+template <int BN, bool A_MN, bool B_MN, int CG, int MODE, bool FUSE = false, bool SK = false>
 __global__ void __launch_bounds__(kUmmaThreads, 1)
 umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams p)
 {
+    static_assert(!SK || (MODE == 0 && !FUSE), "stream-K: plain tiles");
     static_assert(!FUSE || (CG == 1 && (MODE == 0 || MODE == 1 || MODE == 3)), "the fused reduction: 1-CTA tiles, clusters made of the k splits");
     static_assert(!FUSE || BN % 64 == 0, "the fused reduction has no halo tiles");
     constexpr bool A_CLS = MODE == 1;
@@ -248,6 +326,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
     uint8_t* stage_out = bar_gen + kUmmaBarrierBytes;
     // fused split-K: "every rank's partial is in place" / "every rank has read mine", at fixed offsets of the barrier block
     const uint32_t xfull_bar = bar_base + 512u, xempty_bar = bar_base + 520u;
+    int* sk_count = reinterpret_cast<int*>(bar_gen + 528);     // stream-K: epilogue warps that have written their share of a partial
 
     pdl_launch_dependents();
     if (threadIdx.x == 0) ADAPT_TRACE(11, 0);
@@ -258,6 +337,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
 
     if (threadIdx.x == 0) {
         *abort_flag = 0;
+        *sk_count = 0;
         for (int s = 0; s < S; ++s) {
             ptx::mbar_init(full_bar + 8u * s, 1);          // one arrive.expect_tx per phase
             ptx::mbar_init(empty_bar + 8u * s, 1);         // one tcgen05.commit per phase
@@ -332,11 +412,10 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
             };
             const bool is_a = lane < NREQ_A;
             const int jb = lane - NREQ_A;                                     // B box of this lane
-            for (int unit = unit0; ok && unit < p.num_units; unit += unit_step) {
-                int mb, nb, split;
-                decode_unit(p, unit, mb, nb, split);
-                const int kb0 = (B_SPLIT ? (split >> 3) : split) * p.kb_per_split;
-                const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+            for (int it = 0; ok; ++it) {
+                WorkItem w;
+                if (!next_item<SK, B_SPLIT>(p, unit0, unit_step, it, w)) break;
+                const int unit = w.unit, mb = w.mb, nb = w.nb, split = w.split, kb0 = w.kb0, kb1 = w.kb1;
                 // A rows of this CTA: consecutive rows, or in class mode rows 1024*g + j + 8*i read through
                 // map j at class-row index 128*g
                 const int cls = A_CLS ? (mb % NCLS) : 0;
@@ -423,11 +502,11 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                 return __shfl_sync(0xffffffffu, w, 0) != 0;
             };
             bool ok = true;
-            for (int unit = unit0; ok && unit < p.num_units; unit += unit_step) {
-                int mb, nb, split;
-                decode_unit(p, unit, mb, nb, split);
-                const int kb0 = (B_SPLIT ? (split >> 3) : split) * p.kb_per_split;
-                const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+            for (int it = 0; ok; ++it) {
+                WorkItem w;
+                if (!next_item<SK, B_SPLIT>(p, unit0, unit_step, it, w)) break;
+                const int unit = w.unit, mb = w.mb, nb = w.nb, split = w.split, kb0 = w.kb0, kb1 = w.kb1;
+                (void)unit; (void)nb; (void)split;
                 if (warp_wide && kb0 == 0 && kb1 > 0) {
                     // Class tile whose rows are shifted: the sigma elements in front of each row of the first
                     // k-block belong to the previous row of A and are zeroed before the tensor core reads them.
@@ -529,9 +608,11 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
         uint8_t* stg = stage_out + (warp - 2) * kUmmaWarpStagingBytes + lane * kUmmaStageRowBytes;   // this thread's staging row
         unsigned short* srow = reinterpret_cast<unsigned short*>(stg);
         const uintptr_t c_base = reinterpret_cast<uintptr_t>(p.C);
-        for (int unit = unit0; ok && unit < p.num_units; unit += unit_step, ++seq) {
-            int mb, nb, split;
-            decode_unit(p, unit, mb, nb, split);
+        for (int it = 0; ok; ++it, ++seq) {
+            WorkItem w;
+            if (!next_item<SK, B_SPLIT>(p, unit0, unit_step, it, w)) break;
+            const int unit = w.unit, mb = w.mb, nb = w.nb, split = w.split;
+            (void)unit;
             if (!ptx::mbar_wait(tfull_bar + 8u * buf, buf_phase, abort_flag)) { ok = false; break; }
             ptx::tc_fence_after();
             if (warp == 2 && lane == 0) ADAPT_TRACE(4, unit);
@@ -567,7 +648,77 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     if (warp == 2) ADAPT_TRACE(7, unit);
                 }
             };
-            if constexpr (FUSE) {
+            // stream-K: the fp32 partial tiles live in the workspace, one per CTA, [128][BN]; the flag word of a CTA holds
+            // the epoch of the launch whose partial is complete there
+            const int sk_cta = (int)unit0 * CG + (int)cta_rank;
+            if (SK && w.kind == 2 && (seq & 1) == half) {
+                // the slots after this one computed the rest of this tile's k range first thing: wait for their partials
+                bool arrived = true;
+                if (lane == 0) {
+                    for (int j = 1; j <= w.npeers && arrived; ++j) {
+                        const unsigned int* f = p.sk_flags + (sk_cta + j * CG);
+                        uint32_t spins = 0;
+                        uint64_t t0 = 0;
+                        for (;;) {
+                            unsigned int v;
+                            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(f) : "memory");
+                            if (v == p.sk_epoch) break;
+                            if ((++spins & 0x3f) == 0) {
+                                if (*abort_flag) { arrived = false; break; }
+                                const uint64_t now = ptx::globaltimer_ns();
+                                if (t0 == 0) t0 = now;
+                                else if (now - t0 > ptx::kWaitLimitNs) { *abort_flag = 1; arrived = false; break; }
+                            }
+                        }
+                    }
+                }
+                arrived = __shfl_sync(0xffffffffu, arrived ? 1 : 0, 0) != 0;
+                if (!arrived) { ok = false; break; }
+            }
+            // adds the peers' partial values of this thread's row, columns [col, col + 32), in ascending k order
+            auto sk_fixup = [&](uint32_t (&r)[32], int col) {
+                for (int j = 1; j <= w.npeers; ++j) {
+                    // partial tiles are stored [32-column chunk][8-column group][row][8]: a warp's access is 1 KB contiguous
+                    const float4* src = reinterpret_cast<const float4*>(
+                        p.sk_partial + (size_t)(sk_cta + j * CG) * 128 * BN + ((size_t)(col >> 3) * 128 + (size_t)(q * 32 + lane)) * 8);
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) {
+                        const float4 x = __ldcg(src + (v >> 1) * 256 + (v & 1));
+                        r[4 * v + 0] = __float_as_uint(__uint_as_float(r[4 * v + 0]) + x.x);
+                        r[4 * v + 1] = __float_as_uint(__uint_as_float(r[4 * v + 1]) + x.y);
+                        r[4 * v + 2] = __float_as_uint(__uint_as_float(r[4 * v + 2]) + x.z);
+                        r[4 * v + 3] = __float_as_uint(__uint_as_float(r[4 * v + 3]) + x.w);
+                    }
+                }
+            };
+            if (SK && w.kind == 1) {
+                // ---- stream-K: a k range that is not the tile's first: fp32 partial to the workspace, then the flag ----
+                float* mine = p.sk_partial + (size_t)sk_cta * 128 * BN + (size_t)(q * 32 + lane) * 8;
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN; c0 += 32) {
+                    if (n0 + c0 >= p.N) break;                           // uniform; the owner of the tile skips these too
+                    if (((seq * (BN / 32) + (c0 >> 5)) & 1) != half) continue;
+                    uint32_t r[32];
+                    ptx::tmem_ld_32x32(t_row + (uint32_t)c0, r);
+                    ptx::tmem_ld_wait();
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) store_partial8(mine + (size_t)((c0 >> 3) + v) * 128 * 8, r + 8 * v);
+                }
+                release_accumulator();
+                released = true;
+                if (warp == 2 && lane == 0) ADAPT_TRACE(5, unit);
+                // every warp fences its stores and counts itself in; the last one publishes the flag
+                __threadfence();
+                __syncwarp();
+                if (warp == 2 && lane == 0) ADAPT_TRACE(9, unit);
+                if (lane == 0) {
+                    const int old = atomicAdd(sk_count, 1);
+                    if ((old & (kUmmaEpilogueWarps - 1)) == kUmmaEpilogueWarps - 1) {
+                        __threadfence();
+                        asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p.sk_flags + sk_cta), "r"(p.sk_epoch) : "memory");
+                    }
+                }
+            } else if constexpr (FUSE) {
                 // ---- fused split-K: partial -> own shared memory -> sum over the cluster's ranks -> C ----
                 const uint32_t xphase = (uint32_t)(seq & 1);
                 const uint32_t my_rank = ptx::cluster_ctarank();
@@ -713,6 +864,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                                 uint32_t r[32];
                                 ptx::tmem_ld_32x32(t_row + (uint32_t)(off + 64 * pass + 32 * h), r);
                                 ptx::tmem_ld_wait();
+                                if (SK && w.kind == 2) sk_fixup(r, 64 * pass + 32 * h);
                                 if ((pass == PASSES - 1 || x + 64 >= x_end) && (h == 1 || ncols <= 32)) {
                                     // the tile's last read of the accumulator: hand the buffer back now, so the MMA
                                     // of the tile after next starts while this pass is still being packed and stored
@@ -768,6 +920,10 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                             ptx::tmem_ld_32x32(t_row + (uint32_t)c0, r0);
                             if (ncols > 32) ptx::tmem_ld_32x32(t_row + (uint32_t)(c0 + 32), r1);   // uniform
                             ptx::tmem_ld_wait();
+                            if (SK && w.kind == 2) {
+                                sk_fixup(r0, c0);
+                                if (ncols > 32) sk_fixup(r1, c0 + 32);
+                            }
                         }
                         if (warp == 2 && lane == 0) ADAPT_TRACE(5, unit);
                         __syncwarp();                                    // the previous pass has been written out

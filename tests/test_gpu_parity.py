@@ -661,3 +661,55 @@ def test_fused_split_k_matches_the_two_launch_path_bit_for_bit_on_random_values(
             err, mism, n = compare_with_oracle(A, B, C1, M, N, K, dtype)
             assert err <= TOL[dtype]
         ab.adapt_poll_device_status(torch.cuda.current_stream().cuda_stream)
+
+
+# ---- stream-K: the leftover wave's k-blocks shared by all slots, partials fixed up by the tile's owner ---------
+
+def streamk_variants(M, N, K, dtype, lA=ROW, lB=ROW):
+    return [(ab.adapt_matmul_plan_forced(M, N, K, dtype, lA, lB, c.tiling_key), c)
+            for c in ab.adapt_plan_candidates(M, N, K, dtype, lA, lB) if c.streamk]
+
+
+@pytest.mark.parametrize("dtype", [ab.F16, ab.BF16])
+@pytest.mark.parametrize("shape", [(1000, 1024, 1024), (3000, 3000, 512), (300, 520, 1024), (2560, 2048, 2048), (520, 520, 4096),
+                                   (4096, 4096, 256), (5000, 1000, 1000)])
+def test_stream_k_bit_exact(shape, dtype):
+    """Every stream-K configuration (1-CTA and pair tiles, fewer tiles than slots and several waves plus a
+    leftover) against the oracle on position-coded integers, twice in a row on the same workspace."""
+    M, N, K = shape
+    A = synth.position_coded(M, K, dtype, modulus=7, device="cuda")
+    B = synth.position_coded(K, N, dtype, modulus=5, device="cuda").contiguous()
+    variants = streamk_variants(M, N, K, dtype)
+    assert variants, "expected stream-K configurations for this shape"
+    for plan, c in variants:
+        check_case(M, N, K, dtype, A, B, plan=plan, exact=True)
+        check_case(M, N, K, dtype, A, B, plan=plan, exact=True)
+
+
+@pytest.mark.parametrize("lA,lB", [(ROW, COL), (COL, ROW), (COL, COL)])
+def test_stream_k_layouts(lA, lB):
+    M, N, K = 1160, 1000, 1024
+    dtype = ab.BF16
+    A = synth.position_coded(M, K, dtype, 7, "cuda")
+    B = synth.position_coded(K, N, dtype, 5, "cuda")
+    A_st = A.t().contiguous() if lA == COL else A
+    B_st = B.t().contiguous() if lB == COL else B
+    variants = streamk_variants(M, N, K, dtype, lA, lB)
+    assert variants
+    for plan, c in variants:
+        check_case(M, N, K, dtype, A_st, B_st, lA, lB, plan=plan, exact=True)
+
+
+def test_stream_k_random_values_run_twice_bit_identical():
+    for (M, N, K, dtype) in [(4096, 4096, 4096, ab.F16), (3000, 3000, 3000, ab.BF16), (1000, 1024, 1024, ab.F16)]:
+        A = synth.draw_operand(M, K, synth.U11, 31, dtype, "cuda")
+        B = synth.draw_operand(K, N, synth.U11, 32, dtype, "cuda")
+        for plan, c in streamk_variants(M, N, K, dtype)[:4]:
+            C1 = run_library(A, B, M, N, K, dtype, plan=plan).clone()
+            C2 = run_library(A, B, M, N, K, dtype, plan=plan)
+            torch.cuda.synchronize()
+            ab.adapt_poll_device_status(torch.cuda.current_stream().cuda_stream)
+            assert torch.equal(C1.view(torch.int16), C2.view(torch.int16))
+            rows = sample_rows(M, 48, seed=3)
+            err, mism, n = compare_with_oracle(A, B, C1, M, N, K, dtype, rows=rows)
+            assert err <= TOL[dtype], (c.BN, c.family, err)
