@@ -155,6 +155,24 @@ adapt_handle_t adapt_matmul_plan(int64_t M, int64_t N, int64_t K,
  * get different workspaces. */
 adapt_status_t adapt_matmul(adapt_handle_t plan, const void* A, const void* B, void* C, void* cuda_stream);
 
+/* The persisted offline table.  The paper selects configurations offline for a target shape set, registers them in a
+ * hash table and only looks them up online (Section 3.2, Section 5.1); here selection also runs on first sight of a
+ * shape, and these three calls give the offline half back to a deployment that wants it.
+ *
+ * adapt_plan_many: plan `count` shapes in one call (dims: HOST array of 3*count values M, N, K; flags: HOST array of
+ * 3*count values dtype, layoutA, layoutB; handles: optional HOST array of `count` handles to fill).  Returns the
+ * number of shapes planned.
+ * adapt_plan_table_save: write every selected plan of the cache (shape and 64-bit TilingKey, one text line each) to
+ * `path`; returns the number of lines, -1 on error.
+ * adapt_plan_table_load: read such a file and install its TilingKeys as the plans of their shapes, so that the first
+ * online call of a listed shape is already a cache hit and runs exactly the recorded configuration, whatever the
+ * model would choose today.  A shape that already has a plan keeps it; a line whose key is not a legal configuration
+ * of its shape on this machine (another library version, another GPU) is skipped.  Returns the number of plans
+ * installed, -1 if the file cannot be read or is not a table of this library version.  Host work only. */
+int64_t adapt_plan_many(int64_t count, const int64_t* dims, const int32_t* flags, adapt_handle_t* handles);
+int64_t adapt_plan_table_save(const char* path);
+int64_t adapt_plan_table_load(const char* path);
+
 /* The same call for operands that live in HOST memory (A_host, B_host inputs, C_host output,
  * dense, in the plan's layouts; pinned memory makes the copies asynchronous).  The library runs
  * the call on a three-stage pipeline of its own streams (copy A and B into a device staging

@@ -26,7 +26,7 @@ EXPORTS = [
     "adapt_model_pipeline", "adapt_poll_device_status", "adapt_plan_cache_size", "adapt_launch_count",
     "adapt_matmul_noalloc", "adapt_matmul_batch", "adapt_matmul_repeat", "adapt_measure_dispatch",
     "adapt_measure_empty_launch", "adapt_map_encode_count", "adapt_set_map_cache", "adapt_selftest_wait_expiry",
-    "adapt_measure_store_rate",
+    "adapt_measure_store_rate", "adapt_plan_many", "adapt_plan_table_save", "adapt_plan_table_load",
 ]
 
 
@@ -133,6 +133,12 @@ def load():
     lib.adapt_measure_empty_launch.argtypes = [i32, i32, vp, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
     lib.adapt_measure_store_rate.restype = i32
     lib.adapt_measure_store_rate.argtypes = [vp, i64, i64, i32, i32, i32, i32, i32, vp, ctypes.POINTER(dbl)]
+    lib.adapt_plan_many.restype = i64
+    lib.adapt_plan_many.argtypes = [i64, vp, vp, vp]
+    lib.adapt_plan_table_save.restype = i64
+    lib.adapt_plan_table_save.argtypes = [ctypes.c_char_p]
+    lib.adapt_plan_table_load.restype = i64
+    lib.adapt_plan_table_load.argtypes = [ctypes.c_char_p]
     lib.adapt_selftest_wait_expiry.restype = i32
     lib.adapt_selftest_wait_expiry.argtypes = [u64, vp]
     _lib = lib
@@ -222,6 +228,40 @@ def adapt_measure_store_rate(buf_ptr: int, rows: int, cols: int, mode: int, tile
     _check(load().adapt_measure_store_rate(buf_ptr, rows, cols, mode, tile_cols, order, 1 if hint else 0, passes, stream,
                                            ctypes.byref(us)))
     return us.value
+
+
+def adapt_plan_many(shapes):
+    """Plan a list of (M, N, K, dtype[, layoutA, layoutB]) in one call; returns the handles."""
+    n = len(shapes)
+    dims = (ctypes.c_int64 * (3 * n))()
+    flags = (ctypes.c_int32 * (3 * n))()
+    for i, sh in enumerate(shapes):
+        dims[3 * i], dims[3 * i + 1], dims[3 * i + 2] = sh[0], sh[1], sh[2]
+        flags[3 * i] = sh[3]
+        flags[3 * i + 1] = sh[4] if len(sh) > 4 else ROW_MAJOR
+        flags[3 * i + 2] = sh[5] if len(sh) > 5 else ROW_MAJOR
+    handles = (ctypes.c_void_p * n)()
+    planned = load().adapt_plan_many(n, dims, flags, handles)
+    if planned < 0:
+        lib = load()
+        raise AdaptError(lib.adapt_last_error(), lib.adapt_last_error_message().decode())
+    return list(handles)
+
+
+def adapt_plan_table_save(path: str) -> int:
+    n = load().adapt_plan_table_save(path.encode())
+    if n < 0:
+        lib = load()
+        raise AdaptError(lib.adapt_last_error(), lib.adapt_last_error_message().decode())
+    return n
+
+
+def adapt_plan_table_load(path: str) -> int:
+    n = load().adapt_plan_table_load(path.encode())
+    if n < 0:
+        lib = load()
+        raise AdaptError(lib.adapt_last_error(), lib.adapt_last_error_message().decode())
+    return n
 
 
 def adapt_map_encode_count() -> int:

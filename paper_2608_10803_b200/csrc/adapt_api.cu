@@ -65,6 +65,7 @@ constexpr int kMapSlots = 8;   // most recent distinct (pointer, geometry) pairs
 struct adapt_plan_s {
     Shape s;
     Config c;
+    bool selected = false;    // the plan adapt_matmul_plan returns for its shape (not a forced-key plan)
     bool noop = false;        // M == 0 or N == 0
     bool zero_fill = false;   // K == 0
     std::mutex mu;            // guards the tensor-map slots
@@ -140,6 +141,7 @@ struct State {
     std::atomic<int64_t> map_encodes{0};   // tensor maps encoded on the host so far (a cached call encodes none)
     std::atomic<int> map_cache{1};         // 0: every call encodes its maps afresh (measurement of the miss cost)
     int log = 0;
+    int prefetch = 1;                  // L2 prefetch of a kernel's first operands ahead of its dependency wait (ADAPT_PREFETCH=0 turns it off)
     bool class_promo128 = true;        // 128-byte L2 promotion for the strided class views (ADAPT_CLASS_PROMO128=0: 256 as for dense operands)
 };
 
@@ -154,6 +156,7 @@ void apply_env(State& S)
     if (const char* e = getenv("ADAPT_FAMILY_MASK")) S.machine.family_mask = (unsigned)strtoul(e, nullptr, 0);
     if (const char* e = getenv("ADAPT_LOG")) S.log = atoi(e);
     if (const char* e = getenv("ADAPT_NO_PDL")) pdl_enabled() = atoi(e) == 0;
+    if (const char* e = getenv("ADAPT_PREFETCH")) S.prefetch = atoi(e);
     if (const char* e = getenv("ADAPT_CLASS_PROMO128")) S.class_promo128 = atoi(e) != 0;
     if (const char* e = getenv("ADAPT_WORKSPACE_LIMIT_MB")) S.machine.workspace_limit = (int64_t)atoll(e) << 20;
 }
@@ -219,6 +222,45 @@ Plan* make_plan(State& S, const Shape& s, const uint64_t* forced_key)
     return p;
 }
 
+// The plan a shape's adapt_matmul_plan calls return from now on (the caller holds S.mu and has checked that the
+// shape has none yet).
+void insert_selected(State& S, const Shape& s, Plan* p)
+{
+    p->selected = true;
+    S.all_plans.push_back(p);
+    uint64_t w;
+    if (!shape_word(s, &w)) {
+        S.big[State::BigKey(s.M, s.N, s.K, s.dtype, s.layoutA, s.layoutB, 0)] = p;
+        return;
+    }
+    Table* t = S.table.load(std::memory_order_acquire);
+    if (!t || (S.count + 1) * 2 > t->cap) {
+        Table* nt = new Table(t ? t->cap * 2 : (size_t)1 << 14);
+        if (t) {
+            for (size_t i = 0; i < t->cap; ++i) {
+                const uint64_t k = t->keys[i].load(std::memory_order_relaxed);
+                if (k) table_put(nt, k, t->vals[i].load(std::memory_order_relaxed));
+            }
+            S.retired.push_back(t);
+        }
+        S.table.store(nt, std::memory_order_release);
+        t = nt;
+    }
+    table_put(t, w, p);
+    ++S.count;
+}
+
+Plan* find_selected(State& S, const Shape& s)
+{
+    uint64_t w;
+    if (shape_word(s, &w)) {
+        Table* t = S.table.load(std::memory_order_acquire);
+        return t ? table_find(t, w) : nullptr;
+    }
+    auto it = S.big.find(State::BigKey(s.M, s.N, s.K, s.dtype, s.layoutA, s.layoutB, 0));
+    return it == S.big.end() ? nullptr : it->second;
+}
+
 }  // namespace
 
 // ---------------------------------------------------------------------------------------------
@@ -274,22 +316,7 @@ extern "C" adapt_handle_t adapt_matmul_plan(int64_t M, int64_t N, int64_t K, ada
     }
     Plan* p = make_plan(S, s, nullptr);
     if (!p) return nullptr;
-    S.all_plans.push_back(p);
-    if (!small) { S.big[bk] = p; return p; }
-    if (!t || (S.count + 1) * 2 > t->cap) {
-        Table* nt = new Table(t ? t->cap * 2 : (size_t)1 << 14);
-        if (t) {
-            for (size_t i = 0; i < t->cap; ++i) {
-                const uint64_t k = t->keys[i].load(std::memory_order_relaxed);
-                if (k) table_put(nt, k, t->vals[i].load(std::memory_order_relaxed));
-            }
-            S.retired.push_back(t);
-        }
-        S.table.store(nt, std::memory_order_release);
-        t = nt;
-    }
-    table_put(t, w, p);
-    ++S.count;
+    insert_selected(S, s, p);
     return p;
 }
 
@@ -375,6 +402,84 @@ extern "C" int64_t adapt_plan_cache_size(void)
 extern "C" int64_t adapt_launch_count(void) { return st().launches.load(); }
 extern "C" int64_t adapt_map_encode_count(void) { return st().map_encodes.load(); }
 extern "C" void adapt_set_map_cache(int enabled) { st().map_cache.store(enabled ? 1 : 0); }
+
+
+// ---------------------------------------------------------------------------------------------
+// the persisted offline table (Section 3.2: explore offline, look up online)
+// ---------------------------------------------------------------------------------------------
+static const char* kTableHeader = "# adapt_matmul plan table v2: M N K dtype layoutA layoutB tiling_key";
+
+extern "C" int64_t adapt_plan_table_save(const char* path)
+{
+    State& S = st();
+    if (!path) { fail(ADAPT_ERR_INVALID_ARG, "null path%s"); return -1; }
+    FILE* f = fopen(path, "w");
+    if (!f) { fail(ADAPT_ERR_INVALID_ARG, "cannot open %s for writing", path); return -1; }
+    std::lock_guard<std::mutex> lock(S.mu);
+    int64_t n = 0;
+    fprintf(f, "%s\n", kTableHeader);
+    for (Plan* p : S.all_plans) {
+        if (!p->selected || p->noop || p->zero_fill) continue;
+        fprintf(f, "%lld %lld %lld %d %d %d %016llx\n", (long long)p->s.M, (long long)p->s.N, (long long)p->s.K, p->s.dtype,
+                p->s.layoutA, p->s.layoutB, (unsigned long long)pack_tiling_key(p->s, p->c));
+        ++n;
+    }
+    fclose(f);
+    return n;
+}
+
+extern "C" int64_t adapt_plan_table_load(const char* path)
+{
+    State& S = st();
+    if (!path) { fail(ADAPT_ERR_INVALID_ARG, "null path%s"); return -1; }
+    FILE* f = fopen(path, "r");
+    if (!f) { fail(ADAPT_ERR_INVALID_ARG, "cannot open %s", path); return -1; }
+    char line[256];
+    if (!fgets(line, sizeof(line), f) || strncmp(line, kTableHeader, strlen(kTableHeader)) != 0) {
+        fclose(f);
+        fail(ADAPT_ERR_UNSUPPORTED, "%s is not a plan table of this library version", path);
+        return -1;
+    }
+    std::lock_guard<std::mutex> lock(S.mu);
+    if (!S.inited && S.all_plans.empty()) apply_env(S);
+    int64_t loaded = 0;
+    while (fgets(line, sizeof(line), f)) {
+        long long M, N, K;
+        int dt, lA, lB;
+        unsigned long long key;
+        if (line[0] == '#' || sscanf(line, "%lld %lld %lld %d %d %d %llx", &M, &N, &K, &dt, &lA, &lB, &key) != 7) continue;
+        if (M < 1 || N < 1 || K < 1 || M > 2147483647ll || N > 2147483647ll || K > 2147483647ll || (dt | lA | lB) < 0 || dt > 1 || lA > 1 || lB > 1)
+            continue;
+        Shape s;
+        s.M = M; s.N = N; s.K = K; s.dtype = dt; s.layoutA = lA; s.layoutB = lB;
+        if (find_selected(S, s)) continue;                   // a shape keeps the plan it already has
+        // a key is taken over only if it is a legal configuration of this shape on this machine; the selection mask
+        // does not apply (the table's author chose it)
+        Machine saved = S.machine;
+        S.machine.family_mask = 0x1Fu;
+        const uint64_t k64 = (uint64_t)key;
+        Plan* p = make_plan(S, s, &k64);
+        S.machine = saved;
+        if (!p) continue;
+        insert_selected(S, s, p);
+        ++loaded;
+    }
+    fclose(f);
+    return loaded;
+}
+
+extern "C" int64_t adapt_plan_many(int64_t count, const int64_t* dims, const int32_t* flags, adapt_handle_t* handles)
+{
+    if (count < 0 || (count > 0 && (!dims || !flags))) { fail(ADAPT_ERR_INVALID_ARG, "null array%s"); return -1; }
+    int64_t planned = 0;
+    for (int64_t i = 0; i < count; ++i) {
+        adapt_handle_t h = adapt_matmul_plan(dims[3 * i], dims[3 * i + 1], dims[3 * i + 2], (adapt_dtype_t)flags[3 * i],
+                                             (adapt_layout_t)flags[3 * i + 1], (adapt_layout_t)flags[3 * i + 2]);
+        if (handles) handles[i] = h;
+        if (h) ++planned;
+    }
+    return planned;
+}
 
 // ---------------------------------------------------------------------------------------------
 // launch_map: (family, BN, A major, B major) -> compiled kernel
@@ -927,6 +1032,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.raster = (p.P_k == 1 && (double)s.M * (double)s.N >= (double)s.K * ((double)s.M + (double)s.N) &&
                 (s.K >= 32 || p.P_n <= 64 || classesA)) ? 1 : 0;
     if (const char* e = getenv("ADAPT_RASTER")) p.raster = atoi(e);
+    p.prefetch = S.prefetch;
     p.a_shift_any = 0;
     for (int j = 0; j < 16; ++j) p.a_shift_any |= p.a_sigma[j];
     if (p.a_shift_any) p.a_shift_any = 1;
@@ -1026,6 +1132,7 @@ adapt_status_t run_simt(State& S, Plan* pl, const void* A, const void* B, void* 
     p.Np = (int)partial_pitch(s.N);
     p.kb_per_split = (int)ceil_div(ceil_div(s.K, 16), c.P_k);
     p.dtype = s.dtype;
+    p.prefetch = S.prefetch;
     p.C = (unsigned short*)C;
     p.partial = (float*)ws;
     dim3 grid((unsigned)((int64_t)c.P_m * c.P_n), (unsigned)c.P_k, 1);
@@ -1038,7 +1145,7 @@ adapt_status_t run_simt(State& S, Plan* pl, const void* A, const void* B, void* 
 
 adapt_status_t run_cluster(State& S, Plan* pl, const void* A, const void* B, void* C, cudaStream_t stream)
 {
-    if (launch_cluster(pl->s, pl->c, A, B, C, S.d_status, stream) != ADAPT_OK) return fail(ADAPT_ERR_CUDA, "cluster kernel launch failed%s");
+    if (launch_cluster(pl->s, pl->c, A, B, C, S.d_status, stream, S.prefetch) != ADAPT_OK) return fail(ADAPT_ERR_CUDA, "cluster kernel launch failed%s");
     S.launches.fetch_add(1, std::memory_order_relaxed);
     CUDA_TRY(cudaGetLastError());
     return ADAPT_OK;
@@ -1437,6 +1544,7 @@ extern "C" adapt_status_t adapt_matmul_noalloc(int64_t M, int64_t N, int64_t K, 
     p.Np = (int)Np;
     p.kb_per_split = (int)per;
     p.dtype = (int)dtype;
+    p.prefetch = 0;
     p.C = (unsigned short*)C;
     p.partial = scratch;
     const int64_t tiles = ceil_div(M, 64) * ceil_div(N, 64);

@@ -246,6 +246,7 @@ struct SimtParams {
     int P_n, P_k, kb_per_split;  // n tiles; k splits; k-blocks of 16 per split
     int Np;                      // row pitch of the partials (N rounded up to 8)
     int dtype;
+    int prefetch;                // L2 prefetch of the first k steps ahead of the dependency wait
     unsigned short* C;
     float* partial;
 };
@@ -256,12 +257,29 @@ simt_gemm_kernel(const unsigned short* __restrict__ A, const unsigned short* __r
     __shared__ float sA[16][64 + 4];
     __shared__ float sB[16][64 + 4];
     pdl_launch_dependents();
-    pdl_wait();
     const int tid = threadIdx.x;
     const int m0 = (int)(blockIdx.x / p.P_n) * 64, n0 = (int)(blockIdx.x % p.P_n) * 64;
     const int split = blockIdx.y;
     const int k_begin = split * p.kb_per_split * 16;
     const int k_end = min(p.K, k_begin + p.kb_per_split * 16);
+    // Ahead of the wait for the kernel before this one on the stream: ask L2 for the lines the first two k steps
+    // will read (a hint only; the loads proper come after the wait).  A problem this small is mostly the wait for
+    // its first bytes, and this way that wait overlaps the previous kernel's tail.
+    if (p.prefetch) {
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int e = (tid + (it & 3) * 256), k0 = k_begin + (it >> 2) * 16;
+            int am, ak, bn, bk;
+            if (p.a_sk == 1) { ak = e & 15; am = e >> 4; } else { am = e & 63; ak = e >> 6; }
+            if (p.b_sn == 1) { bn = e & 63; bk = e >> 6; } else { bk = e & 15; bn = e >> 4; }
+            // one request per 64-byte stretch of the contiguous dimension is enough
+            if (m0 + am < p.M && k0 + ak < k_end && (((p.a_sk == 1 ? ak : am) & 31) == 0 || (p.a_sk == 1 ? ak : am) == 0))
+                ptx::prefetch_l2(A + (int64_t)(m0 + am) * p.a_sm + (int64_t)(k0 + ak) * p.a_sk);
+            if (n0 + bn < p.N && k0 + bk < k_end && (((p.b_sn == 1 ? bn : bk) & 31) == 0))
+                ptx::prefetch_l2(B + (int64_t)(k0 + bk) * p.b_sk + (int64_t)(n0 + bn) * p.b_sn);
+        }
+    }
+    pdl_wait();
     const int tx = tid & 15, ty = tid >> 4;       // thread's 4 columns: tx*4.., 4 rows: ty*4..
     float acc[4][4];
 #pragma unroll

@@ -47,6 +47,7 @@ struct ClusterParams {
     int CS;                      // CTAs per cluster = pieces of the k range
     int k_per_cta;               // k values per CTA, a multiple of 16
     int ring;                    // raw stages in flight per CTA (1..kClusterMaxRing)
+    int prefetch;                // L2 prefetch of the ring's stages ahead of the dependency wait
     unsigned int* status;        // device status word: bit 0 is set when a bounded wait gave up
 };
 
@@ -110,7 +111,6 @@ cluster_gemm_kernel(const ClusterParams p)
         ptx::fence_barrier_init();
     }
     __syncthreads();
-    pdl_wait();
 
     const uint32_t rank = p.CS > 1 ? cl_rank() : 0u;
     const int tile = (int)(blockIdx.x / (unsigned)p.CS);
@@ -162,6 +162,20 @@ cluster_gemm_kernel(const ClusterParams p)
         cp_meta[j] = mt | ((chunk_live(mt, 64) ? 1u : 0u) << 18);
     }
     const int64_t step_a = A_KC ? 128 : 128 * p.lda, step_b = B_KC ? 128 : 128 * p.ldb;
+    // Ahead of the wait for the kernel before this one on the stream: ask L2 for the lines of the ring's stages (hints
+    // only; the copies proper come after the wait), so that the trip to memory overlaps the previous kernel's tail.
+    if (p.prefetch) {
+#pragma unroll
+        for (int j = 0; j < NCP; ++j) {
+            const uint32_t mt = cp_meta[j];
+            // one request per 128-byte line: chunks 0 and 8 of a row (a row of a stage spans at most two lines)
+            if (!((mt >> 17) & 1) || !((mt >> 18) & 1) || ((mt & 15) != 0 && (mt & 15) != 8)) continue;
+            const char* src = cp_src[j];
+            const int64_t step = ((mt >> 8) & 255) < 64 ? step_a : step_b;
+            for (int s = 0; s < S && s < n_stages; ++s) ptx::prefetch_l2(src + s * step);
+        }
+    }
+    pdl_wait();
     auto issue_stage = [&](int slot, int k0) {
         const int kv = k_end - k0;
 #pragma unroll
@@ -412,7 +426,7 @@ inline int cluster_max_size()
 
 // Host launcher.  c.cluster = CS; c.stages = depth of the raw ring; the grid is CS CTAs per tile, the cluster spans blockIdx.x.
 inline adapt_status_t launch_cluster(const Shape& s, const Config& c, const void* A, const void* B, void* C,
-                                     unsigned int* status, cudaStream_t stream)
+                                     unsigned int* status, cudaStream_t stream, int prefetch = 1)
 {
     ClusterParams p;
     p.A = (const unsigned short*)A;
@@ -426,6 +440,7 @@ inline adapt_status_t launch_cluster(const Shape& s, const Config& c, const void
     p.CS = c.cluster;
     p.k_per_cta = (int)round_up(ceil_div(s.K, c.cluster), 16);
     p.ring = c.stages;
+    p.prefetch = prefetch;
     p.status = status;
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));

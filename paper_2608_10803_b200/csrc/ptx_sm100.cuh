@@ -159,6 +159,17 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const void* tmap,
         ::"r"(dst), "l"(tmap), "r"(bar), "r"(x), "r"(y)
         : "memory");
 }
+// Prefetch of one box into L2: no shared-memory destination, no completion to wait for.  A hint only, so it may be
+// issued before the data dependences of the kernel are resolved (L2 is the point of coherence: later writes to the
+// same lines by other kernels update what was prefetched).
+__device__ __forceinline__ void tma_prefetch_2d(const void* tmap, int x, int y)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tmap), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void prefetch_l2(const void* p)
+{
+    asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
+}
 // Bulk copy shared -> global (no tensor map): both addresses 16-byte aligned, size a multiple of 16.
 // Completion is tracked per thread in bulk groups.
 __device__ __forceinline__ void bulk_store(void* gdst, uint32_t ssrc, uint32_t bytes)

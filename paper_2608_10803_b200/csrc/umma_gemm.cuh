@@ -54,6 +54,7 @@ struct UmmaParams {
     int c_mode;                      // 16-bit output: 0 = stores by the epilogue threads (any N, any alignment),
                                      // 1 = TMA stores through the maps of C (rows of C, or of the tile's row class,
                                      //     start on 32-byte boundaries; class tiles with 16 halo columns shift them there)
+    int prefetch;                    // ask L2 for the first unit's operand boxes before waiting for the kernel ahead on the stream
     int raster;                      // tile visiting order: 0 = m-fastest inside groups of kGroupM m-blocks (operand reuse in L2),
                                      // 1 = n-fastest, row block by row block (write-bound shapes: neighbouring CTAs write
                                      //     neighbouring column blocks of the same rows, and a CTA's consecutive class tiles share their maps)
@@ -382,13 +383,43 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
     }
     ptx::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
+    const int unit0 = (CG == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+    const int unit_step = (CG == 2) ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+
+    // While the kernel ahead of this one on the stream drains, ask L2 for the operand boxes of this CTA's first unit
+    // (up to one ring of k-blocks).  Prefetches are hints: they bring lines (and address translations) in early and
+    // commit to nothing, so they may run ahead of griddepcontrol.wait; the loads proper still come after it.  A problem
+    // of a few tiles spends most of its time waiting for its first bytes (2.5 to 5 us from a cold buffer), and with
+    // programmatic dependent launch that wait now overlaps the previous kernel.
+    if (warp == 0 && !B_CLS && p.prefetch) {
+        constexpr int NREQ_A = A_MN ? 2 : 1;
+        constexpr int NREQ = NREQ_A + (B_MN ? B_BOXES : 1);
+        WorkItem w;
+        if (lane < NREQ && next_item<SK, B_SPLIT>(p, unit0, unit_step, 0, w)) {
+            const int cls = A_CLS ? (w.mb % NCLS) : 0;
+            const int row0 = A_CLS ? (w.mb / NCLS) * 128 : w.mb * (128 * CG) + (int)cta_rank * 128;
+            const int kshift = A_CLS ? p.a_sigma[cls] : 0;
+            const int a_k_off = B_SPLIT ? (w.split & 7) * p.cls_kc : 0;
+            const int col0 = w.nb * TILE_N + (int)cta_rank * BN_CTA;
+            const int jb = lane - NREQ_A;
+            for (int kb = w.kb0; kb < w.kb1 && kb < w.kb0 + S; ++kb) {
+                const int k0 = kb * kUmmaBK;
+                if (lane < NREQ_A) {
+                    if (!A_MN) ptx::tma_prefetch_2d(&maps.a[cls], k0 + a_k_off, row0);
+                    else ptx::tma_prefetch_2d(&maps.a[cls], row0 + lane * 64, k0);
+                } else {
+                    const CUtensorMap* tmB = &maps.b[B_SPLIT ? (w.split & 7) : 0];
+                    if (B_MN) ptx::tma_prefetch_2d(tmB, col0 + jb * 64, k0 - kshift);
+                    else ptx::tma_prefetch_2d(tmB, k0, col0);
+                }
+            }
+        }
+    }
+
     // set-up done: from here on the kernel reads and writes global memory
     if (threadIdx.x == 0) ADAPT_TRACE(12, 0);
     pdl_wait();
     if (threadIdx.x == 0) ADAPT_TRACE(13, 0);
-
-    const int unit0 = (CG == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
-    const int unit_step = (CG == 2) ? (int)(gridDim.x >> 1) : (int)gridDim.x;
 
     if (warp == 0) {
         // ------------------------------ producer -----------------------------------------------

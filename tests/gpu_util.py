@@ -11,14 +11,8 @@ from paper_2608_10803_b200 import synth
 
 TOL = {ab.F16: 1e-3, ab.BF16: 8e-3}     # normwise ||C - C_ref||_F / ||C_ref||_F, norms in fp64
 
-_inited = False
-
-
 def init():
-    global _inited
-    if not _inited:
-        ab.adapt_init(0)
-        _inited = True
+    ab.adapt_init(0)        # idempotent, and a test elsewhere may have shut the library down
 
 
 def run_library(A: torch.Tensor, B: torch.Tensor, M: int, N: int, K: int, dtype: int,

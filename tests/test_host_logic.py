@@ -241,3 +241,56 @@ def test_sweep_csv_matches_recipe():
     assert shapes == synth.sweep_shapes()
     assert shapes[:5] == [(7409, 156, 19633), (3067, 2, 75528), (6392, 8517, 4), (178, 71, 43035), (1657, 12995, 164)]
     assert len(synth.sweep_oracle_subset()) == 200
+
+
+# ---- the persisted offline table (Section 3.2: explore offline, look up online) ---------------------
+
+def test_plan_table_round_trip_and_override(tmp_path):
+    """Plans saved to a table come back with the same TilingKeys in a fresh cache; a table may name any legal
+    configuration of a shape (not only the model's pick) and the online lookup then returns exactly that one;
+    lines that are not legal for their shape are skipped; a shape that already has a plan keeps it."""
+    ab.adapt_shutdown()
+    shapes = [(1000, 1024, 1024, ab.F16), (7, 1024, 1024, ab.F16), (131, 77, 259, ab.BF16), (4096, 4096, 512, ab.BF16),
+              (3, 256, 87087, ab.F16), ((1 << 20) + 3, 8, 24, ab.BF16)]
+    handles = ab.adapt_plan_many(shapes)
+    assert all(handles)
+    keys = [ab.adapt_plan_info(h).tiling_key for h in handles]
+    ab.adapt_matmul_plan(0, 5, 5, ab.F16)            # no-op and zero-fill plans are not part of the table
+    ab.adapt_matmul_plan(5, 5, 0, ab.F16)
+    path = str(tmp_path / "plans.txt")
+    assert ab.adapt_plan_table_save(path) == len(shapes)
+
+    ab.adapt_shutdown()
+    assert ab.adapt_plan_cache_size() == 0
+    assert ab.adapt_plan_table_load(path) == len(shapes)
+    assert ab.adapt_plan_cache_size() == len(shapes)
+    for sh, k in zip(shapes, keys):
+        assert ab.adapt_plan_info(ab.adapt_matmul_plan(*sh)).tiling_key == k
+    assert ab.adapt_plan_cache_size() == len(shapes)  # every lookup was a hit
+    assert ab.adapt_plan_table_load(path) == 0        # shapes that have a plan keep it
+
+    # a hand-written table: the second-best configuration of one shape, one illegal key, one malformed line
+    ab.adapt_shutdown()
+    M, N, K, dt = 1000, 1024, 1024, ab.F16
+    cands = ab.adapt_plan_candidates(M, N, K, dt)
+    second = cands[1]
+    assert second.tiling_key != cands[0].tiling_key
+    lines = open(path).read().splitlines()
+    with open(path, "w") as f:
+        f.write(lines[0] + "\n")
+        f.write(f"{M} {N} {K} {dt} 0 0 {second.tiling_key:016x}\n")
+        f.write(f"64 64 64 0 0 0 {second.tiling_key:016x}\n")     # a 1000-row plan's key on a 64^3 shape: stages / P_k do not fit
+        f.write("this is not a plan\n")
+        f.write(f"-5 64 64 0 0 0 {second.tiling_key:016x}\n")
+    n = ab.adapt_plan_table_load(path)
+    assert n in (1, 2)
+    assert ab.adapt_plan_info(ab.adapt_matmul_plan(M, N, K, dt)).tiling_key == second.tiling_key
+
+    # not a table of this library
+    with open(path, "w") as f:
+        f.write("# some other file\n1 2 3\n")
+    with pytest.raises(ab.AdaptError):
+        ab.adapt_plan_table_load(path)
+    with pytest.raises(ab.AdaptError):
+        ab.adapt_plan_table_load(str(tmp_path / "missing.txt"))
+    ab.adapt_shutdown()
