@@ -719,17 +719,24 @@ def validate_model(args):
     from paper_2608_10803_b200 import synth
     ab.adapt_init(0)
     st = torch.cuda.current_stream().cuda_stream
-    cases = synth.config_sweep()
-    rng = np.random.default_rng(7)
-    order = [int(i) for i in rng.permutation(len(cases))]
+    if args.validate_heldout:
+        # a second shape set drawn with the sweep's recipe from another seed: no model constant was fitted on it
+        cases = synth.sweep_like(args.validate_heldout, 4 * args.validate_model + 200)
+        order = list(range(len(cases)))
+    else:
+        cases = synth.config_sweep()
+        rng = np.random.default_rng(7)
+        order = [int(i) for i in rng.permutation(len(cases))]
     picked = [i for i in order if args.validate_roof_us * 1e-6 <= t_roof_nominal(cases[i]) and cases[i].bytes < 3e9][: args.validate_model]
     cand_rows = []
-    hits, regrets, rows = 0, [], []
+    hits, exact, cut, regrets, rows = 0, 0, 0, [], []
     for i in picked:
         c = cases[i]
         A, B = synth.draw_case(c, "cuda")
         C = torch.empty((c.M, c.N), dtype=A.dtype, device="cuda")
-        cands = ab.adapt_plan_candidates(c.M, c.N, c.K, c.dtype)[:48]
+        all_cands = ab.adapt_plan_candidates(c.M, c.N, c.K, c.dtype)
+        cands = all_cands[:args.validate_cap]
+        cut += int(len(all_cands) > len(cands))
         times = []
         for cand in cands:
             plan = ab.adapt_matmul_plan_forced(c.M, c.N, c.K, c.dtype, 0, 0, cand.tiling_key)
@@ -744,21 +751,27 @@ def validate_model(args):
             torch.cuda.synchronize()
             times.append(e0.elapsed_time(e1) / reps * 1e3)
         for cand, t in zip(cands, times):
-            cand_rows.append((c.M, c.N, c.K, c.dtype, ab.FAMILY_NAMES[cand.family], cand.BN, cand.stages, cand.P_k, cand.srcA,
-                              cand.srcB, cand.predicted_us, cand.t_pro_us, cand.t_main_us, cand.t_epi_us, t))
+            cand_rows.append((c.M, c.N, c.K, c.dtype, ab.FAMILY_NAMES[cand.family], cand.BN, cand.stages, cand.P_k, cand.cluster, cand.fused,
+                              cand.streamk, cand.srcA, cand.srcB, cand.predicted_us, cand.t_pro_us, cand.t_main_us, cand.t_epi_us, t))
         best = int(np.argmin(times))
         hits += int(best == 0 or times[0] <= 1.02 * times[best])
+        exact += int(best == 0)
         regrets.append(times[0] / times[best])
         rows.append((c.M, c.N, c.K, len(cands), times[0], times[best], cands[0].predicted_us))
         del A, B, C
-    out = {"model_validation": {"shapes": len(picked), "top1_hit_rate_within_2pct": hits / max(1, len(picked)),
-                                "mean_regret": float(np.mean(regrets)), "max_regret": float(np.max(regrets)),
+    out = {"model_validation": {"shapes": len(picked), "set": f"held-out, seed {args.validate_heldout}" if args.validate_heldout else "sweep (the set the constants were fitted on)",
+                                "min_t_roof_us": args.validate_roof_us,
+                                "exact_hit_rate": exact / max(1, len(picked)),
+                                "top1_hit_rate_within_2pct": hits / max(1, len(picked)),
+                                "mean_regret": float(np.mean(regrets)), "p95_regret": float(np.percentile(regrets, 95)),
+                                "max_regret": float(np.max(regrets)),
                                 "geomean_regret": geomean(regrets),
+                                "candidates_timed_per_shape_cap": args.validate_cap, "shapes_with_more_candidates_than_cap": cut,
                                 "note": "regret = time of the model's pick / time of the fastest legal configuration; the paper reports 63.86 % exact hits on its own hardware"}}
     print(json.dumps(out))
     if args.dump_candidates:
         with open(args.dump_candidates, "w") as f:
-            f.write("M,N,K,dtype,family,BN,stages,P_k,srcA,srcB,pred_us,t_pro,t_main,t_epi,time_us\n")
+            f.write("M,N,K,dtype,family,BN,stages,P_k,cluster,fused,streamk,srcA,srcB,pred_us,t_pro,t_main,t_epi,time_us\n")
             for r in cand_rows:
                 f.write(",".join(f"{x:.3f}" if isinstance(x, float) else str(x) for x in r) + "\n")
     if args.dump:
@@ -787,6 +800,8 @@ def main():
     ap.add_argument("--vendor", action="store_true", help="also time torch.matmul (cuBLAS) per shape as a vendor reference")
     ap.add_argument("--validate-model", type=int, default=0,
                     help="time every legal configuration of this many seeded sweep shapes and report how often the model's pick is the fastest")
+    ap.add_argument("--validate-heldout", type=int, default=0, help="with --validate-model: draw the shapes with the sweep's recipe from this seed instead of from the sweep")
+    ap.add_argument("--validate-cap", type=int, default=128, help="with --validate-model: time at most this many candidates per shape (best predicted first)")
     ap.add_argument("--validate-roof-us", type=float, default=5.0, help="with --validate-model: only shapes whose nominal roofline time is at least this")
     ap.add_argument("--dump-candidates", default="", help="with --validate-model: write every timed configuration (prediction and time) to this CSV")
     ap.add_argument("--ref-macs", type=float, default=5e10, help="with --impl reference: multiply-accumulates of the oracle's bounded sample per step")

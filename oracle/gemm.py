@@ -55,6 +55,9 @@ def _load():
         lib.oracle_gemm_rows.restype = ctypes.c_int
         lib.oracle_gemm_rows.argtypes = [ctypes.c_int64] * 3 + [ctypes.c_int] * 3 + [
             u16p, u16p, i64p, ctypes.c_int64, f64p, u16p, ctypes.c_int]
+        lib.oracle_addmm_rows.restype = ctypes.c_int
+        lib.oracle_addmm_rows.argtypes = [ctypes.c_int64] * 3 + [ctypes.c_int] * 3 + [
+            u16p, u16p, u16p, ctypes.c_int, ctypes.c_double, ctypes.c_double, i64p, ctypes.c_int64, f64p, u16p, ctypes.c_int]
         lib.oracle_decode16_array.argtypes = [u16p, f64p, ctypes.c_size_t, ctypes.c_int]
         lib.oracle_encode16_array.argtypes = [f64p, u16p, ctypes.c_size_t, ctypes.c_int]
         lib.oracle_fro_accumulate.argtypes = [u16p, f64p, ctypes.c_size_t, ctypes.c_int,
@@ -125,6 +128,34 @@ def gemm_rows(A_bits, B_bits, M: int, N: int, K: int, dtype: int,
 def gemm(A_bits, B_bits, M, N, K, dtype, layoutA=ROW_MAJOR, layoutB=ROW_MAJOR, nthreads=0):
     """Whole product.  Returns (C64, C16)."""
     return gemm_rows(A_bits, B_bits, M, N, K, dtype, layoutA, layoutB, None, True, nthreads)
+
+
+def addmm_rows(A_bits, B_bits, D_bits, M: int, N: int, K: int, dtype: int, alpha: float, beta: float,
+               layoutA: int = ROW_MAJOR, layoutB: int = ROW_MAJOR, rows=None, nthreads: int = 0):
+    """Rows ``rows`` (default: all) of alpha * (A*B) + beta * D (Section 6.5's AddMM operator), D either M x N
+    or a row of N values (a bias, recognised by its size).  alpha and beta are taken at their binary32 values.
+    Returns (O64, O16)."""
+    A = _u16(A_bits).reshape(-1)
+    B = _u16(B_bits).reshape(-1)
+    D = _u16(D_bits).reshape(-1)
+    if A.size != M * K or B.size != K * N or D.size not in (N, M * N):
+        raise ValueError("operand size does not match (M, N, K)")
+    is_vec = 1 if D.size == N else 0      # with M == 1 the two readings coincide
+    if rows is None:
+        rows_arr, nrows = None, M
+    else:
+        rows_arr = np.ascontiguousarray(rows, dtype=np.int64)
+        nrows = rows_arr.size
+    O64 = np.zeros((nrows, N), dtype=np.float64)
+    O16 = np.zeros((nrows, N), dtype=np.uint16)
+    rc = _load().oracle_addmm_rows(
+        M, N, K, dtype, layoutA, layoutB, _ptr(A, ctypes.c_uint16), _ptr(B, ctypes.c_uint16), _ptr(D, ctypes.c_uint16), is_vec,
+        float(np.float32(alpha)), float(np.float32(beta)),
+        _ptr(rows_arr, ctypes.c_int64) if rows_arr is not None else None, nrows,
+        _ptr(O64, ctypes.c_double), _ptr(O16, ctypes.c_uint16), nthreads)
+    if rc != 0:
+        raise ValueError("oracle_addmm_rows rejected its arguments")
+    return O64, O16
 
 
 def rel_fro_error(C_got_bits, C_ref64, dtype: int):

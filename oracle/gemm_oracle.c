@@ -248,3 +248,41 @@ int oracle_max_threads(void)
     return 1;
 #endif
 }
+
+/* ---- the fused-add operator (an extension; the functions above are untouched) ----------- */
+
+/*
+ * Rows rows[0..nrows) of   Out = alpha * (A * B) + beta * D,
+ * the AddMM operator the paper lists beside MatMul among the operators it replaces
+ * (Section 6.5).  The product is the binary64 sum of oracle_gemm_rows (ascending k); alpha and
+ * beta are binary64 (the caller passes the exact values of the binary32 scalars the library
+ * takes); D holds 16-bit words of the same type as A and B and is either a full M x N row-major
+ * matrix (d_is_vector == 0) or one row of N values added to every output row (d_is_vector != 0,
+ * a bias).  One multiplication and one addition per term, in binary64, then ONE rounding to the
+ * 16-bit type: out64 = alpha * sum + beta * d.  O64 / O16 as in oracle_gemm_rows.
+ */
+int oracle_addmm_rows(int64_t M, int64_t N, int64_t K, int dtype, int layoutA, int layoutB,
+                      const uint16_t* A, const uint16_t* B, const uint16_t* D, int d_is_vector,
+                      double alpha, double beta,
+                      const int64_t* rows, int64_t nrows,
+                      double* O64, uint16_t* O16, int nthreads)
+{
+    if (nrows < 0 || N < 0 || !D) return -1;
+    if (nrows == 0 || N == 0) return 0;
+    double* sum = (double*)__builtin_malloc((size_t)nrows * (size_t)N * sizeof(double));
+    if (!sum) return -1;
+    int rc = oracle_gemm_rows(M, N, K, dtype, layoutA, layoutB, A, B, rows, nrows, sum, NULL, nthreads);
+    if (rc == 0) {
+        for (int64_t r = 0; r < nrows; ++r) {
+            int64_t i = rows ? rows[r] : r;
+            for (int64_t j = 0; j < N; ++j) {
+                double d = oracle_decode16(d_is_vector ? D[j] : D[(size_t)i * (size_t)N + (size_t)j], dtype);
+                double v = alpha * sum[(size_t)r * (size_t)N + (size_t)j] + beta * d;
+                if (O64) O64[(size_t)r * (size_t)N + (size_t)j] = v;
+                if (O16) O16[(size_t)r * (size_t)N + (size_t)j] = oracle_encode16(v, dtype);
+            }
+        }
+    }
+    __builtin_free(sum);
+    return rc;
+}

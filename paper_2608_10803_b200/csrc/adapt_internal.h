@@ -30,7 +30,20 @@ inline int umma_cluster_slots(const Machine& m, int cluster)
 // ---- calibration constants of the latency model (Eq. 8: lambda_r, eta_r, BW_r) ------------
 // Measured on B200 with this library's own kernels (CUDA events); the paper's values are for
 // other hardware and are not printed, so these are this library's.
+// Variant groups of the last calibration step: after the terms of Eq. 7 are added up, the prediction of a configuration is
+// scaled by the factor of its group, the geometric mean of measured / predicted time over every timed configuration of
+// that group in the fitting set (paper_2608_10803_b200/calibrate.py computes the table from the CSV that
+// `bench.py --validate-model N --dump-candidates` writes).  The terms rank the configurations inside a group; the factors
+// put the groups, whose kernels differ in what the terms leave out, on one scale.
+constexpr int kCalibGroups = 40;
+struct Config;
+int calib_group(const Config& c);
+
 struct Calib {
+    // fitted on 34,000 timed configurations of 500 sweep shapes (every legal configuration within 3x of its shape's best)
+    double group_bias[kCalibGroups] = {
+        0.718, 0.750, 0.901, 0.909, 1.006, 0.912, 0.878, 1.032, 1.003, 0.984, 0.996, 1.040, 1.191, 0.483, 0.581, 1.004, 1.165, 0.853, 0.979, 1.000,
+        0.746, 0.791, 0.911, 0.935, 1.000, 0.877, 1.000, 1.000, 1.000, 1.000, 1.000, 1.034, 1.000, 1.000, 1.000, 1.000, 1.000, 1.000, 1.000, 1.000};
     double launch_us = 3.0;             // one kernel launch issued back to back on a stream (also per reduce launch)
     double prologue_launch_us = 0.3;    // a re-pitch / regroup launch ahead of the GEMM: its launch overlaps the GEMM's own
                                         // (programmatic dependent launch); fit over 910 timed small configurations: -0.2 us
@@ -57,7 +70,8 @@ struct Calib {
     double simt_step_us = 0.8;          // one 16-k step of a CTA alone on its SM (15 x 30 x 32: two steps, 4.85 us with the launch)
     double halo_edge_tile_us = 0.8;     // row heads or tails of one halo tile (up to 15 elements per row, aligned stores of 2 to 16 bytes)
     double simt_bw_eff = 0.15;          // fraction of hbm_bw its 2-byte accesses reach (K = 1 outer products: 0.13 measured)
-    double skinny_bw_eff_aligned = 0.32;    // fraction of hbm_bw the warp-level streaming kernel reaches, 16-byte aligned rows
+    double skinny_bw_eff_aligned = 0.55;    // fraction of hbm_bw the warp-level streaming kernel reaches, 16-byte aligned rows
+                                            // (16 x 65536 x 4096: 3.5 TB/s with its loads four steps ahead of the MMAs, 1.6 before)
     double skinny_bw_eff_unaligned = 0.10;  // ... rows assembled from two chunks
     double skinny_fixed_us = 2.0;
     double skinny_pass_us = 5.5;        // one 64-row pass over one staged chunk when the streamed rows are k-contiguous

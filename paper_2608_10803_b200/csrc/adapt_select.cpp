@@ -120,10 +120,30 @@ static int64_t outerA(const Shape& s) { return s.layoutA == ADAPT_ROW_MAJOR ? s.
 static int64_t innerB(const Shape& s) { return s.layoutB == ADAPT_ROW_MAJOR ? s.N : s.K; }
 static int64_t outerB(const Shape& s) { return s.layoutB == ADAPT_ROW_MAJOR ? s.K : s.N; }
 
+// Group of a configuration for the last calibration factor: kernel family, tiling mode, and which extra launches
+// (prologue, reduction) or in-kernel exchanges (fused reduction, stream-K) it has.  Pair tiles: + 20.
+int calib_group(const Config& c)
+{
+    const bool pro = c.srcA == ADAPT_SRC_PAD_COPY || c.srcB == ADAPT_SRC_PAD_COPY;
+    int g;
+    switch (c.family) {
+        case ADAPT_FAM_SKINNY: return c.P_k == 1 ? 13 : 14;
+        case ADAPT_FAM_SIMT: return c.P_k == 1 ? 15 : 16;
+        case ADAPT_FAM_CLUSTER: return c.cluster == 1 ? 17 : 18;
+        default: break;
+    }
+    if (c.srcB == ADAPT_SRC_TMA_CLASSES) g = c.BN == 64 ? 10 : (c.fused ? 12 : 11);
+    else if (c.srcA == ADAPT_SRC_TMA_CLASSES) g = c.BN % 64 ? 9 : (c.fused ? 8 : (c.P_k == 1 ? 6 : 7));
+    else if (c.fused) g = 4;
+    else if (c.streamk) g = 5;
+    else g = (c.P_k == 1 ? 0 : 2) + (pro ? 1 : 0);
+    return g + (c.family == ADAPT_FAM_UMMA_2CTA ? 20 : 0);
+}
+
 static void finish_common(const Shape& s, Config& c, const Calib& cal)
 {
     c.workspace_bytes = c.ws_padA + c.ws_padB + c.ws_partial;
-    c.predicted_us = cal.launch_us + c.t_pro_us + c.t_main_us + c.t_epi_us;
+    c.predicted_us = (cal.launch_us + c.t_pro_us + c.t_main_us + c.t_epi_us) * cal.group_bias[calib_group(c)];
     (void)s;
 }
 

@@ -184,13 +184,14 @@ skinny_gemm_kernel(const SkinnyParams p)
             // short k range still keeps all of them busy
             const int k_sub = ((min(kSkinnyKChunk, k_end - kc0) + WK - 1) / WK + 15) & ~15;
             const int kw0 = kc0 + wk * k_sub;
-            // a lane loads rows k+2t, +1, +8, +9 at columns r_warp + 8g .. +7
-#pragma unroll 2
-            for (int ks = 0; ks < k_sub; ks += 16) {
-                const int k = kw0 + ks;
-                if (k >= k_end) break;
+            // a lane loads rows k+2t, +1, +8, +9 at columns r_warp + 8g .. +7.  The loads run kDepth steps ahead of the
+            // MMAs that use them (register ring, indices fixed by full unrolling): with the loads of a step consumed in
+            // the same step a lane had one trip to memory in flight and the kernel streamed at a quarter of the HBM rate
+            const int k_lim = min(k_end, kw0 + k_sub);
+            const int n_steps = kw0 < k_lim ? (k_lim - kw0 + 15) >> 4 : 0;
+            auto load_step = [&](int step, uint4 (&v)[4]) {
+                const int k = kw0 + 16 * step;
                 const int kr[4] = {k + 2 * t, k + 2 * t + 1, k + 2 * t + 8, k + 2 * t + 9};
-                uint4 v[4];
                 if (cols_full && k + 16 <= k_end) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) v[i] = load8<ALIGNED>(p.Str + (int64_t)kr[i] * p.ld + (r_warp + 8 * g));
@@ -201,7 +202,9 @@ skinny_gemm_kernel(const SkinnyParams p)
                         if (kr[i] < k_end && nv > 0) v[i] = load8_edge(p.Str + (int64_t)kr[i] * p.ld + (r_warp + 8 * g), nv);
                     }
                 }
-                const int kl = k - kc0 + 2 * t;          // position inside the staged chunk
+            };
+            auto mma_step = [&](int step, const uint4 (&v)[4]) {
+                const int kl = kw0 + 16 * step - kc0 + 2 * t;      // position inside the staged chunk
                 const uint32_t a0 = *reinterpret_cast<const uint32_t*>(&s_small[g][kl]);
                 const uint32_t a1 = *reinterpret_cast<const uint32_t*>(&s_small[g + 8][kl]);
                 const uint32_t a2 = *reinterpret_cast<const uint32_t*>(&s_small[g][kl + 8]);
@@ -212,6 +215,20 @@ skinny_gemm_kernel(const SkinnyParams p)
                     const uint32_t b0 = __byte_perm(word_of(v[0], j >> 1), word_of(v[1], j >> 1), sel);
                     const uint32_t b1 = __byte_perm(word_of(v[2], j >> 1), word_of(v[3], j >> 1), sel);
                     mma_16816<BF16>(acc[j], a0, a1, a2, a3, b0, b1);
+                }
+            };
+            constexpr int kDepth = 4;
+            uint4 ring[kDepth][4];
+#pragma unroll
+            for (int d = 0; d < kDepth; ++d)
+                if (d < n_steps) load_step(d, ring[d]);
+            for (int st = 0; st < n_steps; st += kDepth) {
+#pragma unroll
+                for (int d = 0; d < kDepth; ++d) {
+                    if (st + d < n_steps) {
+                        mma_step(st + d, ring[d]);
+                        if (st + d + kDepth < n_steps) load_step(st + d + kDepth, ring[d]);
+                    }
                 }
             }
         }

@@ -128,6 +128,12 @@ def config_sweep():
             for i, (M, N, K) in enumerate(sweep_shapes())]
 
 
+def sweep_like(seed: int, count: int):
+    """A second shape set drawn with the sweep's recipe from another seed (held-out shapes for the model check)."""
+    shapes, _ = draw_sweep_shapes(count, seed)
+    return [_case(7, i, M, N, K, F16 if i % 2 == 0 else BF16, U11, U11) for i, (M, N, K) in enumerate(shapes)]
+
+
 def sweep_oracle_subset(count: int = 200, seed: int = 43, total: int = 2000):
     """Indices of the sweep shapes that are checked against the oracle."""
     return sorted(int(i) for i in np.random.default_rng(seed).choice(total, count, replace=False))
