@@ -226,6 +226,24 @@ adapt_status_t adapt_matmul_noalloc(int64_t M, int64_t N, int64_t K, adapt_dtype
 adapt_status_t adapt_matmul_batch(int64_t count, const adapt_handle_t* plans, const void* const* A,
                                   const void* const* B, void* const* C, void* cuda_stream);
 
+/* The other operators the paper replaces beside MatMul (Section 6.5 and the Conclusion: AddMM, BatchMM, GroupMM), on the
+ * same plans.  GroupMM, a list of GEMMs of different shapes, is adapt_matmul_batch above.
+ *
+ * adapt_addmm:  C = alpha * (A * B) + beta * D, with the product accumulated in fp32 as in adapt_matmul, the scaling and
+ * the addition done in fp32 on the accumulated sum, and ONE round-to-nearest-even cast to the 16-bit output.  D (DEVICE,
+ * same 16-bit type) is an M x N row-major matrix (d_is_vector == 0) or one row of N values added to every output row
+ * (d_is_vector != 0, a bias).  C may be D itself (in-place beta * C + alpha * A * B); it must not overlap A, B, or D in
+ * any other way.  The GEMM kernels leave their fp32 sums in the workspace (as a split-K call does) and the fixed-order
+ * reduction kernel applies alpha, beta and D before the cast, so the result is as reproducible as adapt_matmul's; plans
+ * of the warp-level and one-launch families run on the CUDA-core kernel for this call.  K == 0 gives beta * D.
+ *
+ * adapt_matmul_strided_batch:  `batch` GEMMs of the plan's shape on operands stride_a, stride_b, stride_c ELEMENTS apart
+ * (a stride of 0 shares that input across the batch; stride_c must be at least M * N), enqueued in batch order on the stream. */
+adapt_status_t adapt_addmm(adapt_handle_t plan, const void* A, const void* B, const void* D, int d_is_vector,
+                           float alpha, float beta, void* C, void* cuda_stream);
+adapt_status_t adapt_matmul_strided_batch(adapt_handle_t plan, const void* A, int64_t stride_a, const void* B, int64_t stride_b,
+                                          void* C, int64_t stride_c, int64_t batch, void* cuda_stream);
+
 /* Harness support: `calls` back-to-back adapt_matmul calls of one plan, call i on operand set i % sets
  * (A, B, C: HOST arrays of `sets` device pointers).  Used to time one shape with rotating buffers. */
 adapt_status_t adapt_matmul_repeat(adapt_handle_t plan, int sets, const void* const* A, const void* const* B,

@@ -27,6 +27,7 @@ EXPORTS = [
     "adapt_matmul_noalloc", "adapt_matmul_batch", "adapt_matmul_repeat", "adapt_measure_dispatch",
     "adapt_measure_empty_launch", "adapt_map_encode_count", "adapt_set_map_cache", "adapt_selftest_wait_expiry",
     "adapt_measure_store_rate", "adapt_plan_many", "adapt_plan_table_save", "adapt_plan_table_load",
+    "adapt_addmm", "adapt_matmul_strided_batch",
 ]
 
 
@@ -133,6 +134,10 @@ def load():
     lib.adapt_measure_empty_launch.argtypes = [i32, i32, vp, ctypes.POINTER(dbl), ctypes.POINTER(dbl)]
     lib.adapt_measure_store_rate.restype = i32
     lib.adapt_measure_store_rate.argtypes = [vp, i64, i64, i32, i32, i32, i32, i32, vp, ctypes.POINTER(dbl)]
+    lib.adapt_addmm.restype = i32
+    lib.adapt_addmm.argtypes = [vp, vp, vp, vp, i32, ctypes.c_float, ctypes.c_float, vp, vp]
+    lib.adapt_matmul_strided_batch.restype = i32
+    lib.adapt_matmul_strided_batch.argtypes = [vp, vp, i64, vp, i64, vp, i64, i64, vp]
     lib.adapt_plan_many.restype = i64
     lib.adapt_plan_many.argtypes = [i64, vp, vp, vp]
     lib.adapt_plan_table_save.restype = i64
@@ -177,6 +182,17 @@ def adapt_matmul_plan_forced(M, N, K, dtype, layoutA, layoutB, tiling_key):
 def adapt_matmul(plan, A_ptr: int, B_ptr: int, C_ptr: int, stream: int = 0):
     """Enqueue C = A*B.  Pointers are raw device addresses (``tensor.data_ptr()``)."""
     _check(load().adapt_matmul(plan, A_ptr, B_ptr, C_ptr, stream))
+
+
+def adapt_addmm(plan, A_ptr: int, B_ptr: int, D_ptr: int, d_is_vector: bool, alpha: float, beta: float, C_ptr: int, stream: int = 0):
+    """Enqueue C = alpha * (A*B) + beta * D (D: M x N, or a row of N values when d_is_vector)."""
+    _check(load().adapt_addmm(plan, A_ptr, B_ptr, D_ptr, 1 if d_is_vector else 0, alpha, beta, C_ptr, stream))
+
+
+def adapt_matmul_strided_batch(plan, A_ptr: int, stride_a: int, B_ptr: int, stride_b: int, C_ptr: int, stride_c: int, batch: int,
+                               stream: int = 0):
+    """Enqueue `batch` GEMMs of the plan's shape on operands the given numbers of elements apart."""
+    _check(load().adapt_matmul_strided_batch(plan, A_ptr, stride_a, B_ptr, stride_b, C_ptr, stride_c, batch, stream))
 
 
 def adapt_matmul_host(plan, A_host_ptr: int, B_host_ptr: int, C_host_ptr: int, stream: int = 0):

@@ -889,18 +889,22 @@ adapt_status_t launch_pad2(State& S, const void* srcA, void* dstA, int64_t outer
     return ADAPT_OK;
 }
 
-adapt_status_t launch_reduce(State& S, const float* partial, void* C, int64_t M, int64_t N, int P_k, int dtype, cudaStream_t stream)
+adapt_status_t launch_reduce(State& S, const float* partial, void* C, int64_t M, int64_t N, int P_k, int dtype, cudaStream_t stream,
+                             const ReduceEpilogue* epi = nullptr)
 {
+    ReduceEpilogue ep;
+    ep.D = nullptr; ep.d_is_vector = 0; ep.alpha = 1.f; ep.beta = 0.f;
+    if (epi) ep = *epi;
     const int64_t Np = partial_pitch(N);
     const int64_t work = M * (Np / 4);
     const int blocks = (int)std::min<int64_t>(ceil_div(work, 256), (int64_t)S.machine.n_sm * 8);
-    CUDA_TRY(launch_pdl(splitk_reduce_kernel, dim3(blocks), dim3(256), 0, stream, (const float*)partial, (unsigned short*)C, (int)M, (int)N, (int)Np, (int)P_k, (int)dtype));
+    CUDA_TRY(launch_pdl(splitk_reduce_kernel, dim3(blocks), dim3(256), 0, stream, (const float*)partial, (unsigned short*)C, (int)M, (int)N, (int)Np, (int)P_k, (int)dtype, ep));
     S.launches.fetch_add(1, std::memory_order_relaxed);
     CUDA_TRY(cudaGetLastError());
     return ADAPT_OK;
 }
 
-adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* C, cudaStream_t stream)
+adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* C, cudaStream_t stream, const ReduceEpilogue* epi = nullptr)
 {
     const Shape& s = pl->s;
     const Config& c = pl->c;
@@ -948,10 +952,11 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.num_units = p.P_m * p.P_n * p.P_k;
 
     // the plan's fused reduction stands unless a fallback changed the tiling (then: partials in the workspace)
-    const bool fused = c.fused != 0 && p.P_k == c.P_k && !(c.srcB == ADAPT_SRC_TMA_CLASSES && !kclsB);
-    const size_t szP = (p.P_k > 1 && !fused) ? (size_t)round_up((int64_t)p.P_k * s.M * partial_pitch(s.N) * 4, 256) : 0;
+    // (a fused-add epilogue runs in the reduction kernel: the GEMM then always leaves fp32 partials in the workspace)
+    const bool fused = !epi && c.fused != 0 && p.P_k == c.P_k && !(c.srcB == ADAPT_SRC_TMA_CLASSES && !kclsB);
+    const size_t szP = ((p.P_k > 1 || epi) && !fused) ? (size_t)round_up((int64_t)p.P_k * s.M * partial_pitch(s.N) * 4, 256) : 0;
     // stream-K stands unless a fallback changed the tiling; one fp32 partial tile per CTA
-    const bool streamk = c.streamk != 0 && p.P_k == 1 && !classesA && !kclsB;
+    const bool streamk = !epi && c.streamk != 0 && p.P_k == 1 && !classesA && !kclsB;
     const int sk_slots = S.machine.n_sm / c.cluster;
     const size_t szS = streamk ? (size_t)sk_slots * c.cluster * 128 * c.BN * 4 : 0;
     void* ws = nullptr;
@@ -983,7 +988,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
         if ((r = launch_pad(S, B, w8 + szA, outB, inB, pitchB, stream)) != ADAPT_OK) return r;
         b_src = w8 + szA;
     }
-    float* partial = (p.P_k > 1 && !fused) ? (float*)(w8 + szA + szB) : nullptr;
+    float* partial = ((p.P_k > 1 || epi) && !fused) ? (float*)(w8 + szA + szB) : nullptr;
 
     // K-major operand: one box of 64 k x (rows this CTA owns); MN-major operand: boxes of 64 x 64
     if (classesA) {
@@ -1016,7 +1021,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.part_hint = (p.P_k > 1 && szP <= ((size_t)100 << 20)) ? 1 : 0;
     memset(p.c_sigma, 0, sizeof(p.c_sigma));
     memset(p.c_extent, 0, sizeof(p.c_extent));
-    if (p.P_k == 1 && !kclsB && (halo ? ((uintptr_t)C & 15) == 0 : (((uintptr_t)C & 31) == 0 && s.N % 16 == 0))) {
+    if (p.P_k == 1 && !epi && !kclsB && (halo ? ((uintptr_t)C & 15) == 0 : (((uintptr_t)C & 31) == 0 && s.N % 16 == 0))) {
         if (classesA) {
             if ((r = cached_class_maps(S, pl, kMapC, C, s.M, s.N, 32, ncls, 32, true, maps.c, p.c_sigma, p.c_extent)) != ADAPT_OK)
                 return r;
@@ -1033,6 +1038,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
                 (s.K >= 32 || p.P_n <= 64 || classesA)) ? 1 : 0;
     if (const char* e = getenv("ADAPT_RASTER")) p.raster = atoi(e);
     p.prefetch = S.prefetch;
+    p.force_partial = epi ? 1 : 0;
     p.a_shift_any = 0;
     for (int j = 0; j < 16; ++j) p.a_shift_any |= p.a_sigma[j];
     if (p.a_shift_any) p.a_shift_any = 1;
@@ -1111,7 +1117,37 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     }
     CUDA_TRY(launch_exc(&cfg, k, args, arg_bytes, 2));
     S.launches.fetch_add(1, std::memory_order_relaxed);
-    if (p.P_k > 1 && !fused) return launch_reduce(S, partial, C, s.M, s.N, p.P_k, s.dtype, stream);
+    if ((p.P_k > 1 || epi) && !fused) return launch_reduce(S, partial, C, s.M, s.N, p.P_k, s.dtype, stream, epi);
+    return ADAPT_OK;
+}
+
+// The CUDA-core kernel with an explicit split count (the plan's own family, and the stand-in of the families that have
+// no fp32 partial path when a fused-add epilogue is asked for).
+adapt_status_t run_simt_splits(State& S, const Shape& s, int P_k, const void* A, const void* B, void* C, cudaStream_t stream,
+                               const ReduceEpilogue* epi)
+{
+    const bool partials = P_k > 1 || epi;
+    const size_t szP = partials ? (size_t)round_up((int64_t)P_k * s.M * partial_pitch(s.N) * 4, 256) : 0;
+    void* ws = nullptr;
+    adapt_status_t r = get_workspace(S, stream, szP, &ws);
+    if (r != ADAPT_OK) return r;
+    SimtParams p;
+    p.M = (int)s.M; p.N = (int)s.N; p.K = (int)s.K;
+    if (s.layoutA == ADAPT_ROW_MAJOR) { p.a_sm = s.K; p.a_sk = 1; } else { p.a_sm = 1; p.a_sk = s.M; }
+    if (s.layoutB == ADAPT_ROW_MAJOR) { p.b_sk = s.N; p.b_sn = 1; } else { p.b_sk = 1; p.b_sn = s.K; }
+    p.P_n = (int)ceil_div(s.N, 64);
+    p.P_k = partials ? std::max(P_k, 2) : 1;                  // any value > 1 makes the kernel write fp32 partials
+    p.Np = (int)partial_pitch(s.N);
+    p.kb_per_split = (int)ceil_div(ceil_div(s.K, 16), P_k);
+    p.dtype = s.dtype;
+    p.prefetch = S.prefetch;
+    p.C = (unsigned short*)C;
+    p.partial = (float*)ws;
+    dim3 grid((unsigned)(ceil_div(s.M, 64) * ceil_div(s.N, 64)), (unsigned)P_k, 1);
+    CUDA_TRY(launch_pdl(simt_gemm_kernel, grid, dim3(256), 0, stream, (const unsigned short*)A, (const unsigned short*)B, p));
+    S.launches.fetch_add(1, std::memory_order_relaxed);
+    CUDA_TRY(cudaGetLastError());
+    if (partials) return launch_reduce(S, (const float*)ws, C, s.M, s.N, P_k, s.dtype, stream, epi);
     return ADAPT_OK;
 }
 
@@ -1201,6 +1237,59 @@ extern "C" adapt_status_t adapt_matmul(adapt_handle_t plan, const void* A, const
         case ADAPT_FAM_CLUSTER: return run_cluster(S, pl, A, B, C, stream);
     }
     return fail(ADAPT_ERR_UNSUPPORTED, "unknown kernel family%s");
+}
+
+extern "C" adapt_status_t adapt_addmm(adapt_handle_t plan, const void* A, const void* B, const void* D, int d_is_vector,
+                                      float alpha, float beta, void* C, void* cuda_stream)
+{
+    State& S = st();
+    if (!plan) return fail(ADAPT_ERR_INVALID_ARG, "null plan%s");
+    if (!S.inited) return fail(ADAPT_ERR_NOT_INIT, "adapt_init has not been called%s");
+    Plan* pl = plan;
+    const Shape& s = pl->s;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (pl->noop) return ADAPT_OK;
+    if (!C || !D) return fail(ADAPT_ERR_INVALID_ARG, "null C or D%s");
+    if ((!A || !B) && !pl->zero_fill) return fail(ADAPT_ERR_INVALID_ARG, "null operand%s");
+    if (((uintptr_t)A | (uintptr_t)B | (uintptr_t)C | (uintptr_t)D) & 1) return fail(ADAPT_ERR_INVALID_ARG, "operands must be 2-byte aligned%s");
+    const size_t nA = (size_t)s.M * s.K * 2, nB = (size_t)s.K * s.N * 2, nC = (size_t)s.M * s.N * 2;
+    const size_t nD = d_is_vector ? (size_t)s.N * 2 : nC;
+    if (overlaps(C, nC, A, nA) || overlaps(C, nC, B, nB)) return fail(ADAPT_ERR_INVALID_ARG, "C overlaps an input%s");
+    // C may be D itself (the in-place update beta * C + alpha * A * B): every element is read before it is written, by the
+    // same thread; any other overlap is refused
+    if (D != C && overlaps(C, nC, D, nD)) return fail(ADAPT_ERR_INVALID_ARG, "C overlaps D without being D%s");
+    ReduceEpilogue ep;
+    ep.D = (const unsigned short*)D; ep.d_is_vector = d_is_vector ? 1 : 0; ep.alpha = alpha; ep.beta = beta;
+    if (pl->zero_fill) {
+        // K == 0: the product is zero; the reduction kernel over zero partial slabs leaves beta * D
+        return launch_reduce(S, nullptr, C, s.M, s.N, 0, s.dtype, stream, &ep);
+    }
+    switch (pl->c.family) {
+        case ADAPT_FAM_UMMA_1CTA:
+        case ADAPT_FAM_UMMA_2CTA: return run_umma(S, pl, A, B, C, stream, &ep);
+        default: break;
+    }
+    // the warp-level and one-launch families have no fp32 partial path: the CUDA-core kernel stands in, with enough k
+    // splits to fill the machine (their shapes are small or skinny)
+    const int64_t tiles = ceil_div(s.M, 64) * ceil_div(s.N, 64), ksteps = ceil_div(s.K, 16);
+    int64_t pk = pl->c.family == ADAPT_FAM_SIMT ? pl->c.P_k : std::max<int64_t>(1, std::min<int64_t>((4 * (int64_t)S.machine.n_sm) / tiles, ksteps / 4));
+    pk = std::max<int64_t>(1, std::min<int64_t>(pk, 256));
+    pk = ceil_div(ksteps, ceil_div(ksteps, pk));               // no empty split
+    return run_simt_splits(S, s, (int)pk, A, B, C, stream, &ep);
+}
+
+extern "C" adapt_status_t adapt_matmul_strided_batch(adapt_handle_t plan, const void* A, int64_t stride_a, const void* B,
+                                                     int64_t stride_b, void* C, int64_t stride_c, int64_t batch, void* cuda_stream)
+{
+    if (batch < 0 || stride_a < 0 || stride_b < 0 || stride_c < 0) return fail(ADAPT_ERR_INVALID_ARG, "negative batch count or stride%s");
+    if (!plan) return fail(ADAPT_ERR_INVALID_ARG, "null plan%s");
+    if (batch > 1 && !plan->noop && stride_c < plan->s.M * plan->s.N) return fail(ADAPT_ERR_INVALID_ARG, "outputs of the batch overlap%s");
+    for (int64_t i = 0; i < batch; ++i) {
+        const adapt_status_t r = adapt_matmul(plan, (const unsigned short*)A + i * stride_a, (const unsigned short*)B + i * stride_b,
+                                              (unsigned short*)C + i * stride_c, cuda_stream);
+        if (r != ADAPT_OK) return r;
+    }
+    return ADAPT_OK;
 }
 
 extern "C" adapt_status_t adapt_matmul_host(adapt_handle_t plan, const void* A_host, const void* B_host, void* C_host,
@@ -1553,7 +1642,7 @@ extern "C" adapt_status_t adapt_matmul_noalloc(int64_t M, int64_t N, int64_t K, 
     CUDA_TRY(cudaGetLastError());
     const int64_t work = M * (Np / 4);
     const int blocks = (int)std::min<int64_t>(ceil_div(work, 256), 148 * 8);
-    CUDA_TRY(launch_pdl(splitk_reduce_kernel, dim3(blocks), dim3(256), 0, stream, (const float*)scratch, (unsigned short*)C, (int)M, (int)N, (int)Np, (int)pk, (int)dtype));
+    CUDA_TRY(launch_pdl(splitk_reduce_kernel, dim3(blocks), dim3(256), 0, stream, (const float*)scratch, (unsigned short*)C, (int)M, (int)N, (int)Np, (int)pk, (int)dtype, ReduceEpilogue{nullptr, 0, 1.f, 0.f}));
     CUDA_TRY(cudaGetLastError());
     st().launches.fetch_add(2, std::memory_order_relaxed);
     return ADAPT_OK;

@@ -196,9 +196,16 @@ regroup_a_kernel(const unsigned short* __restrict__ A, unsigned short* __restric
 // The order is fixed, so the result does not depend on which CTA finished first.  Partials are
 // stored [P_k][M][Np] with Np = N rounded up to 8, so every row starts on a 32-byte boundary and
 // one thread reduces four consecutive columns with 16-byte loads.
+// Optional fused-add epilogue (the AddMM operator): out = alpha * sum + beta * D in fp32 before the single cast, D either a
+// full M x N 16-bit matrix or one row of N values added to every row.  D == nullptr: plain sum.
+struct ReduceEpilogue {
+    const unsigned short* D;
+    int d_is_vector;
+    float alpha, beta;
+};
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(const float* __restrict__ partial, unsigned short* __restrict__ C,
-                     int M, int N, int Np, int P_k, int dtype)
+                     int M, int N, int Np, int P_k, int dtype, const ReduceEpilogue ep)
 {
     pdl_launch_dependents();
     pdl_wait();
@@ -220,6 +227,14 @@ splitk_reduce_kernel(const float* __restrict__ partial, unsigned short* __restri
 #pragma unroll
             for (int j = 0; j < 8; ++j)
                 if (p0 + j < P_k) { acc.x += v[j].x; acc.y += v[j].y; acc.z += v[j].z; acc.w += v[j].w; }
+        }
+        if (ep.D) {
+            const unsigned short* d = ep.D + (ep.d_is_vector ? (int64_t)n : (int64_t)m * N + n);
+            float v[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (n + j < N) v[j] = fmaf(ep.beta, load16_as_float(d + j, dtype), ep.alpha * v[j]);
+            acc = make_float4(v[0], v[1], v[2], v[3]);
         }
         unsigned short* dst = C + (int64_t)m * N + n;
         if (n + 4 <= N && (reinterpret_cast<uintptr_t>(dst) & 7) == 0) {

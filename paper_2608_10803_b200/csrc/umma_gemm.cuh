@@ -54,6 +54,7 @@ struct UmmaParams {
     int c_mode;                      // 16-bit output: 0 = stores by the epilogue threads (any N, any alignment),
                                      // 1 = TMA stores through the maps of C (rows of C, or of the tile's row class,
                                      //     start on 32-byte boundaries; class tiles with 16 halo columns shift them there)
+    int force_partial;               // write fp32 partials also with P_k = 1 (a fused-add epilogue follows in the reduction kernel)
     int prefetch;                    // ask L2 for the first unit's operand boxes before waiting for the kernel ahead on the stream
     int raster;                      // tile visiting order: 0 = m-fastest inside groups of kGroupM m-blocks (operand reuse in L2),
                                      // 1 = n-fastest, row block by row block (write-bound shapes: neighbouring CTAs write
@@ -821,7 +822,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                 __syncwarp();
                 if (lane == 0)
                     for (int rk = 0; rk < p.P_k; ++rk) ptx::mbar_arrive_cluster(xempty_bar, (uint32_t)rk);
-            } else if (p.P_k == 1) {
+            } else if (p.P_k == 1 && !p.force_partial) {
                 // 16-bit output, any N and any base alignment.  A thread converts 64 columns of its row
                 // and stages them in shared memory shifted by the row's misalignment in C, so that
                 // 16-byte aligned chunks of a staged row are 16-byte aligned chunks of C.  The warp then
