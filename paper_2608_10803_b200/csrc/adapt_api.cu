@@ -557,6 +557,11 @@ static UmmaKernel launch_map_umma(int family, int BN, bool a_mn, bool b_mn, int 
         if (BN == 256) return (const void*)umma_gemm_kernel<256, false, true, 1, 3, true>;
         return nullptr;
     }
+    if (mode == 1 && family == ADAPT_FAM_UMMA_2CTA) {     // 256 rows of one row class per SM pair
+        if (BN == 128) return (const void*)umma_gemm_kernel<128, false, true, 2, 1>;
+        if (BN == 256) return (const void*)umma_gemm_kernel<256, false, true, 2, 1>;
+        return nullptr;
+    }
     if (mode == 1) {                     // row-major A read through per-row-class maps (1-CTA tiles, row-major B)
         if (BN == 64) return (const void*)umma_gemm_kernel<64, false, true, 1, 1>;
         if (BN == 128) return (const void*)umma_gemm_kernel<128, false, true, 1, 1>;
@@ -624,6 +629,9 @@ extern "C" adapt_status_t adapt_init(int device)
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
     CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_2CTA, 256, false, true, 2),
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
+    for (int BN : {128, 256})
+        CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_2CTA, BN, false, true, 1),
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
     for (int BN : {64, 128, 256}) {
         for (int a = 0; a < 2; ++a)
             for (int b = 0; b < 2; ++b)

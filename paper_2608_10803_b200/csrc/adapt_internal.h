@@ -245,8 +245,8 @@ inline int umma_deepest_ring(int BN, int cluster, int a_rows, bool staging, int 
 inline int umma_a_box_rows(const Shape& s, int cluster, int row_classes, bool k_classes)
 {
     const bool a_mn = !k_classes && s.layoutA == ADAPT_COL_MAJOR;
-    if (row_classes)    // 8 or 16 classes: a tile holds every 8th (16th) row of up to 1024 (2048)
-        return s.M < 128 * row_classes ? (int)std::min<int64_t>(128, round_up(ceil_div(s.M, row_classes), 8)) : 128;
+    if (row_classes)    // 8 or 16 classes: a tile holds every 8th (16th) row of up to 1024 (2048); a pair tile of twice as many
+        return (cluster == 1 && s.M < 128 * row_classes) ? (int)std::min<int64_t>(128, round_up(ceil_div(s.M, row_classes), 8)) : 128;
     if (!a_mn && cluster == 1 && s.M < 128) return (int)round_up(s.M, 8);
     return 128;
 }

@@ -488,8 +488,10 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
         if (aligned16(innerB(s)) || s.K < 64 || c.srcA != ADAPT_SRC_PAD_COPY) return false;
     }
     if (classes) {
-        // rows of one residue class share their misalignment: row-major A and B, one CTA per tile
-        if (c.family != ADAPT_FAM_UMMA_1CTA || s.layoutA != ADAPT_ROW_MAJOR || s.layoutB != ADAPT_ROW_MAJOR) return false;
+        // rows of one residue class share their misalignment: row-major A and B; pair tiles (256 rows of one class)
+        // without halo columns only
+        if (s.layoutA != ADAPT_ROW_MAJOR || s.layoutB != ADAPT_ROW_MAJOR) return false;
+        if (c.family != ADAPT_FAM_UMMA_1CTA && (c.BN % 64 != 0 || s.M < 16)) return false;
         // they pay when A's rows are unaligned (no copy), or when C's rows do not start on 32-byte sector
         // boundaries (halo tiles of 16 classes: uniform misalignment per tile, whole-sector TMA stores)
         if ((aligned16(innerA(s)) && c.BN % 64 == 0) || s.M < 8) return false;
@@ -497,7 +499,7 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     if (c.srcA == ADAPT_SRC_PAD_COPY && aligned16(innerA(s)) && !kclasses) return false;    // nothing to pad
     if (c.srcB == ADAPT_SRC_PAD_COPY && aligned16(innerB(s))) return false;
     const int ncls = umma_row_classes(c.srcA, c.BN);
-    c.P_m = classes ? (int)(ncls * ceil_div(s.M, ncls * c.BM)) : (int)ceil_div(s.M, c.BM);   // class tiles: 8 per 1024 rows, 16 per 2048
+    c.P_m = classes ? (int)(ncls * ceil_div(s.M, ncls * c.BM)) : (int)ceil_div(s.M, c.BM);   // class tiles: 8 per 1024 rows (pair tiles: per 2048), 16 per 2048
     c.P_n = (int)ceil_div(s.N, kclasses ? c.BN - 8 : (c.BN % 64 ? c.BN - 16 : c.BN));
     if ((int64_t)c.P_m * c.P_n * c.P_k > (int64_t)1 << 30) return false;
     if (c.streamk) {
@@ -692,6 +694,21 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
                     f.stages = umma_deepest_ring(BN, 1, rows, false, m.smem_bytes, kUmmaMaxStages, umma_fused_bytes(BN, rows));
                     if (f.stages >= 2 && finalize(s, m, cal, f)) out->push_back(f);
                 }
+            }
+        }
+    }
+    // --- the same row-class views on pair tiles (256 rows of one class per SM pair), for an A with unaligned rows ---
+    if (srcA == ADAPT_SRC_PAD_COPY && s.layoutA == ADAPT_ROW_MAJOR && s.layoutB == ADAPT_ROW_MAJOR && s.M >= 16) {
+        for (int BN : {128, 256}) {
+            const int64_t tiles = 8 * ceil_div(s.M, 2048) * ceil_div(s.N, BN);
+            split_candidates(tiles, m.n_sm / 2, ceil_div(s.K + (s.K % 8 ? 7 : 0), 64), 2, &pks);
+            for (int pk : pks) {
+                int deepest = umma_deepest_ring(BN, 2, 128, pk == 1, m.smem_bytes);
+                if (deepest > 8) deepest = 8;
+                Config d;
+                d.family = ADAPT_FAM_UMMA_2CTA; d.BM = 256; d.BN = BN; d.BK = 64; d.cluster = 2;
+                d.stages = deepest; d.P_k = pk; d.srcA = ADAPT_SRC_TMA_CLASSES; d.srcB = srcB;
+                if (deepest >= 2 && finalize(s, m, cal, d)) out->push_back(d);
             }
         }
     }

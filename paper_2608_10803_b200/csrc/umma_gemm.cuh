@@ -287,7 +287,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
     constexpr bool B_CLS = MODE == 2;
     constexpr bool B_SPLIT = MODE == 3;                   // k classes as k splits (see below)
     static_assert(MODE == 0 || (!A_MN && B_MN), "class modes: K-major A, row-major B");
-    static_assert(MODE == 0 || MODE == 3 || CG == 1, "tiles of one row class and tiles with eight class accumulators: one CTA per tile");
+    static_assert(MODE != 2 || CG == 1, "tiles with eight class accumulators: one CTA per tile");
+    static_assert(MODE != 1 || CG == 1 || BN % 64 == 0, "pair tiles of one row class: no halo columns");
     static_assert(!B_CLS || BN == 64, "k-class mode uses 64-column windows");
     // HALO: class tiles for a C whose rows do not start on 32-byte boundaries (N % 16 != 0) own 32-byte
     // units of the shifted rows instead of columns, so they compute 16 columns more than they own (see
@@ -328,6 +329,9 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
     uint8_t* stage_out = bar_gen + kUmmaBarrierBytes;
     // fused split-K: "every rank's partial is in place" / "every rank has read mine", at fixed offsets of the barrier block
     const uint32_t xfull_bar = bar_base + 512u, xempty_bar = bar_base + 520u;
+    // pair tiles of one row class: "this CTA's A box has landed" (each CTA, own loads) and, in the leader, "the peer's A
+    // box has landed and its stale row heads are zeroed"
+    const uint32_t afull_bar = bar_base + 544u, aready_bar = bar_base + 672u;
     int* sk_count = reinterpret_cast<int*>(bar_gen + 528);     // stream-K: epilogue warps that have written their share of a partial
 
     pdl_launch_dependents();
@@ -347,6 +351,12 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
         for (int b = 0; b < NBUF; ++b) {
             ptx::mbar_init(tfull_bar + 8u * b, 1);         // one tcgen05.commit per phase
             ptx::mbar_init(tempty_bar + 8u * b, kUmmaEpilogueWarps * CG);   // one arrive per epilogue warp of the group
+        }
+        if (A_CLS && CG == 2) {
+            for (int st = 0; st < S; ++st) {
+                ptx::mbar_init(afull_bar + 8u * st, 1);
+                ptx::mbar_init(aready_bar + 8u * st, 1);
+            }
         }
         if (FUSE) {
             ptx::mbar_init(xfull_bar, (uint32_t)(kUmmaEpilogueWarps * p.P_k));     // one arrive per epilogue warp of every rank
@@ -398,7 +408,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
         WorkItem w;
         if (lane < NREQ && next_item<SK, B_SPLIT>(p, unit0, unit_step, 0, w)) {
             const int cls = A_CLS ? (w.mb % NCLS) : 0;
-            const int row0 = A_CLS ? (w.mb / NCLS) * 128 : w.mb * (128 * CG) + (int)cta_rank * 128;
+            const int row0 = A_CLS ? (w.mb / NCLS) * (128 * CG) + (int)cta_rank * 128 : w.mb * (128 * CG) + (int)cta_rank * 128;
             const int kshift = A_CLS ? p.a_sigma[cls] : 0;
             const int a_k_off = B_SPLIT ? (w.split & 7) * p.cls_kc : 0;
             const int col0 = w.nb * TILE_N + (int)cta_rank * BN_CTA;
@@ -437,6 +447,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
             // the byte count of a stage is signalled on the leader's barrier (pair form)
             uint32_t full_target = full_bar;
             if (CG == 2) asm volatile("mapa.shared::cluster.u32 %0, %1, 0;" : "=r"(full_target) : "r"(full_bar));
+            uint32_t afull_own = afull_bar;       // pair tiles of one row class: this CTA's own A barrier as a cluster address
+            if (CG == 2) asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(afull_own) : "r"(afull_bar), "r"(cta_rank));
             bool ok = true;
             auto load = [&](uint32_t dst, const CUtensorMap* tm, uint32_t bar, int x, int y) {
                 if (CG == 1) ptx::tma_load_2d(dst, tm, bar, x, y);
@@ -451,7 +463,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                 // A rows of this CTA: consecutive rows, or in class mode rows 1024*g + j + 8*i read through
                 // map j at class-row index 128*g
                 const int cls = A_CLS ? (mb % NCLS) : 0;
-                const int row0 = A_CLS ? (mb / NCLS) * 128 : mb * (128 * CG) + (int)cta_rank * 128;
+                const int row0 = A_CLS ? (mb / NCLS) * (128 * CG) + (int)cta_rank * 128 : mb * (128 * CG) + (int)cta_rank * 128;
                 const int kshift = A_CLS ? p.a_sigma[cls] : 0;                // B's k-rows lag A's kappa by sigma
                 const CUtensorMap* tmA = &maps.a[cls];
                 const CUtensorMap* tmB = &maps.b[B_SPLIT ? (split & 7) : 0];  // k classes as splits: the class's view of B
@@ -486,6 +498,13 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     const uint32_t fb = full_target + 8u * stage;
                     if (lane == 0) {
                         if (CG == 1) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(p.a_tx_bytes + p.b_tx_bytes));
+                        else if (A_CLS && kb == 0 && kshift > 0) {
+                            // pair tiles of one row class, a unit's first k-block with row heads to zero: each CTA's A box
+                            // reports to its own barrier (its warp 1 zeroes the heads there before the MMA); the B boxes of
+                            // both CTAs report to the leader's as always
+                            ptx::mbar_arrive_expect_tx(afull_bar + 8u * stage, (uint32_t)A_BYTES);
+                            if (leader) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(2 * p.b_tx_bytes));
+                        }
                         else if (leader) ptx::mbar_arrive_expect_tx(full_bar + 8u * stage, (uint32_t)(2 * (A_BYTES + p.b_tx_bytes)));
                     }
                     __syncwarp(REQ_MASK);
@@ -503,7 +522,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                         if (B_MN) { dst = sB + (uint32_t)jb * 8192u; x = col0 + jb * 64; y = k0 - kshift; }
                         else { dst = sB; x = k0; y = col0; }
                     }
-                    load(dst, tm, fb, x, y);
+                    if (A_CLS && CG == 2 && is_a && kb == 0 && kshift > 0) load(dst, tm, afull_own + 8u * stage, x, y);   // this CTA's own barrier
+                    else load(dst, tm, fb, x, y);
                     if (++stage == S) { stage = 0; phase ^= 1u; }
                 }
                 if (lane == 0) ADAPT_TRACE(1, unit);
@@ -514,10 +534,65 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
         // one thread issues the MMAs; in class mode the whole warp runs the loop so that its other
         // lanes can zero the stale leading elements of A' in the first k-block
         // (only when some class of A is shifted: with K % 8 == 0 every sigma is zero and one lane is enough)
-        const bool warp_wide = A_CLS && p.a_shift_any != 0;
+        // (pair tiles of one row class: always, and the peer's warp 1 runs the forwarding loop further down)
+        const bool warp_wide = A_CLS && (p.a_shift_any != 0 || CG == 2);
+        // in class mode all 32 lanes run these loops: lane 0 waits and the outcome is broadcast, so
+        // the lanes never part ways before a __syncwarp
+        auto mma_wait = [&](uint32_t bar, uint32_t parity) -> bool {
+            if (!warp_wide) return ptx::mbar_wait(bar, parity, abort_flag);
+            int w = 1;
+            if (lane == 0) w = ptx::mbar_wait(bar, parity, abort_flag) ? 1 : 0;
+            return __shfl_sync(0xffffffffu, w, 0) != 0;
+        };
+        // Class tile whose rows are shifted: the sigma elements in front of each row of the first k-block belong to
+        // the previous row of A and are zeroed before the tensor core reads them.  Rows lane, lane+32, ...: chunk 0
+        // of row r (its first 8 elements) sits at r*128 + ((r & 7) << 4); one masked 16-byte read-modify-write per row.
+        auto zero_row_heads = [&](int stage, int sigma) {
+            uint8_t* genA = gen_base + (size_t)stage * STAGE_BYTES;
+            uint32_t keep[4];
+#pragma unroll
+            for (int w = 0; w < 4; ++w)
+                keep[w] = (2 * w >= sigma ? 0x0000ffffu : 0u) | (2 * w + 1 >= sigma ? 0xffff0000u : 0u);
+            uint4 v[4];
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int r = lane + 32 * t;
+                if (r * 128 < A_BYTES) v[t] = *reinterpret_cast<const uint4*>(genA + r * 128 + ((r & 7) << 4));
+            }
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                const int r = lane + 32 * t;
+                if (r * 128 < A_BYTES)               // rows past the box are not part of the stage
+                    *reinterpret_cast<uint4*>(genA + r * 128 + ((r & 7) << 4)) =
+                        make_uint4(v[t].x & keep[0], v[t].y & keep[1], v[t].z & keep[2], v[t].w & keep[3]);
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+        };
+        if (A_CLS && CG == 2 && !leader) {
+            // Pair tiles of one row class, the peer CTA: the A box of a unit's first k-block reports to this CTA's own
+            // barrier when its rows have stale heads; this warp zeroes them and then tells the leader that the peer's half
+            // of A is ready for the MMA the leader issues for both.  Every other k-block signals the leader directly.
+            int stage = 0;
+            uint32_t aphase = 0;              // per stage: parity of the next use of its A barriers (used by some units only)
+            bool ok = true;
+            for (int it = 0; ok; ++it) {
+                WorkItem w;
+                if (!next_item<SK, B_SPLIT>(p, unit0, unit_step, it, w)) break;
+                const int sigma = p.a_sigma[w.mb % NCLS];
+                if (w.kb0 == 0 && w.kb1 > 0 && sigma > 0) {
+                    if (!mma_wait(afull_bar + 8u * stage, (aphase >> stage) & 1u)) { ok = false; break; }
+                    zero_row_heads(stage, sigma);
+                    if (lane == 0) ptx::mbar_arrive_cluster(aready_bar + 8u * stage, 0);
+                    aphase ^= 1u << stage;
+                }
+                stage = (stage + (w.kb1 - w.kb0)) % S;
+            }
+        }
         if ((lane == 0 || warp_wide) && leader) {
             int stage = 0;
             uint32_t phase = 0;
+            uint32_t aphase = 0;              // pair tiles of one row class: per stage, parity of the next use of its A barriers
             int buf = 0;
             uint32_t buf_phase = 0;
             // K-major operand: rows of 128 B, 8-row groups 1024 B apart, +32 B per 16-element k step.
@@ -525,14 +600,6 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
             // 1024 B apart (SBO), +2048 B per 16-element k step.
             const uint32_t a_lbo = A_MN ? 8192u : 16u, b_lbo = B_MN ? 8192u : 16u;
             const uint32_t a_kstep = A_MN ? 2048u : 32u, b_kstep = B_MN ? 2048u : 32u;
-            // in class mode all 32 lanes run this loop: lane 0 waits and the outcome is broadcast, so
-            // the lanes never part ways before a __syncwarp
-            auto mma_wait = [&](uint32_t bar, uint32_t parity) -> bool {
-                if (!warp_wide) return ptx::mbar_wait(bar, parity, abort_flag);
-                int w = 1;
-                if (lane == 0) w = ptx::mbar_wait(bar, parity, abort_flag) ? 1 : 0;
-                return __shfl_sync(0xffffffffu, w, 0) != 0;
-            };
             bool ok = true;
             for (int it = 0; ok; ++it) {
                 WorkItem w;
@@ -540,35 +607,13 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                 const int unit = w.unit, mb = w.mb, nb = w.nb, split = w.split, kb0 = w.kb0, kb1 = w.kb1;
                 (void)unit; (void)nb; (void)split;
                 if (warp_wide && kb0 == 0 && kb1 > 0) {
-                    // Class tile whose rows are shifted: the sigma elements in front of each row of the first
-                    // k-block belong to the previous row of A and are zeroed before the tensor core reads them.
                     // Done here, before the wait for a free accumulator: the loads run ahead of the drain, so
                     // in the write-bound regime this work hides behind that wait.
                     const int sigma = p.a_sigma[mb % NCLS];
                     if (sigma > 0) {
-                        if (!mma_wait(full_bar + 8u * stage, phase)) { ok = false; break; }
-                        // rows lane, lane+32, ...: chunk 0 of row r (its first 8 elements) sits at
-                        // r*128 + ((r & 7) << 4); one masked 16-byte read-modify-write per row
-                        uint8_t* genA = gen_base + (size_t)stage * STAGE_BYTES;
-                        uint32_t keep[4];
-#pragma unroll
-                        for (int w = 0; w < 4; ++w)
-                            keep[w] = (2 * w >= sigma ? 0x0000ffffu : 0u) | (2 * w + 1 >= sigma ? 0xffff0000u : 0u);
-                        uint4 v[4];
-#pragma unroll
-                        for (int t = 0; t < 4; ++t) {
-                            const int r = lane + 32 * t;
-                            if (r * 128 < A_BYTES) v[t] = *reinterpret_cast<const uint4*>(genA + r * 128 + ((r & 7) << 4));
-                        }
-#pragma unroll
-                        for (int t = 0; t < 4; ++t) {
-                            const int r = lane + 32 * t;
-                            if (r * 128 < A_BYTES)               // rows past the box are not part of the stage
-                                *reinterpret_cast<uint4*>(genA + r * 128 + ((r & 7) << 4)) =
-                                    make_uint4(v[t].x & keep[0], v[t].y & keep[1], v[t].z & keep[2], v[t].w & keep[3]);
-                        }
-                        ptx::fence_proxy_async_smem();
-                        __syncwarp();
+                        if (!mma_wait((A_CLS && CG == 2) ? afull_bar + 8u * stage : full_bar + 8u * stage,
+                                      (A_CLS && CG == 2) ? ((aphase >> stage) & 1u) : phase)) { ok = false; break; }
+                        zero_row_heads(stage, sigma);
                     }
                 }
                 if (!mma_wait(tempty_bar + 8u * buf, buf_phase ^ 1u)) { ok = false; break; }
@@ -592,23 +637,44 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                             if (++stage == S) { stage = 0; phase ^= 1u; }
                         }
                 }
-                for (int kb = kb0; !B_CLS && kb < kb1; ++kb) {
-                    if (!mma_wait(full_bar + 8u * stage, phase)) { ok = false; break; }
-                    ptx::tc_fence_after();
-                    const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
-                    const uint32_t sB = sA + A_BYTES;
+                if (!B_CLS) {
+                    // The k-block loop proper runs in ONE lane, also when the warp came here together (class tiles): a
+                    // warp-wide loop pays a shuffle for every wait, and the MMA thread's loop is what the tensor core waits
+                    // for (pair tiles of one row class: 0.82 us per k-block with the warp-wide loop).  The other lanes step
+                    // their copy of (stage, phase) by the number of k-blocks and pick up the outcome afterwards.
+                    int done = 1;
                     if (lane == 0) {
+                        int st = stage;
+                        uint32_t ph = phase;
+                        for (int kb = kb0; kb < kb1; ++kb) {
+                            if (A_CLS && CG == 2 && kb == 0 && p.a_sigma[mb % NCLS] > 0) {
+                                // the unit's first k-block, row heads zeroed: this CTA's box (waited for above) and the peer's,
+                                // handed over by the peer's warp 1.  The leader reads none of the peer's shared memory itself
+                                // (the peer's tensor core does, after the peer's own proxy fence), so an ordinary wait is enough.
+                                if (!ptx::mbar_wait(aready_bar + 8u * st, (aphase >> st) & 1u, abort_flag)) { done = 0; break; }
+                            }
+                            if (!ptx::mbar_wait(full_bar + 8u * st, ph, abort_flag)) { done = 0; break; }
+                            ptx::tc_fence_after();
+                            const uint32_t sA = smem_base + (uint32_t)st * STAGE_BYTES;
+                            const uint32_t sB = sA + A_BYTES;
 #pragma unroll
-                        for (int k16 = 0; k16 < kUmmaBK / 16; ++k16) {
-                            const uint64_t adesc = ptx::smem_desc_sw128(sA + k16 * a_kstep, a_lbo, 1024u);
-                            const uint64_t bdesc = ptx::smem_desc_sw128(sB + k16 * b_kstep, b_lbo, 1024u);
-                            ptx::umma_f16<CG>(d_tmem, adesc, bdesc, p.idesc, (kb > kb0 || k16 > 0) ? 1u : 0u);
+                            for (int k16 = 0; k16 < kUmmaBK / 16; ++k16) {
+                                const uint64_t adesc = ptx::smem_desc_sw128(sA + k16 * a_kstep, a_lbo, 1024u);
+                                const uint64_t bdesc = ptx::smem_desc_sw128(sB + k16 * b_kstep, b_lbo, 1024u);
+                                ptx::umma_f16<CG>(d_tmem, adesc, bdesc, p.idesc, (kb > kb0 || k16 > 0) ? 1u : 0u);
+                            }
+                            // free the stage (in both CTAs of a pair) once these MMAs have read it
+                            if (CG == 1) ptx::umma_commit_1(empty_bar + 8u * st);
+                            else ptx::umma_commit_2(empty_bar + 8u * st);
+                            if (++st == S) { st = 0; ph ^= 1u; }
                         }
-                        // free the stage (in both CTAs of a pair) once these MMAs have read it
-                        if (CG == 1) ptx::umma_commit_1(empty_bar + 8u * stage);
-                        else ptx::umma_commit_2(empty_bar + 8u * stage);
                     }
-                    if (++stage == S) { stage = 0; phase ^= 1u; }
+                    if (warp_wide) done = __shfl_sync(0xffffffffu, done, 0);
+                    if (!done) { ok = false; break; }
+                    if (A_CLS && CG == 2 && kb0 == 0 && kb1 > 0 && p.a_sigma[mb % NCLS] > 0) aphase ^= 1u << stage;
+                    const int adv = stage + (kb1 - kb0);
+                    phase ^= (uint32_t)((adv / S) & 1);
+                    stage = adv % S;
                 }
                 if (!ok) break;
                 if (lane == 0) {
@@ -650,7 +716,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
             if (warp == 2 && lane == 0) ADAPT_TRACE(4, unit);
             // row of C held by TMEM lane i of this CTA: consecutive rows, or every 8th row of one class
             const int row_step = A_CLS ? NCLS : 1;
-            const int row_base = A_CLS ? (mb / NCLS) * (128 * NCLS) + (mb % NCLS) : mb * (128 * CG) + (int)cta_rank * 128;
+            const int row_base = A_CLS ? (mb / NCLS) * (128 * CG * NCLS) + (mb % NCLS) + NCLS * 128 * (int)cta_rank
+                                       : mb * (128 * CG) + (int)cta_rank * 128;
             const int row = row_base + row_step * (q * 32 + lane);
             const int n0 = nb * TILE_N;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * BN);
@@ -861,7 +928,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                         const int cls = A_CLS ? (mb % NCLS) : 0;
                         const int sig = HALO ? p.c_sigma[cls] : 0;
                         const int off = HALO ? 16 - sig : 0;
-                        const int y0 = A_CLS ? (mb / NCLS) * 128 + q * 32 : row_base + q * 32;
+                        const int y0 = A_CLS ? (mb / NCLS) * (128 * CG) + (int)cta_rank * 128 + q * 32 : row_base + q * 32;
                         const CUtensorMap* tmC = &maps.c[cls];
                         uint8_t* wbuf = stage_out + (warp - 2) * kUmmaWarpStagingBytes;
                         const int x_first = n0 + (HALO ? 16 : 0);

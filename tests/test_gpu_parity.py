@@ -713,3 +713,65 @@ def test_stream_k_random_values_run_twice_bit_identical():
             rows = sample_rows(M, 48, seed=3)
             err, mism, n = compare_with_oracle(A, B, C1, M, N, K, dtype, rows=rows)
             assert err <= TOL[dtype], (c.BN, c.family, err)
+
+
+# ---- row-class views on pair tiles (256 rows of one class per SM pair) ---------------------------------------
+
+def pair_class_variants(M, N, K, dtype):
+    return [(ab.adapt_matmul_plan_forced(M, N, K, dtype, ROW, ROW, c.tiling_key), c)
+            for c in ab.adapt_plan_candidates(M, N, K, dtype) if c.srcA == 3 and c.family == ab.FAM_UMMA_2CTA]
+
+
+@pytest.mark.parametrize("dtype", [ab.F16, ab.BF16])
+@pytest.mark.parametrize("shape", [(131, 77, 259), (1030, 264, 331), (2500, 64, 1001), (16, 8, 9), (300, 520, 12), (2049, 128, 4099),
+                                   (4100, 1000, 70), (5000, 16, 2047), (4096, 512, 1003)])
+def test_pair_tiles_of_one_row_class_bit_exact(shape, dtype):
+    """Both CTAs of a pair read 128 rows each of one row class of an A whose rows are not 16-byte aligned; every such
+    configuration (TMA-store and thread-store epilogues, split-K) against the oracle on position-coded integers."""
+    M, N, K = shape
+    A = synth.position_coded(M, K, dtype, modulus=7, device="cuda")
+    B = synth.position_coded(K, N, dtype, modulus=5, device="cuda")
+    variants = pair_class_variants(M, N, K, dtype)
+    assert variants, "shape must offer pair tiles of one row class"
+    for plan, c in variants[:10]:
+        check_case(M, N, K, dtype, A, B, plan=plan, exact=True)
+
+
+def test_pair_tiles_of_one_row_class_do_not_leak_a_neighbouring_row():
+    """As for the 1-CTA class tiles: non-finite values at the end of a row of A sit in front of the next row's
+    first element in memory and must not reach that row's result, in either CTA of the pair."""
+    M, N, K = 2600, 136, 203
+    dtype = ab.F16
+    A = synth.position_coded(M, K, dtype, 7, "cuda")
+    B = synth.position_coded(K, N, dtype, 5, "cuda")
+    bad_rows = [4, 17, 300, 1029, 1500, 2111]          # classes and halves of both CTAs
+    for r in bad_rows:
+        A[r, K - 1] = float("inf")
+        A[r, K - 2] = float("nan")
+    keep = torch.tensor([i for i in range(M) if i not in bad_rows], device="cuda")
+    variants = pair_class_variants(M, N, K, dtype)
+    assert variants
+    for plan, c in variants[:6]:
+        C = run_library(A, B, M, N, K, dtype, plan=plan)
+        torch.cuda.synchronize()
+        ab.adapt_poll_device_status(torch.cuda.current_stream().cuda_stream)
+        assert torch.isfinite(C.index_select(0, keep)).all()
+        err, mism, n = compare_with_oracle(A, B, C, M, N, K, dtype, rows=keep.cpu().numpy())
+        assert mism == 0
+
+
+def test_pair_tiles_of_one_row_class_random_values_and_unaligned_pointer():
+    M, N, K, dtype = 3000, 688, 1999, ab.BF16
+    A = synth.draw_operand(M, K, synth.U11, 81, dtype, "cuda")
+    B = synth.draw_operand(K, N, synth.U11, 82, dtype, "cuda")
+    bufA = torch.zeros(M * K + 8, dtype=torch.bfloat16, device="cuda")
+    A1 = bufA[3:3 + M * K].view(M, K)
+    A1.copy_(A)
+    for plan, c in pair_class_variants(M, N, K, dtype)[:4]:
+        for Ax in (A, A1):
+            C = run_library(Ax, B, M, N, K, dtype, plan=plan)
+            torch.cuda.synchronize()
+            ab.adapt_poll_device_status(torch.cuda.current_stream().cuda_stream)
+            rows = sample_rows(M, 64, seed=9)
+            err, mism, n = compare_with_oracle(Ax, B, C, M, N, K, dtype, rows=rows)
+            assert err <= TOL[dtype], (c.BN, c.P_k, err)
