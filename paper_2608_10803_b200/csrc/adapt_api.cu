@@ -141,6 +141,7 @@ struct State {
     std::atomic<int64_t> map_encodes{0};   // tensor maps encoded on the host so far (a cached call encodes none)
     std::atomic<int> map_cache{1};         // 0: every call encodes its maps afresh (measurement of the miss cost)
     int log = 0;
+    int shuffle_k = 0;                 // ShuffleK analogue (ADAPT_SHUFFLE_K=1): rotated k-block order per tile; measured, off by default
     int prefetch = 1;                  // L2 prefetch of a kernel's first operands ahead of its dependency wait (ADAPT_PREFETCH=0 turns it off)
     bool class_promo128 = true;        // 128-byte L2 promotion for the strided class views (ADAPT_CLASS_PROMO128=0: 256 as for dense operands)
 };
@@ -157,6 +158,7 @@ void apply_env(State& S)
     if (const char* e = getenv("ADAPT_LOG")) S.log = atoi(e);
     if (const char* e = getenv("ADAPT_NO_PDL")) pdl_enabled() = atoi(e) == 0;
     if (const char* e = getenv("ADAPT_PREFETCH")) S.prefetch = atoi(e);
+    if (const char* e = getenv("ADAPT_SHUFFLE_K")) S.shuffle_k = atoi(e);
     if (const char* e = getenv("ADAPT_CLASS_PROMO128")) S.class_promo128 = atoi(e) != 0;
     if (const char* e = getenv("ADAPT_WORKSPACE_LIMIT_MB")) S.machine.workspace_limit = (int64_t)atoll(e) << 20;
 }
@@ -1046,6 +1048,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
                 (s.K >= 32 || p.P_n <= 64 || classesA)) ? 1 : 0;
     if (const char* e = getenv("ADAPT_RASTER")) p.raster = atoi(e);
     p.prefetch = S.prefetch;
+    p.shuffle_k = S.shuffle_k;
     p.force_partial = epi ? 1 : 0;
     p.a_shift_any = 0;
     for (int j = 0; j < 16; ++j) p.a_shift_any |= p.a_sigma[j];

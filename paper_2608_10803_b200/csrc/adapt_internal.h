@@ -90,9 +90,10 @@ struct Calib {
     double streamk_fixup_us = 10.0;     // stream-K: partial tile out (5 us) and its fence, the flag, the owner's exposed last drain ...
     double streamk_peer_us = 3.0;       // ... and its additions, per slot that shares the tile (2560 x 4096 x 4096, 6 sharers: 87 us
                                         // against 55 us of main loop; 5120 x 4096 x 8192, 3 sharers: 246 us against 226 us)
-    double fused_reduce_us = 2.5;       // fused split-K: cluster scheduling, drain to shared memory, two cluster-wide barrier rounds,
-                                        // first remote reads (1 x 4096 x 4096, 128 x 128 tiles, P_k 4: 12.1 us fused, 11.3 us with the reduce launch)
-    double fused_wave_us = 3.5;         // each further round of clusters starts cold (1 x 4096 x 4096, P_k 8: 3 rounds 26 us, 2 rounds 20 us)
+    double fused_reduce_us = 2.0;       // fused split-K: cluster scheduling, drain to shared memory, two cluster-wide barrier rounds,
+                                        // first remote reads (1 x 4096 x 4096, 128 x 128 tiles, P_k 4: 11.3 us fused, 11.1 us with the reduce launch;
+                                        // 128 x 4096 x 4096: 13.3 against 14.1 us)
+    double fused_wave_us = 3.0;         // each further round of clusters starts cold (1 x 4096 x 4096, P_k 8, 3 rounds: 14.2 us against 11.3 us in one)
     double reduce_launch_us = 1.5;      // the reduce launch behind the GEMM: programmatic dependent launch hides about half of a launch
     double dsmem_bw_per_sm = 60e9;      // B/s one SM reads from its peers' shared memory during the fused reduction
     double copy_bw_eff = 0.85;          // pad-copy and reduce kernels

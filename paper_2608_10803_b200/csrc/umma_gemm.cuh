@@ -55,6 +55,8 @@ struct UmmaParams {
                                      // 1 = TMA stores through the maps of C (rows of C, or of the tile's row class,
                                      //     start on 32-byte boundaries; class tiles with 16 halo columns shift them there)
     int force_partial;               // write fp32 partials also with P_k = 1 (a fused-add epilogue follows in the reduction kernel)
+    int shuffle_k;                   // ShuffleK (Table 2): a tile starts its k range at a k-block that depends on the tile, so the CTAs of a wave
+                                     // do not all ask for the same k slice of a shared operand at the same moment (plain tiles only)
     int prefetch;                    // ask L2 for the first unit's operand boxes before waiting for the kernel ahead on the stream
     int raster;                      // tile visiting order: 0 = m-fastest inside groups of kGroupM m-blocks (operand reuse in L2),
                                      // 1 = n-fastest, row block by row block (write-bound shapes: neighbouring CTAs write
@@ -490,7 +492,11 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                             if (++stage == S) { stage = 0; phase ^= 1u; }
                         }
                 }
-                for (int kb = kb0; !B_CLS && kb < kb1; ++kb) {
+                // ShuffleK: the unit's k-blocks in rotated order (the MMA warp consumes the stages in ring order and sums
+                // whatever arrives, so only the loads know; the order is a function of the tile, hence fixed)
+                const int kb_rot = (MODE == 0 && !SK && p.shuffle_k && kb1 - kb0 > 1) ? ((mb + nb) * 5) % (kb1 - kb0) : 0;
+                for (int kbi = kb0; !B_CLS && kbi < kb1; ++kbi) {
+                    const int kb = (MODE == 0 && !SK) ? kb0 + (kbi - kb0 + kb_rot) % (kb1 - kb0) : kbi;
                     ok = __all_sync(REQ_MASK, ptx::mbar_wait(empty_bar + 8u * stage, phase ^ 1u, abort_flag));
                     if (!ok) break;
                     const uint32_t sA = smem_base + (uint32_t)stage * STAGE_BYTES;
@@ -852,10 +858,11 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                 }
                 release_accumulator();
                 released = true;
-                // this warp's share of the partial is written: tell every rank (release at cluster scope)
+                // this warp's share of the partial is written: tell every rank (release at cluster scope), one lane per rank:
+                // an arrive on another CTA's barrier occupies its thread for the better part of a microsecond, so a single
+                // lane walking the ranks serialised P_k of them (pair tiles hit the same wall: 0.8 us per k-block)
                 __syncwarp();
-                if (lane == 0)
-                    for (int rk = 0; rk < p.P_k; ++rk) ptx::mbar_arrive_cluster(xfull_bar, (uint32_t)rk);
+                if (lane < p.P_k) ptx::mbar_arrive_cluster(xfull_bar, (uint32_t)lane);
                 if (!ptx::mbar_wait_cluster(xfull_bar, xphase, abort_flag)) { ok = false; break; }
                 // rows and 4-column groups of this tile that exist; rank r takes the r-th share of them
                 const int rows_here = A_CLS ? min(128, (p.M - row_base + row_step - 1) / row_step) : min(128, p.M - row_base);
@@ -887,8 +894,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                 }
                 // done reading every rank's partial: each may overwrite it for its next tile
                 __syncwarp();
-                if (lane == 0)
-                    for (int rk = 0; rk < p.P_k; ++rk) ptx::mbar_arrive_cluster(xempty_bar, (uint32_t)rk);
+                if (lane < p.P_k) ptx::mbar_arrive_cluster(xempty_bar, (uint32_t)lane);
             } else if (p.P_k == 1 && !p.force_partial) {
                 // 16-bit output, any N and any base alignment.  A thread converts 64 columns of its row
                 // and stages them in shared memory shifted by the row's misalignment in C, so that
