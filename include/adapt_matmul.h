@@ -288,6 +288,14 @@ adapt_status_t adapt_measure_store_rate(void* buffer, int64_t rows, int64_t cols
 /* Tensor maps encoded on the host since adapt_init; a call whose maps are cached encodes none.  Each plan
  * keeps the encodings of its 8 most recent distinct (pointer, geometry) pairs per operand. */
 int64_t adapt_map_encode_count(void);
+/* Run-time switches of the tcgen05 kernels, applied to calls made after it returns (the environment variables
+ * ADAPT_SHUFFLE_K and ADAPT_PREFETCH set the same at start-up):
+ *   "shuffle_k" (default 0): the ShuffleK module of Table 2: every tile walks its k-blocks in an order rotated by an
+ *               amount that depends on the tile, so that the CTAs of a wave do not all ask for the same k slice of a shared
+ *               operand at once.  The order is a function of the tile, so results stay reproducible, but they may differ
+ *               in the last bit from those with the option off (another summation order).  Plain tiles only.
+ *   "prefetch"  (default 1): L2 prefetch of a kernel's first operand boxes ahead of its wait for the kernel before it. */
+adapt_status_t adapt_set_option(const char* name, int value);
 /* enabled = 0 bypasses the tensor-map cache (every call encodes); 1 restores it.  Measurement only. */
 void adapt_set_map_cache(int enabled);
 

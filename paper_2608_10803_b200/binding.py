@@ -27,7 +27,7 @@ EXPORTS = [
     "adapt_matmul_noalloc", "adapt_matmul_batch", "adapt_matmul_repeat", "adapt_measure_dispatch",
     "adapt_measure_empty_launch", "adapt_map_encode_count", "adapt_set_map_cache", "adapt_selftest_wait_expiry",
     "adapt_measure_store_rate", "adapt_plan_many", "adapt_plan_table_save", "adapt_plan_table_load",
-    "adapt_addmm", "adapt_matmul_strided_batch",
+    "adapt_addmm", "adapt_matmul_strided_batch", "adapt_set_option",
 ]
 
 
@@ -122,6 +122,8 @@ def load():
     lib.adapt_plan_cache_size.restype = i64
     lib.adapt_launch_count.restype = i64
     lib.adapt_map_encode_count.restype = i64
+    lib.adapt_set_option.restype = i32
+    lib.adapt_set_option.argtypes = [ctypes.c_char_p, i32]
     lib.adapt_set_map_cache.restype = None
     lib.adapt_set_map_cache.argtypes = [i32]
     lib.adapt_matmul_batch.restype = i32
@@ -282,6 +284,10 @@ def adapt_plan_table_load(path: str) -> int:
 
 def adapt_map_encode_count() -> int:
     return load().adapt_map_encode_count()
+
+
+def adapt_set_option(name: str, value: int):
+    _check(load().adapt_set_option(name.encode(), int(value)))
 
 
 def adapt_set_map_cache(enabled: bool):

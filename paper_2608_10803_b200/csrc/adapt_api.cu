@@ -404,6 +404,16 @@ extern "C" int64_t adapt_plan_cache_size(void)
 extern "C" int64_t adapt_launch_count(void) { return st().launches.load(); }
 extern "C" int64_t adapt_map_encode_count(void) { return st().map_encodes.load(); }
 extern "C" void adapt_set_map_cache(int enabled) { st().map_cache.store(enabled ? 1 : 0); }
+extern "C" adapt_status_t adapt_set_option(const char* name, int value)
+{
+    State& S = st();
+    if (!name) return fail(ADAPT_ERR_INVALID_ARG, "null option name%s");
+    std::lock_guard<std::mutex> lock(S.mu);
+    if (!strcmp(name, "shuffle_k")) S.shuffle_k = value ? 1 : 0;
+    else if (!strcmp(name, "prefetch")) S.prefetch = value ? 1 : 0;
+    else return fail(ADAPT_ERR_INVALID_ARG, "unknown option %s", name);
+    return ADAPT_OK;
+}
 
 
 // ---------------------------------------------------------------------------------------------
