@@ -129,7 +129,7 @@ def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
                     halo = c.BN % 64 != 0        # class tiles of 16 row classes that own 32-byte units of C's shifted rows
                     ncls = 16 if halo else 8
                     a_rows = 128
-                    if c.srcA == 3:
+                    if c.srcA == 3 and c.cluster == 1:
                         a_rows = min(128, -(-(-(-M // ncls)) // 8) * 8)
                     elif c.cluster == 1 and M < 128:
                         a_rows = -(-M // 8) * 8
@@ -143,8 +143,10 @@ def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
                     if K % 8:
                         assert c.srcA in (1, 3)      # re-pitched copy, or the per-row-class TMA views
                     if c.srcA == 3:
-                        assert (K % 8 or halo) and M >= 8 and c.family == ab.FAM_UMMA_1CTA
-                        assert c.P_m == ncls * -(-M // (128 * ncls))
+                        assert (K % 8 or halo) and M >= 8
+                        # pair tiles of one row class: 256 rows of a class per SM pair, no halo columns
+                        assert c.family == ab.FAM_UMMA_1CTA or (not halo and M >= 16 and c.BN in (128, 256))
+                        assert c.P_m == ncls * -(-M // (128 * c.cluster * ncls))
                     if N % 8:
                         assert c.srcB in (1, 3)      # re-pitched copy, or the per-k-class TMA views
                     if c.srcB == 3:
