@@ -937,12 +937,15 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     const int64_t Kc = round_up(ceil_div(s.K, 8), 64);          // k-class mode: padded class segment of A'
     const int64_t inA = kclsB ? 8 * Kc : (a_mn ? s.M : s.K), outA = a_mn ? s.K : s.M;
     const int64_t inB = b_mn ? s.N : s.K, outB = b_mn ? s.K : s.N;
-    const bool a_inner_ok = (s.layoutA == ADAPT_COL_MAJOR ? s.M : s.K) % 8 == 0;
-    const bool padA = classesA ? ((uintptr_t)A & 15) != 0
+    // in place when the rows suit TMA (16-byte multiples, narrow operands whole sectors) and the base is aligned
+    const bool a_inner_ok = tma_friendly(s.layoutA == ADAPT_COL_MAJOR ? s.M : s.K);
+    const bool padA = classesA ? (((uintptr_t)A & 15) != 0 || class_tiles_copy_a(s))
                                : (!kclsB && (!a_inner_ok || ((uintptr_t)A & 15) != 0));
-    const bool padB = !kclsB && (inB % 8 != 0 || ((uintptr_t)B & 15) != 0);
+    const bool padB = !kclsB && (!tma_friendly(inB) || ((uintptr_t)B & 15) != 0);
     const int64_t pitchA = padA ? padded_pitch(inA) : inA;
     const int64_t pitchB = padB ? padded_pitch(inB) : inB;
+    // a re-pitched narrow operand is read with its pad columns (zeros): whole sectors per row
+    const int64_t extA = (padA && inA < 64) ? pitchA : inA, extB = (padB && inB < 64) ? pitchB : inB;
     const size_t szA = (padA || kclsB) ? (size_t)round_up(outA * pitchA * 2, 256) : 0;
     const size_t szB = padB ? (size_t)round_up(outB * pitchB * 2, 256) : 0;
 
@@ -1019,7 +1022,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
         // a K-major A of fewer than 128 rows is loaded with a box of just those rows (rounded up to 8):
         // the rows of the stage it leaves untouched only feed accumulator rows that are never stored
         a_box_rows = umma_a_box_rows(s, cg, 0, kclsB);
-        if ((r = cached_map(S, pl, kMapA, a_src, inA, outA, pitchA, 64, a_mn ? 64 : a_box_rows, &maps.a[0])) != ADAPT_OK) return r;
+        if ((r = cached_map(S, pl, kMapA, a_src, extA, outA, pitchA, 64, a_mn ? 64 : a_box_rows, &maps.a[0])) != ADAPT_OK) return r;
     }
     if (kclsB) {
         // rows of B (K x N, N % 8 != 0) by class k % 8: the same construction as A's row classes, 64 x 64 boxes
@@ -1028,7 +1031,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
         // a row-major B whose K fits one k-block is loaded with boxes of just the k rows that exist (rounded up to 8; class
         // tiles shift B's rows by up to 7): boxes of 64 rows that lie mostly beyond K load several times slower when B is wide
         if (b_mn && p.kb_total == 1) b_box_k = (int)std::min<int64_t>(64, round_up(s.K + ((classesA && s.K % 8) ? 7 : 0), 8));
-        if ((r = cached_map(S, pl, kMapB, b_src, inB, outB, pitchB, 64, b_mn ? b_box_k : c.BN / cg, &maps.b[0])) != ADAPT_OK) return r;
+        if ((r = cached_map(S, pl, kMapB, b_src, extB, outB, pitchB, 64, b_mn ? b_box_k : c.BN / cg, &maps.b[0])) != ADAPT_OK) return r;
     }
 
     // 16-bit output leaves through TMA stores (boxes of 64 elements x 32 rows, one epilogue warp) when the

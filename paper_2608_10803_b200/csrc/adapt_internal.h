@@ -163,8 +163,18 @@ inline int64_t round_up(int64_t a, int64_t b) { return ceil_div(a, b) * b; }
 // kernels write whole 32-byte sectors (16-byte pieces of a sector halve the store rate).
 inline int64_t partial_pitch(int64_t N) { return round_up(N, 8); }
 
-// Operand pitch in elements after the Padding module (16-byte multiple).
-inline int64_t padded_pitch(int64_t inner) { return round_up(inner, 8); }
+// TMA reads an operand in place when its rows are 16-byte multiples.  Rows shorter than one 128-byte box line must in
+// addition be whole 32-byte sectors: a box whose rows are fractions of a sector loads at a fraction of the rate (a
+// 61370 x 85272 A streams at 6.8 TB/s beside a B of 32 columns, at 5.3 beside one of 5, 8 or 40 columns; a
+// 44239 x 80357 C is written in 1.47 ms beside an A of 16 padded columns, in 1.89 ms beside one of 1).
+inline bool tma_friendly(int64_t inner) { return inner % 8 == 0 && (inner >= 64 || inner % 16 == 0); }
+// Operand pitch in elements after the Padding module: a 16-byte multiple, for narrow operands a 32-byte multiple; the
+// copy fills the pad columns with zeros, and the tensor map of a narrow operand covers them (whole sectors per row).
+inline int64_t padded_pitch(int64_t inner) { return inner < 64 ? round_up(inner, 16) : round_up(inner, 8); }
+
+// Class tiles read a row-major A in place through their per-class views, except a narrow one whose rows are not whole
+// sectors: that one is re-pitched first (the views of the copy are then all aligned).
+inline bool class_tiles_copy_a(const Shape& s) { return s.K < 64 && !tma_friendly(s.K); }
 
 const Calib& default_calib();
 

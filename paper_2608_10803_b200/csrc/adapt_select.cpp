@@ -161,7 +161,8 @@ static void model_prologue(const Shape& s, Config& c, const Calib& cal)
         c.hbm_bytes += src + (double)c.ws_padA;
         return;
     }
-    if (c.srcA == ADAPT_SRC_PAD_COPY) {
+    // (class tiles read a narrow A, whose rows are fractions of a sector, over a sector-pitched copy too)
+    if (c.srcA == ADAPT_SRC_PAD_COPY || (c.srcA == ADAPT_SRC_TMA_CLASSES && class_tiles_copy_a(s))) {
         const double src = 2.0 * (double)s.M * (double)s.K;
         c.ws_padA = round_up(outerA(s) * padded_pitch(innerA(s)) * 2, 256);
         c.t_pro_us += cal.prologue_launch_us + copy_time_us(src + (double)c.ws_padA, cal);
@@ -171,7 +172,7 @@ static void model_prologue(const Shape& s, Config& c, const Calib& cal)
         const double src = 2.0 * (double)s.K * (double)s.N;
         c.ws_padB = round_up(outerB(s) * padded_pitch(innerB(s)) * 2, 256);
         // both operands re-pitched: one launch does both
-        c.t_pro_us += (c.srcA == ADAPT_SRC_PAD_COPY ? 0.0 : cal.prologue_launch_us) + copy_time_us(src + (double)c.ws_padB, cal);
+        c.t_pro_us += (c.ws_padA != 0 ? 0.0 : cal.prologue_launch_us) + copy_time_us(src + (double)c.ws_padB, cal);
         c.hbm_bytes += src + (double)c.ws_padB;
     }
 }
@@ -474,8 +475,8 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     if (c.P_k < 1 || c.P_k > 1023 || pk_blocks > kblocks) return false;
     if (ceil_div(kblocks, ceil_div(kblocks, pk_blocks)) != pk_blocks) return false;   // no empty split
     // operand sources: TMA needs a 16-byte row pitch
-    if (c.srcA == ADAPT_SRC_TMA && !aligned16(innerA(s))) return false;
-    if (c.srcB == ADAPT_SRC_TMA && !aligned16(innerB(s))) return false;
+    if (c.srcA == ADAPT_SRC_TMA && !tma_friendly(innerA(s))) return false;
+    if (c.srcB == ADAPT_SRC_TMA && !tma_friendly(innerB(s))) return false;
     if (c.srcA == ADAPT_SRC_LSU || c.srcB == ADAPT_SRC_LSU) return false;
     const bool classes = c.srcA == ADAPT_SRC_TMA_CLASSES;
     const bool kclasses = c.srcB == ADAPT_SRC_TMA_CLASSES;
@@ -496,8 +497,8 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
         // boundaries (halo tiles of 16 classes: uniform misalignment per tile, whole-sector TMA stores)
         if ((aligned16(innerA(s)) && c.BN % 64 == 0) || s.M < 8) return false;
     }
-    if (c.srcA == ADAPT_SRC_PAD_COPY && aligned16(innerA(s)) && !kclasses) return false;    // nothing to pad
-    if (c.srcB == ADAPT_SRC_PAD_COPY && aligned16(innerB(s))) return false;
+    if (c.srcA == ADAPT_SRC_PAD_COPY && tma_friendly(innerA(s)) && !kclasses) return false;    // nothing to pad
+    if (c.srcB == ADAPT_SRC_PAD_COPY && tma_friendly(innerB(s))) return false;
     const int ncls = umma_row_classes(c.srcA, c.BN);
     c.P_m = classes ? (int)(ncls * ceil_div(s.M, ncls * c.BM)) : (int)ceil_div(s.M, c.BM);   // class tiles: 8 per 1024 rows (pair tiles: per 2048), 16 per 2048
     c.P_n = (int)ceil_div(s.N, kclasses ? c.BN - 8 : (c.BN % 64 ? c.BN - 16 : c.BN));
@@ -632,8 +633,9 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
     if (s.M < 1 || s.N < 1 || s.K < 1) return;
     std::vector<int> pks;
     // --- tcgen05 families ---
-    const int srcA = aligned16(innerA(s)) ? ADAPT_SRC_TMA : ADAPT_SRC_PAD_COPY;
-    const int srcB = aligned16(innerB(s)) ? ADAPT_SRC_TMA : ADAPT_SRC_PAD_COPY;
+    // in place when TMA reads the rows well (16-byte multiples; narrow operands: whole sectors), else over a re-pitched copy
+    const int srcA = tma_friendly(innerA(s)) ? ADAPT_SRC_TMA : ADAPT_SRC_PAD_COPY;
+    const int srcB = tma_friendly(innerB(s)) ? ADAPT_SRC_TMA : ADAPT_SRC_PAD_COPY;
     for (int fam = ADAPT_FAM_UMMA_1CTA; fam <= ADAPT_FAM_UMMA_2CTA; ++fam) {
         const int BM = fam == ADAPT_FAM_UMMA_1CTA ? 128 : 256;
         const int cluster = fam == ADAPT_FAM_UMMA_1CTA ? 1 : 2;
@@ -674,11 +676,12 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
     }
     // --- tcgen05, A read in place through per-row-class views (row-major A, K % 8 != 0): 8 class
     //     tiles per 1024 rows, so the split counts are drawn from that tile count ---
-    if ((srcA == ADAPT_SRC_PAD_COPY || s.N % 16 != 0) && s.layoutA == ADAPT_ROW_MAJOR && s.layoutB == ADAPT_ROW_MAJOR && s.M >= 8) {
+    const bool a_unaligned = !aligned16(innerA(s)), b_unaligned = !aligned16(innerB(s));
+    if ((a_unaligned || s.N % 16 != 0) && s.layoutA == ADAPT_ROW_MAJOR && s.layoutB == ADAPT_ROW_MAJOR && s.M >= 8) {
         for (int BN : {64, 128, 256, 80, 144, 208}) {
             const bool halo = BN % 64 != 0;
             if (halo && (s.N % 16 == 0 || s.M < 16)) continue;             // halo tiles serve a C off 32-byte boundaries only
-            if (!halo && srcA != ADAPT_SRC_PAD_COPY) continue;             // aligned A: class tiles only for their stores
+            if (!halo && !a_unaligned) continue;                           // aligned A: class tiles only for their stores
             const int64_t tiles = (halo ? 16 * ceil_div(s.M, 2048) : 8 * ceil_div(s.M, 1024)) * ceil_div(s.N, halo ? BN - 16 : BN);
             split_candidates(tiles, m.n_sm, ceil_div(s.K + (s.K % 8 ? 7 : 0), 64), 2, &pks);
             for (int pk : pks) {
@@ -698,7 +701,7 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
         }
     }
     // --- the same row-class views on pair tiles (256 rows of one class per SM pair), for an A with unaligned rows ---
-    if (srcA == ADAPT_SRC_PAD_COPY && s.layoutA == ADAPT_ROW_MAJOR && s.layoutB == ADAPT_ROW_MAJOR && s.M >= 16) {
+    if (a_unaligned && s.layoutA == ADAPT_ROW_MAJOR && s.layoutB == ADAPT_ROW_MAJOR && s.M >= 16) {
         for (int BN : {128, 256}) {
             const int64_t tiles = 8 * ceil_div(s.M, 2048) * ceil_div(s.N, BN);
             split_candidates(tiles, m.n_sm / 2, ceil_div(s.K + (s.K % 8 ? 7 : 0), 64), 2, &pks);
@@ -714,7 +717,7 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
     }
     // --- tcgen05, B read in place through per-k-class views (row-major B, N % 8 != 0); A is regrouped by a
     //     prologue copy, so this pays when A is the small operand ---
-    if (srcB == ADAPT_SRC_PAD_COPY && s.layoutB == ADAPT_ROW_MAJOR && s.K >= 64) {
+    if (b_unaligned && s.layoutB == ADAPT_ROW_MAJOR && s.K >= 64) {
         const int64_t tiles = ceil_div(s.M, 128) * ceil_div(s.N, 56);
         split_candidates(tiles, m.n_sm, ceil_div(ceil_div(s.K, 8), 64), 1, &pks);
         for (int pk : pks) {
@@ -726,7 +729,7 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
         }
     }
     // --- the same views with each class a k split: full-width tiles, 8 fp32 partials per output ---
-    if (srcB == ADAPT_SRC_PAD_COPY && s.layoutB == ADAPT_ROW_MAJOR && s.K >= 64) {
+    if (b_unaligned && s.layoutB == ADAPT_ROW_MAJOR && s.K >= 64) {
         for (int v = 0; v < 3; ++v) {                               // 1-CTA tiles of 128 and 256 columns, pair tiles of 256
             const int BN = v == 0 ? 128 : 256, cluster = v == 2 ? 2 : 1, BM = 128 * cluster;
             const int64_t tiles = ceil_div(s.M, BM) * ceil_div(s.N, BN - 8);

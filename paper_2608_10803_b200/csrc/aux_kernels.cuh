@@ -27,9 +27,9 @@ __device__ __forceinline__ unsigned short float_to_16(float a, int dtype)
 }
 
 // ---- Padding: re-pitch a dense [outer][inner] 16-bit matrix to [outer][pitch], pitch % 8 == 0 ----
-// One thread produces one 16-byte chunk of the destination.  The pad columns are never read by
-// the GEMM (the tensor map's extent stays `inner`), so they are written as zeros only to keep
-// the workspace deterministic.
+// One thread produces one 16-byte chunk of the destination.  The pad columns are written as zeros:
+// the tensor map of a narrow operand (inner < 64, pitch a 32-byte multiple) covers them, so that
+// every row TMA fetches is made of whole sectors; they meet zeros or columns that are never stored.
 __device__ __forceinline__ void pad_copy_body(const unsigned short* __restrict__ src, unsigned short* __restrict__ dst,
                                               int64_t outer, int64_t inner, int64_t pitch, int block, int blocks)
 {
