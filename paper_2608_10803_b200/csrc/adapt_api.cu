@@ -944,8 +944,8 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     const bool padB = !kclsB && (!tma_friendly(inB) || ((uintptr_t)B & 15) != 0);
     const int64_t pitchA = padA ? padded_pitch(inA) : inA;
     const int64_t pitchB = padB ? padded_pitch(inB) : inB;
-    // a re-pitched narrow operand is read with its pad columns (zeros): whole sectors per row
-    const int64_t extA = (padA && inA < 64) ? pitchA : inA, extB = (padB && inB < 64) ? pitchB : inB;
+    // a re-pitched operand is read with its pad columns (zeros): whole sectors per row, also in the last box of a row
+    const int64_t extA = padA ? pitchA : inA, extB = padB ? pitchB : inB;
     const size_t szA = (padA || kclsB) ? (size_t)round_up(outA * pitchA * 2, 256) : 0;
     const size_t szB = padB ? (size_t)round_up(outB * pitchB * 2, 256) : 0;
 

@@ -105,7 +105,9 @@ struct Calib {
     double kclass_tile_drain_us = 2.5;  // drain of a tile with eight class accumulators (29 x 58492 x 94: 8 tile rounds in 35 us)
     double oob_box_penalty = 0.05;      // main-loop cost of one B box per stage that lies wholly beyond N
     double reduce_batch_us = 0.8;       // split-K reduction: one batch of eight slabs (13 x 420 x 43580: P_k 72 -> 24 saves 13 us)
-    double class_split_bw_eff = 0.92;   // HBM rate through the k-class views of B with full-width tiles (classes as k splits)
+    double class_split_bw_eff = 0.97;   // HBM rate through the k-class views of B with full-width tiles (classes as k splits) at M = 1 ...
+    double class_split_bw_eff_per_log2m = 0.031;   // ... and what it loses per doubling of M (1 x 50321 x 48452 ... 80 x 23916 x 86044)
+    double class_split_fused_bw_eff = 0.905;       // ... with the classes of a tile as one cluster (36 x 81499 x 66349: 6.3 TB/s)
     double regroup_bw_eff = 0.85;       // class-major regrouping of a row-major A (20000 x 8000: 600 MB in 107 us) relative to hbm_bw
     double class_view_bw_eff = 0.8;     // HBM rate through the per-row-class TMA views of an unaligned A
 };
@@ -168,9 +170,11 @@ inline int64_t partial_pitch(int64_t N) { return round_up(N, 8); }
 // 61370 x 85272 A streams at 6.8 TB/s beside a B of 32 columns, at 5.3 beside one of 5, 8 or 40 columns; a
 // 44239 x 80357 C is written in 1.47 ms beside an A of 16 padded columns, in 1.89 ms beside one of 1).
 inline bool tma_friendly(int64_t inner) { return inner % 8 == 0 && (inner >= 64 || inner % 16 == 0); }
-// Operand pitch in elements after the Padding module: a 16-byte multiple, for narrow operands a 32-byte multiple; the
-// copy fills the pad columns with zeros, and the tensor map of a narrow operand covers them (whole sectors per row).
-inline int64_t padded_pitch(int64_t inner) { return inner < 64 ? round_up(inner, 16) : round_up(inner, 8); }
+// Operand pitch in elements after the Padding module: a 32-byte multiple; the copy fills the pad columns with zeros, and
+// the tensor map covers them, so that every row TMA fetches, also the last box of a row, is made of whole sectors
+// (27239 x 84 x 96056, B re-pitched to 88 columns: the 20-column remainder box of every k-block costs as much as three
+// full ones).
+inline int64_t padded_pitch(int64_t inner) { return round_up(inner, 16); }
 
 // Class tiles read a row-major A in place through their per-class views, except a narrow one whose rows are not whole
 // sectors: that one is re-pitched first (the views of the copy are then all aligned).

@@ -316,7 +316,12 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
     model_prologue(s, c, cal);
     model_epilogue(s, c, cal);
     // strided row-class views stream A at a lower rate than a dense tensor (measured 3.5-4.1 TB/s)
-    const double bw = ksplit_cls ? cal.hbm_bw * cal.class_split_bw_eff
+    // (k classes as splits: the rate falls as the regrouped A, re-read by every column of tiles, grows beside the B
+    // stream: 0.93 of the copy rate at M = 1, 0.80 at M = 30, 0.70 at M = 80; with the eight classes of a tile as
+    // one cluster it stays near 0.87)
+    const double split_eff = c.fused ? cal.class_split_fused_bw_eff
+                                     : std::max(0.6, cal.class_split_bw_eff - cal.class_split_bw_eff_per_log2m * std::log2((double)std::max<int64_t>(1, s.M)));
+    const double bw = ksplit_cls ? cal.hbm_bw * split_eff
                     : (c.srcA == ADAPT_SRC_TMA_CLASSES || kclasses) ? cal.hbm_bw * cal.class_view_bw_eff : cal.hbm_bw;
     // A row-major B arrives as k-rows of BN contiguous columns per tile: short pieces stream below the
     // HBM rate (8 x 30016 x 40000: 3.6 / 5.5 / 6.9 TB/s at 128 / 256 / 512 bytes)
