@@ -84,6 +84,41 @@ def test_layouts_bit_exact(shape, lA, lB, dtype):
         check_case(M, N, K, dtype, A_st, B_st, lA, lB, plan=plan, exact=True)
 
 
+# ---- narrow operands: fewer than 64 contiguous elements, read over a copy with 32-byte rows ----------------
+
+@pytest.mark.parametrize("lA,lB", [(ROW, ROW), (ROW, COL), (COL, ROW), (COL, COL)])
+@pytest.mark.parametrize("shape", [(700, 520, 1), (700, 521, 8), (300, 40, 900), (1100, 5, 1300), (24, 300, 40), (9, 2100, 56),
+                                   (1200, 84, 700), (2100, 330, 24)])
+def test_narrow_operands_bit_exact(shape, lA, lB):
+    """A, B (and through class tiles C) with rows of 2 to 126 bytes: every tensor-core configuration, among them
+    class tiles over the re-pitched A and a B whose last box is a few columns wide, gives the oracle's bits."""
+    M, N, K = shape
+    dtype = ab.F16 if (M + N) % 2 == 0 else ab.BF16
+    A = synth.position_coded(M, K, dtype, 7, "cuda")
+    B = synth.position_coded(K, N, dtype, 5, "cuda")
+    A_st = A.t().contiguous() if lA == COL else A
+    B_st = B.t().contiguous() if lB == COL else B
+    for plan, c in every_variant(M, N, K, dtype, lA, lB, families=(ab.FAM_UMMA_1CTA, ab.FAM_UMMA_2CTA), limit_per_family=10):
+        check_case(M, N, K, dtype, A_st, B_st, lA, lB, plan=plan, exact=True)
+    check_case(M, N, K, dtype, A_st, B_st, lA, lB, exact=True)
+
+
+def test_narrow_operands_random_values_next_to_poisoned_memory():
+    """The pad columns of the re-pitched copies hold zeros whatever follows the operands in memory: A and B sit in
+    buffers whose other bytes are NaN patterns, and the result still meets the bar (a pad column that took a
+    neighbour's value would put NaN into every output)."""
+    for (M, N, K, dtype) in [(900, 5, 1500, ab.F16), (1300, 1031, 3, ab.BF16), (520, 40, 72, ab.F16)]:
+        td = synth.torch_dtype(dtype)
+        bufA = torch.full((M * K + 64,), float("nan"), dtype=td, device="cuda")
+        bufB = torch.full((K * N + 64,), float("nan"), dtype=td, device="cuda")
+        A = bufA[8:8 + M * K].view(M, K)
+        B = bufB[8:8 + K * N].view(K, N)
+        A.copy_(synth.draw_operand(M, K, synth.U11, 21, dtype, "cuda"))
+        B.copy_(synth.draw_operand(K, N, synth.U11, 22, dtype, "cuda"))
+        for plan, c in every_variant(M, N, K, dtype, families=(ab.FAM_UMMA_1CTA, ab.FAM_UMMA_2CTA), limit_per_family=6):
+            check_case(M, N, K, dtype, A, B, plan=plan)
+
+
 # ---- edge tiles: one off the tile sizes, primes, ones --------------------------------------------------
 
 @pytest.mark.parametrize("shape", [(127, 255, 63), (129, 257, 65), (1, 1, 1), (2, 3, 5), (255, 129, 191),
