@@ -296,6 +296,17 @@ int64_t adapt_map_encode_count(void);
  *               in the last bit from those with the option off (another summation order).  Plain tiles only.
  *   "prefetch"  (default 1): L2 prefetch of a kernel's first operand boxes ahead of its wait for the kernel before it. */
 adapt_status_t adapt_set_option(const char* name, int value);
+
+/* The analytical model's calibration constants (Section 5.2's machine terms: bandwidths, latencies, per-tile and
+ * per-launch costs), by name.  adapt_calibration_names writes the comma-separated list of names to out (at most
+ * cap - 1 characters and a terminating zero; out may be null) and returns the length of the whole list plus one.
+ * A value set here is used by every plan made afterwards (adapt_matmul_plan, adapt_plan_candidates); plans already
+ * in the cache keep their selection.  Host only, thread-safe; unknown name or NaN: ADAPT_ERR_INVALID_ARG.  Together
+ * with adapt_plan_candidates and timed configurations (adapt_matmul_plan_forced) this is all a program needs to
+ * refit the model for another machine; paper_2608_10803_b200/calibrate.py does it. */
+adapt_status_t adapt_set_calibration(const char* name, double value);
+adapt_status_t adapt_get_calibration(const char* name, double* value);
+int adapt_calibration_names(char* out, int cap);
 /* enabled = 0 bypasses the tensor-map cache (every call encodes); 1 restores it.  Measurement only. */
 void adapt_set_map_cache(int enabled);
 

@@ -28,6 +28,7 @@ EXPORTS = [
     "adapt_measure_empty_launch", "adapt_map_encode_count", "adapt_set_map_cache", "adapt_selftest_wait_expiry",
     "adapt_measure_store_rate", "adapt_plan_many", "adapt_plan_table_save", "adapt_plan_table_load",
     "adapt_addmm", "adapt_matmul_strided_batch", "adapt_set_option",
+    "adapt_set_calibration", "adapt_get_calibration", "adapt_calibration_names",
 ]
 
 
@@ -124,6 +125,12 @@ def load():
     lib.adapt_map_encode_count.restype = i64
     lib.adapt_set_option.restype = i32
     lib.adapt_set_option.argtypes = [ctypes.c_char_p, i32]
+    lib.adapt_set_calibration.restype = i32
+    lib.adapt_set_calibration.argtypes = [ctypes.c_char_p, ctypes.c_double]
+    lib.adapt_get_calibration.restype = i32
+    lib.adapt_get_calibration.argtypes = [ctypes.c_char_p, ctypes.POINTER(ctypes.c_double)]
+    lib.adapt_calibration_names.restype = i32
+    lib.adapt_calibration_names.argtypes = [ctypes.c_char_p, i32]
     lib.adapt_set_map_cache.restype = None
     lib.adapt_set_map_cache.argtypes = [i32]
     lib.adapt_matmul_batch.restype = i32
@@ -288,6 +295,24 @@ def adapt_map_encode_count() -> int:
 
 def adapt_set_option(name: str, value: int):
     _check(load().adapt_set_option(name.encode(), int(value)))
+
+
+def adapt_set_calibration(name: str, value: float):
+    _check(load().adapt_set_calibration(name.encode(), float(value)))
+
+
+def adapt_get_calibration(name: str) -> float:
+    v = ctypes.c_double(0.0)
+    _check(load().adapt_get_calibration(name.encode(), ctypes.byref(v)))
+    return float(v.value)
+
+
+def adapt_calibration_names():
+    lib = load()
+    need = lib.adapt_calibration_names(None, 0)
+    buf = ctypes.create_string_buffer(need + 1)
+    lib.adapt_calibration_names(buf, need + 1)
+    return buf.value.decode().split(",")
 
 
 def adapt_set_map_cache(enabled: bool):

@@ -1,4 +1,17 @@
-"""Last calibration step of the latency model: one scale factor per variant group.
+"""Calibration of the latency model from timed configurations.
+
+Two tools over the same input, the CSV that ``bench.py --validate-model N --dump-candidates cand.csv`` writes on
+a B200 (every legal configuration of the sampled shapes, with the model's prediction and the measured time):
+
+``python -m paper_2608_10803_b200.calibrate fit train.csv [more.csv] [--check other_seed.csv]`` moves the model's
+constants (``adapt_get_calibration`` / ``adapt_set_calibration``) by coordinate descent so that the configuration
+the model picks is, on average, as close as possible to the fastest timed one (mean regret), and prints the
+constants that changed; ``--check`` reports the same figures on a shape set the fit has not seen.  It needs no GPU:
+the model runs on the host.
+
+``python -m paper_2608_10803_b200.calibrate cand.csv`` (no sub-command) is the older per-group report:
+
+Last calibration step of the latency model: one scale factor per variant group.
 
     python bench.py --validate-model 400 --validate-roof-us 0.3 --dump-candidates cand.csv     (on a B200)
     python -m paper_2608_10803_b200.calibrate cand.csv                                          (anywhere)
@@ -48,7 +61,105 @@ def group_of(row) -> int:
     return g + (20 if fam == "umma_2cta" else 0)
 
 
+FAMILY_ID = {"umma_1cta": 0, "umma_2cta": 1, "skinny": 2, "simt": 3, "cluster": 4}
+
+
+class TimedSet:
+    """Timed configurations of a set of shapes, keyed the way the model's candidates are."""
+
+    def __init__(self, paths):
+        self.shapes = {}
+        for path in paths:
+            with open(path, newline="") as f:
+                for r in csv.DictReader(f):
+                    shape = (int(r["M"]), int(r["N"]), int(r["K"]), int(r["dtype"]))
+                    cfg = (FAMILY_ID[r["family"]], int(r["BN"]), int(r["stages"]), int(r["P_k"]), int(r["cluster"]), int(r["fused"]),
+                           int(r["streamk"]), int(r["srcA"]), int(r["srcB"]))
+                    t = float(r["time_us"])
+                    d = self.shapes.setdefault(shape, {})
+                    d[cfg] = min(d.get(cfg, float("inf")), t)
+
+    def metrics(self, ab):
+        """Regret of the model's pick among the timed configurations of every shape, with the constants now set."""
+        regrets, picked, best_sum, sq, n_near = [], 0.0, 0.0, 0.0, 0
+        for (M, N, K, dt), timed in self.shapes.items():
+            best = min(timed.values())
+            pick_pred, pick_t = float("inf"), None
+            for c in ab.adapt_plan_candidates(M, N, K, dt):
+                t = timed.get((c.family, c.BN, c.stages, c.P_k, c.cluster, c.fused, c.streamk, c.srcA, c.srcB))
+                if t is None:
+                    continue
+                if c.predicted_us < pick_pred:
+                    pick_pred, pick_t = c.predicted_us, t
+                if t <= 1.5 * best:
+                    sq += math.log(c.predicted_us / t) ** 2
+                    n_near += 1
+            if pick_t is None:
+                continue
+            regrets.append(pick_t / best)
+            picked += pick_t
+            best_sum += best
+        regrets.sort()
+        n = len(regrets)
+        return {"shapes": n, "mean": sum(regrets) / n, "p95": regrets[min(n - 1, int(0.95 * n))], "max": regrets[-1],
+                "exact": sum(1 for r in regrets if r <= 1.0001) / n, "within_2pct": sum(1 for r in regrets if r <= 1.02) / n,
+                "time_weighted": picked / best_sum, "rms_log_error_near_best": math.sqrt(sq / max(1, n_near))}
+
+
+def fit(argv):
+    ap = argparse.ArgumentParser(prog="calibrate fit")
+    ap.add_argument("csv", nargs="+", help="timed configurations to fit on")
+    ap.add_argument("--check", nargs="*", default=[], help="timed configurations of shapes the fit does not see")
+    ap.add_argument("--rounds", type=int, default=1)
+    ap.add_argument("--steps", default="0.8,0.9,1.1,1.25", help="factors tried on each constant")
+    ap.add_argument("--only", default="", help="comma-separated names of the constants to move (default: all)")
+    args = ap.parse_args(argv)
+    from . import binding as ab
+    train = TimedSet(args.csv)
+    check = TimedSet(args.check) if args.check else None
+    names = [x for x in args.only.split(",") if x] or ab.adapt_calibration_names()
+    steps = [float(x) for x in args.steps.split(",")]
+    start = {k: ab.adapt_get_calibration(k) for k in names}
+
+    def objective(m):      # the regret decides; the prediction error only breaks ties between equal selections
+        return m["mean"] + 0.5 * (m["time_weighted"] - 1.0) + 0.05 * m["rms_log_error_near_best"]
+
+    def show(tag, m):
+        print(tag, " ".join(f"{k}={v:.4f}" if isinstance(v, float) else f"{k}={v}" for k, v in m.items()), flush=True)
+
+    m0 = train.metrics(ab)
+    show("fit set, before:  ", m0)
+    if check:
+        show("check set, before:", check.metrics(ab))
+    best = objective(m0)
+    for rnd in range(args.rounds):
+        moved = False
+        for k in names:
+            x0 = ab.adapt_get_calibration(k)
+            for f in steps:
+                ab.adapt_set_calibration(k, x0 * f)
+                m = train.metrics(ab)
+                if objective(m) < best - 2e-4:
+                    best, moved = objective(m), True
+                    print(f"round {rnd}: {k} {x0:g} -> {x0 * f:g}  mean regret {m['mean']:.4f}", flush=True)
+                    x0 = x0 * f
+                else:
+                    ab.adapt_set_calibration(k, x0)
+        if not moved:
+            break
+    show("fit set, after:   ", train.metrics(ab))
+    if check:
+        show("check set, after: ", check.metrics(ab))
+    for k in names:
+        v = ab.adapt_get_calibration(k)
+        if v != start[k]:
+            print(f"    double {k} = {v:.4g};    // was {start[k]:g}")
+
+
 def main():
+    import sys
+    if len(sys.argv) > 1 and sys.argv[1] == "fit":
+        return fit(sys.argv[2:])
     ap = argparse.ArgumentParser()
     ap.add_argument("csv", nargs="+")
     ap.add_argument("--current", default="", help="comma-separated factors the library was built with (default: all 1)")

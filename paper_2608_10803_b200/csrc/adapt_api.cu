@@ -404,6 +404,61 @@ extern "C" int64_t adapt_plan_cache_size(void)
 extern "C" int64_t adapt_launch_count(void) { return st().launches.load(); }
 extern "C" int64_t adapt_map_encode_count(void) { return st().map_encodes.load(); }
 extern "C" void adapt_set_map_cache(int enabled) { st().map_cache.store(enabled ? 1 : 0); }
+// the model's calibration constants by name (the fields of Calib that are plain doubles)
+#define ADAPT_CALIB_FIELDS(X) X(launch_us) X(prologue_launch_us) X(hbm_bw) X(l2_bw_per_sm) X(tensor_flops) X(eta_mma_bn128) X(eta_mma_bn64) \
+    X(eta_2cta) X(mem_latency_us) X(hbm_latency_us) X(hbm_latency_views_us) X(umma_fixed_us) X(epi_tile_fixed_us) X(epi_us_per_kb) \
+    X(pair_drain_factor) X(epi_partial_fixed_us) X(epi_partial_us_per_kb) X(epi_tile_fixed_unaligned_us) X(epi_us_per_kb_unaligned) \
+    X(thread_store_exposed) X(thread_store_exposed_pair) X(simt_flops) X(simt_fixed_us) X(simt_step_us) X(halo_edge_tile_us) X(simt_bw_eff) \
+    X(skinny_bw_eff_aligned) X(skinny_bw_eff_unaligned) X(skinny_fixed_us) X(skinny_pass_us) X(skinny_step_unaligned_us) X(skinny_mac_rate) \
+    X(cluster_fixed_us) X(cluster_stage_us) X(cluster_reduce_us) X(cluster_crowd_us) X(cluster_crowd_stage_us) X(cluster_wave_us) \
+    X(cluster_bw_eff) X(streamk_fixup_us) X(streamk_peer_us) X(fused_reduce_us) X(fused_wave_us) X(reduce_launch_us) X(dsmem_bw_per_sm) \
+    X(copy_bw_eff) X(hbm_bw_per_sm) X(class_view_sm_eff) X(class_tile_fixed_us) X(class_tile_fixed_unaligned_us) X(kclass_view_sm_eff) \
+    X(kclass_unit_fixed_us) X(kclass_tile_drain_us) X(oob_box_penalty) X(reduce_batch_us) X(class_split_bw_eff) \
+    X(class_split_bw_eff_per_log2m) X(class_split_fused_bw_eff) X(regroup_bw_eff) X(class_view_bw_eff)
+
+static double* calib_field(Calib& c, const char* name)
+{
+#define X(f) if (!strcmp(name, #f)) return &c.f;
+    ADAPT_CALIB_FIELDS(X)
+#undef X
+    return nullptr;
+}
+extern "C" adapt_status_t adapt_set_calibration(const char* name, double value)
+{
+    State& S = st();
+    if (!name || !(value == value)) return fail(ADAPT_ERR_INVALID_ARG, "calibration: null name or NaN%s");
+    std::lock_guard<std::mutex> lock(S.mu);
+    double* f = calib_field(S.calib, name);
+    if (!f) return fail(ADAPT_ERR_INVALID_ARG, "unknown calibration constant %s", name);
+    *f = value;
+    return ADAPT_OK;
+}
+extern "C" adapt_status_t adapt_get_calibration(const char* name, double* value)
+{
+    State& S = st();
+    if (!name || !value) return fail(ADAPT_ERR_INVALID_ARG, "calibration: null argument%s");
+    std::lock_guard<std::mutex> lock(S.mu);
+    const double* f = calib_field(S.calib, name);
+    if (!f) return fail(ADAPT_ERR_INVALID_ARG, "unknown calibration constant %s", name);
+    *value = *f;
+    return ADAPT_OK;
+}
+extern "C" int adapt_calibration_names(char* out, int cap)
+{
+    static const char names[] =
+#define X(f) #f ","
+        ADAPT_CALIB_FIELDS(X)
+#undef X
+        ;
+    const int need = (int)sizeof(names) - 1;      // drop the last comma
+    if (out && cap > 0) {
+        const int n = need - 1 < cap - 1 ? need - 1 : cap - 1;
+        memcpy(out, names, (size_t)n);
+        out[n] = 0;
+    }
+    return need;
+}
+
 extern "C" adapt_status_t adapt_set_option(const char* name, int value)
 {
     State& S = st();

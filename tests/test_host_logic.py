@@ -296,3 +296,55 @@ def test_plan_table_round_trip_and_override(tmp_path):
     with pytest.raises(ab.AdaptError):
         ab.adapt_plan_table_load(str(tmp_path / "missing.txt"))
     ab.adapt_shutdown()
+
+
+def test_calibration_constants_round_trip_and_steer_the_model():
+    """The model's machine constants can be read and set by name; a plan made afterwards uses the new value
+    (halving the HBM rate makes a memory-bound shape's prediction longer), and unknown names are refused."""
+    names = ab.adapt_calibration_names()
+    assert "hbm_bw" in names and "launch_us" in names and len(names) == len(set(names)) >= 40
+    M, N, K, dt = 40000, 8, 40000, ab.F16         # memory-bound: 3.2 GB of A against 26 GFLOP
+    before = min(c.predicted_us for c in ab.adapt_plan_candidates(M, N, K, dt))
+    old = ab.adapt_get_calibration("hbm_bw")
+    try:
+        ab.adapt_set_calibration("hbm_bw", old / 2)
+        assert ab.adapt_get_calibration("hbm_bw") == old / 2
+        after = min(c.predicted_us for c in ab.adapt_plan_candidates(M, N, K, dt))
+        assert after > 1.3 * before
+    finally:
+        ab.adapt_set_calibration("hbm_bw", old)
+    assert min(c.predicted_us for c in ab.adapt_plan_candidates(M, N, K, dt)) == before
+    with pytest.raises(ab.AdaptError) as e:
+        ab.adapt_set_calibration("no_such_constant", 1.0)
+    assert e.value.status == ab.ERR_INVALID_ARG
+    with pytest.raises(ab.AdaptError):
+        ab.adapt_set_calibration("hbm_bw", float("nan"))
+
+
+def test_calibrate_fit_improves_or_keeps_the_regret_on_its_own_input(tmp_path):
+    """The fitting tool on a small synthetic table of timed configurations: times made from the model's own
+    predictions with one constant changed are explained again by moving that constant (the regret it reports
+    does not get worse, and the constant moves in the right direction)."""
+    import csv as _csv
+    from paper_2608_10803_b200 import calibrate
+    shapes = [(3000, 3000, 3000, 0), (5000, 40, 20000, 1), (64, 6000, 9000, 0), (9000, 9000, 24, 1), (300, 300, 30000, 0)]
+    old = ab.adapt_get_calibration("hbm_bw")
+    path = tmp_path / "cand.csv"
+    try:
+        ab.adapt_set_calibration("hbm_bw", old * 0.8)          # the "machine": a slower memory system
+        with open(path, "w", newline="") as f:
+            w = _csv.writer(f)
+            w.writerow("M,N,K,dtype,family,BN,stages,P_k,cluster,fused,streamk,srcA,srcB,pred_us,t_pro,t_main,t_epi,time_us".split(","))
+            for (M, N, K, dt) in shapes:
+                for c in ab.adapt_plan_candidates(M, N, K, dt)[:60]:
+                    w.writerow([M, N, K, dt, ab.FAMILY_NAMES[c.family], c.BN, c.stages, c.P_k, c.cluster, c.fused, c.streamk, c.srcA, c.srcB,
+                                0, 0, 0, 0, f"{c.predicted_us:.4f}"])
+        ab.adapt_set_calibration("hbm_bw", old)
+        ts = calibrate.TimedSet([str(path)])
+        m0 = ts.metrics(ab)
+        calibrate.fit([str(path), "--only", "hbm_bw"])
+        m1 = ts.metrics(ab)
+        assert m1["mean"] <= m0["mean"] + 1e-9 and m1["rms_log_error_near_best"] <= m0["rms_log_error_near_best"] + 1e-9
+        assert ab.adapt_get_calibration("hbm_bw") <= old
+    finally:
+        ab.adapt_set_calibration("hbm_bw", old)
