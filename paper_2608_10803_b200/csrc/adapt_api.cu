@@ -412,7 +412,7 @@ extern "C" void adapt_set_map_cache(int enabled) { st().map_cache.store(enabled 
     X(skinny_bw_eff_aligned) X(skinny_bw_eff_unaligned) X(skinny_fixed_us) X(skinny_pass_us) X(skinny_step_unaligned_us) X(skinny_mac_rate) \
     X(cluster_fixed_us) X(cluster_stage_us) X(cluster_reduce_us) X(cluster_crowd_us) X(cluster_crowd_stage_us) X(cluster_wave_us) \
     X(cluster_bw_eff) X(streamk_fixup_us) X(streamk_peer_us) X(fused_reduce_us) X(fused_wave_us) X(reduce_launch_us) X(dsmem_bw_per_sm) \
-    X(copy_bw_eff) X(hbm_bw_per_sm) X(class_view_sm_eff) X(class_tile_fixed_us) X(class_tile_fixed_unaligned_us) X(kclass_view_sm_eff) \
+    X(copy_bw_eff) X(hbm_bw_per_sm) X(class_view_sm_eff) X(class_tile_fixed_us) X(class_tile_fixed_unaligned_us) X(pair_class_tile_us) X(kclass_view_sm_eff) \
     X(kclass_unit_fixed_us) X(kclass_tile_drain_us) X(oob_box_penalty) X(reduce_batch_us) X(class_split_bw_eff) \
     X(class_split_bw_eff_per_log2m) X(class_split_fused_bw_eff) X(regroup_bw_eff) X(class_view_bw_eff)
 
@@ -627,6 +627,8 @@ static UmmaKernel launch_map_umma(int family, int BN, bool a_mn, bool b_mn, int 
     if (mode == 1 && family == ADAPT_FAM_UMMA_2CTA) {     // 256 rows of one row class per SM pair
         if (BN == 128) return (const void*)umma_gemm_kernel<128, false, true, 2, 1>;
         if (BN == 256) return (const void*)umma_gemm_kernel<256, false, true, 2, 1>;
+        if (BN == 144) return (const void*)umma_gemm_kernel<144, false, true, 2, 1>;    // 128 / 192 owned + 16 halo columns, 16 row classes
+        if (BN == 208) return (const void*)umma_gemm_kernel<208, false, true, 2, 1>;
         return nullptr;
     }
     if (mode == 1) {                     // row-major A read through per-row-class maps (1-CTA tiles, row-major B)
@@ -696,7 +698,7 @@ extern "C" adapt_status_t adapt_init(int device)
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
     CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_2CTA, 256, false, true, 2),
                                   cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
-    for (int BN : {128, 256})
+    for (int BN : {128, 256, 144, 208})
         CUDA_TRY(cudaFuncSetAttribute(launch_map_umma(ADAPT_FAM_UMMA_2CTA, BN, false, true, 1),
                                       cudaFuncAttributeMaxDynamicSharedMemorySize, S.machine.smem_bytes));
     for (int BN : {64, 128, 256}) {

@@ -107,6 +107,8 @@ struct Calib {
     double hbm_bw_per_sm = 55e9;        // B/s one SM streams from HBM (tail wave of 20000 x 8 x 60001: 15 MB per tile in 0.3 ms)
     double class_view_sm_eff = 0.935;    // per-SM rate through those views relative to l2_bw_per_sm (20000 x 8 x 60001 tail wave)
     double class_tile_fixed_us = 0.5, class_tile_fixed_unaligned_us = 0.99;   // per class tile (44479 x 54634 x 16..72, 64-column tiles)
+    double pair_class_tile_us = 1.0;    // pair tiles of one row class, rows with stale heads: the peer zeroes its half and tells the leader across
+                                        // the cluster before the tile's first MMA (7111 x 97981 x 289: 3.7 us per pair tile of six k-blocks)
     double kclass_view_sm_eff = 0.605;   // per-SM rate through the k-class views of B relative to l2_bw_per_sm (272 x 67839 x 6046: 48 KB per 0.75 us)
     double kclass_unit_fixed_us = 1.65;  // per unit of a k class run as a k split (1 x 80711 x 221: 18 units of one k-block in 37 us)
     double kclass_tile_drain_us = 2.5;  // drain of a tile with eight class accumulators (29 x 58492 x 94: 8 tile rounds in 35 us)

@@ -281,7 +281,7 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
         // (the bubble between the units of a k class shrinks as the unit's main loop grows)
         const double t_fixed = ksplit_cls ? std::max(0.0, cal.kclass_unit_fixed_us - 0.2 * (double)L * ii)
                              : c.srcA != ADAPT_SRC_TMA_CLASSES ? 0.0
-                             : (s.K % 8 ? cal.class_tile_fixed_unaligned_us : cal.class_tile_fixed_us);
+                             : (s.K % 8 ? cal.class_tile_fixed_unaligned_us + (c.cluster == 2 ? cal.pair_class_tile_us : 0.0) : cal.class_tile_fixed_us);
         // eight k-class accumulators fill TMEM: one tile at a time, its drain (eight-way sum, thread stores)
         // is not overlapped with the next tile's main loop
         const bool one_buffer = kclasses && !ksplit_cls;
@@ -451,7 +451,9 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
         if (halo_bn && (c.srcA != ADAPT_SRC_TMA_CLASSES || s.N % 16 == 0 || s.M < 16)) return false;
     } else {
         if (c.BM != 256 || c.cluster != 2) return false;
-        if (c.BN != 128 && c.BN != 256) return false;
+        const bool halo_bn = c.BN == 144 || c.BN == 208;                  // pair class tiles: 128 / 192 owned + 16 halo columns
+        if (c.BN != 128 && c.BN != 256 && !halo_bn) return false;
+        if (halo_bn && (c.srcA != ADAPT_SRC_TMA_CLASSES || s.N % 16 == 0 || s.M < 32)) return false;
     }
     if (c.BN % 16 != 0 || c.BN > 256) return false;                 // UMMA shape rule for M = 128/256
     if (2 * c.BN > m.tmem_cols) return false;                       // at least two accumulator buffers in TMEM
@@ -494,10 +496,10 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
         if (aligned16(innerB(s)) || s.K < 64 || c.srcA != ADAPT_SRC_PAD_COPY) return false;
     }
     if (classes) {
-        // rows of one residue class share their misalignment: row-major A and B; pair tiles (256 rows of one class)
-        // without halo columns only
+        // rows of one residue class share their misalignment: row-major A and B; pair tiles hold 256 rows of one class
+        // (with halo columns: 128 or 192 owned columns)
         if (s.layoutA != ADAPT_ROW_MAJOR || s.layoutB != ADAPT_ROW_MAJOR) return false;
-        if (c.family != ADAPT_FAM_UMMA_1CTA && (c.BN % 64 != 0 || s.M < 16)) return false;
+        if (c.family != ADAPT_FAM_UMMA_1CTA && (c.BN == 80 || s.M < (c.BN % 64 ? 32 : 16))) return false;
         // they pay when A's rows are unaligned (no copy), or when C's rows do not start on 32-byte sector
         // boundaries (halo tiles of 16 classes: uniform misalignment per tile, whole-sector TMA stores)
         if ((aligned16(innerA(s)) && c.BN % 64 == 0) || s.M < 8) return false;
@@ -706,9 +708,12 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
         }
     }
     // --- the same row-class views on pair tiles (256 rows of one class per SM pair), for an A with unaligned rows ---
-    if (a_unaligned && s.layoutA == ADAPT_ROW_MAJOR && s.layoutB == ADAPT_ROW_MAJOR && s.M >= 16) {
-        for (int BN : {128, 256}) {
-            const int64_t tiles = 8 * ceil_div(s.M, 2048) * ceil_div(s.N, BN);
+    //     ... and with halo columns (256 rows of one of 16 classes) for a C whose rows start off 32-byte boundaries
+    if ((a_unaligned || s.N % 16 != 0) && s.layoutA == ADAPT_ROW_MAJOR && s.layoutB == ADAPT_ROW_MAJOR && s.M >= 16) {
+        for (int BN : {128, 256, 144, 208}) {
+            const bool halo = BN % 64 != 0;
+            if (halo ? (s.N % 16 == 0 || s.M < 32) : !a_unaligned) continue;
+            const int64_t tiles = halo ? 16 * ceil_div(s.M, 4096) * ceil_div(s.N, BN - 16) : 8 * ceil_div(s.M, 2048) * ceil_div(s.N, BN);
             split_candidates(tiles, m.n_sm / 2, ceil_div(s.K + (s.K % 8 ? 7 : 0), 64), 2, &pks);
             for (int pk : pks) {
                 int deepest = umma_deepest_ring(BN, 2, 128, pk == 1, m.smem_bytes);

@@ -290,7 +290,6 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
     constexpr bool B_SPLIT = MODE == 3;                   // k classes as k splits (see below)
     static_assert(MODE == 0 || (!A_MN && B_MN), "class modes: K-major A, row-major B");
     static_assert(MODE != 2 || CG == 1, "tiles with eight class accumulators: one CTA per tile");
-    static_assert(MODE != 1 || CG == 1 || BN % 64 == 0, "pair tiles of one row class: no halo columns");
     static_assert(!B_CLS || BN == 64, "k-class mode uses 64-column windows");
     // HALO: class tiles for a C whose rows do not start on 32-byte boundaries (N % 16 != 0) own 32-byte
     // units of the shifted rows instead of columns, so they compute 16 columns more than they own (see

@@ -364,13 +364,15 @@ def synth_bits(t):
 
 # ---- class tiles with halo columns: C with N % 8 != 0 written through per-row-class TMA stores ------
 
-def halo_variants(M, N, K, dtype, limit=8):
-    """Class tiles with halo columns: for every tile width on offer, the best variant that stores C itself
-    (P_k = 1, the TMA-store epilogue) and the best one that writes fp32 partials."""
-    cands = [c for c in ab.adapt_plan_candidates(M, N, K, dtype) if c.srcA == 3 and c.BN % 64 != 0]
+def halo_variants(M, N, K, dtype, limit=12, family=None):
+    """Class tiles with halo columns: for every kernel family and tile width on offer, the best variant that stores
+    C itself (P_k = 1, the TMA-store epilogue) and the best one that writes fp32 partials."""
+    cands = [c for c in ab.adapt_plan_candidates(M, N, K, dtype) if c.srcA == 3 and c.BN % 64 != 0
+             and (family is None or c.family == family)]
     picked = []
-    for bn in sorted({c.BN for c in cands}):
-        picked += [c for c in cands if c.BN == bn and c.P_k == 1][:1] + [c for c in cands if c.BN == bn and c.P_k > 1][:1]
+    for fam, bn in sorted({(c.family, c.BN) for c in cands}):
+        mine = [c for c in cands if c.BN == bn and c.family == fam]
+        picked += [c for c in mine if c.P_k == 1][:1] + [c for c in mine if c.P_k > 1][:1]
     return [(ab.adapt_matmul_plan_forced(M, N, K, dtype, ROW, ROW, c.tiling_key), c) for c in picked[:limit]]
 
 
@@ -386,6 +388,41 @@ def test_halo_class_tiles_bit_exact(shape, dtype):
     assert {c.BN for _, c in variants} == {80, 144, 208}
     for plan, c in variants:
         check_case(M, N, K, dtype, A, B, plan=plan, exact=True)
+
+
+@pytest.mark.parametrize("dtype", [ab.F16, ab.BF16])
+@pytest.mark.parametrize("shape", [(1030, 265, 328), (1030, 265, 331), (4100, 1001, 64), (300, 521, 16), (40, 777, 200),
+                                   (4097, 201, 1003), (9000, 393, 24), (2100, 209, 700), (8200, 1537, 70), (5000, 193, 5)])
+def test_pair_halo_class_tiles_bit_exact(shape, dtype):
+    """Halo class tiles on SM pairs (256 rows of one of 16 row classes, 128 or 192 owned columns + 16 halo columns):
+    aligned and unaligned A, K shorter and longer than a k-block, M below and above one group of 4096 rows,
+    with the TMA-store epilogue and with fp32 partials, against the oracle on position-coded integers."""
+    M, N, K = shape
+    A = synth.position_coded(M, K, dtype, modulus=7, device="cuda")
+    B = synth.position_coded(K, N, dtype, modulus=5, device="cuda")
+    variants = halo_variants(M, N, K, dtype, family=ab.FAM_UMMA_2CTA)
+    assert variants and {c.BN for _, c in variants} == {144, 208}
+    for plan, c in variants:
+        check_case(M, N, K, dtype, A, B, plan=plan, exact=True)
+
+
+def test_pair_halo_class_tiles_random_values_and_guard_bands():
+    """Random values, C inside a buffer whose other bytes must stay as they were (the per-class TMA stores and the
+    narrow stores at the row ends write nothing beyond row M - 1 or column N - 1)."""
+    for (M, N, K, dtype) in [(2300, 1001, 520, ab.F16), (4200, 265, 40, ab.BF16)]:
+        A = synth.draw_operand(M, K, synth.U11, 31, dtype, "cuda")
+        B = synth.draw_operand(K, N, synth.U11, 32, dtype, "cuda")
+        guard = 4096
+        buf = torch.full((M * N + 2 * guard,), 77.0, dtype=A.dtype, device="cuda")
+        C = buf[guard:guard + M * N].view(M, N)
+        for plan, c in halo_variants(M, N, K, dtype, family=ab.FAM_UMMA_2CTA):
+            buf.fill_(77.0)
+            run_library(A, B, M, N, K, dtype, plan=plan, out=C)
+            torch.cuda.synchronize()
+            ab.adapt_poll_device_status(torch.cuda.current_stream().cuda_stream)
+            assert bool((buf[:guard] == 77.0).all()) and bool((buf[guard + M * N:] == 77.0).all())
+            err, mism, n = compare_with_oracle(A, B, C, M, N, K, dtype)
+            assert err <= TOL[dtype], (M, N, K, c.BN, c.P_k, err)
 
 
 def test_halo_class_tiles_with_unaligned_pointers():

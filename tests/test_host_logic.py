@@ -144,8 +144,8 @@ def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
                         assert c.srcA in (1, 3)      # re-pitched copy, or the per-row-class TMA views
                     if c.srcA == 3:
                         assert (K % 8 or halo) and M >= 8
-                        # pair tiles of one row class: 256 rows of a class per SM pair, no halo columns
-                        assert c.family == ab.FAM_UMMA_1CTA or (not halo and M >= 16 and c.BN in (128, 256))
+                        # pair tiles of one row class: 256 rows of a class per SM pair; with halo columns 128 or 192 owned ones
+                        assert c.family == ab.FAM_UMMA_1CTA or (M >= (32 if halo else 16) and c.BN in ((144, 208) if halo else (128, 256)))
                         assert c.P_m == ncls * -(-M // (128 * c.cluster * ncls))
                     if N % 8:
                         assert c.srcB in (1, 3)      # re-pitched copy, or the per-k-class TMA views
