@@ -77,15 +77,20 @@ typedef enum {
 
 /* How an operand reaches shared memory (the paper's Padding module, Table 2). */
 typedef enum {
-    ADAPT_SRC_TMA = 0,        /* TMA straight from the caller's buffer (needs 16 B pitch and base) */
-    ADAPT_SRC_PAD_COPY = 1,   /* prologue kernel re-pitches the operand into the workspace, then TMA (with srcB =
-                                 ADAPT_SRC_TMA_CLASSES: A is regrouped class-major instead) */
+    ADAPT_SRC_TMA = 0,        /* TMA straight from the caller's buffer (needs a 16 B pitch and base; an operand with
+                                 fewer than 64 contiguous elements also a multiple of 16 of them, so that TMA fetches
+                                 whole 32 B sectors) */
+    ADAPT_SRC_PAD_COPY = 1,   /* prologue kernel re-pitches the operand into the workspace (pitch a multiple of 32 B,
+                                 zeros in the pad columns), then TMA (with srcB = ADAPT_SRC_TMA_CLASSES: A is
+                                 regrouped class-major instead) */
     ADAPT_SRC_LSU = 2,        /* ordinary loads (skinny / SIMT / cluster families) */
     ADAPT_SRC_TMA_CLASSES = 3 /* class views, no copy of that operand.
                                  srcA: row-major A read in place through one TMA view per row class; tiles are made
                                  of every 8th row (BN = 64, 128, 256; needs K % 8 != 0) or, with 16 halo columns
                                  (BN = 80, 144, 208; needs N % 16 != 0, any K), of every 16th row, and C is then
-                                 written through per-class TMA stores.
+                                 written through per-class TMA stores; on pair tiles BN = 128, 256 and, with halo
+                                 columns, 144, 208.  An A narrower than 64 columns whose rows are not whole sectors
+                                 is re-pitched first and the views are taken of the copy.
                                  srcB: row-major B with N % 8 != 0 read in place through one view per k class
                                  (k % 8); BN = 64 keeps eight class accumulators per tile, BN = 128 / 256 makes
                                  each class a k split (P_k is then a multiple of 8) */

@@ -148,7 +148,7 @@ static void finish_common(const Shape& s, Config& c, const Calib& cal)
 }
 
 // Prologue (Section 5.2 "Prologue"): the Padding module re-pitches an operand whose rows are not
-// 16-byte multiples, reading it once and writing the padded copy once.
+// 16-byte multiples (or, for a narrow operand, not whole 32-byte sectors), reading it once and writing the padded copy once.
 static void model_prologue(const Shape& s, Config& c, const Calib& cal)
 {
     c.t_pro_us = 0;
