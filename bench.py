@@ -249,6 +249,8 @@ def ours(args):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     ab.adapt_init(local)
+    if args.batch_streams:
+        ab.adapt_set_option("batch_streams", args.batch_streams)
     stream = torch.cuda.current_stream().cuda_stream
     peaks = measured_peaks()
 
@@ -426,7 +428,8 @@ def ours(args):
         "config": {"workload": workload, "shapes": len(cases), "parallelism": f"replicas x{world} (no collective)",
                    "l2": "ring of resident operands (2 x %.0f GiB in, %.0f GiB out), far larger than L2, no reuse between consecutive calls"
                          % (args.pool_gb, out_bytes / gib),
-                   "timing": "CUDA events on the launching stream around K passes; per-shape: events around R back-to-back calls with rotated buffers, median of passes"},
+                   "timing": "CUDA events on the launching stream around K passes; per-shape: events around R back-to-back calls with rotated buffers, median of passes",
+                   "batch": "each pass is one adapt_matmul_batch call; the library spreads its calls over %s internal stream(s) between a fork from and a join to the launching stream and orders calls whose buffers overlap" % (args.batch_streams or 4)},
         "clocks": clocks, "gpu_launches": int(launches), "host_wall_ms_per_step": wall / args.steps * 1e3,
         "plan_ms_cold_total": plan_ms,
         "pointer_policy": {"operand_sets_per_shape_max": n_rot, "map_cache_slots_per_plan": 8,
@@ -796,6 +799,7 @@ def main():
     ap.add_argument("--workload", default="sweep", choices=["sweep", "configs"])
     ap.add_argument("--pool-gb", type=float, default=24.0, help="input pool per dtype, GiB")
     ap.add_argument("--shape-passes", type=int, default=3)
+    ap.add_argument("--batch-streams", type=int, default=0, help="1: the batch entry runs its calls one after the other (library default: four internal streams)")
     ap.add_argument("--e2e-steps", type=int, default=1)
     ap.add_argument("--limit", type=int, default=0)
     ap.add_argument("--no-e2e", action="store_true")

@@ -227,7 +227,14 @@ adapt_status_t adapt_matmul_noalloc(int64_t M, int64_t N, int64_t K, adapt_dtype
  * moved behind the boundary so that a caller in an interpreted language pays its foreign-call cost once per
  * batch, not once per GEMM; each GEMM is still its own launch(es).  The paper replaces the vendor's
  * MatMul / GroupMM operators in recommendation models (Section 6.5), whose layers issue exactly such
- * lists of small GEMMs of different shapes. */
+ * lists of small GEMMs of different shapes.
+ * A batch of eight or more calls is spread over up to four internal streams between a fork from and a join to
+ * cuda_stream (work queued on cuda_stream before the call comes first, work queued after it comes last), so that
+ * the launch gaps and the tail of one GEMM fill with the next one's work.  The result is the one of the calls made
+ * in order: a call whose output overlaps a buffer that an earlier call of the batch still reads or writes on another
+ * internal stream, or whose inputs overlap such an output, waits for that stream first.  Option "batch_streams"
+ * (adapt_set_option; 1 to 4, default 4) sets the number of internal streams; with 1 the calls run one after the
+ * other on cuda_stream itself.  The internal streams keep workspaces of their own. */
 adapt_status_t adapt_matmul_batch(int64_t count, const adapt_handle_t* plans, const void* const* A,
                                   const void* const* B, void* const* C, void* cuda_stream);
 
@@ -299,7 +306,8 @@ int64_t adapt_map_encode_count(void);
  *               amount that depends on the tile, so that the CTAs of a wave do not all ask for the same k slice of a shared
  *               operand at once.  The order is a function of the tile, so results stay reproducible, but they may differ
  *               in the last bit from those with the option off (another summation order).  Plain tiles only.
- *   "prefetch"  (default 1): L2 prefetch of a kernel's first operand boxes ahead of its wait for the kernel before it. */
+ *   "prefetch"  (default 1): L2 prefetch of a kernel's first operand boxes ahead of its wait for the kernel before it.
+ *   "batch_streams" (default 4): internal streams of adapt_matmul_batch, 1 to 4 (see there). */
 adapt_status_t adapt_set_option(const char* name, int value);
 
 /* The analytical model's calibration constants (Section 5.2's machine terms: bandwidths, latencies, per-tile and

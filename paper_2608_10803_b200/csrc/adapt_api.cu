@@ -142,6 +142,14 @@ struct State {
     std::atomic<int> map_cache{1};         // 0: every call encodes its maps afresh (measurement of the miss cost)
     int log = 0;
     int shuffle_k = 0;                 // ShuffleK analogue (ADAPT_SHUFFLE_K=1): rotated k-block order per tile; measured, off by default
+    // adapt_matmul_batch: up to four internal streams (lanes) between a fork from and a join to the caller's stream
+    struct BatchLanes {
+        cudaStream_t s[4] = {nullptr, nullptr, nullptr, nullptr};
+        cudaEvent_t fork = nullptr, join[4] = {nullptr, nullptr, nullptr, nullptr}, cross[4] = {nullptr, nullptr, nullptr, nullptr};
+        bool ready = false;
+    } lanes;
+    std::mutex batch_mu;               // one batch at a time uses the lanes
+    int batch_lanes = 4;               // "batch_streams" option (1 to 4): 1 = the calls of a batch run one after the other on the caller's stream
     int prefetch = 1;                  // L2 prefetch of a kernel's first operands ahead of its dependency wait (ADAPT_PREFETCH=0 turns it off)
     bool class_promo128 = true;        // 128-byte L2 promotion for the strided class views (ADAPT_CLASS_PROMO128=0: 256 as for dense operands)
 };
@@ -466,6 +474,7 @@ extern "C" adapt_status_t adapt_set_option(const char* name, int value)
     std::lock_guard<std::mutex> lock(S.mu);
     if (!strcmp(name, "shuffle_k")) S.shuffle_k = value ? 1 : 0;
     else if (!strcmp(name, "prefetch")) S.prefetch = value ? 1 : 0;
+    else if (!strcmp(name, "batch_streams")) S.batch_lanes = value >= 4 ? 4 : (value >= 2 ? value : 1);
     else return fail(ADAPT_ERR_INVALID_ARG, "unknown option %s", name);
     return ADAPT_OK;
 }
@@ -767,6 +776,15 @@ extern "C" void adapt_shutdown(void)
             if (hp.out) cudaStreamDestroy(hp.out);
         }
         S.pipes.clear();
+        if (S.lanes.ready) {
+            for (int l = 0; l < 4; ++l) {
+                cudaStreamDestroy(S.lanes.s[l]);
+                cudaEventDestroy(S.lanes.join[l]);
+                cudaEventDestroy(S.lanes.cross[l]);
+            }
+            cudaEventDestroy(S.lanes.fork);
+            S.lanes = State::BatchLanes();
+        }
         if (S.d_status) cudaFree(S.d_status);
         S.d_status = nullptr;
     }
@@ -1446,11 +1464,90 @@ extern "C" adapt_status_t adapt_matmul_batch(int64_t count, const adapt_handle_t
                                              const void* const* B, void* const* C, void* cuda_stream)
 {
     if (count < 0 || (count > 0 && (!plans || !A || !B || !C))) return fail(ADAPT_ERR_INVALID_ARG, "null array%s");
-    for (int64_t i = 0; i < count; ++i) {
-        const adapt_status_t r = adapt_matmul(plans[i], A[i], B[i], C[i], cuda_stream);
-        if (r != ADAPT_OK) return r;
+    State& S = st();
+    if (count < 8 || S.batch_lanes < 2 || !S.inited) {
+        for (int64_t i = 0; i < count; ++i) {
+            const adapt_status_t r = adapt_matmul(plans[i], A[i], B[i], C[i], cuda_stream);
+            if (r != ADAPT_OK) return r;
+        }
+        return ADAPT_OK;
     }
-    return ADAPT_OK;
+    // Lanes.  The calls of a batch are handed in turn to the lane with the least predicted work queued, so that the
+    // launch gaps and the tail of one call fill with the next call's work.  The result is the one of running the calls in
+    // order: a call whose output overlaps what the other lane still reads or writes, or whose inputs overlap what it
+    // writes, first waits for that lane; a lane remembers the buffers of its last 16 calls, and when that memory is
+    // full all other lanes are made to wait for it.  A stream-K call runs with nothing beside it: its CTAs wait for one another and
+    // must all be resident, which two such kernels sharing the SMs could deny each other.
+    std::lock_guard<std::mutex> batch_lock(S.batch_mu);
+    State::BatchLanes& L = S.lanes;
+    if (!L.ready) {
+        for (int l = 0; l < 4; ++l) {
+            CUDA_TRY(cudaStreamCreateWithFlags(&L.s[l], cudaStreamNonBlocking));
+            CUDA_TRY(cudaEventCreateWithFlags(&L.join[l], cudaEventDisableTiming));
+            CUDA_TRY(cudaEventCreateWithFlags(&L.cross[l], cudaEventDisableTiming));
+        }
+        CUDA_TRY(cudaEventCreateWithFlags(&L.fork, cudaEventDisableTiming));
+        L.ready = true;
+    }
+    const int NL = S.batch_lanes;
+    cudaStream_t user = (cudaStream_t)cuda_stream;
+    CUDA_TRY(cudaEventRecord(L.fork, user));
+    for (int l = 0; l < NL; ++l) CUDA_TRY(cudaStreamWaitEvent(L.s[l], L.fork, 0));
+    struct Range { uintptr_t lo, hi; };
+    constexpr size_t kLaneMemory = 32;
+    std::vector<Range> reads[4], writes[4];
+    double queued[4] = {0.0, 0.0, 0.0, 0.0};
+    auto hits = [](const std::vector<Range>& v, uintptr_t lo, uintptr_t hi) {
+        for (const Range& r : v) if (lo < r.hi && r.lo < hi) return true;
+        return false;
+    };
+    auto wait_for = [&](int lane, int other) -> adapt_status_t {      // `lane` continues after everything queued on `other`
+        CUDA_TRY(cudaEventRecord(L.cross[other], L.s[other]));
+        CUDA_TRY(cudaStreamWaitEvent(L.s[lane], L.cross[other], 0));
+        return ADAPT_OK;
+    };
+    adapt_status_t status = ADAPT_OK;
+    for (int64_t i = 0; i < count && status == ADAPT_OK; ++i) {
+        Plan* pl = plans[i];
+        if (!pl) { status = fail(ADAPT_ERR_INVALID_ARG, "null plan%s"); break; }
+        const Shape& sh = pl->s;
+        const uintptr_t a0 = (uintptr_t)A[i], b0 = (uintptr_t)B[i], c0 = (uintptr_t)C[i];
+        const uintptr_t a1 = a0 + (uintptr_t)sh.M * sh.K * 2, b1 = b0 + (uintptr_t)sh.K * sh.N * 2, c1 = c0 + (uintptr_t)sh.M * sh.N * 2;
+        int lane = 0;
+        for (int l = 1; l < NL; ++l) if (queued[l] < queued[lane]) lane = l;
+        const bool alone = pl->c.streamk != 0;
+        for (int o = 0; o < NL && status == ADAPT_OK; ++o) {
+            if (o == lane) continue;
+            if (alone || hits(reads[o], c0, c1) || hits(writes[o], c0, c1) || hits(writes[o], a0, a1) || hits(writes[o], b0, b1)) {
+                // everything lane o has queued comes first; what o did before is then ordered before all of this lane's
+                // later calls as well, but the other lanes still have to see it: keep o's memory
+                status = wait_for(lane, o);
+            }
+        }
+        if (status != ADAPT_OK) break;
+        if (reads[lane].size() >= kLaneMemory) {
+            // this lane's memory is full: every other lane waits for it, and it starts a new memory
+            for (int o = 0; o < NL && status == ADAPT_OK; ++o)
+                if (o != lane) status = wait_for(o, lane);
+            if (status != ADAPT_OK) break;
+            reads[lane].clear();
+            writes[lane].clear();
+        }
+        status = adapt_matmul(pl, A[i], B[i], C[i], (void*)L.s[lane]);
+        if (status != ADAPT_OK) break;
+        reads[lane].push_back({a0, a1});
+        reads[lane].push_back({b0, b1});
+        writes[lane].push_back({c0, c1});
+        queued[lane] += std::max(1.0, pl->c.predicted_us);
+        if (alone)
+            for (int o = 0; o < NL && status == ADAPT_OK; ++o)
+                if (o != lane) status = wait_for(o, lane);
+    }
+    // join, also after an error: the caller's stream continues after whatever was queued
+    for (int l = 0; l < NL; ++l) {
+        if (cudaEventRecord(L.join[l], L.s[l]) == cudaSuccess) (void)cudaStreamWaitEvent(user, L.join[l], 0);
+    }
+    return status;
 }
 
 extern "C" adapt_status_t adapt_matmul_repeat(adapt_handle_t plan, int sets, const void* const* A, const void* const* B,

@@ -648,6 +648,55 @@ def test_bounded_wait_expires_and_reports_a_timeout():
     check_case(M, N, K, dtype, A, B, exact=True)
 
 
+def test_batch_of_many_calls_on_internal_streams_matches_single_calls_and_keeps_dependences():
+    """A batch long enough for the internal streams of the batch entry: 40 independent calls of mixed shapes (stream-K, fused and
+    class-tile plans among them) give the bits of the same calls made one by one; then a chain inside one batch, every
+    call reading the output of the one before and the last overwriting the first one's output, gives what the chain gives
+    call by call (the batch entry orders calls whose buffers overlap)."""
+    init()
+    st = torch.cuda.current_stream().cuda_stream
+    base = [(131, 77, 259, ab.BF16), (512, 512, 2048, ab.BF16), (8, 3001, 400, ab.F16), (300, 520, 12, ab.F16), (2560, 2048, 2048, ab.F16),
+            (1, 4096, 4096, ab.BF16), (1030, 265, 331, ab.F16), (64, 64, 8192, ab.F16), (5, 640, 1000, ab.BF16), (2049, 128, 4099, ab.F16)]
+    shapes = [base[i % len(base)] for i in range(40)]
+    plans, As, Bs, C1, C2 = [], [], [], [], []
+    for i, (M, N, K, dt) in enumerate(shapes):
+        plans.append(ab.adapt_matmul_plan(M, N, K, dt))
+        As.append(synth.draw_operand(M, K, synth.U11, 170 + i, dt, "cuda"))
+        Bs.append(synth.draw_operand(K, N, synth.U11, 290 + i, dt, "cuda"))
+        C1.append(torch.full((M, N), float("nan"), dtype=As[-1].dtype, device="cuda"))
+        C2.append(torch.full((M, N), float("nan"), dtype=As[-1].dtype, device="cuda"))
+    for p, a, b, c in zip(plans, As, Bs, C1):
+        ab.adapt_matmul(p, a.data_ptr(), b.data_ptr(), c.data_ptr(), st)
+    for _ in range(2):
+        ab.adapt_matmul_batch(plans, [a.data_ptr() for a in As], [b.data_ptr() for b in Bs], [c.data_ptr() for c in C2], st)
+    torch.cuda.synchronize()
+    ab.adapt_poll_device_status(st)
+    for c1, c2 in zip(C1, C2):
+        assert torch.equal(c1.view(torch.int16), c2.view(torch.int16))
+    # a chain: X_{i+1} = X_i * W_i (square, small integers keep the values exact in fp16 for a while), in one batch
+    n, links = 256, 12
+    plan = ab.adapt_matmul_plan(n, n, n, ab.F16)
+    X0 = synth.position_coded(n, n, ab.F16, 3, "cuda")
+    eye = torch.eye(n, dtype=torch.float16, device="cuda")
+    Ws = [(eye + (torch.roll(eye, i + 1, 1) if i % 2 else 0)).contiguous() for i in range(links)]     # permutation-like, entries 0/1
+    def run(batch):
+        X = [X0.clone()] + [torch.full((n, n), float("nan"), dtype=torch.float16, device="cuda") for _ in range(links - 1)]
+        outs = X[1:] + [X[0]]                      # the last link writes over the first buffer
+        ins = [X[0]] + X[1:]
+        # link 0 reads X[0]; the last link writes X[0]: it must wait for link 0 as well as for its own input
+        ins = [X[i] for i in range(links)]
+        if batch:
+            ab.adapt_matmul_batch([plan] * links, [t.data_ptr() for t in ins], [w.data_ptr() for w in Ws], [t.data_ptr() for t in outs], st)
+        else:
+            for a, w, c in zip(ins, Ws, outs):
+                ab.adapt_matmul(plan, a.data_ptr(), w.data_ptr(), c.data_ptr(), st)
+        torch.cuda.synchronize()
+        return [t.clone() for t in X]
+    ref, got = run(False), run(True)
+    for r, g in zip(ref, got):
+        assert not torch.isnan(g).any() and torch.equal(r.view(torch.int16), g.view(torch.int16))
+
+
 def test_batched_entry_point_matches_single_calls():
     init()
     st = torch.cuda.current_stream().cuda_stream
