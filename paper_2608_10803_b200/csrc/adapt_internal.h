@@ -46,6 +46,10 @@ int calib_group(const Config& c);
 // (steps of 0.8, 0.9, 1.1, 1.25) on the mean regret of the model's pick over 654 sweep shapes with up to 128 timed
 // configurations each; on 300 shapes of another seed the mean regret went from 1.060 to 1.043 and the largest from 1.89 to
 // 1.64, on a third seed it is 1.052 and 1.71.  A second pass with finer steps gained nothing on the other seed and was dropped.
+// A later pass (same steps, two rounds) on 600 sweep shapes of any size, launch-bound ones included, timed with rotating
+// operand sets (cold operands, as in the sweep pass) moved twenty constants again (launch_us, the cluster and warp-level
+// kernels' terms, the thread-store drain, hbm_bw_per_sm among them): seeds 11, 23 and 37 (the last seen by no fit)
+// then give mean regrets 1.047, 1.039, 1.044 and maxima 1.81, 1.51, 1.58, with 45 to 53 % exact picks.
 struct Calib {
     // All ones: factors fitted on 34,000 timed configurations of 500 sweep shapes (0.72 for plain one-split tiles ... 1.19 for
     // fused k classes, 0.48 for the warp-level kernel) raised the mean regret on a held-out shape set from 1.063 to 1.076,
@@ -53,45 +57,45 @@ struct Calib {
     double group_bias[kCalibGroups] = {
         1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0,
         1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0, 1.0};
-    double launch_us = 1.92;             // one kernel launch issued back to back on a stream (also per reduce launch)
+    double launch_us = 1.54;             // one kernel launch issued back to back on a stream (also per reduce launch)
     double prologue_launch_us = 0.3;    // a re-pitch / regroup launch ahead of the GEMM: its launch overlaps the GEMM's own
                                         // (programmatic dependent launch); fit over 910 timed small configurations: -0.2 us
     double hbm_bw = 6.2e12;             // B/s, large streaming transfers
     double l2_bw_per_sm = 1.1e11;        // B/s one SM pulls through TMA from L2 (8192^3, 128 x 256 tiles: 48 KB per 0.48 us)
     double tensor_flops = 1.58e15;      // whole chip, kind::f16, BN = 256 (8192^3 on 256 x 256 pair tiles: 1.56e15)
     double eta_mma_bn128 = 0.518;        // relative tensor efficiency at BN = 128 (0.29 us per 128 x 128 x 64 block)
-    double eta_mma_bn64 = 0.36;         // ... at BN = 64 (A-operand smem reads dominate)
+    double eta_mma_bn64 = 0.324;         // ... at BN = 64 (A-operand smem reads dominate)
     double eta_2cta = 1.0;              // pair tiles share B: no extra tensor cost
     double mem_latency_us = 1.0;        // TMA issue -> data visible (sets Delta_dep with few stages)
-    double hbm_latency_us = 1.6;        // the same under a full HBM stream of a dense operand (128 x 128256 x 4096: 5 stages of 32 KB, 0.41 us each)
+    double hbm_latency_us = 1.04;        // the same under a full HBM stream of a dense operand (128 x 128256 x 4096: 5 stages of 32 KB, 0.41 us each)
     double hbm_latency_views_us = 1.6;  // ... through the strided class views (79457 x 196 x 8325 with 3 stages: 0.75 us per stage)
-    double umma_fixed_us = 1.38;         // barrier init, TMEM alloc, first load, last drain, TMEM free (the same fit: 2.5 was 3 us high)
+    double umma_fixed_us = 1.1;         // barrier init, TMEM alloc, first load, last drain, TMEM free (the same fit: 2.5 was 3 us high)
     // drain of one output tile through the epilogue warps (overlaps the next tile's main loop):
     // fixed part per tile + part per KB written; rows of C that are not 16-byte aligned cost more
     double epi_tile_fixed_us = 0.25, epi_us_per_kb = 0.0275;          // TMA stores (40000 x 40000 x 8: 4.8 TB/s)
-    double pair_drain_factor = 1.26;    // 40000 x 40000 x 8: 780 us on pair tiles, 671 us on 1-CTA tiles
-    double epi_partial_fixed_us = 0.44, epi_partial_us_per_kb = 0.0423;   // fp32 partials, stored by the epilogue threads
-    double epi_tile_fixed_unaligned_us = 1.28, epi_us_per_kb_unaligned = 0.0389;
-    double thread_store_exposed = 0.55;  // share of the main loop that a drain through the epilogue threads does not hide
+    double pair_drain_factor = 1.39;    // 40000 x 40000 x 8: 780 us on pair tiles, 671 us on 1-CTA tiles
+    double epi_partial_fixed_us = 0.44, epi_partial_us_per_kb = 0.0529;   // fp32 partials, stored by the epilogue threads
+    double epi_tile_fixed_unaligned_us = 1.41, epi_us_per_kb_unaligned = 0.0311;
+    double thread_store_exposed = 0.495;  // share of the main loop that a drain through the epilogue threads does not hide
     double thread_store_exposed_pair = 0.25;   // ... on pair tiles (13835 x 3906 x 852 and 7111 x 97981 x 289 bracket it)
-    double simt_flops = 15e12;          // CUDA-core tile kernel (1000^3: 17e12)
+    double simt_flops = 1.65e13;          // CUDA-core tile kernel (1000^3: 17e12)
     double simt_fixed_us = 0.45;
     double simt_step_us = 0.8;          // one 16-k step of a CTA alone on its SM (15 x 30 x 32: two steps, 4.85 us with the launch)
-    double halo_edge_tile_us = 0.8;     // row heads or tails of one halo tile (up to 15 elements per row, aligned stores of 2 to 16 bytes)
+    double halo_edge_tile_us = 0.72;     // row heads or tails of one halo tile (up to 15 elements per row, aligned stores of 2 to 16 bytes)
     double simt_bw_eff = 0.15;          // fraction of hbm_bw its 2-byte accesses reach (K = 1 outer products: 0.13 measured)
     double skinny_bw_eff_aligned = 0.55;    // fraction of hbm_bw the warp-level streaming kernel reaches, 16-byte aligned rows
                                             // (16 x 65536 x 4096: 3.5 TB/s with its loads four steps ahead of the MMAs, 1.6 before)
     double skinny_bw_eff_unaligned = 0.10;  // ... rows assembled from two chunks
-    double skinny_fixed_us = 2.0;
-    double skinny_pass_us = 5.5;        // one 64-row pass over one staged chunk when the streamed rows are k-contiguous
-    double skinny_step_unaligned_us = 2.8;   // one 16-k step of a warp when the streamed rows are unaligned
+    double skinny_fixed_us = 1.6;
+    double skinny_pass_us = 4.4;        // one 64-row pass over one staged chunk when the streamed rows are k-contiguous
+    double skinny_step_unaligned_us = 2.52;   // one 16-k step of a warp when the streamed rows are unaligned
     double skinny_mac_rate = 30e12;     // MAC/s ceiling of the warp-level kernel (small side padded to 16)
     // one-launch cluster kernel (64 x 64 tiles, k split over a cluster); least-squares fit over 180 timed
     // configurations of 2,000-sweep shapes: 3.7 + 0.95 stages + 0.8 (cluster > 1) + crowd (1.6 + 0.44 stages) us
     double cluster_fixed_us = 0.75;     // beyond the launch: barrier set-up, first trip to memory, rounding and store of the tile
-    double cluster_stage_us = 0.95;     // one 64-k stage: copy issue, shift pass, MMAs, each behind a CTA-wide barrier
-    double cluster_reduce_us = 0.8;     // cluster barriers + reading the partial tiles of the peers
-    double cluster_crowd_us = 1.56, cluster_crowd_stage_us = 0.44;   // per CTA per SM beyond one per two SMs
+    double cluster_stage_us = 0.76;     // one 64-k stage: copy issue, shift pass, MMAs, each behind a CTA-wide barrier
+    double cluster_reduce_us = 1.1;     // cluster barriers + reading the partial tiles of the peers
+    double cluster_crowd_us = 1.25, cluster_crowd_stage_us = 0.44;   // per CTA per SM beyond one per two SMs
     double cluster_wave_us = 5.5;       // each further round of clusters
     double cluster_bw_eff = 0.35;       // fraction of hbm_bw its 16-byte copies reach when memory-bound
     double streamk_fixup_us = 10.0;     // stream-K: partial tile out (5 us) and its fence, the flag, the owner's exposed last drain ...
@@ -104,10 +108,10 @@ struct Calib {
     double reduce_launch_us = 1.5;      // the reduce launch behind the GEMM: programmatic dependent launch hides about half of a launch
     double dsmem_bw_per_sm = 60e9;      // B/s one SM reads from its peers' shared memory during the fused reduction
     double copy_bw_eff = 0.935;          // pad-copy and reduce kernels
-    double hbm_bw_per_sm = 55e9;        // B/s one SM streams from HBM (tail wave of 20000 x 8 x 60001: 15 MB per tile in 0.3 ms)
+    double hbm_bw_per_sm = 7.56e10;        // B/s one SM streams from HBM (tail wave of 20000 x 8 x 60001: 15 MB per tile in 0.3 ms)
     double class_view_sm_eff = 0.935;    // per-SM rate through those views relative to l2_bw_per_sm (20000 x 8 x 60001 tail wave)
-    double class_tile_fixed_us = 0.5, class_tile_fixed_unaligned_us = 0.99;   // per class tile (44479 x 54634 x 16..72, 64-column tiles)
-    double pair_class_tile_us = 1.0;    // pair tiles of one row class, rows with stale heads: the peer zeroes its half and tells the leader across
+    double class_tile_fixed_us = 0.625, class_tile_fixed_unaligned_us = 0.99;   // per class tile (44479 x 54634 x 16..72, 64-column tiles)
+    double pair_class_tile_us = 1.1;    // pair tiles of one row class, rows with stale heads: the peer zeroes its half and tells the leader across
                                         // the cluster before the tile's first MMA (7111 x 97981 x 289: 3.7 us per pair tile of six k-blocks)
     double kclass_view_sm_eff = 0.605;   // per-SM rate through the k-class views of B relative to l2_bw_per_sm (272 x 67839 x 6046: 48 KB per 0.75 us)
     double kclass_unit_fixed_us = 1.65;  // per unit of a k class run as a k split (1 x 80711 x 221: 18 units of one k-block in 37 us)
