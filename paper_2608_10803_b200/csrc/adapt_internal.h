@@ -49,7 +49,9 @@ int calib_group(const Config& c);
 // A later pass (same steps, two rounds) on 600 sweep shapes of any size, launch-bound ones included, timed with rotating
 // operand sets (cold operands, as in the sweep pass) moved twenty constants again (launch_us, the cluster and warp-level
 // kernels' terms, the thread-store drain, hbm_bw_per_sm among them): seeds 11, 23 and 37 (the last seen by no fit)
-// then give mean regrets 1.047, 1.039, 1.044 and maxima 1.81, 1.51, 1.58, with 45 to 53 % exact picks.
+// then give mean regrets 1.047, 1.039, 1.044 and maxima 1.81, 1.51, 1.58, with 45 to 53 % exact picks.  Of that pass
+// hbm_bw_per_sm was taken back from 75.6 to 60.5 GB/s: the larger value hides the cost of a partial last wave on the
+// heaviest shapes (61370 x 32 x 85272 picked without split or stream-K: 2275 against 1700 us), 1.4 % of their time in total.
 struct Calib {
     // All ones: factors fitted on 34,000 timed configurations of 500 sweep shapes (0.72 for plain one-split tiles ... 1.19 for
     // fused k classes, 0.48 for the warp-level kernel) raised the mean regret on a held-out shape set from 1.063 to 1.076,
@@ -108,7 +110,7 @@ struct Calib {
     double reduce_launch_us = 1.5;      // the reduce launch behind the GEMM: programmatic dependent launch hides about half of a launch
     double dsmem_bw_per_sm = 60e9;      // B/s one SM reads from its peers' shared memory during the fused reduction
     double copy_bw_eff = 0.935;          // pad-copy and reduce kernels
-    double hbm_bw_per_sm = 7.56e10;        // B/s one SM streams from HBM (tail wave of 20000 x 8 x 60001: 15 MB per tile in 0.3 ms)
+    double hbm_bw_per_sm = 6.05e10;        // B/s one SM streams from HBM (tail wave of 20000 x 8 x 60001: 15 MB per tile in 0.3 ms)
     double class_view_sm_eff = 0.935;    // per-SM rate through those views relative to l2_bw_per_sm (20000 x 8 x 60001 tail wave)
     double class_tile_fixed_us = 0.625, class_tile_fixed_unaligned_us = 0.99;   // per class tile (44479 x 54634 x 16..72, 64-column tiles)
     double pair_class_tile_us = 1.1;    // pair tiles of one row class, rows with stale heads: the peer zeroes its half and tells the leader across
