@@ -697,6 +697,46 @@ def test_batch_of_many_calls_on_internal_streams_matches_single_calls_and_keeps_
         assert not torch.isnan(g).any() and torch.equal(r.view(torch.int16), g.view(torch.int16))
 
 
+def test_batch_entry_can_be_captured_into_a_cuda_graph_and_replayed():
+    """After a warm-up call (workspaces grown, tensor maps cached) the batch entry only launches kernels and records
+    and waits for events, so a stream capture takes it, internal streams included; replays give the bits of the direct
+    calls, also after the inputs change in place."""
+    init()
+    shapes = [(131, 77, 259, ab.BF16), (512, 512, 2048, ab.BF16), (8, 3001, 400, ab.F16), (300, 520, 12, ab.F16), (1030, 265, 331, ab.F16),
+              (64, 64, 8192, ab.F16), (5, 640, 1000, ab.BF16), (1, 4096, 4096, ab.BF16), (200, 264, 328, ab.F16), (77, 50, 1, ab.F16)]
+    plans, As, Bs, Cd, Cg = [], [], [], [], []
+    for i, (M, N, K, dt) in enumerate(shapes):
+        plans.append(ab.adapt_matmul_plan(M, N, K, dt))
+        As.append(synth.draw_operand(M, K, synth.U11, 400 + i, dt, "cuda"))
+        Bs.append(synth.draw_operand(K, N, synth.U11, 500 + i, dt, "cuda"))
+        Cd.append(torch.full((M, N), float("nan"), dtype=As[-1].dtype, device="cuda"))
+        Cg.append(torch.full((M, N), float("nan"), dtype=As[-1].dtype, device="cuda"))
+    pa, pb = ab.pointer_array([t.data_ptr() for t in As]), ab.pointer_array([t.data_ptr() for t in Bs])
+    pd, pg, pp = ab.pointer_array([t.data_ptr() for t in Cd]), ab.pointer_array([t.data_ptr() for t in Cg]), ab.pointer_array(plans)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for _ in range(2):
+            ab.adapt_matmul_batch(pp, pa, pb, pg, side.cuda_stream)          # warm-up on the capturing stream
+        side.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=side):
+            ab.adapt_matmul_batch(pp, pa, pb, pg, side.cuda_stream)
+    torch.cuda.synchronize()
+    st = torch.cuda.current_stream().cuda_stream
+    for round_ in range(2):
+        for c in Cg:
+            c.fill_(float("nan"))
+        torch.cuda.synchronize()
+        graph.replay()
+        ab.adapt_matmul_batch(pp, pa, pb, pd, st)
+        torch.cuda.synchronize()
+        ab.adapt_poll_device_status(st)
+        for cd, cg in zip(Cd, Cg):
+            assert not torch.isnan(cg).any() and torch.equal(cd.view(torch.int16), cg.view(torch.int16))
+        for a in As:                                  # new contents, same buffers: the replay must follow
+            a.mul_(-0.5)
+
+
 def test_batched_entry_point_matches_single_calls():
     init()
     st = torch.cuda.current_stream().cuda_stream
