@@ -1131,9 +1131,10 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
 
     // write-bound shapes (C outweighs the operands) walk the tiles row block by row block
     // (2048 x 97328 x 64: 80 -> 71 us, 94851 x 69977 x 12: 2740 -> 2580 us), unless K is so short that the one A tile all
-    // concurrent CTAs of a row block then read is a handful of cache lines (2048 x 97328 x 8: 86 -> 124 us that way)
+    // concurrent CTAs of a row block then read is a handful of cache lines and the rows are few (2048 x 97328 x 8: 74 -> 84 us
+    // that way; from 64 row blocks on the row-block order wins again: 16384 x 97328 x 8: 653 -> 600 us, 40000 x 40000 x 8: 638 -> 592 us)
     p.raster = (p.P_k == 1 && (double)s.M * (double)s.N >= (double)s.K * ((double)s.M + (double)s.N) &&
-                (s.K >= 32 || p.P_n <= 64 || classesA)) ? 1 : 0;
+                (s.K >= 32 || p.P_n <= 64 || classesA || p.P_m > 32)) ? 1 : 0;
     if (const char* e = getenv("ADAPT_RASTER")) p.raster = atoi(e);
     p.prefetch = S.prefetch;
     p.shuffle_k = S.shuffle_k;
