@@ -1038,7 +1038,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     p.P_m = c.P_m;
     // a plan made for k-class views that has to fall back to a copy of B (unaligned pointer) uses plain tiles
     p.P_n = (c.srcB == ADAPT_SRC_TMA_CLASSES && !kclsB) ? (int)ceil_div(s.N, c.BN) : c.P_n;
-    p.kb_total = kclsB ? (int)(Kc / kUmmaBK) : (int)ceil_div(s.K + ((classesA && s.K % 8) ? 7 : 0), kUmmaBK);
+    p.kb_total = kclsB ? (int)(Kc / kUmmaBK) : (int)ceil_div(s.K + (classesA ? class_k_slack(s) : 0), kUmmaBK);
     const bool ksplit_cls = kclsB && c.BN != 64;            // k classes as k splits: P_k = 8 * (splits per class)
     if (ksplit_cls) {
         p.kb_per_split = (int)ceil_div(p.kb_total, c.P_k / 8);
@@ -1105,7 +1105,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     } else {
         // a row-major B whose K fits one k-block is loaded with boxes of just the k rows that exist (rounded up to 8; class
         // tiles shift B's rows by up to 7): boxes of 64 rows that lie mostly beyond K load several times slower when B is wide
-        if (b_mn && p.kb_total == 1) b_box_k = (int)std::min<int64_t>(64, round_up(s.K + ((classesA && s.K % 8) ? 7 : 0), 8));
+        if (b_mn && p.kb_total == 1) b_box_k = (int)std::min<int64_t>(64, round_up(s.K + (classesA ? class_k_slack(s) : 0), 8));
         if ((r = cached_map(S, pl, kMapB, b_src, extB, outB, pitchB, 64, b_mn ? b_box_k : c.BN / cg, &maps.b[0])) != ADAPT_OK) return r;
     }
 

@@ -194,6 +194,9 @@ inline int64_t padded_pitch(int64_t inner) { return round_up(inner, 16); }
 // Class tiles read a row-major A in place through their per-class views, except a narrow one whose rows are not whole
 // sectors: that one is re-pitched first (the views of the copy are then all aligned).
 inline bool class_tiles_copy_a(const Shape& s) { return s.K < 64 && !tma_friendly(s.K); }
+// Class tiles over an A whose rows are unaligned shift the k index by up to 7 elements (one more k-block at most); over a
+// copy every view is aligned and nothing shifts.
+inline int64_t class_k_slack(const Shape& s) { return (s.K % 8 != 0 && !class_tiles_copy_a(s)) ? 7 : 0; }
 
 const Calib& default_calib();
 

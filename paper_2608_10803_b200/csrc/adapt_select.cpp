@@ -211,7 +211,7 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
 {
     const bool kclasses = c.srcB == ADAPT_SRC_TMA_CLASSES;
     const int64_t kblocks = kclasses ? ceil_div(ceil_div(s.K, 8), c.BK)
-                                     : ceil_div(s.K + ((c.srcA == ADAPT_SRC_TMA_CLASSES && s.K % 8) ? 7 : 0), c.BK);
+                                     : ceil_div(s.K + (c.srcA == ADAPT_SRC_TMA_CLASSES ? class_k_slack(s) : 0), c.BK);
     const bool ksplit_cls = kclasses && c.BN != 64;                       // each class a k split of its own
     const int64_t L = ksplit_cls ? ceil_div(kblocks, c.P_k / 8)
                                  : ceil_div(kblocks, c.P_k) * (kclasses ? 8 : 1);   // BN = 64: the split's blocks of all 8 classes
@@ -474,7 +474,7 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     // in class mode the k index of a tile is shifted by up to 7 elements
     // k-class mode splits the blocks of one class; in row-class mode the k index is shifted by up to 7
     const int64_t kblocks = c.srcB == ADAPT_SRC_TMA_CLASSES ? ceil_div(ceil_div(s.K, 8), c.BK)
-                                                              : ceil_div(s.K + ((c.srcA == ADAPT_SRC_TMA_CLASSES && s.K % 8) ? 7 : 0), c.BK);
+                                                              : ceil_div(s.K + (c.srcA == ADAPT_SRC_TMA_CLASSES ? class_k_slack(s) : 0), c.BK);
     // k classes as k splits (k-class views of B with BN > 64): P_k = 8 * (splits of one class's blocks)
     const bool ksplit_cls = c.srcB == ADAPT_SRC_TMA_CLASSES && c.BN != 64;
     if (ksplit_cls && c.P_k % 8 != 0) return false;
@@ -690,7 +690,7 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
             if (halo && (s.N % 16 == 0 || s.M < 16)) continue;             // halo tiles serve a C off 32-byte boundaries only
             if (!halo && !a_unaligned) continue;                           // aligned A: class tiles only for their stores
             const int64_t tiles = (halo ? 16 * ceil_div(s.M, 2048) : 8 * ceil_div(s.M, 1024)) * ceil_div(s.N, halo ? BN - 16 : BN);
-            split_candidates(tiles, m.n_sm, ceil_div(s.K + (s.K % 8 ? 7 : 0), 64), 2, &pks);
+            split_candidates(tiles, m.n_sm, ceil_div(s.K + class_k_slack(s), 64), 2, &pks);
             for (int pk : pks) {
                 const int deepest = umma_deepest_ring(BN, 1, umma_a_box_rows(s, 1, halo ? 16 : 8, false), pk == 1, m.smem_bytes);
                 Config d;
@@ -714,7 +714,7 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
             const bool halo = BN % 64 != 0;
             if (halo ? (s.N % 16 == 0 || s.M < 32) : !a_unaligned) continue;
             const int64_t tiles = halo ? 16 * ceil_div(s.M, 4096) * ceil_div(s.N, BN - 16) : 8 * ceil_div(s.M, 2048) * ceil_div(s.N, BN);
-            split_candidates(tiles, m.n_sm / 2, ceil_div(s.K + (s.K % 8 ? 7 : 0), 64), 2, &pks);
+            split_candidates(tiles, m.n_sm / 2, ceil_div(s.K + class_k_slack(s), 64), 2, &pks);
             for (int pk : pks) {
                 int deepest = umma_deepest_ring(BN, 2, 128, pk == 1, m.smem_bytes);
                 if (deepest > 8) deepest = 8;
