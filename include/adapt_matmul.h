@@ -87,8 +87,8 @@ typedef enum {
     ADAPT_SRC_TMA_CLASSES = 3 /* class views, no copy of that operand.
                                  srcA: row-major A read in place through one TMA view per row class; tiles are made
                                  of every 8th row (BN = 64, 128, 256; needs K % 8 != 0) or, with 16 halo columns
-                                 (BN = 80, 144, 208; needs N % 16 != 0, any K), of every 16th row, and C is then
-                                 written through per-class TMA stores; on pair tiles BN = 128, 256 and, with halo
+                                 (BN = 80, 144, 208; needs N % 16 != 0, any K), of every 16th row (every 8th, 4th or
+                                 2nd when an even N and K allow it), and C is then written through per-class TMA stores; on pair tiles BN = 128, 256 and, with halo
                                  columns, 144, 208.  An A narrower than 64 columns whose rows are not whole sectors
                                  is re-pitched first and the views are taken of the copy.
                                  srcB: row-major B with N % 8 != 0 read in place through one view per k class

@@ -1026,7 +1026,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
 
     const int cg = c.cluster;
     const bool halo = classesA && c.BN % 64 != 0;           // class tiles with 16 halo columns (C's rows off 32-byte boundaries)
-    const int ncls = halo ? 16 : 8;                         // row classes of a class tile
+    const int ncls = halo ? halo_row_classes(s) : 8;        // row classes of a class tile
     struct { CUtensorMap a[16], b[8], c[16]; } maps;
     UmmaParams p;
     int a_box_rows = 128;
@@ -1138,6 +1138,7 @@ adapt_status_t run_umma(State& S, Plan* pl, const void* A, const void* B, void* 
     if (const char* e = getenv("ADAPT_RASTER")) p.raster = atoi(e);
     p.prefetch = S.prefetch;
     p.shuffle_k = S.shuffle_k;
+    p.ncls_log2 = ncls == 16 ? 4 : (ncls == 8 ? 3 : (ncls == 4 ? 2 : 1));
     p.force_partial = epi ? 1 : 0;
     p.a_shift_any = 0;
     for (int j = 0; j < 16; ++j) p.a_shift_any |= p.a_sigma[j];

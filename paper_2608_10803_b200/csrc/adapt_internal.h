@@ -284,7 +284,19 @@ inline int umma_a_box_rows(const Shape& s, int cluster, int row_classes, bool k_
     return 128;
 }
 
-// Row classes of a configuration's tiles: 0 (plain tiles), 8 (class tiles), 16 (class tiles with halo columns).
-inline int umma_row_classes(int srcA, int BN) { return srcA != ADAPT_SRC_TMA_CLASSES ? 0 : (BN % 64 ? 16 : 8); }
+// Row classes of halo class tiles.  The rows of one class must share their offset from a 32-byte boundary in C (rows j and
+// j + n do when n * N is a multiple of 16 elements: n = 16 for an odd N, 8, 4 or 2 for an even one) and, when A is read in
+// place, their offset from a 16-byte boundary in A (n * K a multiple of 8).  As few classes as that allows: the rows of a
+// tile are then n rows of C apart, and a TMA store box whose rows lie 2 MiB or more apart writes slower (16 classes at
+// N = 99991: 4.2 TB/s; 8 classes at N = 99990: 5.5 TB/s); a smaller n also wastes less of a ragged M.
+inline int gcd_pow2(int64_t v, int p2) { int g = 1; while (g < p2 && v % (2 * g) == 0) g *= 2; return g; }
+inline int halo_row_classes(const Shape& s)
+{
+    const int for_c = 16 / gcd_pow2(s.N % 16 == 0 ? 16 : s.N % 16, 16);
+    const int for_a = class_tiles_copy_a(s) ? 1 : 8 / gcd_pow2(s.K % 8 == 0 ? 8 : s.K % 8, 8);
+    return std::max(2, std::max(for_c, for_a));
+}
+// Row classes of a configuration's tiles: 0 (plain tiles), 8 (class tiles), 2 to 16 (class tiles with halo columns).
+inline int umma_row_classes(const Shape& s, int srcA, int BN) { return srcA != ADAPT_SRC_TMA_CLASSES ? 0 : (BN % 64 ? halo_row_classes(s) : 8); }
 
 }  // namespace adapt

@@ -233,7 +233,7 @@ static void model_umma(const Shape& s, const Machine& m, const Calib& cal, Confi
 
     // per-SM stage: each CTA loads its 128 rows of A and its share of the BN columns of B
     const double bn_per_cta = (double)c.BN / c.cluster;
-    const double a_rows = umma_a_box_rows(s, c.cluster, umma_row_classes(c.srcA, c.BN), kclasses);
+    const double a_rows = umma_a_box_rows(s, c.cluster, umma_row_classes(s, c.srcA, c.BN), kclasses);
     const double stage_bytes = 2.0 * c.BK * (a_rows + (double)round_up((int64_t)bn_per_cta, 64));
     // One SM pulls operands that other SMs also use from L2 at l2_bw_per_sm (a little less through
     // the strided row-class views); a stream that comes from HBM and is used once is bounded by the
@@ -462,7 +462,7 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
         // plain tiles, one split, not fused; needs leftover tiles and at least two k-blocks per slot in the shared part
         if (c.P_k != 1 || c.fused || c.srcA == ADAPT_SRC_TMA_CLASSES || c.srcB == ADAPT_SRC_TMA_CLASSES || c.stages < 2) return false;
     }
-    const int a_rows_box = umma_a_box_rows(s, c.cluster, umma_row_classes(c.srcA, c.BN), c.srcB == ADAPT_SRC_TMA_CLASSES);
+    const int a_rows_box = umma_a_box_rows(s, c.cluster, umma_row_classes(s, c.srcA, c.BN), c.srcB == ADAPT_SRC_TMA_CLASSES);
     if (c.fused) {
         // the k splits of a tile form one cluster: 1-CTA tiles, a portable cluster size, no halo tiles, not the
         // eight-accumulator k-class tiles
@@ -506,7 +506,7 @@ static bool legal_umma(const Shape& s, const Machine& m, Config& c)
     }
     if (c.srcA == ADAPT_SRC_PAD_COPY && tma_friendly(innerA(s)) && !kclasses) return false;    // nothing to pad
     if (c.srcB == ADAPT_SRC_PAD_COPY && tma_friendly(innerB(s))) return false;
-    const int ncls = umma_row_classes(c.srcA, c.BN);
+    const int ncls = umma_row_classes(s, c.srcA, c.BN);
     c.P_m = classes ? (int)(ncls * ceil_div(s.M, ncls * c.BM)) : (int)ceil_div(s.M, c.BM);   // class tiles: 8 per 1024 rows (pair tiles: per 2048), 16 per 2048
     c.P_n = (int)ceil_div(s.N, kclasses ? c.BN - 8 : (c.BN % 64 ? c.BN - 16 : c.BN));
     if ((int64_t)c.P_m * c.P_n * c.P_k > (int64_t)1 << 30) return false;
@@ -689,10 +689,11 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
             const bool halo = BN % 64 != 0;
             if (halo && (s.N % 16 == 0 || s.M < 16)) continue;             // halo tiles serve a C off 32-byte boundaries only
             if (!halo && !a_unaligned) continue;                           // aligned A: class tiles only for their stores
-            const int64_t tiles = (halo ? 16 * ceil_div(s.M, 2048) : 8 * ceil_div(s.M, 1024)) * ceil_div(s.N, halo ? BN - 16 : BN);
+            const int hc = halo_row_classes(s);
+            const int64_t tiles = (halo ? hc * ceil_div(s.M, 128 * hc) : 8 * ceil_div(s.M, 1024)) * ceil_div(s.N, halo ? BN - 16 : BN);
             split_candidates(tiles, m.n_sm, ceil_div(s.K + class_k_slack(s), 64), 2, &pks);
             for (int pk : pks) {
-                const int deepest = umma_deepest_ring(BN, 1, umma_a_box_rows(s, 1, halo ? 16 : 8, false), pk == 1, m.smem_bytes);
+                const int deepest = umma_deepest_ring(BN, 1, umma_a_box_rows(s, 1, halo ? hc : 8, false), pk == 1, m.smem_bytes);
                 Config d;
                 d.family = ADAPT_FAM_UMMA_1CTA; d.BM = 128; d.BN = BN; d.BK = 64; d.cluster = 1;
                 d.stages = deepest; d.P_k = pk; d.srcA = ADAPT_SRC_TMA_CLASSES; d.srcB = srcB;
@@ -713,7 +714,8 @@ void enumerate_configs(const Shape& s, const Machine& m, const Calib& cal, std::
         for (int BN : {128, 256, 144, 208}) {
             const bool halo = BN % 64 != 0;
             if (halo ? (s.N % 16 == 0 || s.M < 32) : !a_unaligned) continue;
-            const int64_t tiles = halo ? 16 * ceil_div(s.M, 4096) * ceil_div(s.N, BN - 16) : 8 * ceil_div(s.M, 2048) * ceil_div(s.N, BN);
+            const int hc = halo_row_classes(s);
+            const int64_t tiles = halo ? hc * ceil_div(s.M, 256 * hc) * ceil_div(s.N, BN - 16) : 8 * ceil_div(s.M, 2048) * ceil_div(s.N, BN);
             split_candidates(tiles, m.n_sm / 2, ceil_div(s.K + class_k_slack(s), 64), 2, &pks);
             for (int pk : pks) {
                 int deepest = umma_deepest_ring(BN, 2, 128, pk == 1, m.smem_bytes);

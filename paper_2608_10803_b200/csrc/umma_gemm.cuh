@@ -73,6 +73,7 @@ struct UmmaParams {
     unsigned int sk_epoch;           // this launch's epoch (unique per workspace)
     int x_rows, x_pitch;             // fused split-K: rows and row pitch (fp32 elements) of the partial tile each CTA of the
                                      // cluster keeps in its shared memory for the exchange
+    int ncls_log2;                   // halo class tiles: log2 of the number of row classes (1 .. 4)
     unsigned int* status;            // device status word: bit 0 = a bounded wait expired
     unsigned long long* trace;       // timestamp trace of one CTA (diagnostic builds only), else null
     int trace_cta;
@@ -296,7 +297,10 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
     // the epilogue); they use 16 row classes, since rows 16 apart share their offset from such a boundary
     constexpr bool HALO = A_CLS && (BN % 64 != 0);
     static_assert(BN % 64 == 0 || (A_CLS && (BN - 16) % 64 == 0), "BN is a multiple of 64, plus 16 halo columns for class tiles");
-    constexpr int NCLS = HALO ? 16 : 8;                   // row classes of a class tile: rows NCLS*128*g + j + NCLS*i
+    // row classes of a class tile (rows NCLS*128*g + j + NCLS*i): 8, or for halo tiles as many as C's rows need to share
+    // their offset from a 32-byte boundary (16 for an odd N, 8, 4 or 2 for an even one: p.ncls_log2)
+    const int NSH = HALO ? p.ncls_log2 : 3;
+    const int NCLS = 1 << NSH;
     constexpr int TILE_N = B_CLS ? 56 : (B_SPLIT ? BN - 8 : (HALO ? BN - 16 : BN));   // output columns (HALO: chunk-aligned elements) a tile owns
     constexpr int BN_CTA = BN / CG;                       // B columns this CTA loads
     // the A region of a stage holds the rows one box brings (128, or fewer for a short K-major A)
@@ -369,9 +373,9 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
         int mb0 = 0, nb0 = 0, sp0 = 0;
         const int first_unit = (CG == 2) ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
         if (first_unit < p.num_units) decode_unit(p, first_unit, mb0, nb0, sp0);
-        ptx::prefetch_tensormap(&maps.a[A_CLS ? (mb0 % NCLS) : 0]);
+        ptx::prefetch_tensormap(&maps.a[A_CLS ? (mb0 & (NCLS - 1)) : 0]);
         ptx::prefetch_tensormap(&maps.b[(B_SPLIT || B_CLS) ? (sp0 & 7) : 0]);
-        if (p.c_mode != 0) ptx::prefetch_tensormap(&maps.c[A_CLS ? (mb0 % NCLS) : 0]);
+        if (p.c_mode != 0) ptx::prefetch_tensormap(&maps.c[A_CLS ? (mb0 & (NCLS - 1)) : 0]);
     }
     if (warp == 1) {
         ptx::tmem_alloc<CG>(tmem_slot, TMEM_COLS);
@@ -408,8 +412,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
         constexpr int NREQ = NREQ_A + (B_MN ? B_BOXES : 1);
         WorkItem w;
         if (lane < NREQ && next_item<SK, B_SPLIT>(p, unit0, unit_step, 0, w)) {
-            const int cls = A_CLS ? (w.mb % NCLS) : 0;
-            const int row0 = A_CLS ? (w.mb / NCLS) * (128 * CG) + (int)cta_rank * 128 : w.mb * (128 * CG) + (int)cta_rank * 128;
+            const int cls = A_CLS ? (w.mb & (NCLS - 1)) : 0;
+            const int row0 = A_CLS ? (w.mb >> NSH) * (128 * CG) + (int)cta_rank * 128 : w.mb * (128 * CG) + (int)cta_rank * 128;
             const int kshift = A_CLS ? p.a_sigma[cls] : 0;
             const int a_k_off = B_SPLIT ? (w.split & 7) * p.cls_kc : 0;
             const int col0 = w.nb * TILE_N + (int)cta_rank * BN_CTA;
@@ -463,8 +467,8 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                 const int unit = w.unit, mb = w.mb, nb = w.nb, split = w.split, kb0 = w.kb0, kb1 = w.kb1;
                 // A rows of this CTA: consecutive rows, or in class mode rows 1024*g + j + 8*i read through
                 // map j at class-row index 128*g
-                const int cls = A_CLS ? (mb % NCLS) : 0;
-                const int row0 = A_CLS ? (mb / NCLS) * (128 * CG) + (int)cta_rank * 128 : mb * (128 * CG) + (int)cta_rank * 128;
+                const int cls = A_CLS ? (mb & (NCLS - 1)) : 0;
+                const int row0 = A_CLS ? (mb >> NSH) * (128 * CG) + (int)cta_rank * 128 : mb * (128 * CG) + (int)cta_rank * 128;
                 const int kshift = A_CLS ? p.a_sigma[cls] : 0;                // B's k-rows lag A's kappa by sigma
                 const CUtensorMap* tmA = &maps.a[cls];
                 const CUtensorMap* tmB = &maps.b[B_SPLIT ? (split & 7) : 0];  // k classes as splits: the class's view of B
@@ -472,7 +476,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     // the next unit may go through other maps: fetch their descriptors while this unit loads
                     int mb2, nb2, sp2;
                     decode_unit(p, unit + unit_step, mb2, nb2, sp2);
-                    if (A_CLS && (mb2 % NCLS) != cls) ptx::prefetch_tensormap(&maps.a[mb2 % NCLS]);
+                    if (A_CLS && (mb2 & (NCLS - 1)) != cls) ptx::prefetch_tensormap(&maps.a[mb2 & (NCLS - 1)]);
                     if (B_SPLIT && (sp2 & 7) != (split & 7)) ptx::prefetch_tensormap(&maps.b[sp2 & 7]);
                 }
                 const int a_k_off = B_SPLIT ? (split & 7) * p.cls_kc : 0;     // ... and its segment of the regrouped A
@@ -584,7 +588,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
             for (int it = 0; ok; ++it) {
                 WorkItem w;
                 if (!next_item<SK, B_SPLIT>(p, unit0, unit_step, it, w)) break;
-                const int sigma = p.a_sigma[w.mb % NCLS];
+                const int sigma = p.a_sigma[w.mb & (NCLS - 1)];
                 if (w.kb0 == 0 && w.kb1 > 0 && sigma > 0) {
                     if (!mma_wait(afull_bar + 8u * stage, (aphase >> stage) & 1u)) { ok = false; break; }
                     zero_row_heads(stage, sigma);
@@ -614,7 +618,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                 if (warp_wide && kb0 == 0 && kb1 > 0) {
                     // Done here, before the wait for a free accumulator: the loads run ahead of the drain, so
                     // in the write-bound regime this work hides behind that wait.
-                    const int sigma = p.a_sigma[mb % NCLS];
+                    const int sigma = p.a_sigma[mb & (NCLS - 1)];
                     if (sigma > 0) {
                         if (!mma_wait((A_CLS && CG == 2) ? afull_bar + 8u * stage : full_bar + 8u * stage,
                                       (A_CLS && CG == 2) ? ((aphase >> stage) & 1u) : phase)) { ok = false; break; }
@@ -652,7 +656,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                         int st = stage;
                         uint32_t ph = phase;
                         for (int kb = kb0; kb < kb1; ++kb) {
-                            if (A_CLS && CG == 2 && kb == 0 && p.a_sigma[mb % NCLS] > 0) {
+                            if (A_CLS && CG == 2 && kb == 0 && p.a_sigma[mb & (NCLS - 1)] > 0) {
                                 // the unit's first k-block, row heads zeroed: this CTA's box (waited for above) and the peer's,
                                 // handed over by the peer's warp 1.  The leader reads none of the peer's shared memory itself
                                 // (the peer's tensor core does, after the peer's own proxy fence), so an ordinary wait is enough.
@@ -676,7 +680,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                     }
                     if (warp_wide) done = __shfl_sync(0xffffffffu, done, 0);
                     if (!done) { ok = false; break; }
-                    if (A_CLS && CG == 2 && kb0 == 0 && kb1 > 0 && p.a_sigma[mb % NCLS] > 0) aphase ^= 1u << stage;
+                    if (A_CLS && CG == 2 && kb0 == 0 && kb1 > 0 && p.a_sigma[mb & (NCLS - 1)] > 0) aphase ^= 1u << stage;
                     const int adv = stage + (kb1 - kb0);
                     phase ^= (uint32_t)((adv / S) & 1);
                     stage = adv % S;
@@ -721,7 +725,7 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
             if (warp == 2 && lane == 0) ADAPT_TRACE(4, unit);
             // row of C held by TMEM lane i of this CTA: consecutive rows, or every 8th row of one class
             const int row_step = A_CLS ? NCLS : 1;
-            const int row_base = A_CLS ? (mb / NCLS) * (128 * CG * NCLS) + (mb % NCLS) + NCLS * 128 * (int)cta_rank
+            const int row_base = A_CLS ? (mb >> NSH) * (128 * CG * NCLS) + (mb & (NCLS - 1)) + NCLS * 128 * (int)cta_rank
                                        : mb * (128 * CG) + (int)cta_rank * 128;
             const int row = row_base + row_step * (q * 32 + lane);
             const int n0 = nb * TILE_N;
@@ -927,13 +931,13 @@ umma_gemm_kernel(const __grid_constant__ TmapPackT<MODE> maps, const UmmaParams 
                         // the other warp of the quarter stores this tile; this one stores the next: fetch its map's descriptor now
                         int mb2, nb2, sp2;
                         decode_unit(p, unit + unit_step, mb2, nb2, sp2);
-                        ptx::prefetch_tensormap(&maps.c[mb2 % NCLS]);
+                        ptx::prefetch_tensormap(&maps.c[mb2 & (NCLS - 1)]);
                     }
                     if ((seq & 1) == half) {
-                        const int cls = A_CLS ? (mb % NCLS) : 0;
+                        const int cls = A_CLS ? (mb & (NCLS - 1)) : 0;
                         const int sig = HALO ? p.c_sigma[cls] : 0;
                         const int off = HALO ? 16 - sig : 0;
-                        const int y0 = A_CLS ? (mb / NCLS) * (128 * CG) + (int)cta_rank * 128 + q * 32 : row_base + q * 32;
+                        const int y0 = A_CLS ? (mb >> NSH) * (128 * CG) + (int)cta_rank * 128 + q * 32 : row_base + q * 32;
                         const CUtensorMap* tmC = &maps.c[cls];
                         uint8_t* wbuf = stage_out + (warp - 2) * kUmmaWarpStagingBytes;
                         const int x_first = n0 + (HALO ? 16 : 0);

@@ -378,7 +378,10 @@ def halo_variants(M, N, K, dtype, limit=12, family=None):
 
 @pytest.mark.parametrize("dtype", [ab.F16, ab.BF16])
 @pytest.mark.parametrize("shape", [(1030, 265, 328), (1030, 265, 331), (2500, 77, 1000), (4100, 1001, 64), (300, 521, 16),
-                                   (16, 9, 8), (129, 3, 40), (1024, 201, 4099), (3000, 40, 24), (2100, 8, 16), (77, 1537, 70), (2049, 193, 5)])
+                                   (16, 9, 8), (129, 3, 40), (1024, 201, 4099), (3000, 40, 24), (2100, 8, 16), (77, 1537, 70), (2049, 193, 5),
+                                   # even N: 8, 4 or 2 row classes instead of 16 (and what an A read in place adds to that)
+                                   (1030, 266, 331), (1030, 268, 328), (4100, 1000, 64), (2049, 200, 5), (300, 518, 20), (2100, 12, 16),
+                                   (999, 36, 100), (1500, 104, 70), (5000, 1032, 257)])
 def test_halo_class_tiles_bit_exact(shape, dtype):
     M, N, K = shape
     A = synth.position_coded(M, K, dtype, modulus=7, device="cuda")
@@ -392,7 +395,8 @@ def test_halo_class_tiles_bit_exact(shape, dtype):
 
 @pytest.mark.parametrize("dtype", [ab.F16, ab.BF16])
 @pytest.mark.parametrize("shape", [(1030, 265, 328), (1030, 265, 331), (4100, 1001, 64), (300, 521, 16), (40, 777, 200),
-                                   (4097, 201, 1003), (9000, 393, 24), (2100, 209, 700), (8200, 1537, 70), (5000, 193, 5)])
+                                   (4097, 201, 1003), (9000, 393, 24), (2100, 209, 700), (8200, 1537, 70), (5000, 193, 5),
+                                   (4097, 204, 1003), (9000, 392, 24), (2100, 210, 700), (1100, 1000, 72)])
 def test_pair_halo_class_tiles_bit_exact(shape, dtype):
     """Halo class tiles on SM pairs (256 rows of one of 16 row classes, 128 or 192 owned columns + 16 halo columns):
     aligned and unaligned A, K shorter and longer than a k-block, M below and above one group of 4096 rows,

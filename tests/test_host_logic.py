@@ -126,8 +126,16 @@ def test_every_shape_has_a_legal_candidate_and_info_is_consistent():
                 if c.family in (ab.FAM_UMMA_1CTA, ab.FAM_UMMA_2CTA):
                     bn_cta = c.BN // c.cluster
                     # a stage holds the rows of A one box brings (128, or fewer for a short A) and BN columns of B
-                    halo = c.BN % 64 != 0        # class tiles of 16 row classes that own 32-byte units of C's shifted rows
-                    ncls = 16 if halo else 8
+                    halo = c.BN % 64 != 0        # class tiles that own 32-byte units of C's shifted rows
+                    # as few row classes as keep the rows of a class at one offset from a 32-byte boundary in C (and from a
+                    # 16-byte one in an A read in place): 16 for an odd N, fewer for an even one
+                    if halo:
+                        for_c = next(n for n in (2, 4, 8, 16) if (n * N) % 16 == 0)
+                        a_copied = K < 64 and not (K % 8 == 0 and K % 16 == 0)
+                        for_a = 1 if a_copied else next(n for n in (1, 2, 4, 8) if (n * K) % 8 == 0)
+                        ncls = max(2, for_c, for_a)
+                    else:
+                        ncls = 8
                     a_rows = 128
                     if c.srcA == 3 and c.cluster == 1:
                         a_rows = min(128, -(-(-(-M // ncls)) // 8) * 8)
